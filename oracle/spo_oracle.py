@@ -1,0 +1,322 @@
+"""Float64 CPU oracle for the SPO (Single-stream Policy Optimization) hot path.
+
+TEST INFRASTRUCTURE ONLY.  This module is the slow, plain restatement of what
+the paper defines; the CUDA library is checked against it.  It shares no code
+with the CUDA path, imports nothing from it, and must never be called from the
+product path (only from tests, the smoke check and the CPU-baseline leg of the
+benchmark).
+
+Everything is numpy float64 unless a function name ends in ``_f32``: those
+restate, in IEEE fp32 with one correctly rounded operation per step, the few
+places where floating point decides an integer (the quantised sampling
+weights), so that both sides take that decision in the same precision.
+
+Pinned by tests/test_oracle_pins.py against closed forms, brute force, finite
+differences and the constants the paper prints.  Pieces whose parameters the
+paper never gives a value for (``d_half``; the whole-step composition, for
+which no worked example is printed) are "parity unpinned" by the paper itself
+and are pinned only through the identities listed in that test file.
+
+Paper sections: Sec. 3.1 (KL-adaptive value tracker), Sec. 3.2 (advantage,
+global normalisation, PPO-Clip objective), Sec. 3.3 and Eq. "sampling_coef"
+(prioritised sampling), Algorithm 1 (training loop), Algorithm 2
+(initialisation), appendix "Training and Evaluation Details" (constants).
+"""
+
+from __future__ import annotations
+
+import numpy as np
+
+# Constants printed in the appendix "Training and Evaluation Details" and Sec. 3.3.
+RHO_MIN = 0.875
+RHO_MAX = 0.96
+EPS_EXPLORE = 0.05
+CLIP_LO = 0.2
+CLIP_HI = 0.28
+N0_SAMPLES = 8
+
+
+# --------------------------------------------------------------------------
+# Sec. 3.1 -- value tracker
+# --------------------------------------------------------------------------
+
+def tracker_init(v0, rho_min=RHO_MIN):
+    """Algorithm 2: N0 = 1/(1-rho_min); alpha0 = N0*v0; beta0 = N0*(1-v0)."""
+    v0 = np.asarray(v0, dtype=np.float64)
+    n0 = 1.0 / (1.0 - float(rho_min))
+    return n0 * v0, n0 * (1.0 - v0)
+
+
+def value_estimate(alpha, beta):
+    """Posterior mean v = alpha/(alpha+beta) (Sec. 3.1).
+
+    The paper does not say what an empty tracker (alpha+beta = 0) estimates;
+    the reading taken is the uninformed 0.5.
+    """
+    alpha = np.asarray(alpha, dtype=np.float64)
+    beta = np.asarray(beta, dtype=np.float64)
+    n = alpha + beta
+    safe = np.where(n > 0.0, n, 1.0)
+    return np.where(n > 0.0, alpha / safe, 0.5)
+
+
+def forgetting_factor(kl, d_half, rho_min=RHO_MIN, rho_max=RHO_MAX):
+    """rho = 2^(-D/D_half), kept inside [rho_min, rho_max] by a hard clamp (Sec. 3.1)."""
+    kl = np.asarray(kl, dtype=np.float64)
+    rho = np.exp2(-kl / float(d_half))
+    return np.minimum(np.maximum(rho, float(rho_min)), float(rho_max))
+
+
+def tracker_update(alpha, beta, ids, r, kl, d_half, rho_min=RHO_MIN, rho_max=RHO_MAX):
+    """Tracker update equation of Sec. 3.1, applied to the batch entries in order.
+
+    alpha <- rho*alpha + r ; beta <- rho*beta + (1-r), at table row ids[j].
+    ``kl`` holds one divergence per batch entry.  Returns new copies.
+    """
+    alpha = np.array(alpha, dtype=np.float64, copy=True)
+    beta = np.array(beta, dtype=np.float64, copy=True)
+    r = np.asarray(r, dtype=np.float64)
+    rho = forgetting_factor(kl, d_half, rho_min, rho_max)
+    for j in range(len(ids)):
+        i = int(ids[j])
+        alpha[i] = rho[j] * alpha[i] + r[j]
+        beta[i] = rho[j] * beta[i] + (1.0 - r[j])
+    return alpha, beta
+
+
+def ema_update(v_prev, n_prev, r, rho):
+    """EMA restatement of the same update (Sec. 3.1, second display).
+
+    v = v_prev + eta*(r - v_prev) with eta = 1/(rho*n_prev + 1), where n_prev is
+    alpha+beta before the update.  (The paper's "N_eff = alpha+beta+1" next to
+    this formula does not satisfy the Beta update by algebra; the Beta update is
+    taken as the definition and eta is what it implies.)
+    """
+    eta = 1.0 / (rho * n_prev + 1.0)
+    return v_prev + eta * (r - v_prev)
+
+
+# --------------------------------------------------------------------------
+# Sec. 3.2 -- advantage and global normalisation
+# --------------------------------------------------------------------------
+
+def raw_advantage(alpha, beta, ids, r):
+    """A = r - v_{-1}(x): the table is read before this batch's update (Sec. 3.2)."""
+    v = value_estimate(alpha, beta)
+    ids = np.asarray(ids, dtype=np.int64)
+    return np.asarray(r, dtype=np.float64) - v[ids]
+
+
+def normalise_advantages(a, ddof=0, eps=1e-8):
+    """A~ = (A - mu_B)/sigma_B over the whole batch (Sec. 3.2).
+
+    Population standard deviation by default; ``eps`` is added to sigma so that
+    an all-equal batch gives zeros.  Returns (A~, mu, sigma).
+    """
+    a = np.asarray(a, dtype=np.float64)
+    b = a.shape[0]
+    if b == 0:
+        return a.copy(), 0.0, 0.0
+    mu = a.sum() / b
+    denom = b - ddof
+    if denom <= 0:
+        sigma = 0.0
+    else:
+        sigma = float(np.sqrt(((a - mu) ** 2).sum() / denom))
+    return (a - mu) / (sigma + eps), float(mu), sigma
+
+
+# --------------------------------------------------------------------------
+# Sec. 3.3 -- prioritised sampling
+# --------------------------------------------------------------------------
+
+def sampling_weights(alpha, beta, eps_explore=EPS_EXPLORE):
+    """w = sqrt(v(1-v)) + eps (Eq. "sampling_coef"), unnormalised."""
+    v = value_estimate(alpha, beta)
+    return np.sqrt(v * (1.0 - v)) + float(eps_explore)
+
+
+def sampling_weights_f32(alpha32, beta32, eps_explore=EPS_EXPLORE):
+    """The same weights in IEEE fp32, one correctly rounded operation per step.
+
+    v(1-v) is formed as alpha*beta/(alpha+beta)^2, which is the same quantity
+    without the cancellation of 1-v near v = 1.  Order of operations:
+    n = alpha+beta; num = alpha*beta; den = n*n; p = num/den (0.25 if n == 0);
+    s = sqrt(p); w = s + eps.  numpy's float32 add, multiply, divide and sqrt
+    are each correctly rounded, so any IEEE implementation that performs these
+    steps without fusing them gives the same bits.
+    """
+    a = np.asarray(alpha32, dtype=np.float32)
+    b = np.asarray(beta32, dtype=np.float32)
+    n = a + b
+    num = a * b
+    den = n * n
+    pos = n > np.float32(0.0)
+    p = np.where(pos, num / np.where(pos, den, np.float32(1.0)), np.float32(0.25)).astype(np.float32)
+    s = np.sqrt(p)
+    w = s + np.float32(eps_explore)
+    return w.astype(np.float32)
+
+
+def quantise_weights(w32):
+    """q = floor(w * 2^32) as unsigned 64-bit integers (exact: a power-of-two scale)."""
+    w = np.asarray(w32, dtype=np.float32).astype(np.float64)
+    if np.any(w < 0) or not np.all(np.isfinite(w)):
+        raise ValueError("weights must be finite and non-negative")
+    return np.floor(w * 4294967296.0).astype(np.uint64)
+
+
+def sample_prompts(w32, uniforms32, batch):
+    """Draw ``batch`` distinct prompts by weight (Algorithm 1, "Sample a batch ... according to weights").
+
+    Successive weighted sampling without replacement, realised as inverse-CDF
+    draws with replacement whose repeats are skipped (equal in distribution to
+    removing each chosen prompt and renormalising).  The CDF is over integers:
+    q_i = floor(w_i*2^32), C_i = q_0+...+q_i, Wtot = C_{N-1}.  For the k-th
+    uniform u_k in [0,1): U_k = floor(u_k*2^32), t_k = floor(U_k*Wtot / 2^32),
+    candidate = the first i with C_i > t_k.  Candidates are accepted in order
+    unless already accepted; stops at ``batch`` accepted.  Raises if the
+    uniforms run out.  Returns int64 ids in acceptance order.
+    """
+    q = quantise_weights(w32)
+    csum = np.cumsum(q, dtype=np.uint64)
+    wtot = int(csum[-1]) if len(csum) else 0
+    if wtot == 0:
+        raise ValueError("total weight is zero")
+    u = np.asarray(uniforms32, dtype=np.float32).astype(np.float64)
+    if np.any(u < 0.0) or np.any(u >= 1.0):
+        raise ValueError("uniforms must lie in [0,1)")
+    chosen = []
+    seen = set()
+    for k in range(len(u)):
+        if len(chosen) == batch:
+            break
+        big_u = int(np.floor(u[k] * 4294967296.0))
+        t = (big_u * wtot) >> 32
+        i = int(np.searchsorted(csum, np.uint64(t), side="right"))
+        if i not in seen:
+            seen.add(i)
+            chosen.append(i)
+    if len(chosen) < batch:
+        raise RuntimeError("not enough uniforms to accept %d distinct prompts" % batch)
+    return np.asarray(chosen, dtype=np.int64)
+
+
+# --------------------------------------------------------------------------
+# Sec. 3.2 -- PPO-Clip objective on log-probs from the LM head
+# --------------------------------------------------------------------------
+
+def token_sequence_ids(cu_seqlens, n_tokens):
+    """seq(t) for packed rows: the s with cu_seqlens[s] <= t < cu_seqlens[s+1]."""
+    cu = np.asarray(cu_seqlens, dtype=np.int64)
+    t = np.arange(n_tokens, dtype=np.int64)
+    return np.searchsorted(cu, t, side="right") - 1
+
+
+def logits(h, w):
+    """z[t, v] = sum_k W[v, k] * H[t, k] (the LM head; no bias, temperature 1)."""
+    return np.asarray(h, dtype=np.float64) @ np.asarray(w, dtype=np.float64).T
+
+
+def loss_forward(h, w, y, logp_old, mask, cu_seqlens, a_norm,
+                 clip_lo=CLIP_LO, clip_hi=CLIP_HI):
+    """Token-level PPO-Clip surrogate of Sec. 3.2 with Clip-Higher bounds.
+
+    Per token t (row of ``h``): z = W h_t; lse = log sum_v exp(z_v);
+    logp = z[y_t] - lse; ratio = exp(logp - logp_old_t); a = A~[seq(t)];
+    s = min(ratio*a, clip(ratio, 1-clip_lo, 1+clip_hi)*a).
+    The expectation over (s,t) is read as the mean over all unmasked tokens of
+    the batch, n_tok = sum(mask); the exported loss is the negated objective.
+
+    Returns a dict: loss, logp[T], lse[T], ratio[T], surrogate[T], unclipped[T]
+    (bool: the gradient passes through the ratio), coef[T] = d loss / d logp_t
+    = -mask*a*ratio*unclipped/n_tok, n_tok, and seq_sums[S,3] = per sequence
+    (sum mask*logp, sum mask*(logp_old - logp), sum mask).
+    """
+    z = logits(h, w)
+    n_tok_rows = z.shape[0]
+    y = np.asarray(y, dtype=np.int64)
+    logp_old = np.asarray(logp_old, dtype=np.float64)
+    if mask is None:
+        m = np.ones(n_tok_rows, dtype=np.float64)
+    else:
+        m = (np.asarray(mask) != 0).astype(np.float64)
+    zmax = z.max(axis=1) if z.shape[1] else np.zeros(n_tok_rows)
+    lse = zmax + np.log(np.exp(z - zmax[:, None]).sum(axis=1))
+    logp = z[np.arange(n_tok_rows), y] - lse
+    ratio = np.exp(logp - logp_old)
+    seq = token_sequence_ids(cu_seqlens, n_tok_rows)
+    a = np.asarray(a_norm, dtype=np.float64)[seq]
+    clipped_ratio = np.minimum(np.maximum(ratio, 1.0 - clip_lo), 1.0 + clip_hi)
+    surrogate = np.minimum(ratio * a, clipped_ratio * a)
+    n_tok = m.sum()
+    loss = -(m * surrogate).sum() / n_tok if n_tok > 0 else 0.0
+    # The min picks the unclipped branch (and so carries gradient) when the
+    # ratio is on the inside of the bound that matters for the sign of a;
+    # the boundary itself counts as inside.
+    unclipped = np.where(a >= 0.0, ratio <= 1.0 + clip_hi, ratio >= 1.0 - clip_lo)
+    coef = -(m * a * ratio * unclipped) / n_tok if n_tok > 0 else np.zeros(n_tok_rows)
+    n_seq = len(cu_seqlens) - 1
+    seq_sums = np.zeros((n_seq, 3), dtype=np.float64)
+    np.add.at(seq_sums[:, 0], seq, m * logp)
+    np.add.at(seq_sums[:, 1], seq, m * (logp_old - logp))
+    np.add.at(seq_sums[:, 2], seq, m)
+    return {
+        "loss": float(loss), "logp": logp, "lse": lse, "ratio": ratio,
+        "surrogate": surrogate, "unclipped": unclipped, "coef": coef,
+        "n_tok": float(n_tok), "seq_sums": seq_sums,
+    }
+
+
+def loss_backward(h, w, y, lse, coef, grad_loss=1.0):
+    """Gradients of the exported loss with respect to H and W.
+
+    With p = exp(z - lse) (the softmax) the logit gradient is
+    g[t, v] = grad_loss * coef_t * (1[v = y_t] - p[t, v]);
+    dH = g W ; dW = g^T H.
+    """
+    h = np.asarray(h, dtype=np.float64)
+    w = np.asarray(w, dtype=np.float64)
+    z = h @ w.T
+    p = np.exp(z - np.asarray(lse, dtype=np.float64)[:, None])
+    g = -p
+    g[np.arange(z.shape[0]), np.asarray(y, dtype=np.int64)] += 1.0
+    g *= (float(grad_loss) * np.asarray(coef, dtype=np.float64))[:, None]
+    return g @ w, g.T @ h
+
+
+def loss_rows(h_rows, w, y_rows, logp_old_rows, mask_rows, a_rows, n_tok,
+              clip_lo=CLIP_LO, clip_hi=CLIP_HI, grad_loss=1.0, v_chunk=8192):
+    """Row-local outputs for a handful of token rows of a large problem.
+
+    Every per-token output of loss_forward and the dH row of loss_backward
+    depends only on that token's hidden state, W and batch-level scalars
+    (the advantage of its sequence, n_tok).  This evaluates exactly those
+    formulas for the given rows, streaming W in chunks of ``v_chunk`` rows so
+    that W never has to exist in float64 at once.  Returns dict(logp, lse,
+    ratio, coef, dH).
+    """
+    h = np.asarray(h_rows, dtype=np.float64)
+    n, d = h.shape
+    v_total = w.shape[0]
+    z = np.empty((n, v_total), dtype=np.float64)
+    for v0 in range(0, v_total, v_chunk):
+        wc = np.asarray(w[v0:v0 + v_chunk], dtype=np.float64)
+        z[:, v0:v0 + wc.shape[0]] = h @ wc.T
+    zmax = z.max(axis=1)
+    lse = zmax + np.log(np.exp(z - zmax[:, None]).sum(axis=1))
+    y = np.asarray(y_rows, dtype=np.int64)
+    logp = z[np.arange(n), y] - lse
+    ratio = np.exp(logp - np.asarray(logp_old_rows, dtype=np.float64))
+    a = np.asarray(a_rows, dtype=np.float64)
+    m = (np.asarray(mask_rows) != 0).astype(np.float64)
+    unclipped = np.where(a >= 0.0, ratio <= 1.0 + clip_hi, ratio >= 1.0 - clip_lo)
+    coef = -(m * a * ratio * unclipped) / float(n_tok)
+    g = -np.exp(z - lse[:, None])
+    g[np.arange(n), y] += 1.0
+    g *= (float(grad_loss) * coef)[:, None]
+    dh = np.zeros((n, d), dtype=np.float64)
+    for v0 in range(0, v_total, v_chunk):
+        wc = np.asarray(w[v0:v0 + v_chunk], dtype=np.float64)
+        dh += g[:, v0:v0 + wc.shape[0]] @ wc
+    return {"logp": logp, "lse": lse, "ratio": ratio, "coef": coef, "dH": dh}

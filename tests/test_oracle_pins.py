@@ -1,0 +1,476 @@
+"""Pins for the CPU oracle: closed forms, hand-worked values, brute force, finite
+differences, library routines and the constants the paper prints.  No GPU."""
+
+import math
+import os
+from fractions import Fraction
+
+import numpy as np
+import pytest
+import scipy.special
+import scipy.stats
+
+from oracle import spo_oracle as O
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "paper_constants.txt")
+
+
+def paper_constants():
+    out = {}
+    with open(GOLDEN) as f:
+        for line in f:
+            line = line.split("#")[0].strip()
+            if line:
+                k, v = line.split()
+                out[k] = float(v)
+    return out
+
+
+# ------------------------------------------------------------------ tracker
+
+def test_paper_constants_match_oracle_defaults():
+    c = paper_constants()
+    assert O.RHO_MIN == c["rho_min"] and O.RHO_MAX == c["rho_max"]
+    assert O.EPS_EXPLORE == c["eps_explore"]
+    assert O.CLIP_LO == c["clip_low"] and O.CLIP_HI == c["clip_high"]
+    assert O.N0_SAMPLES == c["n0"]
+
+
+def test_init_effective_sample_size_is_window_min():
+    c = paper_constants()
+    v0 = np.array([0.0, 0.125, 0.5, 1.0])
+    a, b = O.tracker_init(v0, c["rho_min"])
+    np.testing.assert_allclose(a + b, c["window_min"], rtol=0, atol=1e-12)
+    np.testing.assert_allclose(O.value_estimate(a, b), v0, atol=1e-15)
+
+
+@pytest.mark.parametrize("key_rho,key_win", [("rho_min", "window_min"), ("rho_max", "window_max")])
+def test_equilibrium_window_sizes(key_rho, key_win):
+    """alpha+beta converges to 1/(1-rho): 8 at rho_min and 25 at rho_max."""
+    c = paper_constants()
+    rho = c[key_rho]
+    d_half = 1.0
+    kl = -math.log2(rho) * d_half          # 2^(-kl/d_half) == rho, inside the clamp
+    a, b = np.array([3.0]), np.array([1.0])
+    rng = np.random.default_rng(0)
+    for _ in range(600):
+        r = float(rng.random() < 0.3)
+        a, b = O.tracker_update(a, b, [0], [r], [kl], d_half, c["rho_min"], c["rho_max"])
+    assert abs((a + b)[0] - c[key_win]) < 1e-6
+
+
+def test_equilibrium_start_is_fixed_point_and_constant_reward_closed_form():
+    rho, c_reward, v0 = 0.875, 1.0, 0.25
+    a, b = O.tracker_init(np.array([v0]), rho)
+    kl = -math.log2(rho) * 0.1
+    for k in range(1, 40):
+        a, b = O.tracker_update(a, b, [0], [c_reward], [kl], 0.1, 0.875, 0.96)
+        assert abs((a + b)[0] - 8.0) < 1e-12
+        expect = c_reward + rho ** k * (v0 - c_reward)
+        assert abs(O.value_estimate(a, b)[0] - expect) < 1e-12
+    # the estimate is driven to the constant reward
+    for _ in range(400):
+        a, b = O.tracker_update(a, b, [0], [c_reward], [kl], 0.1, 0.875, 0.96)
+    assert abs(O.value_estimate(a, b)[0] - 1.0) < 1e-9
+
+
+def test_constant_zero_reward_drives_estimate_to_zero():
+    a, b = O.tracker_init(np.array([0.9]), 0.875)
+    for _ in range(300):
+        a, b = O.tracker_update(a, b, [0], [0.0], [0.05], 0.1)
+    assert O.value_estimate(a, b)[0] < 1e-9
+
+
+def test_rho_one_is_beta_bernoulli_counting():
+    """With no forgetting the update is the textbook conjugate count update."""
+    rs = [1, 0, 0, 1, 1, 1, 0]
+    a, b = np.array([2.0]), np.array([5.0])
+    for r in rs:
+        a, b = O.tracker_update(a, b, [0], [float(r)], [0.0], 1.0, rho_min=0.0, rho_max=1.0)
+    assert a[0] == 2.0 + sum(rs) and b[0] == 5.0 + len(rs) - sum(rs)
+    post = scipy.stats.beta(2.0 + sum(rs), 5.0 + len(rs) - sum(rs))
+    assert abs(O.value_estimate(a, b)[0] - post.mean()) < 1e-15
+
+
+def test_forgetting_factor_values_and_clamp():
+    # 2^(-1) = 0.5 is below rho_min; 2^0 = 1 above rho_max; 2^(-1/8) is inside.
+    rho = O.forgetting_factor([1.0, 0.0, 0.125, -3.0], 1.0, 0.875, 0.96)
+    np.testing.assert_allclose(rho, [0.875, 0.96, 0.9170040432046712, 0.96], atol=1e-15)
+    # halving: D = D_half halves the memory when the clamp is open
+    assert O.forgetting_factor([0.3], 0.3, 0.0, 1.0)[0] == 0.5
+
+
+def test_bayes_update_equals_ema_form():
+    rng = np.random.default_rng(1)
+    for _ in range(50):
+        a0, b0 = rng.uniform(0.1, 20, 2)
+        r = float(rng.random() < 0.5)
+        kl = rng.lognormal(-4, 1)
+        rho = O.forgetting_factor([kl], 0.1)[0]
+        a, b = O.tracker_update([a0], [b0], [0], [r], [kl], 0.1)
+        ema = O.ema_update(a0 / (a0 + b0), a0 + b0, r, rho)
+        assert abs(O.value_estimate(a, b)[0] - ema) < 1e-14
+        # the learning rate is one over the new effective sample size
+        assert abs(1.0 / (rho * (a0 + b0) + 1.0) - 1.0 / (a + b)[0]) < 1e-15
+
+
+def test_update_touches_only_batch_rows_and_keeps_domain():
+    rng = np.random.default_rng(2)
+    a0, b0 = rng.uniform(0, 5, 10), rng.uniform(0, 5, 10)
+    ids = [7, 2, 5]
+    a, b = O.tracker_update(a0, b0, ids, [1.0, 0.0, 1.0], [0.01, 0.2, 5.0], 0.1)
+    untouched = [i for i in range(10) if i not in ids]
+    assert np.array_equal(a[untouched], a0[untouched]) and np.array_equal(b[untouched], b0[untouched])
+    assert np.all(a >= 0) and np.all(b >= 0)
+    v = O.value_estimate(a, b)
+    assert np.all((v >= 0) & (v <= 1))
+    # one row by hand: kl=5 -> rho clamps to 0.875; r=1
+    assert abs(a[5] - (0.875 * a0[5] + 1.0)) < 1e-15 and abs(b[5] - 0.875 * b0[5]) < 1e-15
+    # r=0 row by hand: kl = 0.2, d_half 0.1 -> 2^-2 = 0.25 -> clamp 0.875
+    assert abs(a[2] - 0.875 * a0[2]) < 1e-15 and abs(b[2] - (0.875 * b0[2] + 1.0)) < 1e-15
+
+
+def test_empty_tracker_estimates_half_then_first_reward():
+    assert O.value_estimate([0.0], [0.0])[0] == 0.5
+    a, b = O.tracker_update([0.0], [0.0], [0], [1.0], [0.01], 0.1)
+    assert O.value_estimate(a, b)[0] == 1.0
+
+
+# ---------------------------------------------------------------- advantage
+
+def test_no_baseline_table_gives_reward_as_advantage():
+    a, b = np.zeros(4), np.ones(4)            # v = 0 everywhere
+    r = np.array([1.0, 0.0, 1.0, 1.0])
+    np.testing.assert_array_equal(O.raw_advantage(a, b, [3, 1, 0, 2], r), r)
+
+
+def test_advantage_uses_table_rows_by_id():
+    a, b = np.array([1.0, 3.0, 1.0]), np.array([3.0, 1.0, 1.0])   # v = .25 .75 .5
+    out = O.raw_advantage(a, b, [2, 0, 1], [1.0, 1.0, 0.0])
+    np.testing.assert_allclose(out, [0.5, 0.75, -0.75], atol=1e-15)
+
+
+@pytest.mark.parametrize("ddof", [0, 1])
+def test_normalisation_against_library_zscore(ddof):
+    rng = np.random.default_rng(3)
+    a = rng.uniform(-1, 1, 257)
+    out, mu, sigma = O.normalise_advantages(a, ddof=ddof, eps=0.0)
+    np.testing.assert_allclose(out, scipy.stats.zscore(a, ddof=ddof), atol=1e-12)
+    assert abs(out.mean()) < 1e-12
+    assert abs(out.std(ddof=ddof) - 1.0) < 1e-12
+    assert abs(mu - a.mean()) < 1e-15 and abs(sigma - a.std(ddof=ddof)) < 1e-15
+
+
+def test_normalisation_affine_invariance_and_degenerate_cases():
+    rng = np.random.default_rng(4)
+    a = rng.uniform(-1, 1, 64)
+    base, _, _ = O.normalise_advantages(a, eps=0.0)
+    moved, _, _ = O.normalise_advantages(3.5 * a - 2.0, eps=0.0)
+    np.testing.assert_allclose(moved, base, atol=1e-12)
+    flat, _, sigma = O.normalise_advantages(np.full(9, 0.3))
+    assert sigma == 0.0 and np.all(flat == 0.0)
+    one, _, _ = O.normalise_advantages(np.array([0.7]))
+    assert one[0] == 0.0
+
+
+# ----------------------------------------------------------------- sampling
+
+def test_weight_range_endpoints():
+    eps = paper_constants()["eps_explore"]
+    a = np.array([0.0, 8.0, 4.0])
+    b = np.array([8.0, 0.0, 4.0])
+    w = O.sampling_weights(a, b, eps)
+    np.testing.assert_allclose(w, [eps, eps, 0.5 + eps], atol=1e-15)
+    rng = np.random.default_rng(5)
+    aa, bb = rng.uniform(0, 10, 1000), rng.uniform(0, 10, 1000)
+    ww = O.sampling_weights(aa, bb, eps)
+    assert ww.min() >= eps and ww.max() <= 0.5 + eps + 1e-15
+
+
+def test_fp32_weights_track_the_fp64_definition():
+    rng = np.random.default_rng(6)
+    a = rng.uniform(0, 20, 5000).astype(np.float32)
+    b = rng.uniform(0, 20, 5000).astype(np.float32)
+    a[:3], b[:3] = [0, 0, 5], [0, 5, 0]
+    w32 = O.sampling_weights_f32(a, b)
+    assert w32.dtype == np.float32
+    np.testing.assert_allclose(w32, O.sampling_weights(a, b), rtol=2e-6, atol=1e-7)
+    assert w32[0] == np.float32(0.55)
+
+
+def test_quantised_weights_are_exact_scalings():
+    w = np.array([0.05, 0.55, 0.3, 2.0 ** -8], dtype=np.float32)
+    q = O.quantise_weights(w)
+    for wi, qi in zip(w, q):
+        assert int(qi) == int(Fraction(float(wi)) * 2 ** 32)     # exact rational floor
+
+
+def _first_index_by_rationals(w32, u):
+    q = [int(Fraction(float(x)) * 2 ** 32) for x in w32]
+    tot = sum(q)
+    c = 0
+    for i, qi in enumerate(q):
+        c += qi
+        if Fraction(c, tot) > Fraction(float(u)):
+            return i
+    raise AssertionError
+
+
+def test_first_draw_matches_exact_rational_inverse_cdf():
+    rng = np.random.default_rng(7)
+    for n in (1, 2, 3, 6):
+        w = rng.uniform(0.05, 0.55, n).astype(np.float32)
+        if n >= 3:
+            w[1] = 0.0                      # a zero weight can never be chosen
+        us = np.concatenate([rng.random(300), [0.0, 1 - 2.0 ** -24]]).astype(np.float32)
+        us = us[us < 1.0]
+        for u in us:
+            got = O.sample_prompts(w, [u], 1)[0]
+            assert got == _first_index_by_rationals(w, u)
+            assert w[got] > 0
+
+
+def test_equal_weights_systematic_uniforms_hit_every_index():
+    n = 64
+    w = np.full(n, 0.25, dtype=np.float32)
+    u = ((np.arange(n) + 0.5) / n).astype(np.float32)
+    np.testing.assert_array_equal(O.sample_prompts(w, u, n), np.arange(n))
+
+
+def test_repeats_are_skipped_and_full_batch_is_a_permutation():
+    w = np.array([0.5, 0.25, 0.25], dtype=np.float32)
+    u = np.array([0.1, 0.2, 0.6, 0.55, 0.9], dtype=np.float32)
+    np.testing.assert_array_equal(O.sample_prompts(w, u, 3), [0, 1, 2])
+    rng = np.random.default_rng(8)
+    ww = rng.uniform(0.05, 0.55, 40).astype(np.float32)
+    ids = O.sample_prompts(ww, rng.random(4000).astype(np.float32), 40)
+    assert sorted(ids.tolist()) == list(range(40))
+    with pytest.raises(RuntimeError):
+        O.sample_prompts(w, np.array([0.1, 0.2], dtype=np.float32), 3)
+
+
+def test_first_draw_frequencies_chi_square():
+    rng = np.random.default_rng(9)
+    n, draws = 64, 100_000
+    a = rng.uniform(0, 8, n).astype(np.float32)
+    b = rng.uniform(0, 8, n).astype(np.float32)
+    w = O.sampling_weights_f32(a, b)
+    u = rng.random(draws).astype(np.float32)
+    u = u[u < 1.0]
+    counts = np.zeros(n)
+    for x in u:
+        counts[O.sample_prompts(w, [x], 1)[0]] += 1
+    p = w.astype(np.float64) / w.astype(np.float64).sum()
+    chi2 = ((counts - len(u) * p) ** 2 / (len(u) * p)).sum()
+    assert chi2 < scipy.stats.chi2.ppf(0.9999, n - 1)
+
+
+def test_successive_sampling_pair_frequencies():
+    """Ordered pairs (i,j) appear with probability p_i * p_j / (1 - p_i)."""
+    rng = np.random.default_rng(10)
+    w = np.array([0.55, 0.05, 0.3, 0.2, 0.4], dtype=np.float32)
+    p = w.astype(np.float64) / w.astype(np.float64).sum()
+    draws = 40_000
+    counts = np.zeros((5, 5))
+    for _ in range(draws):
+        u = rng.random(64).astype(np.float32)
+        u = u[u < 1.0]
+        i, j = O.sample_prompts(w, u, 2)
+        counts[i, j] += 1
+    expect = draws * np.outer(p, p) / (1 - p)[:, None]
+    off = ~np.eye(5, dtype=bool)
+    assert counts[~off].sum() == 0
+    chi2 = ((counts[off] - expect[off]) ** 2 / expect[off]).sum()
+    assert chi2 < scipy.stats.chi2.ppf(0.9999, 19)
+
+
+# --------------------------------------------------------------------- loss
+
+def _identity_problem(z, y, logp_old, a_tok):
+    """H = I makes the logits equal to W^T, so arbitrary logits can be fed in."""
+    t, v = z.shape
+    h = np.eye(t)
+    w = z.T.copy()
+    cu = np.arange(t + 1)          # one token per sequence -> per-token advantage
+    return h, w, np.asarray(y), np.asarray(logp_old), None, cu, np.asarray(a_tok)
+
+
+def test_uniform_logits_give_minus_log_v():
+    t, d, v = 5, 7, 33
+    h = np.random.default_rng(11).standard_normal((t, d))
+    out = O.loss_forward(h, np.zeros((v, d)), [0, 5, 32, 7, 1], np.zeros(t), None, [0, 2, 5], [1.0, -1.0])
+    np.testing.assert_allclose(out["logp"], -math.log(v), atol=1e-14)
+    np.testing.assert_allclose(out["lse"], math.log(v), atol=1e-14)
+
+
+def test_logp_against_naive_softmax_and_library_and_shift_invariance():
+    rng = np.random.default_rng(12)
+    z = rng.standard_normal((6, 9)) * 3
+    y = rng.integers(0, 9, 6)
+    args = _identity_problem(z, y, np.zeros(6), np.ones(6))
+    out = O.loss_forward(*args)
+    naive = np.log(np.exp(z[np.arange(6), y]) / np.exp(z).sum(axis=1))
+    np.testing.assert_allclose(out["logp"], naive, atol=1e-13)
+    np.testing.assert_allclose(out["lse"], scipy.special.logsumexp(z, axis=1), atol=1e-13)
+    shifted = O.loss_forward(*_identity_problem(z + 1000.0, y, np.zeros(6), np.ones(6)))
+    np.testing.assert_allclose(shifted["logp"], out["logp"], atol=1e-10)
+    # one dominant logit -> probability one
+    z2 = np.zeros((1, 9)); z2[0, 4] = 80.0
+    assert abs(O.loss_forward(*_identity_problem(z2, [4], [0.0], [1.0]))["logp"][0]) < 1e-30
+
+
+def test_logits_orientation_is_w_times_h():
+    """z[t,v] = <W[v,:], H[t,:]> -- a transposed operand would fail this."""
+    h = np.array([[1.0, 2.0]])
+    w = np.array([[1.0, 0.0], [0.0, 1.0], [1.0, 1.0]])
+    np.testing.assert_array_equal(O.logits(h, w), [[1.0, 2.0, 3.0]])
+
+
+def test_ratio_one_gives_minus_mean_advantage():
+    rng = np.random.default_rng(13)
+    t, d, v = 12, 5, 17
+    h, w = rng.standard_normal((t, d)), rng.standard_normal((v, d))
+    y = rng.integers(0, v, t)
+    cu = [0, 3, 4, 12]
+    a = np.array([0.7, -1.3, 0.2])
+    mask = np.array([1, 1, 0, 1, 1, 1, 1, 0, 1, 1, 1, 1], dtype=np.uint8)
+    first = O.loss_forward(h, w, y, np.zeros(t), mask, cu, a)
+    out = O.loss_forward(h, w, y, first["logp"], mask, cu, a)
+    np.testing.assert_allclose(out["ratio"], 1.0, atol=1e-15)
+    a_tok = np.repeat(a, np.diff(cu))
+    assert abs(out["loss"] + (mask * a_tok).sum() / mask.sum()) < 1e-14
+    assert out["n_tok"] == 10
+    np.testing.assert_allclose(out["seq_sums"][:, 2], [2, 1, 7])
+    np.testing.assert_allclose(out["seq_sums"][:, 1], 0.0, atol=1e-13)
+    np.testing.assert_allclose(out["seq_sums"][:, 0],
+                               [(mask * out["logp"])[lo:hi].sum() for lo, hi in zip(cu[:-1], cu[1:])], atol=1e-13)
+
+
+def test_clip_branches_hand_worked():
+    """Clip-Higher bounds 0.8 / 1.28; hand-computed surrogate and gradient gate."""
+    cases = [  # ratio, advantage, surrogate, gradient passes
+        (1.5, 1.0, 1.28, False),
+        (1.5, -1.0, -1.5, True),
+        (0.5, 1.0, 0.5, True),
+        (0.5, -1.0, -0.8, False),
+        (1.0, 2.0, 2.0, True),
+        (1.28, 1.0, 1.28, True),     # boundary counts as inside
+        (0.8, -1.0, -0.8, True),
+        (1.1, 0.0, 0.0, True),
+    ]
+    for ratio, adv, s_expect, passes in cases:
+        z = np.zeros((1, 4))
+        logp_new = -math.log(4)
+        logp_old = logp_new - math.log(ratio)
+        out = O.loss_forward(*_identity_problem(z, [2], [logp_old], [adv]))
+        assert abs(out["ratio"][0] - ratio) < 1e-12
+        assert abs(out["surrogate"][0] - s_expect) < 1e-12, (ratio, adv)
+        assert abs(out["loss"] + s_expect) < 1e-12
+        if ratio not in (1.28, 0.8):       # exactly on the boundary rounding may fall either side
+            assert bool(out["unclipped"][0]) == passes
+        expect_coef = -adv * ratio if passes else 0.0
+        if ratio not in (1.28, 0.8):
+            assert abs(out["coef"][0] - expect_coef) < 1e-12
+
+
+def test_logit_gradient_is_advantage_times_softmax_minus_onehot():
+    rng = np.random.default_rng(14)
+    t, v = 5, 8
+    z = rng.standard_normal((t, v))
+    y = rng.integers(0, v, t)
+    a = np.array([1.0, -0.5, 2.0, 0.3, -1.2])
+    probe = O.loss_forward(*_identity_problem(z, y, np.zeros(t), a))
+    # tokens 0..2 at ratio 1 (inside), token 3 clipped from above (a>0), token 4 clipped from below (a<0)
+    logp_old = probe["logp"].copy()
+    logp_old[3] -= math.log(1.6)
+    logp_old[4] += math.log(2.0)
+    args = _identity_problem(z, y, logp_old, a)
+    fwd = O.loss_forward(*args)
+    _, dw = O.loss_backward(args[0], args[1], y, fwd["lse"], fwd["coef"])
+    g = dw.T                                   # H = I  ->  dW = g^T
+    p = scipy.special.softmax(z, axis=1)
+    onehot = np.eye(v)[y]
+    expect = a[:, None] * (p - onehot) / t
+    np.testing.assert_allclose(g[:3], expect[:3], atol=1e-14)
+    assert np.all(g[3:] == 0.0)
+    np.testing.assert_allclose(g.sum(axis=1), 0.0, atol=1e-15)
+
+
+def test_gradients_against_central_finite_differences():
+    rng = np.random.default_rng(15)
+    t, d, v = 7, 6, 11
+    h, w = rng.standard_normal((t, d)), rng.standard_normal((v, d)) * 0.5
+    y = rng.integers(0, v, t)
+    cu = [0, 2, 7]
+    a = np.array([0.9, -1.1])
+    mask = np.array([1, 1, 1, 0, 1, 1, 1], dtype=np.uint8)
+    base = O.loss_forward(h, w, y, np.zeros(t), mask, cu, a)
+    # offsets chosen so that tokens 1 (a>0, ratio 1.5) and 5 (a<0, ratio 0.6) clip; none sits on a bound
+    logp_old = base["logp"] - np.log([1.1, 1.5, 0.7, 1.0, 1.2, 0.6, 0.9])
+    fwd = O.loss_forward(h, w, y, logp_old, mask, cu, a)
+    assert 0 < fwd["unclipped"].sum() < t
+    gl = 1.7
+    dh, dw = O.loss_backward(h, w, y, fwd["lse"], fwd["coef"], grad_loss=gl)
+
+    def loss_at(hh, ww):
+        return gl * O.loss_forward(hh, ww, y, logp_old, mask, cu, a)["loss"]
+
+    step = 1e-6
+    for arr, grad in ((h, dh), (w, dw)):
+        num = np.zeros_like(arr)
+        for idx in np.ndindex(arr.shape):
+            keep = arr[idx]
+            arr[idx] = keep + step
+            up = loss_at(h, w)
+            arr[idx] = keep - step
+            dn = loss_at(h, w)
+            arr[idx] = keep
+            num[idx] = (up - dn) / (2 * step)
+        assert np.linalg.norm(num - grad) <= 1e-6 * np.linalg.norm(grad)
+    assert np.all(dh[3] == 0.0)                              # masked token
+
+
+def test_backward_matches_library_autograd():
+    torch = pytest.importorskip("torch")
+    rng = np.random.default_rng(16)
+    t, d, v = 9, 4, 13
+    h, w = rng.standard_normal((t, d)), rng.standard_normal((v, d))
+    y = rng.integers(0, v, t)
+    cu, a = [0, 4, 9], np.array([1.0, -0.6])
+    logp_old = O.loss_forward(h, w, y, np.zeros(t), None, cu, a)["logp"] + rng.normal(0, 0.2, t)
+    fwd = O.loss_forward(h, w, y, logp_old, None, cu, a)
+    dh, dw = O.loss_backward(h, w, y, fwd["lse"], fwd["coef"])
+    ht = torch.tensor(h, requires_grad=True)
+    wt = torch.tensor(w, requires_grad=True)
+    lp = torch.log_softmax(ht @ wt.T, dim=1)[torch.arange(t), torch.tensor(y)]
+    ratio = torch.exp(lp - torch.tensor(logp_old))
+    at = torch.tensor(np.repeat(a, np.diff(cu)))
+    loss = -torch.minimum(ratio * at, torch.clamp(ratio, 0.8, 1.28) * at).mean()
+    loss.backward()
+    assert abs(loss.item() - fwd["loss"]) < 1e-13
+    np.testing.assert_allclose(dh, ht.grad.numpy(), atol=1e-13)
+    np.testing.assert_allclose(dw, wt.grad.numpy(), atol=1e-13)
+
+
+def test_row_local_helper_equals_full_definition():
+    rng = np.random.default_rng(17)
+    t, d, v = 20, 8, 50
+    h, w = rng.standard_normal((t, d)), rng.standard_normal((v, d))
+    y = rng.integers(0, v, t)
+    cu, a = [0, 5, 20], np.array([0.4, -1.5])
+    mask = (rng.random(t) > 0.2).astype(np.uint8)
+    logp_old = rng.normal(-4, 0.3, t)
+    fwd = O.loss_forward(h, w, y, logp_old, mask, cu, a)
+    dh, _ = O.loss_backward(h, w, y, fwd["lse"], fwd["coef"], grad_loss=0.5)
+    rows = [0, 4, 5, 19]
+    a_tok = np.repeat(a, np.diff(cu))
+    sub = O.loss_rows(h[rows], w, y[rows], logp_old[rows], mask[rows], a_tok[rows], fwd["n_tok"],
+                      grad_loss=0.5, v_chunk=16)
+    np.testing.assert_allclose(sub["logp"], fwd["logp"][rows], atol=1e-13)
+    np.testing.assert_allclose(sub["lse"], fwd["lse"][rows], atol=1e-13)
+    np.testing.assert_allclose(sub["coef"], fwd["coef"][rows], atol=1e-15)
+    np.testing.assert_allclose(sub["dH"], dh[rows], atol=1e-14)
+
+
+def test_token_to_sequence_map():
+    np.testing.assert_array_equal(O.token_sequence_ids([0, 2, 2, 5], 5), [0, 0, 2, 2, 2])
