@@ -1,0 +1,207 @@
+/*
+ * libspo -- the data-parallel hot path of Single-stream Policy Optimization (SPO)
+ * on NVIDIA B200 (sm_100a).  Plain C ABI.
+ *
+ * Conventions (every entry point):
+ *   - Every pointer named d_* or documented "device" is device memory owned by the
+ *     caller; the library allocates nothing and frees nothing.  Pointers must be
+ *     16-byte aligned unless stated otherwise.  NULL is allowed only where marked
+ *     "optional".
+ *   - Work is enqueued on the caller's stream (`stream` is a cudaStream_t passed as
+ *     void*; NULL = the default stream).  No call synchronises the host.
+ *   - The return value is a host-side status (SPO_OK or a negative SPO_ERR_*),
+ *     produced by argument checks and launch errors only.  Conditions found on
+ *     the device (an id out of range, too few uniforms, a non-finite input, a
+ *     bounded wait that ran out) are OR-ed as SPO_DEV_* bits into the caller's
+ *     `d_status` word (device int32, must be zeroed by the caller beforehand);
+ *     the offending element is skipped, nothing traps.  d_status may be NULL.
+ *   - The device must be compute capability 10.x; otherwise SPO_ERR_UNSUPPORTED_ARCH.
+ *   - Tracker table layout: `ab` is [N][2] fp32, interleaved (alpha, beta) per prompt.
+ *   - Token rows are packed: sequence s owns rows cu_seqlens[s] .. cu_seqlens[s+1]-1.
+ */
+#ifndef SPO_H_
+#define SPO_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* host-side status */
+#define SPO_OK                        0
+#define SPO_ERR_INVALID_ARG          -1   /* NULL where required, negative size, bad flag */
+#define SPO_ERR_BAD_SHAPE            -2   /* size outside what the kernels support */
+#define SPO_ERR_BAD_ALIGNMENT        -3
+#define SPO_ERR_UNSUPPORTED_DTYPE    -4
+#define SPO_ERR_UNSUPPORTED_ARCH     -5
+#define SPO_ERR_WORKSPACE_TOO_SMALL  -6
+#define SPO_ERR_CUDA                 -7   /* see spo_last_cuda_error() */
+
+/* device-side status bits (OR-ed into *d_status) */
+#define SPO_DEV_ID_OUT_OF_RANGE       1   /* prompt id or target token outside its table */
+#define SPO_DEV_NONFINITE             2   /* NaN/Inf reward, divergence or table entry */
+#define SPO_DEV_UNIFORMS_EXHAUSTED    4   /* fewer than B distinct prompts accepted */
+#define SPO_DEV_TIMEOUT               8   /* a bounded wait inside a kernel ran out */
+#define SPO_DEV_ZERO_TOTAL_WEIGHT    16   /* all sampling weights are zero */
+
+/* element types of H / W / dH */
+#define SPO_DTYPE_F32   0
+#define SPO_DTYPE_BF16  1
+
+/* selectors for spo_workspace_bytes */
+#define SPO_WS_SAMPLE      0
+#define SPO_WS_ADVANTAGES  1
+#define SPO_WS_LOSS_FWD    2
+#define SPO_WS_LOSS_BWD    3
+
+/*
+ * Hyper-parameters.  Defaults (spo_default_params) are the values the paper prints:
+ * rho_min 0.875, rho_max 0.96, clip_lo 0.2, clip_hi 0.28 (appendix "Training and
+ * Evaluation Details"), eps_explore 0.05 (Sec. 3.3).  The paper names D_half but
+ * gives no value; the default here is 0.1.  norm_eps and norm_ddof settle what the
+ * paper leaves open about the batch standard deviation (population, +1e-8).
+ */
+typedef struct spo_params {
+  float   rho_min;
+  float   rho_max;
+  float   d_half;
+  float   eps_explore;
+  float   clip_lo;
+  float   clip_hi;
+  float   norm_eps;
+  int32_t norm_ddof;
+} spo_params;
+
+int32_t spo_default_params(spo_params* p /* host, out */);
+
+/*
+ * Algorithm 2 (SPO Initialization): N0 = 1/(1-rho_min); alpha0 = N0*v0; beta0 = N0*(1-v0).
+ *   ab  device out [N][2];  v0  device in [N] initial estimates in [0,1].
+ */
+int32_t spo_tracker_init(float* ab, const float* v0, int64_t N,
+                         const spo_params* params, void* stream);
+
+/*
+ * Prioritised sampling (Sec. 3.3, Eq. "sampling_coef"; Algorithm 1, the two
+ * sampling steps): w(x) = sqrt(v(1-v)) + eps_explore with v = alpha/(alpha+beta)
+ * (0.5 for an empty entry), then B distinct prompts drawn by weight.
+ *
+ * The draw is successive weighted sampling without replacement, made
+ * reproducible bit for bit: weights are computed in fp32 with IEEE-rounded
+ * operations in the order n=a+b, num=a*b, den=n*n, p=num/den, s=sqrt(p),
+ * w=s+eps; q_i = floor(w_i * 2^32) (uint64); C_i = q_0+..+q_i; Wtot = C_{N-1};
+ * for the k-th uniform U_k = floor(u_k * 2^32), t_k = floor(U_k*Wtot / 2^32),
+ * candidate = first i with C_i > t_k; candidates are accepted in order k unless
+ * already accepted, until B are accepted.
+ *
+ *   ab        device in  [N][2]
+ *   uniforms  device in  [M] fp32 in [0,1); M >= B (M = 2B is ample for N >> B)
+ *   out_ids   device out [B] int32, in acceptance order
+ *   out_w     device out [N] fp32 weights, optional
+ *   ws        device scratch, spo_workspace_bytes(SPO_WS_SAMPLE, ..., N, B, M) bytes
+ * Limits: 1 <= N < 2^31, 1 <= B <= M <= 2^20.
+ * Device status: SPO_DEV_UNIFORMS_EXHAUSTED if fewer than B distinct candidates
+ * (the tail of out_ids is then filled with -1), SPO_DEV_ZERO_TOTAL_WEIGHT,
+ * SPO_DEV_NONFINITE for a negative or non-finite table entry (weight treated as 0).
+ */
+int32_t spo_sample_prompts(const float* ab, int64_t N, const float* uniforms, int32_t M, int32_t B,
+                           int32_t* out_ids, float* out_w, void* ws, size_t ws_bytes,
+                           const spo_params* params, int32_t* d_status, void* stream);
+
+/*
+ * Advantage with the pre-update baseline and global normalisation (Sec. 3.2;
+ * Algorithm 1, "Compute raw advantage" and "Normalize advantages"):
+ *   A_j = r_j - v(ids_j);  mu, sigma over the B values;  A~_j = (A_j - mu)/(sigma + norm_eps)
+ * with sigma^2 = sum (A-mu)^2 / (B - norm_ddof).  Must be called BEFORE
+ * spo_tracker_update for the same batch: the baseline is the table as it stood.
+ *
+ *   ids     device in  [B] int32 in [0,N)
+ *   r       device in  [B] fp32 rewards
+ *   a_raw   device out [B] fp32, optional
+ *   a_norm  device out [B] fp32
+ *   stats   device out [4] fp32 = (mu, sigma, B, 0), optional
+ *   ws      device scratch, spo_workspace_bytes(SPO_WS_ADVANTAGES, ..., B, ...) bytes
+ * An id outside [0,N) sets SPO_DEV_ID_OUT_OF_RANGE and contributes A = 0.
+ */
+int32_t spo_advantages(const float* ab, int64_t N, const int32_t* ids, const float* r, int32_t B,
+                       float* a_raw, float* a_norm, float* stats, void* ws, size_t ws_bytes,
+                       const spo_params* params, int32_t* d_status, void* stream);
+
+/*
+ * KL-adaptive tracker update (Sec. 3.1, the update equation; Algorithm 1, "Update tracker"):
+ *   rho = clamp(2^(-D/D_half), rho_min, rho_max); alpha <- rho*alpha + r; beta <- rho*beta + (1-r)
+ * at row ids[j], in place.  ids must be distinct within a call (what sampling
+ * without replacement yields); duplicates race.
+ *
+ *   kl           device in: [B] per batch entry (kl_is_table = 0) or [N] per prompt,
+ *                gathered by id (kl_is_table = 1)
+ * A NaN divergence or reward sets SPO_DEV_NONFINITE and leaves the row untouched.
+ */
+int32_t spo_tracker_update(float* ab, int64_t N, const int32_t* ids, const float* r, const float* kl,
+                           int32_t kl_is_table, int32_t B,
+                           const spo_params* params, int32_t* d_status, void* stream);
+
+/*
+ * Policy loss forward (Sec. 3.2, the PPO-Clip objective with Clip-Higher bounds,
+ * evaluated from final hidden states).  Per token row t:
+ *   z = W h_t (never stored), lse = log sum_v exp z_v, logp = z[y_t] - lse,
+ *   ratio = exp(logp - logp_old_t), a = a_norm[seq(t)],
+ *   s_t = min(ratio*a, clip(ratio, 1-clip_lo, 1+clip_hi)*a),
+ *   loss = - sum_t mask_t s_t / n_tok,  n_tok = sum_t mask_t  (0 if n_tok = 0),
+ *   coef_t = d loss / d logp_t = -mask_t * a * ratio * [gradient passes the clip] / n_tok.
+ *
+ *   H           device in  [T][d], row-major, dtype as given (bf16: d % 64 == 0)
+ *   W           device in  [V][d], row-major, same dtype
+ *   y           device in  [T] int32 target token of each row
+ *   logp_old    device in  [T] fp32
+ *   mask        device in  [T] uint8, optional (NULL = all ones)
+ *   cu_seqlens  device in  [S+1] int32, cu_seqlens[0] = 0, cu_seqlens[S] = T
+ *   a_norm      device in  [S] fp32 normalised advantage per response
+ *   loss        device out [1] fp32
+ *   logp, lse, coef   device out [T] fp32 each
+ *   seq_sums    device out [S][3] fp32 = per response (sum mask*logp,
+ *               sum mask*(logp_old-logp), sum mask), optional
+ *   ws          device scratch, spo_workspace_bytes(SPO_WS_LOSS_FWD, T, d, V, ...) bytes
+ * A target outside [0,V) sets SPO_DEV_ID_OUT_OF_RANGE (the row gets logp = -inf, coef = 0).
+ */
+int32_t spo_loss_fwd(const void* H, const void* W, int32_t dtype,
+                     const int32_t* y, const float* logp_old, const uint8_t* mask,
+                     const int32_t* cu_seqlens, const float* a_norm,
+                     int64_t T, int32_t d, int32_t V, int32_t S,
+                     float* loss, float* logp, float* lse, float* coef, float* seq_sums,
+                     void* ws, size_t ws_bytes,
+                     const spo_params* params, int32_t* d_status, void* stream);
+
+/*
+ * Policy loss backward: with p = exp(z - lse) recomputed tile by tile,
+ *   g[t,v] = grad_loss * coef_t * (1[v = y_t] - p[t,v]);  dH = g W;  dW (+)= g^T H.
+ * lse and coef are the forward's outputs for the same H, W, y.
+ *
+ *   dH        device out [T][d], dtype dH_dtype (bf16 or fp32)
+ *   dW        device out [V][d] fp32; overwritten, or added to when dW_accumulate != 0
+ *   ws        device scratch, spo_workspace_bytes(SPO_WS_LOSS_BWD, T, d, V, ...) bytes.
+ *             For bf16 it holds a bounded chunk of g (a few thousand token rows
+ *             by V, bf16), never the whole [T][V] matrix.
+ */
+int32_t spo_loss_bwd(const void* H, const void* W, int32_t dtype, const int32_t* y,
+                     const float* lse, const float* coef, float grad_loss,
+                     int64_t T, int32_t d, int32_t V,
+                     void* dH, int32_t dH_dtype, float* dW, int32_t dW_accumulate,
+                     void* ws, size_t ws_bytes,
+                     const spo_params* params, int32_t* d_status, void* stream);
+
+/* Scratch size in bytes for one call of the selected entry point (host only, no CUDA call
+ * except a device-property query).  Arguments that the selected call does not use are ignored. */
+size_t spo_workspace_bytes(int32_t which, int64_t T, int32_t d, int32_t V,
+                           int64_t N, int32_t B, int32_t M);
+
+const char* spo_status_string(int32_t status);
+int32_t     spo_last_cuda_error(void);   /* cudaError_t of the last SPO_ERR_CUDA on this thread */
+int32_t     spo_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif  /* SPO_H_ */

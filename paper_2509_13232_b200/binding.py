@@ -1,0 +1,163 @@
+"""ctypes binding of libspo.so: one Python function per C entry point, same names.
+
+Argument marshalling only.  Tensors are torch CUDA tensors used as device
+buffers (``data_ptr()``), the stream is torch's current stream; every step of
+the path runs inside the library's CUDA kernels.  There is no CPU fallback: if
+the shared library has not been built, loading it raises.
+"""
+
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import POINTER, Structure, c_char_p, c_float, c_int32, c_int64, c_size_t, c_void_p
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libspo.so")
+
+SPO_OK = 0
+ERR_INVALID_ARG, ERR_BAD_SHAPE, ERR_BAD_ALIGNMENT = -1, -2, -3
+ERR_UNSUPPORTED_DTYPE, ERR_UNSUPPORTED_ARCH, ERR_WORKSPACE_TOO_SMALL, ERR_CUDA = -4, -5, -6, -7
+DEV_ID_OUT_OF_RANGE, DEV_NONFINITE, DEV_UNIFORMS_EXHAUSTED, DEV_TIMEOUT, DEV_ZERO_TOTAL_WEIGHT = 1, 2, 4, 8, 16
+DTYPE_F32, DTYPE_BF16 = 0, 1
+WS_SAMPLE, WS_ADVANTAGES, WS_LOSS_FWD, WS_LOSS_BWD = 0, 1, 2, 3
+
+EXPORTS = [
+    "spo_default_params", "spo_tracker_init", "spo_sample_prompts", "spo_advantages",
+    "spo_tracker_update", "spo_loss_fwd", "spo_loss_bwd", "spo_workspace_bytes",
+    "spo_status_string", "spo_last_cuda_error", "spo_version",
+]
+
+
+class SpoParams(Structure):
+    _fields_ = [
+        ("rho_min", c_float), ("rho_max", c_float), ("d_half", c_float), ("eps_explore", c_float),
+        ("clip_lo", c_float), ("clip_hi", c_float), ("norm_eps", c_float), ("norm_ddof", c_int32),
+    ]
+
+
+class SpoError(RuntimeError):
+    def __init__(self, status, where):
+        self.status = status
+        msg = lib().spo_status_string(status).decode()
+        if status == ERR_CUDA:
+            msg += " [cudaError %d]" % lib().spo_last_cuda_error()
+        super().__init__("%s: %s (%d)" % (where, msg, status))
+
+
+_lib = None
+
+
+def lib():
+    """The loaded shared library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise RuntimeError(
+                "libspo.so is missing (%s): build it with `python -m paper_2509_13232_b200.build`; "
+                "there is no fallback path" % _LIB_PATH)
+        L = ctypes.CDLL(_LIB_PATH)
+        P = POINTER(SpoParams)
+        L.spo_default_params.argtypes = [P]
+        L.spo_tracker_init.argtypes = [c_void_p, c_void_p, c_int64, P, c_void_p]
+        L.spo_sample_prompts.argtypes = [c_void_p, c_int64, c_void_p, c_int32, c_int32, c_void_p, c_void_p,
+                                         c_void_p, c_size_t, P, c_void_p, c_void_p]
+        L.spo_advantages.argtypes = [c_void_p, c_int64, c_void_p, c_void_p, c_int32, c_void_p, c_void_p,
+                                     c_void_p, c_void_p, c_size_t, P, c_void_p, c_void_p]
+        L.spo_tracker_update.argtypes = [c_void_p, c_int64, c_void_p, c_void_p, c_void_p, c_int32, c_int32,
+                                         P, c_void_p, c_void_p]
+        L.spo_loss_fwd.argtypes = [c_void_p, c_void_p, c_int32, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
+                                   c_int64, c_int32, c_int32, c_int32,
+                                   c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
+                                   c_void_p, c_size_t, P, c_void_p, c_void_p]
+        L.spo_loss_bwd.argtypes = [c_void_p, c_void_p, c_int32, c_void_p, c_void_p, c_void_p, c_float,
+                                   c_int64, c_int32, c_int32, c_void_p, c_int32, c_void_p, c_int32,
+                                   c_void_p, c_size_t, P, c_void_p, c_void_p]
+        L.spo_workspace_bytes.argtypes = [c_int32, c_int64, c_int32, c_int32, c_int64, c_int32, c_int32]
+        L.spo_workspace_bytes.restype = c_size_t
+        L.spo_status_string.argtypes = [c_int32]
+        L.spo_status_string.restype = c_char_p
+        for name in EXPORTS:
+            if name not in ("spo_workspace_bytes", "spo_status_string"):
+                getattr(L, name).restype = c_int32
+        _lib = L
+    return _lib
+
+
+def default_params(**overrides) -> SpoParams:
+    p = SpoParams()
+    rc = lib().spo_default_params(ctypes.byref(p))
+    if rc != SPO_OK:
+        raise SpoError(rc, "spo_default_params")
+    for k, v in overrides.items():
+        setattr(p, k, v)
+    return p
+
+
+def _ptr(t):
+    return None if t is None else c_void_p(t.data_ptr())
+
+
+def _stream():
+    import torch
+    return c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _check(rc, where):
+    if rc != SPO_OK:
+        raise SpoError(rc, where)
+
+
+def _dtype_code(t):
+    import torch
+    if t.dtype == torch.bfloat16:
+        return DTYPE_BF16
+    if t.dtype == torch.float32:
+        return DTYPE_F32
+    raise TypeError("H/W/dH must be float32 or bfloat16, got %s" % t.dtype)
+
+
+def spo_workspace_bytes(which, T=0, d=0, V=0, N=0, B=0, M=0) -> int:
+    return int(lib().spo_workspace_bytes(which, T, d, V, N, B, M))
+
+
+def spo_tracker_init(ab, v0, params):
+    _check(lib().spo_tracker_init(_ptr(ab), _ptr(v0), v0.numel(), ctypes.byref(params), _stream()),
+           "spo_tracker_init")
+
+
+def spo_sample_prompts(ab, uniforms, B, out_ids, out_w, ws, params, d_status):
+    _check(lib().spo_sample_prompts(_ptr(ab), ab.shape[0], _ptr(uniforms), uniforms.numel(), B, _ptr(out_ids),
+                                    _ptr(out_w), _ptr(ws), ws.numel() * ws.element_size(), ctypes.byref(params),
+                                    _ptr(d_status), _stream()), "spo_sample_prompts")
+
+
+def spo_advantages(ab, ids, r, a_raw, a_norm, stats, ws, params, d_status):
+    _check(lib().spo_advantages(_ptr(ab), ab.shape[0], _ptr(ids), _ptr(r), ids.numel(), _ptr(a_raw), _ptr(a_norm),
+                                _ptr(stats), _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size(),
+                                ctypes.byref(params), _ptr(d_status), _stream()), "spo_advantages")
+
+
+def spo_tracker_update(ab, ids, r, kl, kl_is_table, params, d_status):
+    _check(lib().spo_tracker_update(_ptr(ab), ab.shape[0], _ptr(ids), _ptr(r), _ptr(kl), int(kl_is_table),
+                                    ids.numel(), ctypes.byref(params), _ptr(d_status), _stream()),
+           "spo_tracker_update")
+
+
+def spo_loss_fwd(H, W, y, logp_old, mask, cu_seqlens, a_norm, loss, logp, lse, coef, seq_sums, ws, params,
+                 d_status):
+    T, d = H.shape
+    V = W.shape[0]
+    S = cu_seqlens.numel() - 1
+    _check(lib().spo_loss_fwd(_ptr(H), _ptr(W), _dtype_code(W), _ptr(y), _ptr(logp_old), _ptr(mask),
+                              _ptr(cu_seqlens), _ptr(a_norm), T, d, V, S, _ptr(loss), _ptr(logp), _ptr(lse),
+                              _ptr(coef), _ptr(seq_sums), _ptr(ws), ws.numel() * ws.element_size(),
+                              ctypes.byref(params), _ptr(d_status), _stream()), "spo_loss_fwd")
+
+
+def spo_loss_bwd(H, W, y, lse, coef, grad_loss, dH, dW, dW_accumulate, ws, params, d_status):
+    T, d = H.shape
+    V = W.shape[0]
+    _check(lib().spo_loss_bwd(_ptr(H), _ptr(W), _dtype_code(W), _ptr(y), _ptr(lse), _ptr(coef),
+                              c_float(grad_loss), T, d, V, _ptr(dH), _dtype_code(dH), _ptr(dW),
+                              int(dW_accumulate), _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size(),
+                              ctypes.byref(params), _ptr(d_status), _stream()), "spo_loss_bwd")

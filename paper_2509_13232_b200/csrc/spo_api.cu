@@ -1,0 +1,254 @@
+// C-ABI entry points of libspo: argument checks, workspace carving, dispatch.
+// See include/spo.h for the contract of every call.
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <string.h>
+
+#include "spo_internal.h"
+
+namespace spo {
+
+static thread_local int32_t g_last_cuda_error = 0;
+
+int sm_count() {
+  static int cached[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return 148; }
+  if (dev < 0 || dev >= 64) return 148;
+  if (cached[dev] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+      cudaGetLastError();
+      return 148;
+    }
+    cached[dev] = n;
+  }
+  return cached[dev];
+}
+
+int device_is_sm100() {
+  int dev = 0, major = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return 0; }
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) {
+    cudaGetLastError();
+    return 0;
+  }
+  return major == 10;
+}
+
+int fwd_bf16_nsplit(int64_t T, int32_t V);   // spo_loss_tc.cu
+
+FwdWs fwd_ws_layout(int64_t T, int32_t d, int32_t V, int32_t dtype) {
+  (void)d;
+  FwdWs L{};
+  L.nsplit = dtype == SPO_DTYPE_BF16 ? fwd_bf16_nsplit(T, V) : 1;
+  L.fin_blocks = ceil_div(T > 0 ? T : 1, kFinalizeThreads);
+  size_t off = 0;
+  L.partials = off;   off = align_up(off + sizeof(FwdPartial) * (size_t)L.nsplit * (size_t)(T > 0 ? T : 1), 256);
+  L.block_sums = off; off = align_up(off + sizeof(double) * (size_t)L.fin_blocks, 256);
+  L.counters = off;   off = align_up(off + 4 * sizeof(int32_t), 256);
+  L.total = off;
+  return L;
+}
+
+static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static inline int32_t cuda_fail(cudaError_t e) {
+  g_last_cuda_error = (int32_t)e;
+  return SPO_ERR_CUDA;
+}
+
+static bool params_ok(const spo_params* p) {
+  if (!p) return false;
+  if (!(p->rho_min >= 0.0f) || !(p->rho_max <= 1.0f) || !(p->rho_min <= p->rho_max)) return false;
+  if (!(p->d_half > 0.0f)) return false;
+  if (!(p->eps_explore >= 0.0f)) return false;
+  if (!(p->clip_lo >= 0.0f) || !(p->clip_lo < 1.0f) || !(p->clip_hi >= 0.0f)) return false;
+  if (!(p->norm_eps >= 0.0f)) return false;
+  if (p->norm_ddof != 0 && p->norm_ddof != 1) return false;
+  return true;
+}
+
+}  // namespace spo
+
+using namespace spo;
+
+extern "C" {
+
+int32_t spo_default_params(spo_params* p) {
+  if (!p) return SPO_ERR_INVALID_ARG;
+  p->rho_min = 0.875f;
+  p->rho_max = 0.96f;
+  p->d_half = 0.1f;
+  p->eps_explore = 0.05f;
+  p->clip_lo = 0.2f;
+  p->clip_hi = 0.28f;
+  p->norm_eps = 1e-8f;
+  p->norm_ddof = 0;
+  return SPO_OK;
+}
+
+int32_t spo_tracker_init(float* ab, const float* v0, int64_t N, const spo_params* params, void* stream) {
+  if (!params_ok(params) || N < 0 || (N > 0 && (!ab || !v0))) return SPO_ERR_INVALID_ARG;
+  if (!(params->rho_min < 1.0f)) return SPO_ERR_INVALID_ARG;
+  if (N >= ((int64_t)1 << 31)) return SPO_ERR_BAD_SHAPE;
+  if (!aligned16(ab) || !aligned16(v0)) return SPO_ERR_BAD_ALIGNMENT;
+  if (!device_is_sm100()) return SPO_ERR_UNSUPPORTED_ARCH;
+  const float n0 = 1.0f / (1.0f - params->rho_min);
+  cudaError_t e = launch_tracker_init(ab, v0, N, n0, (cudaStream_t)stream);
+  return e == cudaSuccess ? SPO_OK : cuda_fail(e);
+}
+
+int32_t spo_sample_prompts(const float* ab, int64_t N, const float* uniforms, int32_t M, int32_t B,
+                           int32_t* out_ids, float* out_w, void* ws, size_t ws_bytes,
+                           const spo_params* params, int32_t* d_status, void* stream) {
+  if (!params_ok(params) || !ab || !uniforms || !out_ids || !ws) return SPO_ERR_INVALID_ARG;
+  if (N < 1 || N >= ((int64_t)1 << 31) || B < 1 || M < B || M > (1 << 20)) return SPO_ERR_BAD_SHAPE;
+  if (!aligned16(ab) || !aligned16(uniforms) || !aligned16(out_ids) || !aligned16(out_w) || !aligned16(ws))
+    return SPO_ERR_BAD_ALIGNMENT;
+  if (!device_is_sm100()) return SPO_ERR_UNSUPPORTED_ARCH;
+  const SampleWs L = sample_ws_layout(N, M);
+  if (ws_bytes < L.total) return SPO_ERR_WORKSPACE_TOO_SMALL;
+  cudaError_t e = launch_sample(ab, N, uniforms, M, B, out_ids, out_w, (char*)ws, L, params->eps_explore, d_status,
+                                (cudaStream_t)stream);
+  return e == cudaSuccess ? SPO_OK : cuda_fail(e);
+}
+
+int32_t spo_advantages(const float* ab, int64_t N, const int32_t* ids, const float* r, int32_t B,
+                       float* a_raw, float* a_norm, float* stats, void* ws, size_t ws_bytes,
+                       const spo_params* params, int32_t* d_status, void* stream) {
+  if (!params_ok(params) || !ab || !ids || !r || !a_norm) return SPO_ERR_INVALID_ARG;
+  if (N < 1 || N >= ((int64_t)1 << 31) || B < 1) return SPO_ERR_BAD_SHAPE;
+  if (!aligned16(ab) || !aligned16(ids) || !aligned16(r) || !aligned16(a_raw) || !aligned16(a_norm) ||
+      !aligned16(stats) || !aligned16(ws))
+    return SPO_ERR_BAD_ALIGNMENT;
+  if (!device_is_sm100()) return SPO_ERR_UNSUPPORTED_ARCH;
+  if (B > kAdvSingleBlockMax) {
+    if (!ws) return SPO_ERR_INVALID_ARG;
+    if (ws_bytes < spo_workspace_bytes(SPO_WS_ADVANTAGES, 0, 0, 0, N, B, 0)) return SPO_ERR_WORKSPACE_TOO_SMALL;
+  }
+  cudaError_t e = launch_advantages(ab, N, ids, r, B, a_raw, a_norm, stats, (char*)ws, params->norm_eps,
+                                    params->norm_ddof, d_status, (cudaStream_t)stream);
+  return e == cudaSuccess ? SPO_OK : cuda_fail(e);
+}
+
+int32_t spo_tracker_update(float* ab, int64_t N, const int32_t* ids, const float* r, const float* kl,
+                           int32_t kl_is_table, int32_t B, const spo_params* params, int32_t* d_status,
+                           void* stream) {
+  if (!params_ok(params) || !ab || B < 0 || (B > 0 && (!ids || !r || !kl))) return SPO_ERR_INVALID_ARG;
+  if (kl_is_table != 0 && kl_is_table != 1) return SPO_ERR_INVALID_ARG;
+  if (N < 1 || N >= ((int64_t)1 << 31)) return SPO_ERR_BAD_SHAPE;
+  if (!aligned16(ab) || !aligned16(ids) || !aligned16(r) || !aligned16(kl)) return SPO_ERR_BAD_ALIGNMENT;
+  if (!device_is_sm100()) return SPO_ERR_UNSUPPORTED_ARCH;
+  cudaError_t e = launch_tracker_update(ab, N, ids, r, kl, kl_is_table, B, params->rho_min, params->rho_max,
+                                        params->d_half, d_status, (cudaStream_t)stream);
+  return e == cudaSuccess ? SPO_OK : cuda_fail(e);
+}
+
+static int32_t check_loss_shape(int32_t dtype, int64_t T, int32_t d, int32_t V) {
+  if (dtype != SPO_DTYPE_F32 && dtype != SPO_DTYPE_BF16) return SPO_ERR_UNSUPPORTED_DTYPE;
+  if (T < 0 || d < 1 || V < 1) return SPO_ERR_INVALID_ARG;
+  if (T >= ((int64_t)1 << 31) - 256) return SPO_ERR_BAD_SHAPE;
+  if (dtype == SPO_DTYPE_BF16 && (d % 64) != 0) return SPO_ERR_BAD_SHAPE;
+  if (dtype == SPO_DTYPE_F32 && (d > 4096 || (d % 4) != 0)) return SPO_ERR_BAD_SHAPE;
+  return SPO_OK;
+}
+
+int32_t spo_loss_fwd(const void* H, const void* W, int32_t dtype, const int32_t* y, const float* logp_old,
+                     const uint8_t* mask, const int32_t* cu_seqlens, const float* a_norm, int64_t T, int32_t d,
+                     int32_t V, int32_t S, float* loss, float* logp, float* lse, float* coef, float* seq_sums,
+                     void* ws, size_t ws_bytes, const spo_params* params, int32_t* d_status, void* stream) {
+  int32_t rc = check_loss_shape(dtype, T, d, V);
+  if (rc != SPO_OK) return rc;
+  if (!params_ok(params) || !W || !loss || !ws || !cu_seqlens || S < 0) return SPO_ERR_INVALID_ARG;
+  if (T > 0 && (!H || !y || !logp_old || !a_norm || !logp || !lse || !coef || S < 1)) return SPO_ERR_INVALID_ARG;
+  if (!aligned16(H) || !aligned16(W) || !aligned16(y) || !aligned16(logp_old) || !aligned16(cu_seqlens) ||
+      !aligned16(a_norm) || !aligned16(logp) || !aligned16(lse) || !aligned16(coef) || !aligned16(ws))
+    return SPO_ERR_BAD_ALIGNMENT;
+  if (!device_is_sm100()) return SPO_ERR_UNSUPPORTED_ARCH;
+  const FwdWs L = fwd_ws_layout(T, d, V, dtype);
+  if (ws_bytes < L.total) return SPO_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t st = (cudaStream_t)stream;
+  char* w8 = (char*)ws;
+  FwdPartial* partials = reinterpret_cast<FwdPartial*>(w8 + L.partials);
+  double* block_sums = reinterpret_cast<double*>(w8 + L.block_sums);
+  int32_t* counters = reinterpret_cast<int32_t*>(w8 + L.counters);
+  cudaError_t e = launch_fwd_prepare(mask, T, counters, st);
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (dtype == SPO_DTYPE_BF16)
+    e = launch_fwd_bf16(H, W, y, T, d, V, partials, L.nsplit, d_status, st);
+  else
+    e = launch_fwd_f32((const float*)H, (const float*)W, y, T, d, V, partials, st);
+  if (e != cudaSuccess) return cuda_fail(e);
+  e = launch_fwd_finalize(partials, L.nsplit, y, logp_old, mask, cu_seqlens, a_norm, T, V, S, params->clip_lo,
+                          params->clip_hi, loss, logp, lse, coef, seq_sums, block_sums, counters, L.fin_blocks,
+                          d_status, st);
+  return e == cudaSuccess ? SPO_OK : cuda_fail(e);
+}
+
+int32_t spo_loss_bwd(const void* H, const void* W, int32_t dtype, const int32_t* y, const float* lse,
+                     const float* coef, float grad_loss, int64_t T, int32_t d, int32_t V, void* dH,
+                     int32_t dH_dtype, float* dW, int32_t dW_accumulate, void* ws, size_t ws_bytes,
+                     const spo_params* params, int32_t* d_status, void* stream) {
+  int32_t rc = check_loss_shape(dtype, T, d, V);
+  if (rc != SPO_OK) return rc;
+  if (dH_dtype != SPO_DTYPE_F32 && dH_dtype != SPO_DTYPE_BF16) return SPO_ERR_UNSUPPORTED_DTYPE;
+  if (!params_ok(params) || !W || !dW) return SPO_ERR_INVALID_ARG;
+  if (T > 0 && (!H || !y || !lse || !coef || !dH)) return SPO_ERR_INVALID_ARG;
+  if (dtype == SPO_DTYPE_BF16 && !ws) return SPO_ERR_INVALID_ARG;
+  if (!aligned16(H) || !aligned16(W) || !aligned16(y) || !aligned16(lse) || !aligned16(coef) || !aligned16(dH) ||
+      !aligned16(dW) || !aligned16(ws))
+    return SPO_ERR_BAD_ALIGNMENT;
+  if (!device_is_sm100()) return SPO_ERR_UNSUPPORTED_ARCH;
+  cudaStream_t st = (cudaStream_t)stream;
+  cudaError_t e;
+  if (dtype == SPO_DTYPE_BF16) {
+    const BwdWs L = bwd_ws_layout(T, d, V);
+    if (ws_bytes < L.total) return SPO_ERR_WORKSPACE_TOO_SMALL;
+    e = launch_bwd_bf16(H, W, y, lse, coef, grad_loss, T, d, V, dH, dH_dtype, dW, dW_accumulate, (char*)ws, L,
+                        d_status, st);
+  } else {
+    e = launch_bwd_f32((const float*)H, (const float*)W, y, lse, coef, grad_loss, T, d, V, dH, dH_dtype, dW,
+                       dW_accumulate, st);
+  }
+  return e == cudaSuccess ? SPO_OK : cuda_fail(e);
+}
+
+size_t spo_workspace_bytes(int32_t which, int64_t T, int32_t d, int32_t V, int64_t N, int32_t B, int32_t M) {
+  switch (which) {
+    case SPO_WS_SAMPLE:
+      if (N < 1 || M < 1) return 0;
+      return sample_ws_layout(N, M).total;
+    case SPO_WS_ADVANTAGES:
+      if (B <= kAdvSingleBlockMax) return 256;
+      return align_up(sizeof(double) * 2 * (size_t)adv_blocks(B), 256);
+    case SPO_WS_LOSS_FWD:
+      if (T < 0 || V < 1) return 0;
+      return fwd_ws_layout(T, d, V, (d % 64) == 0 ? SPO_DTYPE_BF16 : SPO_DTYPE_F32).total;
+    case SPO_WS_LOSS_BWD:
+      if (T < 0 || V < 1 || d < 1) return 0;
+      return bwd_ws_layout(T, d, V).total;
+    default:
+      return 0;
+  }
+}
+
+const char* spo_status_string(int32_t status) {
+  switch (status) {
+    case SPO_OK: return "ok";
+    case SPO_ERR_INVALID_ARG: return "invalid argument";
+    case SPO_ERR_BAD_SHAPE: return "unsupported shape";
+    case SPO_ERR_BAD_ALIGNMENT: return "pointer not 16-byte aligned";
+    case SPO_ERR_UNSUPPORTED_DTYPE: return "unsupported element type";
+    case SPO_ERR_UNSUPPORTED_ARCH: return "device is not compute capability 10.x";
+    case SPO_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case SPO_ERR_CUDA: return "CUDA error (see spo_last_cuda_error)";
+    default: return "unknown status";
+  }
+}
+
+int32_t spo_last_cuda_error(void) { return g_last_cuda_error; }
+
+int32_t spo_version(void) { return 100; }
+
+}  // extern "C"

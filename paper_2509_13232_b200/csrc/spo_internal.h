@@ -1,0 +1,95 @@
+// Internal declarations shared by the translation units of libspo.
+// Nothing here is part of the public ABI (see include/spo.h).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "spo.h"
+
+namespace spo {
+
+// ---- small helpers ------------------------------------------------------
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+int sm_count();                       // SMs of the current device (cached per device)
+int device_is_sm100();                // 1 when the current device is compute capability 10.x
+
+// ---- sampler ------------------------------------------------------------
+constexpr int kSampleTile = 2048;     // table entries per partial-sum tile
+
+struct SampleWs {
+  size_t tile_sums, tile_offsets, cand, keys, vals, total;
+  int64_t n_tiles;
+  int64_t hash_slots;
+};
+SampleWs sample_ws_layout(int64_t N, int32_t M);
+
+cudaError_t launch_tracker_init(float* ab, const float* v0, int64_t N, float n0, cudaStream_t st);
+cudaError_t launch_sample(const float* ab, int64_t N, const float* u, int32_t M, int32_t B,
+                          int32_t* out_ids, float* out_w, char* ws, const SampleWs& L,
+                          float eps, int32_t* d_status, cudaStream_t st);
+
+// ---- advantages / tracker ------------------------------------------------
+constexpr int kAdvSingleBlockMax = 8192;
+int adv_blocks(int32_t B);
+cudaError_t launch_advantages(const float* ab, int64_t N, const int32_t* ids, const float* r, int32_t B,
+                              float* a_raw, float* a_norm, float* stats, char* ws,
+                              float norm_eps, int32_t ddof, int32_t* d_status, cudaStream_t st);
+cudaError_t launch_tracker_update(float* ab, int64_t N, const int32_t* ids, const float* r,
+                                  const float* kl, int kl_is_table, int32_t B,
+                                  float rho_min, float rho_max, float d_half,
+                                  int32_t* d_status, cudaStream_t st);
+
+// ---- loss: pieces shared by the fp32 and bf16 paths ------------------------
+// Forward partial statistics of one vocabulary split, per token row:
+// (running max of z*log2(e), sum of 2^(z*log2(e) - max), target logit or -inf).
+struct FwdPartial { float m2, l, zt; float pad; };
+
+constexpr int kFinalizeThreads = 256;
+
+struct FwdWs {
+  size_t partials;      // FwdPartial [nsplit][T]
+  size_t block_sums;    // double [finalize blocks]
+  size_t counters;      // int32 [4]: n_tok, ticket
+  size_t total;
+  int nsplit;
+  int64_t fin_blocks;
+};
+FwdWs fwd_ws_layout(int64_t T, int32_t d, int32_t V, int32_t dtype);
+
+cudaError_t launch_fwd_prepare(const uint8_t* mask, int64_t T, int32_t* counters, cudaStream_t st);
+cudaError_t launch_fwd_finalize(const FwdPartial* partials, int nsplit, const int32_t* y,
+                                const float* logp_old, const uint8_t* mask, const int32_t* cu_seqlens,
+                                const float* a_norm, int64_t T, int32_t V, int32_t S,
+                                float clip_lo, float clip_hi,
+                                float* loss, float* logp, float* lse, float* coef, float* seq_sums,
+                                double* block_sums, int32_t* counters, int64_t fin_blocks,
+                                int32_t* d_status, cudaStream_t st);
+
+// fp32 SIMT path
+cudaError_t launch_fwd_f32(const float* H, const float* W, const int32_t* y, int64_t T, int32_t d, int32_t V,
+                           FwdPartial* partials, cudaStream_t st);
+cudaError_t launch_bwd_f32(const float* H, const float* W, const int32_t* y, const float* lse,
+                           const float* coef, float grad_loss, int64_t T, int32_t d, int32_t V,
+                           void* dH, int32_t dH_dtype, float* dW, int accumulate, cudaStream_t st);
+
+// bf16 tensor-core path
+struct BwdWs {
+  size_t g;             // bf16 [chunk_rows][ldg]
+  size_t total;
+  int64_t chunk_rows;   // token rows per chunk (multiple of 128)
+  int64_t ldg;          // row pitch of g in elements (multiple of 256)
+};
+BwdWs bwd_ws_layout(int64_t T, int32_t d, int32_t V);
+
+cudaError_t launch_fwd_bf16(const void* H, const void* W, const int32_t* y, int64_t T, int32_t d, int32_t V,
+                            FwdPartial* partials, int nsplit, int32_t* d_status, cudaStream_t st);
+cudaError_t launch_bwd_bf16(const void* H, const void* W, const int32_t* y, const float* lse,
+                            const float* coef, float grad_loss, int64_t T, int32_t d, int32_t V,
+                            void* dH, int32_t dH_dtype, float* dW, int accumulate,
+                            char* ws, const BwdWs& L, int32_t* d_status, cudaStream_t st);
+
+}  // namespace spo

@@ -1,0 +1,335 @@
+// Loss pieces shared by both element types (token count, per-token finalisation of the
+// clipped surrogate, per-response sums) and the plain fp32 SIMT forward / backward used
+// for fp32 inputs.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <math_constants.h>
+#include <stdint.h>
+
+#include "spo_internal.h"
+
+namespace spo {
+
+namespace {
+
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+__device__ __forceinline__ void flag(int32_t* d_status, int bit) {
+  if (d_status) atomicOr(d_status, bit);
+}
+
+__device__ __forceinline__ double warp_sum_f64(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+__device__ __forceinline__ float warp_sum_f32(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// counters[0] = number of unmasked token rows
+__global__ void __launch_bounds__(256)
+count_mask_kernel(const uint8_t* __restrict__ mask, int64_t T, int32_t* counters) {
+  int local = 0;
+  for (int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x; i < T; i += (int64_t)gridDim.x * 256)
+    local += mask[i] != 0;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) local += __shfl_xor_sync(0xffffffffu, local, o);
+  if ((threadIdx.x & 31) == 0 && local) atomicAdd(&counters[0], local);
+}
+
+__global__ void set_count_kernel(int32_t value, int32_t* counters) { counters[0] = value; }
+
+// Per token: merge the vocabulary splits' (max, sum-exp, target logit), then the
+// importance ratio, the clipped surrogate (Sec. 3.2) and d loss / d logp.
+__global__ void __launch_bounds__(kFinalizeThreads)
+fwd_finalize_kernel(const FwdPartial* __restrict__ partials, int nsplit, const int32_t* __restrict__ y,
+                    const float* __restrict__ logp_old, const uint8_t* __restrict__ mask,
+                    const int32_t* __restrict__ cu_seqlens, const float* __restrict__ a_norm,
+                    int64_t T, int32_t V, int32_t S, float clip_lo, float clip_hi,
+                    float* __restrict__ loss, float* __restrict__ logp_out, float* __restrict__ lse_out,
+                    float* __restrict__ coef_out, double* block_sums, int32_t* counters, int32_t* d_status) {
+  const int64_t t = (int64_t)blockIdx.x * kFinalizeThreads + threadIdx.x;
+  const int32_t n_tok = counters[0];
+  double contrib = 0.0;
+  if (t < T) {
+    float m2 = -CUDART_INF_F, zt = -CUDART_INF_F;
+    for (int s = 0; s < nsplit; ++s) {
+      FwdPartial p = partials[(int64_t)s * T + t];
+      m2 = fmaxf(m2, p.m2);
+      zt = fmaxf(zt, p.zt);
+    }
+    float l = 0.0f;
+    for (int s = 0; s < nsplit; ++s) {
+      FwdPartial p = partials[(int64_t)s * T + t];
+      l += p.l * exp2f(p.m2 - m2);
+    }
+    const float lse = (m2 + log2f(l)) * kLn2;
+    const int32_t yt = y[t];
+    float lp, coef = 0.0f;
+    if (yt < 0 || yt >= V) {
+      flag(d_status, SPO_DEV_ID_OUT_OF_RANGE);
+      lp = -CUDART_INF_F;
+    } else {
+      lp = zt - lse;
+      const float ratio = expf(lp - logp_old[t]);
+      int lo = 0, hi = S;                    // sequence with cu[lo] <= t < cu[lo+1]
+      while (hi - lo > 1) {
+        int mid = (lo + hi) >> 1;
+        if ((int64_t)cu_seqlens[mid] <= t) lo = mid; else hi = mid;
+      }
+      const float a = a_norm[lo];
+      const bool on = mask ? mask[t] != 0 : true;
+      const float hi_b = 1.0f + clip_hi, lo_b = 1.0f - clip_lo;
+      const float sur = fminf(ratio * a, fminf(fmaxf(ratio, lo_b), hi_b) * a);
+      const bool passes = a >= 0.0f ? ratio <= hi_b : ratio >= lo_b;
+      if (on) {
+        contrib = (double)sur;
+        if (passes && n_tok > 0) coef = -a * ratio / (float)n_tok;
+      }
+    }
+    logp_out[t] = lp;
+    lse_out[t] = lse;
+    coef_out[t] = coef;
+  }
+  __shared__ double s_part[kFinalizeThreads / 32];
+  __shared__ int s_last;
+  contrib = warp_sum_f64(contrib);
+  if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = contrib;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double b = 0.0;
+#pragma unroll
+    for (int w = 0; w < kFinalizeThreads / 32; ++w) b += s_part[w];
+    block_sums[blockIdx.x] = b;
+    __threadfence();
+    int ticket = atomicAdd(&counters[1], 1);
+    s_last = (ticket == (int)gridDim.x - 1);
+  }
+  __syncthreads();
+  if (s_last) {                              // the last block to finish folds all blocks in index order
+    __threadfence();
+    double acc = 0.0;
+    const volatile double* bs = block_sums;
+    for (int i = threadIdx.x; i < (int)gridDim.x; i += kFinalizeThreads) acc += bs[i];
+    acc = warp_sum_f64(acc);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = acc;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      double tot = 0.0;
+#pragma unroll
+      for (int w = 0; w < kFinalizeThreads / 32; ++w) tot += s_part[w];
+      loss[0] = n_tok > 0 ? (float)(-tot / (double)n_tok) : 0.0f;
+    }
+  }
+}
+
+// One block per response: (sum mask*logp, sum mask*(logp_old - logp), sum mask).
+__global__ void __launch_bounds__(256)
+seq_sums_kernel(const float* __restrict__ logp, const float* __restrict__ logp_old, const uint8_t* __restrict__ mask,
+                const int32_t* __restrict__ cu_seqlens, float* __restrict__ seq_sums) {
+  const int s = blockIdx.x;
+  const int64_t lo = cu_seqlens[s], hi = cu_seqlens[s + 1];
+  double a = 0.0, b = 0.0, c = 0.0;
+  for (int64_t t = lo + threadIdx.x; t < hi; t += 256) {
+    if (mask && mask[t] == 0) continue;
+    float lp = logp[t];
+    a += lp;
+    b += (double)logp_old[t] - lp;
+    c += 1.0;
+  }
+  __shared__ double s_a[8], s_b[8], s_c[8];
+  a = warp_sum_f64(a); b = warp_sum_f64(b); c = warp_sum_f64(c);
+  if ((threadIdx.x & 31) == 0) { s_a[threadIdx.x >> 5] = a; s_b[threadIdx.x >> 5] = b; s_c[threadIdx.x >> 5] = c; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double ta = 0, tb = 0, tc = 0;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) { ta += s_a[w]; tb += s_b[w]; tc += s_c[w]; }
+    seq_sums[3 * s + 0] = (float)ta;
+    seq_sums[3 * s + 1] = (float)tb;
+    seq_sums[3 * s + 2] = (float)tc;
+  }
+}
+
+// ---------------------------------------------------------------------------
+// fp32 SIMT forward: one block per token row, one warp per vocabulary row at a time.
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(128)
+fwd_f32_kernel(const float* __restrict__ H, const float* __restrict__ W, const int32_t* __restrict__ y,
+               int32_t d, int32_t V, FwdPartial* __restrict__ partials) {
+  extern __shared__ float s_h[];
+  const int64_t t = blockIdx.x;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (int k = threadIdx.x; k < d; k += 128) s_h[k] = H[t * d + k];
+  __syncthreads();
+  const int32_t yt = y[t];
+  float m2 = -CUDART_INF_F, l = 0.0f, zt = -CUDART_INF_F;
+  for (int v = warp; v < V; v += 4) {
+    const float* wr = W + (int64_t)v * d;
+    float acc = 0.0f;
+    for (int k = lane; k < d; k += 32) acc = fmaf(wr[k], s_h[k], acc);
+    const float z = warp_sum_f32(acc);
+    const float z2 = z * kLog2e;
+    const float mn = fmaxf(m2, z2);
+    l = l * exp2f(m2 - mn) + exp2f(z2 - mn);
+    m2 = mn;
+    if (v == yt) zt = z;
+  }
+  __shared__ float s_m[4], s_l[4], s_z[4];
+  if (lane == 0) { s_m[warp] = m2; s_l[warp] = l; s_z[warp] = zt; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float mm = fmaxf(fmaxf(s_m[0], s_m[1]), fmaxf(s_m[2], s_m[3]));
+    float ll = 0.0f, zz = -CUDART_INF_F;
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+      if (s_l[w] > 0.0f) ll += s_l[w] * exp2f(s_m[w] - mm);
+      zz = fmaxf(zz, s_z[w]);
+    }
+    FwdPartial p;
+    p.m2 = mm; p.l = ll; p.zt = zz; p.pad = 0.0f;
+    partials[t] = p;
+  }
+}
+
+// ---------------------------------------------------------------------------
+// fp32 SIMT backward.  One block per output row x (a token row of dH, or a vocabulary
+// row of dW).  For every row j of the other matrix Y: s = <x, Y_j>, g = c*(1[v=y_t] - e^{s-lse_t}),
+// out += g * Y_j.  DW = false: x = H[t], Y = W.  DW = true: x = W[v], Y = H.
+// ---------------------------------------------------------------------------
+constexpr int kBwdChunk = 256;
+constexpr int kBwdMaxPerThread = 32;       // d <= 128 * 32
+
+template <bool DW>
+__global__ void __launch_bounds__(128)
+bwd_f32_kernel(const float* __restrict__ H, const float* __restrict__ W, const int32_t* __restrict__ y,
+               const float* __restrict__ lse, const float* __restrict__ coef, float grad_loss,
+               int64_t T, int32_t d, int32_t V, void* out, int out_bf16, int accumulate) {
+  extern __shared__ float s_mem[];
+  float* s_x = s_mem;                       // [d]
+  float* s_g = s_mem + d;                   // [kBwdChunk]
+  const int64_t row = blockIdx.x;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const float* X = DW ? W : H;
+  const float* Y = DW ? H : W;
+  const int64_t n_other = DW ? T : (int64_t)V;
+  for (int k = threadIdx.x; k < d; k += 128) s_x[k] = X[row * d + k];
+  float acc[kBwdMaxPerThread];
+#pragma unroll
+  for (int i = 0; i < kBwdMaxPerThread; ++i) acc[i] = 0.0f;
+  float c_row = 0.0f, lse_row = 0.0f;
+  int32_t y_row = -1;
+  if (!DW) { c_row = grad_loss * coef[row]; lse_row = lse[row]; y_row = y[row]; }
+  __syncthreads();
+  for (int64_t j0 = 0; j0 < n_other; j0 += kBwdChunk) {
+    const int n_here = (int)((n_other - j0) < kBwdChunk ? (n_other - j0) : kBwdChunk);
+    for (int jj = warp; jj < n_here; jj += 4) {
+      const int64_t j = j0 + jj;
+      float c = c_row, ls = lse_row;
+      bool hit;
+      if (DW) { c = grad_loss * coef[j]; ls = lse[j]; hit = (y[j] == (int32_t)row); }
+      else    { hit = ((int32_t)j == y_row); }
+      float g = 0.0f;
+      if (c != 0.0f) {                      // warp-uniform
+        const float* yr = Y + j * d;
+        float a = 0.0f;
+        for (int k = lane; k < d; k += 32) a = fmaf(yr[k], s_x[k], a);
+        const float s = warp_sum_f32(a);
+        g = c * ((hit ? 1.0f : 0.0f) - expf(s - ls));
+      }
+      if (lane == 0) s_g[jj] = g;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < kBwdMaxPerThread; ++i) {
+      const int k = threadIdx.x + 128 * i;
+      if (k < d) {
+        float a = acc[i];
+        for (int jj = 0; jj < n_here; ++jj) a = fmaf(s_g[jj], Y[(j0 + jj) * d + k], a);
+        acc[i] = a;
+      }
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int i = 0; i < kBwdMaxPerThread; ++i) {
+    const int k = threadIdx.x + 128 * i;
+    if (k < d) {
+      const int64_t o = row * d + k;
+      if (out_bf16) {
+        reinterpret_cast<__nv_bfloat16*>(out)[o] = __float2bfloat16_rn(acc[i]);
+      } else {
+        float* of = reinterpret_cast<float*>(out);
+        of[o] = accumulate ? of[o] + acc[i] : acc[i];
+      }
+    }
+  }
+}
+
+}  // namespace
+
+// ---------------------------------------------------------------------------
+// host launchers
+// ---------------------------------------------------------------------------
+
+cudaError_t launch_fwd_prepare(const uint8_t* mask, int64_t T, int32_t* counters, cudaStream_t st) {
+  cudaError_t e = cudaMemsetAsync(counters, 0, 4 * sizeof(int32_t), st);
+  if (e != cudaSuccess) return e;
+  if (mask) {
+    int64_t blocks = ceil_div(T > 0 ? T : 1, 256 * 8);
+    int64_t cap = (int64_t)sm_count() * 8;
+    if (blocks > cap) blocks = cap;
+    count_mask_kernel<<<(unsigned)blocks, 256, 0, st>>>(mask, T, counters);
+  } else {
+    set_count_kernel<<<1, 1, 0, st>>>((int32_t)T, counters);
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_fwd_finalize(const FwdPartial* partials, int nsplit, const int32_t* y,
+                                const float* logp_old, const uint8_t* mask, const int32_t* cu_seqlens,
+                                const float* a_norm, int64_t T, int32_t V, int32_t S,
+                                float clip_lo, float clip_hi,
+                                float* loss, float* logp, float* lse, float* coef, float* seq_sums,
+                                double* block_sums, int32_t* counters, int64_t fin_blocks,
+                                int32_t* d_status, cudaStream_t st) {
+  fwd_finalize_kernel<<<(unsigned)fin_blocks, kFinalizeThreads, 0, st>>>(
+      partials, nsplit, y, logp_old, mask, cu_seqlens, a_norm, T, V, S, clip_lo, clip_hi,
+      loss, logp, lse, coef, block_sums, counters, d_status);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  if (seq_sums && S > 0) {
+    seq_sums_kernel<<<S, 256, 0, st>>>(logp, logp_old, mask, cu_seqlens, seq_sums);
+    e = cudaGetLastError();
+  }
+  return e;
+}
+
+cudaError_t launch_fwd_f32(const float* H, const float* W, const int32_t* y, int64_t T, int32_t d, int32_t V,
+                           FwdPartial* partials, cudaStream_t st) {
+  if (T == 0) return cudaSuccess;
+  fwd_f32_kernel<<<(unsigned)T, 128, sizeof(float) * d, st>>>(H, W, y, d, V, partials);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_bwd_f32(const float* H, const float* W, const int32_t* y, const float* lse,
+                           const float* coef, float grad_loss, int64_t T, int32_t d, int32_t V,
+                           void* dH, int32_t dH_dtype, float* dW, int accumulate, cudaStream_t st) {
+  const size_t smem = sizeof(float) * (d + kBwdChunk);
+  if (T > 0) {
+    bwd_f32_kernel<false><<<(unsigned)T, 128, smem, st>>>(H, W, y, lse, coef, grad_loss, T, d, V, dH,
+                                                          dH_dtype == SPO_DTYPE_BF16, 0);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+  }
+  bwd_f32_kernel<true><<<(unsigned)V, 128, smem, st>>>(H, W, y, lse, coef, grad_loss, T, d, V, dW, 0, accumulate);
+  return cudaGetLastError();
+}
+
+}  // namespace spo

@@ -1,0 +1,78 @@
+"""Shared helpers for the GPU parity tests: upload inputs, call the C-ABI binding, fetch results."""
+
+import numpy as np
+
+
+def rel_fro(got, want):
+    got = np.asarray(got, dtype=np.float64)
+    want = np.asarray(want, dtype=np.float64)
+    den = np.linalg.norm(want)
+    return np.linalg.norm(got - want) / (den if den > 0 else 1.0)
+
+
+def dev(x, dtype=None):
+    import torch
+    t = torch.from_numpy(np.ascontiguousarray(x)).cuda()
+    return t if dtype is None else t.to(dtype)
+
+
+def status_word():
+    import torch
+    return torch.zeros(4, dtype=torch.int32, device="cuda")
+
+
+def ws_bytes(which, **kw):
+    import torch
+    from paper_2509_13232_b200 import binding as B
+    n = B.spo_workspace_bytes(which, **kw)
+    return torch.empty(max(n, 256), dtype=torch.uint8, device="cuda")
+
+
+def run_loss(lb, params=None, grad_loss=1.0, dh_bf16=None, want_seq_sums=True, dw_init=None, mask_none=False):
+    """Forward + backward through the binding for a LossBatch; returns numpy outputs."""
+    import torch
+    from paper_2509_13232_b200 import binding as B
+    params = params or B.default_params()
+    tdt = torch.bfloat16 if lb.bf16 else torch.float32
+    H, W = dev(lb.h, tdt), dev(lb.w, tdt)
+    T, d = H.shape
+    V = W.shape[0]
+    S = len(lb.cu_seqlens) - 1
+    y, lo = dev(lb.y), dev(lb.logp_old)
+    mask = None if mask_none else dev(lb.mask)
+    cu, an = dev(lb.cu_seqlens), dev(lb.a_norm)
+    f32 = dict(dtype=torch.float32, device="cuda")
+    loss = torch.zeros(4, **f32)
+    logp, lse, coef = (torch.full((max(T, 1),), float("nan"), **f32) for _ in range(3))
+    seq = torch.zeros((max(S, 1), 3), **f32) if want_seq_sums else None
+    st = status_word()
+    wsf = ws_bytes(B.WS_LOSS_FWD, T=T, d=d, V=V)
+    B.spo_loss_fwd(H, W, y, lo, mask, cu, an, loss, logp, lse, coef, seq, wsf, params, st)
+    if dh_bf16 is None:
+        dh_bf16 = lb.bf16
+    dH = torch.full((max(T, 1), d), float("nan"), dtype=torch.bfloat16 if dh_bf16 else torch.float32, device="cuda")
+    if dw_init is None:
+        dW = torch.full((V, d), float("nan"), **f32)
+        acc = 0
+    else:
+        dW = dev(dw_init).clone()
+        acc = 1
+    wsb = ws_bytes(B.WS_LOSS_BWD, T=T, d=d, V=V)
+    B.spo_loss_bwd(H, W, y, lse, coef, grad_loss, dH, dW, acc, wsb, params, st)
+    torch.cuda.synchronize()
+    return {
+        "loss": float(loss[0].item()), "logp": logp[:T].cpu().numpy(), "lse": lse[:T].cpu().numpy(),
+        "coef": coef[:T].cpu().numpy(), "seq_sums": None if seq is None else seq[:S].cpu().numpy(),
+        "dH": dH[:T].float().cpu().numpy(), "dW": dW.cpu().numpy(), "status": int(st[0].item()),
+    }
+
+
+def oracle_loss(lb, params=None, grad_loss=1.0, mask_none=False):
+    from oracle import spo_oracle as O
+    clip_lo = 0.2 if params is None else float(np.float32(params.clip_lo))
+    clip_hi = 0.28 if params is None else float(np.float32(params.clip_hi))
+    mask = None if mask_none else lb.mask
+    fwd = O.loss_forward(lb.h, lb.w, lb.y, lb.logp_old, mask, lb.cu_seqlens, lb.a_norm, clip_lo, clip_hi)
+    dh, dw = O.loss_backward(lb.h, lb.w, lb.y, fwd["lse"], fwd["coef"], grad_loss)
+    fwd["dH"], fwd["dW"] = dh, dw
+    return fwd

@@ -1,0 +1,110 @@
+"""GPU parity of the fused loss forward / backward against the CPU oracle.
+
+Tolerances (bf16 inputs, fp32 accumulation): loss and per-token log-probs within 2e-3
+absolute; gradients within 1e-2 relative Frobenius error.  The fp32 path is held to
+1e-4 absolute / 1e-4 relative Frobenius.
+"""
+
+import numpy as np
+import pytest
+
+from oracle import spo_oracle as O
+from paper_2509_13232_b200 import inputs
+from tests.helpers import oracle_loss, rel_fro, run_loss
+
+pytestmark = pytest.mark.gpu
+
+
+def check(lb, got, want, abs_tol, fro_tol):
+    assert got["status"] == 0
+    assert abs(got["loss"] - want["loss"]) <= abs_tol
+    np.testing.assert_allclose(got["logp"], want["logp"], rtol=0, atol=abs_tol)
+    np.testing.assert_allclose(got["lse"], want["lse"], rtol=0, atol=abs_tol)
+    assert rel_fro(got["coef"], want["coef"]) <= fro_tol
+    if got["seq_sums"] is not None:
+        scale = np.maximum(1.0, want["seq_sums"][:, 2:3])
+        np.testing.assert_allclose(got["seq_sums"] / scale, want["seq_sums"] / scale, rtol=0, atol=abs_tol)
+    assert rel_fro(got["dH"], want["dH"]) <= fro_tol
+    assert rel_fro(got["dW"], want["dW"]) <= fro_tol
+
+
+def test_cfg1_tiny_fp32_full_parity():
+    tb, lb = inputs.cfg1_tiny()
+    # advantages of the tiny step come from the oracle's own tracker pieces
+    a0, b0 = O.tracker_init(tb.v0, 0.875)
+    a_norm, _, _ = O.normalise_advantages(O.raw_advantage(a0, b0, tb.ids, tb.rewards))
+    lb.a_norm = a_norm.astype(np.float32)
+    got = run_loss(lb)
+    want = oracle_loss(lb)
+    check(lb, got, want, 1e-4, 1e-4)
+    assert abs(want["n_tok"] - lb.h.shape[0]) == 0
+
+
+def _clip_batch(cfg, lengths, d, v, bf16, w_std=0.05):
+    """Old log-probs far enough from the new ones that all four (sign x side) clip branches occur."""
+    rng = np.random.default_rng(cfg)
+    a = rng.standard_normal(len(lengths)).astype(np.float32)
+    a[0] = 0.0
+    return inputs.loss_batch(cfg, lengths, d, v, w_std, bf16, 0.3, target="softmax", mask_p=0.15, a_norm=a)
+
+
+def test_fp32_clip_branches_mask_and_grad_scale():
+    lb = _clip_batch(11, [5, 17, 1, 30, 9], 32, 257, False)
+    got = run_loss(lb, grad_loss=0.37, dh_bf16=False)
+    want = oracle_loss(lb, grad_loss=0.37)
+    assert 0.05 < want["unclipped"].mean() < 0.95
+    check(lb, got, want, 1e-4, 1e-4)
+    masked = lb.mask == 0
+    assert masked.any() and np.all(got["dH"][masked] == 0.0)
+
+
+def test_fp32_dw_accumulate_and_no_mask():
+    lb = inputs.loss_batch(12, [7, 8], 16, 50, 0.1, False, 0.05)
+    init = np.random.default_rng(1).standard_normal((50, 16)).astype(np.float32)
+    got = run_loss(lb, dw_init=init, mask_none=True)
+    want = oracle_loss(lb, mask_none=True)
+    assert rel_fro(got["dW"] - init, want["dW"]) <= 1e-4
+    assert abs(got["loss"] - want["loss"]) <= 1e-4
+
+
+BF16_CASES = [
+    # name, lengths, d, V
+    ("one_tile_ragged", [40, 60], 64, 200),
+    ("tails_everywhere", [100, 1, 200, 29], 128, 1000),
+    ("short_k_many_vocab_tiles", [300, 500, 240], 192, 5000),
+    ("several_token_tiles", [700, 900, 404], 256, 2304),
+]
+
+
+@pytest.mark.parametrize("name,lengths,d,v", BF16_CASES, ids=[c[0] for c in BF16_CASES])
+def test_bf16_parity_small_shapes(name, lengths, d, v):
+    lb = _clip_batch(20 + len(lengths) + d, lengths, d, v, True, w_std=0.05)
+    got = run_loss(lb, grad_loss=1.0)
+    want = oracle_loss(lb)
+    assert 0.02 < 1.0 - want["unclipped"].mean()
+    check(lb, got, want, 2e-3, 1e-2)
+
+
+def test_bf16_fp32_dh_output_and_dw_accumulate_across_chunks():
+    """More token rows than one backward chunk holds: dW is accumulated chunk by chunk."""
+    lengths = [2000, 1500, 1100, 97]
+    lb = inputs.loss_batch(31, lengths, 128, 1200, 0.05, True, 0.05, target="softmax")
+    init = np.full((1200, 128), 0.25, dtype=np.float32)
+    got = run_loss(lb, dh_bf16=False, dw_init=init)
+    want = oracle_loss(lb)
+    assert got["status"] == 0
+    np.testing.assert_allclose(got["logp"], want["logp"], rtol=0, atol=2e-3)
+    assert rel_fro(got["dH"], want["dH"]) <= 1e-2
+    assert rel_fro(got["dW"] - init, want["dW"]) <= 1e-2
+
+
+def test_bf16_uniform_logits_and_bad_target():
+    """W = 0 gives logp = -log V exactly; a target outside the vocabulary is flagged."""
+    lb = inputs.loss_batch(32, [50, 78], 64, 300, 0.05, True, 0.05, target="uniform")
+    lb.w[:] = 0.0
+    got = run_loss(lb)
+    np.testing.assert_allclose(got["logp"], -np.log(300.0), atol=1e-5)
+    lb.y[3] = 300
+    got = run_loss(lb)
+    assert got["status"] & 1
+    assert np.isneginf(got["logp"][3]) and got["coef"][3] == 0.0

@@ -1,0 +1,206 @@
+"""GPU parity of the tracker, advantage and sampling kernels against the CPU oracle.
+
+Tolerances: tracker / advantage / normalisation values 1e-5 relative in fp32 (plus an
+absolute floor of 1e-6 where values pass through zero); sampled ids bit-exact.
+"""
+
+import numpy as np
+import pytest
+
+from oracle import spo_oracle as O
+from paper_2509_13232_b200 import inputs
+from tests.helpers import dev, status_word, ws_bytes
+
+pytestmark = pytest.mark.gpu
+
+RTOL, ATOL = 1e-5, 1e-6
+
+
+def B():
+    from paper_2509_13232_b200 import binding
+    return binding
+
+
+def gpu_init(v0, params):
+    import torch
+    ab = torch.empty((len(v0), 2), dtype=torch.float32, device="cuda")
+    B().spo_tracker_init(ab, dev(v0), params)
+    return ab
+
+
+def gpu_sample(ab_t, u, batch, params, want_w=True):
+    import torch
+    n = ab_t.shape[0]
+    ids = torch.full((batch,), -7, dtype=torch.int32, device="cuda")
+    w = torch.empty(n, dtype=torch.float32, device="cuda") if want_w else None
+    st = status_word()
+    ws = ws_bytes(B().WS_SAMPLE, N=n, M=len(u))
+    B().spo_sample_prompts(ab_t, dev(u), batch, ids, w, ws, params, st)
+    torch.cuda.synchronize()
+    return ids.cpu().numpy(), (None if w is None else w.cpu().numpy()), int(st[0].item())
+
+
+def gpu_advantages(ab_t, ids, r, params, want_raw=True):
+    import torch
+    b = len(ids)
+    a_raw = torch.empty(b, dtype=torch.float32, device="cuda") if want_raw else None
+    a_norm = torch.empty(b, dtype=torch.float32, device="cuda")
+    stats = torch.zeros(4, dtype=torch.float32, device="cuda")
+    st = status_word()
+    ws = ws_bytes(B().WS_ADVANTAGES, B=b)
+    B().spo_advantages(ab_t, dev(ids), dev(r), a_raw, a_norm, stats, ws, params, st)
+    torch.cuda.synchronize()
+    return (None if a_raw is None else a_raw.cpu().numpy()), a_norm.cpu().numpy(), stats.cpu().numpy(), int(st[0].item())
+
+
+def gpu_update(ab_t, ids, r, kl, is_table, params):
+    import torch
+    st = status_word()
+    B().spo_tracker_update(ab_t, dev(ids), dev(r), dev(kl), is_table, params, st)
+    torch.cuda.synchronize()
+    return int(st[0].item())
+
+
+def test_cfg1_tracker_step_matches_oracle():
+    """Tiny step: Algorithm 2 init, sampling, advantage (pre-update), update, normalisation."""
+    tb, _ = inputs.cfg1_tiny()
+    p = B().default_params()
+    ab_t = gpu_init(tb.v0, p)
+    a0, b0 = O.tracker_init(tb.v0, 0.875)
+    ab = ab_t.cpu().numpy()
+    np.testing.assert_allclose(ab[:, 0], a0, rtol=RTOL, atol=ATOL)
+    np.testing.assert_allclose(ab[:, 1], b0, rtol=RTOL, atol=ATOL)
+    assert np.allclose(ab.sum(axis=1), 8.0)
+    # sampling: all 16 of 16 -> a permutation, bit-exact
+    ids, w, st = gpu_sample(ab_t, tb.uniforms, 16, p)
+    w_or = O.sampling_weights_f32(ab[:, 0], ab[:, 1], np.float32(p.eps_explore))
+    assert st == 0
+    np.testing.assert_array_equal(w, w_or)
+    np.testing.assert_allclose(w, O.sampling_weights(a0, b0, float(np.float32(p.eps_explore))), rtol=RTOL)
+    np.testing.assert_array_equal(ids, O.sample_prompts(w_or, tb.uniforms, 16))
+    assert sorted(ids.tolist()) == list(range(16))
+    # advantage before the update, then the update
+    a_raw, a_norm, stats, st = gpu_advantages(ab_t, tb.ids, tb.rewards, p)
+    assert st == 0
+    want_raw = O.raw_advantage(ab[:, 0].astype(np.float64), ab[:, 1].astype(np.float64), tb.ids, tb.rewards)
+    want_norm, mu, sigma = O.normalise_advantages(want_raw, 0, float(np.float32(p.norm_eps)))
+    np.testing.assert_allclose(a_raw, want_raw, rtol=RTOL, atol=ATOL)
+    np.testing.assert_allclose(a_norm, want_norm, rtol=RTOL, atol=ATOL)
+    np.testing.assert_allclose(stats[:3], [mu, sigma, 16], rtol=RTOL, atol=ATOL)
+    assert gpu_update(ab_t, tb.ids, tb.rewards, tb.kl, 0, p) == 0
+    a1, b1 = O.tracker_update(ab[:, 0].astype(np.float64), ab[:, 1].astype(np.float64), tb.ids, tb.rewards,
+                              tb.kl.astype(np.float64), float(np.float32(p.d_half)))
+    ab1 = ab_t.cpu().numpy()
+    np.testing.assert_allclose(ab1[:, 0], a1, rtol=RTOL, atol=ATOL)
+    np.testing.assert_allclose(ab1[:, 1], b1, rtol=RTOL, atol=ATOL)
+
+
+@pytest.fixture(scope="module")
+def cfg2():
+    return inputs.tracker_batch(2, 1_000_000, 4096, 8192)
+
+
+def test_cfg2_advantages_and_update_at_scale(cfg2):
+    tb = cfg2
+    p = B().default_params()
+    ab_t = dev(tb.ab)
+    a64, b64 = tb.ab[:, 0].astype(np.float64), tb.ab[:, 1].astype(np.float64)
+    a_raw, a_norm, stats, st = gpu_advantages(ab_t, tb.ids, tb.rewards, p)
+    assert st == 0
+    want_raw = O.raw_advantage(a64, b64, tb.ids, tb.rewards)
+    want_norm, mu, sigma = O.normalise_advantages(want_raw, 0, float(np.float32(p.norm_eps)))
+    np.testing.assert_allclose(a_raw, want_raw, rtol=RTOL, atol=ATOL)
+    np.testing.assert_allclose(a_norm, want_norm, rtol=RTOL, atol=2e-6)
+    np.testing.assert_allclose(stats[:2], [mu, sigma], rtol=RTOL, atol=ATOL)
+    # per-prompt divergence table gathered by id
+    assert gpu_update(ab_t, tb.ids, tb.rewards, tb.kl_table, 1, p) == 0
+    a1, b1 = O.tracker_update(a64, b64, tb.ids, tb.rewards, tb.kl.astype(np.float64), float(np.float32(p.d_half)))
+    ab1 = ab_t.cpu().numpy()
+    np.testing.assert_allclose(ab1[:, 0], a1, rtol=RTOL, atol=ATOL)
+    np.testing.assert_allclose(ab1[:, 1], b1, rtol=RTOL, atol=ATOL)
+    # all three branches of the clamp occur in this workload
+    rho = O.forgetting_factor(tb.kl.astype(np.float64), float(np.float32(p.d_half)))
+    assert (rho == 0.875).any() and (rho == 0.96).any() and ((rho > 0.875) & (rho < 0.96)).any()
+
+
+def test_cfg2_sampling_bit_exact(cfg2):
+    tb = cfg2
+    p = B().default_params()
+    ids, w, st = gpu_sample(dev(tb.ab), tb.uniforms, 4096, p)
+    assert st == 0
+    w_or = O.sampling_weights_f32(tb.ab[:, 0], tb.ab[:, 1], np.float32(p.eps_explore))
+    np.testing.assert_array_equal(w, w_or)
+    np.testing.assert_array_equal(ids, O.sample_prompts(w_or, tb.uniforms, 4096))
+    assert len(set(ids.tolist())) == 4096
+
+
+@pytest.mark.parametrize("n,m,b", [(1, 4, 1), (5, 64, 5), (2047, 300, 100), (2049, 128, 64), (70001, 4096, 2048)])
+def test_sampling_ragged_sizes_and_repeats(n, m, b):
+    """Odd table sizes (tile tails), heavy repetition (small N), no weight output."""
+    rng = np.random.default_rng(100 + n)
+    ab = rng.uniform(0.0, 12.0, (n, 2)).astype(np.float32)
+    if n > 4:
+        ab[1] = 0.0            # empty entry -> v = 0.5
+        ab[2, 0] = 0.0         # v = 0 -> weight eps
+    u = inputs.uniforms_f32(rng, m)
+    p = B().default_params()
+    ids, _, st = gpu_sample(dev(ab), u, b, p, want_w=False)
+    w_or = O.sampling_weights_f32(ab[:, 0], ab[:, 1], np.float32(p.eps_explore))
+    assert st == 0
+    np.testing.assert_array_equal(ids, O.sample_prompts(w_or, u, b))
+
+
+def test_sampling_reports_exhausted_uniforms():
+    ab = np.ones((4, 2), dtype=np.float32)
+    u = np.array([0.1, 0.1, 0.1, 0.1], dtype=np.float32)       # always the same prompt
+    ids, _, st = gpu_sample(dev(ab), u, 3, B().default_params())
+    assert st & B().DEV_UNIFORMS_EXHAUSTED
+    assert ids[0] == 0 and (ids[1:] == -1).all()
+
+
+def test_advantages_large_batch_two_pass_path():
+    rng = np.random.default_rng(7)
+    n, b = 300_000, 200_000
+    ab = rng.uniform(0.1, 12.0, (n, 2)).astype(np.float32)
+    ids = rng.permutation(n)[:b].astype(np.int32)
+    r = (rng.random(b) < 0.4).astype(np.float32)
+    for ddof, want_raw in ((0, True), (1, False)):
+        p = B().default_params(norm_ddof=ddof)
+        a_raw, a_norm, stats, st = gpu_advantages(dev(ab), ids, r, p, want_raw=want_raw)
+        want = O.raw_advantage(ab[:, 0].astype(np.float64), ab[:, 1].astype(np.float64), ids, r)
+        want_norm, mu, sigma = O.normalise_advantages(want, ddof, float(np.float32(p.norm_eps)))
+        assert st == 0
+        if want_raw:
+            np.testing.assert_allclose(a_raw, want, rtol=RTOL, atol=ATOL)
+        np.testing.assert_allclose(a_norm, want_norm, rtol=RTOL, atol=2e-6)
+        np.testing.assert_allclose(stats[:2], [mu, sigma], rtol=RTOL, atol=ATOL)
+
+
+def test_advantages_degenerate_batches():
+    p = B().default_params()
+    ab = np.array([[2.0, 2.0], [0.0, 0.0], [0.0, 4.0]], dtype=np.float32)
+    # one entry: normalised advantage is zero
+    _, a_norm, _, _ = gpu_advantages(dev(ab), np.array([0], np.int32), np.array([1.0], np.float32), p)
+    assert a_norm[0] == 0.0
+    # all-equal advantages -> zeros; empty entry estimates 0.5; zero table -> A = r
+    a_raw, a_norm, stats, _ = gpu_advantages(dev(ab), np.array([0, 1], np.int32), np.array([1.0, 1.0], np.float32), p)
+    np.testing.assert_array_equal(a_raw, [0.5, 0.5])
+    np.testing.assert_array_equal(a_norm, [0.0, 0.0])
+    a_raw, _, _, _ = gpu_advantages(dev(ab), np.array([2], np.int32), np.array([1.0], np.float32), p)
+    assert a_raw[0] == 1.0
+    # an id outside the table is reported, not dereferenced
+    _, _, _, st = gpu_advantages(dev(ab), np.array([0, 9], np.int32), np.array([1.0, 0.0], np.float32), p)
+    assert st & B().DEV_ID_OUT_OF_RANGE
+
+
+def test_update_flags_bad_entries_and_leaves_them_untouched():
+    p = B().default_params()
+    ab = np.array([[2.0, 2.0], [1.0, 3.0], [3.0, 1.0]], dtype=np.float32)
+    ab_t = dev(ab)
+    st = gpu_update(ab_t, np.array([0, 5, 2], np.int32), np.array([1.0, 1.0, 0.0], np.float32),
+                    np.array([0.01, 0.01, np.nan], np.float32), 0, p)
+    assert st & B().DEV_ID_OUT_OF_RANGE and st & B().DEV_NONFINITE
+    out = ab_t.cpu().numpy()
+    np.testing.assert_array_equal(out[1:], ab[1:])
+    a1, b1 = O.tracker_update([2.0], [2.0], [0], [1.0], [np.float64(np.float32(0.01))], float(np.float32(p.d_half)))
+    np.testing.assert_allclose(out[0], [a1[0], b1[0]], rtol=RTOL)
