@@ -1,0 +1,382 @@
+#!/usr/bin/env python
+"""Benchmark of the SPO hot path on B200.
+
+One "step" is one pass of the whole path over one synthetic mini-batch:
+prioritised sampling -> advantages (pre-update baseline) + normalisation ->
+tracker update -> fused loss forward -> fused loss backward (dH, dW).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+Prints one JSON line (rank 0).  `value` is response tokens/s with inputs resident
+in HBM; `e2e` is the same step fed from pinned host buffers with the copies inside
+the timed region.  `--impl reference` times the float64 CPU oracle on a bounded
+sample of the same workload instead.
+"""
+
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "response tokens/s, fused SPO loss fwd+bwd (d4096,V151936,bf16); % bf16 peak"
+UNIT = "tokens/s"
+TABLE_N = 1_000_000          # tracker table the step samples from and updates
+
+LOSS_SHAPES = {
+    # workload: (d, V, w_std, old-logprob noise, reward probability)
+    "cfg3_small_bf16": (1024, 151936, 0.02, 0.02, 0.4),
+    "cfg4_8b_bf16": (4096, 151936, 0.02, 0.02, 0.3),
+    "cfg5_longtail_bf16": (4096, 151936, 0.02, 0.02, 0.3),
+}
+
+
+def read_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            p = json.load(f)
+        return {"tflops": float(p["bf16_tflops_sustained"]), "tflops_burst": float(p["bf16_tflops"]),
+                "hbm_gbs": float(p["hbm_gbs"]), "source": "measured"}
+    except Exception:
+        return {"tflops": 1400.0, "tflops_burst": 1590.0, "hbm_gbs": 6650.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+
+    QUERY = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.rows = []
+        self._stop = threading.Event()
+        self._thr = threading.Thread(target=self._run, daemon=True)
+
+    def _run(self):
+        while not self._stop.is_set():
+            try:
+                out = subprocess.run(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.QUERY,
+                                      "--format=csv,noheader,nounits"], capture_output=True, text=True, timeout=5)
+                parts = [x.strip() for x in out.stdout.strip().split(",")]
+                if len(parts) == 6:
+                    self.rows.append(parts)
+            except Exception:
+                pass
+            self._stop.wait(0.2)
+
+    def __enter__(self):
+        self._thr.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        self._thr.join(timeout=6)
+
+    def summary(self):
+        if not self.rows:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unsampled"]}
+        sm = sorted(float(r[0]) for r in self.rows)
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any(r[2 + i].lower().startswith("active") for r in self.rows)]
+        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": float(self.rows[0][1]), "reasons": reasons,
+                "samples": len(self.rows)}
+
+
+class Step:
+    """Device buffers of one workload and the call sequence of one step."""
+
+    def __init__(self, workload, device, rank):
+        import torch
+        from paper_2509_13232_b200 import binding as B
+        from paper_2509_13232_b200 import inputs
+        self.B, self.torch = B, torch
+        d, V, w_std, noise, rew_p = LOSS_SHAPES[workload]
+        lengths = inputs.workload_lengths(workload)
+        cfg = int(workload[3])
+        data = inputs.loss_batch_device(cfg * 10 + rank, lengths, d, V, w_std, noise, device, adv_p=rew_p)
+        self.data = data
+        self.T, self.d, self.V, self.S = data["T"], d, V, data["S"]
+        self.n_tok = int(data["mask"].sum().item())
+        tb = inputs.tracker_batch(cfg * 10 + rank, TABLE_N, self.S, 2 * self.S)
+        f32 = dict(dtype=torch.float32, device=device)
+        self.ab0 = torch.from_numpy(tb.ab).to(device)
+        self.ab = self.ab0.clone()
+        self.kl_table = torch.from_numpy(tb.kl_table).to(device)
+        self.uniforms = torch.from_numpy(tb.uniforms).to(device)
+        self.rewards = data["rewards"]
+        self.params = B.default_params()
+        self.ids = torch.empty(self.S, dtype=torch.int32, device=device)
+        self.a_norm = torch.empty(self.S, **f32)
+        self.stats = torch.empty(4, **f32)
+        self.loss = torch.zeros(4, **f32)
+        self.logp, self.lse, self.coef = (torch.empty(self.T, **f32) for _ in range(3))
+        self.dH = torch.empty((self.T, d), dtype=torch.bfloat16, device=device)
+        self.dW = torch.empty((V, d), **f32)
+        self.status = torch.zeros(4, dtype=torch.int32, device=device)
+        u8 = dict(dtype=torch.uint8, device=device)
+        self.ws_sample = torch.empty(B.spo_workspace_bytes(B.WS_SAMPLE, N=TABLE_N, M=2 * self.S), **u8)
+        self.ws_adv = torch.empty(B.spo_workspace_bytes(B.WS_ADVANTAGES, B=self.S), **u8)
+        self.ws_fwd = torch.empty(B.spo_workspace_bytes(B.WS_LOSS_FWD, T=self.T, d=d, V=V), **u8)
+        self.ws_bwd_bytes = B.spo_workspace_bytes(B.WS_LOSS_BWD, T=self.T, d=d, V=V)
+        self.ws_bwd = torch.empty(self.ws_bwd_bytes, **u8)
+        chunk_rows = self.ws_bwd_bytes // (((V + 255) // 256) * 256 * 2)
+        self.bwd_chunks = -(-self.T // chunk_rows)
+        # kernels launched by one step: sampling 4, advantages 1, update 1,
+        # forward 3 (count, contraction, finalise), backward 3 per chunk
+        self.launches = 4 + 1 + 1 + 3 + 3 * self.bwd_chunks
+        self.flops_fwd = 2.0 * self.T * d * V
+        self.flops_bwd = 6.0 * self.T * d * V
+
+    def small(self):
+        B = self.B
+        B.spo_sample_prompts(self.ab, self.uniforms, self.S, self.ids, None, self.ws_sample, self.params, self.status)
+        B.spo_advantages(self.ab, self.ids, self.rewards, None, self.a_norm, self.stats, self.ws_adv, self.params,
+                         self.status)
+        B.spo_tracker_update(self.ab, self.ids, self.rewards, self.kl_table, 1, self.params, self.status)
+
+    def fwd(self, h=None, y=None, logp_old=None, mask=None, cu=None):
+        D = self.data
+        self.B.spo_loss_fwd(D["h"] if h is None else h, D["w"], D["y"] if y is None else y,
+                            D["logp_old"] if logp_old is None else logp_old, D["mask"] if mask is None else mask,
+                            D["cu_seqlens"] if cu is None else cu, self.a_norm, self.loss, self.logp, self.lse,
+                            self.coef, None, self.ws_fwd, self.params, self.status)
+
+    def bwd(self, h=None, y=None):
+        D = self.data
+        self.B.spo_loss_bwd(D["h"] if h is None else h, D["w"], D["y"] if y is None else y, self.lse, self.coef,
+                            1.0, self.dH, self.dW, 0, self.ws_bwd, self.params, self.status)
+
+    def run(self):
+        self.small()
+        self.fwd()
+        self.bwd()
+
+
+def run_ours(args, rank, world, local_rank):
+    import torch
+    import torch.distributed as dist
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    from paper_2509_13232_b200 import build as spo_build
+    if rank == 0:
+        spo_build.build()
+    if world > 1:
+        dist.barrier()
+    step = Step(args.workload, device, rank)
+    peaks = read_peaks()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    ev = lambda: torch.cuda.Event(enable_timing=True)  # noqa: E731  (timed on torch's current stream, which the library launches on)
+    for _ in range(args.warmup):
+        step.run()
+    barrier()
+    t_small = t_fwd = t_bwd = 0.0
+    with ClockSampler(local_rank) as clocks:
+        barrier()
+        wall0 = time.perf_counter()
+        marks = []
+        for _ in range(args.steps):
+            a, b, c, dd = ev(), ev(), ev(), ev()
+            a.record(); step.small(); b.record(); step.fwd(); c.record(); step.bwd(); dd.record()
+            marks.append((a, b, c, dd))
+        barrier()
+        wall = time.perf_counter() - wall0
+    total_ms = marks[0][0].elapsed_time(marks[-1][3])
+    for a, b, c, dd in marks:
+        t_small += a.elapsed_time(b); t_fwd += b.elapsed_time(c); t_bwd += c.elapsed_time(dd)
+    status = int(step.status[0].item())
+
+    # end to end: the step's inputs come from pinned host memory every step, the loss goes back
+    D = step.data
+    host = {k: D[k].cpu().pin_memory() for k in ("h", "y", "logp_old", "mask", "cu_seqlens")}
+    host["rewards"] = step.rewards.cpu().pin_memory()
+    host["uniforms"] = step.uniforms.cpu().pin_memory()
+    devbuf = {k: torch.empty_like(D[k]) for k in ("h", "y", "logp_old", "mask", "cu_seqlens")}
+    loss_host = torch.zeros(4, dtype=torch.float32).pin_memory()
+    ids_host = torch.zeros(step.S, dtype=torch.int32).pin_memory()
+    h2d = sum(v.numel() * v.element_size() for v in host.values())
+    d2h = loss_host.numel() * 4 + ids_host.numel() * 4
+
+    def e2e_step():
+        for k in devbuf:
+            devbuf[k].copy_(host[k], non_blocking=True)
+        step.rewards.copy_(host["rewards"], non_blocking=True)
+        step.uniforms.copy_(host["uniforms"], non_blocking=True)
+        step.small()
+        step.fwd(devbuf["h"], devbuf["y"], devbuf["logp_old"], devbuf["mask"], devbuf["cu_seqlens"])
+        step.bwd(devbuf["h"], devbuf["y"])
+        loss_host.copy_(step.loss, non_blocking=True)
+        ids_host.copy_(step.ids, non_blocking=True)
+
+    e2e_steps = max(1, min(args.steps, 3))
+    e2e_step()
+    barrier()
+    s0, s1 = ev(), ev()
+    s0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    s1.record()
+    barrier()
+    e2e_ms = s0.elapsed_time(s1)
+
+    # max over ranks, sum of tokens
+    vals = torch.tensor([total_ms, e2e_ms, t_fwd, t_bwd, t_small], dtype=torch.float64, device=device)
+    toks = torch.tensor([float(step.n_tok)], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(vals, op=dist.ReduceOp.MAX)
+        dist.all_reduce(toks, op=dist.ReduceOp.SUM)
+    total_ms, e2e_ms, t_fwd, t_bwd, t_small = [float(x) for x in vals.tolist()]
+    tokens_all = float(toks.item())
+    if rank != 0:
+        return
+    ms_per_step = total_ms / args.steps
+    value = tokens_all / (ms_per_step / 1e3)
+    gemm_ms = (t_fwd + t_bwd) / args.steps
+    achieved = (step.flops_fwd + step.flops_bwd) / (gemm_ms / 1e3) / 1e12
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": args.workload, "responses": step.S, "tokens": step.T, "d": step.d, "V": step.V,
+                   "tracker_prompts": TABLE_N, "l2": "inputs_exceed_l2", "bwd_chunks": step.bwd_chunks,
+                   "parallelism": "replicas" if world > 1 else "single"},
+        "gpu_launches": step.launches * args.steps,
+        "device_status": status,
+        "wall_s": wall,
+        "breakdown_ms": {"small": t_small / args.steps, "loss_fwd": t_fwd / args.steps, "loss_bwd": t_bwd / args.steps},
+        "roofline": {
+            "bound": "tensor", "kernel": "spo_gemm_kernel (FWD, G, DH, DW instantiations; all launches of a step)",
+            "achieved": achieved, "peak": peaks["tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["tflops"],
+            "peak_source": peaks["source"] + " sustained cuBLAS bf16",
+            "frac_of_nominal_2250": achieved / 2250.0, "frac_of_burst": achieved / peaks["tflops_burst"],
+            "flops_per_step": step.flops_fwd + step.flops_bwd,
+            "fwd_tflops": step.flops_fwd / (t_fwd / args.steps / 1e3) / 1e12,
+            "bwd_tflops": step.flops_bwd / (t_bwd / args.steps / 1e3) / 1e12,
+            "traffic": None,
+        },
+        "e2e": {"value": tokens_all / (e2e_ms / e2e_steps / 1e3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+        "clocks": clocks.summary(),
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        out["cpu_baseline"] = cpu_baseline_sample(step, args.cpu_tokens)
+    print(json.dumps(out), flush=True)
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        return max(n) if n else (os.cpu_count() or 1)
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def oracle_slice_seconds(h, w, y, logp_old, a_tok, n_rows):
+    """Time the oracle, as it stands, on the first n_rows token rows (forward + backward)."""
+    from oracle import spo_oracle as O
+    cu = np.arange(n_rows + 1)
+    t0 = time.perf_counter()
+    fwd = O.loss_forward(h, w, y, logp_old, None, cu, a_tok)
+    O.loss_backward(h, w, y, fwd["lse"], fwd["coef"], 1.0)
+    return time.perf_counter() - t0
+
+
+def cpu_baseline_sample(step, n_rows):
+    D = step.data
+    h = D["h"][:n_rows].float().cpu().numpy()
+    w = D["w"].float().cpu().numpy()
+    y = D["y"][:n_rows].cpu().numpy()
+    lo = D["logp_old"][:n_rows].cpu().numpy()
+    a_tok = np.full(n_rows, 0.5, dtype=np.float32)
+    sec = oracle_slice_seconds(h, w, y, lo, a_tok, n_rows)
+    return {"value": n_rows / sec, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+            "sample": "loss forward+backward of the first %d token rows at full d=%d, V=%d (numpy float64); "
+                      "the tracker/sampling steps are negligible beside it" % (n_rows, step.d, step.V),
+            "seconds": sec}
+
+
+def run_reference(args, rank, world):
+    """The reference arm: the float64 CPU oracle on a bounded sample per step (rank 0 only)."""
+    if rank != 0:
+        return
+    from paper_2509_13232_b200 import inputs
+    d, V, w_std, noise, _ = LOSS_SHAPES[args.workload]
+    n_rows = args.cpu_tokens
+    rng = inputs.rng_for(int(args.workload[3]), 9)
+    h = inputs.round_to_bf16(rng.standard_normal((n_rows, d)).astype(np.float32))
+    w = inputs.round_to_bf16((rng.standard_normal((V, d)) * w_std).astype(np.float32))
+    y = rng.integers(0, V, n_rows).astype(np.int32)
+    lo = np.full(n_rows, -np.log(V), dtype=np.float32)
+    a_tok = np.full(n_rows, 0.5, dtype=np.float32)
+    for _ in range(args.warmup):
+        oracle_slice_seconds(h, w, y, lo, a_tok, n_rows)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_slice_seconds(h, w, y, lo, a_tok, n_rows)
+    sec = (time.perf_counter() - t0) / args.steps
+    value = n_rows / sec
+    sample = ("each step = oracle loss forward+backward on %d synthetic token rows at full d=%d, V=%d "
+              "(numpy float64)" % (n_rows, d, V))
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.workload, "tokens": n_rows, "d": d, "V": V},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=4)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg4_8b_bf16", choices=sorted(LOSS_SHAPES))
+    ap.add_argument("--cpu-tokens", type=int, default=None, help="token rows of the CPU-oracle sample")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        if args.cpu_tokens is None:
+            args.cpu_tokens = 16
+        run_reference(args, rank, world)
+        return
+    if args.cpu_tokens is None:
+        args.cpu_tokens = 256
+    if world > 1:
+        import torch
+        import torch.distributed as dist
+        torch.cuda.set_device(local_rank)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    try:
+        run_ours(args, rank, world, local_rank)
+    finally:
+        if world > 1:
+            import torch.distributed as dist
+            dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
