@@ -97,13 +97,15 @@ class ClockSampler:
 class Step:
     """Device buffers of one workload and the call sequence of one step."""
 
-    def __init__(self, workload, device, rank):
+    def __init__(self, workload, device, rank, responses=None):
         import torch
         from paper_2509_13232_b200 import binding as B
         from paper_2509_13232_b200 import inputs
         self.B, self.torch = B, torch
         d, V, w_std, noise, rew_p = LOSS_SHAPES[workload]
         lengths = inputs.workload_lengths(workload)
+        if responses:
+            lengths = lengths[:responses]
         cfg = int(workload[3])
         data = inputs.loss_batch_device(cfg * 10 + rank, lengths, d, V, w_std, noise, device, adv_p=rew_p)
         self.data = data
@@ -174,7 +176,7 @@ def run_ours(args, rank, world, local_rank):
         spo_build.build()
     if world > 1:
         dist.barrier()
-    step = Step(args.workload, device, rank)
+    step = Step(args.workload, device, rank, args.responses)
     peaks = read_peaks()
 
     def barrier():
@@ -354,6 +356,8 @@ def main():
     ap.add_argument("--workload", default="cfg4_8b_bf16", choices=sorted(LOSS_SHAPES))
     ap.add_argument("--cpu-tokens", type=int, default=None, help="token rows of the CPU-oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--responses", type=int, default=None,
+                    help="use only the first S responses of the workload (small cases for profiling)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
