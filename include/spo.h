@@ -130,6 +130,37 @@ int32_t spo_advantages(const float* ab, int64_t N, const int32_t* ids, const flo
                        const spo_params* params, int32_t* d_status, void* stream);
 
 /*
+ * spo_advantages with no scratch argument and no allocation anywhere.  (The paper has no
+ * counterpart to this call: it computes exactly what spo_advantages computes and exists
+ * only for the memory situation described here.)
+ *
+ * Who needs it: code that runs where device memory can no longer be obtained -- a
+ * trainer whose framework has already handed every free byte of HBM to its own caching
+ * allocator, a plug-in that is given input and output buffers but no allocator handle,
+ * a step function that must never touch cudaMalloc because an allocation there would
+ * synchronise the device or fail outright.  Such a caller cannot produce the `ws`
+ * buffer that spo_advantages asks for large batches.
+ *
+ * Here the block partials of the two-pass path live in a fixed 16 KB array inside the
+ * library's device image (each GPU that loads the library holds it until the process
+ * exits).  Consequences the caller must know:
+ *   - B may not exceed SPO_ADVANTAGES_STATIC_MAX_B; a larger B returns SPO_ERR_BAD_SHAPE
+ *     and launches nothing.
+ *   - The first call on a device looks up the array's device address (once per device,
+ *     with that device current).  Make that first call outside any stream capture.
+ *   - All calls share the one array.  Each call overwrites the part it later reads, so
+ *     stale contents are harmless, but two calls whose kernels overlap on the GPU (two
+ *     streams, two host threads) race on it: serialise them.
+ *   - It calls no cudaMalloc/cudaFree or any allocating routine; inputs and outputs are
+ *     still the caller's, with the same meaning, alignment and status bits as
+ *     spo_advantages.  Always takes the two-kernel path, whatever B is.
+ */
+#define SPO_ADVANTAGES_STATIC_MAX_B  4194304
+int32_t spo_advantages_static(const float* ab, int64_t N, const int32_t* ids, const float* r, int32_t B,
+                              float* a_raw, float* a_norm, float* stats,
+                              const spo_params* params, int32_t* d_status, void* stream);
+
+/*
  * KL-adaptive tracker update (Sec. 3.1, the update equation; Algorithm 1, "Update tracker"):
  *   rho = clamp(2^(-D/D_half), rho_min, rho_max); alpha <- rho*alpha + r; beta <- rho*beta + (1-r)
  * at row ids[j], in place.  ids must be distinct within a call (what sampling

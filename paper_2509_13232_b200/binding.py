@@ -23,6 +23,7 @@ WS_SAMPLE, WS_ADVANTAGES, WS_LOSS_FWD, WS_LOSS_BWD = 0, 1, 2, 3
 
 EXPORTS = [
     "spo_default_params", "spo_tracker_init", "spo_sample_prompts", "spo_advantages",
+    "spo_advantages_static",
     "spo_tracker_update", "spo_loss_fwd", "spo_loss_bwd", "spo_workspace_bytes",
     "spo_status_string", "spo_last_cuda_error", "spo_version",
 ]
@@ -63,6 +64,8 @@ def lib():
                                          c_void_p, c_size_t, P, c_void_p, c_void_p]
         L.spo_advantages.argtypes = [c_void_p, c_int64, c_void_p, c_void_p, c_int32, c_void_p, c_void_p,
                                      c_void_p, c_void_p, c_size_t, P, c_void_p, c_void_p]
+        L.spo_advantages_static.argtypes = [c_void_p, c_int64, c_void_p, c_void_p, c_int32, c_void_p, c_void_p,
+                                            c_void_p, P, c_void_p, c_void_p]
         L.spo_tracker_update.argtypes = [c_void_p, c_int64, c_void_p, c_void_p, c_void_p, c_int32, c_int32,
                                          P, c_void_p, c_void_p]
         L.spo_loss_fwd.argtypes = [c_void_p, c_void_p, c_int32, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
@@ -135,6 +138,18 @@ def spo_advantages(ab, ids, r, a_raw, a_norm, stats, ws, params, d_status):
     _check(lib().spo_advantages(_ptr(ab), ab.shape[0], _ptr(ids), _ptr(r), ids.numel(), _ptr(a_raw), _ptr(a_norm),
                                 _ptr(stats), _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size(),
                                 ctypes.byref(params), _ptr(d_status), _stream()), "spo_advantages")
+
+
+ADVANTAGES_STATIC_MAX_B = 4194304
+
+
+def spo_advantages_static(ab, ids, r, a_raw, a_norm, stats, params, d_status):
+    """spo_advantages for callers that cannot supply scratch memory: same inputs and outputs,
+    no `ws`; the library's own fixed device array holds the partial sums (B <= ADVANTAGES_STATIC_MAX_B;
+    calls must not overlap on the GPU)."""
+    _check(lib().spo_advantages_static(_ptr(ab), ab.shape[0], _ptr(ids), _ptr(r), ids.numel(), _ptr(a_raw),
+                                       _ptr(a_norm), _ptr(stats), ctypes.byref(params), _ptr(d_status),
+                                       _stream()), "spo_advantages_static")
 
 
 def spo_tracker_update(ab, ids, r, kl, kl_is_table, params, d_status):

@@ -4,6 +4,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <mutex>
+
 #include "spo_internal.h"
 
 namespace spo {
@@ -466,3 +468,71 @@ cudaError_t launch_tracker_update(float* ab, int64_t N, const int32_t* ids, cons
 }
 
 }  // namespace spo
+
+// ---------------------------------------------------------------------------
+// spo_advantages_static: the two-pass advantage kernels with their scratch in a
+// fixed device array instead of a caller buffer (see include/spo.h).
+// ---------------------------------------------------------------------------
+namespace spo {
+namespace {
+
+constexpr int kStaticAdvMaxBlocks = 1024;
+
+// Per-block (sum, sum of squares) partials of pass 1.  Lives in every GPU context that
+// loads this library, 16 KB, until the process exits.  In host code this name is only a
+// handle for cudaGetSymbolAddress, never a device address.
+static __device__ __align__(256) double2 g_adv_static_scratch[kStaticAdvMaxBlocks];
+
+std::mutex g_adv_static_mutex;
+double2* g_adv_static_ptr[64] = {};
+
+// Device address of the scratch array for the current device (looked up once per device).
+cudaError_t adv_static_scratch(double2** out) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(g_adv_static_mutex);
+  if (!g_adv_static_ptr[dev]) {
+    void* ptr = nullptr;
+    e = cudaGetSymbolAddress(&ptr, g_adv_static_scratch);
+    if (e != cudaSuccess) return e;
+    g_adv_static_ptr[dev] = static_cast<double2*>(ptr);
+  }
+  *out = g_adv_static_ptr[dev];
+  return cudaSuccess;
+}
+
+}  // namespace
+}  // namespace spo
+
+extern "C" int32_t spo_advantages_static(const float* ab, int64_t N, const int32_t* ids, const float* r, int32_t B,
+                                         float* a_raw, float* a_norm, float* stats, const spo_params* params,
+                                         int32_t* d_status, void* stream) {
+  using namespace spo;
+  if (!params || !ab || !ids || !r || !a_norm) return SPO_ERR_INVALID_ARG;
+  if (!(params->norm_eps >= 0.0f) || (params->norm_ddof != 0 && params->norm_ddof != 1)) return SPO_ERR_INVALID_ARG;
+  if (N < 1 || N >= ((int64_t)1 << 31) || B < 1) return SPO_ERR_BAD_SHAPE;
+  if (B > SPO_ADVANTAGES_STATIC_MAX_B) return SPO_ERR_BAD_SHAPE;   // beyond what the fixed scratch is sized for
+  const uintptr_t all = reinterpret_cast<uintptr_t>(ab) | reinterpret_cast<uintptr_t>(ids) |
+                        reinterpret_cast<uintptr_t>(r) | reinterpret_cast<uintptr_t>(a_raw) |
+                        reinterpret_cast<uintptr_t>(a_norm) | reinterpret_cast<uintptr_t>(stats);
+  if (all & 15u) return SPO_ERR_BAD_ALIGNMENT;
+  if (!device_is_sm100()) return SPO_ERR_UNSUPPORTED_ARCH;
+  double2* partials = nullptr;
+  cudaError_t e = adv_static_scratch(&partials);
+  if (e != cudaSuccess) return SPO_ERR_CUDA;
+  int blocks = adv_blocks(B);
+  if (blocks > kStaticAdvMaxBlocks) blocks = kStaticAdvMaxBlocks;
+  cudaStream_t st = (cudaStream_t)stream;
+  const float2* ab2 = reinterpret_cast<const float2*>(ab);
+  float* tmp = a_raw ? a_raw : a_norm;
+  // Pass 1 overwrites partials[0..blocks) and pass 2 reads exactly those, so nothing left
+  // over from an earlier call is ever read and nothing needs clearing.
+  advantages_partial_kernel<<<blocks, 256, 0, st>>>(ab2, N, ids, r, B, tmp, partials, d_status);
+  if ((e = cudaGetLastError()) != cudaSuccess) return SPO_ERR_CUDA;
+  advantages_normalise_kernel<<<blocks, 256, 0, st>>>(partials, blocks, tmp, B, a_norm, stats, params->norm_eps,
+                                                      params->norm_ddof);
+  if ((e = cudaGetLastError()) != cudaSuccess) return SPO_ERR_CUDA;
+  return SPO_OK;
+}
