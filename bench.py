@@ -166,6 +166,19 @@ class Step:
         self.bwd()
 
 
+def reduce_over_ranks(times_ms, tokens, world, device):
+    """Replicas run independent mini-batches: the job's time is the slowest rank's (MAX of every
+    timing), its work is the sum of the ranks' tokens (SUM).  Returns (times, tokens) on every rank."""
+    import torch
+    import torch.distributed as dist
+    vals = torch.tensor(list(times_ms), dtype=torch.float64, device=device)
+    toks = torch.tensor([float(tokens)], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(vals, op=dist.ReduceOp.MAX)
+        dist.all_reduce(toks, op=dist.ReduceOp.SUM)
+    return [float(x) for x in vals.tolist()], float(toks.item())
+
+
 def run_ours(args, rank, world, local_rank):
     import torch
     import torch.distributed as dist
@@ -237,14 +250,8 @@ def run_ours(args, rank, world, local_rank):
     barrier()
     e2e_ms = s0.elapsed_time(s1)
 
-    # max over ranks, sum of tokens
-    vals = torch.tensor([total_ms, e2e_ms, t_fwd, t_bwd, t_small], dtype=torch.float64, device=device)
-    toks = torch.tensor([float(step.n_tok)], dtype=torch.float64, device=device)
-    if world > 1:
-        dist.all_reduce(vals, op=dist.ReduceOp.MAX)
-        dist.all_reduce(toks, op=dist.ReduceOp.SUM)
-    total_ms, e2e_ms, t_fwd, t_bwd, t_small = [float(x) for x in vals.tolist()]
-    tokens_all = float(toks.item())
+    (total_ms, e2e_ms, t_fwd, t_bwd, t_small), tokens_all = reduce_over_ranks(
+        [total_ms, e2e_ms, t_fwd, t_bwd, t_small], step.n_tok, world, device)
     if rank != 0:
         return
     ms_per_step = total_ms / args.steps

@@ -12,7 +12,8 @@ import ctypes
 import os
 from ctypes import POINTER, Structure, c_char_p, c_float, c_int32, c_int64, c_size_t, c_void_p
 
-_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libspo.so")
+# SPO_LIBRARY_PATH points at another build of the same library (e.g. one compiled with different tile options).
+_LIB_PATH = os.environ.get("SPO_LIBRARY_PATH") or os.path.join(os.path.dirname(os.path.abspath(__file__)), "libspo.so")
 
 SPO_OK = 0
 ERR_INVALID_ARG, ERR_BAD_SHAPE, ERR_BAD_ALIGNMENT = -1, -2, -3

@@ -8,12 +8,19 @@
 //   DH  : dH_chunk = G W        (A = G, K-major;  B = W read as an N-major operand)
 //   DW  : dW (+)= G^T H_chunk   (A = G read as an M-major operand; B = H, N-major)
 //
+// CTAs run as pairs (a cluster of two SMs, tcgen05 cta_group::2): one MMA covers a
+// 256 x 256 output tile, each CTA holding 128 rows of A, half of B's 256 columns and
+// the 128 accumulator rows of its own tensor memory.  Pairing halves the shared-memory
+// fill per FLOP and leaves room for a 6-stage ring.  (CG = 1 is the unpaired form.)
+//
 // Pipeline per CTA (one CTA per SM, 192 threads):
 //   warp 0 : allocates tensor memory; lane 0 issues the TMA loads (128-byte swizzle)
-//            into a 4-stage shared-memory ring, signalling "full" mbarriers.
-//   warp 1 : lane 0 issues tcgen05.mma (128x256x16, bf16 -> fp32) into one of two
-//            256-column accumulators in tensor memory; tcgen05.commit releases the
-//            stage ("empty") and, after the last k-block, publishes the accumulator.
+//            of this CTA's operand halves into its shared-memory ring; completion is
+//            signalled on the "full" mbarrier of the pair's leader CTA.
+//   warp 1 : (leader CTA only) lane 0 issues tcgen05.mma (bf16 -> fp32) into one of two
+//            256-column accumulators in tensor memory; tcgen05.commit, multicast to both
+//            CTAs, releases the stage ("empty") and, after the last k-block, publishes
+//            the accumulator.
 //   warps 2-5 : epilogue; each owns the 32 accumulator lanes its warp id selects,
 //            reads them with tcgen05.ld and applies the mode's fused epilogue while
 //            the next tile accumulates in the other buffer.
@@ -31,24 +38,38 @@ namespace spo {
 
 namespace {
 
-constexpr int BM = 128;
-constexpr int BN = 256;
+constexpr int BM = 128;                 // rows of A (and of the accumulator) per CTA
+constexpr int BN = 256;                 // columns of one output tile
 constexpr int BK = 64;
-constexpr int STAGES = 4;
 constexpr int A_BYTES = BM * BK * 2;
-constexpr int B_BYTES = BN * BK * 2;
-constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int NUM_THREADS = 192;
 constexpr int TMEM_COLS = 512;
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256;
+
+// Per-CTA shared-memory plan for a CTA group of CG CTAs.
+template <int CG>
+struct Plan {
+  static constexpr int kStages = CG == 2 ? 6 : 4;
+  static constexpr int kBRows = BN / CG;                  // columns of B held by this CTA
+  static constexpr int kBBytes = kBRows * BK * 2;
+  static constexpr int kStageBytes = A_BYTES + kBBytes;
+  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 + 256;
+};
 constexpr unsigned long long kWaitLimitNs = 4000000000ull;
+#ifndef SPO_EPI_SLEEP
+#define SPO_EPI_SLEEP 128
+#endif
+#ifndef SPO_PROD_SLEEP
+#define SPO_PROD_SLEEP 32
+#endif
+constexpr int kEpilogueSleepNs = SPO_EPI_SLEEP;
+constexpr int kProducerSleepNs = SPO_PROD_SLEEP;
 
 constexpr float kLog2e = 1.4426950408889634f;
 
 enum : int { MODE_FWD = 0, MODE_G = 1, MODE_DH = 2, MODE_DW = 3 };
 
 struct GemmParams {
-  int m_tiles, n_tiles, nsplit, per_split;   // work decomposition: unit = (m tile, split of the n tiles)
+  int m_tiles, n_tiles, nsplit, per_split;   // work decomposition: unit = (row tile of the CTA group, split of the n tiles)
   int k_blocks;                              // K / 64, rounded up
   int a_row0;                                // added to A's row coordinate (K-major A) or k coordinate (M-major A)
   int b_k0;                                  // added to B's k coordinate (N-major B)
@@ -77,6 +98,22 @@ struct GemmParams {
 // ---------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// Address of the same shared-memory offset in CTA `rank` of this cluster.
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
@@ -86,11 +123,27 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
+// Arrive on a barrier given by a shared::cluster address (possibly in the peer CTA).
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
 __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
       "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok;
+}
+// Same, with cluster-scope acquire: for barriers that the peer CTA arrives on.
+__device__ __forceinline__ uint32_t mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
       "selp.b32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
       : "r"(bar), "r"(parity)
@@ -104,10 +157,15 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
 }
 
 // Bounded wait.  Returns false when the wait ran out or another role already gave up.
+// SLEEP_NS > 0 backs off between polls (for roles that wait long and need not react within
+// nanoseconds): a spinning warp occupies an issue slot every cycle and costs power that the
+// tensor pipe could use.
+template <bool CLUSTER_SCOPE = false, int SLEEP_NS = 0>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* d_status) {
   uint32_t spins = 0;
   unsigned long long t0 = 0;
-  while (!mbar_try_wait(bar, parity)) {
+  while (!(CLUSTER_SCOPE ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity))) {
+    if (SLEEP_NS > 0) __nanosleep(SLEEP_NS);
     if ((++spins & 255u) == 0) {
       if (*abort_flag) return false;
       unsigned long long now = global_timer_ns();
@@ -123,26 +181,55 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   return true;
 }
 
+// TMA tile load into this CTA's shared memory; completion bytes are counted on `bar`, which for
+// CG == 2 is a shared::cluster address and may belong to the pair's leader CTA.
+template <int CG>
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar)
-      : "memory");
+  if (CG == 1) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar)
+        : "memory");
+  } else {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar)
+        : "memory");
+  }
 }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
+template <int CG>
 __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t acc) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(acc)
-      : "memory");
+  if (CG == 1) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(acc)
+        : "memory");
+  } else {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(acc)
+        : "memory");
+  }
 }
+// Arrive on `bar` once all MMAs issued so far have completed; for CG == 2 the arrival is
+// delivered to the barrier at the same offset in both CTAs of the pair.
+template <int CG>
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+  if (CG == 1) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+  } else {
+    const uint16_t mask = 3;
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"(mask) : "memory");
+  }
 }
 
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
@@ -159,6 +246,12 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+__device__ __forceinline__ float fast_exp2(float x) {
+  float r;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+  return r;
+}
+
 // Shared-memory matrix descriptor, 128-byte swizzle (layout type 2), descriptor version 1.
 // lbo / sbo in bytes.
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo) {
@@ -171,10 +264,10 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint3
   return d;
 }
 
-// Instruction descriptor for kind::f16: fp32 accumulate, bf16 A and B, M = 128, N = 256.
-__host__ __device__ constexpr uint32_t instr_desc(bool a_mn, bool b_mn) {
+// Instruction descriptor for kind::f16: fp32 accumulate, bf16 A and B, M = 128 per CTA of the group, N = 256.
+__host__ __device__ constexpr uint32_t instr_desc(bool a_mn, bool b_mn, int cg) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
-         ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+         ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((BM * cg) >> 4) << 24);
 }
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
@@ -195,11 +288,16 @@ __device__ __forceinline__ Unit unit_of(int u, const GemmParams& p) {
 // ---------------------------------------------------------------------------
 // the kernel
 // ---------------------------------------------------------------------------
-template <int MODE>
+template <int MODE, int CG>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmParams p) {
   constexpr bool A_MN = (MODE == MODE_DW);
   constexpr bool B_MN = (MODE == MODE_DH || MODE == MODE_DW);
+  using P = Plan<CG>;
+  constexpr int STAGES = P::kStages;
+  constexpr int STAGE_BYTES = P::kStageBytes;
+  constexpr int B_ROWS = P::kBRows;
+  constexpr int GROUP_M = BM * CG;                   // rows of one output tile of the CTA group
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
@@ -211,20 +309,28 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + STAGES * STAGE_BYTES + 16 * STAGES + 40);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = CG == 2 ? cluster_ctarank() : 0u;     // 0 = leader of the pair
+  const int group = blockIdx.x / CG, n_groups = gridDim.x / CG;
   const int total_units = p.m_tiles * p.nsplit;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(tfull0 + 8 * a, 1); mbar_init(tempty0 + 8 * a, 4); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull0 + 8 * a, 1); mbar_init(tempty0 + 8 * a, 4 * CG); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 0) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if (CG == 1) {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
   }
   tc_fence_before();
   __syncthreads();
+  if (CG == 2) cluster_sync_all();          // the peer's barriers exist before anything signals them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
@@ -233,72 +339,80 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
-      for (int u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
+      for (int u = group; u < total_units && ok; u += n_groups) {
         const Unit un = unit_of(u, p);
+        const int row_base = un.m_tile * GROUP_M + (int)rank * BM;      // this CTA's rows of the tile
         for (int n = un.n_begin; n < un.n_end && ok; ++n) {
+          const int col_base = n * BN + (int)rank * B_ROWS;             // this CTA's columns of B
           for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
             const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
-            if (!mbar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag, p.d_status)) { ok = false; break; }
-            const uint32_t fb = full0 + 8 * s;
+            if (!mbar_wait<CG == 2, kProducerSleepNs>(empty0 + 8 * s, ph ^ 1u, abort_flag, p.d_status)) { ok = false; break; }
             const uint32_t sa = base + s * STAGE_BYTES, sb = sa + A_BYTES;
-            mbar_expect_tx(fb, STAGE_BYTES);
+            uint32_t fb = full0 + 8 * s;
+            if (CG == 1) {
+              mbar_expect_tx(fb, STAGE_BYTES);
+            } else {
+              if (rank == 0) mbar_expect_tx(fb, 2 * STAGE_BYTES);        // both CTAs' bytes land on the leader's barrier
+              fb = map_to_cta(fb, 0);
+            }
             if (!A_MN) {
-              tma_load_2d(sa, &tmA, kb * BK, p.a_row0 + un.m_tile * BM, fb);
+              tma_load_2d<CG>(sa, &tmA, kb * BK, p.a_row0 + row_base, fb);
             } else {
 #pragma unroll
               for (int b = 0; b < BM / 64; ++b)
-                tma_load_2d(sa + b * 8192, &tmA, un.m_tile * BM + b * 64, p.a_row0 + kb * BK, fb);
+                tma_load_2d<CG>(sa + b * 8192, &tmA, row_base + b * 64, p.a_row0 + kb * BK, fb);
             }
             if (!B_MN) {
-              tma_load_2d(sb, &tmB, kb * BK, n * BN, fb);
+              tma_load_2d<CG>(sb, &tmB, kb * BK, col_base, fb);
             } else {
 #pragma unroll
-              for (int b = 0; b < BN / 64; ++b)
-                tma_load_2d(sb + b * 8192, &tmB, n * BN + b * 64, p.b_k0 + kb * BK, fb);
+              for (int b = 0; b < B_ROWS / 64; ++b)
+                tma_load_2d<CG>(sb + b * 8192, &tmB, col_base + b * 64, p.b_k0 + kb * BK, fb);
             }
           }
         }
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      constexpr uint32_t idesc = instr_desc(A_MN, B_MN);
+    // ------------------------------------------------------------------ MMA issuer (leader CTA)
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = instr_desc(A_MN, B_MN, CG);
       uint32_t it = 0, tile = 0;
       bool ok = true;
-      for (int u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
+      for (int u = group; u < total_units && ok; u += n_groups) {
         const Unit un = unit_of(u, p);
         for (int n = un.n_begin; n < un.n_end && ok; ++n, ++tile) {
           const uint32_t acc = tile & 1u, aph = (tile >> 1) & 1u;
-          if (!mbar_wait(tempty0 + 8 * acc, aph ^ 1u, abort_flag, p.d_status)) { ok = false; break; }
+          if (!mbar_wait<CG == 2>(tempty0 + 8 * acc, aph ^ 1u, abort_flag, p.d_status)) { ok = false; break; }
           tc_fence_after();
           const uint32_t tmem_d = tmem_base + acc * BN;
           for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
             const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
-            if (!mbar_wait(full0 + 8 * s, ph, abort_flag, p.d_status)) { ok = false; break; }
+            if (!mbar_wait<CG == 2>(full0 + 8 * s, ph, abort_flag, p.d_status)) { ok = false; break; }
             tc_fence_after();
             const uint32_t sa = base + s * STAGE_BYTES, sb = sa + A_BYTES;
 #pragma unroll
             for (int j = 0; j < BK / 16; ++j) {
               const uint64_t da = A_MN ? smem_desc(sa + j * 2048, 8192, 1024) : smem_desc(sa + j * 32, 16, 1024);
               const uint64_t db = B_MN ? smem_desc(sb + j * 2048, 8192, 1024) : smem_desc(sb + j * 32, 16, 1024);
-              umma_bf16(tmem_d, da, db, idesc, (kb | j) != 0 ? 1u : 0u);
+              umma_bf16<CG>(tmem_d, da, db, idesc, (kb | j) != 0 ? 1u : 0u);
             }
-            umma_commit(empty0 + 8 * s);
+            umma_commit<CG>(empty0 + 8 * s);
           }
-          if (ok) umma_commit(tfull0 + 8 * acc);
+          if (ok) umma_commit<CG>(tfull0 + 8 * acc);
         }
       }
     }
   } else {
     // ------------------------------------------------------------------ epilogue (warps 2..5)
     const int quarter = warp & 3;                    // tensor-memory lanes this warp may read
-    const int row = quarter * 32 + lane;             // row of the 128-row tile
+    const int row = (int)rank * BM + quarter * 32 + lane;   // row of the group's tile
+    const uint32_t tempty_leader0 = CG == 2 ? map_to_cta(tempty0, 0) : tempty0;
     uint32_t tile = 0;
     bool ok = true;
-    for (int u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
+    for (int u = group; u < total_units && ok; u += n_groups) {
       const Unit un = unit_of(u, p);
-      const int64_t grow = p.out_row0 + (int64_t)un.m_tile * BM + row;   // global output row
+      const int64_t grow = p.out_row0 + (int64_t)un.m_tile * GROUP_M + row;   // global output row
       const bool row_ok = grow < p.rows_valid;
       // per-row state
       float m2 = -CUDART_INF_F, l = 0.0f, zt = -CUDART_INF_F;             // FWD
@@ -310,7 +424,12 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       }
       for (int n = un.n_begin; n < un.n_end && ok; ++n, ++tile) {
         const uint32_t acc = tile & 1u, aph = (tile >> 1) & 1u;
-        if (!mbar_wait(tfull0 + 8 * acc, aph, abort_flag, p.d_status)) { ok = false; break; }
+        {                                   // one lane polls (with backoff); the warp reconverges on its verdict
+          int good = 1;
+          if (lane == 0) good = mbar_wait<CG == 2, kEpilogueSleepNs>(tfull0 + 8 * acc, aph, abort_flag, p.d_status) ? 1 : 0;
+          good = __shfl_sync(0xffffffffu, good, 0);
+          if (!good) { ok = false; break; }
+        }
         tc_fence_after();
         const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN;
         const int col_tile = n * BN;
@@ -332,8 +451,8 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             const float mn = fmaxf(m2, cmax * kLog2e);
             float sum = 0.0f;
 #pragma unroll
-            for (int j = 0; j < 32; ++j) sum += exp2f(fmaf(__uint_as_float(v[j]), kLog2e, -mn));
-            l = l * exp2f(m2 - mn) + sum;
+            for (int j = 0; j < 32; ++j) sum += fast_exp2(fmaf(__uint_as_float(v[j]), kLog2e, -mn));
+            l = l * fast_exp2(m2 - mn) + sum;
             m2 = mn;
             if (yt >= col0 && yt < col0 + 32) {
               const int jj = yt - col0;
@@ -347,8 +466,8 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
               for (int j = 0; j < 32; j += 2) {
                 float g0 = 0.0f, g1 = 0.0f;
                 if (c != 0.0f) {
-                  const float p0 = exp2f(fmaf(__uint_as_float(v[j]), kLog2e, -lse2));
-                  const float p1 = exp2f(fmaf(__uint_as_float(v[j + 1]), kLog2e, -lse2));
+                  const float p0 = fast_exp2(fmaf(__uint_as_float(v[j]), kLog2e, -lse2));
+                  const float p1 = fast_exp2(fmaf(__uint_as_float(v[j + 1]), kLog2e, -lse2));
                   g0 = c * ((col0 + j == yt ? 1.0f : 0.0f) - p0);
                   g1 = c * ((col0 + j + 1 == yt ? 1.0f : 0.0f) - p1);
                 }
@@ -356,7 +475,7 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 if (col0 + j + 1 >= p.cols_valid) g1 = 0.0f;
                 o[j >> 1] = pack_bf16(g0, g1);
               }
-              uint4* dst = reinterpret_cast<uint4*>(p.G + ((int64_t)un.m_tile * BM + row) * p.ldg + col0);
+              uint4* dst = reinterpret_cast<uint4*>(p.G + ((int64_t)un.m_tile * GROUP_M + row) * p.ldg + col0);
 #pragma unroll
               for (int q = 0; q < 4; ++q) dst[q] = make_uint4(o[4 * q], o[4 * q + 1], o[4 * q + 2], o[4 * q + 3]);
             }
@@ -392,7 +511,10 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         }
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(tempty0 + 8 * acc);
+        if (lane == 0) {
+          if (CG == 1) mbar_arrive(tempty0 + 8 * acc);
+          else mbar_arrive_cluster(tempty_leader0 + 8 * acc);
+        }
       }
       if (MODE == MODE_FWD && ok && row_ok) {
         FwdPartial part;
@@ -409,14 +531,23 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   }
   tc_fence_before();
   __syncthreads();
+  if (CG == 2) cluster_sync_all();          // the peer may still be reading this CTA's shared / tensor memory
   if (warp == 0) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    if (CG == 1)
+      asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    else
+      asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
   }
 }
 
 // ---------------------------------------------------------------------------
 // host side: tensor maps and launches
 // ---------------------------------------------------------------------------
+#ifndef SPO_CTA_GROUP
+#define SPO_CTA_GROUP 2
+#endif
+constexpr int kCG = SPO_CTA_GROUP;         // CTAs per MMA group used by the launches below
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -447,29 +578,49 @@ bool make_map(CUtensorMap* m, const void* ptr, uint64_t inner, uint64_t outer, u
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// CTA groups that can be resident at once (one CTA per SM).
+int group_count() { return sm_count() / kCG; }
+
 template <int MODE>
 cudaError_t launch_gemm(const CUtensorMap& a, const CUtensorMap& b, const GemmParams& p, cudaStream_t st) {
   static bool configured[64] = {};
   int dev = 0;
   cudaGetDevice(&dev);
+  constexpr int smem = Plan<kCG>::kSmemBytes;
   if (dev >= 0 && dev < 64 && !configured[dev]) {
-    cudaError_t e = cudaFuncSetAttribute(spo_gemm_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    cudaError_t e = cudaFuncSetAttribute(spo_gemm_kernel<MODE, kCG>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     configured[dev] = true;
   }
   const int units = p.m_tiles * p.nsplit;
   if (units <= 0) return cudaSuccess;
-  const int grid = units < sm_count() ? units : sm_count();
-  spo_gemm_kernel<MODE><<<grid, NUM_THREADS, SMEM_BYTES, st>>>(a, b, p);
-  return cudaGetLastError();
+  const int groups = units < group_count() ? units : group_count();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(groups * kCG, 1, 1);
+  cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = kCG;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, spo_gemm_kernel<MODE, kCG>, a, b, p);
 }
 
+// Operand box heights: A rows per CTA, B rows (columns of the output) per CTA.
+constexpr uint32_t kBoxA = BM;
+constexpr uint32_t kBoxB = BN / kCG;
+constexpr int kGroupM = BM * kCG;
+
 int pick_fwd_split(int64_t m_tiles, int n_tiles) {
-  // Enough units to fill the machine, and several splits so that CTAs running together
+  // Enough units to fill the machine, and several splits so that CTA groups running together
   // share token tiles (which then stay in L2) while sweeping different parts of W.
-  int sms = sm_count();
+  int groups = group_count();
   int nsplit = 4;
-  while (m_tiles * nsplit < 2 * (int64_t)sms && nsplit < n_tiles) nsplit *= 2;
+  while (m_tiles * nsplit < 2 * (int64_t)groups && nsplit < n_tiles) nsplit *= 2;
   if (nsplit > n_tiles) nsplit = n_tiles;
   if (nsplit < 1) nsplit = 1;
   return nsplit;
@@ -479,7 +630,7 @@ int pick_fwd_split(int64_t m_tiles, int n_tiles) {
 
 // nsplit used by the forward for a given shape (the workspace layout depends on it).
 int fwd_bf16_nsplit(int64_t T, int32_t V) {
-  const int64_t m_tiles = ceil_div(T, BM);
+  const int64_t m_tiles = ceil_div(T, kGroupM);
   const int n_tiles = (int)ceil_div(V, BN);
   int nsplit = pick_fwd_split(m_tiles, n_tiles);
   const int per = (int)ceil_div(n_tiles, nsplit);
@@ -490,9 +641,9 @@ cudaError_t launch_fwd_bf16(const void* H, const void* W, const int32_t* y, int6
                             FwdPartial* partials, int nsplit, int32_t* d_status, cudaStream_t st) {
   if (T == 0) return cudaSuccess;
   CUtensorMap ma, mb;
-  if (!make_map(&ma, H, d, T, d, BM) || !make_map(&mb, W, d, V, d, BN)) return cudaErrorInvalidValue;
+  if (!make_map(&ma, H, d, T, d, kBoxA) || !make_map(&mb, W, d, V, d, kBoxB)) return cudaErrorInvalidValue;
   GemmParams p{};
-  p.m_tiles = (int)ceil_div(T, BM);
+  p.m_tiles = (int)ceil_div(T, kGroupM);
   p.n_tiles = (int)ceil_div(V, BN);
   p.per_split = (int)ceil_div(p.n_tiles, nsplit);
   p.nsplit = nsplit;
@@ -509,15 +660,15 @@ cudaError_t launch_fwd_bf16(const void* H, const void* W, const int32_t* y, int6
 
 BwdWs bwd_ws_layout(int64_t T, int32_t d, int32_t V) {
   BwdWs L{};
-  // Token rows per chunk: a multiple of 128 chosen so that the dH tiles of a full chunk
-  // (row tiles x d/256 column tiles) fill the SMs a whole number of times.
-  const int sms = sm_count();
+  // Token rows per chunk: a multiple of the group tile height chosen so that the dH tiles of a
+  // full chunk (row tiles x d/256 column tiles) fill the CTA groups a whole number of times.
+  const int groups = group_count();
   const int n_tiles_d = (int)ceil_div(d, BN);
   int64_t m_tiles = 32;
   for (int64_t cand = 24; cand <= 64; ++cand)
-    if ((cand * n_tiles_d) % sms == 0) { m_tiles = cand; break; }
-  int64_t rows = m_tiles * BM;
-  const int64_t t_pad = ceil_div(T > 0 ? T : 1, BM) * BM;
+    if ((cand * n_tiles_d) % groups == 0) { m_tiles = cand; break; }
+  int64_t rows = m_tiles * kGroupM;
+  const int64_t t_pad = ceil_div(T > 0 ? T : 1, kGroupM) * kGroupM;
   if (rows > t_pad) rows = t_pad;
   L.chunk_rows = rows;
   L.ldg = ceil_div(V, BN) * BN;
@@ -536,7 +687,7 @@ cudaError_t launch_bwd_bf16(const void* H, const void* W, const int32_t* y, cons
     return cudaSuccess;
   }
   CUtensorMap mH_k, mW_k, mW_mn, mH_mn;
-  if (!make_map(&mH_k, H, d, T, d, BM) || !make_map(&mW_k, W, d, V, d, BN) ||
+  if (!make_map(&mH_k, H, d, T, d, kBoxA) || !make_map(&mW_k, W, d, V, d, kBoxB) ||
       !make_map(&mW_mn, W, d, V, d, 64) || !make_map(&mH_mn, H, d, T, d, 64))
     return cudaErrorInvalidValue;
   const int n_tiles_v = (int)ceil_div(V, BN);
@@ -545,9 +696,9 @@ cudaError_t launch_bwd_bf16(const void* H, const void* W, const int32_t* y, cons
   int chunk = 0;
   for (int64_t t0 = 0; t0 < T; t0 += L.chunk_rows, ++chunk) {
     const int64_t rows = (T - t0) < L.chunk_rows ? (T - t0) : L.chunk_rows;
-    const int m_tiles = (int)ceil_div(rows, BM);
+    const int m_tiles = (int)ceil_div(rows, kGroupM);
     CUtensorMap mG_k, mG_mn;
-    if (!make_map(&mG_k, G, V, rows, L.ldg, BM) || !make_map(&mG_mn, G, V, rows, L.ldg, 64))
+    if (!make_map(&mG_k, G, V, rows, L.ldg, kBoxA) || !make_map(&mG_mn, G, V, rows, L.ldg, 64))
       return cudaErrorInvalidValue;
     // 1) logits of the chunk, rewritten in place as g (bf16)
     {
@@ -588,7 +739,7 @@ cudaError_t launch_bwd_bf16(const void* H, const void* W, const int32_t* y, cons
     // 3) dW (+)= G^T H_chunk
     {
       GemmParams p{};
-      p.m_tiles = (int)ceil_div(V, BM);
+      p.m_tiles = (int)ceil_div(V, kGroupM);
       p.n_tiles = n_tiles_d;
       p.nsplit = n_tiles_d;
       p.per_split = 1;
