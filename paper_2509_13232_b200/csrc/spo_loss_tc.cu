@@ -8,22 +8,24 @@
 //   DH  : dH_chunk = G W        (A = G, K-major;  B = W read as an N-major operand)
 //   DW  : dW (+)= G^T H_chunk   (A = G read as an M-major operand; B = H, N-major)
 //
-// CTAs run as pairs (a cluster of two SMs, tcgen05 cta_group::2): one MMA covers a
-// 256 x 256 output tile, each CTA holding 128 rows of A, half of B's 256 columns and
-// the 128 accumulator rows of its own tensor memory.  Pairing halves the shared-memory
-// fill per FLOP and leaves room for a 6-stage ring.  (CG = 1 is the unpaired form.)
+// CTAs run as pairs (a cluster of two SMs, tcgen05 cta_group::2).  A pair owns a
+// 256 x 512 output tile: per 64-deep k-block each CTA stages 128 rows of A and its
+// half (2 x 128 columns) of B, and the leader issues two 256x256x16 MMAs per k-step
+// that share the A operand and fill the two 256-column halves of tensor memory.
+// The wide tile is what keeps the L2 -> shared-memory traffic (48 KB per 256x256x64
+// block of MACs) under the L2 bandwidth; the price is that the accumulator is not
+// double-buffered, so the epilogue is kept short: eight warps drain it in parallel.
 //
-// Pipeline per CTA (one CTA per SM, 192 threads):
+// Pipeline per CTA (one CTA per SM, 320 threads):
 //   warp 0 : allocates tensor memory; lane 0 issues the TMA loads (128-byte swizzle)
-//            of this CTA's operand halves into its shared-memory ring; completion is
-//            signalled on the "full" mbarrier of the pair's leader CTA.
-//   warp 1 : (leader CTA only) lane 0 issues tcgen05.mma (bf16 -> fp32) into one of two
-//            256-column accumulators in tensor memory; tcgen05.commit, multicast to both
-//            CTAs, releases the stage ("empty") and, after the last k-block, publishes
-//            the accumulator.
-//   warps 2-5 : epilogue; each owns the 32 accumulator lanes its warp id selects,
-//            reads them with tcgen05.ld and applies the mode's fused epilogue while
-//            the next tile accumulates in the other buffer.
+//            of this CTA's operand parts into its 4-stage shared-memory ring; completion
+//            is signalled on the "full" mbarrier of the pair's leader CTA.
+//   warp 1 : (leader CTA only) lane 0 issues tcgen05.mma (bf16 -> fp32);
+//            tcgen05.commit, multicast to both CTAs, releases the stage ("empty") and,
+//            after the last k-block, publishes the accumulator ("tfull").
+//   warps 2-9 : epilogue; each owns the 32 accumulator lanes its warp id selects and one
+//            256-column half, reads them with tcgen05.ld and applies the mode's fused
+//            epilogue, then releases the accumulator ("tempty", on the leader).
 // Every mbarrier wait is bounded: when it runs out the CTA raises SPO_DEV_TIMEOUT,
 // all roles leave their loops, tensor memory is released and the kernel returns.
 #include <cuda.h>
@@ -38,38 +40,31 @@ namespace spo {
 
 namespace {
 
-constexpr int BM = 128;                 // rows of A (and of the accumulator) per CTA
-constexpr int BN = 256;                 // columns of one output tile
+constexpr int CG = 2;                   // CTAs per MMA group (cluster size)
+constexpr int BM = 128;                 // rows of A (and accumulator lanes) per CTA
+constexpr int GROUP_M = BM * CG;        // rows of one output tile
+constexpr int HALF_N = 256;             // columns of one MMA / one accumulator half
+constexpr int BN = 2 * HALF_N;          // columns of one output tile
 constexpr int BK = 64;
-constexpr int A_BYTES = BM * BK * 2;
-constexpr int NUM_THREADS = 192;
+constexpr int STAGES = 4;
+constexpr int A_BYTES = BM * BK * 2;                 // 16 KB
+constexpr int BSUB_ROWS = HALF_N / CG;               // B columns per CTA per half (128)
+constexpr int BSUB_BYTES = BSUB_ROWS * BK * 2;       // 16 KB
+constexpr int STAGE_BYTES = A_BYTES + 2 * BSUB_BYTES;  // 48 KB
+constexpr int EPI_WARPS = 8;
+constexpr int NUM_THREADS = 32 * (2 + EPI_WARPS);
 constexpr int TMEM_COLS = 512;
-
-// Per-CTA shared-memory plan for a CTA group of CG CTAs.
-template <int CG>
-struct Plan {
-  static constexpr int kStages = CG == 2 ? 6 : 4;
-  static constexpr int kBRows = BN / CG;                  // columns of B held by this CTA
-  static constexpr int kBBytes = kBRows * BK * 2;
-  static constexpr int kStageBytes = A_BYTES + kBBytes;
-  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 + 256;
-};
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256;
 constexpr unsigned long long kWaitLimitNs = 4000000000ull;
-#ifndef SPO_EPI_SLEEP
-#define SPO_EPI_SLEEP 128
-#endif
-#ifndef SPO_PROD_SLEEP
-#define SPO_PROD_SLEEP 32
-#endif
-constexpr int kEpilogueSleepNs = SPO_EPI_SLEEP;
-constexpr int kProducerSleepNs = SPO_PROD_SLEEP;
+constexpr int kEpilogueSleepNs = 64;
+constexpr int kProducerSleepNs = 32;
 
 constexpr float kLog2e = 1.4426950408889634f;
 
 enum : int { MODE_FWD = 0, MODE_G = 1, MODE_DH = 2, MODE_DW = 3 };
 
 struct GemmParams {
-  int m_tiles, n_tiles, nsplit, per_split;   // work decomposition: unit = (row tile of the CTA group, split of the n tiles)
+  int m_tiles, n_tiles, nsplit, per_split;   // work decomposition: unit = (row tile, split of the column tiles)
   int k_blocks;                              // K / 64, rounded up
   int a_row0;                                // added to A's row coordinate (K-major A) or k coordinate (M-major A)
   int b_k0;                                  // added to B's k coordinate (N-major B)
@@ -120,26 +115,12 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
 // Arrive on a barrier given by a shared::cluster address (possibly in the peer CTA).
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
+// Cluster-scope acquire: the barriers here are arrived on by the peer CTA or by tcgen05.commit.
 __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.b32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok;
-}
-// Same, with cluster-scope acquire: for barriers that the peer CTA arrives on.
-__device__ __forceinline__ uint32_t mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
@@ -157,14 +138,12 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
 }
 
 // Bounded wait.  Returns false when the wait ran out or another role already gave up.
-// SLEEP_NS > 0 backs off between polls (for roles that wait long and need not react within
-// nanoseconds): a spinning warp occupies an issue slot every cycle and costs power that the
-// tensor pipe could use.
-template <bool CLUSTER_SCOPE = false, int SLEEP_NS = 0>
+// SLEEP_NS > 0 backs off between polls (roles that wait long and need not react within nanoseconds).
+template <int SLEEP_NS = 0>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* d_status) {
   uint32_t spins = 0;
   unsigned long long t0 = 0;
-  while (!(CLUSTER_SCOPE ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity))) {
+  while (!mbar_try_wait(bar, parity)) {
     if (SLEEP_NS > 0) __nanosleep(SLEEP_NS);
     if ((++spins & 255u) == 0) {
       if (*abort_flag) return false;
@@ -181,55 +160,31 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   return true;
 }
 
-// TMA tile load into this CTA's shared memory; completion bytes are counted on `bar`, which for
-// CG == 2 is a shared::cluster address and may belong to the pair's leader CTA.
-template <int CG>
+// TMA tile load into this CTA's shared memory; completion bytes are counted on `bar`, a
+// shared::cluster address that belongs to the pair's leader CTA.
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
-  if (CG == 1) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar)
-        : "memory");
-  } else {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar)
-        : "memory");
-  }
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar)
+      : "memory");
 }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-template <int CG>
 __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t acc) {
-  if (CG == 1) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(acc)
-        : "memory");
-  } else {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(acc)
-        : "memory");
-  }
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(acc)
+      : "memory");
 }
-// Arrive on `bar` once all MMAs issued so far have completed; for CG == 2 the arrival is
-// delivered to the barrier at the same offset in both CTAs of the pair.
-template <int CG>
+// Arrive, once all MMAs issued so far have completed, on the barrier at this offset in both CTAs.
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
-  if (CG == 1) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-  } else {
-    const uint16_t mask = 3;
-    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-                 ::"r"(bar), "h"(mask) : "memory");
-  }
+  const uint16_t mask = 3;
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"(mask) : "memory");
 }
 
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
@@ -264,10 +219,10 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint3
   return d;
 }
 
-// Instruction descriptor for kind::f16: fp32 accumulate, bf16 A and B, M = 128 per CTA of the group, N = 256.
-__host__ __device__ constexpr uint32_t instr_desc(bool a_mn, bool b_mn, int cg) {
+// Instruction descriptor for kind::f16: fp32 accumulate, bf16 A and B, M = 256 over the pair, N = 256.
+__host__ __device__ constexpr uint32_t instr_desc(bool a_mn, bool b_mn) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
-         ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((BM * cg) >> 4) << 24);
+         ((uint32_t)(HALF_N >> 3) << 17) | ((uint32_t)(GROUP_M >> 4) << 24);
 }
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
@@ -288,49 +243,40 @@ __device__ __forceinline__ Unit unit_of(int u, const GemmParams& p) {
 // ---------------------------------------------------------------------------
 // the kernel
 // ---------------------------------------------------------------------------
-template <int MODE, int CG>
+template <int MODE>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmParams p) {
   constexpr bool A_MN = (MODE == MODE_DW);
   constexpr bool B_MN = (MODE == MODE_DH || MODE == MODE_DW);
-  using P = Plan<CG>;
-  constexpr int STAGES = P::kStages;
-  constexpr int STAGE_BYTES = P::kStageBytes;
-  constexpr int B_ROWS = P::kBRows;
-  constexpr int GROUP_M = BM * CG;                   // rows of one output tile of the CTA group
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* gen = smem_raw + (base - raw);
   const uint32_t bars = base + STAGES * STAGE_BYTES;
-  const uint32_t full0 = bars, empty0 = bars + 8 * STAGES, tfull0 = bars + 16 * STAGES, tempty0 = tfull0 + 16;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen + STAGES * STAGE_BYTES + 16 * STAGES + 32);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + STAGES * STAGE_BYTES + 16 * STAGES + 40);
+  const uint32_t full0 = bars, empty0 = bars + 8 * STAGES, tfull = bars + 16 * STAGES, tempty = tfull + 8;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen + STAGES * STAGE_BYTES + 16 * STAGES + 16);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + STAGES * STAGE_BYTES + 16 * STAGES + 24);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const uint32_t rank = CG == 2 ? cluster_ctarank() : 0u;     // 0 = leader of the pair
+  const uint32_t rank = cluster_ctarank();                    // 0 = leader of the pair
   const int group = blockIdx.x / CG, n_groups = gridDim.x / CG;
   const int total_units = p.m_tiles * p.nsplit;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(tfull0 + 8 * a, 1); mbar_init(tempty0 + 8 * a, 4 * CG); }
+    mbar_init(tfull, 1);
+    mbar_init(tempty, EPI_WARPS * CG);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 0) {
-    if (CG == 1) {
-      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
-      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    } else {
-      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
-      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
-    }
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
   __syncthreads();
-  if (CG == 2) cluster_sync_all();          // the peer's barriers exist before anything signals them
+  cluster_sync_all();                       // the peer's barriers exist before anything signals them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
@@ -341,33 +287,33 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       bool ok = true;
       for (int u = group; u < total_units && ok; u += n_groups) {
         const Unit un = unit_of(u, p);
-        const int row_base = un.m_tile * GROUP_M + (int)rank * BM;      // this CTA's rows of the tile
+        const int row_base = un.m_tile * GROUP_M + (int)rank * BM;       // this CTA's rows of the tile
         for (int n = un.n_begin; n < un.n_end && ok; ++n) {
-          const int col_base = n * BN + (int)rank * B_ROWS;             // this CTA's columns of B
+          const int col_base = n * BN + (int)rank * BSUB_ROWS;           // this CTA's columns of half 0
           for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
             const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
-            if (!mbar_wait<CG == 2, kProducerSleepNs>(empty0 + 8 * s, ph ^ 1u, abort_flag, p.d_status)) { ok = false; break; }
+            if (!mbar_wait<kProducerSleepNs>(empty0 + 8 * s, ph ^ 1u, abort_flag, p.d_status)) { ok = false; break; }
             const uint32_t sa = base + s * STAGE_BYTES, sb = sa + A_BYTES;
-            uint32_t fb = full0 + 8 * s;
-            if (CG == 1) {
-              mbar_expect_tx(fb, STAGE_BYTES);
-            } else {
-              if (rank == 0) mbar_expect_tx(fb, 2 * STAGE_BYTES);        // both CTAs' bytes land on the leader's barrier
-              fb = map_to_cta(fb, 0);
-            }
+            if (rank == 0) mbar_expect_tx(full0 + 8 * s, CG * STAGE_BYTES);   // both CTAs' bytes land on the leader's barrier
+            const uint32_t fb = map_to_cta(full0 + 8 * s, 0);
             if (!A_MN) {
-              tma_load_2d<CG>(sa, &tmA, kb * BK, p.a_row0 + row_base, fb);
+              tma_load_2d(sa, &tmA, kb * BK, p.a_row0 + row_base, fb);
             } else {
 #pragma unroll
               for (int b = 0; b < BM / 64; ++b)
-                tma_load_2d<CG>(sa + b * 8192, &tmA, row_base + b * 64, p.a_row0 + kb * BK, fb);
+                tma_load_2d(sa + b * 8192, &tmA, row_base + b * 64, p.a_row0 + kb * BK, fb);
             }
-            if (!B_MN) {
-              tma_load_2d<CG>(sb, &tmB, kb * BK, col_base, fb);
-            } else {
 #pragma unroll
-              for (int b = 0; b < B_ROWS / 64; ++b)
-                tma_load_2d<CG>(sb + b * 8192, &tmB, col_base + b * 64, p.b_k0 + kb * BK, fb);
+            for (int h = 0; h < 2; ++h) {
+              const uint32_t sbh = sb + h * BSUB_BYTES;
+              const int col = col_base + h * HALF_N;
+              if (!B_MN) {
+                tma_load_2d(sbh, &tmB, kb * BK, col, fb);
+              } else {
+#pragma unroll
+                for (int b = 0; b < BSUB_ROWS / 64; ++b)
+                  tma_load_2d(sbh + b * 8192, &tmB, col + b * 64, p.b_k0 + kb * BK, fb);
+              }
             }
           }
         }
@@ -376,38 +322,42 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer (leader CTA)
     if (lane == 0 && rank == 0) {
-      constexpr uint32_t idesc = instr_desc(A_MN, B_MN, CG);
+      constexpr uint32_t idesc = instr_desc(A_MN, B_MN);
       uint32_t it = 0, tile = 0;
       bool ok = true;
       for (int u = group; u < total_units && ok; u += n_groups) {
         const Unit un = unit_of(u, p);
         for (int n = un.n_begin; n < un.n_end && ok; ++n, ++tile) {
-          const uint32_t acc = tile & 1u, aph = (tile >> 1) & 1u;
-          if (!mbar_wait<CG == 2>(tempty0 + 8 * acc, aph ^ 1u, abort_flag, p.d_status)) { ok = false; break; }
+          if (!mbar_wait(tempty, (tile & 1u) ^ 1u, abort_flag, p.d_status)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t tmem_d = tmem_base + acc * BN;
           for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
             const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
-            if (!mbar_wait<CG == 2>(full0 + 8 * s, ph, abort_flag, p.d_status)) { ok = false; break; }
+            if (!mbar_wait(full0 + 8 * s, ph, abort_flag, p.d_status)) { ok = false; break; }
             tc_fence_after();
             const uint32_t sa = base + s * STAGE_BYTES, sb = sa + A_BYTES;
 #pragma unroll
             for (int j = 0; j < BK / 16; ++j) {
               const uint64_t da = A_MN ? smem_desc(sa + j * 2048, 8192, 1024) : smem_desc(sa + j * 32, 16, 1024);
-              const uint64_t db = B_MN ? smem_desc(sb + j * 2048, 8192, 1024) : smem_desc(sb + j * 32, 16, 1024);
-              umma_bf16<CG>(tmem_d, da, db, idesc, (kb | j) != 0 ? 1u : 0u);
+#pragma unroll
+              for (int h = 0; h < 2; ++h) {
+                const uint32_t sbh = sb + h * BSUB_BYTES;
+                const uint64_t db = B_MN ? smem_desc(sbh + j * 2048, 8192, 1024) : smem_desc(sbh + j * 32, 16, 1024);
+                umma_bf16(tmem_base + h * HALF_N, da, db, idesc, (kb | j) != 0 ? 1u : 0u);
+              }
             }
-            umma_commit<CG>(empty0 + 8 * s);
+            umma_commit(empty0 + 8 * s);
           }
-          if (ok) umma_commit<CG>(tfull0 + 8 * acc);
+          if (ok) umma_commit(tfull);
         }
       }
     }
   } else {
-    // ------------------------------------------------------------------ epilogue (warps 2..5)
-    const int quarter = warp & 3;                    // tensor-memory lanes this warp may read
-    const int row = (int)rank * BM + quarter * 32 + lane;   // row of the group's tile
-    const uint32_t tempty_leader0 = CG == 2 ? map_to_cta(tempty0, 0) : tempty0;
+    // ------------------------------------------------------------------ epilogue (warps 2..9)
+    const int quarter = warp & 3;                            // tensor-memory lanes this warp may read
+    const int half = (warp - 2) >> 2;                        // which 256-column half of the tile
+    const int row = (int)rank * BM + quarter * 32 + lane;    // row of the pair's tile
+    const uint32_t tempty_leader = map_to_cta(tempty, 0);
+    const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + half * HALF_N;
     uint32_t tile = 0;
     bool ok = true;
     for (int u = group; u < total_units && ok; u += n_groups) {
@@ -423,36 +373,41 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         if (MODE == MODE_G && row_ok) { c = p.grad_loss * p.coef[grow]; lse2 = p.lse[grow] * kLog2e; }
       }
       for (int n = un.n_begin; n < un.n_end && ok; ++n, ++tile) {
-        const uint32_t acc = tile & 1u, aph = (tile >> 1) & 1u;
         {                                   // one lane polls (with backoff); the warp reconverges on its verdict
           int good = 1;
-          if (lane == 0) good = mbar_wait<CG == 2, kEpilogueSleepNs>(tfull0 + 8 * acc, aph, abort_flag, p.d_status) ? 1 : 0;
+          if (lane == 0) good = mbar_wait<kEpilogueSleepNs>(tfull, tile & 1u, abort_flag, p.d_status) ? 1 : 0;
           good = __shfl_sync(0xffffffffu, good, 0);
           if (!good) { ok = false; break; }
         }
         tc_fence_after();
-        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN;
-        const int col_tile = n * BN;
+        const int col_half = n * BN + half * HALF_N;
 #pragma unroll 1
-        for (int ch = 0; ch < BN / 32; ++ch) {
-          const int col0 = col_tile + ch * 32;
+        for (int ch = 0; ch < HALF_N / 32; ++ch) {
+          const int col0 = col_half + ch * 32;
           if (col0 >= p.cols_valid && MODE != MODE_G) break;          // nothing valid further right
           uint32_t v[32];
           tmem_ld32(taddr + ch * 32, v);
           if (MODE == MODE_FWD) {
-            const bool tail = col0 + 32 > p.cols_valid;
-            float cmax = -CUDART_INF_F;
+            if (col0 + 32 > p.cols_valid) {                            // ragged last chunk of the vocabulary
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-              float z = __uint_as_float(v[j]);
-              if (tail && col0 + j >= p.cols_valid) { z = -CUDART_INF_F; v[j] = __float_as_uint(z); }
-              cmax = fmaxf(cmax, z);
+              for (int j = 0; j < 32; ++j)
+                if (col0 + j >= p.cols_valid) v[j] = __float_as_uint(-CUDART_INF_F);
             }
-            const float mn = fmaxf(m2, cmax * kLog2e);
-            float sum = 0.0f;
+            float mx0 = __uint_as_float(v[0]), mx1 = __uint_as_float(v[1]);
 #pragma unroll
-            for (int j = 0; j < 32; ++j) sum += fast_exp2(fmaf(__uint_as_float(v[j]), kLog2e, -mn));
-            l = l * fast_exp2(m2 - mn) + sum;
+            for (int j = 2; j < 32; j += 2) {
+              mx0 = fmaxf(mx0, __uint_as_float(v[j]));
+              mx1 = fmaxf(mx1, __uint_as_float(v[j + 1]));
+            }
+            const float mn = fmaxf(m2, fmaxf(mx0, mx1) * kLog2e);
+            const float neg = -mn;
+            float s0 = 0.0f, s1 = 0.0f;
+#pragma unroll
+            for (int j = 0; j < 32; j += 2) {
+              s0 += fast_exp2(fmaf(__uint_as_float(v[j]), kLog2e, neg));
+              s1 += fast_exp2(fmaf(__uint_as_float(v[j + 1]), kLog2e, neg));
+            }
+            l = fmaf(l, fast_exp2(m2 - mn), s0 + s1);
             m2 = mn;
             if (yt >= col0 && yt < col0 + 32) {
               const int jj = yt - col0;
@@ -461,23 +416,29 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             }
           } else if (MODE == MODE_G) {
             if (row_ok) {
-              uint32_t o[16];
+              float g[32];
+              if (c != 0.0f) {
+                const float nc = -c;
 #pragma unroll
-              for (int j = 0; j < 32; j += 2) {
-                float g0 = 0.0f, g1 = 0.0f;
-                if (c != 0.0f) {
-                  const float p0 = fast_exp2(fmaf(__uint_as_float(v[j]), kLog2e, -lse2));
-                  const float p1 = fast_exp2(fmaf(__uint_as_float(v[j + 1]), kLog2e, -lse2));
-                  g0 = c * ((col0 + j == yt ? 1.0f : 0.0f) - p0);
-                  g1 = c * ((col0 + j + 1 == yt ? 1.0f : 0.0f) - p1);
+                for (int j = 0; j < 32; ++j) g[j] = nc * fast_exp2(fmaf(__uint_as_float(v[j]), kLog2e, -lse2));
+                if (yt >= col0 && yt < col0 + 32) {
+                  const int jj = yt - col0;
+#pragma unroll
+                  for (int j = 0; j < 32; ++j) if (j == jj) g[j] += c;
                 }
-                if (col0 + j >= p.cols_valid) g0 = 0.0f;
-                if (col0 + j + 1 >= p.cols_valid) g1 = 0.0f;
-                o[j >> 1] = pack_bf16(g0, g1);
+                if (col0 + 32 > p.cols_valid) {
+#pragma unroll
+                  for (int j = 0; j < 32; ++j) if (col0 + j >= p.cols_valid) g[j] = 0.0f;
+                }
+              } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) g[j] = 0.0f;
               }
               uint4* dst = reinterpret_cast<uint4*>(p.G + ((int64_t)un.m_tile * GROUP_M + row) * p.ldg + col0);
 #pragma unroll
-              for (int q = 0; q < 4; ++q) dst[q] = make_uint4(o[4 * q], o[4 * q + 1], o[4 * q + 2], o[4 * q + 3]);
+              for (int q = 0; q < 4; ++q)
+                dst[q] = make_uint4(pack_bf16(g[8 * q + 0], g[8 * q + 1]), pack_bf16(g[8 * q + 2], g[8 * q + 3]),
+                                    pack_bf16(g[8 * q + 4], g[8 * q + 5]), pack_bf16(g[8 * q + 6], g[8 * q + 7]));
             }
           } else {
             if (row_ok) {
@@ -492,12 +453,14 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
               } else {
                 float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + grow * p.ldo + col0);
                 if (p.accumulate) {
+                  float4 old[8];
+#pragma unroll
+                  for (int q = 0; q < 8; ++q) old[q] = dst[q];
 #pragma unroll
                   for (int q = 0; q < 8; ++q) {
-                    float4 old = dst[q];
-                    old.x += __uint_as_float(v[4 * q + 0]); old.y += __uint_as_float(v[4 * q + 1]);
-                    old.z += __uint_as_float(v[4 * q + 2]); old.w += __uint_as_float(v[4 * q + 3]);
-                    dst[q] = old;
+                    old[q].x += __uint_as_float(v[4 * q + 0]); old[q].y += __uint_as_float(v[4 * q + 1]);
+                    old[q].z += __uint_as_float(v[4 * q + 2]); old[q].w += __uint_as_float(v[4 * q + 3]);
+                    dst[q] = old[q];
                   }
                 } else {
 #pragma unroll
@@ -511,15 +474,12 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         }
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) {
-          if (CG == 1) mbar_arrive(tempty0 + 8 * acc);
-          else mbar_arrive_cluster(tempty_leader0 + 8 * acc);
-        }
+        if (lane == 0) mbar_arrive_cluster(tempty_leader);
       }
       if (MODE == MODE_FWD && ok && row_ok) {
         FwdPartial part;
         part.m2 = m2; part.l = l; part.zt = zt; part.pad = 0.0f;
-        p.partials[(int64_t)(u % p.nsplit) * p.T + grow] = part;
+        p.partials[(int64_t)((u % p.nsplit) * 2 + half) * p.T + grow] = part;
       }
     }
   }
@@ -531,23 +491,14 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   }
   tc_fence_before();
   __syncthreads();
-  if (CG == 2) cluster_sync_all();          // the peer may still be reading this CTA's shared / tensor memory
-  if (warp == 0) {
-    if (CG == 1)
-      asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
-    else
-      asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
-  }
+  cluster_sync_all();                       // the peer may still be reading this CTA's shared / tensor memory
+  if (warp == 0)
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
 }
 
 // ---------------------------------------------------------------------------
 // host side: tensor maps and launches
 // ---------------------------------------------------------------------------
-#ifndef SPO_CTA_GROUP
-#define SPO_CTA_GROUP 2
-#endif
-constexpr int kCG = SPO_CTA_GROUP;         // CTAs per MMA group used by the launches below
-
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -578,17 +529,16 @@ bool make_map(CUtensorMap* m, const void* ptr, uint64_t inner, uint64_t outer, u
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// CTA groups that can be resident at once (one CTA per SM).
-int group_count() { return sm_count() / kCG; }
+// CTA pairs that can be resident at once (one CTA per SM).
+int group_count() { return sm_count() / CG; }
 
 template <int MODE>
 cudaError_t launch_gemm(const CUtensorMap& a, const CUtensorMap& b, const GemmParams& p, cudaStream_t st) {
   static bool configured[64] = {};
   int dev = 0;
   cudaGetDevice(&dev);
-  constexpr int smem = Plan<kCG>::kSmemBytes;
   if (dev >= 0 && dev < 64 && !configured[dev]) {
-    cudaError_t e = cudaFuncSetAttribute(spo_gemm_kernel<MODE, kCG>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    cudaError_t e = cudaFuncSetAttribute(spo_gemm_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (e != cudaSuccess) return e;
     configured[dev] = true;
   }
@@ -596,27 +546,26 @@ cudaError_t launch_gemm(const CUtensorMap& a, const CUtensorMap& b, const GemmPa
   if (units <= 0) return cudaSuccess;
   const int groups = units < group_count() ? units : group_count();
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(groups * kCG, 1, 1);
+  cfg.gridDim = dim3(groups * CG, 1, 1);
   cfg.blockDim = dim3(NUM_THREADS, 1, 1);
-  cfg.dynamicSmemBytes = smem;
+  cfg.dynamicSmemBytes = SMEM_BYTES;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = kCG;
+  attr[0].val.clusterDim.x = CG;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, spo_gemm_kernel<MODE, kCG>, a, b, p);
+  return cudaLaunchKernelEx(&cfg, spo_gemm_kernel<MODE>, a, b, p);
 }
 
-// Operand box heights: A rows per CTA, B rows (columns of the output) per CTA.
+// Operand box heights (rows per TMA box) for K-major operands.
 constexpr uint32_t kBoxA = BM;
-constexpr uint32_t kBoxB = BN / kCG;
-constexpr int kGroupM = BM * kCG;
+constexpr uint32_t kBoxB = BSUB_ROWS;
 
 int pick_fwd_split(int64_t m_tiles, int n_tiles) {
-  // Enough units to fill the machine, and several splits so that CTA groups running together
+  // Enough units to fill the machine, and several splits so that CTA pairs running together
   // share token tiles (which then stay in L2) while sweeping different parts of W.
   int groups = group_count();
   int nsplit = 4;
@@ -626,16 +575,20 @@ int pick_fwd_split(int64_t m_tiles, int n_tiles) {
   return nsplit;
 }
 
-}  // namespace
-
-// nsplit used by the forward for a given shape (the workspace layout depends on it).
-int fwd_bf16_nsplit(int64_t T, int32_t V) {
-  const int64_t m_tiles = ceil_div(T, kGroupM);
+// Splits of the vocabulary tiles actually used for a given shape.
+int fwd_unit_splits(int64_t T, int32_t V) {
+  const int64_t m_tiles = ceil_div(T, GROUP_M);
   const int n_tiles = (int)ceil_div(V, BN);
   int nsplit = pick_fwd_split(m_tiles, n_tiles);
   const int per = (int)ceil_div(n_tiles, nsplit);
   return (int)ceil_div(n_tiles, per);
 }
+
+}  // namespace
+
+// Number of forward partials per token row (two column halves per vocabulary split);
+// the workspace layout depends on it.
+int fwd_bf16_nsplit(int64_t T, int32_t V) { return 2 * fwd_unit_splits(T, V); }
 
 cudaError_t launch_fwd_bf16(const void* H, const void* W, const int32_t* y, int64_t T, int32_t d, int32_t V,
                             FwdPartial* partials, int nsplit, int32_t* d_status, cudaStream_t st) {
@@ -643,10 +596,10 @@ cudaError_t launch_fwd_bf16(const void* H, const void* W, const int32_t* y, int6
   CUtensorMap ma, mb;
   if (!make_map(&ma, H, d, T, d, kBoxA) || !make_map(&mb, W, d, V, d, kBoxB)) return cudaErrorInvalidValue;
   GemmParams p{};
-  p.m_tiles = (int)ceil_div(T, kGroupM);
+  p.m_tiles = (int)ceil_div(T, GROUP_M);
   p.n_tiles = (int)ceil_div(V, BN);
-  p.per_split = (int)ceil_div(p.n_tiles, nsplit);
-  p.nsplit = nsplit;
+  p.nsplit = nsplit / 2;
+  p.per_split = (int)ceil_div(p.n_tiles, p.nsplit);
   p.k_blocks = (int)ceil_div(d, BK);
   p.rows_valid = T;
   p.cols_valid = V;
@@ -660,15 +613,15 @@ cudaError_t launch_fwd_bf16(const void* H, const void* W, const int32_t* y, int6
 
 BwdWs bwd_ws_layout(int64_t T, int32_t d, int32_t V) {
   BwdWs L{};
-  // Token rows per chunk: a multiple of the group tile height chosen so that the dH tiles of a
-  // full chunk (row tiles x d/256 column tiles) fill the CTA groups a whole number of times.
+  // Token rows per chunk: a multiple of the tile height chosen so that the dH tiles of a
+  // full chunk (row tiles x d/512 column tiles) fill the CTA pairs a whole number of times.
   const int groups = group_count();
   const int n_tiles_d = (int)ceil_div(d, BN);
   int64_t m_tiles = 32;
-  for (int64_t cand = 24; cand <= 64; ++cand)
+  for (int64_t cand = 24; cand <= 80; ++cand)
     if ((cand * n_tiles_d) % groups == 0) { m_tiles = cand; break; }
-  int64_t rows = m_tiles * kGroupM;
-  const int64_t t_pad = ceil_div(T > 0 ? T : 1, kGroupM) * kGroupM;
+  int64_t rows = m_tiles * GROUP_M;
+  const int64_t t_pad = ceil_div(T > 0 ? T : 1, GROUP_M) * GROUP_M;
   if (rows > t_pad) rows = t_pad;
   L.chunk_rows = rows;
   L.ldg = ceil_div(V, BN) * BN;
@@ -696,7 +649,7 @@ cudaError_t launch_bwd_bf16(const void* H, const void* W, const int32_t* y, cons
   int chunk = 0;
   for (int64_t t0 = 0; t0 < T; t0 += L.chunk_rows, ++chunk) {
     const int64_t rows = (T - t0) < L.chunk_rows ? (T - t0) : L.chunk_rows;
-    const int m_tiles = (int)ceil_div(rows, kGroupM);
+    const int m_tiles = (int)ceil_div(rows, GROUP_M);
     CUtensorMap mG_k, mG_mn;
     if (!make_map(&mG_k, G, V, rows, L.ldg, kBoxA) || !make_map(&mG_mn, G, V, rows, L.ldg, 64))
       return cudaErrorInvalidValue;
@@ -739,7 +692,7 @@ cudaError_t launch_bwd_bf16(const void* H, const void* W, const int32_t* y, cons
     // 3) dW (+)= G^T H_chunk
     {
       GemmParams p{};
-      p.m_tiles = (int)ceil_div(V, kGroupM);
+      p.m_tiles = (int)ceil_div(V, GROUP_M);
       p.n_tiles = n_tiles_d;
       p.nsplit = n_tiles_d;
       p.per_split = 1;
