@@ -36,14 +36,14 @@ int device_is_sm100() {
   return major == 10;
 }
 
-int fwd_bf16_nsplit(int64_t T, int32_t V);   // spo_loss_tc.cu
+int fwd_bf16_nsplit(int64_t T, int32_t d, int32_t V);   // spo_loss_tc.cu
 
 FwdWs fwd_ws_layout(int64_t T, int32_t d, int32_t V, int32_t dtype) {
-  (void)d;
   FwdWs L{};
-  L.nsplit = dtype == SPO_DTYPE_BF16 ? fwd_bf16_nsplit(T, V) : 1;
+  L.nsplit = dtype == SPO_DTYPE_BF16 ? fwd_bf16_nsplit(T, d, V) : 1;
   L.fin_blocks = ceil_div(T > 0 ? T : 1, kFinalizeThreads);
   size_t off = 0;
+  L.progress = off;   off = align_up(off + kProgressBytes, 256);
   L.partials = off;   off = align_up(off + sizeof(FwdPartial) * (size_t)L.nsplit * (size_t)(T > 0 ? T : 1), 256);
   L.block_sums = off; off = align_up(off + sizeof(double) * (size_t)L.fin_blocks, 256);
   L.counters = off;   off = align_up(off + 4 * sizeof(int32_t), 256);
@@ -176,7 +176,7 @@ int32_t spo_loss_fwd(const void* H, const void* W, int32_t dtype, const int32_t*
   cudaError_t e = launch_fwd_prepare(mask, T, counters, st);
   if (e != cudaSuccess) return cuda_fail(e);
   if (dtype == SPO_DTYPE_BF16)
-    e = launch_fwd_bf16(H, W, y, T, d, V, partials, L.nsplit, d_status, st);
+    e = launch_fwd_bf16(H, W, y, T, d, V, partials, L.nsplit, reinterpret_cast<uint32_t*>(w8 + L.progress), d_status, st);
   else
     e = launch_fwd_f32((const float*)H, (const float*)W, y, T, d, V, partials, st);
   if (e != cudaSuccess) return cuda_fail(e);

@@ -50,7 +50,10 @@ struct FwdPartial { float m2, l, zt; float pad; };
 
 constexpr int kFinalizeThreads = 256;
 
+constexpr size_t kProgressBytes = 1024;   // per-launch progress words of the CTA pairs (bf16 path)
+
 struct FwdWs {
+  size_t progress;      // uint32 [256]
   size_t partials;      // FwdPartial [nsplit][T]
   size_t block_sums;    // double [finalize blocks]
   size_t counters;      // int32 [4]: n_tok, ticket
@@ -79,6 +82,7 @@ cudaError_t launch_bwd_f32(const float* H, const float* W, const int32_t* y, con
 // bf16 tensor-core path
 struct BwdWs {
   size_t g;             // bf16 [chunk_rows][ldg]
+  size_t progress;      // uint32 [256]
   size_t total;
   int64_t chunk_rows;   // token rows per chunk (multiple of 128)
   int64_t ldg;          // row pitch of g in elements (multiple of 256)
@@ -86,7 +90,7 @@ struct BwdWs {
 BwdWs bwd_ws_layout(int64_t T, int32_t d, int32_t V);
 
 cudaError_t launch_fwd_bf16(const void* H, const void* W, const int32_t* y, int64_t T, int32_t d, int32_t V,
-                            FwdPartial* partials, int nsplit, int32_t* d_status, cudaStream_t st);
+                            FwdPartial* partials, int nsplit, uint32_t* progress, int32_t* d_status, cudaStream_t st);
 cudaError_t launch_bwd_bf16(const void* H, const void* W, const int32_t* y, const float* lse,
                             const float* coef, float grad_loss, int64_t T, int32_t d, int32_t V,
                             void* dH, int32_t dH_dtype, float* dW, int accumulate,

@@ -33,6 +33,7 @@
 #include <cuda_runtime.h>
 #include <math_constants.h>
 #include <stdint.h>
+#include <stdlib.h>
 
 #include "spo_internal.h"
 
@@ -54,7 +55,8 @@ constexpr int STAGE_BYTES = A_BYTES + 2 * BSUB_BYTES;  // 48 KB
 constexpr int EPI_WARPS = 8;
 constexpr int NUM_THREADS = 32 * (2 + EPI_WARPS);
 constexpr int TMEM_COLS = 512;
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256;
+constexpr int STAGING_BYTES = 4096;                    // per epilogue warp: 32 rows x 128 bytes, for coalesced stores
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256 + EPI_WARPS * STAGING_BYTES;
 constexpr unsigned long long kWaitLimitNs = 4000000000ull;
 constexpr int kEpilogueSleepNs = 64;
 constexpr int kProducerSleepNs = 32;
@@ -86,6 +88,9 @@ struct GemmParams {
   int64_t ldo;
   int accumulate;
   int32_t* d_status;
+  // Soft lock-step between CTA pairs (FWD / G): progress[g] = tiles started by pair g (+1), ~0u when done.
+  uint32_t* progress;
+  int window;
 };
 
 // ---------------------------------------------------------------------------
@@ -207,6 +212,80 @@ __device__ __forceinline__ float fast_exp2(float x) {
   return r;
 }
 
+__device__ __forceinline__ void tmem_ld32_nowait(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+        "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+        "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// The lane that owns tile row `lane` deposits its 128 bytes (eight 16-byte pieces) into the warp's
+// staging buffer; piece c of row r sits at position c ^ (r & 7) so that both this row-wise write and
+// the piece-wise read-back below are free of bank conflicts.
+__device__ __forceinline__ void stage_put(uint8_t* stage, int lane, const uint4 (&piece)[8]) {
+  __syncwarp();                                   // earlier read-backs of this buffer are done
+#pragma unroll
+  for (int c = 0; c < 8; ++c)
+    *reinterpret_cast<uint4*>(stage + lane * 128 + ((c ^ (lane & 7)) << 4)) = piece[c];
+  __syncwarp();
+}
+// Read-back i (0..7): lanes 8j..8j+7 fetch the eight pieces of row 4i + j, so one warp-wide global
+// access covers four whole 128-byte rows.
+__device__ __forceinline__ uint4 stage_get(const uint8_t* stage, int lane, int i, int& r, int& c) {
+  r = 4 * i + (lane >> 3);
+  c = lane & 7;
+  return *reinterpret_cast<const uint4*>(stage + r * 128 + ((c ^ (r & 7)) << 4));
+}
+
+// g = c_t (1[v = y_t] - 2^(z log2e - lse_t log2e)) for 32 consecutive columns, packed to bf16.
+__device__ __forceinline__ void g_values(const uint32_t (&v)[32], int col0, float c, float lse2, int yt,
+                                         int cols_valid, uint4* out4) {
+  float g[32];
+  if (c != 0.0f) {
+    const float nc = -c;
+#pragma unroll
+    for (int j = 0; j < 32; ++j) g[j] = nc * fast_exp2(fmaf(__uint_as_float(v[j]), kLog2e, -lse2));
+    if (yt >= col0 && yt < col0 + 32) {
+      const int jj = yt - col0;
+#pragma unroll
+      for (int j = 0; j < 32; ++j) if (j == jj) g[j] += c;
+    }
+    if (col0 + 32 > cols_valid) {
+#pragma unroll
+      for (int j = 0; j < 32; ++j) if (col0 + j >= cols_valid) g[j] = 0.0f;
+    }
+  } else {
+#pragma unroll
+    for (int j = 0; j < 32; ++j) g[j] = 0.0f;
+  }
+#pragma unroll
+  for (int q = 0; q < 4; ++q)
+    out4[q] = make_uint4(pack_bf16(g[8 * q + 0], g[8 * q + 1]), pack_bf16(g[8 * q + 2], g[8 * q + 3]),
+                         pack_bf16(g[8 * q + 4], g[8 * q + 5]), pack_bf16(g[8 * q + 6], g[8 * q + 7]));
+}
+
+__device__ __forceinline__ void bf16_values(const uint32_t (&v)[32], uint4* out4) {
+#pragma unroll
+  for (int q = 0; q < 4; ++q)
+    out4[q] = make_uint4(pack_bf16(__uint_as_float(v[8 * q + 0]), __uint_as_float(v[8 * q + 1])),
+                         pack_bf16(__uint_as_float(v[8 * q + 2]), __uint_as_float(v[8 * q + 3])),
+                         pack_bf16(__uint_as_float(v[8 * q + 4]), __uint_as_float(v[8 * q + 5])),
+                         pack_bf16(__uint_as_float(v[8 * q + 6]), __uint_as_float(v[8 * q + 7])));
+}
+
+
 // Shared-memory matrix descriptor, 128-byte swizzle (layout type 2), descriptor version 1.
 // lbo / sbo in bytes.
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo) {
@@ -225,10 +304,6 @@ __host__ __device__ constexpr uint32_t instr_desc(bool a_mn, bool b_mn) {
          ((uint32_t)(HALF_N >> 3) << 17) | ((uint32_t)(GROUP_M >> 4) << 24);
 }
 
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-  return *reinterpret_cast<uint32_t*>(&v);
-}
 
 struct Unit { int m_tile, n_begin, n_end; };
 __device__ __forceinline__ Unit unit_of(int u, const GemmParams& p) {
@@ -282,17 +357,38 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
-    if (lane == 0) {
-      uint32_t it = 0;
-      bool ok = true;
-      for (int u = group; u < total_units && ok; u += n_groups) {
-        const Unit un = unit_of(u, p);
-        const int row_base = un.m_tile * GROUP_M + (int)rank * BM;       // this CTA's rows of the tile
-        for (int n = un.n_begin; n < un.n_end && ok; ++n) {
+    // Lane 0 issues the loads.  At every tile boundary the whole warp compares this pair's tile
+    // count with the other pairs' and holds back while it is more than `window` tiles ahead of the
+    // slowest: pairs that sweep the same part of W then stay close enough in time for its tiles to
+    // be served from L2 instead of being streamed from HBM once per pair.  The hold is bounded and
+    // advisory (after ~100 us the pair goes on regardless), so it can never dead-lock.
+    uint32_t it = 0, tseq = 0;
+    int ok = 1;
+    volatile uint32_t* progress = (rank == 0) ? p.progress : nullptr;
+    for (int u = group; u < total_units && ok; u += n_groups) {
+      const Unit un = unit_of(u, p);
+      const int row_base = un.m_tile * GROUP_M + (int)rank * BM;       // this CTA's rows of the tile
+      for (int n = un.n_begin; n < un.n_end && ok; ++n) {
+        if (progress) {
+          ++tseq;
+          if (lane == 0) progress[group] = tseq;
+          if ((int)tseq > p.window) {
+            for (int tries = 0; tries < 128; ++tries) {
+              uint32_t mn = 0xFFFFFFFFu;
+              for (int g = lane; g < n_groups; g += 32) mn = min(mn, progress[g]);
+#pragma unroll
+              for (int o = 16; o > 0; o >>= 1) mn = min(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+              if (mn + (uint32_t)p.window >= tseq) break;
+              __nanosleep(256);
+            }
+          }
+          __syncwarp();
+        }
+        if (lane == 0) {
           const int col_base = n * BN + (int)rank * BSUB_ROWS;           // this CTA's columns of half 0
           for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
             const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
-            if (!mbar_wait<kProducerSleepNs>(empty0 + 8 * s, ph ^ 1u, abort_flag, p.d_status)) { ok = false; break; }
+            if (!mbar_wait<kProducerSleepNs>(empty0 + 8 * s, ph ^ 1u, abort_flag, p.d_status)) { ok = 0; break; }
             const uint32_t sa = base + s * STAGE_BYTES, sb = sa + A_BYTES;
             if (rank == 0) mbar_expect_tx(full0 + 8 * s, CG * STAGE_BYTES);   // both CTAs' bytes land on the leader's barrier
             const uint32_t fb = map_to_cta(full0 + 8 * s, 0);
@@ -317,8 +413,10 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             }
           }
         }
+        ok = __shfl_sync(0xffffffffu, ok, 0);
       }
     }
+    if (progress && lane == 0) progress[group] = 0xFFFFFFFFu;          // done: never hold anyone back
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer (leader CTA)
     if (lane == 0 && rank == 0) {
@@ -356,13 +454,16 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     const int quarter = warp & 3;                            // tensor-memory lanes this warp may read
     const int half = (warp - 2) >> 2;                        // which 256-column half of the tile
     const int row = (int)rank * BM + quarter * 32 + lane;    // row of the pair's tile
+    const int warp_row0 = (int)rank * BM + quarter * 32;     // tile row of the warp's first lane
+    uint8_t* stage = gen + STAGES * STAGE_BYTES + 256 + (warp - 2) * STAGING_BYTES;
     const uint32_t tempty_leader = map_to_cta(tempty, 0);
     const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + half * HALF_N;
     uint32_t tile = 0;
     bool ok = true;
     for (int u = group; u < total_units && ok; u += n_groups) {
       const Unit un = unit_of(u, p);
-      const int64_t grow = p.out_row0 + (int64_t)un.m_tile * GROUP_M + row;   // global output row
+      const int64_t grow = p.out_row0 + (int64_t)un.m_tile * GROUP_M + row;   // global output row of this lane
+      const int64_t grow_warp0 = grow - lane;                                  // ... and of the warp's first lane
       const bool row_ok = grow < p.rows_valid;
       // per-row state
       float m2 = -CUDART_INF_F, l = 0.0f, zt = -CUDART_INF_F;             // FWD
@@ -381,13 +482,13 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         }
         tc_fence_after();
         const int col_half = n * BN + half * HALF_N;
+        if (MODE == MODE_FWD) {
 #pragma unroll 1
-        for (int ch = 0; ch < HALF_N / 32; ++ch) {
-          const int col0 = col_half + ch * 32;
-          if (col0 >= p.cols_valid && MODE != MODE_G) break;          // nothing valid further right
-          uint32_t v[32];
-          tmem_ld32(taddr + ch * 32, v);
-          if (MODE == MODE_FWD) {
+          for (int ch = 0; ch < HALF_N / 32; ++ch) {
+            const int col0 = col_half + ch * 32;
+            if (col0 >= p.cols_valid) break;                           // nothing valid further right
+            uint32_t v[32];
+            tmem_ld32(taddr + ch * 32, v);
             if (col0 + 32 > p.cols_valid) {                            // ragged last chunk of the vocabulary
 #pragma unroll
               for (int j = 0; j < 32; ++j)
@@ -414,61 +515,70 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 #pragma unroll
               for (int j = 0; j < 32; ++j) if (j == jj) zt = __uint_as_float(v[j]);
             }
-          } else if (MODE == MODE_G) {
-            if (row_ok) {
-              float g[32];
-              if (c != 0.0f) {
-                const float nc = -c;
-#pragma unroll
-                for (int j = 0; j < 32; ++j) g[j] = nc * fast_exp2(fmaf(__uint_as_float(v[j]), kLog2e, -lse2));
-                if (yt >= col0 && yt < col0 + 32) {
-                  const int jj = yt - col0;
-#pragma unroll
-                  for (int j = 0; j < 32; ++j) if (j == jj) g[j] += c;
-                }
-                if (col0 + 32 > p.cols_valid) {
-#pragma unroll
-                  for (int j = 0; j < 32; ++j) if (col0 + j >= p.cols_valid) g[j] = 0.0f;
-                }
-              } else {
-#pragma unroll
-                for (int j = 0; j < 32; ++j) g[j] = 0.0f;
-              }
-              uint4* dst = reinterpret_cast<uint4*>(p.G + ((int64_t)un.m_tile * GROUP_M + row) * p.ldg + col0);
-#pragma unroll
-              for (int q = 0; q < 4; ++q)
-                dst[q] = make_uint4(pack_bf16(g[8 * q + 0], g[8 * q + 1]), pack_bf16(g[8 * q + 2], g[8 * q + 3]),
-                                    pack_bf16(g[8 * q + 4], g[8 * q + 5]), pack_bf16(g[8 * q + 6], g[8 * q + 7]));
+          }
+        } else if (MODE == MODE_G || (MODE == MODE_DH && p.out_bf16)) {
+          // bf16 outputs: 64 columns (128 bytes per row) per staging round
+          __nv_bfloat16* obase = MODE == MODE_G
+              ? p.G + ((int64_t)un.m_tile * GROUP_M + warp_row0) * p.ldg
+              : reinterpret_cast<__nv_bfloat16*>(p.out) + grow_warp0 * p.ldo;
+          const int64_t ld = MODE == MODE_G ? p.ldg : p.ldo;
+#pragma unroll 1
+          for (int r2 = 0; r2 < HALF_N / 64; ++r2) {
+            const int col0 = col_half + r2 * 64;
+            if (MODE != MODE_G && col0 >= p.cols_valid) break;
+            uint32_t v0[32], v1[32];
+            tmem_ld32_nowait(taddr + r2 * 64, v0);
+            tmem_ld32_nowait(taddr + r2 * 64 + 32, v1);
+            tmem_wait_ld();
+            uint4 piece[8];
+            if (MODE == MODE_G) {
+              g_values(v0, col0, c, lse2, yt, p.cols_valid, piece);
+              g_values(v1, col0 + 32, c, lse2, yt, p.cols_valid, piece + 4);
+            } else {
+              bf16_values(v0, piece);
+              bf16_values(v1, piece + 4);
             }
-          } else {
-            if (row_ok) {
-              if (p.out_bf16) {
-                uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.out) + grow * p.ldo + col0);
+            stage_put(stage, lane, piece);
 #pragma unroll
-                for (int q = 0; q < 4; ++q)
-                  dst[q] = make_uint4(pack_bf16(__uint_as_float(v[8 * q + 0]), __uint_as_float(v[8 * q + 1])),
-                                      pack_bf16(__uint_as_float(v[8 * q + 2]), __uint_as_float(v[8 * q + 3])),
-                                      pack_bf16(__uint_as_float(v[8 * q + 4]), __uint_as_float(v[8 * q + 5])),
-                                      pack_bf16(__uint_as_float(v[8 * q + 6]), __uint_as_float(v[8 * q + 7])));
-              } else {
-                float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + grow * p.ldo + col0);
-                if (p.accumulate) {
-                  float4 old[8];
+            for (int i = 0; i < 8; ++i) {
+              int r, cc;
+              const uint4 val = stage_get(stage, lane, i, r, cc);
+              if (grow_warp0 + r < p.rows_valid)
+                *reinterpret_cast<uint4*>(obase + (int64_t)r * ld + col0 + cc * 8) = val;
+            }
+          }
+        } else {
+          // fp32 outputs: 32 columns (128 bytes per row) per staging round; dW may accumulate
+          float* obase = reinterpret_cast<float*>(p.out) + grow_warp0 * p.ldo;
+#pragma unroll 1
+          for (int ch = 0; ch < HALF_N / 32; ++ch) {
+            const int col0 = col_half + ch * 32;
+            if (col0 >= p.cols_valid) break;
+            uint32_t v[32];
+            tmem_ld32(taddr + ch * 32, v);
+            uint4 piece[8];
 #pragma unroll
-                  for (int q = 0; q < 8; ++q) old[q] = dst[q];
+            for (int q = 0; q < 8; ++q) piece[q] = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+            stage_put(stage, lane, piece);
+            float4 old[8];
+            if (p.accumulate) {
 #pragma unroll
-                  for (int q = 0; q < 8; ++q) {
-                    old[q].x += __uint_as_float(v[4 * q + 0]); old[q].y += __uint_as_float(v[4 * q + 1]);
-                    old[q].z += __uint_as_float(v[4 * q + 2]); old[q].w += __uint_as_float(v[4 * q + 3]);
-                    dst[q] = old[q];
-                  }
-                } else {
-#pragma unroll
-                  for (int q = 0; q < 8; ++q)
-                    dst[q] = make_float4(__uint_as_float(v[4 * q + 0]), __uint_as_float(v[4 * q + 1]),
-                                         __uint_as_float(v[4 * q + 2]), __uint_as_float(v[4 * q + 3]));
-                }
+              for (int i = 0; i < 8; ++i) {
+                const int r = 4 * i + (lane >> 3), cc = lane & 7;
+                old[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (grow_warp0 + r < p.rows_valid)
+                  old[i] = *reinterpret_cast<const float4*>(obase + (int64_t)r * p.ldo + col0 + cc * 4);
               }
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              int r, cc;
+              const uint4 raw4 = stage_get(stage, lane, i, r, cc);
+              float4 val = make_float4(__uint_as_float(raw4.x), __uint_as_float(raw4.y), __uint_as_float(raw4.z),
+                                       __uint_as_float(raw4.w));
+              if (p.accumulate) { val.x += old[i].x; val.y += old[i].y; val.z += old[i].z; val.w += old[i].w; }
+              if (grow_warp0 + r < p.rows_valid)
+                *reinterpret_cast<float4*>(obase + (int64_t)r * p.ldo + col0 + cc * 4) = val;
             }
           }
         }
@@ -529,11 +639,18 @@ bool make_map(CUtensorMap* m, const void* ptr, uint64_t inner, uint64_t outer, u
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Window (in tiles) of the lock-step hold between CTA pairs; 0 disables it.
+int throttle_window() {
+  if (const char* e = getenv("SPO_DEV_WINDOW")) return atoi(e);
+  return 1;
+}
+
 // CTA pairs that can be resident at once (one CTA per SM).
 int group_count() { return sm_count() / CG; }
 
 template <int MODE>
-cudaError_t launch_gemm(const CUtensorMap& a, const CUtensorMap& b, const GemmParams& p, cudaStream_t st) {
+cudaError_t launch_gemm(const CUtensorMap& a, const CUtensorMap& b, const GemmParams& p_in, uint32_t* progress,
+                        cudaStream_t st) {
   static bool configured[64] = {};
   int dev = 0;
   cudaGetDevice(&dev);
@@ -542,8 +659,16 @@ cudaError_t launch_gemm(const CUtensorMap& a, const CUtensorMap& b, const GemmPa
     if (e != cudaSuccess) return e;
     configured[dev] = true;
   }
-  const int units = p.m_tiles * p.nsplit;
+  const int units = p_in.m_tiles * p_in.nsplit;
   if (units <= 0) return cudaSuccess;
+  GemmParams p = p_in;
+  p.window = throttle_window();
+  p.progress = nullptr;
+  if (p.window > 0 && progress) {
+    cudaError_t e = cudaMemsetAsync(progress, 0, kProgressBytes, st);
+    if (e != cudaSuccess) return e;
+    p.progress = progress;
+  }
   const int groups = units < group_count() ? units : group_count();
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(groups * CG, 1, 1);
@@ -564,34 +689,49 @@ cudaError_t launch_gemm(const CUtensorMap& a, const CUtensorMap& b, const GemmPa
 constexpr uint32_t kBoxA = BM;
 constexpr uint32_t kBoxB = BSUB_ROWS;
 
-int pick_fwd_split(int64_t m_tiles, int n_tiles) {
-  // Enough units to fill the machine, and several splits so that CTA pairs running together
-  // share token tiles (which then stay in L2) while sweeping different parts of W.
-  int groups = group_count();
-  int nsplit = 4;
-  while (m_tiles * nsplit < 2 * (int64_t)groups && nsplit < n_tiles) nsplit *= 2;
-  if (nsplit > n_tiles) nsplit = n_tiles;
-  if (nsplit < 1) nsplit = 1;
-  return nsplit;
+// How many splits of the column tiles a FWD / G launch uses.  All pairs running at one time form
+// a rectangle of (pairs / nsplit) row tiles x nsplit column positions; per sweep step L2 has to hold
+// that many A tiles (re-read every step) plus nsplit B tiles (streamed).  Fewer splits mean fewer
+// re-reads of W from HBM; the choice also avoids a short last split (pairs would fall out of step)
+// and a nearly empty last round of units.
+int pick_fwd_split(int64_t m_tiles, int n_tiles, int d) {
+  if (const char* e = getenv("SPO_DEV_FWD_SPLIT")) { int v = atoi(e); if (v > 0) return v < n_tiles ? v : n_tiles; }
+  const int groups = group_count();
+  const double a_tile = (double)GROUP_M * d * 2, b_tile = (double)BN * d * 2;
+  const double l2_budget = 56e6;
+  int best = 1;
+  double best_score = -1.0;
+  for (int ns = 1; ns <= n_tiles && ns <= 256; ++ns) {
+    const int per = (int)ceil_div(n_tiles, ns);
+    if ((int)ceil_div(n_tiles, per) != ns) continue;               // not a distinct partition
+    const double ragged = (double)(ns * per - n_tiles) / (double)(ns * per);
+    const int64_t units = m_tiles * ns;
+    const int64_t rounds = ceil_div(units, groups);
+    const double fill = (double)units / (double)(rounds * groups);
+    const double rows_live = (double)(m_tiles < (groups + ns - 1) / ns ? m_tiles : (groups + ns - 1) / ns);
+    const double footprint = rows_live * a_tile + ns * b_tile;
+    double score = fill * (1.0 - ragged) / (1.0 + 0.01 * ns);
+    if (footprint > l2_budget) score *= l2_budget / footprint;
+    if (score > best_score) { best_score = score; best = ns; }
+  }
+  return best;
 }
 
 // Splits of the vocabulary tiles actually used for a given shape.
-int fwd_unit_splits(int64_t T, int32_t V) {
+int fwd_unit_splits(int64_t T, int32_t d, int32_t V) {
   const int64_t m_tiles = ceil_div(T, GROUP_M);
   const int n_tiles = (int)ceil_div(V, BN);
-  int nsplit = pick_fwd_split(m_tiles, n_tiles);
-  const int per = (int)ceil_div(n_tiles, nsplit);
-  return (int)ceil_div(n_tiles, per);
+  return pick_fwd_split(m_tiles, n_tiles, d);
 }
 
 }  // namespace
 
 // Number of forward partials per token row (two column halves per vocabulary split);
 // the workspace layout depends on it.
-int fwd_bf16_nsplit(int64_t T, int32_t V) { return 2 * fwd_unit_splits(T, V); }
+int fwd_bf16_nsplit(int64_t T, int32_t d, int32_t V) { return 2 * fwd_unit_splits(T, d, V); }
 
 cudaError_t launch_fwd_bf16(const void* H, const void* W, const int32_t* y, int64_t T, int32_t d, int32_t V,
-                            FwdPartial* partials, int nsplit, int32_t* d_status, cudaStream_t st) {
+                            FwdPartial* partials, int nsplit, uint32_t* progress, int32_t* d_status, cudaStream_t st) {
   if (T == 0) return cudaSuccess;
   CUtensorMap ma, mb;
   if (!make_map(&ma, H, d, T, d, kBoxA) || !make_map(&mb, W, d, V, d, kBoxB)) return cudaErrorInvalidValue;
@@ -608,25 +748,25 @@ cudaError_t launch_fwd_bf16(const void* H, const void* W, const int32_t* y, int6
   p.partials = partials;
   p.T = T;
   p.d_status = d_status;
-  return launch_gemm<MODE_FWD>(ma, mb, p, st);
+  return launch_gemm<MODE_FWD>(ma, mb, p, progress, st);
 }
 
 BwdWs bwd_ws_layout(int64_t T, int32_t d, int32_t V) {
   BwdWs L{};
-  // Token rows per chunk: a multiple of the tile height chosen so that the dH tiles of a
-  // full chunk (row tiles x d/512 column tiles) fill the CTA pairs a whole number of times.
+  // Token rows per chunk: half as many row tiles as there are CTA pairs.  With d/512 column
+  // tiles (a multiple of 2 for the usual hidden sizes) the dH tiles of a full chunk then fill the
+  // pairs a whole number of times, and the chunk buffer stays at a few GB.
   const int groups = group_count();
-  const int n_tiles_d = (int)ceil_div(d, BN);
-  int64_t m_tiles = 32;
-  for (int64_t cand = 24; cand <= 80; ++cand)
-    if ((cand * n_tiles_d) % groups == 0) { m_tiles = cand; break; }
+  int64_t m_tiles = groups / 2 > 0 ? groups / 2 : 1;
+  if (const char* e = getenv("SPO_DEV_CHUNK_TILES")) { int v = atoi(e); if (v > 0) m_tiles = v; }
   int64_t rows = m_tiles * GROUP_M;
   const int64_t t_pad = ceil_div(T > 0 ? T : 1, GROUP_M) * GROUP_M;
   if (rows > t_pad) rows = t_pad;
   L.chunk_rows = rows;
   L.ldg = ceil_div(V, BN) * BN;
   L.g = 0;
-  L.total = align_up((size_t)rows * (size_t)L.ldg * 2, 256);
+  L.progress = align_up((size_t)rows * (size_t)L.ldg * 2, 256);
+  L.total = L.progress + kProgressBytes;
   return L;
 }
 
@@ -635,6 +775,7 @@ cudaError_t launch_bwd_bf16(const void* H, const void* W, const int32_t* y, cons
                             void* dH, int32_t dH_dtype, float* dW, int accumulate,
                             char* ws, const BwdWs& L, int32_t* d_status, cudaStream_t st) {
   __nv_bfloat16* G = reinterpret_cast<__nv_bfloat16*>(ws + L.g);
+  uint32_t* progress = reinterpret_cast<uint32_t*>(ws + L.progress);
   if (T == 0) {
     if (!accumulate) return cudaMemsetAsync(dW, 0, sizeof(float) * (size_t)V * d, st);
     return cudaSuccess;
@@ -658,9 +799,8 @@ cudaError_t launch_bwd_bf16(const void* H, const void* W, const int32_t* y, cons
       GemmParams p{};
       p.m_tiles = m_tiles;
       p.n_tiles = n_tiles_v;
-      int nsplit = pick_fwd_split(m_tiles, n_tiles_v);
-      p.per_split = (int)ceil_div(n_tiles_v, nsplit);
-      p.nsplit = (int)ceil_div(n_tiles_v, p.per_split);
+      p.nsplit = pick_fwd_split(m_tiles, n_tiles_v, d);
+      p.per_split = (int)ceil_div(n_tiles_v, p.nsplit);
       p.k_blocks = (int)ceil_div(d, BK);
       p.a_row0 = (int)t0;
       p.rows_valid = T;
@@ -670,7 +810,7 @@ cudaError_t launch_bwd_bf16(const void* H, const void* W, const int32_t* y, cons
       p.T = T;
       p.G = G; p.ldg = L.ldg;
       p.d_status = d_status;
-      if ((e = launch_gemm<MODE_G>(mH_k, mW_k, p, st)) != cudaSuccess) return e;
+      if ((e = launch_gemm<MODE_G>(mH_k, mW_k, p, progress, st)) != cudaSuccess) return e;
     }
     // 2) dH rows of the chunk = G W
     {
@@ -687,7 +827,7 @@ cudaError_t launch_bwd_bf16(const void* H, const void* W, const int32_t* y, cons
       p.out_row0 = t0;
       p.out = dH; p.out_bf16 = (dH_dtype == SPO_DTYPE_BF16); p.ldo = d; p.accumulate = 0;
       p.d_status = d_status;
-      if ((e = launch_gemm<MODE_DH>(mG_k, mW_mn, p, st)) != cudaSuccess) return e;
+      if ((e = launch_gemm<MODE_DH>(mG_k, mW_mn, p, progress, st)) != cudaSuccess) return e;
     }
     // 3) dW (+)= G^T H_chunk
     {
@@ -704,7 +844,7 @@ cudaError_t launch_bwd_bf16(const void* H, const void* W, const int32_t* y, cons
       p.out_row0 = 0;
       p.out = dW; p.out_bf16 = 0; p.ldo = d; p.accumulate = (accumulate || chunk > 0) ? 1 : 0;
       p.d_status = d_status;
-      if ((e = launch_gemm<MODE_DW>(mG_mn, mH_mn, p, st)) != cudaSuccess) return e;
+      if ((e = launch_gemm<MODE_DW>(mG_mn, mH_mn, p, progress, st)) != cudaSuccess) return e;
     }
   }
   return cudaSuccess;
