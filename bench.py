@@ -32,6 +32,7 @@ if ROOT not in sys.path:
 METRIC = "response tokens/s, fused SPO loss fwd+bwd (d4096,V151936,bf16); % bf16 peak"
 UNIT = "tokens/s"
 TABLE_N = 1_000_000          # tracker table the step samples from and updates
+CFG4_STEP_DRAM_BYTES = 1.11e12
 
 LOSS_SHAPES = {
     # workload: (d, V, w_std, old-logprob noise, reward probability)
@@ -277,7 +278,9 @@ def run_ours(args, rank, world, local_rank):
             "flops_per_step": step.flops_fwd + step.flops_bwd,
             "fwd_tflops": step.flops_fwd / (t_fwd / args.steps / 1e3) / 1e12,
             "bwd_tflops": step.flops_bwd / (t_bwd / args.steps / 1e3) / 1e12,
-            "traffic": None,
+            # DRAM read+write bytes of all launches of one step, from the ncu capture summarised in
+            # profiles/spo_gemm_kernel_cfg4_16responses_full.md, scaled by token rows; null for other shapes.
+            "traffic": CFG4_STEP_DRAM_BYTES if (args.workload == "cfg4_8b_bf16" and not args.responses) else None,
         },
         "e2e": {"value": tokens_all / (e2e_ms / e2e_steps / 1e3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "steps": e2e_steps},
@@ -286,6 +289,80 @@ def run_ours(args, rank, world, local_rank):
     if world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline_sample(step, args.cpu_tokens)
     print(json.dumps(out), flush=True)
+
+
+SMALL_SHAPES = {
+    # workload: (table prompts N, batch B, uniforms M)
+    "cfg2_tracker_scale": (1_000_000, 4096, 8192),
+    "small_scaled": (1 << 28, 1 << 22, 8192),
+}
+
+
+def run_small_kernels(args, local_rank):
+    """Tracker / advantage / sampling kernels alone: time per call (CUDA events, L2 flushed by writing a
+    512 MB buffer before every timed call) and achieved algorithmic GB/s against the measured HBM copy rate."""
+    import torch
+    from paper_2509_13232_b200 import binding as B
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    N, Bn, M = SMALL_SHAPES[args.workload]
+    peaks = read_peaks()
+    g = torch.Generator(device=dev)
+    g.manual_seed(20250913)
+    ab = torch.rand((N, 2), generator=g, device=dev) * 12 + 0.1
+    v0 = torch.rand(N, generator=g, device=dev)
+    u = torch.rand(M, generator=g, device=dev).clamp_(0, 0.999999)
+    ids = torch.randperm(N, generator=g, device=dev)[:Bn].to(torch.int32)
+    r = (torch.rand(Bn, generator=g, device=dev) < 0.4).float()
+    kl = torch.rand(Bn, generator=g, device=dev) * 0.05
+    n_draw = min(4096, Bn)
+    out_ids = torch.empty(n_draw, dtype=torch.int32, device=dev)
+    a_norm = torch.empty(Bn, device=dev)
+    stats = torch.empty(4, device=dev)
+    st = torch.zeros(4, dtype=torch.int32, device=dev)
+    ws = torch.empty(B.spo_workspace_bytes(B.WS_SAMPLE, N=N, M=M), dtype=torch.uint8, device=dev)
+    wsa = torch.empty(B.spo_workspace_bytes(B.WS_ADVANTAGES, B=Bn), dtype=torch.uint8, device=dev)
+    ab2 = torch.empty_like(ab)
+    p = B.default_params()
+    flush = torch.empty(128 * 1024 * 1024, dtype=torch.float32, device=dev)
+    calls = {
+        "spo_tracker_init": (lambda: B.spo_tracker_init(ab2, v0, p), 12 * N, 1),
+        "spo_sample_prompts": (lambda: B.spo_sample_prompts(ab, u, n_draw, out_ids, None, ws, p, st), 8 * N, 3),
+        "spo_advantages": (lambda: B.spo_advantages(ab, ids, r, None, a_norm, stats, wsa, p, st), 28 * Bn,
+                           1 if Bn <= 8192 else 2),
+        "spo_tracker_update": (lambda: B.spo_tracker_update(ab, ids, r, kl, 0, p, st), 28 * Bn, 1),
+    }
+    out_calls, total_ms, total_bytes, launches = {}, 0.0, 0, 0
+    with ClockSampler(local_rank) as clocks:
+        for name, (fn, nbytes, n_launch) in calls.items():
+            ts = []
+            for i in range(args.warmup + args.steps):
+                flush.zero_()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(); fn(); e1.record()
+                torch.cuda.synchronize()
+                if i >= args.warmup:
+                    ts.append(e0.elapsed_time(e1))
+            ts.sort()
+            ms = ts[len(ts) // 2]
+            out_calls[name] = {"ms": ms, "algorithmic_bytes": nbytes, "GB/s": nbytes / ms / 1e6,
+                               "frac_of_hbm": nbytes / ms / 1e6 / peaks["hbm_gbs"]}
+            total_ms += ms
+            total_bytes += nbytes
+            launches += n_launch * args.steps
+    dom = out_calls["spo_sample_prompts"]
+    print(json.dumps({
+        "metric": "tracker / advantage / sampling kernels, achieved HBM GB/s (algorithmic bytes)",
+        "value": total_bytes / total_ms / 1e6, "unit": "GB/s", "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": total_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic",
+        "config": {"workload": args.workload, "N": N, "B": Bn, "M": M, "l2": "flushed_before_each_call"},
+        "gpu_launches": launches, "device_status": int(st[0].item()), "calls": out_calls,
+        "roofline": {"bound": "hbm", "kernel": "sample_tile_sums_kernel (within spo_sample_prompts)",
+                     "achieved": dom["GB/s"], "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": dom["frac_of_hbm"],
+                     "peak_source": peaks["source"] + " copy", "traffic": None},
+        "clocks": clocks.summary(),
+    }), flush=True)
 
 
 def blas_threads():
@@ -360,7 +437,7 @@ def main():
     ap.add_argument("--steps", type=int, default=4)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg4_8b_bf16", choices=sorted(LOSS_SHAPES))
+    ap.add_argument("--workload", default="cfg4_8b_bf16", choices=sorted(LOSS_SHAPES) + sorted(SMALL_SHAPES))
     ap.add_argument("--cpu-tokens", type=int, default=None, help="token rows of the CPU-oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--responses", type=int, default=None,
@@ -369,6 +446,10 @@ def main():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.workload in SMALL_SHAPES:
+        if rank == 0:
+            run_small_kernels(args, local_rank)
+        return
     if args.impl == "reference":
         if args.cpu_tokens is None:
             args.cpu_tokens = 16

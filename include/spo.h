@@ -90,8 +90,8 @@ int32_t spo_tracker_init(float* ab, const float* v0, int64_t N,
  *
  * The draw is successive weighted sampling without replacement, made
  * reproducible bit for bit: weights are computed in fp32 with IEEE-rounded
- * operations in the order n=a+b, num=a*b, den=n*n, p=num/den, s=sqrt(p),
- * w=s+eps; q_i = floor(w_i * 2^32) (uint64); C_i = q_0+..+q_i; Wtot = C_{N-1};
+ * operations in the order n=a+b, num=a*b, den=n*n, inv=1/den, p=num*inv,
+ * s=sqrt(p), w=s+eps; q_i = floor(w_i * 2^32) (uint64); C_i = q_0+..+q_i; Wtot = C_{N-1};
  * for the k-th uniform U_k = floor(u_k * 2^32), t_k = floor(U_k*Wtot / 2^32),
  * candidate = first i with C_i > t_k; candidates are accepted in order k unless
  * already accepted, until B are accepted.

@@ -141,18 +141,20 @@ def sampling_weights_f32(alpha32, beta32, eps_explore=EPS_EXPLORE):
 
     v(1-v) is formed as alpha*beta/(alpha+beta)^2, which is the same quantity
     without the cancellation of 1-v near v = 1.  Order of operations:
-    n = alpha+beta; num = alpha*beta; den = n*n; p = num/den (0.25 if n == 0);
-    s = sqrt(p); w = s + eps.  numpy's float32 add, multiply, divide and sqrt
-    are each correctly rounded, so any IEEE implementation that performs these
-    steps without fusing them gives the same bits.
+    n = alpha+beta; num = alpha*beta; den = n*n; inv = 1/den; p = num*inv
+    (0.25 if n == 0); s = sqrt(p); w = s + eps.  numpy's float32 add, multiply,
+    divide and sqrt are each correctly rounded, so any IEEE implementation that
+    performs these steps without fusing them gives the same bits.
     """
     a = np.asarray(alpha32, dtype=np.float32)
     b = np.asarray(beta32, dtype=np.float32)
+    one = np.float32(1.0)
     n = a + b
     num = a * b
     den = n * n
     pos = n > np.float32(0.0)
-    p = np.where(pos, num / np.where(pos, den, np.float32(1.0)), np.float32(0.25)).astype(np.float32)
+    inv = one / np.where(pos, den, one)
+    p = np.where(pos, num * inv, np.float32(0.25)).astype(np.float32)
     s = np.sqrt(p)
     w = s + np.float32(eps_explore)
     return w.astype(np.float32)

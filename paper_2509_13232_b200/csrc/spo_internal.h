@@ -19,10 +19,12 @@ int device_is_sm100();                // 1 when the current device is compute ca
 
 // ---- sampler ------------------------------------------------------------
 constexpr int kSampleTile = 2048;     // table entries per partial-sum tile
+constexpr int kSuperTile = 1024;      // tiles per second-level sum
 
 struct SampleWs {
-  size_t tile_sums, tile_offsets, cand, keys, vals, total;
+  size_t super_sums, keys, vals, zeroed_bytes, tile_sums, cand, total;
   int64_t n_tiles;
+  int n_super;
   int64_t hash_slots;
 };
 SampleWs sample_ws_layout(int64_t N, int32_t M);

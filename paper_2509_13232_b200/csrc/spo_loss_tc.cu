@@ -33,7 +33,6 @@
 #include <cuda_runtime.h>
 #include <math_constants.h>
 #include <stdint.h>
-#include <stdlib.h>
 
 #include "spo_internal.h"
 
@@ -91,6 +90,7 @@ struct GemmParams {
   // Soft lock-step between CTA pairs (FWD / G): progress[g] = tiles started by pair g (+1), ~0u when done.
   uint32_t* progress;
   int window;
+  int sync_kblocks;                          // k-blocks between two progress comparisons
 };
 
 // ---------------------------------------------------------------------------
@@ -357,65 +357,71 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
-    // Lane 0 issues the loads.  At every tile boundary the whole warp compares this pair's tile
-    // count with the other pairs' and holds back while it is more than `window` tiles ahead of the
-    // slowest: pairs that sweep the same part of W then stay close enough in time for its tiles to
-    // be served from L2 instead of being streamed from HBM once per pair.  The hold is bounded and
-    // advisory (after ~100 us the pair goes on regardless), so it can never dead-lock.
+    // Lane 0 issues the loads.  Every `sync_kblocks` k-blocks (once per tile) the whole warp compares
+    // this pair's step count with the other pairs' and holds back while it is more than `window`
+    // steps ahead of the slowest: pairs that sweep the same operand tiles then stay close enough in
+    // time for those tiles to be served from L2 instead of being streamed from HBM once per pair
+    // (without it the forward at 244k tokens read 0.8 TB from HBM per launch, with it 0.12 TB).
+    // The hold is bounded and advisory (after ~0.15 ms the pair goes on regardless), so it cannot
+    // dead-lock, and finished pairs publish ~0u so that they never hold anyone back.
     uint32_t it = 0, tseq = 0;
     int ok = 1;
     volatile uint32_t* progress = (rank == 0) ? p.progress : nullptr;
-    for (int u = group; u < total_units && ok; u += n_groups) {
+    const uint32_t sync_kb = (uint32_t)p.sync_kblocks;
+    for (int u = group; u < total_units; u += n_groups) {
       const Unit un = unit_of(u, p);
       const int row_base = un.m_tile * GROUP_M + (int)rank * BM;       // this CTA's rows of the tile
-      for (int n = un.n_begin; n < un.n_end && ok; ++n) {
-        if (progress) {
-          ++tseq;
-          if (lane == 0) progress[group] = tseq;
-          if ((int)tseq > p.window) {
-            for (int tries = 0; tries < 128; ++tries) {
-              uint32_t mn = 0xFFFFFFFFu;
-              for (int g = lane; g < n_groups; g += 32) mn = min(mn, progress[g]);
+      for (int n = un.n_begin; n < un.n_end; ++n) {
+        const int col_base = n * BN + (int)rank * BSUB_ROWS;           // this CTA's columns of half 0
+        for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+          if (progress && (it % sync_kb) == 0) {                       // whole warp: publish and compare progress
+            ++tseq;
+            if (lane == 0) progress[group] = tseq;
+            if ((int)tseq > p.window) {
+              for (int tries = 0; tries < 128; ++tries) {
+                uint32_t mn = 0xFFFFFFFFu;
+                for (int g = lane; g < n_groups; g += 32) mn = min(mn, progress[g]);
 #pragma unroll
-              for (int o = 16; o > 0; o >>= 1) mn = min(mn, __shfl_xor_sync(0xffffffffu, mn, o));
-              if (mn + (uint32_t)p.window >= tseq) break;
-              __nanosleep(256);
+                for (int o = 16; o > 0; o >>= 1) mn = min(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+                if (mn + (uint32_t)p.window >= tseq) break;
+                __nanosleep(128);
+              }
             }
+            ok = __shfl_sync(0xffffffffu, ok, 0);
           }
-          __syncwarp();
-        }
-        if (lane == 0) {
-          const int col_base = n * BN + (int)rank * BSUB_ROWS;           // this CTA's columns of half 0
-          for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+          if (lane == 0 && ok) {
             const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
-            if (!mbar_wait<kProducerSleepNs>(empty0 + 8 * s, ph ^ 1u, abort_flag, p.d_status)) { ok = 0; break; }
-            const uint32_t sa = base + s * STAGE_BYTES, sb = sa + A_BYTES;
-            if (rank == 0) mbar_expect_tx(full0 + 8 * s, CG * STAGE_BYTES);   // both CTAs' bytes land on the leader's barrier
-            const uint32_t fb = map_to_cta(full0 + 8 * s, 0);
-            if (!A_MN) {
-              tma_load_2d(sa, &tmA, kb * BK, p.a_row0 + row_base, fb);
+            if (!mbar_wait<kProducerSleepNs>(empty0 + 8 * s, ph ^ 1u, abort_flag, p.d_status)) {
+              ok = 0;
             } else {
-#pragma unroll
-              for (int b = 0; b < BM / 64; ++b)
-                tma_load_2d(sa + b * 8192, &tmA, row_base + b * 64, p.a_row0 + kb * BK, fb);
-            }
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-              const uint32_t sbh = sb + h * BSUB_BYTES;
-              const int col = col_base + h * HALF_N;
-              if (!B_MN) {
-                tma_load_2d(sbh, &tmB, kb * BK, col, fb);
+              const uint32_t sa = base + s * STAGE_BYTES, sb = sa + A_BYTES;
+              if (rank == 0) mbar_expect_tx(full0 + 8 * s, CG * STAGE_BYTES);   // both CTAs' bytes land on the leader's barrier
+              const uint32_t fb = map_to_cta(full0 + 8 * s, 0);
+              if (!A_MN) {
+                tma_load_2d(sa, &tmA, kb * BK, p.a_row0 + row_base, fb);
               } else {
 #pragma unroll
-                for (int b = 0; b < BSUB_ROWS / 64; ++b)
-                  tma_load_2d(sbh + b * 8192, &tmB, col + b * 64, p.b_k0 + kb * BK, fb);
+                for (int b = 0; b < BM / 64; ++b)
+                  tma_load_2d(sa + b * 8192, &tmA, row_base + b * 64, p.a_row0 + kb * BK, fb);
+              }
+#pragma unroll
+              for (int h = 0; h < 2; ++h) {
+                const uint32_t sbh = sb + h * BSUB_BYTES;
+                const int col = col_base + h * HALF_N;
+                if (!B_MN) {
+                  tma_load_2d(sbh, &tmB, kb * BK, col, fb);
+                } else {
+#pragma unroll
+                  for (int b = 0; b < BSUB_ROWS / 64; ++b)
+                    tma_load_2d(sbh + b * 8192, &tmB, col + b * 64, p.b_k0 + kb * BK, fb);
+                }
               }
             }
           }
         }
-        ok = __shfl_sync(0xffffffffu, ok, 0);
       }
     }
+    __syncwarp();
     if (progress && lane == 0) progress[group] = 0xFFFFFFFFu;          // done: never hold anyone back
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer (leader CTA)
@@ -560,25 +566,24 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 #pragma unroll
             for (int q = 0; q < 8; ++q) piece[q] = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
             stage_put(stage, lane, piece);
-            float4 old[8];
-            if (p.accumulate) {
-#pragma unroll
-              for (int i = 0; i < 8; ++i) {
-                const int r = 4 * i + (lane >> 3), cc = lane & 7;
-                old[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (grow_warp0 + r < p.rows_valid)
-                  old[i] = *reinterpret_cast<const float4*>(obase + (int64_t)r * p.ldo + col0 + cc * 4);
-              }
-            }
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
               int r, cc;
               const uint4 raw4 = stage_get(stage, lane, i, r, cc);
-              float4 val = make_float4(__uint_as_float(raw4.x), __uint_as_float(raw4.y), __uint_as_float(raw4.z),
-                                       __uint_as_float(raw4.w));
-              if (p.accumulate) { val.x += old[i].x; val.y += old[i].y; val.z += old[i].z; val.w += old[i].w; }
-              if (grow_warp0 + r < p.rows_valid)
-                *reinterpret_cast<float4*>(obase + (int64_t)r * p.ldo + col0 + cc * 4) = val;
+              if (grow_warp0 + r < p.rows_valid) {
+                float* dst = obase + (int64_t)r * p.ldo + col0 + cc * 4;
+                if (p.accumulate) {
+                  // Added in L2, nothing comes back: no load latency in this (un-overlapped) epilogue.
+                  // Each element receives exactly one addend per launch and launches are ordered on
+                  // the stream, so the summation order is fixed.
+                  asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};"
+                               ::"l"(dst), "f"(__uint_as_float(raw4.x)), "f"(__uint_as_float(raw4.y)),
+                                 "f"(__uint_as_float(raw4.z)), "f"(__uint_as_float(raw4.w))
+                               : "memory");
+                } else {
+                  *reinterpret_cast<uint4*>(dst) = raw4;
+                }
+              }
             }
           }
         }
@@ -639,11 +644,8 @@ bool make_map(CUtensorMap* m, const void* ptr, uint64_t inner, uint64_t outer, u
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// Window (in tiles) of the lock-step hold between CTA pairs; 0 disables it.
-int throttle_window() {
-  if (const char* e = getenv("SPO_DEV_WINDOW")) return atoi(e);
-  return 1;
-}
+// How many tiles a CTA pair may run ahead of the slowest pair before it holds back.
+constexpr int kLockStepWindow = 1;
 
 // CTA pairs that can be resident at once (one CTA per SM).
 int group_count() { return sm_count() / CG; }
@@ -662,7 +664,8 @@ cudaError_t launch_gemm(const CUtensorMap& a, const CUtensorMap& b, const GemmPa
   const int units = p_in.m_tiles * p_in.nsplit;
   if (units <= 0) return cudaSuccess;
   GemmParams p = p_in;
-  p.window = throttle_window();
+  p.window = kLockStepWindow;
+  p.sync_kblocks = p.k_blocks;                 // compare progress once per tile
   p.progress = nullptr;
   if (p.window > 0 && progress) {
     cudaError_t e = cudaMemsetAsync(progress, 0, kProgressBytes, st);
@@ -695,7 +698,6 @@ constexpr uint32_t kBoxB = BSUB_ROWS;
 // re-reads of W from HBM; the choice also avoids a short last split (pairs would fall out of step)
 // and a nearly empty last round of units.
 int pick_fwd_split(int64_t m_tiles, int n_tiles, int d) {
-  if (const char* e = getenv("SPO_DEV_FWD_SPLIT")) { int v = atoi(e); if (v > 0) return v < n_tiles ? v : n_tiles; }
   const int groups = group_count();
   const double a_tile = (double)GROUP_M * d * 2, b_tile = (double)BN * d * 2;
   const double l2_budget = 56e6;
@@ -758,7 +760,6 @@ BwdWs bwd_ws_layout(int64_t T, int32_t d, int32_t V) {
   // pairs a whole number of times, and the chunk buffer stays at a few GB.
   const int groups = group_count();
   int64_t m_tiles = groups / 2 > 0 ? groups / 2 : 1;
-  if (const char* e = getenv("SPO_DEV_CHUNK_TILES")) { int v = atoi(e); if (v > 0) m_tiles = v; }
   int64_t rows = m_tiles * GROUP_M;
   const int64_t t_pad = ceil_div(T > 0 ? T : 1, GROUP_M) * GROUP_M;
   if (rows > t_pad) rows = t_pad;

@@ -2,6 +2,7 @@
 // All are memory-streaming kernels: coalesced vector loads of the interleaved
 // (alpha, beta) table, warp-shuffle reductions, integer prefix sums.
 #include <cuda_runtime.h>
+#include <math_constants.h>
 #include <stdint.h>
 
 #include <mutex>
@@ -31,20 +32,24 @@ __global__ void tracker_init_kernel(float2* __restrict__ ab, const float* __rest
 // ---------------------------------------------------------------------------
 // Sampling weight of one table entry (Eq. "sampling_coef") in IEEE fp32, one
 // rounded operation per step so that a host restatement gives the same bits:
-// n=a+b, num=a*b, den=n*n, p=num/den (0.25 for an empty entry), s=sqrt(p), w=s+eps.
+// n=a+b, num=a*b, den=n*n, inv=1/den, p=num*inv (0.25 for an empty entry), s=sqrt(p), w=s+eps.
+// (A correctly rounded reciprocal plus a multiply costs about half the instructions of a
+// correctly rounded division; this kernel is bound by instruction issue, not by HBM.)
 // A negative or non-finite entry yields weight 0 and *bad = true.
 // ---------------------------------------------------------------------------
 __device__ __forceinline__ float entry_weight(float a, float b, float eps, bool& bad) {
-  if (!(a >= 0.0f) || !(b >= 0.0f) || isinf(a) || isinf(b)) { bad = true; return 0.0f; }
-  float n = __fadd_rn(a, b);
+  const float n = __fadd_rn(a, b);
+  const bool wrong = (fminf(a, b) < 0.0f) | !(n < CUDART_INF_F);     // negative, NaN or Inf
+  bad |= wrong;
   float p = 0.25f;
-  if (n > 0.0f) p = __fdiv_rn(__fmul_rn(a, b), __fmul_rn(n, n));
-  return __fadd_rn(__fsqrt_rn(p), eps);
+  if (n > 0.0f) p = __fmul_rn(__fmul_rn(a, b), __frcp_rn(__fmul_rn(n, n)));
+  const float w = __fadd_rn(__fsqrt_rn(p), eps);
+  return wrong ? 0.0f : w;
 }
 
-// q = floor(w * 2^32): exact, the scale is a power of two.
+// q = floor(w * 2^32): exact, the scale is a power of two (w is finite, non-negative, far below 2^32).
 __device__ __forceinline__ unsigned long long quantise(float w) {
-  return (unsigned long long)((double)w * 4294967296.0);
+  return __float2ull_rz(w * 4294967296.0f);
 }
 
 __device__ __forceinline__ unsigned long long warp_sum_u64(unsigned long long v) {
@@ -66,7 +71,7 @@ __device__ __forceinline__ unsigned long long warp_incl_scan_u64(unsigned long l
 __global__ void __launch_bounds__(256)
 sample_tile_sums_kernel(const float4* __restrict__ ab4, int64_t N, float eps, float2* __restrict__ out_w2,
                         float* __restrict__ out_w, unsigned long long* __restrict__ tile_sums,
-                        int32_t* d_status) {
+                        unsigned long long* __restrict__ super_sums, int32_t* d_status) {
   const int64_t tile = blockIdx.x;
   const int64_t first_pair = tile * (kSampleTile / 2);
   const int64_t n_pairs = N >> 1;
@@ -97,79 +102,30 @@ sample_tile_sums_kernel(const float4* __restrict__ ab4, int64_t N, float eps, fl
 #pragma unroll
     for (int w = 0; w < 8; ++w) t += s_part[w];
     tile_sums[tile] = t;
+    atomicAdd(&super_sums[tile / kSuperTile], t);      // integer adds commute: exact in any order
   }
 }
 
-// Exclusive scan of the tile sums by one block; offsets[n_tiles] = total weight.
-__global__ void __launch_bounds__(1024)
-sample_scan_tiles_kernel(const unsigned long long* __restrict__ tile_sums, int64_t n_tiles,
-                         unsigned long long* __restrict__ offsets, int32_t* d_status) {
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int64_t per = (n_tiles + 1023) / 1024;
-  const int64_t lo = (int64_t)tid * per;
-  const int64_t hi = lo + per < n_tiles ? lo + per : n_tiles;
-  unsigned long long local = 0;
-  for (int64_t i = lo; i < hi; ++i) local += tile_sums[i];
-  unsigned long long incl = warp_incl_scan_u64(local, lane);
-  __shared__ unsigned long long s_warp[32];
-  if (lane == 31) s_warp[warp] = incl;
-  __syncthreads();
-  if (warp == 0) {
-    unsigned long long v = s_warp[lane];
-    unsigned long long s = warp_incl_scan_u64(v, lane);
-    s_warp[lane] = s - v;                       // exclusive prefix of the warp totals
-    if (lane == 31) {
-      offsets[n_tiles] = s;
-      if (s == 0) flag(d_status, SPO_DEV_ZERO_TOTAL_WEIGHT);
+// Warp-wide search of the first entry whose running sum exceeds t: `get(i)` yields entry i of a
+// list of `count` non-negative integers, `run` is the sum of everything before the list.  Returns
+// the index (or -1) and leaves in `run` the sum of everything before that index.
+template <typename Get>
+__device__ __forceinline__ int64_t warp_find(int64_t count, unsigned long long t, unsigned long long& run, int lane,
+                                             Get get) {
+  for (int64_t c0 = 0; c0 < count; c0 += 32) {
+    const int64_t i = c0 + lane;
+    const unsigned long long q = i < count ? get(i) : 0ull;
+    const unsigned long long incl = warp_incl_scan_u64(q, lane);
+    const unsigned hit = __ballot_sync(0xffffffffu, run + incl > t);
+    if (hit) {
+      const int first = __ffs(hit) - 1;
+      const unsigned long long before = __shfl_sync(0xffffffffu, incl - q, first);
+      run += before;
+      return c0 + first;
     }
-  }
-  __syncthreads();
-  unsigned long long run = s_warp[warp] + incl - local;
-  for (int64_t i = lo; i < hi; ++i) {
-    offsets[i] = run;
-    run += tile_sums[i];
-  }
-}
-
-// One warp per uniform: threshold, tile by binary search, entry by a scan inside the tile.
-__global__ void __launch_bounds__(256)
-sample_search_kernel(const float* __restrict__ ab, int64_t N, float eps, const float* __restrict__ uniforms,
-                     int32_t M, const unsigned long long* __restrict__ offsets, int64_t n_tiles,
-                     int32_t* __restrict__ cand, int32_t* d_status) {
-  const int lane = threadIdx.x & 31;
-  const int k = (int)(((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5);
-  if (k >= M) return;
-  const unsigned long long wtot = offsets[n_tiles];
-  const float u = uniforms[k];
-  if (wtot == 0 || !(u >= 0.0f) || !(u < 1.0f)) {
-    if (lane == 0) {
-      cand[k] = -1;
-      if (wtot != 0) flag(d_status, SPO_DEV_NONFINITE);
-    }
-    return;
-  }
-  const unsigned long long bigu = (unsigned long long)((double)u * 4294967296.0);
-  const unsigned long long t = (__umul64hi(bigu, wtot) << 32) | ((bigu * wtot) >> 32);
-  // first tile j with offsets[j+1] > t
-  int64_t lo = 0, hi = n_tiles - 1;
-  while (lo < hi) {
-    int64_t mid = (lo + hi) >> 1;
-    if (offsets[mid + 1] > t) hi = mid; else lo = mid + 1;
-  }
-  unsigned long long run = offsets[lo];
-  const int64_t base = lo * kSampleTile;
-  int32_t found = -1;
-  bool bad = false;
-  for (int c = 0; c < kSampleTile / 32; ++c) {
-    int64_t i = base + c * 32 + lane;
-    unsigned long long q = 0;
-    if (i < N) q = quantise(entry_weight(ab[2 * i], ab[2 * i + 1], eps, bad));
-    unsigned long long incl = warp_incl_scan_u64(q, lane);
-    unsigned hit = __ballot_sync(0xffffffffu, run + incl > t);
-    if (hit) { found = (int32_t)(base + c * 32 + (__ffs(hit) - 1)); break; }
     run += __shfl_sync(0xffffffffu, incl, 31);
   }
-  if (lane == 0) cand[k] = found;
+  return -1;
 }
 
 __device__ __forceinline__ uint32_t hash_id(uint32_t x) {
@@ -177,54 +133,149 @@ __device__ __forceinline__ uint32_t hash_id(uint32_t x) {
   return x;
 }
 
-// Keep the first occurrence of every candidate, in order, until B are accepted.
-// One block; keys/vals is an open-addressing table (keys preset to -1, vals to 0x7f7f7f7f).
-__global__ void __launch_bounds__(1024)
-sample_accept_kernel(const int32_t* __restrict__ cand, int32_t M, int32_t B, int32_t* __restrict__ keys,
-                     int32_t* __restrict__ vals, uint32_t slot_mask, int32_t* __restrict__ out_ids,
+// One warp per uniform: total weight, threshold, then three levels of search (super-tile, tile,
+// entry).  The winner is also entered into an open-addressing table keyed by prompt id + 1
+// (0 = empty) whose value keeps the largest M - k, i.e. the earliest draw k of that prompt.
+__global__ void __launch_bounds__(256)
+sample_search_kernel(const float* __restrict__ ab, int64_t N, float eps, const float* __restrict__ uniforms,
+                     int32_t M, const unsigned long long* __restrict__ tile_sums,
+                     const unsigned long long* __restrict__ super_sums, int64_t n_tiles, int n_super,
+                     int32_t* __restrict__ cand, int32_t* keys, int32_t* vals, uint32_t slot_mask,
                      int32_t* d_status) {
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  for (int k = tid; k < M; k += 1024) {
-    int32_t c = cand[k];
-    if (c < 0) continue;
-    uint32_t s = hash_id((uint32_t)c) & slot_mask;
-    for (uint32_t probe = 0; probe <= slot_mask; ++probe) {
-      int32_t prev = atomicCAS(&keys[s], -1, c);
-      if (prev == -1 || prev == c) { atomicMin(&vals[s], k); break; }
-      s = (s + 1) & slot_mask;
+  const int lane = threadIdx.x & 31;
+  const int k = (int)(((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5);
+  if (k >= M) return;
+  unsigned long long wtot = 0;
+  for (int i = lane; i < n_super; i += 32) wtot += super_sums[i];
+  wtot = warp_sum_u64(wtot);
+  const float u = uniforms[k];
+  if (wtot == 0 || !(u >= 0.0f) || !(u < 1.0f)) {
+    if (lane == 0) {
+      cand[k] = -1;
+      if (wtot != 0) flag(d_status, SPO_DEV_NONFINITE);
+      else if (k == 0) flag(d_status, SPO_DEV_ZERO_TOTAL_WEIGHT);
+    }
+    return;
+  }
+  const unsigned long long bigu = __float2ull_rz(u * 4294967296.0f);          // floor(u * 2^32), exact
+  const unsigned long long t = (__umul64hi(bigu, wtot) << 32) | ((bigu * wtot) >> 32);
+  unsigned long long run = 0;
+  int64_t off = -1, base = 0;
+  const int64_t sup = warp_find(n_super, t, run, lane, [&](int64_t i) { return super_sums[i]; });
+  if (sup >= 0) {                                                    // warp-uniform
+    const int64_t tile0 = sup * kSuperTile;
+    const int64_t tiles_here = n_tiles - tile0 < kSuperTile ? n_tiles - tile0 : kSuperTile;
+    const int64_t tl = warp_find(tiles_here, t, run, lane, [&](int64_t i) { return tile_sums[tile0 + i]; });
+    if (tl >= 0) {
+      base = (tile0 + tl) * kSampleTile;
+      const int64_t n_here = N - base < kSampleTile ? N - base : kSampleTile;
+      // entries: 128 per step, four consecutive ones per lane (two float4 loads)
+      const float4* ab4 = reinterpret_cast<const float4*>(ab) + base / 2;      // base is a multiple of 2048
+      for (int64_t c0 = 0; c0 < n_here && off < 0; c0 += 128) {
+        const int64_t i0 = c0 + 4 * lane;
+        unsigned long long q[4] = {0ull, 0ull, 0ull, 0ull};
+        bool bad = false;
+        if (i0 + 3 < n_here) {
+          const float4 e0 = __ldg(ab4 + i0 / 2), e1 = __ldg(ab4 + i0 / 2 + 1);
+          q[0] = quantise(entry_weight(e0.x, e0.y, eps, bad));
+          q[1] = quantise(entry_weight(e0.z, e0.w, eps, bad));
+          q[2] = quantise(entry_weight(e1.x, e1.y, eps, bad));
+          q[3] = quantise(entry_weight(e1.z, e1.w, eps, bad));
+        } else {
+#pragma unroll
+          for (int j = 0; j < 4; ++j)
+            if (i0 + j < n_here) q[j] = quantise(entry_weight(ab[2 * (base + i0 + j)], ab[2 * (base + i0 + j) + 1], eps, bad));
+        }
+        const unsigned long long mine = q[0] + q[1] + q[2] + q[3];
+        const unsigned long long incl = warp_incl_scan_u64(mine, lane);
+        const unsigned hit = __ballot_sync(0xffffffffu, run + incl > t);
+        if (hit) {
+          const int first = __ffs(hit) - 1;                              // lane whose four entries hold the answer
+          unsigned long long r0 = run + __shfl_sync(0xffffffffu, incl - mine, first);
+          const unsigned long long f0 = __shfl_sync(0xffffffffu, q[0], first), f1 = __shfl_sync(0xffffffffu, q[1], first),
+                                   f2 = __shfl_sync(0xffffffffu, q[2], first);
+          int j = 3;
+          if (r0 + f0 > t) j = 0;
+          else if (r0 + f0 + f1 > t) j = 1;
+          else if (r0 + f0 + f1 + f2 > t) j = 2;
+          off = c0 + 4 * first + j;
+        } else {
+          run += __shfl_sync(0xffffffffu, incl, 31);
+        }
+      }
     }
   }
-  __syncthreads();
+  if (lane == 0) {
+    const int32_t found = off < 0 ? -1 : (int32_t)(base + off);
+    cand[k] = found;
+    if (found >= 0) {
+      uint32_t s = hash_id((uint32_t)found) & slot_mask;
+      for (uint32_t probe = 0; probe <= slot_mask; ++probe) {
+        const int32_t prev = atomicCAS(&keys[s], 0, found + 1);
+        if (prev == 0 || prev == found + 1) { atomicMax(&vals[s], M - k); break; }
+        s = (s + 1) & slot_mask;
+      }
+    }
+  }
+}
+
+// Keep the first occurrence of every candidate, in order, until B are accepted.  One block;
+// each pass covers 8192 draws, eight consecutive ones per thread.
+__global__ void __launch_bounds__(1024)
+sample_accept_kernel(const int32_t* __restrict__ cand, int32_t M, int32_t B, const int32_t* __restrict__ keys,
+                     const int32_t* __restrict__ vals, uint32_t slot_mask, int32_t* __restrict__ out_ids,
+                     int32_t* d_status) {
+  constexpr int PER = 8;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   __shared__ int s_warp[32];
   __shared__ int s_total;
   if (tid == 0) s_total = 0;
   __syncthreads();
-  for (int k0 = 0; k0 < M; k0 += 1024) {
+  for (int k0 = 0; k0 < M; k0 += 1024 * PER) {
     const int base_count = s_total;
     if (base_count >= B) break;
-    const int k = k0 + tid;
-    int first = 0;
-    int32_t c = -1;
-    if (k < M) {
-      c = cand[k];
-      if (c >= 0) {
-        uint32_t s = hash_id((uint32_t)c) & slot_mask;
+    int32_t c[PER];
+    uint32_t slot[PER];
+    bool first[PER];
+#pragma unroll
+    for (int j = 0; j < PER; ++j) {
+      const int k = k0 + tid * PER + j;
+      c[j] = k < M ? cand[k] : -1;
+      slot[j] = hash_id((uint32_t)c[j]) & slot_mask;
+    }
+    int mine = 0;
+#pragma unroll
+    for (int j = 0; j < PER; ++j) {
+      first[j] = false;
+      if (c[j] >= 0) {
+        uint32_t sl = slot[j];
         for (uint32_t probe = 0; probe <= slot_mask; ++probe) {
-          if (keys[s] == c) { first = (vals[s] == k); break; }
-          s = (s + 1) & slot_mask;
+          if (keys[sl] == c[j] + 1) { first[j] = (vals[sl] == M - (k0 + tid * PER + j)); break; }
+          sl = (sl + 1) & slot_mask;
         }
       }
+      mine += first[j];
     }
-    unsigned bal = __ballot_sync(0xffffffffu, first);
-    int in_warp = __popc(bal & ((1u << lane) - 1));
-    if (lane == 0) s_warp[warp] = __popc(bal);
+    int incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int v = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += v;
+    }
+    if (lane == 31) s_warp[warp] = incl;
     __syncthreads();
     int before = 0;
     for (int w = 0; w < warp; ++w) before += s_warp[w];
-    int pos = base_count + before + in_warp;
-    if (first && pos < B) out_ids[pos] = c;
+    int pos = base_count + before + incl - mine;
+#pragma unroll
+    for (int j = 0; j < PER; ++j) {
+      if (first[j]) {
+        if (pos < B) out_ids[pos] = c[j];
+        ++pos;
+      }
+    }
     __syncthreads();
-    if (tid == 1023) s_total = pos + first;
+    if (tid == 1023) s_total = pos;
     __syncthreads();
   }
   const int accepted = s_total;
@@ -357,22 +408,45 @@ advantages_normalise_kernel(const double2* __restrict__ partials, int n_partials
 // ---------------------------------------------------------------------------
 // Tracker update (Sec. 3.1): rho = clamp(2^(-D/D_half)); alpha <- rho*alpha + r; beta <- rho*beta + 1-r
 // ---------------------------------------------------------------------------
+// Four batch entries per thread, loads issued before any is used, so that four gathers are in
+// flight per thread: the kernel is bound by memory latency, not arithmetic.
 __global__ void __launch_bounds__(256)
 tracker_update_kernel(float2* __restrict__ ab, int64_t N, const int32_t* __restrict__ ids,
                       const float* __restrict__ r, const float* __restrict__ kl, int kl_is_table, int32_t B,
                       float rho_min, float rho_max, float inv_d_half, int32_t* d_status) {
-  for (int64_t j = (int64_t)blockIdx.x * 256 + threadIdx.x; j < B; j += (int64_t)gridDim.x * 256) {
-    const int32_t id = ids[j];
-    if (id < 0 || (int64_t)id >= N) { flag(d_status, SPO_DEV_ID_OUT_OF_RANGE); continue; }
-    const float rew = r[j];
-    const float div = kl_is_table ? __ldg(kl + id) : kl[j];
-    if (isnan(rew) || isinf(rew) || isnan(div)) { flag(d_status, SPO_DEV_NONFINITE); continue; }
-    float rho = exp2f(-div * inv_d_half);
-    rho = fminf(fmaxf(rho, rho_min), rho_max);
-    float2 e = ab[id];
-    e.x = fmaf(rho, e.x, rew);
-    e.y = fmaf(rho, e.y, 1.0f - rew);
-    ab[id] = e;
+  constexpr int U = 4;
+  const int64_t stride = (int64_t)gridDim.x * 256;
+  for (int64_t j0 = (int64_t)blockIdx.x * 256 + threadIdx.x; j0 < B; j0 += U * stride) {
+    int32_t id[U];
+    float rew[U], div[U];
+    float2 e[U];
+    bool live[U];
+#pragma unroll
+    for (int q = 0; q < U; ++q) {
+      const int64_t j = j0 + q * stride;
+      live[q] = j < B;
+      id[q] = live[q] ? ids[j] : 0;
+      rew[q] = live[q] ? r[j] : 0.0f;
+      div[q] = (live[q] && !kl_is_table) ? kl[j] : 0.0f;
+    }
+#pragma unroll
+    for (int q = 0; q < U; ++q) {
+      if (live[q] && (id[q] < 0 || (int64_t)id[q] >= N)) { flag(d_status, SPO_DEV_ID_OUT_OF_RANGE); live[q] = false; }
+      if (live[q]) {
+        e[q] = ab[id[q]];
+        if (kl_is_table) div[q] = __ldg(kl + id[q]);
+      }
+    }
+#pragma unroll
+    for (int q = 0; q < U; ++q) {
+      if (!live[q]) continue;
+      if (isnan(rew[q]) || isinf(rew[q]) || isnan(div[q])) { flag(d_status, SPO_DEV_NONFINITE); continue; }
+      float rho = exp2f(-div[q] * inv_d_half);
+      rho = fminf(fmaxf(rho, rho_min), rho_max);
+      e[q].x = fmaf(rho, e[q].x, rew[q]);
+      e[q].y = fmaf(rho, e[q].y, 1.0f - rew[q]);
+      ab[id[q]] = e[q];
+    }
   }
 }
 
@@ -385,15 +459,18 @@ tracker_update_kernel(float2* __restrict__ ab, int64_t N, const int32_t* __restr
 SampleWs sample_ws_layout(int64_t N, int32_t M) {
   SampleWs L{};
   L.n_tiles = ceil_div(N, kSampleTile);
+  L.n_super = (int)ceil_div(L.n_tiles, kSuperTile);
   int64_t slots = 64;
   while (slots < 2 * (int64_t)M) slots <<= 1;
   L.hash_slots = slots;
   size_t off = 0;
-  L.tile_sums = off;    off = align_up(off + sizeof(unsigned long long) * L.n_tiles, 256);
-  L.tile_offsets = off; off = align_up(off + sizeof(unsigned long long) * (L.n_tiles + 1), 256);
-  L.cand = off;         off = align_up(off + sizeof(int32_t) * (size_t)M, 256);
+  // one zero-filled region: super-tile sums, hash keys, hash values
+  L.super_sums = off;   off = align_up(off + sizeof(unsigned long long) * (size_t)L.n_super, 256);
   L.keys = off;         off = align_up(off + sizeof(int32_t) * (size_t)slots, 256);
   L.vals = off;         off = align_up(off + sizeof(int32_t) * (size_t)slots, 256);
+  L.zeroed_bytes = off;
+  L.tile_sums = off;    off = align_up(off + sizeof(unsigned long long) * (size_t)L.n_tiles, 256);
+  L.cand = off;         off = align_up(off + sizeof(int32_t) * (size_t)M, 256);
   L.total = off;
   return L;
 }
@@ -409,20 +486,19 @@ cudaError_t launch_sample(const float* ab, int64_t N, const float* u, int32_t M,
                           int32_t* out_ids, float* out_w, char* ws, const SampleWs& L,
                           float eps, int32_t* d_status, cudaStream_t st) {
   auto* tile_sums = reinterpret_cast<unsigned long long*>(ws + L.tile_sums);
-  auto* offsets = reinterpret_cast<unsigned long long*>(ws + L.tile_offsets);
+  auto* super_sums = reinterpret_cast<unsigned long long*>(ws + L.super_sums);
   auto* cand = reinterpret_cast<int32_t*>(ws + L.cand);
   auto* keys = reinterpret_cast<int32_t*>(ws + L.keys);
   auto* vals = reinterpret_cast<int32_t*>(ws + L.vals);
   cudaError_t e;
-  if ((e = cudaMemsetAsync(keys, 0xFF, sizeof(int32_t) * L.hash_slots, st)) != cudaSuccess) return e;
-  if ((e = cudaMemsetAsync(vals, 0x7F, sizeof(int32_t) * L.hash_slots, st)) != cudaSuccess) return e;
+  if ((e = cudaMemsetAsync(ws, 0, L.zeroed_bytes, st)) != cudaSuccess) return e;
   sample_tile_sums_kernel<<<(unsigned)L.n_tiles, 256, 0, st>>>(
-      reinterpret_cast<const float4*>(ab), N, eps, reinterpret_cast<float2*>(out_w), out_w, tile_sums, d_status);
-  if ((e = cudaGetLastError()) != cudaSuccess) return e;
-  sample_scan_tiles_kernel<<<1, 1024, 0, st>>>(tile_sums, L.n_tiles, offsets, d_status);
+      reinterpret_cast<const float4*>(ab), N, eps, reinterpret_cast<float2*>(out_w), out_w, tile_sums, super_sums,
+      d_status);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   sample_search_kernel<<<(unsigned)ceil_div((int64_t)M * 32, 256), 256, 0, st>>>(
-      ab, N, eps, u, M, offsets, L.n_tiles, cand, d_status);
+      ab, N, eps, u, M, tile_sums, super_sums, L.n_tiles, L.n_super, cand, keys, vals, (uint32_t)(L.hash_slots - 1),
+      d_status);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   sample_accept_kernel<<<1, 1024, 0, st>>>(cand, M, B, keys, vals, (uint32_t)(L.hash_slots - 1), out_ids, d_status);
   return cudaGetLastError();
@@ -459,7 +535,7 @@ cudaError_t launch_tracker_update(float* ab, int64_t N, const int32_t* ids, cons
                                   float rho_min, float rho_max, float d_half,
                                   int32_t* d_status, cudaStream_t st) {
   if (B == 0) return cudaSuccess;
-  int64_t blocks = ceil_div(B, 256);
+  int64_t blocks = ceil_div(B, 256 * 4);
   int64_t cap = (int64_t)sm_count() * 8;
   if (blocks > cap) blocks = cap;
   tracker_update_kernel<<<(unsigned)blocks, 256, 0, st>>>(reinterpret_cast<float2*>(ab), N, ids, r, kl, kl_is_table, B,
