@@ -108,3 +108,71 @@ def test_bf16_uniform_logits_and_bad_target():
     got = run_loss(lb)
     assert got["status"] & 1
     assert np.isneginf(got["logp"][3]) and got["coef"][3] == 0.0
+
+
+def test_empty_batch_is_a_no_op_with_zero_loss():
+    """T = 0: loss 0, dW zeroed (or left alone when accumulating), nothing else touched."""
+    import torch
+    from paper_2509_13232_b200 import binding as B
+    from tests.helpers import status_word, ws_bytes
+    p = B.default_params()
+    for dt, d, v in ((torch.bfloat16, 64, 300), (torch.float32, 16, 40)):
+        H = torch.empty((0, d), dtype=dt, device="cuda")
+        W = torch.randn((v, d), device="cuda").to(dt)
+        z = lambda n, t=torch.float32: torch.zeros(max(n, 1), dtype=t, device="cuda")  # noqa: E731
+        loss = torch.full((4,), 7.0, device="cuda")
+        cu = torch.zeros(1, dtype=torch.int32, device="cuda")
+        st = status_word()
+        B.spo_loss_fwd(H, W, z(0, torch.int32), z(0), None, cu, z(0), loss, z(0), z(0), z(0), None,
+                       ws_bytes(B.WS_LOSS_FWD, T=0, d=d, V=v), p, st)
+        dW = torch.full((v, d), 3.0, device="cuda")
+        dH = torch.empty((0, d), dtype=dt, device="cuda")
+        B.spo_loss_bwd(H, W, z(0, torch.int32), z(0), z(0), 1.0, dH, dW, 0, ws_bytes(B.WS_LOSS_BWD, T=0, d=d, V=v), p, st)
+        torch.cuda.synchronize()
+        assert loss[0].item() == 0.0 and int(st[0].item()) == 0
+        if dt == torch.bfloat16:
+            assert float(dW.abs().max().item()) == 0.0
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+def test_all_tokens_masked_gives_zero_loss_and_zero_gradients(bf16):
+    lb = inputs.loss_batch(51, [20, 13], 64, 200, 0.05, bf16, 0.1)
+    lb.mask[:] = 0
+    got = run_loss(lb)
+    want = oracle_loss(lb)
+    assert want["loss"] == 0.0 and got["loss"] == 0.0 and got["status"] == 0
+    assert np.all(got["coef"] == 0.0) and np.all(got["dH"] == 0.0) and np.all(got["dW"] == 0.0)
+    np.testing.assert_allclose(got["logp"], want["logp"], rtol=0, atol=2e-3)
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+def test_single_token_and_empty_sequences(bf16):
+    """One token row; and responses of length zero in the middle of the batch."""
+    tol = (2e-3, 1e-2) if bf16 else (1e-4, 1e-4)
+    one = inputs.loss_batch(52, [1], 64, 130, 0.05, bf16, 0.1)
+    check(one, run_loss(one), oracle_loss(one), *tol)
+    gaps = inputs.loss_batch(53, [5, 0, 0, 9, 0, 3], 64, 130, 0.05, bf16, 0.3,
+                             a_norm=np.array([1.0, 9.0, -9.0, -0.7, 5.0, 0.4], dtype=np.float32))
+    got, want = run_loss(gaps), oracle_loss(gaps)
+    check(gaps, got, want, *tol)
+    np.testing.assert_array_equal(got["seq_sums"][[1, 2, 4]], 0.0)
+
+
+@pytest.mark.parametrize("v", [100, 512, 1024, 1025])
+def test_bf16_vocabulary_edges(v):
+    """Vocabulary below one tile, exactly one and two tiles, and one column over."""
+    lb = _clip_batch(60 + v, [70, 61], 64, v, True)
+    check(lb, run_loss(lb), oracle_loss(lb), 2e-3, 1e-2)
+
+
+def test_bf16_targets_on_tile_and_half_boundaries():
+    """Targets at the first/last column of accumulator halves and tiles are gathered correctly."""
+    lb = inputs.loss_batch(70, [64], 64, 1200, 0.05, True, 0.05, target="uniform")
+    edges = [0, 31, 32, 255, 256, 511, 512, 767, 768, 1023, 1024, 1199]
+    lb.y[:len(edges)] = edges
+    z = lb.h.astype(np.float64) @ lb.w.astype(np.float64).T
+    from scipy.special import log_softmax
+    lb.logp_old[:] = log_softmax(z, axis=1)[np.arange(64), lb.y].astype(np.float32)
+    got, want = run_loss(lb), oracle_loss(lb)
+    check(lb, got, want, 2e-3, 1e-2)
+    np.testing.assert_allclose(want["ratio"], 1.0, atol=1e-6)

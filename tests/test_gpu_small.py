@@ -204,3 +204,42 @@ def test_update_flags_bad_entries_and_leaves_them_untouched():
     np.testing.assert_array_equal(out[1:], ab[1:])
     a1, b1 = O.tracker_update([2.0], [2.0], [0], [1.0], [np.float64(np.float32(0.01))], float(np.float32(p.d_half)))
     np.testing.assert_allclose(out[0], [a1[0], b1[0]], rtol=RTOL)
+
+
+def test_sampling_single_prompt_table_and_full_draw():
+    p = B().default_params()
+    ids, w, st = gpu_sample(dev(np.array([[3.0, 1.0]], np.float32)), np.array([0.7, 0.2], np.float32), 1, p)
+    assert st == 0 and ids.tolist() == [0]
+    np.testing.assert_array_equal(w, O.sampling_weights_f32([3.0], [1.0], np.float32(p.eps_explore)))
+    # B = M = N: every uniform must land on a new prompt, else the call reports exhaustion
+    n = 8
+    ab = np.full((n, 2), 2.0, dtype=np.float32)
+    u = ((np.arange(n) + 0.5) / n).astype(np.float32)
+    ids, _, st = gpu_sample(dev(ab), u, n, p)
+    assert st == 0 and ids.tolist() == list(range(n))
+
+
+def test_sampling_flags_bad_table_entries_and_zero_total_weight():
+    p = B().default_params()
+    ab = np.array([[2.0, 2.0], [-1.0, 2.0], [np.nan, 1.0], [1.0, 3.0]], dtype=np.float32)
+    u = inputs.uniforms_f32(np.random.default_rng(3), 64)
+    ids, w, st = gpu_sample(dev(ab), u, 2, p)
+    assert st & B().DEV_NONFINITE
+    assert w[1] == 0.0 and w[2] == 0.0 and set(ids.tolist()) == {0, 3}
+    p0 = B().default_params(eps_explore=0.0)
+    dead = np.array([[0.0, 5.0], [4.0, 0.0]], dtype=np.float32)      # v = 0 and v = 1: weight eps = 0
+    ids, _, st = gpu_sample(dev(dead), u, 1, p0)
+    assert st & B().DEV_ZERO_TOTAL_WEIGHT and ids[0] == -1
+
+
+def test_sampling_across_super_tile_boundaries():
+    """A table larger than one second-level group (1024 tiles of 2048 prompts)."""
+    n = 2048 * 1024 * 2 + 777
+    rng = np.random.default_rng(11)
+    ab = rng.uniform(0.0, 9.0, (n, 2)).astype(np.float32)
+    u = inputs.uniforms_f32(rng, 512)
+    p = B().default_params()
+    ids, _, st = gpu_sample(dev(ab), u, 256, p, want_w=False)
+    w_or = O.sampling_weights_f32(ab[:, 0], ab[:, 1], np.float32(p.eps_explore))
+    assert st == 0
+    np.testing.assert_array_equal(ids, O.sample_prompts(w_or, u, 256))
