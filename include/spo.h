@@ -223,6 +223,15 @@ int32_t spo_loss_bwd(const void* H, const void* W, int32_t dtype, const int32_t*
                      void* ws, size_t ws_bytes,
                      const spo_params* params, int32_t* d_status, void* stream);
 
+/*
+ * Diagnostic (no counterpart in the paper): runs the kernels' bounded mbarrier wait on a barrier
+ * that nothing ever signals, with a limit of `limit_us` microseconds (1 .. 1 000 000).  A healthy
+ * build sets SPO_DEV_TIMEOUT in *d_status, writes 1 to *reached_end (device int32, optional) and the
+ * kernel returns normally; the context stays usable.  It shows that a stuck pipeline stage ends in a
+ * status bit, not in a hang.  One tiny launch on `stream`.
+ */
+int32_t spo_selftest_bounded_wait(uint32_t limit_us, int32_t* reached_end, int32_t* d_status, void* stream);
+
 /* Scratch size in bytes for one call of the selected entry point (host only, no CUDA call
  * except a device-property query).  Arguments that the selected call does not use are ignored. */
 size_t spo_workspace_bytes(int32_t which, int64_t T, int32_t d, int32_t V,

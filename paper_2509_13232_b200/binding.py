@@ -26,7 +26,7 @@ EXPORTS = [
     "spo_default_params", "spo_tracker_init", "spo_sample_prompts", "spo_advantages",
     "spo_advantages_static",
     "spo_tracker_update", "spo_loss_fwd", "spo_loss_bwd", "spo_workspace_bytes",
-    "spo_status_string", "spo_last_cuda_error", "spo_version",
+    "spo_status_string", "spo_last_cuda_error", "spo_version", "spo_selftest_bounded_wait",
 ]
 
 
@@ -76,6 +76,7 @@ def lib():
         L.spo_loss_bwd.argtypes = [c_void_p, c_void_p, c_int32, c_void_p, c_void_p, c_void_p, c_float,
                                    c_int64, c_int32, c_int32, c_void_p, c_int32, c_void_p, c_int32,
                                    c_void_p, c_size_t, P, c_void_p, c_void_p]
+        L.spo_selftest_bounded_wait.argtypes = [ctypes.c_uint32, c_void_p, c_void_p, c_void_p]
         L.spo_workspace_bytes.argtypes = [c_int32, c_int64, c_int32, c_int32, c_int64, c_int32, c_int32]
         L.spo_workspace_bytes.restype = c_size_t
         L.spo_status_string.argtypes = [c_int32]
@@ -177,3 +178,8 @@ def spo_loss_bwd(H, W, y, lse, coef, grad_loss, dH, dW, dW_accumulate, ws, param
                               c_float(grad_loss), T, d, V, _ptr(dH), _dtype_code(dH), _ptr(dW),
                               int(dW_accumulate), _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size(),
                               ctypes.byref(params), _ptr(d_status), _stream()), "spo_loss_bwd")
+
+
+def spo_selftest_bounded_wait(limit_us, reached_end, d_status):
+    _check(lib().spo_selftest_bounded_wait(int(limit_us), _ptr(reached_end), _ptr(d_status), _stream()),
+           "spo_selftest_bounded_wait")

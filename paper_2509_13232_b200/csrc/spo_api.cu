@@ -233,6 +233,13 @@ size_t spo_workspace_bytes(int32_t which, int64_t T, int32_t d, int32_t V, int64
   }
 }
 
+int32_t spo_selftest_bounded_wait(uint32_t limit_us, int32_t* reached_end, int32_t* d_status, void* stream) {
+  if (!d_status || limit_us == 0 || limit_us > 1000000u) return SPO_ERR_INVALID_ARG;
+  if (!device_is_sm100()) return SPO_ERR_UNSUPPORTED_ARCH;
+  cudaError_t e = launch_bounded_wait_probe(d_status, limit_us, reached_end, (cudaStream_t)stream);
+  return e == cudaSuccess ? SPO_OK : cuda_fail(e);
+}
+
 const char* spo_status_string(int32_t status) {
   switch (status) {
     case SPO_OK: return "ok";

@@ -98,4 +98,6 @@ cudaError_t launch_bwd_bf16(const void* H, const void* W, const int32_t* y, cons
                             void* dH, int32_t dH_dtype, float* dW, int accumulate,
                             char* ws, const BwdWs& L, int32_t* d_status, cudaStream_t st);
 
+cudaError_t launch_bounded_wait_probe(int32_t* d_status, uint32_t limit_us, int32_t* reached_end, cudaStream_t st);
+
 }  // namespace spo

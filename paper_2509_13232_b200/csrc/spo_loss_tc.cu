@@ -145,7 +145,8 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
 // Bounded wait.  Returns false when the wait ran out or another role already gave up.
 // SLEEP_NS > 0 backs off between polls (roles that wait long and need not react within nanoseconds).
 template <int SLEEP_NS = 0>
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* d_status) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* d_status,
+                                          unsigned long long limit_ns = kWaitLimitNs) {
   uint32_t spins = 0;
   unsigned long long t0 = 0;
   while (!mbar_try_wait(bar, parity)) {
@@ -155,7 +156,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       unsigned long long now = global_timer_ns();
       if (t0 == 0) {
         t0 = now;
-      } else if (now - t0 > kWaitLimitNs) {
+      } else if (now - t0 > limit_ns) {
         *abort_flag = 1;
         if (d_status) atomicOr(d_status, SPO_DEV_TIMEOUT);
         return false;
@@ -611,6 +612,23 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
 }
 
+// A wait that nothing ever satisfies, through the same bounded-wait routine the pipeline uses:
+// checks that a stuck barrier ends in SPO_DEV_TIMEOUT and a clean return instead of a hang.
+__global__ void bounded_wait_probe_kernel(int32_t* d_status, unsigned long long limit_ns, int* reached_end) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    mbar_init(smem_u32(&bar), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  bool ok = true;
+  if (threadIdx.x == 0) ok = mbar_wait<64>(smem_u32(&bar), 0, &abort_flag, d_status, limit_ns);
+  __syncthreads();
+  if (threadIdx.x == 0 && reached_end) *reached_end = ok ? 2 : 1;
+}
+
 // ---------------------------------------------------------------------------
 // host side: tensor maps and launches
 // ---------------------------------------------------------------------------
@@ -849,6 +867,11 @@ cudaError_t launch_bwd_bf16(const void* H, const void* W, const int32_t* y, cons
     }
   }
   return cudaSuccess;
+}
+
+cudaError_t launch_bounded_wait_probe(int32_t* d_status, uint32_t limit_us, int32_t* reached_end, cudaStream_t st) {
+  bounded_wait_probe_kernel<<<1, 32, 0, st>>>(d_status, (unsigned long long)limit_us * 1000ull, reached_end);
+  return cudaGetLastError();
 }
 
 }  // namespace spo

@@ -176,3 +176,22 @@ def test_bf16_targets_on_tile_and_half_boundaries():
     got, want = run_loss(lb), oracle_loss(lb)
     check(lb, got, want, 2e-3, 1e-2)
     np.testing.assert_allclose(want["ratio"], 1.0, atol=1e-6)
+
+
+def test_bounded_wait_ends_in_a_status_bit_not_a_hang():
+    """A barrier nobody signals: the wait gives up after its limit, the kernel returns, the context lives on."""
+    import time
+    import torch
+    from paper_2509_13232_b200 import binding as B
+    st = torch.zeros(4, dtype=torch.int32, device="cuda")
+    end = torch.zeros(4, dtype=torch.int32, device="cuda")
+    t0 = time.perf_counter()
+    B.spo_selftest_bounded_wait(2000, end, st)          # 2 ms limit
+    torch.cuda.synchronize()
+    elapsed = time.perf_counter() - t0
+    assert int(st[0].item()) & B.DEV_TIMEOUT
+    assert int(end[0].item()) == 1
+    assert elapsed < 1.0
+    # the device is still usable afterwards
+    lb = inputs.loss_batch(80, [33], 64, 200, 0.05, True, 0.05)
+    assert run_loss(lb)["status"] == 0
