@@ -40,6 +40,8 @@ LOSS_SHAPES = {
     "cfg4_8b_bf16": (4096, 151936, 0.02, 0.02, 0.3),
     "cfg5_longtail_bf16": (4096, 151936, 0.02, 0.02, 0.3),
 }
+# prompts in the tracker table of each workload (cfg5 names a 100 000-prompt table)
+TABLE_PROMPTS = {"cfg5_longtail_bf16": 100_000}
 
 
 def read_peaks():
@@ -112,7 +114,8 @@ class Step:
         self.data = data
         self.T, self.d, self.V, self.S = data["T"], d, V, data["S"]
         self.n_tok = int(data["mask"].sum().item())
-        tb = inputs.tracker_batch(cfg * 10 + rank, TABLE_N, self.S, 2 * self.S)
+        self.table_n = TABLE_PROMPTS.get(workload, TABLE_N)
+        tb = inputs.tracker_batch(cfg * 10 + rank, self.table_n, self.S, 2 * self.S)
         f32 = dict(dtype=torch.float32, device=device)
         self.ab0 = torch.from_numpy(tb.ab).to(device)
         self.ab = self.ab0.clone()
@@ -129,7 +132,7 @@ class Step:
         self.dW = torch.empty((V, d), **f32)
         self.status = torch.zeros(4, dtype=torch.int32, device=device)
         u8 = dict(dtype=torch.uint8, device=device)
-        self.ws_sample = torch.empty(B.spo_workspace_bytes(B.WS_SAMPLE, N=TABLE_N, M=2 * self.S), **u8)
+        self.ws_sample = torch.empty(B.spo_workspace_bytes(B.WS_SAMPLE, N=self.table_n, M=2 * self.S), **u8)
         self.ws_adv = torch.empty(B.spo_workspace_bytes(B.WS_ADVANTAGES, B=self.S), **u8)
         self.ws_fwd = torch.empty(B.spo_workspace_bytes(B.WS_LOSS_FWD, T=self.T, d=d, V=V), **u8)
         self.ws_bwd_bytes = B.spo_workspace_bytes(B.WS_LOSS_BWD, T=self.T, d=d, V=V)
@@ -264,7 +267,7 @@ def run_ours(args, rank, world, local_rank):
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": args.workload, "responses": step.S, "tokens": step.T, "d": step.d, "V": step.V,
-                   "tracker_prompts": TABLE_N, "l2": "inputs_exceed_l2", "bwd_chunks": step.bwd_chunks,
+                   "tracker_prompts": step.table_n, "l2": "inputs_exceed_l2", "bwd_chunks": step.bwd_chunks,
                    "parallelism": "replicas" if world > 1 else "single"},
         "gpu_launches": step.launches * args.steps,
         "device_status": status,

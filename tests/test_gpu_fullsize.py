@@ -36,10 +36,11 @@ def test_real_vocab_and_hidden_small_token_count_full_oracle():
     assert rel_fro(got["dW"][-64:], want["dW"][-64:]) <= 1e-2
 
 
-def test_cfg4_full_size_sampled_rows_and_identities():
+@pytest.mark.parametrize("workload", ["cfg3_small_bf16", "cfg4_8b_bf16", "cfg5_longtail_bf16"])
+def test_full_size_sampled_rows_and_identities(workload):
     import torch
     import bench
-    step = bench.Step("cfg4_8b_bf16", torch.device("cuda", 0), 0)
+    step = bench.Step(workload, torch.device("cuda", 0), 0)
     step.run()
     torch.cuda.synchronize()
     assert int(step.status[0].item()) == 0
