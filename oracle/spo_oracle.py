@@ -220,8 +220,35 @@ def logits(h, w):
     return np.asarray(h, dtype=np.float64) @ np.asarray(w, dtype=np.float64).T
 
 
+AGG_TOKEN_MEAN = 0      # mean over all unmasked tokens of the batch
+AGG_SEQ_MEAN = 1        # mean over responses of each response's own token mean
+
+
+def aggregation_weights(mask01, seq, n_seq, agg_mode):
+    """Weight u_t of token t in the expectation E_{s,t} of the objective; the weights sum to 1.
+
+    The paper writes E_{s,t} without saying how tokens of responses of different
+    length are weighted.  Mode 0 (the reading taken as default): every unmasked token
+    counts alike, u_t = m_t / n_tok.  Mode 1: every response that has an unmasked
+    token counts alike and its tokens share its weight, u_t = m_t / (S_act * n_s(t)).
+    """
+    m = np.asarray(mask01, dtype=np.float64)
+    if agg_mode == AGG_TOKEN_MEAN:
+        n_tok = m.sum()
+        return m / n_tok if n_tok > 0 else np.zeros_like(m)
+    if agg_mode == AGG_SEQ_MEAN:
+        per_seq = np.zeros(n_seq, dtype=np.float64)
+        np.add.at(per_seq, seq, m)
+        s_act = float((per_seq > 0).sum())
+        if s_act == 0:
+            return np.zeros_like(m)
+        denom = np.where(per_seq[seq] > 0, per_seq[seq], 1.0)
+        return m / (s_act * denom)
+    raise ValueError("agg_mode")
+
+
 def loss_forward(h, w, y, logp_old, mask, cu_seqlens, a_norm,
-                 clip_lo=CLIP_LO, clip_hi=CLIP_HI):
+                 clip_lo=CLIP_LO, clip_hi=CLIP_HI, agg_mode=AGG_TOKEN_MEAN):
     """Token-level PPO-Clip surrogate of Sec. 3.2 with Clip-Higher bounds.
 
     Per token t (row of ``h``): z = W h_t; lse = log sum_v exp(z_v);
@@ -232,7 +259,8 @@ def loss_forward(h, w, y, logp_old, mask, cu_seqlens, a_norm,
 
     Returns a dict: loss, logp[T], lse[T], ratio[T], surrogate[T], unclipped[T]
     (bool: the gradient passes through the ratio), coef[T] = d loss / d logp_t
-    = -mask*a*ratio*unclipped/n_tok, n_tok, and seq_sums[S,3] = per sequence
+    = -u_t*a*ratio*unclipped with u_t the aggregation weight (mask/n_tok by
+    default, see aggregation_weights), n_tok, and seq_sums[S,3] = per sequence
     (sum mask*logp, sum mask*(logp_old - logp), sum mask).
     """
     z = logits(h, w)
@@ -252,13 +280,14 @@ def loss_forward(h, w, y, logp_old, mask, cu_seqlens, a_norm,
     clipped_ratio = np.minimum(np.maximum(ratio, 1.0 - clip_lo), 1.0 + clip_hi)
     surrogate = np.minimum(ratio * a, clipped_ratio * a)
     n_tok = m.sum()
-    loss = -(m * surrogate).sum() / n_tok if n_tok > 0 else 0.0
+    n_seq = len(cu_seqlens) - 1
+    u = aggregation_weights(m, seq, n_seq, agg_mode)
+    loss = -(u * surrogate).sum()
     # The min picks the unclipped branch (and so carries gradient) when the
     # ratio is on the inside of the bound that matters for the sign of a;
     # the boundary itself counts as inside.
     unclipped = np.where(a >= 0.0, ratio <= 1.0 + clip_hi, ratio >= 1.0 - clip_lo)
-    coef = -(m * a * ratio * unclipped) / n_tok if n_tok > 0 else np.zeros(n_tok_rows)
-    n_seq = len(cu_seqlens) - 1
+    coef = -(u * a * ratio * unclipped)
     seq_sums = np.zeros((n_seq, 3), dtype=np.float64)
     np.add.at(seq_sums[:, 0], seq, m * logp)
     np.add.at(seq_sums[:, 1], seq, m * (logp_old - logp))

@@ -474,3 +474,57 @@ def test_row_local_helper_equals_full_definition():
 
 def test_token_to_sequence_map():
     np.testing.assert_array_equal(O.token_sequence_ids([0, 2, 2, 5], 5), [0, 0, 2, 2, 2])
+
+
+# ------------------------------------------------------ aggregation variants
+
+def test_aggregation_weights_sum_to_one_and_hand_values():
+    seq = np.array([0, 1, 1, 1, 2, 2])
+    m = np.array([1, 1, 0, 1, 0, 0], dtype=float)          # response 2 fully masked
+    u0 = O.aggregation_weights(m, seq, 3, O.AGG_TOKEN_MEAN)
+    u1 = O.aggregation_weights(m, seq, 3, O.AGG_SEQ_MEAN)
+    np.testing.assert_allclose(u0, [1 / 3, 1 / 3, 0, 1 / 3, 0, 0])
+    np.testing.assert_allclose(u1, [1 / 2, 1 / 4, 0, 1 / 4, 0, 0])
+    assert abs(u0.sum() - 1) < 1e-15 and abs(u1.sum() - 1) < 1e-15
+    assert O.aggregation_weights(np.zeros(4), np.zeros(4, int), 1, O.AGG_SEQ_MEAN).sum() == 0.0
+
+
+def test_sequence_mean_at_ratio_one_is_minus_mean_of_response_advantages():
+    rng = np.random.default_rng(21)
+    t, d, v = 9, 4, 12
+    h, w = rng.standard_normal((t, d)), rng.standard_normal((v, d))
+    y = rng.integers(0, v, t)
+    cu, a = [0, 1, 4, 9], np.array([2.0, -1.0, 0.5])
+    new = O.loss_forward(h, w, y, np.zeros(t), None, cu, a)["logp"]
+    tok = O.loss_forward(h, w, y, new, None, cu, a, agg_mode=O.AGG_TOKEN_MEAN)
+    seq = O.loss_forward(h, w, y, new, None, cu, a, agg_mode=O.AGG_SEQ_MEAN)
+    assert abs(seq["loss"] + a.mean()) < 1e-14                       # each response counts once
+    assert abs(tok["loss"] + (1 * 2.0 - 3 * 1.0 + 5 * 0.5) / 9) < 1e-14  # each token counts once
+    # equal lengths: the two readings coincide
+    same = [O.loss_forward(h[:8], w, y[:8], new[:8], None, [0, 4, 8], a[:2], agg_mode=k)["loss"] for k in (0, 1)]
+    assert abs(same[0] - same[1]) < 1e-15
+
+
+def test_sequence_mean_gradients_against_finite_differences():
+    rng = np.random.default_rng(22)
+    t, d, v = 7, 5, 9
+    h, w = rng.standard_normal((t, d)), rng.standard_normal((v, d)) * 0.5
+    y = rng.integers(0, v, t)
+    cu, a = [0, 2, 3, 7], np.array([0.9, -1.1, 0.4])
+    mask = np.array([1, 1, 1, 0, 1, 1, 1], dtype=np.uint8)
+    base = O.loss_forward(h, w, y, np.zeros(t), mask, cu, a)["logp"]
+    logp_old = base - np.log([1.1, 1.5, 0.6, 1.0, 1.2, 0.9, 1.05])
+    fwd = O.loss_forward(h, w, y, logp_old, mask, cu, a, agg_mode=O.AGG_SEQ_MEAN)
+    dh, dw = O.loss_backward(h, w, y, fwd["lse"], fwd["coef"])
+    step = 1e-6
+    for arr, grad in ((h, dh), (w, dw)):
+        num = np.zeros_like(arr)
+        for idx in np.ndindex(arr.shape):
+            keep = arr[idx]
+            arr[idx] = keep + step
+            up = O.loss_forward(h, w, y, logp_old, mask, cu, a, agg_mode=O.AGG_SEQ_MEAN)["loss"]
+            arr[idx] = keep - step
+            dn = O.loss_forward(h, w, y, logp_old, mask, cu, a, agg_mode=O.AGG_SEQ_MEAN)["loss"]
+            arr[idx] = keep
+            num[idx] = (up - dn) / (2 * step)
+        assert np.linalg.norm(num - grad) <= 1e-6 * np.linalg.norm(grad)
