@@ -134,7 +134,7 @@ class Step:
         u8 = dict(dtype=torch.uint8, device=device)
         self.ws_sample = torch.empty(B.spo_workspace_bytes(B.WS_SAMPLE, N=self.table_n, M=2 * self.S), **u8)
         self.ws_adv = torch.empty(B.spo_workspace_bytes(B.WS_ADVANTAGES, B=self.S), **u8)
-        self.ws_fwd = torch.empty(B.spo_workspace_bytes(B.WS_LOSS_FWD, T=self.T, d=d, V=V), **u8)
+        self.ws_fwd = torch.empty(B.spo_workspace_bytes(B.WS_LOSS_FWD, T=self.T, d=d, V=V, B=self.S), **u8)
         self.ws_bwd_bytes = B.spo_workspace_bytes(B.WS_LOSS_BWD, T=self.T, d=d, V=V)
         self.ws_bwd = torch.empty(self.ws_bwd_bytes, **u8)
         chunk_rows = self.ws_bwd_bytes // (((V + 255) // 256) * 256 * 2)

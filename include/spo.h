@@ -50,6 +50,12 @@ extern "C" {
 #define SPO_DTYPE_F32   0
 #define SPO_DTYPE_BF16  1
 
+/* token weights in the objective's expectation E_{s,t} (the paper does not say how responses of
+ * different length are weighted): every unmasked token alike (default), or every response alike
+ * with its tokens sharing the response's weight */
+#define SPO_AGG_TOKEN_MEAN  0
+#define SPO_AGG_SEQ_MEAN    1
+
 /* selectors for spo_workspace_bytes */
 #define SPO_WS_SAMPLE      0
 #define SPO_WS_ADVANTAGES  1
@@ -72,6 +78,7 @@ typedef struct spo_params {
   float   clip_hi;
   float   norm_eps;
   int32_t norm_ddof;
+  int32_t agg_mode;       /* SPO_AGG_*: how E_{s,t} of the objective weights tokens */
 } spo_params;
 
 int32_t spo_default_params(spo_params* p /* host, out */);
@@ -180,8 +187,11 @@ int32_t spo_tracker_update(float* ab, int64_t N, const int32_t* ids, const float
  *   z = W h_t (never stored), lse = log sum_v exp z_v, logp = z[y_t] - lse,
  *   ratio = exp(logp - logp_old_t), a = a_norm[seq(t)],
  *   s_t = min(ratio*a, clip(ratio, 1-clip_lo, 1+clip_hi)*a),
- *   loss = - sum_t mask_t s_t / n_tok,  n_tok = sum_t mask_t  (0 if n_tok = 0),
- *   coef_t = d loss / d logp_t = -mask_t * a * ratio * [gradient passes the clip] / n_tok.
+ *   loss = - sum_t u_t s_t with token weights u_t that sum to one: u_t = mask_t / n_tok,
+ *   n_tok = sum_t mask_t (SPO_AGG_TOKEN_MEAN), or u_t = mask_t / (S_act * n_seq(t)) with n_s the
+ *   unmasked tokens of response s and S_act the responses that have any (SPO_AGG_SEQ_MEAN);
+ *   loss = 0 if n_tok = 0;
+ *   coef_t = d loss / d logp_t = -u_t * a * ratio * [gradient passes the clip].
  *
  *   H           device in  [T][d], row-major, dtype as given (bf16: d % 64 == 0)
  *   W           device in  [V][d], row-major, same dtype
@@ -194,7 +204,8 @@ int32_t spo_tracker_update(float* ab, int64_t N, const int32_t* ids, const float
  *   logp, lse, coef   device out [T] fp32 each
  *   seq_sums    device out [S][3] fp32 = per response (sum mask*logp,
  *               sum mask*(logp_old-logp), sum mask), optional
- *   ws          device scratch, spo_workspace_bytes(SPO_WS_LOSS_FWD, T, d, V, ...) bytes
+ *   ws          device scratch, spo_workspace_bytes(SPO_WS_LOSS_FWD, T, d, V, 0, S, 0) bytes
+ *               (the B argument of that query carries the number of responses S)
  * A target outside [0,V) sets SPO_DEV_ID_OUT_OF_RANGE (the row gets logp = -inf, coef = 0).
  */
 int32_t spo_loss_fwd(const void* H, const void* W, int32_t dtype,

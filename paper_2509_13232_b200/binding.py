@@ -21,6 +21,7 @@ ERR_UNSUPPORTED_DTYPE, ERR_UNSUPPORTED_ARCH, ERR_WORKSPACE_TOO_SMALL, ERR_CUDA =
 DEV_ID_OUT_OF_RANGE, DEV_NONFINITE, DEV_UNIFORMS_EXHAUSTED, DEV_TIMEOUT, DEV_ZERO_TOTAL_WEIGHT = 1, 2, 4, 8, 16
 DTYPE_F32, DTYPE_BF16 = 0, 1
 WS_SAMPLE, WS_ADVANTAGES, WS_LOSS_FWD, WS_LOSS_BWD = 0, 1, 2, 3
+AGG_TOKEN_MEAN, AGG_SEQ_MEAN = 0, 1
 
 EXPORTS = [
     "spo_default_params", "spo_tracker_init", "spo_sample_prompts", "spo_advantages",
@@ -34,6 +35,7 @@ class SpoParams(Structure):
     _fields_ = [
         ("rho_min", c_float), ("rho_max", c_float), ("d_half", c_float), ("eps_explore", c_float),
         ("clip_lo", c_float), ("clip_hi", c_float), ("norm_eps", c_float), ("norm_ddof", c_int32),
+        ("agg_mode", c_int32),
     ]
 
 

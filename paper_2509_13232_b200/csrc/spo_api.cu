@@ -38,7 +38,7 @@ int device_is_sm100() {
 
 int fwd_bf16_nsplit(int64_t T, int32_t d, int32_t V);   // spo_loss_tc.cu
 
-FwdWs fwd_ws_layout(int64_t T, int32_t d, int32_t V, int32_t dtype) {
+FwdWs fwd_ws_layout(int64_t T, int32_t d, int32_t V, int32_t dtype, int32_t S) {
   FwdWs L{};
   L.nsplit = dtype == SPO_DTYPE_BF16 ? fwd_bf16_nsplit(T, d, V) : 1;
   L.fin_blocks = ceil_div(T > 0 ? T : 1, kFinalizeThreads);
@@ -47,6 +47,7 @@ FwdWs fwd_ws_layout(int64_t T, int32_t d, int32_t V, int32_t dtype) {
   L.partials = off;   off = align_up(off + sizeof(FwdPartial) * (size_t)L.nsplit * (size_t)(T > 0 ? T : 1), 256);
   L.block_sums = off; off = align_up(off + sizeof(double) * (size_t)L.fin_blocks, 256);
   L.counters = off;   off = align_up(off + 4 * sizeof(int32_t), 256);
+  L.seq_cnt = off;    off = align_up(off + sizeof(int32_t) * (size_t)(S > 0 ? S : 1), 256);
   L.total = off;
   return L;
 }
@@ -66,6 +67,7 @@ static bool params_ok(const spo_params* p) {
   if (!(p->clip_lo >= 0.0f) || !(p->clip_lo < 1.0f) || !(p->clip_hi >= 0.0f)) return false;
   if (!(p->norm_eps >= 0.0f)) return false;
   if (p->norm_ddof != 0 && p->norm_ddof != 1) return false;
+  if (p->agg_mode != SPO_AGG_TOKEN_MEAN && p->agg_mode != SPO_AGG_SEQ_MEAN) return false;
   return true;
 }
 
@@ -85,6 +87,7 @@ int32_t spo_default_params(spo_params* p) {
   p->clip_hi = 0.28f;
   p->norm_eps = 1e-8f;
   p->norm_ddof = 0;
+  p->agg_mode = SPO_AGG_TOKEN_MEAN;
   return SPO_OK;
 }
 
@@ -166,14 +169,15 @@ int32_t spo_loss_fwd(const void* H, const void* W, int32_t dtype, const int32_t*
       !aligned16(a_norm) || !aligned16(logp) || !aligned16(lse) || !aligned16(coef) || !aligned16(ws))
     return SPO_ERR_BAD_ALIGNMENT;
   if (!device_is_sm100()) return SPO_ERR_UNSUPPORTED_ARCH;
-  const FwdWs L = fwd_ws_layout(T, d, V, dtype);
+  const FwdWs L = fwd_ws_layout(T, d, V, dtype, S);
   if (ws_bytes < L.total) return SPO_ERR_WORKSPACE_TOO_SMALL;
   cudaStream_t st = (cudaStream_t)stream;
   char* w8 = (char*)ws;
   FwdPartial* partials = reinterpret_cast<FwdPartial*>(w8 + L.partials);
   double* block_sums = reinterpret_cast<double*>(w8 + L.block_sums);
   int32_t* counters = reinterpret_cast<int32_t*>(w8 + L.counters);
-  cudaError_t e = launch_fwd_prepare(mask, T, counters, st);
+  int32_t* seq_cnt = reinterpret_cast<int32_t*>(w8 + L.seq_cnt);
+  cudaError_t e = launch_fwd_prepare(mask, T, cu_seqlens, S, params->agg_mode, seq_cnt, counters, st);
   if (e != cudaSuccess) return cuda_fail(e);
   if (dtype == SPO_DTYPE_BF16)
     e = launch_fwd_bf16(H, W, y, T, d, V, partials, L.nsplit, reinterpret_cast<uint32_t*>(w8 + L.progress), d_status, st);
@@ -181,7 +185,8 @@ int32_t spo_loss_fwd(const void* H, const void* W, int32_t dtype, const int32_t*
     e = launch_fwd_f32((const float*)H, (const float*)W, y, T, d, V, partials, st);
   if (e != cudaSuccess) return cuda_fail(e);
   e = launch_fwd_finalize(partials, L.nsplit, y, logp_old, mask, cu_seqlens, a_norm, T, V, S, params->clip_lo,
-                          params->clip_hi, loss, logp, lse, coef, seq_sums, block_sums, counters, L.fin_blocks,
+                          params->clip_hi, loss, logp, lse, coef, seq_sums, block_sums, counters, seq_cnt, params->agg_mode,
+                          L.fin_blocks,
                           d_status, st);
   return e == cudaSuccess ? SPO_OK : cuda_fail(e);
 }
@@ -224,7 +229,7 @@ size_t spo_workspace_bytes(int32_t which, int64_t T, int32_t d, int32_t V, int64
       return align_up(sizeof(double) * 2 * (size_t)adv_blocks(B), 256);
     case SPO_WS_LOSS_FWD:
       if (T < 0 || V < 1) return 0;
-      return fwd_ws_layout(T, d, V, (d % 64) == 0 ? SPO_DTYPE_BF16 : SPO_DTYPE_F32).total;
+      return fwd_ws_layout(T, d, V, (d % 64) == 0 ? SPO_DTYPE_BF16 : SPO_DTYPE_F32, B).total;
     case SPO_WS_LOSS_BWD:
       if (T < 0 || V < 1 || d < 1) return 0;
       return bwd_ws_layout(T, d, V).total;

@@ -58,21 +58,23 @@ struct FwdWs {
   size_t progress;      // uint32 [256]
   size_t partials;      // FwdPartial [nsplit][T]
   size_t block_sums;    // double [finalize blocks]
-  size_t counters;      // int32 [4]: n_tok, ticket
+  size_t counters;      // int32 [4]: n_tok, ticket, responses with an unmasked token
+  size_t seq_cnt;       // int32 [S]: unmasked tokens per response (sequence-mean aggregation)
   size_t total;
   int nsplit;
   int64_t fin_blocks;
 };
-FwdWs fwd_ws_layout(int64_t T, int32_t d, int32_t V, int32_t dtype);
+FwdWs fwd_ws_layout(int64_t T, int32_t d, int32_t V, int32_t dtype, int32_t S);
 
-cudaError_t launch_fwd_prepare(const uint8_t* mask, int64_t T, int32_t* counters, cudaStream_t st);
+cudaError_t launch_fwd_prepare(const uint8_t* mask, int64_t T, const int32_t* cu_seqlens, int32_t S, int agg_mode,
+                               int32_t* seq_cnt, int32_t* counters, cudaStream_t st);
 cudaError_t launch_fwd_finalize(const FwdPartial* partials, int nsplit, const int32_t* y,
                                 const float* logp_old, const uint8_t* mask, const int32_t* cu_seqlens,
                                 const float* a_norm, int64_t T, int32_t V, int32_t S,
                                 float clip_lo, float clip_hi,
                                 float* loss, float* logp, float* lse, float* coef, float* seq_sums,
-                                double* block_sums, int32_t* counters, int64_t fin_blocks,
-                                int32_t* d_status, cudaStream_t st);
+                                double* block_sums, int32_t* counters, const int32_t* seq_cnt, int agg_mode,
+                                int64_t fin_blocks, int32_t* d_status, cudaStream_t st);
 
 // fp32 SIMT path
 cudaError_t launch_fwd_f32(const float* H, const float* W, const int32_t* y, int64_t T, int32_t d, int32_t V,

@@ -44,6 +44,33 @@ count_mask_kernel(const uint8_t* __restrict__ mask, int64_t T, int32_t* counters
 
 __global__ void set_count_kernel(int32_t value, int32_t* counters) { counters[0] = value; }
 
+// Sequence-mean aggregation: seq_cnt[s] = unmasked tokens of response s; counters[2] = responses
+// that have at least one.
+__global__ void __launch_bounds__(256)
+seq_count_kernel(const uint8_t* __restrict__ mask, const int32_t* __restrict__ cu_seqlens, int32_t* __restrict__ seq_cnt,
+                 int32_t* counters) {
+  const int s = blockIdx.x;
+  const int64_t lo = cu_seqlens[s], hi = cu_seqlens[s + 1];
+  int local = 0;
+  if (mask) {
+    for (int64_t t = lo + threadIdx.x; t < hi; t += 256) local += mask[t] != 0;
+  } else if (threadIdx.x == 0) {
+    local = (int)(hi - lo);
+  }
+  __shared__ int s_w[8];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) local += __shfl_xor_sync(0xffffffffu, local, o);
+  if ((threadIdx.x & 31) == 0) s_w[threadIdx.x >> 5] = local;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int tot = 0;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) tot += s_w[w];
+    seq_cnt[s] = tot;
+    if (tot > 0) atomicAdd(&counters[2], 1);
+  }
+}
+
 // Per token: merge the vocabulary splits' (max, sum-exp, target logit), then the
 // importance ratio, the clipped surrogate (Sec. 3.2) and d loss / d logp.
 __global__ void __launch_bounds__(kFinalizeThreads)
@@ -52,9 +79,11 @@ fwd_finalize_kernel(const FwdPartial* __restrict__ partials, int nsplit, const i
                     const int32_t* __restrict__ cu_seqlens, const float* __restrict__ a_norm,
                     int64_t T, int32_t V, int32_t S, float clip_lo, float clip_hi,
                     float* __restrict__ loss, float* __restrict__ logp_out, float* __restrict__ lse_out,
-                    float* __restrict__ coef_out, double* block_sums, int32_t* counters, int32_t* d_status) {
+                    float* __restrict__ coef_out, double* block_sums, int32_t* counters,
+                    const int32_t* __restrict__ seq_cnt, int agg_mode, int32_t* d_status) {
   const int64_t t = (int64_t)blockIdx.x * kFinalizeThreads + threadIdx.x;
   const int32_t n_tok = counters[0];
+  const int32_t s_act = counters[2];
   double contrib = 0.0;
   if (t < T) {
     float m2 = -CUDART_INF_F, zt = -CUDART_INF_F;
@@ -87,9 +116,16 @@ fwd_finalize_kernel(const FwdPartial* __restrict__ partials, int nsplit, const i
       const float hi_b = 1.0f + clip_hi, lo_b = 1.0f - clip_lo;
       const float sur = fminf(ratio * a, fminf(fmaxf(ratio, lo_b), hi_b) * a);
       const bool passes = a >= 0.0f ? ratio <= hi_b : ratio >= lo_b;
-      if (on) {
-        contrib = (double)sur;
-        if (passes && n_tok > 0) coef = -a * ratio / (float)n_tok;
+      if (on && n_tok > 0) {
+        // weight of this token in the expectation: 1/n_tok, or 1/(responses * tokens of its response)
+        if (agg_mode == 0) {
+          contrib = (double)sur;
+          if (passes) coef = -a * ratio / (float)n_tok;
+        } else {
+          const float u = 1.0f / ((float)s_act * (float)seq_cnt[lo]);
+          contrib = (double)sur * (double)u;
+          if (passes) coef = -a * ratio * u;
+        }
       }
     }
     logp_out[t] = lp;
@@ -124,7 +160,8 @@ fwd_finalize_kernel(const FwdPartial* __restrict__ partials, int nsplit, const i
       double tot = 0.0;
 #pragma unroll
       for (int w = 0; w < kFinalizeThreads / 32; ++w) tot += s_part[w];
-      loss[0] = n_tok > 0 ? (float)(-tot / (double)n_tok) : 0.0f;
+      if (n_tok <= 0) loss[0] = 0.0f;
+      else loss[0] = agg_mode == 0 ? (float)(-tot / (double)n_tok) : (float)(-tot);
     }
   }
 }
@@ -278,9 +315,14 @@ bwd_f32_kernel(const float* __restrict__ H, const float* __restrict__ W, const i
 // host launchers
 // ---------------------------------------------------------------------------
 
-cudaError_t launch_fwd_prepare(const uint8_t* mask, int64_t T, int32_t* counters, cudaStream_t st) {
+cudaError_t launch_fwd_prepare(const uint8_t* mask, int64_t T, const int32_t* cu_seqlens, int32_t S, int agg_mode,
+                               int32_t* seq_cnt, int32_t* counters, cudaStream_t st) {
   cudaError_t e = cudaMemsetAsync(counters, 0, 4 * sizeof(int32_t), st);
   if (e != cudaSuccess) return e;
+  if (agg_mode != 0 && S > 0 && T > 0) {
+    seq_count_kernel<<<S, 256, 0, st>>>(mask, cu_seqlens, seq_cnt, counters);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  }
   if (mask) {
     int64_t blocks = ceil_div(T > 0 ? T : 1, 256 * 8);
     int64_t cap = (int64_t)sm_count() * 8;
@@ -297,11 +339,11 @@ cudaError_t launch_fwd_finalize(const FwdPartial* partials, int nsplit, const in
                                 const float* a_norm, int64_t T, int32_t V, int32_t S,
                                 float clip_lo, float clip_hi,
                                 float* loss, float* logp, float* lse, float* coef, float* seq_sums,
-                                double* block_sums, int32_t* counters, int64_t fin_blocks,
-                                int32_t* d_status, cudaStream_t st) {
+                                double* block_sums, int32_t* counters, const int32_t* seq_cnt, int agg_mode,
+                                int64_t fin_blocks, int32_t* d_status, cudaStream_t st) {
   fwd_finalize_kernel<<<(unsigned)fin_blocks, kFinalizeThreads, 0, st>>>(
       partials, nsplit, y, logp_old, mask, cu_seqlens, a_norm, T, V, S, clip_lo, clip_hi,
-      loss, logp, lse, coef, block_sums, counters, d_status);
+      loss, logp, lse, coef, block_sums, counters, seq_cnt, agg_mode, d_status);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   if (seq_sums && S > 0) {

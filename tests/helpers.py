@@ -46,7 +46,7 @@ def run_loss(lb, params=None, grad_loss=1.0, dh_bf16=None, want_seq_sums=True, d
     logp, lse, coef = (torch.full((max(T, 1),), float("nan"), **f32) for _ in range(3))
     seq = torch.zeros((max(S, 1), 3), **f32) if want_seq_sums else None
     st = status_word()
-    wsf = ws_bytes(B.WS_LOSS_FWD, T=T, d=d, V=V)
+    wsf = ws_bytes(B.WS_LOSS_FWD, T=T, d=d, V=V, B=S)
     B.spo_loss_fwd(H, W, y, lo, mask, cu, an, loss, logp, lse, coef, seq, wsf, params, st)
     if dh_bf16 is None:
         dh_bf16 = lb.bf16
@@ -72,7 +72,8 @@ def oracle_loss(lb, params=None, grad_loss=1.0, mask_none=False):
     clip_lo = 0.2 if params is None else float(np.float32(params.clip_lo))
     clip_hi = 0.28 if params is None else float(np.float32(params.clip_hi))
     mask = None if mask_none else lb.mask
-    fwd = O.loss_forward(lb.h, lb.w, lb.y, lb.logp_old, mask, lb.cu_seqlens, lb.a_norm, clip_lo, clip_hi)
+    agg = 0 if params is None else int(params.agg_mode)
+    fwd = O.loss_forward(lb.h, lb.w, lb.y, lb.logp_old, mask, lb.cu_seqlens, lb.a_norm, clip_lo, clip_hi, agg)
     dh, dw = O.loss_backward(lb.h, lb.w, lb.y, fwd["lse"], fwd["coef"], grad_loss)
     fwd["dH"], fwd["dW"] = dh, dw
     return fwd

@@ -124,7 +124,7 @@ def test_empty_batch_is_a_no_op_with_zero_loss():
         cu = torch.zeros(1, dtype=torch.int32, device="cuda")
         st = status_word()
         B.spo_loss_fwd(H, W, z(0, torch.int32), z(0), None, cu, z(0), loss, z(0), z(0), z(0), None,
-                       ws_bytes(B.WS_LOSS_FWD, T=0, d=d, V=v), p, st)
+                       ws_bytes(B.WS_LOSS_FWD, T=0, d=d, V=v, B=1), p, st)
         dW = torch.full((v, d), 3.0, device="cuda")
         dH = torch.empty((0, d), dtype=dt, device="cuda")
         B.spo_loss_bwd(H, W, z(0, torch.int32), z(0), z(0), 1.0, dH, dW, 0, ws_bytes(B.WS_LOSS_BWD, T=0, d=d, V=v), p, st)
@@ -195,3 +195,24 @@ def test_bounded_wait_ends_in_a_status_bit_not_a_hang():
     # the device is still usable afterwards
     lb = inputs.loss_batch(80, [33], 64, 200, 0.05, True, 0.05)
     assert run_loss(lb)["status"] == 0
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+def test_sequence_mean_aggregation(bf16):
+    """Each response weighs the same whatever its length; fully masked and empty responses drop out."""
+    from paper_2509_13232_b200 import binding as B
+    params = B.default_params(agg_mode=B.AGG_SEQ_MEAN)
+    lb = _clip_batch(90, [3, 40, 0, 17, 1, 9], 64, 333, bf16)
+    lb.mask[3:43] = 0                                   # response 1 entirely masked
+    lb.mask[50] = 0
+    got = run_loss(lb, params=params, grad_loss=0.8)
+    want = oracle_loss(lb, params=params, grad_loss=0.8)
+    tol = (2e-3, 1e-2) if bf16 else (1e-4, 1e-4)
+    check(lb, got, want, *tol)
+    # and it differs from the token mean on this batch, so the switch is really exercised
+    other = oracle_loss(lb, grad_loss=0.8)
+    assert abs(other["loss"] - want["loss"]) > 1e-3
+    for mask_none in (True,):
+        got = run_loss(lb, params=params, mask_none=mask_none)
+        want = oracle_loss(lb, params=params, mask_none=mask_none)
+        check(lb, got, want, *tol)
