@@ -61,6 +61,7 @@ extern "C" {
 #define SPO_WS_ADVANTAGES  1
 #define SPO_WS_LOSS_FWD    2
 #define SPO_WS_LOSS_BWD    3
+#define SPO_WS_UPDATE_REPEATS 4
 
 /*
  * Hyper-parameters.  Defaults (spo_default_params) are the values the paper prints:
@@ -180,6 +181,21 @@ int32_t spo_advantages_static(const float* ab, int64_t N, const int32_t* ids, co
 int32_t spo_tracker_update(float* ab, int64_t N, const int32_t* ids, const float* r, const float* kl,
                            int32_t kl_is_table, int32_t B,
                            const spo_params* params, int32_t* d_status, void* stream);
+
+/*
+ * Tracker update for batch SPO (appendix "Batch Extensions": every prompt rolled out G times per
+ * batch against a shared baseline): like spo_tracker_update, but `ids` may repeat.  The entries
+ * of one prompt are applied one after the other in batch order (the update equation of Sec. 3.1
+ * composed G times), the same result as G successive calls; the outcome does not depend on
+ * thread scheduling.  spo_advantages already accepts repeated ids (every copy reads the same
+ * pre-update estimate), so a batch-SPO step is spo_advantages, then this call.
+ *
+ *   ws   device scratch, spo_workspace_bytes(SPO_WS_UPDATE_REPEATS, ..., B, ...) bytes
+ * Limit: B <= 65536 (one thread block walks the rounds).  Status bits as spo_tracker_update.
+ */
+int32_t spo_tracker_update_repeats(float* ab, int64_t N, const int32_t* ids, const float* r, const float* kl,
+                                   int32_t kl_is_table, int32_t B, void* ws, size_t ws_bytes,
+                                   const spo_params* params, int32_t* d_status, void* stream);
 
 /*
  * Policy loss forward (Sec. 3.2, the PPO-Clip objective with Clip-Higher bounds,

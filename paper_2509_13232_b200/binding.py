@@ -20,13 +20,13 @@ ERR_INVALID_ARG, ERR_BAD_SHAPE, ERR_BAD_ALIGNMENT = -1, -2, -3
 ERR_UNSUPPORTED_DTYPE, ERR_UNSUPPORTED_ARCH, ERR_WORKSPACE_TOO_SMALL, ERR_CUDA = -4, -5, -6, -7
 DEV_ID_OUT_OF_RANGE, DEV_NONFINITE, DEV_UNIFORMS_EXHAUSTED, DEV_TIMEOUT, DEV_ZERO_TOTAL_WEIGHT = 1, 2, 4, 8, 16
 DTYPE_F32, DTYPE_BF16 = 0, 1
-WS_SAMPLE, WS_ADVANTAGES, WS_LOSS_FWD, WS_LOSS_BWD = 0, 1, 2, 3
+WS_SAMPLE, WS_ADVANTAGES, WS_LOSS_FWD, WS_LOSS_BWD, WS_UPDATE_REPEATS = 0, 1, 2, 3, 4
 AGG_TOKEN_MEAN, AGG_SEQ_MEAN = 0, 1
 
 EXPORTS = [
     "spo_default_params", "spo_tracker_init", "spo_sample_prompts", "spo_advantages",
     "spo_advantages_static",
-    "spo_tracker_update", "spo_loss_fwd", "spo_loss_bwd", "spo_workspace_bytes",
+    "spo_tracker_update", "spo_tracker_update_repeats", "spo_loss_fwd", "spo_loss_bwd", "spo_workspace_bytes",
     "spo_status_string", "spo_last_cuda_error", "spo_version", "spo_selftest_bounded_wait",
 ]
 
@@ -71,6 +71,8 @@ def lib():
                                             c_void_p, P, c_void_p, c_void_p]
         L.spo_tracker_update.argtypes = [c_void_p, c_int64, c_void_p, c_void_p, c_void_p, c_int32, c_int32,
                                          P, c_void_p, c_void_p]
+        L.spo_tracker_update_repeats.argtypes = [c_void_p, c_int64, c_void_p, c_void_p, c_void_p, c_int32, c_int32,
+                                                 c_void_p, c_size_t, P, c_void_p, c_void_p]
         L.spo_loss_fwd.argtypes = [c_void_p, c_void_p, c_int32, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                                    c_int64, c_int32, c_int32, c_int32,
                                    c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
@@ -160,6 +162,13 @@ def spo_tracker_update(ab, ids, r, kl, kl_is_table, params, d_status):
     _check(lib().spo_tracker_update(_ptr(ab), ab.shape[0], _ptr(ids), _ptr(r), _ptr(kl), int(kl_is_table),
                                     ids.numel(), ctypes.byref(params), _ptr(d_status), _stream()),
            "spo_tracker_update")
+
+
+def spo_tracker_update_repeats(ab, ids, r, kl, kl_is_table, ws, params, d_status):
+    _check(lib().spo_tracker_update_repeats(_ptr(ab), ab.shape[0], _ptr(ids), _ptr(r), _ptr(kl), int(kl_is_table),
+                                            ids.numel(), _ptr(ws), ws.numel() * ws.element_size(),
+                                            ctypes.byref(params), _ptr(d_status), _stream()),
+           "spo_tracker_update_repeats")
 
 
 def spo_loss_fwd(H, W, y, logp_old, mask, cu_seqlens, a_norm, loss, logp, lse, coef, seq_sums, ws, params,

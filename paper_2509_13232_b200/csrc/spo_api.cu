@@ -148,6 +148,22 @@ int32_t spo_tracker_update(float* ab, int64_t N, const int32_t* ids, const float
   return e == cudaSuccess ? SPO_OK : cuda_fail(e);
 }
 
+int32_t spo_tracker_update_repeats(float* ab, int64_t N, const int32_t* ids, const float* r, const float* kl,
+                                   int32_t kl_is_table, int32_t B, void* ws, size_t ws_bytes,
+                                   const spo_params* params, int32_t* d_status, void* stream) {
+  if (!params_ok(params) || !ab || B < 0 || (B > 0 && (!ids || !r || !kl || !ws))) return SPO_ERR_INVALID_ARG;
+  if (kl_is_table != 0 && kl_is_table != 1) return SPO_ERR_INVALID_ARG;
+  if (N < 1 || N >= ((int64_t)1 << 31) || B > kRepeatsMaxBatch) return SPO_ERR_BAD_SHAPE;
+  if (!aligned16(ab) || !aligned16(ids) || !aligned16(r) || !aligned16(kl) || !aligned16(ws))
+    return SPO_ERR_BAD_ALIGNMENT;
+  if (!device_is_sm100()) return SPO_ERR_UNSUPPORTED_ARCH;
+  const RepeatsWs L = repeats_ws_layout(B);
+  if (B > 0 && ws_bytes < L.total) return SPO_ERR_WORKSPACE_TOO_SMALL;
+  cudaError_t e = launch_tracker_update_repeats(ab, N, ids, r, kl, kl_is_table, B, (char*)ws, L, params->rho_min,
+                                                params->rho_max, params->d_half, d_status, (cudaStream_t)stream);
+  return e == cudaSuccess ? SPO_OK : cuda_fail(e);
+}
+
 static int32_t check_loss_shape(int32_t dtype, int64_t T, int32_t d, int32_t V) {
   if (dtype != SPO_DTYPE_F32 && dtype != SPO_DTYPE_BF16) return SPO_ERR_UNSUPPORTED_DTYPE;
   if (T < 0 || d < 1 || V < 1) return SPO_ERR_INVALID_ARG;
@@ -227,6 +243,9 @@ size_t spo_workspace_bytes(int32_t which, int64_t T, int32_t d, int32_t V, int64
     case SPO_WS_ADVANTAGES:
       if (B <= kAdvSingleBlockMax) return 256;
       return align_up(sizeof(double) * 2 * (size_t)adv_blocks(B), 256);
+    case SPO_WS_UPDATE_REPEATS:
+      if (B < 0 || B > kRepeatsMaxBatch) return 0;
+      return repeats_ws_layout(B).total;
     case SPO_WS_LOSS_FWD:
       if (T < 0 || V < 1) return 0;
       return fwd_ws_layout(T, d, V, (d % 64) == 0 ? SPO_DTYPE_BF16 : SPO_DTYPE_F32, B).total;

@@ -45,6 +45,16 @@ cudaError_t launch_tracker_update(float* ab, int64_t N, const int32_t* ids, cons
                                   float rho_min, float rho_max, float d_half,
                                   int32_t* d_status, cudaStream_t st);
 
+constexpr int kRepeatsMaxBatch = 65536;
+struct RepeatsWs {
+  size_t keys, zeroed_bytes, cur, slot_of, total;
+  int64_t hash_slots;
+};
+RepeatsWs repeats_ws_layout(int32_t B);
+cudaError_t launch_tracker_update_repeats(float* ab, int64_t N, const int32_t* ids, const float* r, const float* kl,
+                                          int kl_is_table, int32_t B, char* ws, const RepeatsWs& L, float rho_min,
+                                          float rho_max, float d_half, int32_t* d_status, cudaStream_t st);
+
 // ---- loss: pieces shared by the fp32 and bf16 paths ------------------------
 // Forward partial statistics of one vocabulary split, per token row:
 // (running max of z*log2(e), sum of 2^(z*log2(e) - max), target logit or -inf).

@@ -450,6 +450,76 @@ tracker_update_kernel(float2* __restrict__ ab, int64_t N, const int32_t* __restr
   }
 }
 
+// Tracker update for a batch in which a prompt may appear several times (batch SPO: each prompt is
+// rolled out G times against a shared baseline).  The occurrences of one prompt are applied in batch
+// order, one per round: in every round each prompt's earliest not-yet-applied occurrence wins an
+// integer atomicMin and performs its update, so the result does not depend on thread timing.
+// One block; keys/cur is an open-addressing table over the distinct ids (keys preset to 0, id+1 stored).
+__global__ void __launch_bounds__(1024)
+tracker_update_repeats_kernel(float2* __restrict__ ab, int64_t N, const int32_t* __restrict__ ids,
+                              const float* __restrict__ r, const float* __restrict__ kl, int kl_is_table, int32_t B,
+                              int32_t* keys, int32_t* cur, int32_t* slot_of, uint32_t slot_mask,
+                              float rho_min, float rho_max, float inv_d_half, int32_t* d_status) {
+  const int tid = threadIdx.x;
+  __shared__ int s_remaining;
+  for (int j = tid; j < B; j += 1024) {
+    const int32_t id = ids[j];
+    int32_t slot = -1;
+    if (id < 0 || (int64_t)id >= N) {
+      flag(d_status, SPO_DEV_ID_OUT_OF_RANGE);
+    } else {
+      const float rew = r[j];
+      const float div = kl_is_table ? kl[id] : kl[j];
+      if (isnan(rew) || isinf(rew) || isnan(div)) {
+        flag(d_status, SPO_DEV_NONFINITE);
+      } else {
+        uint32_t s = hash_id((uint32_t)id) & slot_mask;
+        for (uint32_t probe = 0; probe <= slot_mask; ++probe) {
+          const int32_t prev = atomicCAS(&keys[s], 0, id + 1);
+          if (prev == 0 || prev == id + 1) { slot = (int32_t)s; break; }
+          s = (s + 1) & slot_mask;
+        }
+      }
+    }
+    slot_of[j] = slot;
+  }
+  __syncthreads();
+  for (int round = 0; round <= B; ++round) {
+    if (tid == 0) s_remaining = 0;
+    for (int j = tid; j < B; j += 1024) {
+      const int32_t slot = slot_of[j];
+      if (slot >= 0) cur[slot] = 0x7fffffff;
+    }
+    __syncthreads();
+    for (int j = tid; j < B; j += 1024) {
+      const int32_t slot = slot_of[j];
+      if (slot >= 0) atomicMin(&cur[slot], j);
+    }
+    __syncthreads();
+    for (int j = tid; j < B; j += 1024) {
+      const int32_t slot = slot_of[j];
+      if (slot < 0) continue;
+      if (__ldcg(&cur[slot]) == j) {                  // read at L2, where the atomics were performed
+        const int32_t id = ids[j];
+        const float rew = r[j];
+        const float div = kl_is_table ? kl[id] : kl[j];
+        float rho = exp2f(-div * inv_d_half);
+        rho = fminf(fmaxf(rho, rho_min), rho_max);
+        float2 e = ab[id];
+        e.x = fmaf(rho, e.x, rew);
+        e.y = fmaf(rho, e.y, 1.0f - rew);
+        ab[id] = e;
+        slot_of[j] = -1;
+      } else {
+        s_remaining = 1;
+      }
+    }
+    __syncthreads();
+    if (s_remaining == 0) break;
+    __syncthreads();
+  }
+}
+
 }  // namespace
 
 // ---------------------------------------------------------------------------
@@ -501,6 +571,33 @@ cudaError_t launch_sample(const float* ab, int64_t N, const float* u, int32_t M,
       d_status);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   sample_accept_kernel<<<1, 1024, 0, st>>>(cand, M, B, keys, vals, (uint32_t)(L.hash_slots - 1), out_ids, d_status);
+  return cudaGetLastError();
+}
+
+RepeatsWs repeats_ws_layout(int32_t B) {
+  RepeatsWs L{};
+  int64_t slots = 64;
+  while (slots < 2 * (int64_t)B) slots <<= 1;
+  L.hash_slots = slots;
+  size_t off = 0;
+  L.keys = off;    off = align_up(off + sizeof(int32_t) * (size_t)slots, 256);
+  L.zeroed_bytes = off;
+  L.cur = off;     off = align_up(off + sizeof(int32_t) * (size_t)slots, 256);
+  L.slot_of = off; off = align_up(off + sizeof(int32_t) * (size_t)(B > 0 ? B : 1), 256);
+  L.total = off;
+  return L;
+}
+
+cudaError_t launch_tracker_update_repeats(float* ab, int64_t N, const int32_t* ids, const float* r, const float* kl,
+                                          int kl_is_table, int32_t B, char* ws, const RepeatsWs& L, float rho_min,
+                                          float rho_max, float d_half, int32_t* d_status, cudaStream_t st) {
+  if (B == 0) return cudaSuccess;
+  cudaError_t e = cudaMemsetAsync(ws + L.keys, 0, L.zeroed_bytes, st);
+  if (e != cudaSuccess) return e;
+  tracker_update_repeats_kernel<<<1, 1024, 0, st>>>(
+      reinterpret_cast<float2*>(ab), N, ids, r, kl, kl_is_table, B, reinterpret_cast<int32_t*>(ws + L.keys),
+      reinterpret_cast<int32_t*>(ws + L.cur), reinterpret_cast<int32_t*>(ws + L.slot_of),
+      (uint32_t)(L.hash_slots - 1), rho_min, rho_max, 1.0f / d_half, d_status);
   return cudaGetLastError();
 }
 

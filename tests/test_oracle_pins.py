@@ -528,3 +528,43 @@ def test_sequence_mean_gradients_against_finite_differences():
             arr[idx] = keep
             num[idx] = (up - dn) / (2 * step)
         assert np.linalg.norm(num - grad) <= 1e-6 * np.linalg.norm(grad)
+
+
+def test_general_rewards_follow_the_ema_form():
+    """Sec. 3.1, last sentence: for non-binary rewards the same EMA tracks the value.  With
+    (alpha, beta) carried as before, alpha/(alpha+beta) obeys that EMA for any real reward."""
+    rng = np.random.default_rng(23)
+    v, n = 0.3, 8.0
+    a, b = np.array([v * n]), np.array([(1 - v) * n])
+    for _ in range(200):
+        r = float(rng.uniform(0.0, 1.0))
+        kl = float(rng.lognormal(-4, 1))
+        rho = O.forgetting_factor([kl], 0.1)[0]
+        v = O.ema_update(v, n, r, rho)
+        n = rho * n + 1.0
+        a, b = O.tracker_update(a, b, [0], [r], [kl], 0.1)
+        assert abs(O.value_estimate(a, b)[0] - v) < 1e-12
+        assert abs((a + b)[0] - n) < 1e-12
+    # a constant fractional reward is tracked to that reward
+    a, b = O.tracker_init(np.array([0.9]), 0.875)
+    for _ in range(400):
+        a, b = O.tracker_update(a, b, [0], [0.37], [0.05], 0.1)
+    assert abs(O.value_estimate(a, b)[0] - 0.37) < 1e-9
+
+
+def test_repeated_ids_apply_in_batch_order():
+    """Batch SPO: several outcomes of one prompt in a batch compose the update in order."""
+    a0, b0 = np.array([2.0, 1.0]), np.array([3.0, 4.0])
+    ids, r, kl = [0, 1, 0, 0], [1.0, 0.0, 0.0, 1.0], [0.01, 0.02, 0.2, 0.005]
+    a, b = O.tracker_update(a0, b0, ids, r, kl, 0.1)
+    sa, sb = a0.copy(), b0.copy()
+    for j in range(4):                               # one call per entry
+        sa, sb = O.tracker_update(sa, sb, [ids[j]], [r[j]], [kl[j]], 0.1)
+    np.testing.assert_array_equal(a, sa)
+    np.testing.assert_array_equal(b, sb)
+    # order matters: swapping the two zero/one rewards of prompt 0 changes the estimate
+    a2, b2 = O.tracker_update(a0, b0, [0, 1, 0, 0], [1.0, 0.0, 1.0, 0.0], kl, 0.1)
+    assert abs(O.value_estimate(a, b)[0] - O.value_estimate(a2, b2)[0]) > 1e-3
+    # every copy of a prompt sees the same pre-update baseline
+    adv = O.raw_advantage(a0, b0, ids, r)
+    assert adv[0] == 1.0 - 0.4 and adv[2] == 0.0 - 0.4 and adv[3] == 1.0 - 0.4
