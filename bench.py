@@ -139,9 +139,9 @@ class Step:
         self.ws_bwd = torch.empty(self.ws_bwd_bytes, **u8)
         chunk_rows = self.ws_bwd_bytes // (((V + 255) // 256) * 256 * 2)
         self.bwd_chunks = -(-self.T // chunk_rows)
-        # kernels launched by one step: sampling 4, advantages 1, update 1,
-        # forward 3 (count, contraction, finalise), backward 3 per chunk
-        self.launches = 4 + 1 + 1 + 3 + 3 * self.bwd_chunks
+        # kernels launched by one step: sampling 3 (tile sums, search, accept), advantages 1, update 1,
+        # forward 3 (count, contraction, finalise), backward 3 per chunk (memsets are not counted)
+        self.launches = 3 + 1 + 1 + 3 + 3 * self.bwd_chunks
         self.flops_fwd = 2.0 * self.T * d * V
         self.flops_bwd = 6.0 * self.T * d * V
 
@@ -459,7 +459,7 @@ def main():
         run_reference(args, rank, world)
         return
     if args.cpu_tokens is None:
-        args.cpu_tokens = 256
+        args.cpu_tokens = 512
     if world > 1:
         import torch
         import torch.distributed as dist
