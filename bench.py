@@ -226,33 +226,52 @@ def run_ours(args, rank, world, local_rank):
     host = {k: D[k].cpu().pin_memory() for k in ("h", "y", "logp_old", "mask", "cu_seqlens")}
     host["rewards"] = step.rewards.cpu().pin_memory()
     host["uniforms"] = step.uniforms.cpu().pin_memory()
-    devbuf = {k: torch.empty_like(D[k]) for k in ("h", "y", "logp_old", "mask", "cu_seqlens")}
+    names = ("h", "y", "logp_old", "mask", "cu_seqlens")
+    # two sets of device input buffers: a copy stream fills one while the step runs on the other
+    bufs = [{k: torch.empty_like(D[k]) for k in names} for _ in range(2)]
+    small_bufs = [{"rewards": torch.empty_like(step.rewards), "uniforms": torch.empty_like(step.uniforms)}
+                  for _ in range(2)]
     loss_host = torch.zeros(4, dtype=torch.float32).pin_memory()
     ids_host = torch.zeros(step.S, dtype=torch.int32).pin_memory()
     h2d = sum(v.numel() * v.element_size() for v in host.values())
     d2h = loss_host.numel() * 4 + ids_host.numel() * 4
+    main = torch.cuda.current_stream()
+    copy_stream = torch.cuda.Stream(device=device)
 
-    def e2e_step():
-        for k in devbuf:
-            devbuf[k].copy_(host[k], non_blocking=True)
-        step.rewards.copy_(host["rewards"], non_blocking=True)
-        step.uniforms.copy_(host["uniforms"], non_blocking=True)
-        step.small()
-        step.fwd(devbuf["h"], devbuf["y"], devbuf["logp_old"], devbuf["mask"], devbuf["cu_seqlens"])
-        step.bwd(devbuf["h"], devbuf["y"])
-        loss_host.copy_(step.loss, non_blocking=True)
-        ids_host.copy_(step.ids, non_blocking=True)
+    def e2e_run(n_steps):
+        """n_steps whole steps, every one fed from pinned host memory; returns device milliseconds."""
+        ready = [torch.cuda.Event() for _ in range(n_steps)]
+        done = [torch.cuda.Event() for _ in range(n_steps)]
+        s0, s1 = ev(), ev()
+        s0.record(main)
+        copy_stream.wait_event(s0)                      # the first copy starts inside the timed region
+        for i in range(n_steps):
+            b = i % 2
+            with torch.cuda.stream(copy_stream):
+                if i >= 2:
+                    copy_stream.wait_event(done[i - 2])  # the step that last used this buffer has finished
+                for k in names:
+                    bufs[b][k].copy_(host[k], non_blocking=True)
+                small_bufs[b]["rewards"].copy_(host["rewards"], non_blocking=True)
+                small_bufs[b]["uniforms"].copy_(host["uniforms"], non_blocking=True)
+                ready[i].record(copy_stream)
+            main.wait_event(ready[i])
+            step.rewards, step.uniforms = small_bufs[b]["rewards"], small_bufs[b]["uniforms"]
+            step.small()
+            step.fwd(bufs[b]["h"], bufs[b]["y"], bufs[b]["logp_old"], bufs[b]["mask"], bufs[b]["cu_seqlens"])
+            step.bwd(bufs[b]["h"], bufs[b]["y"])
+            loss_host.copy_(step.loss, non_blocking=True)
+            ids_host.copy_(step.ids, non_blocking=True)
+            done[i].record(main)
+        s1.record(main)
+        torch.cuda.synchronize()
+        return s0.elapsed_time(s1)
 
-    e2e_steps = max(1, min(args.steps, 3))
-    e2e_step()
+    e2e_steps = max(1, args.steps)
+    e2e_run(1)
     barrier()
-    s0, s1 = ev(), ev()
-    s0.record()
-    for _ in range(e2e_steps):
-        e2e_step()
-    s1.record()
+    e2e_ms = e2e_run(e2e_steps)
     barrier()
-    e2e_ms = s0.elapsed_time(s1)
 
     (total_ms, e2e_ms, t_fwd, t_bwd, t_small), tokens_all = reduce_over_ranks(
         [total_ms, e2e_ms, t_fwd, t_bwd, t_small], step.n_tok, world, device)
