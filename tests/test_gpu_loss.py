@@ -216,3 +216,14 @@ def test_sequence_mean_aggregation(bf16):
         got = run_loss(lb, params=params, mask_none=mask_none)
         want = oracle_loss(lb, params=params, mask_none=mask_none)
         check(lb, got, want, *tol)
+
+
+def test_results_are_bitwise_reproducible():
+    """Fixed reduction orders everywhere: two runs on the same inputs agree bit for bit
+    (loss fold, split merge, chunked dW accumulation)."""
+    lb = inputs.loss_batch(95, [2000, 1500, 1100, 97, 5300], 128, 1200, 0.05, True, 0.3, target="softmax", mask_p=0.1)
+    a = run_loss(lb, grad_loss=0.9)
+    b = run_loss(lb, grad_loss=0.9)
+    assert a["loss"] == b["loss"]
+    for k in ("logp", "lse", "coef", "dH", "dW", "seq_sums"):
+        np.testing.assert_array_equal(a[k], b[k])

@@ -317,3 +317,16 @@ def test_batch_spo_update_skips_bad_entries():
     a1, b1 = O.tracker_update([2.0, 1.0], [2.0, 3.0], [0, 1], [1.0, 0.0], [np.float64(np.float32(0.01))] * 2,
                               float(np.float32(p.d_half)))
     np.testing.assert_allclose(ab_t.cpu().numpy(), np.stack([a1, b1], 1), rtol=RTOL)
+
+
+@pytest.mark.parametrize("n", [1, 2047, 4097])
+def test_sampling_weight_output_for_odd_table_sizes(n):
+    rng = np.random.default_rng(300 + n)
+    ab = rng.uniform(0.0, 12.0, (n, 2)).astype(np.float32)
+    u = inputs.uniforms_f32(rng, 32)
+    p = B().default_params()
+    ids, w, st = gpu_sample(dev(ab), u, 1, p, want_w=True)
+    want = O.sampling_weights_f32(ab[:, 0], ab[:, 1], np.float32(p.eps_explore))
+    assert st == 0
+    np.testing.assert_array_equal(w, want)
+    np.testing.assert_array_equal(ids, O.sample_prompts(want, u, 1))
