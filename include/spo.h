@@ -80,6 +80,10 @@ typedef struct spo_params {
   float   norm_eps;
   int32_t norm_ddof;
   int32_t agg_mode;       /* SPO_AGG_*: how E_{s,t} of the objective weights tokens */
+  /* Data-parallel training: when the mini-batch is spread over several ranks, the denominators of
+   * the objective are those of the whole mini-batch.  0 = use this call's own counts. */
+  int32_t global_tokens;     /* unmasked tokens of the whole mini-batch (n_tok) */
+  int32_t global_responses;  /* responses with an unmasked token in the whole mini-batch (S_act) */
 } spo_params;
 
 int32_t spo_default_params(spo_params* p /* host, out */);
@@ -129,13 +133,23 @@ int32_t spo_sample_prompts(const float* ab, int64_t N, const float* uniforms, in
  *   r       device in  [B] fp32 rewards
  *   a_raw   device out [B] fp32, optional
  *   a_norm  device out [B] fp32
- *   stats   device out [4] fp32 = (mu, sigma, B, 0), optional
+ *   stats   device out [4] fp32 = (mu, sigma, B, M2 = sum (A-mu)^2), optional; (mu, M2, B) of
+ *           several ranks merge exactly (pairwise: M2 = M2a + M2b + (mub-mua)^2 Ba Bb/(Ba+Bb))
  *   ws      device scratch, spo_workspace_bytes(SPO_WS_ADVANTAGES, ..., B, ...) bytes
  * An id outside [0,N) sets SPO_DEV_ID_OUT_OF_RANGE and contributes A = 0.
  */
 int32_t spo_advantages(const float* ab, int64_t N, const int32_t* ids, const float* r, int32_t B,
                        float* a_raw, float* a_norm, float* stats, void* ws, size_t ws_bytes,
                        const spo_params* params, int32_t* d_status, void* stream);
+
+/*
+ * Second half of spo_advantages for a batch whose statistics were merged elsewhere (data-parallel
+ * ranks each call spo_advantages for a_raw and stats, merge (mu, M2, B) on the host, then call
+ * this): a_norm_j = (a_raw_j - mu) / (sigma + norm_eps)  (Sec. 3.2, global normalisation).
+ * a_raw and a_norm may be the same buffer.
+ */
+int32_t spo_advantages_apply(const float* a_raw, int32_t B, float mu, float sigma, float* a_norm,
+                             const spo_params* params, void* stream);
 
 /*
  * spo_advantages with no scratch argument and no allocation anywhere.  (The paper has no
@@ -206,7 +220,9 @@ int32_t spo_tracker_update_repeats(float* ab, int64_t N, const int32_t* ids, con
  *   loss = - sum_t u_t s_t with token weights u_t that sum to one: u_t = mask_t / n_tok,
  *   n_tok = sum_t mask_t (SPO_AGG_TOKEN_MEAN), or u_t = mask_t / (S_act * n_seq(t)) with n_s the
  *   unmasked tokens of response s and S_act the responses that have any (SPO_AGG_SEQ_MEAN);
- *   loss = 0 if n_tok = 0;
+ *   loss = 0 if n_tok = 0.  With params->global_tokens / global_responses set, n_tok and S_act are
+ *   those values (the whole data-parallel mini-batch) and `loss` is this rank's share: the ranks'
+ *   losses and dW add up to the mini-batch's, dH rows are final;
  *   coef_t = d loss / d logp_t = -u_t * a * ratio * [gradient passes the clip].
  *
  *   H           device in  [T][d], row-major, dtype as given (bf16: d % 64 == 0)

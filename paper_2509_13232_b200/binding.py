@@ -25,7 +25,7 @@ AGG_TOKEN_MEAN, AGG_SEQ_MEAN = 0, 1
 
 EXPORTS = [
     "spo_default_params", "spo_tracker_init", "spo_sample_prompts", "spo_advantages",
-    "spo_advantages_static",
+    "spo_advantages_static", "spo_advantages_apply",
     "spo_tracker_update", "spo_tracker_update_repeats", "spo_loss_fwd", "spo_loss_bwd", "spo_workspace_bytes",
     "spo_status_string", "spo_last_cuda_error", "spo_version", "spo_selftest_bounded_wait",
 ]
@@ -35,7 +35,7 @@ class SpoParams(Structure):
     _fields_ = [
         ("rho_min", c_float), ("rho_max", c_float), ("d_half", c_float), ("eps_explore", c_float),
         ("clip_lo", c_float), ("clip_hi", c_float), ("norm_eps", c_float), ("norm_ddof", c_int32),
-        ("agg_mode", c_int32),
+        ("agg_mode", c_int32), ("global_tokens", c_int32), ("global_responses", c_int32),
     ]
 
 
@@ -69,6 +69,7 @@ def lib():
                                      c_void_p, c_void_p, c_size_t, P, c_void_p, c_void_p]
         L.spo_advantages_static.argtypes = [c_void_p, c_int64, c_void_p, c_void_p, c_int32, c_void_p, c_void_p,
                                             c_void_p, P, c_void_p, c_void_p]
+        L.spo_advantages_apply.argtypes = [c_void_p, c_int32, c_float, c_float, c_void_p, P, c_void_p]
         L.spo_tracker_update.argtypes = [c_void_p, c_int64, c_void_p, c_void_p, c_void_p, c_int32, c_int32,
                                          P, c_void_p, c_void_p]
         L.spo_tracker_update_repeats.argtypes = [c_void_p, c_int64, c_void_p, c_void_p, c_void_p, c_int32, c_int32,
@@ -144,6 +145,11 @@ def spo_advantages(ab, ids, r, a_raw, a_norm, stats, ws, params, d_status):
     _check(lib().spo_advantages(_ptr(ab), ab.shape[0], _ptr(ids), _ptr(r), ids.numel(), _ptr(a_raw), _ptr(a_norm),
                                 _ptr(stats), _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size(),
                                 ctypes.byref(params), _ptr(d_status), _stream()), "spo_advantages")
+
+
+def spo_advantages_apply(a_raw, mu, sigma, a_norm, params):
+    _check(lib().spo_advantages_apply(_ptr(a_raw), a_raw.numel(), c_float(mu), c_float(sigma), _ptr(a_norm),
+                                      ctypes.byref(params), _stream()), "spo_advantages_apply")
 
 
 ADVANTAGES_STATIC_MAX_B = 4194304

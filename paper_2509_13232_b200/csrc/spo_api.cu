@@ -68,6 +68,7 @@ static bool params_ok(const spo_params* p) {
   if (!(p->norm_eps >= 0.0f)) return false;
   if (p->norm_ddof != 0 && p->norm_ddof != 1) return false;
   if (p->agg_mode != SPO_AGG_TOKEN_MEAN && p->agg_mode != SPO_AGG_SEQ_MEAN) return false;
+  if (p->global_tokens < 0 || p->global_responses < 0) return false;
   return true;
 }
 
@@ -88,6 +89,8 @@ int32_t spo_default_params(spo_params* p) {
   p->norm_eps = 1e-8f;
   p->norm_ddof = 0;
   p->agg_mode = SPO_AGG_TOKEN_MEAN;
+  p->global_tokens = 0;
+  p->global_responses = 0;
   return SPO_OK;
 }
 
@@ -132,6 +135,16 @@ int32_t spo_advantages(const float* ab, int64_t N, const int32_t* ids, const flo
   }
   cudaError_t e = launch_advantages(ab, N, ids, r, B, a_raw, a_norm, stats, (char*)ws, params->norm_eps,
                                     params->norm_ddof, d_status, (cudaStream_t)stream);
+  return e == cudaSuccess ? SPO_OK : cuda_fail(e);
+}
+
+int32_t spo_advantages_apply(const float* a_raw, int32_t B, float mu, float sigma, float* a_norm,
+                             const spo_params* params, void* stream) {
+  if (!params_ok(params) || B < 0 || (B > 0 && (!a_raw || !a_norm))) return SPO_ERR_INVALID_ARG;
+  if (!(sigma >= 0.0f) || !(mu == mu)) return SPO_ERR_INVALID_ARG;
+  if (!aligned16(a_raw) || !aligned16(a_norm)) return SPO_ERR_BAD_ALIGNMENT;
+  if (!device_is_sm100()) return SPO_ERR_UNSUPPORTED_ARCH;
+  cudaError_t e = launch_advantages_apply(a_raw, B, mu, sigma, params->norm_eps, a_norm, (cudaStream_t)stream);
   return e == cudaSuccess ? SPO_OK : cuda_fail(e);
 }
 
@@ -202,7 +215,7 @@ int32_t spo_loss_fwd(const void* H, const void* W, int32_t dtype, const int32_t*
   if (e != cudaSuccess) return cuda_fail(e);
   e = launch_fwd_finalize(partials, L.nsplit, y, logp_old, mask, cu_seqlens, a_norm, T, V, S, params->clip_lo,
                           params->clip_hi, loss, logp, lse, coef, seq_sums, block_sums, counters, seq_cnt, params->agg_mode,
-                          L.fin_blocks,
+                          params->global_tokens, params->global_responses, L.fin_blocks,
                           d_status, st);
   return e == cudaSuccess ? SPO_OK : cuda_fail(e);
 }

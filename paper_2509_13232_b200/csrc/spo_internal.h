@@ -37,6 +37,8 @@ cudaError_t launch_sample(const float* ab, int64_t N, const float* u, int32_t M,
 // ---- advantages / tracker ------------------------------------------------
 constexpr int kAdvSingleBlockMax = 8192;
 int adv_blocks(int32_t B);
+cudaError_t launch_advantages_apply(const float* a_raw, int32_t B, float mu, float sigma, float norm_eps, float* a_norm,
+                                    cudaStream_t st);
 cudaError_t launch_advantages(const float* ab, int64_t N, const int32_t* ids, const float* r, int32_t B,
                               float* a_raw, float* a_norm, float* stats, char* ws,
                               float norm_eps, int32_t ddof, int32_t* d_status, cudaStream_t st);
@@ -84,6 +86,7 @@ cudaError_t launch_fwd_finalize(const FwdPartial* partials, int nsplit, const in
                                 float clip_lo, float clip_hi,
                                 float* loss, float* logp, float* lse, float* coef, float* seq_sums,
                                 double* block_sums, int32_t* counters, const int32_t* seq_cnt, int agg_mode,
+                                int32_t global_tokens, int32_t global_responses,
                                 int64_t fin_blocks, int32_t* d_status, cudaStream_t st);
 
 // fp32 SIMT path

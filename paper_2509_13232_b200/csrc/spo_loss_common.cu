@@ -80,10 +80,12 @@ fwd_finalize_kernel(const FwdPartial* __restrict__ partials, int nsplit, const i
                     int64_t T, int32_t V, int32_t S, float clip_lo, float clip_hi,
                     float* __restrict__ loss, float* __restrict__ logp_out, float* __restrict__ lse_out,
                     float* __restrict__ coef_out, double* block_sums, int32_t* counters,
-                    const int32_t* __restrict__ seq_cnt, int agg_mode, int32_t* d_status) {
+                    const int32_t* __restrict__ seq_cnt, int agg_mode, int32_t global_tokens,
+                    int32_t global_responses, int32_t* d_status) {
   const int64_t t = (int64_t)blockIdx.x * kFinalizeThreads + threadIdx.x;
-  const int32_t n_tok = counters[0];
-  const int32_t s_act = counters[2];
+  // denominators of the expectation: this call's own counts, or the whole data-parallel batch's
+  const int32_t n_tok = global_tokens > 0 ? global_tokens : counters[0];
+  const int32_t s_act = global_responses > 0 ? global_responses : counters[2];
   double contrib = 0.0;
   if (t < T) {
     float m2 = -CUDART_INF_F, zt = -CUDART_INF_F;
@@ -340,10 +342,11 @@ cudaError_t launch_fwd_finalize(const FwdPartial* partials, int nsplit, const in
                                 float clip_lo, float clip_hi,
                                 float* loss, float* logp, float* lse, float* coef, float* seq_sums,
                                 double* block_sums, int32_t* counters, const int32_t* seq_cnt, int agg_mode,
+                                int32_t global_tokens, int32_t global_responses,
                                 int64_t fin_blocks, int32_t* d_status, cudaStream_t st) {
   fwd_finalize_kernel<<<(unsigned)fin_blocks, kFinalizeThreads, 0, st>>>(
       partials, nsplit, y, logp_old, mask, cu_seqlens, a_norm, T, V, S, clip_lo, clip_hi,
-      loss, logp, lse, coef, block_sums, counters, seq_cnt, agg_mode, d_status);
+      loss, logp, lse, coef, block_sums, counters, seq_cnt, agg_mode, global_tokens, global_responses, d_status);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   if (seq_sums && S > 0) {

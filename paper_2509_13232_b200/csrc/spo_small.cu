@@ -318,7 +318,8 @@ __device__ __forceinline__ void block_sum2(double& a, double& b, double* s_a, do
   __syncthreads();
 }
 
-__device__ __forceinline__ void mean_sigma(double sum, double sumsq, int32_t B, int32_t ddof, float& mu, float& sigma) {
+__device__ __forceinline__ void mean_sigma(double sum, double sumsq, int32_t B, int32_t ddof, float& mu, float& sigma,
+                                           float& m2) {
   double m = B > 0 ? sum / B : 0.0;
   double ss = sumsq - sum * m;                 // sum (A - mu)^2
   if (ss < 0.0) ss = 0.0;
@@ -326,6 +327,7 @@ __device__ __forceinline__ void mean_sigma(double sum, double sumsq, int32_t B, 
   double var = den > 0 ? ss / den : 0.0;
   mu = (float)m;
   sigma = (float)sqrt(var);
+  m2 = (float)ss;
 }
 
 // Whole batch in one block: one launch for gather, statistics and normalisation.
@@ -352,15 +354,15 @@ advantages_single_kernel(const float2* __restrict__ ab, int64_t N, const int32_t
   }
   if (bad) flag(d_status, SPO_DEV_ID_OUT_OF_RANGE);
   block_sum2<1024>(sum, sumsq, s_a, s_b);
-  float mu, sigma;
-  mean_sigma(sum, sumsq, B, ddof, mu, sigma);
+  float mu, sigma, m2;
+  mean_sigma(sum, sumsq, B, ddof, mu, sigma, m2);
   const float inv = 1.0f / (sigma + norm_eps);
 #pragma unroll
   for (int j = 0; j < PER; ++j) {
     int i = j * 1024 + threadIdx.x;
     if (i < B) a_norm[i] = (a[j] - mu) * inv;
   }
-  if (stats && threadIdx.x == 0) { stats[0] = mu; stats[1] = sigma; stats[2] = (float)B; stats[3] = 0.0f; }
+  if (stats && threadIdx.x == 0) { stats[0] = mu; stats[1] = sigma; stats[2] = (float)B; stats[3] = m2; }
 }
 
 // Large batches, pass 1: raw advantages (stored into `tmp`) and per-block (sum, sum of squares).
@@ -395,13 +397,13 @@ advantages_normalise_kernel(const double2* __restrict__ partials, int n_partials
     sumsq += p.y;
   }
   block_sum2<256>(sum, sumsq, s_a, s_b);
-  float mu, sigma;
-  mean_sigma(sum, sumsq, B, ddof, mu, sigma);
+  float mu, sigma, m2;
+  mean_sigma(sum, sumsq, B, ddof, mu, sigma, m2);
   const float inv = 1.0f / (sigma + norm_eps);
   for (int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x; i < B; i += (int64_t)gridDim.x * 256)
     a_norm[i] = (tmp[i] - mu) * inv;
   if (stats && blockIdx.x == 0 && threadIdx.x == 0) {
-    stats[0] = mu; stats[1] = sigma; stats[2] = (float)B; stats[3] = 0.0f;
+    stats[0] = mu; stats[1] = sigma; stats[2] = (float)B; stats[3] = m2;
   }
 }
 
@@ -520,6 +522,13 @@ tracker_update_repeats_kernel(float2* __restrict__ ab, int64_t N, const int32_t*
   }
 }
 
+// Normalisation with statistics supplied by the caller (e.g. merged over data-parallel ranks).
+__global__ void __launch_bounds__(256)
+advantages_apply_kernel(const float* a_raw, int32_t B, float mu, float inv, float* a_norm) {
+  for (int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x; i < B; i += (int64_t)gridDim.x * 256)
+    a_norm[i] = (a_raw[i] - mu) * inv;
+}
+
 }  // namespace
 
 // ---------------------------------------------------------------------------
@@ -598,6 +607,13 @@ cudaError_t launch_tracker_update_repeats(float* ab, int64_t N, const int32_t* i
       reinterpret_cast<float2*>(ab), N, ids, r, kl, kl_is_table, B, reinterpret_cast<int32_t*>(ws + L.keys),
       reinterpret_cast<int32_t*>(ws + L.cur), reinterpret_cast<int32_t*>(ws + L.slot_of),
       (uint32_t)(L.hash_slots - 1), rho_min, rho_max, 1.0f / d_half, d_status);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_advantages_apply(const float* a_raw, int32_t B, float mu, float sigma, float norm_eps, float* a_norm,
+                                    cudaStream_t st) {
+  if (B == 0) return cudaSuccess;
+  advantages_apply_kernel<<<adv_blocks(B), 256, 0, st>>>(a_raw, B, mu, 1.0f / (sigma + norm_eps), a_norm);
   return cudaGetLastError();
 }
 

@@ -1,0 +1,74 @@
+"""Host-side glue for data-parallel training over responses (one process per GPU).
+
+Each rank holds its share of the mini-batch's responses and the replicated W and tracker table.
+Three small exchanges make the ranks' results those of the whole mini-batch:
+
+  1. advantage statistics: every rank calls spo_advantages for its raw advantages and
+     (mu, sigma, B, M2); `global_advantage_stats` gathers the 16-byte records, merges them and
+     returns the mini-batch mu and sigma for spo_advantages_apply;
+  2. denominators of the objective: `global_counts` sums the ranks' unmasked-token and active-
+     response counts; they go into spo_params.global_tokens / global_responses;
+  3. after spo_loss_bwd: `allreduce_sum` on dW (and on the scalar loss); dH rows are already final.
+
+Only torch.distributed calls and a few lines of float64 arithmetic live here; nothing of the
+path itself.
+"""
+
+from __future__ import annotations
+
+import math
+
+
+def merge_moments(parts):
+    """Merge (mean, M2, count) records, M2 = sum of squared deviations from the record's own mean
+    (pairwise update of Chan et al.).  Returns (mean, M2, count)."""
+    mean, m2, n = 0.0, 0.0, 0.0
+    for mu_b, m2_b, n_b in parts:
+        mu_b, m2_b, n_b = float(mu_b), float(m2_b), float(n_b)
+        if n_b <= 0:
+            continue
+        tot = n + n_b
+        delta = mu_b - mean
+        mean += delta * n_b / tot
+        m2 += m2_b + delta * delta * n * n_b / tot
+        n = tot
+    return mean, m2, n
+
+
+def sigma_from(m2, n, ddof=0):
+    den = n - ddof
+    return math.sqrt(m2 / den) if den > 0 else 0.0
+
+
+def global_advantage_stats(stats, ddof=0, group=None):
+    """`stats` is this rank's [4] tensor (mu, sigma, B, M2) from spo_advantages.  Returns the
+    mini-batch (mu, sigma) as Python floats, identical on every rank."""
+    import torch
+    import torch.distributed as dist
+    world = dist.get_world_size(group) if dist.is_initialized() else 1
+    if world == 1:
+        rows = [stats.detach().cpu().double()]
+    else:
+        bucket = [torch.empty_like(stats) for _ in range(world)]
+        dist.all_gather(bucket, stats.contiguous(), group=group)
+        rows = [b.detach().cpu().double() for b in bucket]
+    mean, m2, n = merge_moments([(float(r[0]), float(r[3]), float(r[2])) for r in rows])
+    return mean, sigma_from(m2, n, ddof)
+
+
+def global_counts(n_tokens, n_responses, device=None, group=None):
+    """Sum of the ranks' unmasked-token and active-response counts."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([int(n_tokens), int(n_responses)], dtype=torch.int64, device=device)
+    if dist.is_initialized() and dist.get_world_size(group) > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.SUM, group=group)
+    return int(t[0].item()), int(t[1].item())
+
+
+def allreduce_sum(tensor, group=None):
+    """In-place sum over ranks (dW, the scalar loss)."""
+    import torch.distributed as dist
+    if dist.is_initialized() and dist.get_world_size(group) > 1:
+        dist.all_reduce(tensor, op=dist.ReduceOp.SUM, group=group)
+    return tensor

@@ -1,0 +1,77 @@
+"""Data-parallel decomposition on one GPU: the mini-batch is split over two emulated ranks that run
+one after the other; with the merged advantage statistics and the global denominators their losses
+and dW add up to, and their dH rows equal, what the oracle gives for the whole mini-batch."""
+
+import numpy as np
+import pytest
+
+from oracle import spo_oracle as O
+from paper_2509_13232_b200 import dp, inputs
+from tests.helpers import dev, rel_fro, run_loss, status_word, ws_bytes
+
+pytestmark = pytest.mark.gpu
+
+
+def _slice_batch(lb, s0, s1):
+    t0, t1 = int(lb.cu_seqlens[s0]), int(lb.cu_seqlens[s1])
+    return inputs.LossBatch(h=lb.h[t0:t1], w=lb.w, y=lb.y[t0:t1], logp_old=lb.logp_old[t0:t1], mask=lb.mask[t0:t1],
+                            cu_seqlens=(lb.cu_seqlens[s0:s1 + 1] - lb.cu_seqlens[s0]).astype(np.int32),
+                            a_norm=lb.a_norm[s0:s1], bf16=lb.bf16)
+
+
+@pytest.mark.parametrize("agg", [0, 1])
+def test_two_emulated_ranks_equal_the_whole_mini_batch(agg):
+    import torch
+    from paper_2509_13232_b200 import binding as B
+    rng = np.random.default_rng(77)
+    lengths = [300, 40, 0, 520, 75, 260, 9, 410]
+    n = 5000
+    ab = rng.uniform(0.1, 12.0, (n, 2)).astype(np.float32)
+    ids = rng.permutation(n)[:len(lengths)].astype(np.int32)
+    rewards = (rng.random(len(lengths)) < 0.5).astype(np.float32)
+    lb = inputs.loss_batch(78, lengths, 128, 900, 0.05, True, 0.3, target="softmax", mask_p=0.1,
+                           a_norm=np.zeros(len(lengths), np.float32))
+    lb.mask[int(lb.cu_seqlens[4]):int(lb.cu_seqlens[5])] = 0          # one response fully masked
+    # oracle on the whole mini-batch
+    raw = O.raw_advantage(ab[:, 0].astype(np.float64), ab[:, 1].astype(np.float64), ids, rewards)
+    a_norm, mu, sigma = O.normalise_advantages(raw, 0, 1e-8)
+    lb.a_norm = a_norm.astype(np.float32)
+    want = O.loss_forward(lb.h, lb.w, lb.y, lb.logp_old, lb.mask, lb.cu_seqlens, lb.a_norm, agg_mode=agg)
+    want_dh, want_dw = O.loss_backward(lb.h, lb.w, lb.y, want["lse"], want["coef"])
+    # two ranks: responses [0,3) and [3,8)
+    splits = [(0, 3), (3, 8)]
+    ab_t = dev(ab)
+    p0 = B.default_params()
+    recs, raws = [], []
+    for s0, s1 in splits:
+        a_raw = torch.empty(s1 - s0, dtype=torch.float32, device="cuda")
+        a_tmp = torch.empty_like(a_raw)
+        stats = torch.zeros(4, dtype=torch.float32, device="cuda")
+        B.spo_advantages(ab_t, dev(ids[s0:s1]), dev(rewards[s0:s1]), a_raw, a_tmp, stats, ws_bytes(B.WS_ADVANTAGES, B=s1 - s0),
+                         p0, status_word())
+        torch.cuda.synchronize()
+        r = stats.cpu().numpy()
+        recs.append((r[0], r[3], r[2]))
+        raws.append(a_raw)
+    g_mu, g_m2, g_n = dp.merge_moments(recs)
+    g_sigma = dp.sigma_from(g_m2, g_n, 0)
+    assert abs(g_mu - mu) < 1e-6 and abs(g_sigma - sigma) < 1e-6
+    seq_tok = [int(lb.mask[int(a):int(b)].sum()) for a, b in zip(lb.cu_seqlens[:-1], lb.cu_seqlens[1:])]
+    n_tok, n_resp = sum(seq_tok), sum(1 for c in seq_tok if c > 0)
+    params = B.default_params(agg_mode=agg, global_tokens=n_tok, global_responses=n_resp)
+    loss_sum, dws, dhs = 0.0, [], []
+    for (s0, s1), a_raw in zip(splits, raws):
+        a_n = torch.empty_like(a_raw)
+        B.spo_advantages_apply(a_raw, g_mu, g_sigma, a_n, params)
+        torch.cuda.synchronize()
+        np.testing.assert_allclose(a_n.cpu().numpy(), a_norm[s0:s1], rtol=1e-5, atol=2e-6)
+        part = _slice_batch(lb, s0, s1)
+        part.a_norm = a_n.cpu().numpy()
+        got = run_loss(part, params=params)
+        assert got["status"] == 0
+        loss_sum += got["loss"]
+        dws.append(got["dW"])
+        dhs.append(got["dH"])
+    assert abs(loss_sum - want["loss"]) <= 2e-3
+    assert rel_fro(np.concatenate(dhs, 0), want_dh) <= 1e-2
+    assert rel_fro(dws[0] + dws[1], want_dw) <= 1e-2
