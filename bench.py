@@ -100,16 +100,23 @@ class ClockSampler:
 class Step:
     """Device buffers of one workload and the call sequence of one step."""
 
-    def __init__(self, workload, device, rank, responses=None):
+    def __init__(self, workload, device, rank, responses=None, custom=None):
         import torch
         from paper_2509_13232_b200 import binding as B
         from paper_2509_13232_b200 import inputs
         self.B, self.torch = B, torch
-        d, V, w_std, noise, rew_p = LOSS_SHAPES[workload]
-        lengths = inputs.workload_lengths(workload)
-        if responses:
-            lengths = lengths[:responses]
-        cfg = int(workload[3])
+        if custom:                       # T,d,V: eight equal responses, weights scaled to unit-variance logits
+            t_c, d, V = custom
+            w_std, noise, rew_p = 1.3 / d ** 0.5, 0.02, 0.3
+            lengths = np.full(8, t_c // 8, dtype=np.int64)
+            lengths[-1] += t_c - int(lengths.sum())
+            cfg = 9
+        else:
+            d, V, w_std, noise, rew_p = LOSS_SHAPES[workload]
+            lengths = inputs.workload_lengths(workload)
+            if responses:
+                lengths = lengths[:responses]
+            cfg = int(workload[3])
         data = inputs.loss_batch_device(cfg * 10 + rank, lengths, d, V, w_std, noise, device, adv_p=rew_p)
         self.data = data
         self.T, self.d, self.V, self.S = data["T"], d, V, data["S"]
@@ -193,7 +200,7 @@ def run_ours(args, rank, world, local_rank):
         spo_build.build()
     if world > 1:
         dist.barrier()
-    step = Step(args.workload, device, rank, args.responses)
+    step = Step(args.workload, device, rank, args.responses, args.custom)
     peaks = read_peaks()
 
     def barrier():
@@ -285,7 +292,7 @@ def run_ours(args, rank, world, local_rank):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": args.workload, "responses": step.S, "tokens": step.T, "d": step.d, "V": step.V,
+        "config": {"workload": "custom" if args.custom else args.workload, "responses": step.S, "tokens": step.T, "d": step.d, "V": step.V,
                    "tracker_prompts": step.table_n, "l2": "inputs_exceed_l2", "bwd_chunks": step.bwd_chunks,
                    "parallelism": "replicas" if world > 1 else "single"},
         "gpu_launches": step.launches * args.steps,
@@ -302,7 +309,7 @@ def run_ours(args, rank, world, local_rank):
             "bwd_tflops": step.flops_bwd / (t_bwd / args.steps / 1e3) / 1e12,
             # DRAM read+write bytes of all launches of one step, from the ncu capture summarised in
             # profiles/spo_gemm_kernel_cfg4_16responses_full.md, scaled by token rows; null for other shapes.
-            "traffic": CFG4_STEP_DRAM_BYTES if (args.workload == "cfg4_8b_bf16" and not args.responses) else None,
+            "traffic": CFG4_STEP_DRAM_BYTES if (args.workload == "cfg4_8b_bf16" and not args.responses and not args.custom) else None,
         },
         "e2e": {"value": tokens_all / (e2e_ms / e2e_steps / 1e3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "steps": e2e_steps},
@@ -462,6 +469,8 @@ def main():
     ap.add_argument("--workload", default="cfg4_8b_bf16", choices=sorted(LOSS_SHAPES) + sorted(SMALL_SHAPES))
     ap.add_argument("--cpu-tokens", type=int, default=None, help="token rows of the CPU-oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--custom", type=lambda v: tuple(int(x) for x in v.split(",")), default=None,
+                    help="T,d,V: time the loss path on another LM-head shape (eight equal responses)")
     ap.add_argument("--responses", type=int, default=None,
                     help="use only the first S responses of the workload (small cases for profiling)")
     args = ap.parse_args()
