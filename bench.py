@@ -324,6 +324,7 @@ SMALL_SHAPES = {
     # workload: (table prompts N, batch B, uniforms M)
     "cfg2_tracker_scale": (1_000_000, 4096, 8192),
     "small_scaled": (1 << 28, 1 << 22, 8192),
+    "small_scaled_26": (1 << 26, 1 << 22, 8192),      # a size that profiler captures with many passes can hold
 }
 
 
