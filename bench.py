@@ -32,7 +32,7 @@ if ROOT not in sys.path:
 METRIC = "response tokens/s, fused SPO loss fwd+bwd (d4096,V151936,bf16); % bf16 peak"
 UNIT = "tokens/s"
 TABLE_N = 1_000_000          # tracker table the step samples from and updates
-CFG4_STEP_DRAM_BYTES = 1.14e12
+CFG4_STEP_DRAM_BYTES = 1.23e12
 
 LOSS_SHAPES = {
     # workload: (d, V, w_std, old-logprob noise, reward probability)

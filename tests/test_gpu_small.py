@@ -330,3 +330,18 @@ def test_sampling_weight_output_for_odd_table_sizes(n):
     assert st == 0
     np.testing.assert_array_equal(w, want)
     np.testing.assert_array_equal(ids, O.sample_prompts(want, u, 1))
+
+
+def test_sampling_at_the_maximum_number_of_uniforms():
+    """M = 2^20 draws (the documented limit) with many repeats; ids still bit-exact and in order."""
+    n, m, b = 3_000_000, 1 << 20, 500_000
+    rng = np.random.default_rng(404)
+    ab = rng.uniform(0.0, 12.0, (n, 2)).astype(np.float32)
+    u = inputs.uniforms_f32(rng, m)
+    p = B().default_params()
+    ids, _, st = gpu_sample(dev(ab), u, b, p, want_w=False)
+    w_or = O.sampling_weights_f32(ab[:, 0], ab[:, 1], np.float32(p.eps_explore))
+    want = O.sample_prompts(w_or, u, b)
+    assert st == 0
+    np.testing.assert_array_equal(ids, want)
+    assert len(set(ids.tolist())) == b
