@@ -672,13 +672,31 @@ int group_count() { return sm_count() / CG; }
 template <int MODE>
 cudaError_t launch_gemm(const CUtensorMap& a, const CUtensorMap& b, const GemmParams& p_in, uint32_t* progress,
                         cudaStream_t st) {
-  static bool configured[64] = {};
+  static int max_groups[64] = {};            // CTA pairs that can be resident together, per device (0 = not yet asked)
   int dev = 0;
   cudaGetDevice(&dev);
-  if (dev >= 0 && dev < 64 && !configured[dev]) {
+  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  if (max_groups[dev] == 0) {
     cudaError_t e = cudaFuncSetAttribute(spo_gemm_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (e != cudaSuccess) return e;
-    configured[dev] = true;
+    // The kernel is persistent and its pairs pace one another, so the grid must not exceed what the
+    // device can hold at one time.
+    cudaLaunchConfig_t q = {};
+    q.gridDim = dim3(group_count() * CG, 1, 1);
+    q.blockDim = dim3(NUM_THREADS, 1, 1);
+    q.dynamicSmemBytes = SMEM_BYTES;
+    cudaLaunchAttribute qa[1];
+    qa[0].id = cudaLaunchAttributeClusterDimension;
+    qa[0].val.clusterDim.x = CG;
+    qa[0].val.clusterDim.y = 1;
+    qa[0].val.clusterDim.z = 1;
+    q.attrs = qa;
+    q.numAttrs = 1;
+    int n = 0;
+    e = cudaOccupancyMaxActiveClusters(&n, spo_gemm_kernel<MODE>, &q);
+    if (e != cudaSuccess) return e;
+    if (n < 1) return cudaErrorLaunchOutOfResources;
+    max_groups[dev] = n < group_count() ? n : group_count();
   }
   const int units = p_in.m_tiles * p_in.nsplit;
   if (units <= 0) return cudaSuccess;
@@ -691,7 +709,7 @@ cudaError_t launch_gemm(const CUtensorMap& a, const CUtensorMap& b, const GemmPa
     if (e != cudaSuccess) return e;
     p.progress = progress;
   }
-  const int groups = units < group_count() ? units : group_count();
+  const int groups = units < max_groups[dev] ? units : max_groups[dev];
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(groups * CG, 1, 1);
   cfg.blockDim = dim3(NUM_THREADS, 1, 1);
