@@ -100,7 +100,7 @@ class ClockSampler:
 class Step:
     """Device buffers of one workload and the call sequence of one step."""
 
-    def __init__(self, workload, device, rank, responses=None, custom=None):
+    def __init__(self, workload, device, rank, responses=None, custom=None, mask_frac=0.0):
         import torch
         from paper_2509_13232_b200 import binding as B
         from paper_2509_13232_b200 import inputs
@@ -120,6 +120,16 @@ class Step:
         data = inputs.loss_batch_device(cfg * 10 + rank, lengths, d, V, w_std, noise, device, adv_p=rew_p)
         self.data = data
         self.T, self.d, self.V, self.S = data["T"], d, V, data["S"]
+        self.mask_frac = float(mask_frac)
+        if self.mask_frac > 0.0:
+            # contiguous masked spans inside the responses, the way tool output sits inside a
+            # tool-integrated-reasoning response: spans of 32..256 tokens until the share is reached
+            rng = inputs.rng_for(cfg * 10 + rank, 7)
+            m = np.ones(self.T, dtype=np.uint8)
+            while 1.0 - m.mean() < self.mask_frac:
+                a = int(rng.integers(0, self.T))
+                m[a:a + int(rng.integers(32, 257))] = 0
+            data["mask"] = torch.from_numpy(m).to(device)
         self.n_tok = int(data["mask"].sum().item())
         self.table_n = TABLE_PROMPTS.get(workload, TABLE_N)
         tb = inputs.tracker_batch(cfg * 10 + rank, self.table_n, self.S, 2 * self.S)
@@ -143,7 +153,13 @@ class Step:
         self.ws_adv = torch.empty(B.spo_workspace_bytes(B.WS_ADVANTAGES, B=self.S), **u8)
         self.ws_fwd = torch.empty(B.spo_workspace_bytes(B.WS_LOSS_FWD, T=self.T, d=d, V=V, B=self.S), **u8)
         self.ws_bwd_bytes = B.spo_workspace_bytes(B.WS_LOSS_BWD, T=self.T, d=d, V=V)
-        self.ws_bwd = torch.empty(self.ws_bwd_bytes, **u8)
+        if self.mask_frac > 0.0:        # backward over the rows with gradient only
+            self.rows = torch.empty(self.T, dtype=torch.int32, device=device)
+            self.n_active = torch.zeros(4, dtype=torch.int32, device=device)
+            self.ws_rows = torch.empty(B.spo_workspace_bytes(B.WS_ACTIVE_ROWS, T=self.T), **u8)
+            self.ws_bwd = torch.empty(B.spo_workspace_bytes(B.WS_LOSS_BWD_ROWS, T=self.n_tok, d=d, V=V), **u8)
+        else:
+            self.ws_bwd = torch.empty(self.ws_bwd_bytes, **u8)
         chunk_rows = self.ws_bwd_bytes // (((V + 255) // 256) * 256 * 2)
         self.bwd_chunks = -(-self.T // chunk_rows)
         # kernels launched by one step: sampling 3 (tile sums, search, accept), advantages 1, update 1,
@@ -168,6 +184,13 @@ class Step:
 
     def bwd(self, h=None, y=None):
         D = self.data
+        if self.mask_frac > 0.0:
+            B = self.B
+            B.spo_loss_active_rows(self.coef, self.rows, self.n_active, self.ws_rows)
+            n_act = int(self.n_active[0].item())          # the one host read-back of this path
+            B.spo_loss_bwd_rows(D["h"] if h is None else h, D["w"], D["y"] if y is None else y, self.lse, self.coef,
+                                1.0, self.rows, n_act, self.dH, self.dW, 0, self.ws_bwd, self.params, self.status)
+            return
         self.B.spo_loss_bwd(D["h"] if h is None else h, D["w"], D["y"] if y is None else y, self.lse, self.coef,
                             1.0, self.dH, self.dW, 0, self.ws_bwd, self.params, self.status)
 
@@ -200,7 +223,7 @@ def run_ours(args, rank, world, local_rank):
         spo_build.build()
     if world > 1:
         dist.barrier()
-    step = Step(args.workload, device, rank, args.responses, args.custom)
+    step = Step(args.workload, device, rank, args.responses, args.custom, args.mask_frac)
     peaks = read_peaks()
 
     def barrier():
@@ -293,7 +316,7 @@ def run_ours(args, rank, world, local_rank):
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": "custom" if args.custom else args.workload, "responses": step.S, "tokens": step.T, "d": step.d, "V": step.V,
-                   "tracker_prompts": step.table_n, "l2": "inputs_exceed_l2", "bwd_chunks": step.bwd_chunks,
+                   "tracker_prompts": step.table_n, "l2": "inputs_exceed_l2", "bwd_chunks": step.bwd_chunks, "mask_frac": step.mask_frac,
                    "parallelism": "replicas" if world > 1 else "single"},
         "gpu_launches": step.launches * args.steps,
         "device_status": status,
@@ -309,7 +332,7 @@ def run_ours(args, rank, world, local_rank):
             "bwd_tflops": step.flops_bwd / (t_bwd / args.steps / 1e3) / 1e12,
             # DRAM read+write bytes of all launches of one step, from the ncu capture summarised in
             # profiles/spo_gemm_kernel_cfg4_16responses_full.md, scaled by token rows; null for other shapes.
-            "traffic": CFG4_STEP_DRAM_BYTES if (args.workload == "cfg4_8b_bf16" and not args.responses and not args.custom) else None,
+            "traffic": CFG4_STEP_DRAM_BYTES if (args.workload == "cfg4_8b_bf16" and not args.responses and not args.custom and not args.mask_frac) else None,
         },
         "e2e": {"value": tokens_all / (e2e_ms / e2e_steps / 1e3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "steps": e2e_steps},
@@ -472,6 +495,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--custom", type=lambda v: tuple(int(x) for x in v.split(",")), default=None,
                     help="T,d,V: time the loss path on another LM-head shape (eight equal responses)")
+    ap.add_argument("--mask-frac", type=float, default=0.0,
+                    help="mask this share of the tokens in contiguous spans and run the backward over the "
+                         "rows with gradient only (spo_loss_bwd_rows)")
     ap.add_argument("--responses", type=int, default=None,
                     help="use only the first S responses of the workload (small cases for profiling)")
     args = ap.parse_args()

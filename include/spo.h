@@ -62,6 +62,8 @@ extern "C" {
 #define SPO_WS_LOSS_FWD    2
 #define SPO_WS_LOSS_BWD    3
 #define SPO_WS_UPDATE_REPEATS 4
+#define SPO_WS_ACTIVE_ROWS    5
+#define SPO_WS_LOSS_BWD_ROWS  6
 
 /*
  * Hyper-parameters.  Defaults (spo_default_params) are the values the paper prints:
@@ -274,6 +276,31 @@ int32_t spo_loss_bwd(const void* H, const void* W, int32_t dtype, const int32_t*
  * status bit, not in a hang.  One tiny launch on `stream`.
  */
 int32_t spo_selftest_bounded_wait(uint32_t limit_us, int32_t* reached_end, int32_t* d_status, void* stream);
+
+/*
+ * Backward over the rows that carry gradient only.  A token whose coef is zero -- masked out of the
+ * loss (e.g. tool output inside a response) or clipped on the side that stops the gradient --
+ * contributes nothing to dH or dW, so the three contractions of spo_loss_bwd can run on the other
+ * rows alone; their cost falls in proportion.  Two calls, because the number of such rows has to
+ * reach the host to size the second one (the library itself never synchronises):
+ *
+ *   spo_loss_active_rows: rows[0..count) = ascending indices t with coef[t] != 0, *d_count = count.
+ *     rows    device out [T] int32;  d_count  device out [1] int32
+ *     ws      device scratch, spo_workspace_bytes(SPO_WS_ACTIVE_ROWS, T, ...) bytes
+ *   (the caller reads *d_count back, e.g. after a stream synchronise)
+ *   spo_loss_bwd_rows: same results as spo_loss_bwd(H, W, ..., T, ...): dH[t] for the listed rows,
+ *     zeros elsewhere; dW as in spo_loss_bwd.  bf16 H / W only.
+ *     rows    device in [T_act] from the first call;  T_act  host value of *d_count
+ *     ws      device scratch, spo_workspace_bytes(SPO_WS_LOSS_BWD_ROWS, T_act, d, V, ...) bytes
+ *             (holds the gathered rows of H and dH besides the chunk buffer)
+ */
+int32_t spo_loss_active_rows(const float* coef, int64_t T, int32_t* rows, int32_t* d_count,
+                             void* ws, size_t ws_bytes, void* stream);
+int32_t spo_loss_bwd_rows(const void* H, const void* W, int32_t dtype, const int32_t* y,
+                          const float* lse, const float* coef, float grad_loss,
+                          int64_t T, int32_t d, int32_t V, const int32_t* rows, int64_t T_act,
+                          void* dH, int32_t dH_dtype, float* dW, int32_t dW_accumulate,
+                          void* ws, size_t ws_bytes, const spo_params* params, int32_t* d_status, void* stream);
 
 /* Scratch size in bytes for one call of the selected entry point (host only, no CUDA call
  * except a device-property query).  Arguments that the selected call does not use are ignored. */

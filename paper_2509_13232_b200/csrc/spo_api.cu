@@ -248,6 +248,80 @@ int32_t spo_loss_bwd(const void* H, const void* W, int32_t dtype, const int32_t*
   return e == cudaSuccess ? SPO_OK : cuda_fail(e);
 }
 
+namespace {
+struct BwdRowsWs {
+  size_t bwd, h_act, dh_act, y_act, lse_act, coef_act, total;
+  BwdWs inner;
+};
+BwdRowsWs bwd_rows_ws_layout(int64_t T_act, int32_t d, int32_t V, int32_t dh_elem) {
+  BwdRowsWs L{};
+  const int64_t n = T_act > 0 ? T_act : 1;
+  L.inner = bwd_ws_layout(T_act, d, V);
+  size_t off = 0;
+  L.bwd = off;      off = align_up(off + L.inner.total, 256);
+  L.h_act = off;    off = align_up(off + (size_t)n * d * 2, 256);
+  L.dh_act = off;   off = align_up(off + (size_t)n * d * dh_elem, 256);
+  L.y_act = off;    off = align_up(off + (size_t)n * 4, 256);
+  L.lse_act = off;  off = align_up(off + (size_t)n * 4, 256);
+  L.coef_act = off; off = align_up(off + (size_t)n * 4, 256);
+  L.total = off;
+  return L;
+}
+}  // namespace
+
+int32_t spo_loss_active_rows(const float* coef, int64_t T, int32_t* rows, int32_t* d_count, void* ws, size_t ws_bytes,
+                             void* stream) {
+  if (T < 0 || !d_count || (T > 0 && (!coef || !rows || !ws))) return SPO_ERR_INVALID_ARG;
+  if (T >= ((int64_t)1 << 31) - 256) return SPO_ERR_BAD_SHAPE;
+  if (!aligned16(coef) || !aligned16(rows) || !aligned16(ws)) return SPO_ERR_BAD_ALIGNMENT;
+  if (!device_is_sm100()) return SPO_ERR_UNSUPPORTED_ARCH;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (T == 0) {
+    cudaError_t e0 = cudaMemsetAsync(d_count, 0, sizeof(int32_t), st);
+    return e0 == cudaSuccess ? SPO_OK : cuda_fail(e0);
+  }
+  if (ws_bytes < active_rows_ws_bytes(T)) return SPO_ERR_WORKSPACE_TOO_SMALL;
+  cudaError_t e = launch_active_rows(coef, T, rows, d_count, (int32_t*)ws, st);
+  return e == cudaSuccess ? SPO_OK : cuda_fail(e);
+}
+
+int32_t spo_loss_bwd_rows(const void* H, const void* W, int32_t dtype, const int32_t* y, const float* lse,
+                          const float* coef, float grad_loss, int64_t T, int32_t d, int32_t V, const int32_t* rows,
+                          int64_t T_act, void* dH, int32_t dH_dtype, float* dW, int32_t dW_accumulate, void* ws,
+                          size_t ws_bytes, const spo_params* params, int32_t* d_status, void* stream) {
+  int32_t rc = check_loss_shape(dtype, T, d, V);
+  if (rc != SPO_OK) return rc;
+  if (dtype != SPO_DTYPE_BF16) return SPO_ERR_UNSUPPORTED_DTYPE;
+  if (dH_dtype != SPO_DTYPE_F32 && dH_dtype != SPO_DTYPE_BF16) return SPO_ERR_UNSUPPORTED_DTYPE;
+  if (!params_ok(params) || !W || !dW || !ws || T_act < 0 || T_act > T) return SPO_ERR_INVALID_ARG;
+  if (T > 0 && (!H || !y || !lse || !coef || !dH)) return SPO_ERR_INVALID_ARG;
+  if (T_act > 0 && !rows) return SPO_ERR_INVALID_ARG;
+  if (!aligned16(H) || !aligned16(W) || !aligned16(y) || !aligned16(lse) || !aligned16(coef) || !aligned16(dH) ||
+      !aligned16(dW) || !aligned16(ws) || !aligned16(rows))
+    return SPO_ERR_BAD_ALIGNMENT;
+  if (!device_is_sm100()) return SPO_ERR_UNSUPPORTED_ARCH;
+  const int32_t dh_elem = dH_dtype == SPO_DTYPE_BF16 ? 2 : 4;
+  const BwdRowsWs L = bwd_rows_ws_layout(T_act, d, V, dh_elem);
+  if (ws_bytes < L.total) return SPO_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t st = (cudaStream_t)stream;
+  char* w8 = (char*)ws;
+  cudaError_t e;
+  // rows without gradient get zeros; the others are overwritten by the scatter below
+  if (T > 0 && (e = cudaMemsetAsync(dH, 0, (size_t)T * d * dh_elem, st)) != cudaSuccess) return cuda_fail(e);
+  void* h_act = w8 + L.h_act;
+  void* dh_act = w8 + L.dh_act;
+  int32_t* y_act = reinterpret_cast<int32_t*>(w8 + L.y_act);
+  float* lse_act = reinterpret_cast<float*>(w8 + L.lse_act);
+  float* coef_act = reinterpret_cast<float*>(w8 + L.coef_act);
+  if ((e = launch_gather_rows(H, y, lse, coef, rows, T_act, d * 2, h_act, y_act, lse_act, coef_act, st)) != cudaSuccess)
+    return cuda_fail(e);
+  if ((e = launch_bwd_bf16(h_act, W, y_act, lse_act, coef_act, grad_loss, T_act, d, V, dh_act, dH_dtype, dW,
+                           dW_accumulate, w8 + L.bwd, L.inner, d_status, st)) != cudaSuccess)
+    return cuda_fail(e);
+  if ((e = launch_scatter_rows(dh_act, rows, T_act, d * dh_elem, dH, st)) != cudaSuccess) return cuda_fail(e);
+  return SPO_OK;
+}
+
 size_t spo_workspace_bytes(int32_t which, int64_t T, int32_t d, int32_t V, int64_t N, int32_t B, int32_t M) {
   switch (which) {
     case SPO_WS_SAMPLE:
@@ -262,6 +336,12 @@ size_t spo_workspace_bytes(int32_t which, int64_t T, int32_t d, int32_t V, int64
     case SPO_WS_LOSS_FWD:
       if (T < 0 || V < 1) return 0;
       return fwd_ws_layout(T, d, V, (d % 64) == 0 ? SPO_DTYPE_BF16 : SPO_DTYPE_F32, B).total;
+    case SPO_WS_ACTIVE_ROWS:
+      if (T < 0) return 0;
+      return active_rows_ws_bytes(T);
+    case SPO_WS_LOSS_BWD_ROWS:          /* T = number of active rows; sized for an fp32 dH */
+      if (T < 0 || V < 1 || d < 1) return 0;
+      return bwd_rows_ws_layout(T, d, V, 4).total;
     case SPO_WS_LOSS_BWD:
       if (T < 0 || V < 1 || d < 1) return 0;
       return bwd_ws_layout(T, d, V).total;

@@ -113,6 +113,16 @@ cudaError_t launch_bwd_bf16(const void* H, const void* W, const int32_t* y, cons
                             void* dH, int32_t dH_dtype, float* dW, int accumulate,
                             char* ws, const BwdWs& L, int32_t* d_status, cudaStream_t st);
 
+// row compaction for the backward
+cudaError_t launch_active_rows(const float* coef, int64_t T, int32_t* rows, int32_t* d_count, int32_t* block_cnt,
+                               cudaStream_t st);
+size_t active_rows_ws_bytes(int64_t T);
+cudaError_t launch_gather_rows(const void* H, const int32_t* y, const float* lse, const float* coef,
+                               const int32_t* rows, int64_t n_act, int32_t row_bytes, void* H_act, int32_t* y_act,
+                               float* lse_act, float* coef_act, cudaStream_t st);
+cudaError_t launch_scatter_rows(const void* dH_act, const int32_t* rows, int64_t n_act, int32_t row_bytes, void* dH,
+                                cudaStream_t st);
+
 cudaError_t launch_bounded_wait_probe(int32_t* d_status, uint32_t limit_us, int32_t* reached_end, cudaStream_t st);
 
 }  // namespace spo

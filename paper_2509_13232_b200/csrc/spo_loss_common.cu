@@ -311,6 +311,88 @@ bwd_f32_kernel(const float* __restrict__ H, const float* __restrict__ W, const i
   }
 }
 
+// ---------------------------------------------------------------------------
+// Row compaction for the backward: tokens whose coef is zero (masked, or clipped on the side
+// that stops the gradient) contribute nothing to dH or dW.
+// ---------------------------------------------------------------------------
+constexpr int kRowsPerBlock = 1024;
+
+__global__ void __launch_bounds__(1024)
+active_count_kernel(const float* __restrict__ coef, int64_t T, int32_t* __restrict__ block_cnt) {
+  const int64_t t = (int64_t)blockIdx.x * kRowsPerBlock + threadIdx.x;
+  const int on = (t < T && coef[t] != 0.0f) ? 1 : 0;
+  const int total = __syncthreads_count(on);
+  if (threadIdx.x == 0) block_cnt[blockIdx.x] = total;
+}
+
+// Exclusive scan of the block counts by one block; *d_count = number of active rows.
+__global__ void __launch_bounds__(1024)
+active_scan_kernel(int32_t* block_cnt, int64_t n_blocks, int32_t* __restrict__ d_count) {
+  __shared__ int s_warp[32];
+  __shared__ int s_run;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 0) s_run = 0;
+  __syncthreads();
+  for (int64_t b0 = 0; b0 < n_blocks; b0 += 1024) {
+    const int64_t b = b0 + tid;
+    const int v = b < n_blocks ? block_cnt[b] : 0;
+    int incl = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int x = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += x;
+    }
+    if (lane == 31) s_warp[warp] = incl;
+    __syncthreads();
+    int before = s_run;
+    for (int w = 0; w < warp; ++w) before += s_warp[w];
+    if (b < n_blocks) block_cnt[b] = before + incl - v;
+    __syncthreads();
+    if (tid == 1023) s_run = before + incl;
+    __syncthreads();
+  }
+  if (tid == 0) *d_count = s_run;
+}
+
+__global__ void __launch_bounds__(1024)
+active_write_kernel(const float* __restrict__ coef, int64_t T, const int32_t* __restrict__ block_off,
+                    int32_t* __restrict__ rows) {
+  __shared__ int s_warp[32];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int64_t t = (int64_t)blockIdx.x * kRowsPerBlock + tid;
+  const int on = (t < T && coef[t] != 0.0f) ? 1 : 0;
+  const unsigned bal = __ballot_sync(0xffffffffu, on);
+  if (lane == 0) s_warp[warp] = __popc(bal);
+  __syncthreads();
+  int before = block_off[blockIdx.x];
+  for (int w = 0; w < warp; ++w) before += s_warp[w];
+  if (on) rows[before + __popc(bal & ((1u << lane) - 1))] = (int32_t)t;
+}
+
+// One warp per active row: copy the row of H (16-byte pieces) and its per-token scalars.
+__global__ void __launch_bounds__(256)
+gather_rows_kernel(const uint4* __restrict__ H, const int32_t* __restrict__ y, const float* __restrict__ lse,
+                   const float* __restrict__ coef, const int32_t* __restrict__ rows, int64_t n_act, int row_vec,
+                   uint4* __restrict__ H_act, int32_t* __restrict__ y_act, float* __restrict__ lse_act,
+                   float* __restrict__ coef_act) {
+  const int lane = threadIdx.x & 31;
+  for (int64_t i = ((int64_t)blockIdx.x * 256 + threadIdx.x) >> 5; i < n_act; i += ((int64_t)gridDim.x * 256) >> 5) {
+    const int64_t t = rows[i];
+    for (int k = lane; k < row_vec; k += 32) H_act[i * row_vec + k] = __ldg(H + t * row_vec + k);
+    if (lane == 0) { y_act[i] = y[t]; lse_act[i] = lse[t]; coef_act[i] = coef[t]; }
+  }
+}
+
+__global__ void __launch_bounds__(256)
+scatter_rows_kernel(const uint4* __restrict__ dH_act, const int32_t* __restrict__ rows, int64_t n_act, int row_vec,
+                    uint4* __restrict__ dH) {
+  const int lane = threadIdx.x & 31;
+  for (int64_t i = ((int64_t)blockIdx.x * 256 + threadIdx.x) >> 5; i < n_act; i += ((int64_t)gridDim.x * 256) >> 5) {
+    const int64_t t = rows[i];
+    for (int k = lane; k < row_vec; k += 32) dH[t * row_vec + k] = dH_act[i * row_vec + k];
+  }
+}
+
 }  // namespace
 
 // ---------------------------------------------------------------------------
@@ -374,6 +456,46 @@ cudaError_t launch_bwd_f32(const float* H, const float* W, const int32_t* y, con
     if (e != cudaSuccess) return e;
   }
   bwd_f32_kernel<true><<<(unsigned)V, 128, smem, st>>>(H, W, y, lse, coef, grad_loss, T, d, V, dW, 0, accumulate);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_active_rows(const float* coef, int64_t T, int32_t* rows, int32_t* d_count, int32_t* block_cnt,
+                               cudaStream_t st) {
+  const int64_t n_blocks = ceil_div(T > 0 ? T : 1, kRowsPerBlock);
+  active_count_kernel<<<(unsigned)n_blocks, 1024, 0, st>>>(coef, T, block_cnt);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  active_scan_kernel<<<1, 1024, 0, st>>>(block_cnt, n_blocks, d_count);
+  if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  active_write_kernel<<<(unsigned)n_blocks, 1024, 0, st>>>(coef, T, block_cnt, rows);
+  return cudaGetLastError();
+}
+
+size_t active_rows_ws_bytes(int64_t T) {
+  return align_up(sizeof(int32_t) * (size_t)ceil_div(T > 0 ? T : 1, kRowsPerBlock), 256);
+}
+
+cudaError_t launch_gather_rows(const void* H, const int32_t* y, const float* lse, const float* coef,
+                               const int32_t* rows, int64_t n_act, int32_t row_bytes, void* H_act, int32_t* y_act,
+                               float* lse_act, float* coef_act, cudaStream_t st) {
+  if (n_act == 0) return cudaSuccess;
+  int64_t blocks = ceil_div(n_act * 32, 256);
+  const int64_t cap = (int64_t)sm_count() * 16;
+  if (blocks > cap) blocks = cap;
+  gather_rows_kernel<<<(unsigned)blocks, 256, 0, st>>>(reinterpret_cast<const uint4*>(H), y, lse, coef, rows, n_act,
+                                                       row_bytes / 16, reinterpret_cast<uint4*>(H_act), y_act, lse_act,
+                                                       coef_act);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_scatter_rows(const void* dH_act, const int32_t* rows, int64_t n_act, int32_t row_bytes, void* dH,
+                                cudaStream_t st) {
+  if (n_act == 0) return cudaSuccess;
+  int64_t blocks = ceil_div(n_act * 32, 256);
+  const int64_t cap = (int64_t)sm_count() * 16;
+  if (blocks > cap) blocks = cap;
+  scatter_rows_kernel<<<(unsigned)blocks, 256, 0, st>>>(reinterpret_cast<const uint4*>(dH_act), rows, n_act,
+                                                        row_bytes / 16, reinterpret_cast<uint4*>(dH));
   return cudaGetLastError();
 }
 

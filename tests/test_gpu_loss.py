@@ -227,3 +227,64 @@ def test_results_are_bitwise_reproducible():
     assert a["loss"] == b["loss"]
     for k in ("logp", "lse", "coef", "dH", "dW", "seq_sums"):
         np.testing.assert_array_equal(a[k], b[k])
+
+
+@pytest.mark.parametrize("dh_f32", [False, True])
+def test_backward_over_active_rows_only(dh_f32):
+    """40 % of the tokens masked (plus clipped ones): the row-compacted backward gives the oracle's gradients,
+    zeros in the rows without gradient, and lists exactly the rows with coef != 0."""
+    import torch
+    from paper_2509_13232_b200 import binding as B
+    from tests.helpers import dev, status_word, ws_bytes
+    lb = _clip_batch(110, [900, 1300, 2, 700, 2500, 61], 128, 1500, True)
+    rng = np.random.default_rng(3)
+    lb.mask[:] = (rng.random(lb.mask.shape[0]) > 0.4).astype(np.uint8)
+    lb.mask[900:2200] = 0                                # a whole response (tool output) masked
+    want = oracle_loss(lb, grad_loss=0.7)
+    p = B.default_params()
+    H, W = dev(lb.h, torch.bfloat16), dev(lb.w, torch.bfloat16)
+    T, d = H.shape
+    V = W.shape[0]
+    y = dev(lb.y)
+    lse, coef = dev(want["lse"].astype(np.float32)), dev(want["coef"].astype(np.float32))
+    rows = torch.full((T,), -1, dtype=torch.int32, device="cuda")
+    count = torch.zeros(4, dtype=torch.int32, device="cuda")
+    B.spo_loss_active_rows(coef, rows, count, ws_bytes(B.WS_ACTIVE_ROWS, T=T))
+    torch.cuda.synchronize()
+    n_act = int(count[0].item())
+    want_rows = np.nonzero(want["coef"].astype(np.float32) != 0)[0]
+    assert n_act == len(want_rows) and 0 < n_act < 0.7 * T
+    np.testing.assert_array_equal(rows[:n_act].cpu().numpy(), want_rows)
+    dH = torch.full((T, d), float("nan"), dtype=torch.float32 if dh_f32 else torch.bfloat16, device="cuda")
+    dW = torch.full((V, d), float("nan"), dtype=torch.float32, device="cuda")
+    st = status_word()
+    B.spo_loss_bwd_rows(H, W, y, lse, coef, 0.7, rows, n_act, dH, dW, 0, ws_bytes(B.WS_LOSS_BWD_ROWS, T=n_act, d=d, V=V),
+                        p, st)
+    torch.cuda.synchronize()
+    assert int(st[0].item()) == 0
+    got_dh = dH.float().cpu().numpy()
+    inactive = np.setdiff1d(np.arange(T), want_rows)
+    assert np.all(got_dh[inactive] == 0.0)
+    assert rel_fro(got_dh, want["dH"]) <= 1e-2
+    assert rel_fro(dW.cpu().numpy(), want["dW"]) <= 1e-2
+
+
+def test_backward_over_active_rows_with_nothing_active():
+    import torch
+    from paper_2509_13232_b200 import binding as B
+    from tests.helpers import dev, status_word, ws_bytes
+    T, d, V = 300, 64, 200
+    H = torch.randn((T, d), device="cuda").to(torch.bfloat16)
+    W = torch.randn((V, d), device="cuda").to(torch.bfloat16)
+    zeros = torch.zeros(T, device="cuda")
+    rows = torch.zeros(T, dtype=torch.int32, device="cuda")
+    count = torch.full((4,), 9, dtype=torch.int32, device="cuda")
+    B.spo_loss_active_rows(zeros, rows, count, ws_bytes(B.WS_ACTIVE_ROWS, T=T))
+    torch.cuda.synchronize()
+    assert int(count[0].item()) == 0
+    dH = torch.full((T, d), 1.0, dtype=torch.bfloat16, device="cuda")
+    dW = torch.full((V, d), 1.0, device="cuda")
+    B.spo_loss_bwd_rows(H, W, torch.zeros(T, dtype=torch.int32, device="cuda"), zeros, zeros, 1.0, rows, 0, dH, dW, 0,
+                        ws_bytes(B.WS_LOSS_BWD_ROWS, T=0, d=d, V=V), B.default_params(), status_word())
+    torch.cuda.synchronize()
+    assert float(dH.float().abs().max().item()) == 0.0 and float(dW.abs().max().item()) == 0.0
