@@ -3,7 +3,10 @@
 
 One "step" is one pass of the whole path over one synthetic mini-batch:
 prioritised sampling -> advantages (pre-update baseline) + normalisation ->
-tracker update -> fused loss forward -> fused loss backward (dH, dW).
+tracker update -> fused loss forward + backward (loss, logp, lse, coef, dH, dW).
+The loss runs as the one-pass call spo_loss_fwd_bwd (three LM-head contractions per
+token) by default, or as spo_loss_fwd followed by spo_loss_bwd with `--path split`
+(four: the backward recomputes the logits).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
 
@@ -32,7 +35,9 @@ if ROOT not in sys.path:
 METRIC = "response tokens/s, fused SPO loss fwd+bwd (d4096,V151936,bf16); % bf16 peak"
 UNIT = "tokens/s"
 TABLE_N = 1_000_000          # tracker table the step samples from and updates
-CFG4_STEP_DRAM_BYTES = 1.23e12
+# DRAM read+write bytes of all launches of one cfg4 step, from ncu captures (profiles/); None = the
+# kernels of that path changed after the counters were taken
+CFG4_STEP_DRAM_BYTES = {"split": 1.23e12, "onepass": None}
 
 LOSS_SHAPES = {
     # workload: (d, V, w_std, old-logprob noise, reward probability)
@@ -100,7 +105,7 @@ class ClockSampler:
 class Step:
     """Device buffers of one workload and the call sequence of one step."""
 
-    def __init__(self, workload, device, rank, responses=None, custom=None, mask_frac=0.0):
+    def __init__(self, workload, device, rank, responses=None, custom=None, mask_frac=0.0, path="onepass"):
         import torch
         from paper_2509_13232_b200 import binding as B
         from paper_2509_13232_b200 import inputs
@@ -121,6 +126,7 @@ class Step:
         self.data = data
         self.T, self.d, self.V, self.S = data["T"], d, V, data["S"]
         self.mask_frac = float(mask_frac)
+        self.onepass = (path == "onepass") and not self.mask_frac > 0.0
         if self.mask_frac > 0.0:
             # contiguous masked spans inside the responses, the way tool output sits inside a
             # tool-integrated-reasoning response: spans of 32..256 tokens until the share is reached
@@ -151,22 +157,30 @@ class Step:
         u8 = dict(dtype=torch.uint8, device=device)
         self.ws_sample = torch.empty(B.spo_workspace_bytes(B.WS_SAMPLE, N=self.table_n, M=2 * self.S), **u8)
         self.ws_adv = torch.empty(B.spo_workspace_bytes(B.WS_ADVANTAGES, B=self.S), **u8)
-        self.ws_fwd = torch.empty(B.spo_workspace_bytes(B.WS_LOSS_FWD, T=self.T, d=d, V=V, B=self.S), **u8)
         self.ws_bwd_bytes = B.spo_workspace_bytes(B.WS_LOSS_BWD, T=self.T, d=d, V=V)
-        if self.mask_frac > 0.0:        # backward over the rows with gradient only
-            self.rows = torch.empty(self.T, dtype=torch.int32, device=device)
-            self.n_active = torch.zeros(4, dtype=torch.int32, device=device)
-            self.ws_rows = torch.empty(B.spo_workspace_bytes(B.WS_ACTIVE_ROWS, T=self.T), **u8)
-            self.ws_bwd = torch.empty(B.spo_workspace_bytes(B.WS_LOSS_BWD_ROWS, T=self.n_tok, d=d, V=V), **u8)
+        if self.onepass:
+            self.ws_loss = torch.empty(B.spo_workspace_bytes(B.WS_LOSS_FWD_BWD, T=self.T, d=d, V=V, B=self.S), **u8)
         else:
-            self.ws_bwd = torch.empty(self.ws_bwd_bytes, **u8)
+            self.ws_fwd = torch.empty(B.spo_workspace_bytes(B.WS_LOSS_FWD, T=self.T, d=d, V=V, B=self.S), **u8)
+            if self.mask_frac > 0.0:    # backward over the rows with gradient only
+                self.rows = torch.empty(self.T, dtype=torch.int32, device=device)
+                self.n_active = torch.zeros(4, dtype=torch.int32, device=device)
+                self.ws_rows = torch.empty(B.spo_workspace_bytes(B.WS_ACTIVE_ROWS, T=self.T), **u8)
+                self.ws_bwd = torch.empty(B.spo_workspace_bytes(B.WS_LOSS_BWD_ROWS, T=self.n_tok, d=d, V=V), **u8)
+            else:
+                self.ws_bwd = torch.empty(self.ws_bwd_bytes, **u8)
         chunk_rows = self.ws_bwd_bytes // (((V + 255) // 256) * 256 * 2)
         self.bwd_chunks = -(-self.T // chunk_rows)
-        # kernels launched by one step: sampling 3 (tile sums, search, accept), advantages 1, update 1,
-        # forward 3 (count, contraction, finalise), backward 3 per chunk (memsets are not counted)
-        self.launches = 3 + 1 + 1 + 3 + 3 * self.bwd_chunks
+        # kernels launched by one step: sampling 3 (tile sums, search, accept), advantages 1, update 1, then
+        # split path: forward 3 (count, contraction, finalise), backward 3 per chunk;
+        # one-pass path: count 1, per chunk 5 (logits contraction, finalise, e->g, dH, dW).  Memsets are not counted.
         self.flops_fwd = 2.0 * self.T * d * V
-        self.flops_bwd = 6.0 * self.T * d * V
+        if self.onepass:
+            self.launches = 3 + 1 + 1 + 1 + 5 * self.bwd_chunks
+            self.flops_bwd = 4.0 * self.T * d * V
+        else:
+            self.launches = 3 + 1 + 1 + 3 + 3 * self.bwd_chunks
+            self.flops_bwd = 6.0 * self.T * d * V
 
     def small(self):
         B = self.B
@@ -194,10 +208,24 @@ class Step:
         self.B.spo_loss_bwd(D["h"] if h is None else h, D["w"], D["y"] if y is None else y, self.lse, self.coef,
                             1.0, self.dH, self.dW, 0, self.ws_bwd, self.params, self.status)
 
+    def loss_onepass(self, h=None, y=None, logp_old=None, mask=None, cu=None):
+        D = self.data
+        self.B.spo_loss_fwd_bwd(D["h"] if h is None else h, D["w"], D["y"] if y is None else y,
+                                D["logp_old"] if logp_old is None else logp_old, D["mask"] if mask is None else mask,
+                                D["cu_seqlens"] if cu is None else cu, self.a_norm, 1.0, self.loss, self.logp,
+                                self.lse, self.coef, None, self.dH, self.dW, 0, self.ws_loss, self.params, self.status)
+
+    def loss_calls(self, h=None, y=None, logp_old=None, mask=None, cu=None):
+        """The loss calls of one step on the chosen path."""
+        if self.onepass:
+            self.loss_onepass(h, y, logp_old, mask, cu)
+        else:
+            self.fwd(h, y, logp_old, mask, cu)
+            self.bwd(h, y)
+
     def run(self):
         self.small()
-        self.fwd()
-        self.bwd()
+        self.loss_calls()
 
 
 def reduce_over_ranks(times_ms, tokens, world, device):
@@ -223,7 +251,7 @@ def run_ours(args, rank, world, local_rank):
         spo_build.build()
     if world > 1:
         dist.barrier()
-    step = Step(args.workload, device, rank, args.responses, args.custom, args.mask_frac)
+    step = Step(args.workload, device, rank, args.responses, args.custom, args.mask_frac, args.path)
     peaks = read_peaks()
 
     def barrier():
@@ -242,7 +270,11 @@ def run_ours(args, rank, world, local_rank):
         marks = []
         for _ in range(args.steps):
             a, b, c, dd = ev(), ev(), ev(), ev()
-            a.record(); step.small(); b.record(); step.fwd(); c.record(); step.bwd(); dd.record()
+            a.record(); step.small(); b.record()
+            if step.onepass:
+                c.record(); step.loss_onepass(); dd.record()        # no forward / backward boundary to time
+            else:
+                step.fwd(); c.record(); step.bwd(); dd.record()
             marks.append((a, b, c, dd))
         barrier()
         wall = time.perf_counter() - wall0
@@ -288,8 +320,7 @@ def run_ours(args, rank, world, local_rank):
             main.wait_event(ready[i])
             step.rewards, step.uniforms = small_bufs[b]["rewards"], small_bufs[b]["uniforms"]
             step.small()
-            step.fwd(bufs[b]["h"], bufs[b]["y"], bufs[b]["logp_old"], bufs[b]["mask"], bufs[b]["cu_seqlens"])
-            step.bwd(bufs[b]["h"], bufs[b]["y"])
+            step.loss_calls(bufs[b]["h"], bufs[b]["y"], bufs[b]["logp_old"], bufs[b]["mask"], bufs[b]["cu_seqlens"])
             loss_host.copy_(step.loss, non_blocking=True)
             ids_host.copy_(step.ids, non_blocking=True)
             done[i].record(main)
@@ -316,23 +347,30 @@ def run_ours(args, rank, world, local_rank):
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": "custom" if args.custom else args.workload, "responses": step.S, "tokens": step.T, "d": step.d, "V": step.V,
-                   "tracker_prompts": step.table_n, "l2": "inputs_exceed_l2", "bwd_chunks": step.bwd_chunks, "mask_frac": step.mask_frac,
+                   "tracker_prompts": step.table_n, "l2": "inputs_exceed_l2", "loss_path": "onepass" if step.onepass else "split",
+                   "bwd_chunks": step.bwd_chunks, "mask_frac": step.mask_frac,
                    "parallelism": "replicas" if world > 1 else "single"},
         "gpu_launches": step.launches * args.steps,
         "device_status": status,
         "wall_s": wall,
-        "breakdown_ms": {"small": t_small / args.steps, "loss_fwd": t_fwd / args.steps, "loss_bwd": t_bwd / args.steps},
+        "breakdown_ms": ({"small": t_small / args.steps, "loss_fwd_bwd": t_bwd / args.steps} if step.onepass else
+                         {"small": t_small / args.steps, "loss_fwd": t_fwd / args.steps, "loss_bwd": t_bwd / args.steps}),
         "roofline": {
-            "bound": "tensor", "kernel": "spo_gemm_kernel (FWD, G, DH, DW instantiations; all launches of a step)",
+            "bound": "tensor",
+            "kernel": ("spo_gemm_kernel (E, DH, DW instantiations; all launches of a step; the duration is the whole "
+                       "spo_loss_fwd_bwd call, which also holds the streaming e->g and finalisation kernels)" if step.onepass
+                       else "spo_gemm_kernel (FWD, G, DH, DW instantiations; all launches of a step)"),
             "achieved": achieved, "peak": peaks["tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["tflops"],
             "peak_source": peaks["source"] + " sustained cuBLAS bf16",
             "frac_of_nominal_2250": achieved / 2250.0, "frac_of_burst": achieved / peaks["tflops_burst"],
             "flops_per_step": step.flops_fwd + step.flops_bwd,
-            "fwd_tflops": step.flops_fwd / (t_fwd / args.steps / 1e3) / 1e12,
-            "bwd_tflops": step.flops_bwd / (t_bwd / args.steps / 1e3) / 1e12,
+            "flops_per_token": (6 if step.onepass else 8) * step.d * step.V,
+            "fwd_tflops": None if step.onepass else step.flops_fwd / (t_fwd / args.steps / 1e3) / 1e12,
+            "bwd_tflops": None if step.onepass else step.flops_bwd / (t_bwd / args.steps / 1e3) / 1e12,
             # DRAM read+write bytes of all launches of one step, from the ncu capture summarised in
             # profiles/spo_gemm_kernel_cfg4_16responses_full.md, scaled by token rows; null for other shapes.
-            "traffic": CFG4_STEP_DRAM_BYTES if (args.workload == "cfg4_8b_bf16" and not args.responses and not args.custom and not args.mask_frac) else None,
+            "traffic": CFG4_STEP_DRAM_BYTES.get("onepass" if step.onepass else "split") if (
+                args.workload == "cfg4_8b_bf16" and not args.responses and not args.custom and not args.mask_frac) else None,
         },
         "e2e": {"value": tokens_all / (e2e_ms / e2e_steps / 1e3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "steps": e2e_steps},
@@ -498,6 +536,8 @@ def main():
     ap.add_argument("--mask-frac", type=float, default=0.0,
                     help="mask this share of the tokens in contiguous spans and run the backward over the "
                          "rows with gradient only (spo_loss_bwd_rows)")
+    ap.add_argument("--path", default="onepass", choices=["onepass", "split"],
+                    help="loss as one spo_loss_fwd_bwd call (default) or as spo_loss_fwd + spo_loss_bwd")
     ap.add_argument("--responses", type=int, default=None,
                     help="use only the first S responses of the workload (small cases for profiling)")
     args = ap.parse_args()

@@ -64,6 +64,7 @@ extern "C" {
 #define SPO_WS_UPDATE_REPEATS 4
 #define SPO_WS_ACTIVE_ROWS    5
 #define SPO_WS_LOSS_BWD_ROWS  6
+#define SPO_WS_LOSS_FWD_BWD   7
 
 /*
  * Hyper-parameters.  Defaults (spo_default_params) are the values the paper prints:
@@ -267,6 +268,37 @@ int32_t spo_loss_bwd(const void* H, const void* W, int32_t dtype, const int32_t*
                      void* dH, int32_t dH_dtype, float* dW, int32_t dW_accumulate,
                      void* ws, size_t ws_bytes,
                      const spo_params* params, int32_t* d_status, void* stream);
+
+/*
+ * Policy loss forward and backward in one pass: every output of spo_loss_fwd (loss, logp, lse,
+ * coef, seq_sums; Sec. 3.2, the PPO-Clip objective) and of spo_loss_bwd (dH, dW) for the same
+ * inputs, with three LM-head-sized contractions per token instead of four.  The loss is the last
+ * node of the training graph, so its upstream gradient (`grad_loss`, e.g. 1 or a loss scale) is
+ * known before the forward runs; that is what lets the two halves share their logits.
+ *
+ * bf16: token rows are processed in chunks (the chunk of spo_loss_bwd).  The logits of a chunk
+ * are contracted once; the epilogue keeps the online (max, sum-exp, target logit) of every row and
+ * also stores each logit as e = 2^(z log2(e) - ref), bf16, with one fp32 reference exponent `ref`
+ * per row and 64 columns (that group's largest logit, so e <= 1 and its relative error is bf16's
+ * whatever the range of the logits).  After the chunk's rows are finalised (lse, coef), a streaming
+ * kernel rewrites the buffer in place as g = grad_loss coef_t (1[v = y_t] - e 2^(ref - lse_t log2(e)))
+ * and dH, dW follow as in spo_loss_bwd.  loss, logp, lse and coef never see the bf16 rounding of e;
+ * dH and dW carry it in place of spo_loss_bwd's own bf16 rounding of g (same size).
+ * fp32: the two SIMT halves run back to back (nothing to share).
+ *
+ *   arguments   as in spo_loss_fwd and spo_loss_bwd; lse and coef are outputs here
+ *   ws          device scratch, spo_workspace_bytes(SPO_WS_LOSS_FWD_BWD, T, d, V, 0, S, 0) bytes:
+ *               the chunk buffer, its reference exponents (1/32 of it) and the forward's partials
+ * Status bits as spo_loss_fwd.
+ */
+int32_t spo_loss_fwd_bwd(const void* H, const void* W, int32_t dtype,
+                         const int32_t* y, const float* logp_old, const uint8_t* mask,
+                         const int32_t* cu_seqlens, const float* a_norm,
+                         int64_t T, int32_t d, int32_t V, int32_t S, float grad_loss,
+                         float* loss, float* logp, float* lse, float* coef, float* seq_sums,
+                         void* dH, int32_t dH_dtype, float* dW, int32_t dW_accumulate,
+                         void* ws, size_t ws_bytes,
+                         const spo_params* params, int32_t* d_status, void* stream);
 
 /*
  * Diagnostic (no counterpart in the paper): runs the kernels' bounded mbarrier wait on a barrier

@@ -248,6 +248,55 @@ int32_t spo_loss_bwd(const void* H, const void* W, int32_t dtype, const int32_t*
   return e == cudaSuccess ? SPO_OK : cuda_fail(e);
 }
 
+int32_t spo_loss_fwd_bwd(const void* H, const void* W, int32_t dtype, const int32_t* y, const float* logp_old,
+                         const uint8_t* mask, const int32_t* cu_seqlens, const float* a_norm, int64_t T, int32_t d,
+                         int32_t V, int32_t S, float grad_loss, float* loss, float* logp, float* lse, float* coef,
+                         float* seq_sums, void* dH, int32_t dH_dtype, float* dW, int32_t dW_accumulate, void* ws,
+                         size_t ws_bytes, const spo_params* params, int32_t* d_status, void* stream) {
+  int32_t rc = check_loss_shape(dtype, T, d, V);
+  if (rc != SPO_OK) return rc;
+  if (dH_dtype != SPO_DTYPE_F32 && dH_dtype != SPO_DTYPE_BF16) return SPO_ERR_UNSUPPORTED_DTYPE;
+  if (!params_ok(params) || !W || !loss || !dW || !ws || !cu_seqlens || S < 0) return SPO_ERR_INVALID_ARG;
+  if (T > 0 && (!H || !y || !logp_old || !a_norm || !logp || !lse || !coef || !dH || S < 1)) return SPO_ERR_INVALID_ARG;
+  if (!aligned16(H) || !aligned16(W) || !aligned16(y) || !aligned16(logp_old) || !aligned16(cu_seqlens) ||
+      !aligned16(a_norm) || !aligned16(logp) || !aligned16(lse) || !aligned16(coef) || !aligned16(dH) ||
+      !aligned16(dW) || !aligned16(ws))
+    return SPO_ERR_BAD_ALIGNMENT;
+  if (!device_is_sm100()) return SPO_ERR_UNSUPPORTED_ARCH;
+  cudaStream_t st = (cudaStream_t)stream;
+  char* w8 = (char*)ws;
+  cudaError_t e;
+  if (dtype == SPO_DTYPE_BF16) {
+    const FusedWs L = fused_ws_layout(T, d, V, S);
+    if (ws_bytes < L.total) return SPO_ERR_WORKSPACE_TOO_SMALL;
+    FusedArgs a{};
+    a.H = H; a.W = W; a.y = y; a.logp_old = logp_old; a.mask = mask; a.cu_seqlens = cu_seqlens; a.a_norm = a_norm;
+    a.T = T; a.d = d; a.V = V; a.S = S; a.grad_loss = grad_loss;
+    a.loss = loss; a.logp = logp; a.lse = lse; a.coef = coef; a.seq_sums = seq_sums;
+    a.dH = dH; a.dH_dtype = dH_dtype; a.dW = dW; a.accumulate = dW_accumulate;
+    a.params = params; a.d_status = d_status;
+    e = launch_fused_bf16(a, w8, L, st);
+    return e == cudaSuccess ? SPO_OK : cuda_fail(e);
+  }
+  // fp32 inputs: nothing to share between the two halves of the SIMT path; run them back to back
+  const FwdWs L = fwd_ws_layout(T, d, V, dtype, S);
+  if (ws_bytes < L.total) return SPO_ERR_WORKSPACE_TOO_SMALL;
+  FwdPartial* partials = reinterpret_cast<FwdPartial*>(w8 + L.partials);
+  double* block_sums = reinterpret_cast<double*>(w8 + L.block_sums);
+  int32_t* counters = reinterpret_cast<int32_t*>(w8 + L.counters);
+  int32_t* seq_cnt = reinterpret_cast<int32_t*>(w8 + L.seq_cnt);
+  if ((e = launch_fwd_prepare(mask, T, cu_seqlens, S, params->agg_mode, seq_cnt, counters, st)) != cudaSuccess)
+    return cuda_fail(e);
+  if ((e = launch_fwd_f32((const float*)H, (const float*)W, y, T, d, V, partials, st)) != cudaSuccess) return cuda_fail(e);
+  e = launch_fwd_finalize(partials, L.nsplit, y, logp_old, mask, cu_seqlens, a_norm, T, V, S, params->clip_lo,
+                          params->clip_hi, loss, logp, lse, coef, seq_sums, block_sums, counters, seq_cnt,
+                          params->agg_mode, params->global_tokens, params->global_responses, L.fin_blocks, d_status, st);
+  if (e != cudaSuccess) return cuda_fail(e);
+  e = launch_bwd_f32((const float*)H, (const float*)W, y, lse, coef, grad_loss, T, d, V, dH, dH_dtype, dW,
+                     dW_accumulate, st);
+  return e == cudaSuccess ? SPO_OK : cuda_fail(e);
+}
+
 namespace {
 struct BwdRowsWs {
   size_t bwd, h_act, dh_act, y_act, lse_act, coef_act, total;
@@ -345,6 +394,13 @@ size_t spo_workspace_bytes(int32_t which, int64_t T, int32_t d, int32_t V, int64
     case SPO_WS_LOSS_BWD:
       if (T < 0 || V < 1 || d < 1) return 0;
       return bwd_ws_layout(T, d, V).total;
+    case SPO_WS_LOSS_FWD_BWD: {         /* enough for either element type */
+      if (T < 0 || V < 1 || d < 1) return 0;
+      const size_t f32 = fwd_ws_layout(T, d, V, SPO_DTYPE_F32, B).total;
+      if ((d % 64) != 0) return f32;
+      const size_t bf16 = fused_ws_layout(T, d, V, B).total;
+      return bf16 > f32 ? bf16 : f32;
+    }
     default:
       return 0;
   }

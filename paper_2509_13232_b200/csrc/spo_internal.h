@@ -78,6 +78,15 @@ struct FwdWs {
 };
 FwdWs fwd_ws_layout(int64_t T, int32_t d, int32_t V, int32_t dtype, int32_t S);
 
+// Rows a finalisation launch covers when the batch is finalised piecewise (one-pass forward+backward).
+struct FinalizeRange {
+  int64_t t_begin;      // first token row of this launch (a multiple of kFinalizeThreads)
+  int64_t part_ld;      // rows between two splits' partials; partial 0 of a split belongs to row t_begin
+  int block0;           // index of this launch's first block among all finalisation blocks
+  int total_blocks;     // finalisation blocks over the whole batch; the last one to finish folds the loss
+  int last;             // 1 when this launch covers the final rows (per-response sums are taken then)
+};
+
 cudaError_t launch_fwd_prepare(const uint8_t* mask, int64_t T, const int32_t* cu_seqlens, int32_t S, int agg_mode,
                                int32_t* seq_cnt, int32_t* counters, cudaStream_t st);
 cudaError_t launch_fwd_finalize(const FwdPartial* partials, int nsplit, const int32_t* y,
@@ -87,7 +96,8 @@ cudaError_t launch_fwd_finalize(const FwdPartial* partials, int nsplit, const in
                                 float* loss, float* logp, float* lse, float* coef, float* seq_sums,
                                 double* block_sums, int32_t* counters, const int32_t* seq_cnt, int agg_mode,
                                 int32_t global_tokens, int32_t global_responses,
-                                int64_t fin_blocks, int32_t* d_status, cudaStream_t st);
+                                int64_t fin_blocks, int32_t* d_status, cudaStream_t st,
+                                const FinalizeRange* range = nullptr);
 
 // fp32 SIMT path
 cudaError_t launch_fwd_f32(const float* H, const float* W, const int32_t* y, int64_t T, int32_t d, int32_t V,
@@ -105,6 +115,37 @@ struct BwdWs {
   int64_t ldg;          // row pitch of g in elements (multiple of 256)
 };
 BwdWs bwd_ws_layout(int64_t T, int32_t d, int32_t V);
+
+// one-pass forward+backward (bf16)
+struct FusedWs {
+  size_t g;             // bf16 [chunk_rows][ldg]: e, then g, of one chunk
+  size_t ref;           // float [ldg/64][chunk_rows]: reference exponents of e
+  size_t partials;      // FwdPartial [2*nsplit][rows of the chunk]
+  size_t progress, block_sums, counters, seq_cnt;
+  size_t total;
+  int64_t chunk_rows, ldg;
+  int64_t fin_blocks;
+};
+FusedWs fused_ws_layout(int64_t T, int32_t d, int32_t V, int32_t S);
+struct FusedArgs {
+  const void *H, *W;
+  const int32_t* y;
+  const float* logp_old;
+  const uint8_t* mask;
+  const int32_t* cu_seqlens;
+  const float* a_norm;
+  int64_t T;
+  int32_t d, V, S;
+  float grad_loss;
+  float *loss, *logp, *lse, *coef, *seq_sums;
+  void* dH;
+  int32_t dH_dtype;
+  float* dW;
+  int accumulate;
+  const spo_params* params;
+  int32_t* d_status;
+};
+cudaError_t launch_fused_bf16(const FusedArgs& a, char* ws, const FusedWs& L, cudaStream_t st);
 
 cudaError_t launch_fwd_bf16(const void* H, const void* W, const int32_t* y, int64_t T, int32_t d, int32_t V,
                             FwdPartial* partials, int nsplit, uint32_t* progress, int32_t* d_status, cudaStream_t st);

@@ -81,22 +81,25 @@ fwd_finalize_kernel(const FwdPartial* __restrict__ partials, int nsplit, const i
                     float* __restrict__ loss, float* __restrict__ logp_out, float* __restrict__ lse_out,
                     float* __restrict__ coef_out, double* block_sums, int32_t* counters,
                     const int32_t* __restrict__ seq_cnt, int agg_mode, int32_t global_tokens,
-                    int32_t global_responses, int32_t* d_status) {
-  const int64_t t = (int64_t)blockIdx.x * kFinalizeThreads + threadIdx.x;
+                    int32_t global_responses, int32_t* d_status, FinalizeRange rg) {
+  // This launch covers token rows [rg.t_begin, T_end); its blocks are blocks rg.block0.. of the
+  // rg.total_blocks that cover all rows (one launch, or one per chunk of the one-pass path).
+  const int64_t t = rg.t_begin + (int64_t)blockIdx.x * kFinalizeThreads + threadIdx.x;
   // denominators of the expectation: this call's own counts, or the whole data-parallel batch's
   const int32_t n_tok = global_tokens > 0 ? global_tokens : counters[0];
   const int32_t s_act = global_responses > 0 ? global_responses : counters[2];
   double contrib = 0.0;
   if (t < T) {
+    const int64_t tp = t - rg.t_begin;
     float m2 = -CUDART_INF_F, zt = -CUDART_INF_F;
     for (int s = 0; s < nsplit; ++s) {
-      FwdPartial p = partials[(int64_t)s * T + t];
+      FwdPartial p = partials[(int64_t)s * rg.part_ld + tp];
       m2 = fmaxf(m2, p.m2);
       zt = fmaxf(zt, p.zt);
     }
     float l = 0.0f;
     for (int s = 0; s < nsplit; ++s) {
-      FwdPartial p = partials[(int64_t)s * T + t];
+      FwdPartial p = partials[(int64_t)s * rg.part_ld + tp];
       l += p.l * exp2f(p.m2 - m2);
     }
     const float lse = (m2 + log2f(l)) * kLn2;
@@ -143,17 +146,17 @@ fwd_finalize_kernel(const FwdPartial* __restrict__ partials, int nsplit, const i
     double b = 0.0;
 #pragma unroll
     for (int w = 0; w < kFinalizeThreads / 32; ++w) b += s_part[w];
-    block_sums[blockIdx.x] = b;
+    block_sums[rg.block0 + blockIdx.x] = b;
     __threadfence();
     int ticket = atomicAdd(&counters[1], 1);
-    s_last = (ticket == (int)gridDim.x - 1);
+    s_last = (ticket == rg.total_blocks - 1);
   }
   __syncthreads();
   if (s_last) {                              // the last block to finish folds all blocks in index order
     __threadfence();
     double acc = 0.0;
     const volatile double* bs = block_sums;
-    for (int i = threadIdx.x; i < (int)gridDim.x; i += kFinalizeThreads) acc += bs[i];
+    for (int i = threadIdx.x; i < rg.total_blocks; i += kFinalizeThreads) acc += bs[i];
     acc = warp_sum_f64(acc);
     __syncthreads();
     if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = acc;
@@ -425,13 +428,25 @@ cudaError_t launch_fwd_finalize(const FwdPartial* partials, int nsplit, const in
                                 float* loss, float* logp, float* lse, float* coef, float* seq_sums,
                                 double* block_sums, int32_t* counters, const int32_t* seq_cnt, int agg_mode,
                                 int32_t global_tokens, int32_t global_responses,
-                                int64_t fin_blocks, int32_t* d_status, cudaStream_t st) {
-  fwd_finalize_kernel<<<(unsigned)fin_blocks, kFinalizeThreads, 0, st>>>(
+                                int64_t fin_blocks, int32_t* d_status, cudaStream_t st,
+                                const FinalizeRange* range) {
+  // Default: one launch over all rows.  With a range: rows [t_begin, T) of a larger batch whose
+  // blocks are numbered from block0; T is then the end of the range and the per-response sums
+  // are left to the launch that covers the last rows.
+  FinalizeRange rg;
+  rg.t_begin = 0; rg.part_ld = T; rg.block0 = 0; rg.total_blocks = (int)fin_blocks; rg.last = 1;
+  unsigned blocks = (unsigned)fin_blocks;
+  if (range) {
+    rg = *range;
+    blocks = (unsigned)ceil_div(T - rg.t_begin, kFinalizeThreads);
+  }
+  if (blocks == 0) return cudaSuccess;
+  fwd_finalize_kernel<<<blocks, kFinalizeThreads, 0, st>>>(
       partials, nsplit, y, logp_old, mask, cu_seqlens, a_norm, T, V, S, clip_lo, clip_hi,
-      loss, logp, lse, coef, block_sums, counters, seq_cnt, agg_mode, global_tokens, global_responses, d_status);
+      loss, logp, lse, coef, block_sums, counters, seq_cnt, agg_mode, global_tokens, global_responses, d_status, rg);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  if (seq_sums && S > 0) {
+  if (seq_sums && S > 0 && rg.last) {
     seq_sums_kernel<<<S, 256, 0, st>>>(logp, logp_old, mask, cu_seqlens, seq_sums);
     e = cudaGetLastError();
   }

@@ -5,6 +5,11 @@
 //         per token row in registers across the vocabulary tiles of its split.
 //   G   : the same contraction for one chunk of token rows; epilogue turns each logit
 //         into g = c_t (1[v=y_t] - e^{z-lse_t}) and writes it as bf16 into the chunk buffer.
+//   E   : the same contraction again, for the one-pass forward+backward: epilogue keeps the
+//         forward's online statistics AND writes every logit of the chunk as
+//         e = 2^(z log2e - ref), bf16, with one reference exponent per row and 64 columns;
+//         a streaming kernel turns e into g once the row's lse is known, so the backward
+//         needs no second logits contraction.
 //   DH  : dH_chunk = G W        (A = G, K-major;  B = W read as an N-major operand)
 //   DW  : dW (+)= G^T H_chunk   (A = G read as an M-major operand; B = H, N-major)
 //
@@ -62,7 +67,7 @@ constexpr int kProducerSleepNs = 32;
 
 constexpr float kLog2e = 1.4426950408889634f;
 
-enum : int { MODE_FWD = 0, MODE_G = 1, MODE_DH = 2, MODE_DW = 3 };
+enum : int { MODE_FWD = 0, MODE_G = 1, MODE_DH = 2, MODE_DW = 3, MODE_E = 4 };
 
 struct GemmParams {
   int m_tiles, n_tiles, nsplit, per_split;   // work decomposition: unit = (row tile, split of the column tiles)
@@ -78,9 +83,12 @@ struct GemmParams {
   const float* coef;
   float grad_loss;
   FwdPartial* partials;
-  int64_t T;
+  int64_t T;                                 // stride between the splits' partials (rows they cover)
+  int64_t part_row0;                         // global row that partial 0 of a split belongs to
   __nv_bfloat16* G;
   int64_t ldg;
+  float* ref;                                // E: reference exponent of (64-column group, chunk row), [groups][ref_ld]
+  int64_t ref_ld;
   // DH / DW
   void* out;
   int out_bf16;
@@ -476,7 +484,7 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       float m2 = -CUDART_INF_F, l = 0.0f, zt = -CUDART_INF_F;             // FWD
       int32_t yt = -1;
       float c = 0.0f, lse2 = 0.0f;                                         // G
-      if (MODE == MODE_FWD || MODE == MODE_G) {
+      if (MODE == MODE_FWD || MODE == MODE_G || MODE == MODE_E) {
         if (row_ok) yt = p.y[grow];
         if (MODE == MODE_G && row_ok) { c = p.grad_loss * p.coef[grow]; lse2 = p.lse[grow] * kLog2e; }
       }
@@ -521,6 +529,80 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
               const int jj = yt - col0;
 #pragma unroll
               for (int j = 0; j < 32; ++j) if (j == jj) zt = __uint_as_float(v[j]);
+            }
+          }
+        } else if (MODE == MODE_E) {
+          // Forward statistics and the stored exponentials in one pass.  Per 64 columns the row's
+          // largest logit gives the reference: e = 2^(z log2e - ref) <= 1 keeps full bf16 precision
+          // for the entries that matter whatever the range of the logits, and ref is written once
+          // per (64-column group, row) -- lanes are consecutive rows, so the store is coalesced.
+          __nv_bfloat16* obase = p.G + ((int64_t)un.m_tile * GROUP_M + warp_row0) * p.ldg;
+          float* ref_row = p.ref + (int64_t)un.m_tile * GROUP_M + row;
+#pragma unroll 1
+          for (int r2 = 0; r2 < HALF_N / 64; ++r2) {
+            const int col0 = col_half + r2 * 64;
+            uint4 piece[8];
+            float ref2 = 0.0f;
+            if (col0 < p.cols_valid) {
+              uint32_t v0[32], v1[32];
+              tmem_ld32_nowait(taddr + r2 * 64, v0);
+              tmem_ld32_nowait(taddr + r2 * 64 + 32, v1);
+              tmem_wait_ld(v0);
+              tmem_wait_ld(v1);
+              if (col0 + 64 > p.cols_valid) {                          // ragged end of the vocabulary
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                  if (col0 + j >= p.cols_valid) v0[j] = __float_as_uint(-CUDART_INF_F);
+                  if (col0 + 32 + j >= p.cols_valid) v1[j] = __float_as_uint(-CUDART_INF_F);
+                }
+              }
+              float mx0 = __uint_as_float(v0[0]), mx1 = __uint_as_float(v0[1]);
+              float mx2 = __uint_as_float(v1[0]), mx3 = __uint_as_float(v1[1]);
+#pragma unroll
+              for (int j = 2; j < 32; j += 2) {
+                mx0 = fmaxf(mx0, __uint_as_float(v0[j]));
+                mx1 = fmaxf(mx1, __uint_as_float(v0[j + 1]));
+                mx2 = fmaxf(mx2, __uint_as_float(v1[j]));
+                mx3 = fmaxf(mx3, __uint_as_float(v1[j + 1]));
+              }
+              ref2 = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * kLog2e;
+              if (yt >= col0 && yt < col0 + 64) {
+                const int jj = yt - col0;
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                  if (j == jj) zt = __uint_as_float(v0[j]);
+                  if (j + 32 == jj) zt = __uint_as_float(v1[j]);
+                }
+              }
+              const float neg = -ref2;
+              float s0 = 0.0f, s1 = 0.0f, s2 = 0.0f, s3 = 0.0f;
+#pragma unroll
+              for (int j = 0; j < 32; j += 2) {
+                const float e0 = fast_exp2(fmaf(__uint_as_float(v0[j]), kLog2e, neg));
+                const float e1 = fast_exp2(fmaf(__uint_as_float(v0[j + 1]), kLog2e, neg));
+                const float e2 = fast_exp2(fmaf(__uint_as_float(v1[j]), kLog2e, neg));
+                const float e3 = fast_exp2(fmaf(__uint_as_float(v1[j + 1]), kLog2e, neg));
+                s0 += e0; s1 += e1; s2 += e2; s3 += e3;
+                v0[j] = __float_as_uint(e0); v0[j + 1] = __float_as_uint(e1);
+                v1[j] = __float_as_uint(e2); v1[j + 1] = __float_as_uint(e3);
+              }
+              const float mn = fmaxf(m2, ref2);
+              l = fmaf(l, fast_exp2(m2 - mn), ((s0 + s1) + (s2 + s3)) * fast_exp2(ref2 - mn));
+              m2 = mn;
+              bf16_values(v0, piece);
+              bf16_values(v1, piece + 4);
+            } else {                                                   // pad columns: e = 0
+#pragma unroll
+              for (int q = 0; q < 8; ++q) piece[q] = make_uint4(0u, 0u, 0u, 0u);
+            }
+            ref_row[(int64_t)(col0 >> 6) * p.ref_ld] = ref2;
+            stage_put(stage, lane, piece);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              int r, cc;
+              const uint4 val = stage_get(stage, lane, i, r, cc);
+              if (grow_warp0 + r < p.rows_valid)
+                *reinterpret_cast<uint4*>(obase + (int64_t)r * p.ldg + col0 + cc * 8) = val;
             }
           }
         } else if (MODE == MODE_G || (MODE == MODE_DH && p.out_bf16)) {
@@ -593,10 +675,10 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         __syncwarp();
         if (lane == 0) mbar_arrive_cluster(tempty_leader);
       }
-      if (MODE == MODE_FWD && ok && row_ok) {
+      if ((MODE == MODE_FWD || MODE == MODE_E) && ok && row_ok) {
         FwdPartial part;
         part.m2 = m2; part.l = l; part.zt = zt; part.pad = 0.0f;
-        p.partials[(int64_t)((u % p.nsplit) * 2 + half) * p.T + grow] = part;
+        p.partials[(int64_t)((u % p.nsplit) * 2 + half) * p.T + (grow - p.part_row0)] = part;
       }
     }
   }
@@ -611,6 +693,69 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   cluster_sync_all();                       // the peer may still be reading this CTA's shared / tensor memory
   if (warp == 0)
     asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+}
+
+// One-pass forward+backward, second half: once a row's lse and coef exist, turn the stored
+// e = 2^(z log2e - ref) of the chunk into g = c_t (1[v = y_t] - e 2^(ref - lse_t log2e)), in place.
+// A block covers 32 rows x 64 columns per step (lane -> row lane/8, 16-byte piece lane%8), so every
+// warp-wide access is four whole 128-byte row pieces and the four references a warp needs share a
+// sector.  Rows without gradient are zero-filled without being read.  Streaming: 4 bytes per logit.
+constexpr int kE2gThreads = 256;
+constexpr int kE2gRows = 32;
+constexpr int kE2gUnroll = 4;
+
+__global__ void __launch_bounds__(kE2gThreads)
+e_to_g_kernel(__nv_bfloat16* __restrict__ G, int64_t ldg, const float* __restrict__ ref, int64_t ref_ld,
+              int64_t rows, int n_groups, int groups_per_block, const int32_t* __restrict__ y,
+              const float* __restrict__ lse, const float* __restrict__ coef, float grad_loss, int64_t row0) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int64_t r = (int64_t)blockIdx.x * kE2gRows + warp * 4 + (lane >> 3);
+  if (r >= rows) return;
+  const int piece = lane & 7;
+  const float c = grad_loss * coef[row0 + r];
+  const float lse2 = lse[row0 + r] * kLog2e;
+  const int32_t yt = y[row0 + r];
+  uint4* grow = reinterpret_cast<uint4*>(G + r * ldg) + piece;       // + 8 per 64-column group
+  const float* rrow = ref + r;
+  const int g_begin = blockIdx.y * groups_per_block;
+  const int g_end = min(g_begin + groups_per_block, n_groups);
+  if (c == 0.0f) {
+    for (int g = g_begin; g < g_end; ++g) grow[(int64_t)g * 8] = make_uint4(0u, 0u, 0u, 0u);
+    return;
+  }
+  const float nc = -c;
+  for (int g0 = g_begin; g0 < g_end; g0 += kE2gUnroll) {
+    uint4 v[kE2gUnroll];
+    float sc[kE2gUnroll];
+#pragma unroll
+    for (int i = 0; i < kE2gUnroll; ++i) {
+      if (g0 + i < g_end) {
+        v[i] = grow[(int64_t)(g0 + i) * 8];
+        sc[i] = rrow[(int64_t)(g0 + i) * ref_ld];
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < kE2gUnroll; ++i) {
+      if (g0 + i < g_end) {
+        const float scale = nc * fast_exp2(sc[i] - lse2);
+        const int col0 = (g0 + i) * 64 + piece * 8;
+        uint32_t w[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
+        float f[8];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          f[2 * q] = __uint_as_float(w[q] << 16) * scale;
+          f[2 * q + 1] = __uint_as_float(w[q] & 0xFFFF0000u) * scale;
+        }
+        if (yt >= col0 && yt < col0 + 8) {
+          const int jj = yt - col0;
+#pragma unroll
+          for (int j = 0; j < 8; ++j) if (j == jj) f[j] += c;
+        }
+        grow[(int64_t)(g0 + i) * 8] = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]),
+                                                 pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
+      }
+    }
+  }
 }
 
 // A wait that nothing ever satisfies, through the same bounded-wait routine the pipeline uses:
@@ -808,6 +953,53 @@ BwdWs bwd_ws_layout(int64_t T, int32_t d, int32_t V) {
   return L;
 }
 
+namespace {
+
+// The two output contractions of one chunk whose g sits in the chunk buffer:
+// dH rows of the chunk = G W, then dW (+)= G^T H_chunk.
+cudaError_t launch_chunk_dh_dw(const CUtensorMap& mG_k, const CUtensorMap& mG_mn, const CUtensorMap& mW_mn,
+                               const CUtensorMap& mH_mn, int64_t t0, int64_t rows, int64_t T, int32_t d, int32_t V,
+                               void* dH, int32_t dH_dtype, float* dW, int dw_accumulate, uint32_t* progress,
+                               int32_t* d_status, cudaStream_t st) {
+  const int n_tiles_d = (int)ceil_div(d, BN);
+  cudaError_t e;
+  {
+    GemmParams p{};
+    p.m_tiles = (int)ceil_div(rows, GROUP_M);
+    p.n_tiles = n_tiles_d;
+    p.nsplit = n_tiles_d;
+    p.per_split = 1;
+    p.k_blocks = (int)ceil_div(V, BK);
+    p.a_row0 = 0;
+    p.b_k0 = 0;
+    p.rows_valid = T;
+    p.cols_valid = d;
+    p.out_row0 = t0;
+    p.out = dH; p.out_bf16 = (dH_dtype == SPO_DTYPE_BF16); p.ldo = d; p.accumulate = 0;
+    p.d_status = d_status;
+    if ((e = launch_gemm<MODE_DH>(mG_k, mW_mn, p, progress, st)) != cudaSuccess) return e;
+  }
+  {
+    GemmParams p{};
+    p.m_tiles = (int)ceil_div(V, GROUP_M);
+    p.n_tiles = n_tiles_d;
+    p.nsplit = n_tiles_d;
+    p.per_split = 1;
+    p.k_blocks = (int)ceil_div(rows, BK);
+    p.a_row0 = 0;
+    p.b_k0 = (int)t0;
+    p.rows_valid = V;
+    p.cols_valid = d;
+    p.out_row0 = 0;
+    p.out = dW; p.out_bf16 = 0; p.ldo = d; p.accumulate = dw_accumulate;
+    p.d_status = d_status;
+    if ((e = launch_gemm<MODE_DW>(mG_mn, mH_mn, p, progress, st)) != cudaSuccess) return e;
+  }
+  return cudaSuccess;
+}
+
+}  // namespace
+
 cudaError_t launch_bwd_bf16(const void* H, const void* W, const int32_t* y, const float* lse,
                             const float* coef, float grad_loss, int64_t T, int32_t d, int32_t V,
                             void* dH, int32_t dH_dtype, float* dW, int accumulate,
@@ -823,7 +1015,6 @@ cudaError_t launch_bwd_bf16(const void* H, const void* W, const int32_t* y, cons
       !make_map(&mW_mn, W, d, V, d, 64) || !make_map(&mH_mn, H, d, T, d, 64))
     return cudaErrorInvalidValue;
   const int n_tiles_v = (int)ceil_div(V, BN);
-  const int n_tiles_d = (int)ceil_div(d, BN);
   cudaError_t e;
   int chunk = 0;
   for (int64_t t0 = 0; t0 < T; t0 += L.chunk_rows, ++chunk) {
@@ -850,40 +1041,137 @@ cudaError_t launch_bwd_bf16(const void* H, const void* W, const int32_t* y, cons
       p.d_status = d_status;
       if ((e = launch_gemm<MODE_G>(mH_k, mW_k, p, progress, st)) != cudaSuccess) return e;
     }
-    // 2) dH rows of the chunk = G W
+    // 2) dH rows of the chunk = G W;  3) dW (+)= G^T H_chunk
+    if ((e = launch_chunk_dh_dw(mG_k, mG_mn, mW_mn, mH_mn, t0, rows, T, d, V, dH, dH_dtype, dW,
+                                (accumulate || chunk > 0) ? 1 : 0, progress, d_status, st)) != cudaSuccess)
+      return e;
+  }
+  return cudaSuccess;
+}
+
+// ---------------------------------------------------------------------------
+// One-pass forward+backward.  Per chunk of token rows: E contraction (forward statistics + stored
+// exponentials) -> per-token finalisation (lse, logp, coef, loss terms) -> e -> g in place ->
+// dH, dW.  Three contractions per token instead of the four of forward-then-backward.
+// ---------------------------------------------------------------------------
+FusedWs fused_ws_layout(int64_t T, int32_t d, int32_t V, int32_t S) {
+  FusedWs L{};
+  const BwdWs b = bwd_ws_layout(T, d, V);
+  L.chunk_rows = b.chunk_rows;
+  L.ldg = b.ldg;
+  const int n_tiles_v = (int)ceil_div(V, BN);
+  const int64_t t_eff = T > 0 ? T : 1;
+  // partials: the full chunk and the (shorter) last chunk may pick different split counts
+  const int64_t full_rows = t_eff < L.chunk_rows ? ceil_div(t_eff, GROUP_M) * GROUP_M : L.chunk_rows;
+  size_t part_elems = (size_t)2 * pick_fwd_split(full_rows / GROUP_M, n_tiles_v, d) * (size_t)full_rows;
+  const int64_t tail = t_eff % L.chunk_rows;
+  if (t_eff > L.chunk_rows && tail > 0) {
+    const int64_t tail_rows = ceil_div(tail, GROUP_M) * GROUP_M;
+    const size_t e2 = (size_t)2 * pick_fwd_split(tail_rows / GROUP_M, n_tiles_v, d) * (size_t)tail_rows;
+    if (e2 > part_elems) part_elems = e2;
+  }
+  L.fin_blocks = ceil_div(t_eff, kFinalizeThreads);
+  size_t off = 0;
+  L.g = off;          off = align_up(off + (size_t)L.chunk_rows * (size_t)L.ldg * 2, 256);
+  L.ref = off;        off = align_up(off + sizeof(float) * (size_t)(L.ldg / 64) * (size_t)L.chunk_rows, 256);
+  L.partials = off;   off = align_up(off + sizeof(FwdPartial) * part_elems, 256);
+  L.progress = off;   off = align_up(off + kProgressBytes, 256);
+  L.block_sums = off; off = align_up(off + sizeof(double) * (size_t)L.fin_blocks, 256);
+  L.counters = off;   off = align_up(off + 4 * sizeof(int32_t), 256);
+  L.seq_cnt = off;    off = align_up(off + sizeof(int32_t) * (size_t)(S > 0 ? S : 1), 256);
+  L.total = off;
+  return L;
+}
+
+cudaError_t launch_fused_bf16(const FusedArgs& a, char* ws, const FusedWs& L, cudaStream_t st) {
+  __nv_bfloat16* G = reinterpret_cast<__nv_bfloat16*>(ws + L.g);
+  float* ref = reinterpret_cast<float*>(ws + L.ref);
+  FwdPartial* partials = reinterpret_cast<FwdPartial*>(ws + L.partials);
+  uint32_t* progress = reinterpret_cast<uint32_t*>(ws + L.progress);
+  double* block_sums = reinterpret_cast<double*>(ws + L.block_sums);
+  int32_t* counters = reinterpret_cast<int32_t*>(ws + L.counters);
+  int32_t* seq_cnt = reinterpret_cast<int32_t*>(ws + L.seq_cnt);
+  const spo_params& pr = *a.params;
+  const int64_t T = a.T;
+  const int32_t d = a.d, V = a.V;
+  cudaError_t e = launch_fwd_prepare(a.mask, T, a.cu_seqlens, a.S, pr.agg_mode, seq_cnt, counters, st);
+  if (e != cudaSuccess) return e;
+  if (T == 0) {
+    e = launch_fwd_finalize(partials, 0, a.y, a.logp_old, a.mask, a.cu_seqlens, a.a_norm, 0, V, a.S, pr.clip_lo,
+                            pr.clip_hi, a.loss, a.logp, a.lse, a.coef, a.seq_sums, block_sums, counters, seq_cnt,
+                            pr.agg_mode, pr.global_tokens, pr.global_responses, L.fin_blocks, a.d_status, st);
+    if (e != cudaSuccess) return e;
+    if (!a.accumulate) return cudaMemsetAsync(a.dW, 0, sizeof(float) * (size_t)V * d, st);
+    return cudaSuccess;
+  }
+  CUtensorMap mH_k, mW_k, mW_mn, mH_mn;
+  if (!make_map(&mH_k, a.H, d, T, d, kBoxA) || !make_map(&mW_k, a.W, d, V, d, kBoxB) ||
+      !make_map(&mW_mn, a.W, d, V, d, 64) || !make_map(&mH_mn, a.H, d, T, d, 64))
+    return cudaErrorInvalidValue;
+  const int n_tiles_v = (int)ceil_div(V, BN);
+  const int n_groups = (int)(L.ldg / 64);
+  int chunk = 0;
+  for (int64_t t0 = 0; t0 < T; t0 += L.chunk_rows, ++chunk) {
+    const int64_t rows = (T - t0) < L.chunk_rows ? (T - t0) : L.chunk_rows;
+    const int m_tiles = (int)ceil_div(rows, GROUP_M);
+    const int64_t rows_pad = (int64_t)m_tiles * GROUP_M;
+    CUtensorMap mG_k, mG_mn;
+    if (!make_map(&mG_k, G, V, rows, L.ldg, kBoxA) || !make_map(&mG_mn, G, V, rows, L.ldg, 64))
+      return cudaErrorInvalidValue;
+    // 1) logits of the chunk: online (max, sum, target logit) per row and split, e into the chunk buffer
+    const int nsplit = pick_fwd_split(m_tiles, n_tiles_v, d);
     {
       GemmParams p{};
       p.m_tiles = m_tiles;
-      p.n_tiles = n_tiles_d;
-      p.nsplit = n_tiles_d;
-      p.per_split = 1;
-      p.k_blocks = (int)ceil_div(V, BK);
-      p.a_row0 = 0;
-      p.b_k0 = 0;
+      p.n_tiles = n_tiles_v;
+      p.nsplit = nsplit;
+      p.per_split = (int)ceil_div(n_tiles_v, p.nsplit);
+      p.k_blocks = (int)ceil_div(d, BK);
+      p.a_row0 = (int)t0;
       p.rows_valid = T;
-      p.cols_valid = d;
+      p.cols_valid = V;
       p.out_row0 = t0;
-      p.out = dH; p.out_bf16 = (dH_dtype == SPO_DTYPE_BF16); p.ldo = d; p.accumulate = 0;
-      p.d_status = d_status;
-      if ((e = launch_gemm<MODE_DH>(mG_k, mW_mn, p, progress, st)) != cudaSuccess) return e;
+      p.y = a.y;
+      p.partials = partials;
+      p.T = rows_pad;
+      p.part_row0 = t0;
+      p.G = G; p.ldg = L.ldg;
+      p.ref = ref; p.ref_ld = L.chunk_rows;
+      p.d_status = a.d_status;
+      if ((e = launch_gemm<MODE_E>(mH_k, mW_k, p, progress, st)) != cudaSuccess) return e;
     }
-    // 3) dW (+)= G^T H_chunk
+    // 2) lse, logp, ratio, clipped surrogate and coef of the chunk's rows; loss terms per block
     {
-      GemmParams p{};
-      p.m_tiles = (int)ceil_div(V, GROUP_M);
-      p.n_tiles = n_tiles_d;
-      p.nsplit = n_tiles_d;
-      p.per_split = 1;
-      p.k_blocks = (int)ceil_div(rows, BK);
-      p.a_row0 = 0;
-      p.b_k0 = (int)t0;
-      p.rows_valid = V;
-      p.cols_valid = d;
-      p.out_row0 = 0;
-      p.out = dW; p.out_bf16 = 0; p.ldo = d; p.accumulate = (accumulate || chunk > 0) ? 1 : 0;
-      p.d_status = d_status;
-      if ((e = launch_gemm<MODE_DW>(mG_mn, mH_mn, p, progress, st)) != cudaSuccess) return e;
+      FinalizeRange rg;
+      rg.t_begin = t0;
+      rg.part_ld = rows_pad;
+      rg.block0 = (int)(t0 / kFinalizeThreads);
+      rg.total_blocks = (int)L.fin_blocks;
+      rg.last = (t0 + rows >= T) ? 1 : 0;
+      e = launch_fwd_finalize(partials, 2 * nsplit, a.y, a.logp_old, a.mask, a.cu_seqlens, a.a_norm, t0 + rows, V,
+                              a.S, pr.clip_lo, pr.clip_hi, a.loss, a.logp, a.lse, a.coef, a.seq_sums, block_sums,
+                              counters, seq_cnt, pr.agg_mode, pr.global_tokens, pr.global_responses, L.fin_blocks,
+                              a.d_status, st, &rg);
+      if (e != cudaSuccess) return e;
     }
+    // 3) e -> g in place
+    {
+      const int64_t row_blocks = ceil_div(rows, kE2gRows);
+      int col_blocks = (int)ceil_div((int64_t)sm_count() * 16, row_blocks);     // enough blocks to fill the device
+      if (col_blocks < 1) col_blocks = 1;
+      if (col_blocks > n_groups) col_blocks = n_groups;
+      int per = (int)ceil_div(n_groups, col_blocks);
+      per = (int)ceil_div(per, kE2gUnroll) * kE2gUnroll;
+      col_blocks = (int)ceil_div(n_groups, per);
+      dim3 grid((unsigned)row_blocks, (unsigned)col_blocks, 1);
+      e_to_g_kernel<<<grid, kE2gThreads, 0, st>>>(G, L.ldg, ref, L.chunk_rows, rows, n_groups, per, a.y, a.lse, a.coef,
+                                                  a.grad_loss, t0);
+      if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    }
+    // 4) dH rows of the chunk = G W;  5) dW (+)= G^T H_chunk
+    if ((e = launch_chunk_dh_dw(mG_k, mG_mn, mW_mn, mH_mn, t0, rows, T, d, V, a.dH, a.dH_dtype, a.dW,
+                                (a.accumulate || chunk > 0) ? 1 : 0, progress, a.d_status, st)) != cudaSuccess)
+      return e;
   }
   return cudaSuccess;
 }

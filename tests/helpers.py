@@ -28,8 +28,10 @@ def ws_bytes(which, **kw):
     return torch.empty(max(n, 256), dtype=torch.uint8, device="cuda")
 
 
-def run_loss(lb, params=None, grad_loss=1.0, dh_bf16=None, want_seq_sums=True, dw_init=None, mask_none=False):
-    """Forward + backward through the binding for a LossBatch; returns numpy outputs."""
+def run_loss(lb, params=None, grad_loss=1.0, dh_bf16=None, want_seq_sums=True, dw_init=None, mask_none=False,
+             one_pass=False):
+    """Forward + backward through the binding for a LossBatch; returns numpy outputs.
+    one_pass: a single spo_loss_fwd_bwd call instead of spo_loss_fwd followed by spo_loss_bwd."""
     import torch
     from paper_2509_13232_b200 import binding as B
     params = params or B.default_params()
@@ -46,8 +48,6 @@ def run_loss(lb, params=None, grad_loss=1.0, dh_bf16=None, want_seq_sums=True, d
     logp, lse, coef = (torch.full((max(T, 1),), float("nan"), **f32) for _ in range(3))
     seq = torch.zeros((max(S, 1), 3), **f32) if want_seq_sums else None
     st = status_word()
-    wsf = ws_bytes(B.WS_LOSS_FWD, T=T, d=d, V=V, B=S)
-    B.spo_loss_fwd(H, W, y, lo, mask, cu, an, loss, logp, lse, coef, seq, wsf, params, st)
     if dh_bf16 is None:
         dh_bf16 = lb.bf16
     dH = torch.full((max(T, 1), d), float("nan"), dtype=torch.bfloat16 if dh_bf16 else torch.float32, device="cuda")
@@ -57,8 +57,15 @@ def run_loss(lb, params=None, grad_loss=1.0, dh_bf16=None, want_seq_sums=True, d
     else:
         dW = dev(dw_init).clone()
         acc = 1
-    wsb = ws_bytes(B.WS_LOSS_BWD, T=T, d=d, V=V)
-    B.spo_loss_bwd(H, W, y, lse, coef, grad_loss, dH, dW, acc, wsb, params, st)
+    if one_pass:
+        ws = ws_bytes(B.WS_LOSS_FWD_BWD, T=T, d=d, V=V, B=S)
+        B.spo_loss_fwd_bwd(H, W, y, lo, mask, cu, an, grad_loss, loss, logp, lse, coef, seq, dH[:T], dW, acc, ws,
+                           params, st)
+    else:
+        wsf = ws_bytes(B.WS_LOSS_FWD, T=T, d=d, V=V, B=S)
+        B.spo_loss_fwd(H, W, y, lo, mask, cu, an, loss, logp, lse, coef, seq, wsf, params, st)
+        wsb = ws_bytes(B.WS_LOSS_BWD, T=T, d=d, V=V)
+        B.spo_loss_bwd(H, W, y, lse, coef, grad_loss, dH, dW, acc, wsb, params, st)
     torch.cuda.synchronize()
     return {
         "loss": float(loss[0].item()), "logp": logp[:T].cpu().numpy(), "lse": lse[:T].cpu().numpy(),

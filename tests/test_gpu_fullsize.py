@@ -36,11 +36,13 @@ def test_real_vocab_and_hidden_small_token_count_full_oracle():
     assert rel_fro(got["dW"][-64:], want["dW"][-64:]) <= 1e-2
 
 
+@pytest.mark.parametrize("path", ["onepass", "split"])
 @pytest.mark.parametrize("workload", ["cfg3_small_bf16", "cfg4_8b_bf16", "cfg5_longtail_bf16"])
-def test_full_size_sampled_rows_and_identities(workload):
+def test_full_size_sampled_rows_and_identities(workload, path):
+    """Both loss paths bench.py can time: one spo_loss_fwd_bwd call, or spo_loss_fwd then spo_loss_bwd."""
     import torch
     import bench
-    step = bench.Step(workload, torch.device("cuda", 0), 0)
+    step = bench.Step(workload, torch.device("cuda", 0), 0, path=path)
     step.run()
     torch.cuda.synchronize()
     assert int(step.status[0].item()) == 0
