@@ -37,7 +37,7 @@ UNIT = "tokens/s"
 TABLE_N = 1_000_000          # tracker table the step samples from and updates
 # DRAM read+write bytes of all launches of one cfg4 step, from ncu captures (profiles/); None = the
 # kernels of that path changed after the counters were taken
-CFG4_STEP_DRAM_BYTES = {"split": 1.23e12, "onepass": None}
+CFG4_STEP_DRAM_BYTES = {"split": 1.23e12, "onepass": 1.26e12}
 
 LOSS_SHAPES = {
     # workload: (d, V, w_std, old-logprob noise, reward probability)
@@ -367,8 +367,9 @@ def run_ours(args, rank, world, local_rank):
             "flops_per_token": (6 if step.onepass else 8) * step.d * step.V,
             "fwd_tflops": None if step.onepass else step.flops_fwd / (t_fwd / args.steps / 1e3) / 1e12,
             "bwd_tflops": None if step.onepass else step.flops_bwd / (t_bwd / args.steps / 1e3) / 1e12,
-            # DRAM read+write bytes of all launches of one step, from the ncu capture summarised in
-            # profiles/spo_gemm_kernel_cfg4_16responses_full.md, scaled by token rows; null for other shapes.
+            # DRAM read+write bytes of all launches of one step, from the ncu captures summarised in
+            # profiles/spo_loss_fwd_bwd_cfg4_16responses_full.md (one-pass) and
+            # profiles/spo_gemm_kernel_cfg4_16responses_full.md (split), scaled by token rows; null for other shapes.
             "traffic": CFG4_STEP_DRAM_BYTES.get("onepass" if step.onepass else "split") if (
                 args.workload == "cfg4_8b_bf16" and not args.responses and not args.custom and not args.mask_frac) else None,
         },
