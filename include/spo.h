@@ -104,9 +104,13 @@ int32_t spo_tracker_init(float* ab, const float* v0, int64_t N,
  * (0.5 for an empty entry), then B distinct prompts drawn by weight.
  *
  * The draw is successive weighted sampling without replacement, made
- * reproducible bit for bit: weights are computed in fp32 with IEEE-rounded
- * operations in the order n=a+b, num=a*b, den=n*n, inv=1/den, p=num*inv,
- * s=sqrt(p), w=s+eps; q_i = floor(w_i * 2^32) (uint64); C_i = q_0+..+q_i; Wtot = C_{N-1};
+ * reproducible bit for bit: weights are computed in fp32 by a fixed sequence of
+ * individually rounded operations (nothing fused): n=a+b, t=a*b, x=t*(n*n);
+ * for 2^-100 <= x <= 2^100 and a > 0 (any entry a tracker produces with both parameters
+ * positive): y0 = the float with bits 0x5f3759df - (bits(x) >> 1), three Newton steps
+ * y <- y*(1.5 - (0.5*x)*(y*y)), s = t*y (= sqrt(t)/n to 3e-7 relative); an empty entry has
+ * s = 0.5, an entry with a or b zero s = 0, any other magnitude s = sqrt((a/n)*(b/n));
+ * w = s+eps; q_i = floor(w_i * 2^32) (uint64); C_i = q_0+..+q_i; Wtot = C_{N-1};
  * for the k-th uniform U_k = floor(u_k * 2^32), t_k = floor(U_k*Wtot / 2^32),
  * candidate = first i with C_i > t_k; candidates are accepted in order k unless
  * already accepted, until B are accepted.

@@ -137,26 +137,43 @@ def sampling_weights(alpha, beta, eps_explore=EPS_EXPLORE):
 
 
 def sampling_weights_f32(alpha32, beta32, eps_explore=EPS_EXPLORE):
-    """The same weights in IEEE fp32, one correctly rounded operation per step.
+    """The same weights in IEEE fp32 as a fixed sequence of individually rounded operations.
 
-    v(1-v) is formed as alpha*beta/(alpha+beta)^2, which is the same quantity
-    without the cancellation of 1-v near v = 1.  Order of operations:
-    n = alpha+beta; num = alpha*beta; den = n*n; inv = 1/den; p = num*inv
-    (0.25 if n == 0); s = sqrt(p); w = s + eps.  numpy's float32 add, multiply,
-    divide and sqrt are each correctly rounded, so any IEEE implementation that
-    performs these steps without fusing them gives the same bits.
+    v(1-v) is formed as alpha*beta/(alpha+beta)^2, the same quantity without the
+    cancellation of 1-v near v = 1, and its square root as t/sqrt(t n^2):
+        n = alpha+beta; t = alpha*beta; den = n*n; x = t*den
+        2^-100 <= x <= 2^100 and alpha > 0 (every entry with both parameters positive that a tracker produces):
+            y0 = float32 with the bits 0x5f3759df - (bits(x) >> 1)      (reciprocal-square-root seed)
+            three Newton steps  y <- y * (1.5 - (0.5*x) * (y*y))
+            s = t * y
+        n == 0: s = 0.5;   alpha or beta zero with n > 0: s = 0
+        any other magnitude: s = sqrt((alpha/n) * (beta/n))
+        w = s + eps
+    numpy's float32 add, subtract, multiply, divide and sqrt are each correctly rounded and
+    nothing here is fused, so any IEEE implementation that performs these steps in this order
+    gives the same bits.  (This order of operations is this implementation's own choice for
+    Eq. "sampling_coef"; the pins hold it to the float64 definition.)
     """
+    f = np.float32
     a = np.asarray(alpha32, dtype=np.float32)
     b = np.asarray(beta32, dtype=np.float32)
-    one = np.float32(1.0)
-    n = a + b
-    num = a * b
-    den = n * n
-    pos = n > np.float32(0.0)
-    inv = one / np.where(pos, den, one)
-    p = np.where(pos, num * inv, np.float32(0.25)).astype(np.float32)
-    s = np.sqrt(p)
-    w = s + np.float32(eps_explore)
+    with np.errstate(all="ignore"):
+        n = a + b
+        t = a * b
+        den = n * n
+        x = t * den
+        h = f(0.5) * x
+        y = (np.uint32(0x5F3759DF) - (x.view(np.uint32) >> np.uint32(1))).view(np.float32)
+        for _ in range(3):
+            y = y * (f(1.5) - h * (y * y))
+        s = t * y
+        common = (x >= f(2.0 ** -100)) & (x <= f(2.0 ** 100)) & (a > f(0.0))
+        empty = n == f(0.0)
+        one_zero = (np.minimum(a, b) == f(0.0)) & (n > f(0.0))
+        n_safe = np.where(n > f(0.0), n, f(1.0))
+        rare = np.sqrt((a / n_safe) * (b / n_safe))
+        s = np.where(common, s, np.where(empty, f(0.5), np.where(one_zero, f(0.0), rare))).astype(np.float32)
+        w = s + f(eps_explore)
     return w.astype(np.float32)
 
 

@@ -30,21 +30,46 @@ __global__ void tracker_init_kernel(float2* __restrict__ ab, const float* __rest
 }
 
 // ---------------------------------------------------------------------------
-// Sampling weight of one table entry (Eq. "sampling_coef") in IEEE fp32, one
-// rounded operation per step so that a host restatement gives the same bits:
-// n=a+b, num=a*b, den=n*n, inv=1/den, p=num*inv (0.25 for an empty entry), s=sqrt(p), w=s+eps.
-// (A correctly rounded reciprocal plus a multiply costs about half the instructions of a
-// correctly rounded division; this kernel is bound by instruction issue, not by HBM.)
-// A negative or non-finite entry yields weight 0 and *bad = true.
+// Sampling weight of one table entry (Eq. "sampling_coef"), w = sqrt(v(1-v)) + eps with
+// v(1-v) = alpha beta / (alpha+beta)^2, in fp32 as a fixed sequence of individually rounded
+// operations (no contraction into FMAs) so that a host restatement gives the same bits:
+//   n = a+b; t = a*b; den = n*n; x = t*den;
+//   common case, 2^-100 <= x <= 2^100 and a > 0:  s = t * y  with y ~ 1/sqrt(x) = 1/(sqrt(t) n):
+//     y0 = bits(0x5f3759df - (bits(x) >> 1)); three Newton steps y <- y*(1.5 - (0.5x)*(y*y));
+//   n == 0 (empty entry): s = 0.5;   a or b zero (n > 0): s = 0;
+//   any other magnitude: s = sqrt((a/n)*(b/n)) with IEEE division and square root;
+//   w = s + eps.
+// The Newton form needs 20 plain multiplies / subtracts where a correctly rounded reciprocal and
+// square root need about twice that; the table scan is bound by instruction issue, so this is what
+// sets its speed.  s is within 3e-7 relative of the exact value.
+// A negative or non-finite entry yields weight 0 and sets SPO_DEV_NONFINITE in *d_status.
 // ---------------------------------------------------------------------------
-__device__ __forceinline__ float entry_weight(float a, float b, float eps, bool& bad) {
+// Everything but the common case, out of line so that the scan's hot loop stays short:
+// invalid entries (weight 0, status bit), empty entries, a zero alpha or beta, extreme magnitudes.
+__device__ __noinline__ float entry_weight_uncommon(float a, float b, float eps, int32_t* d_status) {
   const float n = __fadd_rn(a, b);
-  const bool wrong = (fminf(a, b) < 0.0f) | !(n < CUDART_INF_F);     // negative, NaN or Inf
-  bad |= wrong;
-  float p = 0.25f;
-  if (n > 0.0f) p = __fmul_rn(__fmul_rn(a, b), __frcp_rn(__fmul_rn(n, n)));
-  const float w = __fadd_rn(__fsqrt_rn(p), eps);
-  return wrong ? 0.0f : w;
+  if ((fminf(a, b) < 0.0f) | !(n < CUDART_INF_F)) {                  // negative, NaN or Inf
+    flag(d_status, SPO_DEV_NONFINITE);
+    return 0.0f;
+  }
+  float s;
+  if (n == 0.0f) s = 0.5f;
+  else if (fminf(a, b) == 0.0f) s = 0.0f;
+  else s = __fsqrt_rn(__fmul_rn(__fdiv_rn(a, n), __fdiv_rn(b, n)));
+  return __fadd_rn(s, eps);
+}
+
+__device__ __forceinline__ float entry_weight(float a, float b, float eps, int32_t* d_status) {
+  const float n = __fadd_rn(a, b);
+  const float t = __fmul_rn(a, b);
+  const float x = __fmul_rn(t, __fmul_rn(n, n));
+  // x in range and a > 0 imply b > 0 and everything finite: one test covers validity too
+  if (!((x >= 0x1p-100f) & (x <= 0x1p100f) & (a > 0.0f))) return entry_weight_uncommon(a, b, eps, d_status);
+  const float h = __fmul_rn(0.5f, x);
+  float y = __uint_as_float(0x5f3759dfu - (__float_as_uint(x) >> 1));
+#pragma unroll
+  for (int k = 0; k < 3; ++k) y = __fmul_rn(y, __fsub_rn(1.5f, __fmul_rn(h, __fmul_rn(y, y))));
+  return __fadd_rn(__fmul_rn(t, y), eps);
 }
 
 // q = floor(w * 2^32): exact, the scale is a power of two (w is finite, non-negative, far below 2^32).
@@ -68,6 +93,8 @@ __device__ __forceinline__ unsigned long long warp_incl_scan_u64(unsigned long l
 }
 
 // One block = one tile of kSampleTile entries: 256 threads x 4 float4 loads (2 entries each).
+// EMIT: also write the weights.  Full tiles take a path without per-load bounds tests.
+template <bool EMIT>
 __global__ void __launch_bounds__(256)
 sample_tile_sums_kernel(const float4* __restrict__ ab4, int64_t N, float eps, float2* __restrict__ out_w2,
                         float* __restrict__ out_w, unsigned long long* __restrict__ tile_sums,
@@ -76,27 +103,39 @@ sample_tile_sums_kernel(const float4* __restrict__ ab4, int64_t N, float eps, fl
   const int64_t first_pair = tile * (kSampleTile / 2);
   const int64_t n_pairs = N >> 1;
   unsigned long long sum = 0;
-  bool bad = false;
+  if (first_pair + kSampleTile / 2 <= n_pairs) {
+    float4 e[4];
 #pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    int64_t p = first_pair + j * 256 + threadIdx.x;
-    if (p < n_pairs) {
-      float4 e = __ldg(ab4 + p);
-      float w0 = entry_weight(e.x, e.y, eps, bad);
-      float w1 = entry_weight(e.z, e.w, eps, bad);
+    for (int j = 0; j < 4; ++j) e[j] = __ldg(ab4 + first_pair + j * 256 + threadIdx.x);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float w0 = entry_weight(e[j].x, e[j].y, eps, d_status);
+      const float w1 = entry_weight(e[j].z, e[j].w, eps, d_status);
       sum += quantise(w0) + quantise(w1);
-      if (out_w2) out_w2[p] = make_float2(w0, w1);
-    } else if (p == n_pairs && (N & 1)) {      // odd tail entry
-      const float* ab = reinterpret_cast<const float*>(ab4);
-      float w0 = entry_weight(ab[2 * (N - 1)], ab[2 * (N - 1) + 1], eps, bad);
-      sum += quantise(w0);
-      if (out_w) out_w[N - 1] = w0;
+      if (EMIT) out_w2[first_pair + j * 256 + threadIdx.x] = make_float2(w0, w1);
+    }
+  } else {
+#pragma unroll 1
+    for (int j = 0; j < 4; ++j) {
+      const int64_t p = first_pair + j * 256 + threadIdx.x;
+      if (p < n_pairs) {
+        const float4 e = __ldg(ab4 + p);
+        const float w0 = entry_weight(e.x, e.y, eps, d_status);
+        const float w1 = entry_weight(e.z, e.w, eps, d_status);
+        sum += quantise(w0) + quantise(w1);
+        if (EMIT) out_w2[p] = make_float2(w0, w1);
+      } else if (p == n_pairs && (N & 1)) {      // odd tail entry
+        const float* ab = reinterpret_cast<const float*>(ab4);
+        const float w0 = entry_weight(ab[2 * (N - 1)], ab[2 * (N - 1) + 1], eps, d_status);
+        sum += quantise(w0);
+        if (EMIT) out_w[N - 1] = w0;
+      }
     }
   }
   sum = warp_sum_u64(sum);
   __shared__ unsigned long long s_part[8];
   if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = sum;
-  if (__syncthreads_or(bad) && threadIdx.x == 0) flag(d_status, SPO_DEV_NONFINITE);
+  __syncthreads();
   if (threadIdx.x == 0) {
     unsigned long long t = 0;
 #pragma unroll
@@ -174,17 +213,16 @@ sample_search_kernel(const float* __restrict__ ab, int64_t N, float eps, const f
       for (int64_t c0 = 0; c0 < n_here && off < 0; c0 += 128) {
         const int64_t i0 = c0 + 4 * lane;
         unsigned long long q[4] = {0ull, 0ull, 0ull, 0ull};
-        bool bad = false;
         if (i0 + 3 < n_here) {
           const float4 e0 = __ldg(ab4 + i0 / 2), e1 = __ldg(ab4 + i0 / 2 + 1);
-          q[0] = quantise(entry_weight(e0.x, e0.y, eps, bad));
-          q[1] = quantise(entry_weight(e0.z, e0.w, eps, bad));
-          q[2] = quantise(entry_weight(e1.x, e1.y, eps, bad));
-          q[3] = quantise(entry_weight(e1.z, e1.w, eps, bad));
+          q[0] = quantise(entry_weight(e0.x, e0.y, eps, d_status));
+          q[1] = quantise(entry_weight(e0.z, e0.w, eps, d_status));
+          q[2] = quantise(entry_weight(e1.x, e1.y, eps, d_status));
+          q[3] = quantise(entry_weight(e1.z, e1.w, eps, d_status));
         } else {
 #pragma unroll
           for (int j = 0; j < 4; ++j)
-            if (i0 + j < n_here) q[j] = quantise(entry_weight(ab[2 * (base + i0 + j)], ab[2 * (base + i0 + j) + 1], eps, bad));
+            if (i0 + j < n_here) q[j] = quantise(entry_weight(ab[2 * (base + i0 + j)], ab[2 * (base + i0 + j) + 1], eps, d_status));
         }
         const unsigned long long mine = q[0] + q[1] + q[2] + q[3];
         const unsigned long long incl = warp_incl_scan_u64(mine, lane);
@@ -571,9 +609,13 @@ cudaError_t launch_sample(const float* ab, int64_t N, const float* u, int32_t M,
   auto* vals = reinterpret_cast<int32_t*>(ws + L.vals);
   cudaError_t e;
   if ((e = cudaMemsetAsync(ws, 0, L.zeroed_bytes, st)) != cudaSuccess) return e;
-  sample_tile_sums_kernel<<<(unsigned)L.n_tiles, 256, 0, st>>>(
-      reinterpret_cast<const float4*>(ab), N, eps, reinterpret_cast<float2*>(out_w), out_w, tile_sums, super_sums,
-      d_status);
+  if (out_w)
+    sample_tile_sums_kernel<true><<<(unsigned)L.n_tiles, 256, 0, st>>>(
+        reinterpret_cast<const float4*>(ab), N, eps, reinterpret_cast<float2*>(out_w), out_w, tile_sums, super_sums,
+        d_status);
+  else
+    sample_tile_sums_kernel<false><<<(unsigned)L.n_tiles, 256, 0, st>>>(
+        reinterpret_cast<const float4*>(ab), N, eps, nullptr, nullptr, tile_sums, super_sums, d_status);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   sample_search_kernel<<<(unsigned)ceil_div((int64_t)M * 32, 256), 256, 0, st>>>(
       ab, N, eps, u, M, tile_sums, super_sums, L.n_tiles, L.n_super, cand, keys, vals, (uint32_t)(L.hash_slots - 1),
