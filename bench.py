@@ -37,7 +37,7 @@ UNIT = "tokens/s"
 TABLE_N = 1_000_000          # tracker table the step samples from and updates
 # DRAM read+write bytes of all launches of one cfg4 step, from ncu captures (profiles/); None = the
 # kernels of that path changed after the counters were taken
-CFG4_STEP_DRAM_BYTES = {"split": 1.23e12, "onepass": 1.26e12}
+CFG4_STEP_DRAM_BYTES = {"split": 1.23e12, "onepass": 1.03e12}
 
 LOSS_SHAPES = {
     # workload: (d, V, w_std, old-logprob noise, reward probability)
@@ -173,10 +173,11 @@ class Step:
         self.bwd_chunks = -(-self.T // chunk_rows)
         # kernels launched by one step: sampling 3 (tile sums, search, accept), advantages 1, update 1, then
         # split path: forward 3 (count, contraction, finalise), backward 3 per chunk;
-        # one-pass path: count 1, per chunk 5 (logits contraction, finalise, e->g, dH, dW).  Memsets are not counted.
+        # one-pass path: count 1, per chunk 4 (logits contraction [+ e->g of the chunk before on side warps],
+        # finalise, dH, dW), and one e->g kernel for the last chunk.  Memsets are not counted.
         self.flops_fwd = 2.0 * self.T * d * V
         if self.onepass:
-            self.launches = 3 + 1 + 1 + 1 + 5 * self.bwd_chunks
+            self.launches = 3 + 1 + 1 + 1 + 4 * self.bwd_chunks + 1
             self.flops_bwd = 4.0 * self.T * d * V
         else:
             self.launches = 3 + 1 + 1 + 3 + 3 * self.bwd_chunks

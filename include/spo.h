@@ -292,7 +292,9 @@ int32_t spo_loss_bwd(const void* H, const void* W, int32_t dtype, const int32_t*
  *
  *   arguments   as in spo_loss_fwd and spo_loss_bwd; lse and coef are outputs here
  *   ws          device scratch, spo_workspace_bytes(SPO_WS_LOSS_FWD_BWD, T, d, V, 0, S, 0) bytes:
- *               the chunk buffer, its reference exponents (1/32 of it) and the forward's partials
+ *               two chunk buffers when T exceeds one chunk (the chunks are software-pipelined: the
+ *               e -> g pass of one chunk runs on spare warps of the next chunk's logits contraction),
+ *               their reference exponents (1/32 of them) and the forward's partials
  * Status bits as spo_loss_fwd.
  */
 int32_t spo_loss_fwd_bwd(const void* H, const void* W, int32_t dtype,

@@ -118,13 +118,15 @@ BwdWs bwd_ws_layout(int64_t T, int32_t d, int32_t V);
 
 // one-pass forward+backward (bf16)
 struct FusedWs {
-  size_t g;             // bf16 [chunk_rows][ldg]: e, then g, of one chunk
-  size_t ref;           // float [ldg/64][chunk_rows]: reference exponents of e
+  size_t g;             // n_buf x bf16 [chunk_rows][ldg]: e, then g, of one chunk each
+  size_t ref;           // n_buf x float [ldg/64][chunk_rows]: reference exponents of e
+  size_t g_bytes, ref_bytes;   // size of one of them
   size_t partials;      // FwdPartial [2*nsplit][rows of the chunk]
   size_t progress, block_sums, counters, seq_cnt;
   size_t total;
   int64_t chunk_rows, ldg;
   int64_t fin_blocks;
+  int n_buf;            // 2 when there is more than one chunk (chunks are software-pipelined), else 1
 };
 FusedWs fused_ws_layout(int64_t T, int32_t d, int32_t V, int32_t S);
 struct FusedArgs {

@@ -69,6 +69,21 @@ constexpr float kLog2e = 1.4426950408889634f;
 
 enum : int { MODE_FWD = 0, MODE_G = 1, MODE_DH = 2, MODE_DW = 3, MODE_E = 4 };
 
+// Work description of the e -> g pass of the one-pass path (see e_to_g_rows).
+struct E2gJob {
+  __nv_bfloat16* G;        // [rows][ldg]
+  int64_t ldg;
+  const float* ref;        // [n_groups][ref_ld]
+  int64_t ref_ld;
+  int64_t rows;            // rows of the chunk that exist
+  int n_groups;            // ldg / 64
+  const int32_t* y;        // per-token arrays, indexed by row0 + chunk row
+  const float* lse;
+  const float* coef;
+  float grad_loss;
+  int64_t row0;
+};
+
 struct GemmParams {
   int m_tiles, n_tiles, nsplit, per_split;   // work decomposition: unit = (row tile, split of the column tiles)
   int k_blocks;                              // K / 64, rounded up
@@ -89,6 +104,7 @@ struct GemmParams {
   int64_t ldg;
   float* ref;                                // E: reference exponent of (64-column group, chunk row), [groups][ref_ld]
   int64_t ref_ld;
+  E2gJob side;                               // E with side warps: the previous chunk's e -> g (rows = 0: nothing)
   // DH / DW
   void* out;
   int out_bf16;
@@ -314,6 +330,77 @@ __host__ __device__ constexpr uint32_t instr_desc(bool a_mn, bool b_mn) {
 }
 
 
+// ---------------------------------------------------------------------------
+// One-pass forward+backward, second half: once a row's lse and coef exist, the stored
+// e = 2^(z log2e - ref) of a chunk become g = c_t (1[v = y_t] - e 2^(ref - lse_t log2e)), in place.
+// Streaming: 4 bytes per logit.  The work runs either as a kernel of its own or on four extra
+// warps of the next chunk's logits contraction, whose tensor-bound CTAs leave HBM nearly idle.
+// ---------------------------------------------------------------------------
+
+// One warp, 4 rows x 64 columns per step (lane -> row r = first_row + lane/8, 16-byte piece lane%8):
+// every warp-wide access is four whole 128-byte row pieces and the four references the warp needs
+// share a sector.  Rows without gradient are zero-filled without being read.
+template <int UNROLL>
+__device__ __forceinline__ void e_to_g_rows(const E2gJob& j, int64_t first_row, int g_begin, int g_end, int lane) {
+  const int64_t r = first_row + (lane >> 3);
+  if (r >= j.rows) return;
+  const int piece = lane & 7;
+  const float c = j.grad_loss * j.coef[j.row0 + r];
+  const float lse2 = j.lse[j.row0 + r] * kLog2e;
+  const int32_t yt = j.y[j.row0 + r];
+  uint4* grow = reinterpret_cast<uint4*>(j.G + r * j.ldg) + piece;      // + 8 per 64-column group
+  const float* rrow = j.ref + r;
+  if (c == 0.0f) {
+    for (int g = g_begin; g < g_end; ++g) grow[(int64_t)g * 8] = make_uint4(0u, 0u, 0u, 0u);
+    return;
+  }
+  const float nc = -c;
+  for (int g0 = g_begin; g0 < g_end; g0 += UNROLL) {
+    uint4 v[UNROLL];
+    float sc[UNROLL];
+#pragma unroll
+    for (int i = 0; i < UNROLL; ++i) {
+      if (g0 + i < g_end) {
+        v[i] = grow[(int64_t)(g0 + i) * 8];
+        sc[i] = rrow[(int64_t)(g0 + i) * j.ref_ld];
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < UNROLL; ++i) {
+      if (g0 + i < g_end) {
+        const float scale = nc * fast_exp2(sc[i] - lse2);
+        const int col0 = (g0 + i) * 64 + piece * 8;
+        uint32_t w[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
+        float f[8];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          f[2 * q] = __uint_as_float(w[q] << 16) * scale;
+          f[2 * q + 1] = __uint_as_float(w[q] & 0xFFFF0000u) * scale;
+        }
+        if (yt >= col0 && yt < col0 + 8) {
+          const int jj = yt - col0;
+#pragma unroll
+          for (int q = 0; q < 8; ++q) if (q == jj) f[q] += c;
+        }
+        grow[(int64_t)(g0 + i) * 8] = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]),
+                                                 pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
+      }
+    }
+  }
+}
+
+constexpr int kE2gThreads = 256;
+constexpr int kE2gRows = 32;            // rows per block: 8 warps x 4 rows
+constexpr int kE2gUnroll = 4;
+
+__global__ void __launch_bounds__(kE2gThreads)
+e_to_g_kernel(const E2gJob job, int groups_per_block) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int g_begin = blockIdx.y * groups_per_block;
+  e_to_g_rows<kE2gUnroll>(job, (int64_t)blockIdx.x * kE2gRows + warp * 4, g_begin,
+                          min(g_begin + groups_per_block, job.n_groups), lane);
+}
+
 struct Unit { int m_tile, n_begin, n_end; };
 __device__ __forceinline__ Unit unit_of(int u, const GemmParams& p) {
   Unit r;
@@ -327,8 +414,13 @@ __device__ __forceinline__ Unit unit_of(int u, const GemmParams& p) {
 // ---------------------------------------------------------------------------
 // the kernel
 // ---------------------------------------------------------------------------
-template <int MODE>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+// SIDE (E only): two more warps per CTA stream the previous chunk's e -> g while this chunk's
+// logits are contracted.
+constexpr int SIDE_WARPS = 2;
+constexpr int kSideUnroll = 16;
+
+template <int MODE, bool SIDE = false>
+__global__ void __launch_bounds__(NUM_THREADS + (SIDE ? 32 * SIDE_WARPS : 0), 1)
 spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmParams p) {
   constexpr bool A_MN = (MODE == MODE_DW);
   constexpr bool B_MN = (MODE == MODE_DH || MODE == MODE_DW);
@@ -464,7 +556,7 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         }
       }
     }
-  } else {
+  } else if (warp < 2 + EPI_WARPS) {
     // ------------------------------------------------------------------ epilogue (warps 2..9)
     const int quarter = warp & 3;                            // tensor-memory lanes this warp may read
     const int half = (warp - 2) >> 2;                        // which 256-column half of the tile
@@ -681,6 +773,12 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         p.partials[(int64_t)((u % p.nsplit) * 2 + half) * p.T + (grow - p.part_row0)] = part;
       }
     }
+  } else if (SIDE) {
+    // ------------------------------------------------------------------ side warps: e -> g of the previous chunk
+    // Plain loads and stores on memory no other role of this launch touches; no waits.
+    const int sw = warp - (2 + EPI_WARPS);
+    for (int64_t rb = (int64_t)blockIdx.x * SIDE_WARPS + sw; rb * 4 < p.side.rows; rb += (int64_t)gridDim.x * SIDE_WARPS)
+      e_to_g_rows<kSideUnroll>(p.side, rb * 4, 0, p.side.n_groups, lane);
   }
 
   // ------------------------------------------------------------------ teardown
@@ -693,69 +791,6 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   cluster_sync_all();                       // the peer may still be reading this CTA's shared / tensor memory
   if (warp == 0)
     asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
-}
-
-// One-pass forward+backward, second half: once a row's lse and coef exist, turn the stored
-// e = 2^(z log2e - ref) of the chunk into g = c_t (1[v = y_t] - e 2^(ref - lse_t log2e)), in place.
-// A block covers 32 rows x 64 columns per step (lane -> row lane/8, 16-byte piece lane%8), so every
-// warp-wide access is four whole 128-byte row pieces and the four references a warp needs share a
-// sector.  Rows without gradient are zero-filled without being read.  Streaming: 4 bytes per logit.
-constexpr int kE2gThreads = 256;
-constexpr int kE2gRows = 32;
-constexpr int kE2gUnroll = 4;
-
-__global__ void __launch_bounds__(kE2gThreads)
-e_to_g_kernel(__nv_bfloat16* __restrict__ G, int64_t ldg, const float* __restrict__ ref, int64_t ref_ld,
-              int64_t rows, int n_groups, int groups_per_block, const int32_t* __restrict__ y,
-              const float* __restrict__ lse, const float* __restrict__ coef, float grad_loss, int64_t row0) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int64_t r = (int64_t)blockIdx.x * kE2gRows + warp * 4 + (lane >> 3);
-  if (r >= rows) return;
-  const int piece = lane & 7;
-  const float c = grad_loss * coef[row0 + r];
-  const float lse2 = lse[row0 + r] * kLog2e;
-  const int32_t yt = y[row0 + r];
-  uint4* grow = reinterpret_cast<uint4*>(G + r * ldg) + piece;       // + 8 per 64-column group
-  const float* rrow = ref + r;
-  const int g_begin = blockIdx.y * groups_per_block;
-  const int g_end = min(g_begin + groups_per_block, n_groups);
-  if (c == 0.0f) {
-    for (int g = g_begin; g < g_end; ++g) grow[(int64_t)g * 8] = make_uint4(0u, 0u, 0u, 0u);
-    return;
-  }
-  const float nc = -c;
-  for (int g0 = g_begin; g0 < g_end; g0 += kE2gUnroll) {
-    uint4 v[kE2gUnroll];
-    float sc[kE2gUnroll];
-#pragma unroll
-    for (int i = 0; i < kE2gUnroll; ++i) {
-      if (g0 + i < g_end) {
-        v[i] = grow[(int64_t)(g0 + i) * 8];
-        sc[i] = rrow[(int64_t)(g0 + i) * ref_ld];
-      }
-    }
-#pragma unroll
-    for (int i = 0; i < kE2gUnroll; ++i) {
-      if (g0 + i < g_end) {
-        const float scale = nc * fast_exp2(sc[i] - lse2);
-        const int col0 = (g0 + i) * 64 + piece * 8;
-        uint32_t w[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
-        float f[8];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          f[2 * q] = __uint_as_float(w[q] << 16) * scale;
-          f[2 * q + 1] = __uint_as_float(w[q] & 0xFFFF0000u) * scale;
-        }
-        if (yt >= col0 && yt < col0 + 8) {
-          const int jj = yt - col0;
-#pragma unroll
-          for (int j = 0; j < 8; ++j) if (j == jj) f[j] += c;
-        }
-        grow[(int64_t)(g0 + i) * 8] = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]),
-                                                 pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
-      }
-    }
-  }
 }
 
 // A wait that nothing ever satisfies, through the same bounded-wait routine the pipeline uses:
@@ -814,21 +849,22 @@ constexpr int kLockStepWindow = 1;
 // CTA pairs that can be resident at once (one CTA per SM).
 int group_count() { return sm_count() / CG; }
 
-template <int MODE>
+template <int MODE, bool SIDE = false>
 cudaError_t launch_gemm(const CUtensorMap& a, const CUtensorMap& b, const GemmParams& p_in, uint32_t* progress,
                         cudaStream_t st) {
+  constexpr int kThreads = NUM_THREADS + (SIDE ? 32 * SIDE_WARPS : 0);
   static int max_groups[64] = {};            // CTA pairs that can be resident together, per device (0 = not yet asked)
   int dev = 0;
   cudaGetDevice(&dev);
   if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
   if (max_groups[dev] == 0) {
-    cudaError_t e = cudaFuncSetAttribute(spo_gemm_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    cudaError_t e = cudaFuncSetAttribute(spo_gemm_kernel<MODE, SIDE>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (e != cudaSuccess) return e;
     // The kernel is persistent and its pairs pace one another, so the grid must not exceed what the
     // device can hold at one time.
     cudaLaunchConfig_t q = {};
     q.gridDim = dim3(group_count() * CG, 1, 1);
-    q.blockDim = dim3(NUM_THREADS, 1, 1);
+    q.blockDim = dim3(kThreads, 1, 1);
     q.dynamicSmemBytes = SMEM_BYTES;
     cudaLaunchAttribute qa[1];
     qa[0].id = cudaLaunchAttributeClusterDimension;
@@ -838,7 +874,7 @@ cudaError_t launch_gemm(const CUtensorMap& a, const CUtensorMap& b, const GemmPa
     q.attrs = qa;
     q.numAttrs = 1;
     int n = 0;
-    e = cudaOccupancyMaxActiveClusters(&n, spo_gemm_kernel<MODE>, &q);
+    e = cudaOccupancyMaxActiveClusters(&n, spo_gemm_kernel<MODE, SIDE>, &q);
     if (e != cudaSuccess) return e;
     if (n < 1) return cudaErrorLaunchOutOfResources;
     max_groups[dev] = n < group_count() ? n : group_count();
@@ -857,7 +893,7 @@ cudaError_t launch_gemm(const CUtensorMap& a, const CUtensorMap& b, const GemmPa
   const int groups = units < max_groups[dev] ? units : max_groups[dev];
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(groups * CG, 1, 1);
-  cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+  cfg.blockDim = dim3(kThreads, 1, 1);
   cfg.dynamicSmemBytes = SMEM_BYTES;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
@@ -867,7 +903,7 @@ cudaError_t launch_gemm(const CUtensorMap& a, const CUtensorMap& b, const GemmPa
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, spo_gemm_kernel<MODE>, a, b, p);
+  return cudaLaunchKernelEx(&cfg, spo_gemm_kernel<MODE, SIDE>, a, b, p);
 }
 
 // Operand box heights (rows per TMA box) for K-major operands.
@@ -1053,6 +1089,9 @@ cudaError_t launch_bwd_bf16(const void* H, const void* W, const int32_t* y, cons
 // One-pass forward+backward.  Per chunk of token rows: E contraction (forward statistics + stored
 // exponentials) -> per-token finalisation (lse, logp, coef, loss terms) -> e -> g in place ->
 // dH, dW.  Three contractions per token instead of the four of forward-then-backward.
+// The chunks are software-pipelined over two chunk buffers: the e -> g pass of chunk c (HBM-bound)
+// rides on side warps of chunk c+1's E launch (tensor-bound), so only the last chunk pays for it:
+//   E(0) fin(0) | E(1)+e2g(0) fin(1) DH(0) DW(0) | E(2)+e2g(1) fin(2) DH(1) DW(1) | ... | e2g(n-1) DH(n-1) DW(n-1)
 // ---------------------------------------------------------------------------
 FusedWs fused_ws_layout(int64_t T, int32_t d, int32_t V, int32_t S) {
   FusedWs L{};
@@ -1061,6 +1100,7 @@ FusedWs fused_ws_layout(int64_t T, int32_t d, int32_t V, int32_t S) {
   L.ldg = b.ldg;
   const int n_tiles_v = (int)ceil_div(V, BN);
   const int64_t t_eff = T > 0 ? T : 1;
+  L.n_buf = t_eff > L.chunk_rows ? 2 : 1;
   // partials: the full chunk and the (shorter) last chunk may pick different split counts
   const int64_t full_rows = t_eff < L.chunk_rows ? ceil_div(t_eff, GROUP_M) * GROUP_M : L.chunk_rows;
   size_t part_elems = (size_t)2 * pick_fwd_split(full_rows / GROUP_M, n_tiles_v, d) * (size_t)full_rows;
@@ -1071,9 +1111,11 @@ FusedWs fused_ws_layout(int64_t T, int32_t d, int32_t V, int32_t S) {
     if (e2 > part_elems) part_elems = e2;
   }
   L.fin_blocks = ceil_div(t_eff, kFinalizeThreads);
+  L.g_bytes = align_up((size_t)L.chunk_rows * (size_t)L.ldg * 2, 256);
+  L.ref_bytes = align_up(sizeof(float) * (size_t)(L.ldg / 64) * (size_t)L.chunk_rows, 256);
   size_t off = 0;
-  L.g = off;          off = align_up(off + (size_t)L.chunk_rows * (size_t)L.ldg * 2, 256);
-  L.ref = off;        off = align_up(off + sizeof(float) * (size_t)(L.ldg / 64) * (size_t)L.chunk_rows, 256);
+  L.g = off;          off += L.g_bytes * (size_t)L.n_buf;
+  L.ref = off;        off += L.ref_bytes * (size_t)L.n_buf;
   L.partials = off;   off = align_up(off + sizeof(FwdPartial) * part_elems, 256);
   L.progress = off;   off = align_up(off + kProgressBytes, 256);
   L.block_sums = off; off = align_up(off + sizeof(double) * (size_t)L.fin_blocks, 256);
@@ -1084,8 +1126,6 @@ FusedWs fused_ws_layout(int64_t T, int32_t d, int32_t V, int32_t S) {
 }
 
 cudaError_t launch_fused_bf16(const FusedArgs& a, char* ws, const FusedWs& L, cudaStream_t st) {
-  __nv_bfloat16* G = reinterpret_cast<__nv_bfloat16*>(ws + L.g);
-  float* ref = reinterpret_cast<float*>(ws + L.ref);
   FwdPartial* partials = reinterpret_cast<FwdPartial*>(ws + L.partials);
   uint32_t* progress = reinterpret_cast<uint32_t*>(ws + L.progress);
   double* block_sums = reinterpret_cast<double*>(ws + L.block_sums);
@@ -1109,16 +1149,37 @@ cudaError_t launch_fused_bf16(const FusedArgs& a, char* ws, const FusedWs& L, cu
       !make_map(&mW_mn, a.W, d, V, d, 64) || !make_map(&mH_mn, a.H, d, T, d, 64))
     return cudaErrorInvalidValue;
   const int n_tiles_v = (int)ceil_div(V, BN);
-  const int n_groups = (int)(L.ldg / 64);
-  int chunk = 0;
-  for (int64_t t0 = 0; t0 < T; t0 += L.chunk_rows, ++chunk) {
-    const int64_t rows = (T - t0) < L.chunk_rows ? (T - t0) : L.chunk_rows;
+  const int n_chunks = (int)ceil_div(T, L.chunk_rows);
+
+  auto chunk_rows_of = [&](int c) {
+    const int64_t t0 = (int64_t)c * L.chunk_rows;
+    return (T - t0) < L.chunk_rows ? (T - t0) : L.chunk_rows;
+  };
+  auto g_of = [&](int c) { return reinterpret_cast<__nv_bfloat16*>(ws + L.g + L.g_bytes * (size_t)(c % L.n_buf)); };
+  auto ref_of = [&](int c) { return reinterpret_cast<float*>(ws + L.ref + L.ref_bytes * (size_t)(c % L.n_buf)); };
+  auto e2g_job = [&](int c) {
+    E2gJob j{};
+    j.G = g_of(c); j.ldg = L.ldg; j.ref = ref_of(c); j.ref_ld = L.chunk_rows;
+    j.rows = chunk_rows_of(c); j.n_groups = (int)(L.ldg / 64);
+    j.y = a.y; j.lse = a.lse; j.coef = a.coef; j.grad_loss = a.grad_loss; j.row0 = (int64_t)c * L.chunk_rows;
+    return j;
+  };
+  // dH rows of chunk c = G W, then dW (+)= G^T H_chunk
+  auto dh_dw = [&](int c) -> cudaError_t {
+    const int64_t t0 = (int64_t)c * L.chunk_rows, rows = chunk_rows_of(c);
+    CUtensorMap mG_k, mG_mn;
+    if (!make_map(&mG_k, g_of(c), V, rows, L.ldg, kBoxA) || !make_map(&mG_mn, g_of(c), V, rows, L.ldg, 64))
+      return cudaErrorInvalidValue;
+    return launch_chunk_dh_dw(mG_k, mG_mn, mW_mn, mH_mn, t0, rows, T, d, V, a.dH, a.dH_dtype, a.dW,
+                              (a.accumulate || c > 0) ? 1 : 0, progress, a.d_status, st);
+  };
+
+  for (int c = 0; c < n_chunks; ++c) {
+    const int64_t t0 = (int64_t)c * L.chunk_rows, rows = chunk_rows_of(c);
     const int m_tiles = (int)ceil_div(rows, GROUP_M);
     const int64_t rows_pad = (int64_t)m_tiles * GROUP_M;
-    CUtensorMap mG_k, mG_mn;
-    if (!make_map(&mG_k, G, V, rows, L.ldg, kBoxA) || !make_map(&mG_mn, G, V, rows, L.ldg, 64))
-      return cudaErrorInvalidValue;
-    // 1) logits of the chunk: online (max, sum, target logit) per row and split, e into the chunk buffer
+    // 1) logits of chunk c: online (max, sum, target logit) per row and split, e into the chunk buffer;
+    //    its side warps turn chunk c-1's e into g
     const int nsplit = pick_fwd_split(m_tiles, n_tiles_v, d);
     {
       GemmParams p{};
@@ -1135,43 +1196,49 @@ cudaError_t launch_fused_bf16(const FusedArgs& a, char* ws, const FusedWs& L, cu
       p.partials = partials;
       p.T = rows_pad;
       p.part_row0 = t0;
-      p.G = G; p.ldg = L.ldg;
-      p.ref = ref; p.ref_ld = L.chunk_rows;
+      p.G = g_of(c); p.ldg = L.ldg;
+      p.ref = ref_of(c); p.ref_ld = L.chunk_rows;
       p.d_status = a.d_status;
-      if ((e = launch_gemm<MODE_E>(mH_k, mW_k, p, progress, st)) != cudaSuccess) return e;
+      if (c > 0) {
+        p.side = e2g_job(c - 1);
+        e = launch_gemm<MODE_E, true>(mH_k, mW_k, p, progress, st);
+      } else {
+        e = launch_gemm<MODE_E, false>(mH_k, mW_k, p, progress, st);
+      }
+      if (e != cudaSuccess) return e;
     }
-    // 2) lse, logp, ratio, clipped surrogate and coef of the chunk's rows; loss terms per block
+    // 2) lse, logp, ratio, clipped surrogate and coef of chunk c's rows; loss terms per block
     {
       FinalizeRange rg;
       rg.t_begin = t0;
       rg.part_ld = rows_pad;
       rg.block0 = (int)(t0 / kFinalizeThreads);
       rg.total_blocks = (int)L.fin_blocks;
-      rg.last = (t0 + rows >= T) ? 1 : 0;
+      rg.last = (c == n_chunks - 1) ? 1 : 0;
       e = launch_fwd_finalize(partials, 2 * nsplit, a.y, a.logp_old, a.mask, a.cu_seqlens, a.a_norm, t0 + rows, V,
                               a.S, pr.clip_lo, pr.clip_hi, a.loss, a.logp, a.lse, a.coef, a.seq_sums, block_sums,
                               counters, seq_cnt, pr.agg_mode, pr.global_tokens, pr.global_responses, L.fin_blocks,
                               a.d_status, st, &rg);
       if (e != cudaSuccess) return e;
     }
-    // 3) e -> g in place
-    {
-      const int64_t row_blocks = ceil_div(rows, kE2gRows);
-      int col_blocks = (int)ceil_div((int64_t)sm_count() * 16, row_blocks);     // enough blocks to fill the device
-      if (col_blocks < 1) col_blocks = 1;
-      if (col_blocks > n_groups) col_blocks = n_groups;
-      int per = (int)ceil_div(n_groups, col_blocks);
-      per = (int)ceil_div(per, kE2gUnroll) * kE2gUnroll;
-      col_blocks = (int)ceil_div(n_groups, per);
-      dim3 grid((unsigned)row_blocks, (unsigned)col_blocks, 1);
-      e_to_g_kernel<<<grid, kE2gThreads, 0, st>>>(G, L.ldg, ref, L.chunk_rows, rows, n_groups, per, a.y, a.lse, a.coef,
-                                                  a.grad_loss, t0);
-      if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    }
-    // 4) dH rows of the chunk = G W;  5) dW (+)= G^T H_chunk
-    if ((e = launch_chunk_dh_dw(mG_k, mG_mn, mW_mn, mH_mn, t0, rows, T, d, V, a.dH, a.dH_dtype, a.dW,
-                                (a.accumulate || chunk > 0) ? 1 : 0, progress, a.d_status, st)) != cudaSuccess)
-      return e;
+    // 3) the two output contractions of chunk c-1, whose g is complete now
+    if (c > 0 && (e = dh_dw(c - 1)) != cudaSuccess) return e;
+  }
+  // last chunk: e -> g as a kernel of its own, then its output contractions
+  {
+    const int c = n_chunks - 1;
+    const E2gJob job = e2g_job(c);
+    const int64_t row_blocks = ceil_div(job.rows, kE2gRows);
+    int col_blocks = (int)ceil_div((int64_t)sm_count() * 16, row_blocks);       // enough blocks to fill the device
+    if (col_blocks < 1) col_blocks = 1;
+    if (col_blocks > job.n_groups) col_blocks = job.n_groups;
+    int per = (int)ceil_div(job.n_groups, col_blocks);
+    per = (int)ceil_div(per, kE2gUnroll) * kE2gUnroll;
+    col_blocks = (int)ceil_div(job.n_groups, per);
+    dim3 grid((unsigned)row_blocks, (unsigned)col_blocks, 1);
+    e_to_g_kernel<<<grid, kE2gThreads, 0, st>>>(job, per);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    if ((e = dh_dw(c)) != cudaSuccess) return e;
   }
   return cudaSuccess;
 }
