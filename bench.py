@@ -126,7 +126,7 @@ class Step:
         self.data = data
         self.T, self.d, self.V, self.S = data["T"], d, V, data["S"]
         self.mask_frac = float(mask_frac)
-        self.onepass = (path == "onepass") and not self.mask_frac > 0.0
+        self.onepass = path == "onepass"
         if self.mask_frac > 0.0:
             # contiguous masked spans inside the responses, the way tool output sits inside a
             # tool-integrated-reasoning response: spans of 32..256 tokens until the share is reached
@@ -158,14 +158,18 @@ class Step:
         self.ws_sample = torch.empty(B.spo_workspace_bytes(B.WS_SAMPLE, N=self.table_n, M=2 * self.S), **u8)
         self.ws_adv = torch.empty(B.spo_workspace_bytes(B.WS_ADVANTAGES, B=self.S), **u8)
         self.ws_bwd_bytes = B.spo_workspace_bytes(B.WS_LOSS_BWD, T=self.T, d=d, V=V)
-        if self.onepass:
+        if self.mask_frac > 0.0:        # row lists: unmasked rows (one-pass) or rows with gradient (split backward)
+            self.rows = torch.empty(self.T, dtype=torch.int32, device=device)
+            self.n_active = torch.zeros(4, dtype=torch.int32, device=device)
+            self.ws_rows = torch.empty(B.spo_workspace_bytes(B.WS_ACTIVE_ROWS, T=self.T), **u8)
+        if self.onepass and self.mask_frac > 0.0:
+            self.ws_loss = torch.empty(B.spo_workspace_bytes(B.WS_LOSS_FWD_BWD_ROWS, T=self.n_tok, d=d, V=V, B=self.S),
+                                       **u8)
+        elif self.onepass:
             self.ws_loss = torch.empty(B.spo_workspace_bytes(B.WS_LOSS_FWD_BWD, T=self.T, d=d, V=V, B=self.S), **u8)
         else:
             self.ws_fwd = torch.empty(B.spo_workspace_bytes(B.WS_LOSS_FWD, T=self.T, d=d, V=V, B=self.S), **u8)
             if self.mask_frac > 0.0:    # backward over the rows with gradient only
-                self.rows = torch.empty(self.T, dtype=torch.int32, device=device)
-                self.n_active = torch.zeros(4, dtype=torch.int32, device=device)
-                self.ws_rows = torch.empty(B.spo_workspace_bytes(B.WS_ACTIVE_ROWS, T=self.T), **u8)
                 self.ws_bwd = torch.empty(B.spo_workspace_bytes(B.WS_LOSS_BWD_ROWS, T=self.n_tok, d=d, V=V), **u8)
             else:
                 self.ws_bwd = torch.empty(self.ws_bwd_bytes, **u8)
@@ -176,9 +180,19 @@ class Step:
         # one-pass path: count 1, per chunk 4 (logits contraction [+ e->g of the chunk before on side warps],
         # finalise, dH, dW), and one e->g kernel for the last chunk.  Memsets are not counted.
         self.flops_fwd = 2.0 * self.T * d * V
-        if self.onepass:
+        chunks_act = -(-self.n_tok // chunk_rows)          # chunks of the compacted batch (masked workloads)
+        if self.onepass and self.mask_frac > 0.0:
+            # row list 3, gather 1, boundaries 1, one-pass on the compacted batch, two scatters
+            self.launches = 3 + 1 + 1 + 3 + 1 + 1 + (1 + 4 * chunks_act + 1) + 2
+            self.flops_fwd = 2.0 * self.n_tok * d * V
+            self.flops_bwd = 4.0 * self.n_tok * d * V
+        elif self.onepass:
             self.launches = 3 + 1 + 1 + 1 + 4 * self.bwd_chunks + 1
             self.flops_bwd = 4.0 * self.T * d * V
+        elif self.mask_frac > 0.0:
+            # forward over all rows; row list 3, gather 1, backward on the rows with gradient, scatter 1
+            self.launches = 3 + 1 + 1 + 3 + 3 + 1 + 3 * chunks_act + 1
+            self.flops_bwd = 6.0 * self.n_tok * d * V
         else:
             self.launches = 3 + 1 + 1 + 3 + 3 * self.bwd_chunks
             self.flops_bwd = 6.0 * self.T * d * V
@@ -211,6 +225,16 @@ class Step:
 
     def loss_onepass(self, h=None, y=None, logp_old=None, mask=None, cu=None):
         D = self.data
+        if self.mask_frac > 0.0:        # the unmasked rows only
+            B = self.B
+            B.spo_loss_mask_rows(D["mask"] if mask is None else mask, self.rows, self.n_active, self.ws_rows)
+            n_act = int(self.n_active[0].item())          # the one host read-back of this path
+            B.spo_loss_fwd_bwd_rows(D["h"] if h is None else h, D["w"], D["y"] if y is None else y,
+                                    D["logp_old"] if logp_old is None else logp_old,
+                                    D["cu_seqlens"] if cu is None else cu, self.a_norm, self.rows, n_act, 1.0,
+                                    self.loss, self.logp, self.lse, self.coef, None, self.dH, self.dW, 0, self.ws_loss,
+                                    self.params, self.status)
+            return
         self.B.spo_loss_fwd_bwd(D["h"] if h is None else h, D["w"], D["y"] if y is None else y,
                                 D["logp_old"] if logp_old is None else logp_old, D["mask"] if mask is None else mask,
                                 D["cu_seqlens"] if cu is None else cu, self.a_norm, 1.0, self.loss, self.logp,
@@ -536,8 +560,9 @@ def main():
     ap.add_argument("--custom", type=lambda v: tuple(int(x) for x in v.split(",")), default=None,
                     help="T,d,V: time the loss path on another LM-head shape (eight equal responses)")
     ap.add_argument("--mask-frac", type=float, default=0.0,
-                    help="mask this share of the tokens in contiguous spans and run the backward over the "
-                         "rows with gradient only (spo_loss_bwd_rows)")
+                    help="mask this share of the tokens in contiguous spans and run the loss over the unmasked rows "
+                         "only (spo_loss_fwd_bwd_rows; with --path split: the backward over the rows with gradient, "
+                         "spo_loss_bwd_rows)")
     ap.add_argument("--path", default="onepass", choices=["onepass", "split"],
                     help="loss as one spo_loss_fwd_bwd call (default) or as spo_loss_fwd + spo_loss_bwd")
     ap.add_argument("--responses", type=int, default=None,

@@ -65,6 +65,7 @@ extern "C" {
 #define SPO_WS_ACTIVE_ROWS    5
 #define SPO_WS_LOSS_BWD_ROWS  6
 #define SPO_WS_LOSS_FWD_BWD   7
+#define SPO_WS_LOSS_FWD_BWD_ROWS 8
 
 /*
  * Hyper-parameters.  Defaults (spo_default_params) are the values the paper prints:
@@ -339,6 +340,39 @@ int32_t spo_loss_bwd_rows(const void* H, const void* W, int32_t dtype, const int
                           int64_t T, int32_t d, int32_t V, const int32_t* rows, int64_t T_act,
                           void* dH, int32_t dH_dtype, float* dW, int32_t dW_accumulate,
                           void* ws, size_t ws_bytes, const spo_params* params, int32_t* d_status, void* stream);
+
+/*
+ * One-pass loss over the unmasked rows only.  In tool-integrated reasoning the tokens a tool wrote
+ * sit inside the response but carry no loss (mask = 0): they enter neither the objective of Sec. 3.2
+ * nor its gradients, so none of the three contractions has to see them and the cost of the call
+ * falls in proportion to the masked share.  Two calls, because the number of unmasked rows has to
+ * reach the host to size the second one (the library itself never synchronises):
+ *
+ *   spo_loss_mask_rows: rows[0..count) = ascending indices t with mask[t] != 0, *d_count = count.
+ *     mask    device in [T] uint8;  rows  device out [T] int32;  d_count  device out [1] int32
+ *     ws      device scratch, spo_workspace_bytes(SPO_WS_ACTIVE_ROWS, T, ...) bytes
+ *   (the caller reads *d_count back, e.g. after a stream synchronise)
+ *   spo_loss_fwd_bwd_rows: what spo_loss_fwd_bwd(H, W, ..., mask, ...) gives for loss, seq_sums,
+ *     dW, and for logp / lse / coef / dH at the listed rows; at all other rows logp, lse, coef and
+ *     dH are ZERO (spo_loss_fwd_bwd reports logp and lse of masked rows too; use it if you need them).
+ *     The listed rows of H, y and logp_old are gathered into a packed batch of T_act rows whose
+ *     sequence boundaries are the counts of listed rows per response, and the one-pass path runs on
+ *     that batch.  bf16 H / W only.  Every listed row counts as unmasked.
+ *     rows    device in [T_act] from the first call;  T_act  host value of *d_count
+ *     ws      device scratch, spo_workspace_bytes(SPO_WS_LOSS_FWD_BWD_ROWS, T_act, d, V, 0, S, 0) bytes
+ *             (holds the gathered rows of H and dH besides the one-pass scratch)
+ */
+int32_t spo_loss_mask_rows(const uint8_t* mask, int64_t T, int32_t* rows, int32_t* d_count,
+                           void* ws, size_t ws_bytes, void* stream);
+int32_t spo_loss_fwd_bwd_rows(const void* H, const void* W, int32_t dtype,
+                              const int32_t* y, const float* logp_old,
+                              const int32_t* cu_seqlens, const float* a_norm,
+                              int64_t T, int32_t d, int32_t V, int32_t S,
+                              const int32_t* rows, int64_t T_act, float grad_loss,
+                              float* loss, float* logp, float* lse, float* coef, float* seq_sums,
+                              void* dH, int32_t dH_dtype, float* dW, int32_t dW_accumulate,
+                              void* ws, size_t ws_bytes,
+                              const spo_params* params, int32_t* d_status, void* stream);
 
 /* Scratch size in bytes for one call of the selected entry point (host only, no CUDA call
  * except a device-property query).  Arguments that the selected call does not use are ignored. */

@@ -21,13 +21,13 @@ ERR_UNSUPPORTED_DTYPE, ERR_UNSUPPORTED_ARCH, ERR_WORKSPACE_TOO_SMALL, ERR_CUDA =
 DEV_ID_OUT_OF_RANGE, DEV_NONFINITE, DEV_UNIFORMS_EXHAUSTED, DEV_TIMEOUT, DEV_ZERO_TOTAL_WEIGHT = 1, 2, 4, 8, 16
 DTYPE_F32, DTYPE_BF16 = 0, 1
 (WS_SAMPLE, WS_ADVANTAGES, WS_LOSS_FWD, WS_LOSS_BWD, WS_UPDATE_REPEATS, WS_ACTIVE_ROWS, WS_LOSS_BWD_ROWS,
- WS_LOSS_FWD_BWD) = range(8)
+ WS_LOSS_FWD_BWD, WS_LOSS_FWD_BWD_ROWS) = range(9)
 AGG_TOKEN_MEAN, AGG_SEQ_MEAN = 0, 1
 
 EXPORTS = [
     "spo_default_params", "spo_tracker_init", "spo_sample_prompts", "spo_advantages",
     "spo_advantages_static", "spo_advantages_apply",
-    "spo_tracker_update", "spo_tracker_update_repeats", "spo_loss_fwd", "spo_loss_bwd", "spo_loss_fwd_bwd", "spo_loss_active_rows", "spo_loss_bwd_rows", "spo_workspace_bytes",
+    "spo_tracker_update", "spo_tracker_update_repeats", "spo_loss_fwd", "spo_loss_bwd", "spo_loss_fwd_bwd", "spo_loss_mask_rows", "spo_loss_fwd_bwd_rows", "spo_loss_active_rows", "spo_loss_bwd_rows", "spo_workspace_bytes",
     "spo_status_string", "spo_last_cuda_error", "spo_version", "spo_selftest_bounded_wait",
 ]
 
@@ -87,6 +87,12 @@ def lib():
                                        c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                                        c_void_p, c_int32, c_void_p, c_int32,
                                        c_void_p, c_size_t, P, c_void_p, c_void_p]
+        L.spo_loss_mask_rows.argtypes = [c_void_p, c_int64, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
+        L.spo_loss_fwd_bwd_rows.argtypes = [c_void_p, c_void_p, c_int32, c_void_p, c_void_p, c_void_p, c_void_p,
+                                            c_int64, c_int32, c_int32, c_int32, c_void_p, c_int64, c_float,
+                                            c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
+                                            c_void_p, c_int32, c_void_p, c_int32,
+                                            c_void_p, c_size_t, P, c_void_p, c_void_p]
         L.spo_loss_active_rows.argtypes = [c_void_p, c_int64, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
         L.spo_loss_bwd_rows.argtypes = [c_void_p, c_void_p, c_int32, c_void_p, c_void_p, c_void_p, c_float,
                                         c_int64, c_int32, c_int32, c_void_p, c_int64, c_void_p, c_int32, c_void_p,
@@ -217,6 +223,24 @@ def spo_loss_fwd_bwd(H, W, y, logp_old, mask, cu_seqlens, a_norm, grad_loss, los
                                   _ptr(logp), _ptr(lse), _ptr(coef), _ptr(seq_sums), _ptr(dH), _dtype_code(dH),
                                   _ptr(dW), int(dW_accumulate), _ptr(ws), ws.numel() * ws.element_size(),
                                   ctypes.byref(params), _ptr(d_status), _stream()), "spo_loss_fwd_bwd")
+
+
+def spo_loss_mask_rows(mask, rows, d_count, ws):
+    _check(lib().spo_loss_mask_rows(_ptr(mask), mask.numel(), _ptr(rows), _ptr(d_count), _ptr(ws),
+                                    ws.numel() * ws.element_size(), _stream()), "spo_loss_mask_rows")
+
+
+def spo_loss_fwd_bwd_rows(H, W, y, logp_old, cu_seqlens, a_norm, rows, n_listed, grad_loss, loss, logp, lse, coef,
+                          seq_sums, dH, dW, dW_accumulate, ws, params, d_status):
+    T, d = H.shape
+    V = W.shape[0]
+    S = cu_seqlens.numel() - 1
+    _check(lib().spo_loss_fwd_bwd_rows(_ptr(H), _ptr(W), _dtype_code(W), _ptr(y), _ptr(logp_old), _ptr(cu_seqlens),
+                                       _ptr(a_norm), T, d, V, S, _ptr(rows), int(n_listed), c_float(grad_loss),
+                                       _ptr(loss), _ptr(logp), _ptr(lse), _ptr(coef), _ptr(seq_sums), _ptr(dH),
+                                       _dtype_code(dH), _ptr(dW), int(dW_accumulate), _ptr(ws),
+                                       ws.numel() * ws.element_size(), ctypes.byref(params), _ptr(d_status),
+                                       _stream()), "spo_loss_fwd_bwd_rows")
 
 
 def spo_selftest_bounded_wait(limit_us, reached_end, d_status):

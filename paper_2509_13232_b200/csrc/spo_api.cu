@@ -330,7 +330,7 @@ int32_t spo_loss_active_rows(const float* coef, int64_t T, int32_t* rows, int32_
     return e0 == cudaSuccess ? SPO_OK : cuda_fail(e0);
   }
   if (ws_bytes < active_rows_ws_bytes(T)) return SPO_ERR_WORKSPACE_TOO_SMALL;
-  cudaError_t e = launch_active_rows(coef, T, rows, d_count, (int32_t*)ws, st);
+  cudaError_t e = launch_active_rows(coef, nullptr, T, rows, d_count, (int32_t*)ws, st);
   return e == cudaSuccess ? SPO_OK : cuda_fail(e);
 }
 
@@ -371,6 +371,104 @@ int32_t spo_loss_bwd_rows(const void* H, const void* W, int32_t dtype, const int
   return SPO_OK;
 }
 
+int32_t spo_loss_mask_rows(const uint8_t* mask, int64_t T, int32_t* rows, int32_t* d_count, void* ws, size_t ws_bytes,
+                           void* stream) {
+  if (T < 0 || !d_count || (T > 0 && (!mask || !rows || !ws))) return SPO_ERR_INVALID_ARG;
+  if (T >= ((int64_t)1 << 31) - 256) return SPO_ERR_BAD_SHAPE;
+  if (!aligned16(mask) || !aligned16(rows) || !aligned16(ws)) return SPO_ERR_BAD_ALIGNMENT;
+  if (!device_is_sm100()) return SPO_ERR_UNSUPPORTED_ARCH;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (T == 0) {
+    cudaError_t e0 = cudaMemsetAsync(d_count, 0, sizeof(int32_t), st);
+    return e0 == cudaSuccess ? SPO_OK : cuda_fail(e0);
+  }
+  if (ws_bytes < active_rows_ws_bytes(T)) return SPO_ERR_WORKSPACE_TOO_SMALL;
+  cudaError_t e = launch_active_rows(nullptr, mask, T, rows, d_count, (int32_t*)ws, st);
+  return e == cudaSuccess ? SPO_OK : cuda_fail(e);
+}
+
+namespace {
+struct FusedRowsWs {
+  size_t fused, h_act, dh_act, y_act, lo_act, logp_act, lse_act, coef_act, cu_act, total;
+  FusedWs inner;
+};
+FusedRowsWs fused_rows_ws_layout(int64_t T_act, int32_t d, int32_t V, int32_t S, int32_t dh_elem) {
+  FusedRowsWs L{};
+  const int64_t n = T_act > 0 ? T_act : 1;
+  L.inner = fused_ws_layout(T_act, d, V, S);
+  size_t off = 0;
+  L.fused = off;    off = align_up(off + L.inner.total, 256);
+  L.h_act = off;    off = align_up(off + (size_t)n * d * 2, 256);
+  L.dh_act = off;   off = align_up(off + (size_t)n * d * dh_elem, 256);
+  L.y_act = off;    off = align_up(off + (size_t)n * 4, 256);
+  L.lo_act = off;   off = align_up(off + (size_t)n * 4, 256);
+  L.logp_act = off; off = align_up(off + (size_t)n * 4, 256);
+  L.lse_act = off;  off = align_up(off + (size_t)n * 4, 256);
+  L.coef_act = off; off = align_up(off + (size_t)n * 4, 256);
+  L.cu_act = off;   off = align_up(off + (size_t)(S > 0 ? S + 1 : 2) * 4, 256);
+  L.total = off;
+  return L;
+}
+}  // namespace
+
+int32_t spo_loss_fwd_bwd_rows(const void* H, const void* W, int32_t dtype, const int32_t* y, const float* logp_old,
+                              const int32_t* cu_seqlens, const float* a_norm, int64_t T, int32_t d, int32_t V,
+                              int32_t S, const int32_t* rows, int64_t T_act, float grad_loss, float* loss, float* logp,
+                              float* lse, float* coef, float* seq_sums, void* dH, int32_t dH_dtype, float* dW,
+                              int32_t dW_accumulate, void* ws, size_t ws_bytes, const spo_params* params,
+                              int32_t* d_status, void* stream) {
+  int32_t rc = check_loss_shape(dtype, T, d, V);
+  if (rc != SPO_OK) return rc;
+  if (dtype != SPO_DTYPE_BF16) return SPO_ERR_UNSUPPORTED_DTYPE;
+  if (dH_dtype != SPO_DTYPE_F32 && dH_dtype != SPO_DTYPE_BF16) return SPO_ERR_UNSUPPORTED_DTYPE;
+  if (!params_ok(params) || !W || !loss || !dW || !ws || !cu_seqlens || S < 0 || T_act < 0 || T_act > T)
+    return SPO_ERR_INVALID_ARG;
+  if (T > 0 && (!H || !y || !logp_old || !a_norm || !logp || !lse || !coef || !dH || S < 1)) return SPO_ERR_INVALID_ARG;
+  if (T_act > 0 && !rows) return SPO_ERR_INVALID_ARG;
+  if (!aligned16(H) || !aligned16(W) || !aligned16(y) || !aligned16(logp_old) || !aligned16(cu_seqlens) ||
+      !aligned16(a_norm) || !aligned16(logp) || !aligned16(lse) || !aligned16(coef) || !aligned16(dH) ||
+      !aligned16(dW) || !aligned16(ws) || !aligned16(rows))
+    return SPO_ERR_BAD_ALIGNMENT;
+  if (!device_is_sm100()) return SPO_ERR_UNSUPPORTED_ARCH;
+  const int32_t dh_elem = dH_dtype == SPO_DTYPE_BF16 ? 2 : 4;
+  const FusedRowsWs L = fused_rows_ws_layout(T_act, d, V, S, dh_elem);
+  if (ws_bytes < L.total) return SPO_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t st = (cudaStream_t)stream;
+  char* w8 = (char*)ws;
+  cudaError_t e;
+  // rows that are not listed get zeros; the listed ones are overwritten by the scatters below
+  if (T > 0) {
+    if ((e = cudaMemsetAsync(dH, 0, (size_t)T * d * dh_elem, st)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaMemsetAsync(logp, 0, (size_t)T * 4, st)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaMemsetAsync(lse, 0, (size_t)T * 4, st)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaMemsetAsync(coef, 0, (size_t)T * 4, st)) != cudaSuccess) return cuda_fail(e);
+  }
+  void* h_act = w8 + L.h_act;
+  void* dh_act = w8 + L.dh_act;
+  int32_t* y_act = reinterpret_cast<int32_t*>(w8 + L.y_act);
+  float* lo_act = reinterpret_cast<float*>(w8 + L.lo_act);
+  float* logp_act = reinterpret_cast<float*>(w8 + L.logp_act);
+  float* lse_act = reinterpret_cast<float*>(w8 + L.lse_act);
+  float* coef_act = reinterpret_cast<float*>(w8 + L.coef_act);
+  int32_t* cu_act = reinterpret_cast<int32_t*>(w8 + L.cu_act);
+  // the compacted batch: listed rows of H, y, logp_old, and the sequence boundaries among them
+  if ((e = launch_gather_rows(H, y, logp_old, logp_old, rows, T_act, d * 2, h_act, y_act, lo_act, logp_act, st)) !=
+      cudaSuccess)
+    return cuda_fail(e);
+  if ((e = launch_compact_cu_seqlens(rows, T_act, cu_seqlens, S, cu_act, st)) != cudaSuccess) return cuda_fail(e);
+  FusedArgs a{};
+  a.H = h_act; a.W = W; a.y = y_act; a.logp_old = lo_act; a.mask = nullptr; a.cu_seqlens = cu_act; a.a_norm = a_norm;
+  a.T = T_act; a.d = d; a.V = V; a.S = S; a.grad_loss = grad_loss;
+  a.loss = loss; a.logp = logp_act; a.lse = lse_act; a.coef = coef_act; a.seq_sums = seq_sums;
+  a.dH = dh_act; a.dH_dtype = dH_dtype; a.dW = dW; a.accumulate = dW_accumulate;
+  a.params = params; a.d_status = d_status;
+  if ((e = launch_fused_bf16(a, w8 + L.fused, L.inner, st)) != cudaSuccess) return cuda_fail(e);
+  if ((e = launch_scatter_scalars(logp_act, lse_act, coef_act, rows, T_act, logp, lse, coef, st)) != cudaSuccess)
+    return cuda_fail(e);
+  if ((e = launch_scatter_rows(dh_act, rows, T_act, d * dh_elem, dH, st)) != cudaSuccess) return cuda_fail(e);
+  return SPO_OK;
+}
+
 size_t spo_workspace_bytes(int32_t which, int64_t T, int32_t d, int32_t V, int64_t N, int32_t B, int32_t M) {
   switch (which) {
     case SPO_WS_SAMPLE:
@@ -394,6 +492,9 @@ size_t spo_workspace_bytes(int32_t which, int64_t T, int32_t d, int32_t V, int64
     case SPO_WS_LOSS_BWD:
       if (T < 0 || V < 1 || d < 1) return 0;
       return bwd_ws_layout(T, d, V).total;
+    case SPO_WS_LOSS_FWD_BWD_ROWS:      /* T = number of listed rows, B = responses; sized for an fp32 dH */
+      if (T < 0 || V < 1 || d < 1 || (d % 64) != 0) return 0;
+      return fused_rows_ws_layout(T, d, V, B, 4).total;
     case SPO_WS_LOSS_FWD_BWD: {         /* enough for either element type */
       if (T < 0 || V < 1 || d < 1) return 0;
       const size_t f32 = fwd_ws_layout(T, d, V, SPO_DTYPE_F32, B).total;

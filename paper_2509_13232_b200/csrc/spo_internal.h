@@ -157,8 +157,14 @@ cudaError_t launch_bwd_bf16(const void* H, const void* W, const int32_t* y, cons
                             char* ws, const BwdWs& L, int32_t* d_status, cudaStream_t st);
 
 // row compaction for the backward
-cudaError_t launch_active_rows(const float* coef, int64_t T, int32_t* rows, int32_t* d_count, int32_t* block_cnt,
-                               cudaStream_t st);
+// rows listed: coef[t] != 0 (coef given) or mask[t] != 0 (mask given, coef NULL)
+cudaError_t launch_active_rows(const float* coef, const uint8_t* mask, int64_t T, int32_t* rows, int32_t* d_count,
+                               int32_t* block_cnt, cudaStream_t st);
+cudaError_t launch_compact_cu_seqlens(const int32_t* rows, int64_t n_act, const int32_t* cu_seqlens, int32_t S,
+                                      int32_t* cu_act, cudaStream_t st);
+cudaError_t launch_scatter_scalars(const float* logp_act, const float* lse_act, const float* coef_act,
+                                   const int32_t* rows, int64_t n_act, float* logp, float* lse, float* coef,
+                                   cudaStream_t st);
 size_t active_rows_ws_bytes(int64_t T);
 cudaError_t launch_gather_rows(const void* H, const int32_t* y, const float* lse, const float* coef,
                                const int32_t* rows, int64_t n_act, int32_t row_bytes, void* H_act, int32_t* y_act,

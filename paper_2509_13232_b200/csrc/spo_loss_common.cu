@@ -320,10 +320,16 @@ bwd_f32_kernel(const float* __restrict__ H, const float* __restrict__ W, const i
 // ---------------------------------------------------------------------------
 constexpr int kRowsPerBlock = 1024;
 
+// A row is listed when its coef is non-zero (coef given) or when its mask byte is non-zero (mask given).
+__device__ __forceinline__ int row_is_listed(const float* coef, const uint8_t* mask, int64_t t) {
+  return coef ? (coef[t] != 0.0f) : (mask[t] != 0);
+}
+
 __global__ void __launch_bounds__(1024)
-active_count_kernel(const float* __restrict__ coef, int64_t T, int32_t* __restrict__ block_cnt) {
+active_count_kernel(const float* __restrict__ coef, const uint8_t* __restrict__ mask, int64_t T,
+                    int32_t* __restrict__ block_cnt) {
   const int64_t t = (int64_t)blockIdx.x * kRowsPerBlock + threadIdx.x;
-  const int on = (t < T && coef[t] != 0.0f) ? 1 : 0;
+  const int on = (t < T && row_is_listed(coef, mask, t)) ? 1 : 0;
   const int total = __syncthreads_count(on);
   if (threadIdx.x == 0) block_cnt[blockIdx.x] = total;
 }
@@ -358,12 +364,12 @@ active_scan_kernel(int32_t* block_cnt, int64_t n_blocks, int32_t* __restrict__ d
 }
 
 __global__ void __launch_bounds__(1024)
-active_write_kernel(const float* __restrict__ coef, int64_t T, const int32_t* __restrict__ block_off,
-                    int32_t* __restrict__ rows) {
+active_write_kernel(const float* __restrict__ coef, const uint8_t* __restrict__ mask, int64_t T,
+                    const int32_t* __restrict__ block_off, int32_t* __restrict__ rows) {
   __shared__ int s_warp[32];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int64_t t = (int64_t)blockIdx.x * kRowsPerBlock + tid;
-  const int on = (t < T && coef[t] != 0.0f) ? 1 : 0;
+  const int on = (t < T && row_is_listed(coef, mask, t)) ? 1 : 0;
   const unsigned bal = __ballot_sync(0xffffffffu, on);
   if (lane == 0) s_warp[warp] = __popc(bal);
   __syncthreads();
@@ -394,6 +400,36 @@ scatter_rows_kernel(const uint4* __restrict__ dH_act, const int32_t* __restrict_
     const int64_t t = rows[i];
     for (int k = lane; k < row_vec; k += 32) dH[t * row_vec + k] = dH_act[i * row_vec + k];
   }
+}
+
+
+// Sequence boundaries of the compacted batch: cu_act[s] = number of listed rows below cu_seqlens[s]
+// (rows is ascending, so a lower bound).
+__global__ void __launch_bounds__(256)
+compact_cu_seqlens_kernel(const int32_t* __restrict__ rows, int64_t n_act, const int32_t* __restrict__ cu_seqlens,
+                          int32_t S, int32_t* __restrict__ cu_act) {
+  const int s = blockIdx.x * 256 + threadIdx.x;
+  if (s > S) return;
+  const int32_t bound = cu_seqlens[s];
+  int64_t lo = 0, hi = n_act;                 // first i with rows[i] >= bound
+  while (lo < hi) {
+    const int64_t mid = (lo + hi) >> 1;
+    if (rows[mid] < bound) lo = mid + 1; else hi = mid;
+  }
+  cu_act[s] = (int32_t)lo;
+}
+
+// logp / lse / coef of the compacted rows back to their places in the full arrays.
+__global__ void __launch_bounds__(256)
+scatter_scalars_kernel(const float* __restrict__ logp_act, const float* __restrict__ lse_act,
+                       const float* __restrict__ coef_act, const int32_t* __restrict__ rows, int64_t n_act,
+                       float* __restrict__ logp, float* __restrict__ lse, float* __restrict__ coef) {
+  const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
+  if (i >= n_act) return;
+  const int64_t t = rows[i];
+  logp[t] = logp_act[i];
+  lse[t] = lse_act[i];
+  coef[t] = coef_act[i];
 }
 
 }  // namespace
@@ -474,15 +510,15 @@ cudaError_t launch_bwd_f32(const float* H, const float* W, const int32_t* y, con
   return cudaGetLastError();
 }
 
-cudaError_t launch_active_rows(const float* coef, int64_t T, int32_t* rows, int32_t* d_count, int32_t* block_cnt,
-                               cudaStream_t st) {
+cudaError_t launch_active_rows(const float* coef, const uint8_t* mask, int64_t T, int32_t* rows, int32_t* d_count,
+                               int32_t* block_cnt, cudaStream_t st) {
   const int64_t n_blocks = ceil_div(T > 0 ? T : 1, kRowsPerBlock);
-  active_count_kernel<<<(unsigned)n_blocks, 1024, 0, st>>>(coef, T, block_cnt);
+  active_count_kernel<<<(unsigned)n_blocks, 1024, 0, st>>>(coef, mask, T, block_cnt);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   active_scan_kernel<<<1, 1024, 0, st>>>(block_cnt, n_blocks, d_count);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
-  active_write_kernel<<<(unsigned)n_blocks, 1024, 0, st>>>(coef, T, block_cnt, rows);
+  active_write_kernel<<<(unsigned)n_blocks, 1024, 0, st>>>(coef, mask, T, block_cnt, rows);
   return cudaGetLastError();
 }
 
@@ -500,6 +536,21 @@ cudaError_t launch_gather_rows(const void* H, const int32_t* y, const float* lse
   gather_rows_kernel<<<(unsigned)blocks, 256, 0, st>>>(reinterpret_cast<const uint4*>(H), y, lse, coef, rows, n_act,
                                                        row_bytes / 16, reinterpret_cast<uint4*>(H_act), y_act, lse_act,
                                                        coef_act);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_compact_cu_seqlens(const int32_t* rows, int64_t n_act, const int32_t* cu_seqlens, int32_t S,
+                                      int32_t* cu_act, cudaStream_t st) {
+  compact_cu_seqlens_kernel<<<(unsigned)ceil_div(S + 1, 256), 256, 0, st>>>(rows, n_act, cu_seqlens, S, cu_act);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_scatter_scalars(const float* logp_act, const float* lse_act, const float* coef_act,
+                                   const int32_t* rows, int64_t n_act, float* logp, float* lse, float* coef,
+                                   cudaStream_t st) {
+  if (n_act == 0) return cudaSuccess;
+  scatter_scalars_kernel<<<(unsigned)ceil_div(n_act, 256), 256, 0, st>>>(logp_act, lse_act, coef_act, rows, n_act, logp,
+                                                                        lse, coef);
   return cudaGetLastError();
 }
 

@@ -198,3 +198,72 @@ def test_real_vocab_and_hidden_small_token_count_full_oracle():
     assert rel_fro(got["dW"], want["dW"]) <= 1e-2
     assert np.abs(want["dW"][-64:]).max() > 0
     assert rel_fro(got["dW"][-64:], want["dW"][-64:]) <= 1e-2
+
+
+def _run_rows(lb, params, grad_loss, dh_f32):
+    """spo_loss_mask_rows + spo_loss_fwd_bwd_rows through the binding; numpy outputs."""
+    import torch
+    from paper_2509_13232_b200 import binding as B
+    from tests.helpers import dev, status_word, ws_bytes
+    H, W = dev(lb.h, torch.bfloat16), dev(lb.w, torch.bfloat16)
+    T, d = H.shape
+    V = W.shape[0]
+    S = len(lb.cu_seqlens) - 1
+    rows = torch.full((max(T, 1),), -1, dtype=torch.int32, device="cuda")
+    count = torch.zeros(4, dtype=torch.int32, device="cuda")
+    B.spo_loss_mask_rows(dev(lb.mask), rows, count, ws_bytes(B.WS_ACTIVE_ROWS, T=T))
+    torch.cuda.synchronize()
+    n = int(count[0].item())
+    f32 = dict(dtype=torch.float32, device="cuda")
+    loss = torch.zeros(4, **f32)
+    logp, lse, coef = (torch.full((max(T, 1),), float("nan"), **f32) for _ in range(3))
+    seq = torch.zeros((max(S, 1), 3), **f32)
+    dH = torch.full((max(T, 1), d), float("nan"), dtype=torch.float32 if dh_f32 else torch.bfloat16, device="cuda")
+    dW = torch.full((V, d), float("nan"), **f32)
+    st = status_word()
+    B.spo_loss_fwd_bwd_rows(H, W, dev(lb.y), dev(lb.logp_old), dev(lb.cu_seqlens), dev(lb.a_norm), rows, n, grad_loss,
+                            loss, logp, lse, coef, seq, dH[:T], dW, 0,
+                            ws_bytes(B.WS_LOSS_FWD_BWD_ROWS, T=n, d=d, V=V, B=S), params, st)
+    torch.cuda.synchronize()
+    return {"rows": rows[:n].cpu().numpy(), "loss": float(loss[0].item()), "logp": logp[:T].cpu().numpy(),
+            "lse": lse[:T].cpu().numpy(), "coef": coef[:T].cpu().numpy(), "seq_sums": seq[:S].cpu().numpy(),
+            "dH": dH[:T].float().cpu().numpy(), "dW": dW.cpu().numpy(), "status": int(st[0].item())}
+
+
+@pytest.mark.parametrize("agg,dh_f32", [(0, False), (1, True)])
+def test_unmasked_rows_only_matches_the_masked_oracle(agg, dh_f32):
+    """40 % of the tokens masked, one response masked entirely, an empty response, more listed rows
+    than one chunk: the compacted one-pass call gives the oracle's loss, sums and gradients."""
+    from paper_2509_13232_b200 import binding as B
+    lb = _clip_batch(140, [5000, 1300, 0, 700, 9000, 61, 4100], 128, 1500, True)
+    rng = np.random.default_rng(4)
+    lb.mask[:] = (rng.random(lb.mask.shape[0]) > 0.4).astype(np.uint8)
+    lb.mask[5000:6300] = 0
+    params = B.default_params(agg_mode=agg)
+    want = oracle_loss(lb, params=params, grad_loss=0.7)
+    got = _run_rows(lb, params, 0.7, dh_f32)
+    listed = np.nonzero(lb.mask)[0]
+    np.testing.assert_array_equal(got["rows"], listed)
+    assert got["status"] == 0 and len(listed) > 9472
+    assert abs(got["loss"] - want["loss"]) <= 2e-3
+    np.testing.assert_allclose(got["logp"][listed], want["logp"][listed], rtol=0, atol=2e-3)
+    np.testing.assert_allclose(got["lse"][listed], want["lse"][listed], rtol=0, atol=2e-3)
+    assert rel_fro(got["coef"], want["coef"]) <= 1e-2
+    scale = np.maximum(1.0, want["seq_sums"][:, 2:3])
+    np.testing.assert_allclose(got["seq_sums"] / scale, want["seq_sums"] / scale, rtol=0, atol=2e-3)
+    hidden = np.setdiff1d(np.arange(lb.mask.shape[0]), listed)
+    for k in ("logp", "lse", "coef"):
+        assert np.all(got[k][hidden] == 0.0)
+    assert np.all(got["dH"][hidden] == 0.0)
+    assert rel_fro(got["dH"], want["dH"]) <= 1e-2
+    assert rel_fro(got["dW"], want["dW"]) <= 1e-2
+
+
+def test_unmasked_rows_only_with_everything_masked():
+    from paper_2509_13232_b200 import binding as B
+    lb = inputs.loss_batch(141, [20, 13], 64, 200, 0.05, True, 0.1)
+    lb.mask[:] = 0
+    got = _run_rows(lb, B.default_params(), 1.0, False)
+    assert len(got["rows"]) == 0 and got["loss"] == 0.0 and got["status"] == 0
+    for k in ("logp", "lse", "coef", "dH", "dW", "seq_sums"):
+        assert np.all(got[k] == 0.0), k
