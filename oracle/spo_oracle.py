@@ -264,8 +264,13 @@ def aggregation_weights(mask01, seq, n_seq, agg_mode):
     raise ValueError("agg_mode")
 
 
+SUR_PPO_CLIP = 0        # the paper's objective: token-level PPO-Clip
+SUR_CISPO = 1           # clipped importance weight, held constant, times log-prob
+SUR_GSPO = 2            # PPO-Clip on one sequence-level ratio per response
+
+
 def loss_forward(h, w, y, logp_old, mask, cu_seqlens, a_norm,
-                 clip_lo=CLIP_LO, clip_hi=CLIP_HI, agg_mode=AGG_TOKEN_MEAN):
+                 clip_lo=CLIP_LO, clip_hi=CLIP_HI, agg_mode=AGG_TOKEN_MEAN, surrogate=SUR_PPO_CLIP):
     """Token-level PPO-Clip surrogate of Sec. 3.2 with Clip-Higher bounds.
 
     Per token t (row of ``h``): z = W h_t; lse = log sum_v exp(z_v);
@@ -273,6 +278,22 @@ def loss_forward(h, w, y, logp_old, mask, cu_seqlens, a_norm,
     s = min(ratio*a, clip(ratio, 1-clip_lo, 1+clip_hi)*a).
     The expectation over (s,t) is read as the mean over all unmasked tokens of
     the batch, n_tok = sum(mask); the exported loss is the negated objective.
+
+    Sec. 3.2 closes by naming two other objectives the advantage estimator is
+    compatible with, without writing them out; ``surrogate`` selects them in
+    the form their own publications give (this implementation's reading):
+      SUR_CISPO  the importance ratio is truncated to [1-clip_lo, 1+clip_hi] and
+                 enters as a constant weight (no gradient through it) on the
+                 log-prob: term_t = w_t * a * logp_t, w_t = clip(ratio_t);
+                 so d loss / d logp_t = -u_t * w_t * a for every unmasked token.
+      SUR_GSPO   one ratio per response, the geometric mean of its unmasked
+                 tokens' ratios: r_i = exp(mean_t (logp_t - logp_old_t));
+                 term_i = min(r_i*a_i, clip(r_i)*a_i); the objective is the mean
+                 of term_i over the responses that have an unmasked token
+                 (``agg_mode`` does not apply), and
+                 d loss / d logp_t = -(1/S_act) * a_i * r_i * [unclipped_i] / n_i.
+                 ``ratio``, ``surrogate`` and ``unclipped`` then hold each
+                 token's response-level value.
 
     Returns a dict: loss, logp[T], lse[T], ratio[T], surrogate[T], unclipped[T]
     (bool: the gradient passes through the ratio), coef[T] = d loss / d logp_t
@@ -294,24 +315,49 @@ def loss_forward(h, w, y, logp_old, mask, cu_seqlens, a_norm,
     ratio = np.exp(logp - logp_old)
     seq = token_sequence_ids(cu_seqlens, n_tok_rows)
     a = np.asarray(a_norm, dtype=np.float64)[seq]
-    clipped_ratio = np.minimum(np.maximum(ratio, 1.0 - clip_lo), 1.0 + clip_hi)
-    surrogate = np.minimum(ratio * a, clipped_ratio * a)
     n_tok = m.sum()
     n_seq = len(cu_seqlens) - 1
-    u = aggregation_weights(m, seq, n_seq, agg_mode)
-    loss = -(u * surrogate).sum()
-    # The min picks the unclipped branch (and so carries gradient) when the
-    # ratio is on the inside of the bound that matters for the sign of a;
-    # the boundary itself counts as inside.
-    unclipped = np.where(a >= 0.0, ratio <= 1.0 + clip_hi, ratio >= 1.0 - clip_lo)
-    coef = -(u * a * ratio * unclipped)
     seq_sums = np.zeros((n_seq, 3), dtype=np.float64)
     np.add.at(seq_sums[:, 0], seq, m * logp)
     np.add.at(seq_sums[:, 1], seq, m * (logp_old - logp))
     np.add.at(seq_sums[:, 2], seq, m)
+    lo_b, hi_b = 1.0 - clip_lo, 1.0 + clip_hi
+    if surrogate == SUR_GSPO:
+        n_i = seq_sums[:, 2]
+        live = n_i > 0
+        s_act = float(live.sum())
+        r_i = np.exp(-seq_sums[:, 1] / np.where(live, n_i, 1.0))          # exp(mean(logp - logp_old))
+        a_i = np.asarray(a_norm, dtype=np.float64)[:n_seq]
+        term_i = np.minimum(r_i * a_i, np.minimum(np.maximum(r_i, lo_b), hi_b) * a_i)
+        pass_i = np.where(a_i >= 0.0, r_i <= hi_b, r_i >= lo_b)
+        loss = -(term_i[live].sum() / s_act) if s_act > 0 else 0.0
+        ratio = r_i[seq]
+        surrogate_t = term_i[seq]
+        unclipped = pass_i[seq]
+        if s_act > 0:
+            coef = -(m * a * ratio * unclipped) / (s_act * np.where(n_i[seq] > 0, n_i[seq], 1.0))
+        else:
+            coef = np.zeros(n_tok_rows)
+    else:
+        u = aggregation_weights(m, seq, n_seq, agg_mode)
+        clipped_ratio = np.minimum(np.maximum(ratio, lo_b), hi_b)
+        if surrogate == SUR_CISPO:
+            surrogate_t = clipped_ratio * a * logp
+            unclipped = np.ones(n_tok_rows, dtype=bool)
+            coef = -(u * clipped_ratio * a)
+        elif surrogate == SUR_PPO_CLIP:
+            surrogate_t = np.minimum(ratio * a, clipped_ratio * a)
+            # The min picks the unclipped branch (and so carries gradient) when the
+            # ratio is on the inside of the bound that matters for the sign of a;
+            # the boundary itself counts as inside.
+            unclipped = np.where(a >= 0.0, ratio <= hi_b, ratio >= lo_b)
+            coef = -(u * a * ratio * unclipped)
+        else:
+            raise ValueError("surrogate")
+        loss = -(u * surrogate_t).sum()
     return {
         "loss": float(loss), "logp": logp, "lse": lse, "ratio": ratio,
-        "surrogate": surrogate, "unclipped": unclipped, "coef": coef,
+        "surrogate": surrogate_t, "unclipped": unclipped, "coef": coef,
         "n_tok": float(n_tok), "seq_sums": seq_sums,
     }
 

@@ -568,3 +568,131 @@ def test_repeated_ids_apply_in_batch_order():
     # every copy of a prompt sees the same pre-update baseline
     adv = O.raw_advantage(a0, b0, ids, r)
     assert adv[0] == 1.0 - 0.4 and adv[2] == 0.0 - 0.4 and adv[3] == 1.0 - 0.4
+
+
+# ------------------------------------------------------------------ the other objectives Sec. 3.2 names
+
+def _tiny_loss_case(seed, cu, t, d=5, v=9):
+    rng = np.random.default_rng(seed)
+    h, w = rng.standard_normal((t, d)), rng.standard_normal((v, d)) * 0.5
+    y = rng.integers(0, v, t)
+    return h, w, y
+
+
+def test_cispo_hand_values_and_agreement_with_ppo_clip_inside_the_bounds():
+    """Truncated importance weight held constant: coef = -u * clip(ratio) * a for every unmasked token.
+    Inside the clip bounds that is PPO-Clip's own gradient; outside, PPO-Clip gives zero on the
+    clipped side while this objective keeps the truncated weight."""
+    t, cu, a = 6, [0, 3, 6], np.array([2.0, -1.0])
+    h, w, y = _tiny_loss_case(31, cu, t)
+    mask = np.array([1, 1, 1, 1, 0, 1], dtype=np.uint8)
+    base = O.loss_forward(h, w, y, np.zeros(t), mask, cu, a)["logp"]
+    ratios = np.array([1.0, 1.5, 0.5, 1.1, 1.0, 0.6])
+    logp_old = base - np.log(ratios)
+    cis = O.loss_forward(h, w, y, logp_old, mask, cu, a, surrogate=O.SUR_CISPO)
+    ppo = O.loss_forward(h, w, y, logp_old, mask, cu, a)
+    np.testing.assert_allclose(cis["ratio"], ratios, rtol=1e-12)
+    # n_tok = 5; weights: 1, 1.28 (cut from 1.5), 0.8 (raised from 0.5), 1.1, -, 0.8 (raised from 0.6)
+    want = -np.array([1.0 * 2, 1.28 * 2, 0.8 * 2, 1.1 * -1, 0.0, 0.8 * -1]) / 5.0
+    np.testing.assert_allclose(cis["coef"], want, rtol=1e-12, atol=1e-15)
+    inside = (ratios >= 0.8) & (ratios <= 1.28)
+    np.testing.assert_allclose(cis["coef"][inside], ppo["coef"][inside], rtol=1e-12, atol=1e-15)
+    # token 1: a > 0 above the upper bound -> PPO-Clip stops the gradient, the truncated weight does not
+    assert ppo["coef"][1] == 0.0 and cis["coef"][1] != 0.0
+    # loss = -(1/n_tok) sum w a logp
+    wts = np.clip(ratios, 0.8, 1.28)
+    a_tok = np.repeat(a, 3)
+    assert abs(cis["loss"] + (mask * wts * a_tok * cis["logp"]).sum() / 5.0) < 1e-14
+
+
+def test_cispo_gradients_are_those_of_the_weighted_log_likelihood():
+    """With the weights frozen at their current values the objective is a weighted log-likelihood;
+    its central finite differences give dH and dW."""
+    t, cu, a = 7, [0, 2, 7], np.array([0.9, -1.1])
+    h, w, y = _tiny_loss_case(32, cu, t, d=6, v=11)
+    mask = np.array([1, 1, 1, 0, 1, 1, 1], dtype=np.uint8)
+    base = O.loss_forward(h, w, y, np.zeros(t), mask, cu, a)["logp"]
+    logp_old = base - np.log([1.1, 1.5, 0.7, 1.0, 1.2, 0.6, 0.9])
+    fwd = O.loss_forward(h, w, y, logp_old, mask, cu, a, surrogate=O.SUR_CISPO)
+    dh, dw = O.loss_backward(h, w, y, fwd["lse"], fwd["coef"], grad_loss=1.3)
+    frozen = np.clip(fwd["ratio"], 0.8, 1.28) * np.repeat(a, np.diff(cu)) * mask / mask.sum()
+
+    def frozen_loss(hh, ww):
+        lp = scipy.special.log_softmax(hh @ ww.T, axis=1)[np.arange(t), y]
+        return -1.3 * (frozen * lp).sum()
+
+    step = 1e-6
+    for arr, grad in ((h, dh), (w, dw)):
+        num = np.zeros_like(arr)
+        for idx in np.ndindex(arr.shape):
+            keep = arr[idx]
+            arr[idx] = keep + step
+            up = frozen_loss(h, w)
+            arr[idx] = keep - step
+            dn = frozen_loss(h, w)
+            arr[idx] = keep
+            num[idx] = (up - dn) / (2 * step)
+        assert np.linalg.norm(num - grad) <= 1e-6 * np.linalg.norm(grad)
+
+
+def test_gspo_reduces_to_ppo_clip_for_one_token_responses_and_hand_values():
+    """Responses of one token: the sequence-level ratio is the token's ratio, so the objective is the
+    sequence-mean PPO-Clip objective.  A response whose tokens all moved by the same log-ratio has
+    exactly that ratio."""
+    t = 5
+    cu, a = [0, 1, 2, 3, 4, 5], np.array([1.0, -0.5, 2.0, -1.5, 0.3])
+    h, w, y = _tiny_loss_case(33, cu, t)
+    base = O.loss_forward(h, w, y, np.zeros(t), None, cu, a)["logp"]
+    logp_old = base - np.log([1.0, 1.5, 0.5, 0.7, 1.4])
+    g = O.loss_forward(h, w, y, logp_old, None, cu, a, surrogate=O.SUR_GSPO)
+    p = O.loss_forward(h, w, y, logp_old, None, cu, a, agg_mode=O.AGG_SEQ_MEAN)
+    assert abs(g["loss"] - p["loss"]) < 1e-14
+    np.testing.assert_allclose(g["coef"], p["coef"], rtol=1e-12, atol=1e-16)
+    # one response of four tokens, every token's ratio e^0.1; a second, masked out entirely, drops out
+    t = 6
+    cu, a = [0, 4, 6], np.array([-2.0, 7.0])
+    h, w, y = _tiny_loss_case(34, cu, t)
+    mask = np.array([1, 1, 0, 1, 0, 0], dtype=np.uint8)
+    base = O.loss_forward(h, w, y, np.zeros(t), mask, cu, a)["logp"]
+    g = O.loss_forward(h, w, y, base - 0.1, mask, cu, a, surrogate=O.SUR_GSPO)
+    r = math.exp(0.1)
+    np.testing.assert_allclose(g["ratio"][:4], r, rtol=1e-12)
+    assert abs(g["loss"] - 2.0 * r) < 1e-12                     # -(min(r*-2, clip(r)*-2)) / 1 response
+    np.testing.assert_allclose(g["coef"], np.array([1, 1, 0, 1, 0, 0]) * 2.0 * r / 3.0, rtol=1e-12)
+    # geometric mean: ratios 2 and 1/2 on a two-token response give a sequence ratio of 1
+    cu, a = [0, 2], np.array([1.0])
+    h, w, y = _tiny_loss_case(35, cu, 2)
+    base = O.loss_forward(h, w, y, np.zeros(2), None, cu, a)["logp"]
+    g = O.loss_forward(h, w, y, base - np.log([2.0, 0.5]), None, cu, a, surrogate=O.SUR_GSPO)
+    np.testing.assert_allclose(g["ratio"], 1.0, rtol=1e-12)
+    assert abs(g["loss"] + 1.0) < 1e-12
+
+
+def test_gspo_gradients_against_central_finite_differences():
+    t, cu, a = 9, [0, 2, 2, 6, 9], np.array([0.9, 5.0, -1.1, 0.4])
+    h, w, y = _tiny_loss_case(36, cu, t, d=6, v=11)
+    mask = np.array([1, 1, 1, 0, 1, 1, 1, 1, 1], dtype=np.uint8)
+    base = O.loss_forward(h, w, y, np.zeros(t), mask, cu, a)["logp"]
+    # response 0: mean log-ratio above the upper bound with a > 0 (clipped); response 2: inside; 3: inside
+    logp_old = base - np.log([1.5, 1.4, 0.9, 1.0, 0.95, 0.85, 1.1, 1.2, 0.9])
+    fwd = O.loss_forward(h, w, y, logp_old, mask, cu, a, surrogate=O.SUR_GSPO)
+    per_seq_pass = [fwd["unclipped"][0], fwd["unclipped"][2], fwd["unclipped"][6]]
+    assert per_seq_pass == [False, True, True]
+    dh, dw = O.loss_backward(h, w, y, fwd["lse"], fwd["coef"], grad_loss=0.8)
+    assert np.all(dh[:2] == 0.0) and np.all(dh[3] == 0.0)
+
+    def loss_at(hh, ww):
+        return 0.8 * O.loss_forward(hh, ww, y, logp_old, mask, cu, a, surrogate=O.SUR_GSPO)["loss"]
+
+    step = 1e-6
+    for arr, grad in ((h, dh), (w, dw)):
+        num = np.zeros_like(arr)
+        for idx in np.ndindex(arr.shape):
+            keep = arr[idx]
+            arr[idx] = keep + step
+            up = loss_at(h, w)
+            arr[idx] = keep - step
+            dn = loss_at(h, w)
+            arr[idx] = keep
+            num[idx] = (up - dn) / (2 * step)
+        assert np.linalg.norm(num - grad) <= 1e-6 * np.linalg.norm(grad)
