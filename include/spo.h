@@ -56,6 +56,19 @@ extern "C" {
 #define SPO_AGG_TOKEN_MEAN  0
 #define SPO_AGG_SEQ_MEAN    1
 
+/* objective evaluated by the loss calls.  Sec. 3.2 defines the first and names the other two as
+ * compatible with the SPO advantage without writing them out; they follow their own publications:
+ *   PPO_CLIP  sum_t u_t min(ratio_t a, clip(ratio_t, 1-clip_lo, 1+clip_hi) a)          (the default)
+ *   CISPO     sum_t u_t w_t a logp_t with w_t = clip(ratio_t, 1-clip_lo, 1+clip_hi) held constant
+ *             (no gradient through the weight): coef_t = -u_t w_t a for every unmasked token
+ *   GSPO      one ratio per response, r_i = exp(mean over its unmasked tokens of logp_t - logp_old_t);
+ *             (1/S_act) sum_i min(r_i a_i, clip(r_i) a_i); coef_t = -a_i r_i [unclipped_i] / (S_act n_i);
+ *             agg_mode does not apply.  Needs every token of a response before any coef exists, so it
+ *             runs in the two-call path only (spo_loss_fwd, spo_loss_bwd) */
+#define SPO_SUR_PPO_CLIP  0
+#define SPO_SUR_CISPO     1
+#define SPO_SUR_GSPO      2
+
 /* selectors for spo_workspace_bytes */
 #define SPO_WS_SAMPLE      0
 #define SPO_WS_ADVANTAGES  1
@@ -88,6 +101,7 @@ typedef struct spo_params {
    * the objective are those of the whole mini-batch.  0 = use this call's own counts. */
   int32_t global_tokens;     /* unmasked tokens of the whole mini-batch (n_tok) */
   int32_t global_responses;  /* responses with an unmasked token in the whole mini-batch (S_act) */
+  int32_t surrogate;         /* SPO_SUR_*: which objective the loss calls evaluate */
 } spo_params;
 
 int32_t spo_default_params(spo_params* p /* host, out */);
@@ -232,6 +246,7 @@ int32_t spo_tracker_update_repeats(float* ab, int64_t N, const int32_t* ids, con
  *   those values (the whole data-parallel mini-batch) and `loss` is this rank's share: the ranks'
  *   losses and dW add up to the mini-batch's, dH rows are final;
  *   coef_t = d loss / d logp_t = -u_t * a * ratio * [gradient passes the clip].
+ *   params->surrogate selects one of the other objectives (SPO_SUR_*, above) instead.
  *
  *   H           device in  [T][d], row-major, dtype as given (bf16: d % 64 == 0)
  *   W           device in  [V][d], row-major, same dtype
@@ -291,7 +306,9 @@ int32_t spo_loss_bwd(const void* H, const void* W, int32_t dtype, const int32_t*
  * dH and dW carry it in place of spo_loss_bwd's own bf16 rounding of g (same size).
  * fp32: the two SIMT halves run back to back (nothing to share).
  *
- *   arguments   as in spo_loss_fwd and spo_loss_bwd; lse and coef are outputs here
+ *   arguments   as in spo_loss_fwd and spo_loss_bwd; lse and coef are outputs here.
+ *               SPO_SUR_GSPO with bf16 inputs returns SPO_ERR_INVALID_ARG (a response's ratio needs all
+ *               its tokens, which may lie in later chunks): use the two calls.
  *   ws          device scratch, spo_workspace_bytes(SPO_WS_LOSS_FWD_BWD, T, d, V, 0, S, 0) bytes:
  *               two chunk buffers when T exceeds one chunk (the chunks are software-pipelined: the
  *               e -> g pass of one chunk runs on spare warps of the next chunk's logits contraction),

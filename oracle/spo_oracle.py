@@ -7,15 +7,17 @@ product path (only from tests, the smoke check and the CPU-baseline leg of the
 benchmark).
 
 Everything is numpy float64 unless a function name ends in ``_f32``: those
-restate, in IEEE fp32 with one correctly rounded operation per step, the few
+restate, in IEEE fp32 as a fixed sequence of individually rounded operations, the few
 places where floating point decides an integer (the quantised sampling
 weights), so that both sides take that decision in the same precision.
 
 Pinned by tests/test_oracle_pins.py against closed forms, brute force, finite
 differences and the constants the paper prints.  Pieces whose parameters the
-paper never gives a value for (``d_half``; the whole-step composition, for
-which no worked example is printed) are "parity unpinned" by the paper itself
-and are pinned only through the identities listed in that test file.
+paper never gives a value or a formula for (``d_half``; the two objectives
+Sec. 3.2 only names, ``SUR_CISPO`` and ``SUR_GSPO``; the whole-step
+composition, for which no worked example is printed) are "parity unpinned" by
+the paper itself and are pinned only through the identities listed in that
+test file.
 
 Paper sections: Sec. 3.1 (KL-adaptive value tracker), Sec. 3.2 (advantage,
 global normalisation, PPO-Clip objective), Sec. 3.3 and Eq. "sampling_coef"

@@ -23,6 +23,7 @@ DTYPE_F32, DTYPE_BF16 = 0, 1
 (WS_SAMPLE, WS_ADVANTAGES, WS_LOSS_FWD, WS_LOSS_BWD, WS_UPDATE_REPEATS, WS_ACTIVE_ROWS, WS_LOSS_BWD_ROWS,
  WS_LOSS_FWD_BWD, WS_LOSS_FWD_BWD_ROWS) = range(9)
 AGG_TOKEN_MEAN, AGG_SEQ_MEAN = 0, 1
+SUR_PPO_CLIP, SUR_CISPO, SUR_GSPO = 0, 1, 2
 
 EXPORTS = [
     "spo_default_params", "spo_tracker_init", "spo_sample_prompts", "spo_advantages",
@@ -37,6 +38,7 @@ class SpoParams(Structure):
         ("rho_min", c_float), ("rho_max", c_float), ("d_half", c_float), ("eps_explore", c_float),
         ("clip_lo", c_float), ("clip_hi", c_float), ("norm_eps", c_float), ("norm_ddof", c_int32),
         ("agg_mode", c_int32), ("global_tokens", c_int32), ("global_responses", c_int32),
+        ("surrogate", c_int32),
     ]
 
 

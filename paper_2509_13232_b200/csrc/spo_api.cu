@@ -48,6 +48,8 @@ FwdWs fwd_ws_layout(int64_t T, int32_t d, int32_t V, int32_t dtype, int32_t S) {
   L.block_sums = off; off = align_up(off + sizeof(double) * (size_t)L.fin_blocks, 256);
   L.counters = off;   off = align_up(off + 4 * sizeof(int32_t), 256);
   L.seq_cnt = off;    off = align_up(off + sizeof(int32_t) * (size_t)(S > 0 ? S : 1), 256);
+  L.seq_coef = off;   off = align_up(off + sizeof(float) * (size_t)(S > 0 ? S : 1), 256);
+  L.seq_term = off;   off = align_up(off + sizeof(double) * (size_t)(S > 0 ? S : 1), 256);
   L.total = off;
   return L;
 }
@@ -69,7 +71,40 @@ static bool params_ok(const spo_params* p) {
   if (p->norm_ddof != 0 && p->norm_ddof != 1) return false;
   if (p->agg_mode != SPO_AGG_TOKEN_MEAN && p->agg_mode != SPO_AGG_SEQ_MEAN) return false;
   if (p->global_tokens < 0 || p->global_responses < 0) return false;
+  if (p->surrogate != SPO_SUR_PPO_CLIP && p->surrogate != SPO_SUR_CISPO && p->surrogate != SPO_SUR_GSPO) return false;
   return true;
+}
+
+}  // namespace spo
+
+namespace spo {
+
+// The launches of spo_loss_fwd: token count, logits contraction into per-split partials, per-token
+// finalisation, and for the sequence-level objective the pass that needs every token's logp first.
+static cudaError_t forward_launches(const void* H, const void* W, int32_t dtype, const int32_t* y,
+                                    const float* logp_old, const uint8_t* mask, const int32_t* cu_seqlens,
+                                    const float* a_norm, int64_t T, int32_t d, int32_t V, int32_t S, float* loss,
+                                    float* logp, float* lse, float* coef, float* seq_sums, char* w8, const FwdWs& L,
+                                    const spo_params* params, int32_t* d_status, cudaStream_t st) {
+  FwdPartial* partials = reinterpret_cast<FwdPartial*>(w8 + L.partials);
+  double* block_sums = reinterpret_cast<double*>(w8 + L.block_sums);
+  int32_t* counters = reinterpret_cast<int32_t*>(w8 + L.counters);
+  int32_t* seq_cnt = reinterpret_cast<int32_t*>(w8 + L.seq_cnt);
+  const bool seq_level = params->surrogate == SPO_SUR_GSPO;
+  cudaError_t e = launch_fwd_prepare(mask, T, cu_seqlens, S, params->agg_mode != 0 || seq_level, seq_cnt, counters, st);
+  if (e != cudaSuccess) return e;
+  if (dtype == SPO_DTYPE_BF16)
+    e = launch_fwd_bf16(H, W, y, T, d, V, partials, L.nsplit, reinterpret_cast<uint32_t*>(w8 + L.progress), d_status, st);
+  else
+    e = launch_fwd_f32((const float*)H, (const float*)W, y, T, d, V, partials, st);
+  if (e != cudaSuccess) return e;
+  e = launch_fwd_finalize(partials, L.nsplit, y, logp_old, mask, cu_seqlens, a_norm, T, V, S, params->clip_lo,
+                          params->clip_hi, loss, logp, lse, coef, seq_sums, block_sums, counters, seq_cnt, params->agg_mode,
+                          params->surrogate, params->global_tokens, params->global_responses, L.fin_blocks, d_status, st);
+  if (e != cudaSuccess || !seq_level) return e;
+  return launch_seq_level_objective(logp, logp_old, mask, cu_seqlens, a_norm, T, S, params->clip_lo, params->clip_hi,
+                                    counters, params->global_responses, reinterpret_cast<float*>(w8 + L.seq_coef),
+                                    reinterpret_cast<double*>(w8 + L.seq_term), coef, loss, st);
 }
 
 }  // namespace spo
@@ -91,6 +126,7 @@ int32_t spo_default_params(spo_params* p) {
   p->agg_mode = SPO_AGG_TOKEN_MEAN;
   p->global_tokens = 0;
   p->global_responses = 0;
+  p->surrogate = SPO_SUR_PPO_CLIP;
   return SPO_OK;
 }
 
@@ -200,23 +236,8 @@ int32_t spo_loss_fwd(const void* H, const void* W, int32_t dtype, const int32_t*
   if (!device_is_sm100()) return SPO_ERR_UNSUPPORTED_ARCH;
   const FwdWs L = fwd_ws_layout(T, d, V, dtype, S);
   if (ws_bytes < L.total) return SPO_ERR_WORKSPACE_TOO_SMALL;
-  cudaStream_t st = (cudaStream_t)stream;
-  char* w8 = (char*)ws;
-  FwdPartial* partials = reinterpret_cast<FwdPartial*>(w8 + L.partials);
-  double* block_sums = reinterpret_cast<double*>(w8 + L.block_sums);
-  int32_t* counters = reinterpret_cast<int32_t*>(w8 + L.counters);
-  int32_t* seq_cnt = reinterpret_cast<int32_t*>(w8 + L.seq_cnt);
-  cudaError_t e = launch_fwd_prepare(mask, T, cu_seqlens, S, params->agg_mode, seq_cnt, counters, st);
-  if (e != cudaSuccess) return cuda_fail(e);
-  if (dtype == SPO_DTYPE_BF16)
-    e = launch_fwd_bf16(H, W, y, T, d, V, partials, L.nsplit, reinterpret_cast<uint32_t*>(w8 + L.progress), d_status, st);
-  else
-    e = launch_fwd_f32((const float*)H, (const float*)W, y, T, d, V, partials, st);
-  if (e != cudaSuccess) return cuda_fail(e);
-  e = launch_fwd_finalize(partials, L.nsplit, y, logp_old, mask, cu_seqlens, a_norm, T, V, S, params->clip_lo,
-                          params->clip_hi, loss, logp, lse, coef, seq_sums, block_sums, counters, seq_cnt, params->agg_mode,
-                          params->global_tokens, params->global_responses, L.fin_blocks,
-                          d_status, st);
+  cudaError_t e = forward_launches(H, W, dtype, y, logp_old, mask, cu_seqlens, a_norm, T, d, V, S, loss, logp, lse, coef,
+                                   seq_sums, (char*)ws, L, params, d_status, (cudaStream_t)stream);
   return e == cudaSuccess ? SPO_OK : cuda_fail(e);
 }
 
@@ -267,6 +288,7 @@ int32_t spo_loss_fwd_bwd(const void* H, const void* W, int32_t dtype, const int3
   char* w8 = (char*)ws;
   cudaError_t e;
   if (dtype == SPO_DTYPE_BF16) {
+    if (params->surrogate == SPO_SUR_GSPO) return SPO_ERR_INVALID_ARG;     // needs whole responses: two-call path
     const FusedWs L = fused_ws_layout(T, d, V, S);
     if (ws_bytes < L.total) return SPO_ERR_WORKSPACE_TOO_SMALL;
     FusedArgs a{};
@@ -281,17 +303,9 @@ int32_t spo_loss_fwd_bwd(const void* H, const void* W, int32_t dtype, const int3
   // fp32 inputs: nothing to share between the two halves of the SIMT path; run them back to back
   const FwdWs L = fwd_ws_layout(T, d, V, dtype, S);
   if (ws_bytes < L.total) return SPO_ERR_WORKSPACE_TOO_SMALL;
-  FwdPartial* partials = reinterpret_cast<FwdPartial*>(w8 + L.partials);
-  double* block_sums = reinterpret_cast<double*>(w8 + L.block_sums);
-  int32_t* counters = reinterpret_cast<int32_t*>(w8 + L.counters);
-  int32_t* seq_cnt = reinterpret_cast<int32_t*>(w8 + L.seq_cnt);
-  if ((e = launch_fwd_prepare(mask, T, cu_seqlens, S, params->agg_mode, seq_cnt, counters, st)) != cudaSuccess)
+  if ((e = forward_launches(H, W, dtype, y, logp_old, mask, cu_seqlens, a_norm, T, d, V, S, loss, logp, lse, coef,
+                            seq_sums, w8, L, params, d_status, st)) != cudaSuccess)
     return cuda_fail(e);
-  if ((e = launch_fwd_f32((const float*)H, (const float*)W, y, T, d, V, partials, st)) != cudaSuccess) return cuda_fail(e);
-  e = launch_fwd_finalize(partials, L.nsplit, y, logp_old, mask, cu_seqlens, a_norm, T, V, S, params->clip_lo,
-                          params->clip_hi, loss, logp, lse, coef, seq_sums, block_sums, counters, seq_cnt,
-                          params->agg_mode, params->global_tokens, params->global_responses, L.fin_blocks, d_status, st);
-  if (e != cudaSuccess) return cuda_fail(e);
   e = launch_bwd_f32((const float*)H, (const float*)W, y, lse, coef, grad_loss, T, d, V, dH, dH_dtype, dW,
                      dW_accumulate, st);
   return e == cudaSuccess ? SPO_OK : cuda_fail(e);
@@ -423,6 +437,7 @@ int32_t spo_loss_fwd_bwd_rows(const void* H, const void* W, int32_t dtype, const
   if (dH_dtype != SPO_DTYPE_F32 && dH_dtype != SPO_DTYPE_BF16) return SPO_ERR_UNSUPPORTED_DTYPE;
   if (!params_ok(params) || !W || !loss || !dW || !ws || !cu_seqlens || S < 0 || T_act < 0 || T_act > T)
     return SPO_ERR_INVALID_ARG;
+  if (params->surrogate == SPO_SUR_GSPO) return SPO_ERR_INVALID_ARG;       // needs whole responses: two-call path
   if (T > 0 && (!H || !y || !logp_old || !a_norm || !logp || !lse || !coef || !dH || S < 1)) return SPO_ERR_INVALID_ARG;
   if (T_act > 0 && !rows) return SPO_ERR_INVALID_ARG;
   if (!aligned16(H) || !aligned16(W) || !aligned16(y) || !aligned16(logp_old) || !aligned16(cu_seqlens) ||

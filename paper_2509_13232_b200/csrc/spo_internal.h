@@ -72,6 +72,8 @@ struct FwdWs {
   size_t block_sums;    // double [finalize blocks]
   size_t counters;      // int32 [4]: n_tok, ticket, responses with an unmasked token
   size_t seq_cnt;       // int32 [S]: unmasked tokens per response (sequence-mean aggregation)
+  size_t seq_coef;      // float [S]: d loss / d logp of a response's unmasked tokens (sequence-level objective)
+  size_t seq_term;      // double [S]: objective term of each response (sequence-level objective)
   size_t total;
   int nsplit;
   int64_t fin_blocks;
@@ -87,15 +89,21 @@ struct FinalizeRange {
   int last;             // 1 when this launch covers the final rows (per-response sums are taken then)
 };
 
-cudaError_t launch_fwd_prepare(const uint8_t* mask, int64_t T, const int32_t* cu_seqlens, int32_t S, int agg_mode,
-                               int32_t* seq_cnt, int32_t* counters, cudaStream_t st);
+// need_seq_counts: per-response unmasked counts and the number of responses that have any
+cudaError_t launch_fwd_prepare(const uint8_t* mask, int64_t T, const int32_t* cu_seqlens, int32_t S,
+                               int need_seq_counts, int32_t* seq_cnt, int32_t* counters, cudaStream_t st);
+// Sequence-level objective: coef and loss from the finished logp of all tokens.
+cudaError_t launch_seq_level_objective(const float* logp, const float* logp_old, const uint8_t* mask,
+                                       const int32_t* cu_seqlens, const float* a_norm, int64_t T, int32_t S,
+                                       float clip_lo, float clip_hi, const int32_t* counters, int32_t global_responses,
+                                       float* seq_coef, double* seq_term, float* coef, float* loss, cudaStream_t st);
 cudaError_t launch_fwd_finalize(const FwdPartial* partials, int nsplit, const int32_t* y,
                                 const float* logp_old, const uint8_t* mask, const int32_t* cu_seqlens,
                                 const float* a_norm, int64_t T, int32_t V, int32_t S,
                                 float clip_lo, float clip_hi,
                                 float* loss, float* logp, float* lse, float* coef, float* seq_sums,
                                 double* block_sums, int32_t* counters, const int32_t* seq_cnt, int agg_mode,
-                                int32_t global_tokens, int32_t global_responses,
+                                int surrogate, int32_t global_tokens, int32_t global_responses,
                                 int64_t fin_blocks, int32_t* d_status, cudaStream_t st,
                                 const FinalizeRange* range = nullptr);
 

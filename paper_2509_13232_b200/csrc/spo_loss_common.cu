@@ -80,7 +80,7 @@ fwd_finalize_kernel(const FwdPartial* __restrict__ partials, int nsplit, const i
                     int64_t T, int32_t V, int32_t S, float clip_lo, float clip_hi,
                     float* __restrict__ loss, float* __restrict__ logp_out, float* __restrict__ lse_out,
                     float* __restrict__ coef_out, double* block_sums, int32_t* counters,
-                    const int32_t* __restrict__ seq_cnt, int agg_mode, int32_t global_tokens,
+                    const int32_t* __restrict__ seq_cnt, int agg_mode, int surrogate, int32_t global_tokens,
                     int32_t global_responses, int32_t* d_status, FinalizeRange rg) {
   // This launch covers token rows [rg.t_begin, T_end); its blocks are blocks rg.block0.. of the
   // rg.total_blocks that cover all rows (one launch, or one per chunk of the one-pass path).
@@ -119,17 +119,26 @@ fwd_finalize_kernel(const FwdPartial* __restrict__ partials, int nsplit, const i
       const float a = a_norm[lo];
       const bool on = mask ? mask[t] != 0 : true;
       const float hi_b = 1.0f + clip_hi, lo_b = 1.0f - clip_lo;
-      const float sur = fminf(ratio * a, fminf(fmaxf(ratio, lo_b), hi_b) * a);
-      const bool passes = a >= 0.0f ? ratio <= hi_b : ratio >= lo_b;
-      if (on && n_tok > 0) {
+      const float cut = fminf(fmaxf(ratio, lo_b), hi_b);
+      // per unit of token weight: the objective's term and d term / d logp
+      float sur, dsur;
+      if (surrogate == SPO_SUR_CISPO) {        // truncated weight, held constant, on the log-prob
+        sur = cut * a * lp;
+        dsur = cut * a;
+      } else {                                 // PPO-Clip (a sequence-level objective fills coef later)
+        sur = fminf(ratio * a, cut * a);
+        const bool passes = a >= 0.0f ? ratio <= hi_b : ratio >= lo_b;
+        dsur = passes ? a * ratio : 0.0f;
+      }
+      if (on && n_tok > 0 && surrogate != SPO_SUR_GSPO) {
         // weight of this token in the expectation: 1/n_tok, or 1/(responses * tokens of its response)
         if (agg_mode == 0) {
           contrib = (double)sur;
-          if (passes) coef = -a * ratio / (float)n_tok;
+          if (dsur != 0.0f) coef = -dsur / (float)n_tok;
         } else {
           const float u = 1.0f / ((float)s_act * (float)seq_cnt[lo]);
           contrib = (double)sur * (double)u;
-          if (passes) coef = -a * ratio * u;
+          if (dsur != 0.0f) coef = -dsur * u;
         }
       }
     }
@@ -165,7 +174,8 @@ fwd_finalize_kernel(const FwdPartial* __restrict__ partials, int nsplit, const i
       double tot = 0.0;
 #pragma unroll
       for (int w = 0; w < kFinalizeThreads / 32; ++w) tot += s_part[w];
-      if (n_tok <= 0) loss[0] = 0.0f;
+      if (surrogate == SPO_SUR_GSPO) { /* written by the sequence-level pass */ }
+      else if (n_tok <= 0) loss[0] = 0.0f;
       else loss[0] = agg_mode == 0 ? (float)(-tot / (double)n_tok) : (float)(-tot);
     }
   }
@@ -403,6 +413,80 @@ scatter_rows_kernel(const uint4* __restrict__ dH_act, const int32_t* __restrict_
 }
 
 
+// Sequence-level objective, one block per response: r = exp(mean over its unmasked tokens of
+// logp - logp_old), term = min(r a, clip(r) a), and the coef all its unmasked tokens share.
+__global__ void __launch_bounds__(256)
+seq_level_terms_kernel(const float* __restrict__ logp, const float* __restrict__ logp_old,
+                       const uint8_t* __restrict__ mask, const int32_t* __restrict__ cu_seqlens,
+                       const float* __restrict__ a_norm, float clip_lo, float clip_hi,
+                       const int32_t* __restrict__ counters, int32_t global_responses,
+                       float* __restrict__ seq_coef, double* __restrict__ seq_term) {
+  const int s = blockIdx.x;
+  const int64_t lo = cu_seqlens[s], hi = cu_seqlens[s + 1];
+  double sum = 0.0, cnt = 0.0;
+  for (int64_t t = lo + threadIdx.x; t < hi; t += 256) {
+    if (mask && mask[t] == 0) continue;
+    sum += (double)logp[t] - (double)logp_old[t];
+    cnt += 1.0;
+  }
+  __shared__ double s_a[8], s_c[8];
+  sum = warp_sum_f64(sum); cnt = warp_sum_f64(cnt);
+  if ((threadIdx.x & 31) == 0) { s_a[threadIdx.x >> 5] = sum; s_c[threadIdx.x >> 5] = cnt; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double ts = 0, tc = 0;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) { ts += s_a[w]; tc += s_c[w]; }
+    const int32_t s_act = global_responses > 0 ? global_responses : counters[2];
+    float c = 0.0f;
+    double term = 0.0;
+    if (tc > 0.0 && s_act > 0) {
+      const double r = exp(ts / tc);
+      const double a = (double)a_norm[s];
+      const double hi_b = 1.0 + (double)clip_hi, lo_b = 1.0 - (double)clip_lo;
+      term = fmin(r * a, fmin(fmax(r, lo_b), hi_b) * a);
+      const bool passes = a >= 0.0 ? r <= hi_b : r >= lo_b;
+      if (passes) c = (float)(-a * r / ((double)s_act * tc));
+    }
+    seq_coef[s] = c;
+    seq_term[s] = term;
+  }
+}
+
+// coef of every token from its response's value; block 0 also folds the responses' terms (index
+// order, fixed tree) into the loss.
+__global__ void __launch_bounds__(256)
+seq_level_apply_kernel(const uint8_t* __restrict__ mask, const int32_t* __restrict__ cu_seqlens, int64_t T, int32_t S,
+                       const float* __restrict__ seq_coef, const double* __restrict__ seq_term,
+                       const int32_t* __restrict__ counters, int32_t global_responses, float* __restrict__ coef,
+                       float* __restrict__ loss) {
+  const int64_t t = (int64_t)blockIdx.x * 256 + threadIdx.x;
+  if (t < T) {
+    int lo = 0, hi = S;
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if ((int64_t)cu_seqlens[mid] <= t) lo = mid; else hi = mid;
+    }
+    const bool on = mask ? mask[t] != 0 : true;
+    coef[t] = on ? seq_coef[lo] : 0.0f;
+  }
+  if (blockIdx.x == 0) {
+    __shared__ double s_part[8];
+    double acc = 0.0;
+    for (int i = threadIdx.x; i < S; i += 256) acc += seq_term[i];
+    acc = warp_sum_f64(acc);
+    if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = acc;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      double tot = 0.0;
+#pragma unroll
+      for (int w = 0; w < 8; ++w) tot += s_part[w];
+      const int32_t s_act = global_responses > 0 ? global_responses : counters[2];
+      loss[0] = s_act > 0 ? (float)(-tot / (double)s_act) : 0.0f;
+    }
+  }
+}
+
 // Sequence boundaries of the compacted batch: cu_act[s] = number of listed rows below cu_seqlens[s]
 // (rows is ascending, so a lower bound).
 __global__ void __launch_bounds__(256)
@@ -438,11 +522,11 @@ scatter_scalars_kernel(const float* __restrict__ logp_act, const float* __restri
 // host launchers
 // ---------------------------------------------------------------------------
 
-cudaError_t launch_fwd_prepare(const uint8_t* mask, int64_t T, const int32_t* cu_seqlens, int32_t S, int agg_mode,
-                               int32_t* seq_cnt, int32_t* counters, cudaStream_t st) {
+cudaError_t launch_fwd_prepare(const uint8_t* mask, int64_t T, const int32_t* cu_seqlens, int32_t S,
+                               int need_seq_counts, int32_t* seq_cnt, int32_t* counters, cudaStream_t st) {
   cudaError_t e = cudaMemsetAsync(counters, 0, 4 * sizeof(int32_t), st);
   if (e != cudaSuccess) return e;
-  if (agg_mode != 0 && S > 0 && T > 0) {
+  if (need_seq_counts && S > 0 && T > 0) {
     seq_count_kernel<<<S, 256, 0, st>>>(mask, cu_seqlens, seq_cnt, counters);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }
@@ -463,7 +547,7 @@ cudaError_t launch_fwd_finalize(const FwdPartial* partials, int nsplit, const in
                                 float clip_lo, float clip_hi,
                                 float* loss, float* logp, float* lse, float* coef, float* seq_sums,
                                 double* block_sums, int32_t* counters, const int32_t* seq_cnt, int agg_mode,
-                                int32_t global_tokens, int32_t global_responses,
+                                int surrogate, int32_t global_tokens, int32_t global_responses,
                                 int64_t fin_blocks, int32_t* d_status, cudaStream_t st,
                                 const FinalizeRange* range) {
   // Default: one launch over all rows.  With a range: rows [t_begin, T) of a larger batch whose
@@ -479,7 +563,8 @@ cudaError_t launch_fwd_finalize(const FwdPartial* partials, int nsplit, const in
   if (blocks == 0) return cudaSuccess;
   fwd_finalize_kernel<<<blocks, kFinalizeThreads, 0, st>>>(
       partials, nsplit, y, logp_old, mask, cu_seqlens, a_norm, T, V, S, clip_lo, clip_hi,
-      loss, logp, lse, coef, block_sums, counters, seq_cnt, agg_mode, global_tokens, global_responses, d_status, rg);
+      loss, logp, lse, coef, block_sums, counters, seq_cnt, agg_mode, surrogate, global_tokens, global_responses,
+      d_status, rg);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   if (seq_sums && S > 0 && rg.last) {
@@ -487,6 +572,21 @@ cudaError_t launch_fwd_finalize(const FwdPartial* partials, int nsplit, const in
     e = cudaGetLastError();
   }
   return e;
+}
+
+cudaError_t launch_seq_level_objective(const float* logp, const float* logp_old, const uint8_t* mask,
+                                       const int32_t* cu_seqlens, const float* a_norm, int64_t T, int32_t S,
+                                       float clip_lo, float clip_hi, const int32_t* counters, int32_t global_responses,
+                                       float* seq_coef, double* seq_term, float* coef, float* loss, cudaStream_t st) {
+  if (S > 0) {
+    seq_level_terms_kernel<<<S, 256, 0, st>>>(logp, logp_old, mask, cu_seqlens, a_norm, clip_lo, clip_hi, counters,
+                                              global_responses, seq_coef, seq_term);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+  }
+  seq_level_apply_kernel<<<(unsigned)ceil_div(T > 0 ? T : 1, 256), 256, 0, st>>>(
+      mask, cu_seqlens, T, S, seq_coef, seq_term, counters, global_responses, coef, loss);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_fwd_f32(const float* H, const float* W, const int32_t* y, int64_t T, int32_t d, int32_t V,

@@ -1134,12 +1134,13 @@ cudaError_t launch_fused_bf16(const FusedArgs& a, char* ws, const FusedWs& L, cu
   const spo_params& pr = *a.params;
   const int64_t T = a.T;
   const int32_t d = a.d, V = a.V;
-  cudaError_t e = launch_fwd_prepare(a.mask, T, a.cu_seqlens, a.S, pr.agg_mode, seq_cnt, counters, st);
+  cudaError_t e = launch_fwd_prepare(a.mask, T, a.cu_seqlens, a.S, pr.agg_mode != 0, seq_cnt, counters, st);
   if (e != cudaSuccess) return e;
   if (T == 0) {
     e = launch_fwd_finalize(partials, 0, a.y, a.logp_old, a.mask, a.cu_seqlens, a.a_norm, 0, V, a.S, pr.clip_lo,
                             pr.clip_hi, a.loss, a.logp, a.lse, a.coef, a.seq_sums, block_sums, counters, seq_cnt,
-                            pr.agg_mode, pr.global_tokens, pr.global_responses, L.fin_blocks, a.d_status, st);
+                            pr.agg_mode, pr.surrogate, pr.global_tokens, pr.global_responses, L.fin_blocks, a.d_status,
+                            st);
     if (e != cudaSuccess) return e;
     if (!a.accumulate) return cudaMemsetAsync(a.dW, 0, sizeof(float) * (size_t)V * d, st);
     return cudaSuccess;
@@ -1217,8 +1218,8 @@ cudaError_t launch_fused_bf16(const FusedArgs& a, char* ws, const FusedWs& L, cu
       rg.last = (c == n_chunks - 1) ? 1 : 0;
       e = launch_fwd_finalize(partials, 2 * nsplit, a.y, a.logp_old, a.mask, a.cu_seqlens, a.a_norm, t0 + rows, V,
                               a.S, pr.clip_lo, pr.clip_hi, a.loss, a.logp, a.lse, a.coef, a.seq_sums, block_sums,
-                              counters, seq_cnt, pr.agg_mode, pr.global_tokens, pr.global_responses, L.fin_blocks,
-                              a.d_status, st, &rg);
+                              counters, seq_cnt, pr.agg_mode, pr.surrogate, pr.global_tokens, pr.global_responses,
+                              L.fin_blocks, a.d_status, st, &rg);
       if (e != cudaSuccess) return e;
     }
     // 3) the two output contractions of chunk c-1, whose g is complete now

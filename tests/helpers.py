@@ -80,7 +80,8 @@ def oracle_loss(lb, params=None, grad_loss=1.0, mask_none=False):
     clip_hi = 0.28 if params is None else float(np.float32(params.clip_hi))
     mask = None if mask_none else lb.mask
     agg = 0 if params is None else int(params.agg_mode)
-    fwd = O.loss_forward(lb.h, lb.w, lb.y, lb.logp_old, mask, lb.cu_seqlens, lb.a_norm, clip_lo, clip_hi, agg)
+    sur = 0 if params is None else int(params.surrogate)
+    fwd = O.loss_forward(lb.h, lb.w, lb.y, lb.logp_old, mask, lb.cu_seqlens, lb.a_norm, clip_lo, clip_hi, agg, sur)
     dh, dw = O.loss_backward(lb.h, lb.w, lb.y, fwd["lse"], fwd["coef"], grad_loss)
     fwd["dH"], fwd["dW"] = dh, dw
     return fwd
