@@ -19,8 +19,9 @@ def _slice_batch(lb, s0, s1):
                             a_norm=lb.a_norm[s0:s1], bf16=lb.bf16)
 
 
+@pytest.mark.parametrize("one_pass", [False, True])
 @pytest.mark.parametrize("agg", [0, 1])
-def test_two_emulated_ranks_equal_the_whole_mini_batch(agg):
+def test_two_emulated_ranks_equal_the_whole_mini_batch(agg, one_pass):
     import torch
     from paper_2509_13232_b200 import binding as B
     rng = np.random.default_rng(77)
@@ -67,7 +68,7 @@ def test_two_emulated_ranks_equal_the_whole_mini_batch(agg):
         np.testing.assert_allclose(a_n.cpu().numpy(), a_norm[s0:s1], rtol=1e-5, atol=2e-6)
         part = _slice_batch(lb, s0, s1)
         part.a_norm = a_n.cpu().numpy()
-        got = run_loss(part, params=params)
+        got = run_loss(part, params=params, one_pass=one_pass)
         assert got["status"] == 0
         loss_sum += got["loss"]
         dws.append(got["dW"])
