@@ -345,3 +345,25 @@ def test_sampling_at_the_maximum_number_of_uniforms():
     assert st == 0
     np.testing.assert_array_equal(ids, want)
     assert len(set(ids.tolist())) == b
+
+
+def test_sampling_weights_every_branch_of_the_op_sequence_bit_equal():
+    """Common entries (Newton reciprocal square root), empty entries, a zero parameter, tiny and
+    huge magnitudes (the division / square-root branch): the weights equal the oracle's fp32
+    restatement bit for bit, and the draw made from them is the oracle's."""
+    rng = np.random.default_rng(41)
+    special = np.array([[0, 0], [0, 5], [5, 0], [1e-30, 1], [1, 1e-38], [1e-20, 1e-20], [1e25, 1e25],
+                        [3e5, 7e5], [2.0 ** -21, 2.0 ** -21], [1e-39, 1], [8, 8], [0.875, 7.125],
+                        [1e18, 3e18], [1e-19, 4e-19]], dtype=np.float32)
+    ab = np.concatenate([special, rng.uniform(0.0, 25.0, (3000, 2)).astype(np.float32),
+                         (10.0 ** rng.uniform(-12, 12, (3000, 2))).astype(np.float32)])
+    ab = ab[rng.permutation(len(ab))]
+    p = B().default_params()
+    u = inputs.uniforms_f32(rng, 600)
+    ids, w, st = gpu_sample(dev(ab), u, 300, p)
+    w_or = O.sampling_weights_f32(ab[:, 0], ab[:, 1], np.float32(p.eps_explore))
+    assert st == 0
+    np.testing.assert_array_equal(w.view(np.uint32), w_or.view(np.uint32))
+    np.testing.assert_array_equal(ids, O.sample_prompts(w_or, u, 300))
+    np.testing.assert_allclose(w, O.sampling_weights(ab[:, 0].astype(np.float64), ab[:, 1].astype(np.float64),
+                                                     float(np.float32(p.eps_explore))), rtol=1e-5)

@@ -198,6 +198,23 @@ def test_fp32_weights_track_the_fp64_definition():
     assert w32[0] == np.float32(0.55)
 
 
+def test_fp32_weights_uncommon_magnitudes_track_the_fp64_definition():
+    """Entries outside the range the Newton sequence serves (empty, a zero parameter, tiny, huge)
+    take the division / square-root branch; every branch stays within 1e-6 of the definition."""
+    a = np.array([0, 0, 5, 1e-30, 1, 1e-20, 1e25, 3e5, 2.0 ** -21, 1e-39, 1e18, 1e-19], dtype=np.float32)
+    b = np.array([0, 5, 0, 1, 1e-38, 1e-20, 1e25, 7e5, 2.0 ** -21, 1, 3e18, 4e-19], dtype=np.float32)
+    w32 = O.sampling_weights_f32(a, b)
+    want = O.sampling_weights(a.astype(np.float64), b.astype(np.float64))
+    assert np.all(np.isfinite(w32))
+    np.testing.assert_allclose(w32, want, rtol=1e-6)
+    assert w32[0] == np.float32(0.55) and w32[1] == np.float32(0.05) and w32[2] == np.float32(0.05)
+    rng = np.random.default_rng(8)
+    aa = (10.0 ** rng.uniform(-15, 15, 20000)).astype(np.float32)
+    bb = (10.0 ** rng.uniform(-15, 15, 20000)).astype(np.float32)
+    np.testing.assert_allclose(O.sampling_weights_f32(aa, bb),
+                               O.sampling_weights(aa.astype(np.float64), bb.astype(np.float64)), rtol=1e-6)
+
+
 def test_quantised_weights_are_exact_scalings():
     w = np.array([0.05, 0.55, 0.3, 2.0 ** -8], dtype=np.float32)
     q = O.quantise_weights(w)
