@@ -391,6 +391,21 @@ int32_t spo_loss_fwd_bwd_rows(const void* H, const void* W, int32_t dtype,
                               void* ws, size_t ws_bytes,
                               const spo_params* params, int32_t* d_status, void* stream);
 
+/*
+ * Diagnostics of one policy update over the unmasked tokens, from the forward's logp (no counterpart
+ * in the paper's equations; these are the quantities its training curves are read by, and none
+ * enters the objective).  out (device, [8] fp32):
+ *   [0] n_tok   [1] mean importance ratio   [2] share of tokens whose gradient the clip stops
+ *   (ratio beyond the bound that matters for the sign of their advantage; zero advantage: not stopped)
+ *   [3] mean of logp_old - logp (sampled estimate of KL(old || new))   [4] mean of ratio - 1 - log ratio
+ *   (a non-negative estimate of the same)   [5] largest ratio   [6] smallest ratio
+ *   [7] share of tokens whose ratio lies outside [1-clip_lo, 1+clip_hi].  All zeros when n_tok = 0.
+ * One block, fixed reduction order; a few tens of microseconds at 250 k tokens.
+ */
+int32_t spo_loss_stats(const float* logp, const float* logp_old, const uint8_t* mask,
+                       const int32_t* cu_seqlens, const float* a_norm, int64_t T, int32_t S,
+                       float* out, const spo_params* params, void* stream);
+
 /* Scratch size in bytes for one call of the selected entry point (host only, no CUDA call
  * except a device-property query).  Arguments that the selected call does not use are ignored. */
 size_t spo_workspace_bytes(int32_t which, int64_t T, int32_t d, int32_t V,

@@ -364,6 +364,43 @@ def loss_forward(h, w, y, logp_old, mask, cu_seqlens, a_norm,
     }
 
 
+def loss_stats(logp, logp_old, mask, cu_seqlens, a_norm, clip_lo=CLIP_LO, clip_hi=CLIP_HI):
+    """Per-step diagnostics of the policy update over the unmasked tokens (the quantities the
+    paper's training curves are read by; none enters the objective):
+      [0] n_tok            [1] mean importance ratio
+      [2] share of tokens whose gradient the clip stops (ratio beyond the bound that matters
+          for the sign of their advantage; a zero advantage counts as not clipped)
+      [3] mean of logp_old - logp            (the plain sampled estimate of KL(old || new))
+      [4] mean of ratio - 1 - log(ratio)     (a non-negative estimate of the same KL)
+      [5] largest ratio    [6] smallest ratio
+      [7] share of tokens whose ratio lies outside [1-clip_lo, 1+clip_hi], whatever the sign.
+    All zeros when no token is unmasked.
+    """
+    logp = np.asarray(logp, dtype=np.float64)
+    logp_old = np.asarray(logp_old, dtype=np.float64)
+    t = logp.shape[0]
+    m = np.ones(t, dtype=bool) if mask is None else (np.asarray(mask) != 0)
+    out = np.zeros(8, dtype=np.float64)
+    n = int(m.sum())
+    if n == 0:
+        return out
+    seq = token_sequence_ids(cu_seqlens, t)
+    a = np.asarray(a_norm, dtype=np.float64)[seq][m]
+    d = (logp - logp_old)[m]
+    ratio = np.exp(d)
+    lo_b, hi_b = 1.0 - clip_lo, 1.0 + clip_hi
+    stopped = np.where(a > 0.0, ratio > hi_b, np.where(a < 0.0, ratio < lo_b, False))
+    out[0] = n
+    out[1] = ratio.mean()
+    out[2] = stopped.mean()
+    out[3] = (-d).mean()
+    out[4] = (ratio - 1.0 - d).mean()
+    out[5] = ratio.max()
+    out[6] = ratio.min()
+    out[7] = ((ratio > hi_b) | (ratio < lo_b)).mean()
+    return out
+
+
 def loss_backward(h, w, y, lse, coef, grad_loss=1.0):
     """Gradients of the exported loss with respect to H and W.
 

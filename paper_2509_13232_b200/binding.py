@@ -28,7 +28,7 @@ SUR_PPO_CLIP, SUR_CISPO, SUR_GSPO = 0, 1, 2
 EXPORTS = [
     "spo_default_params", "spo_tracker_init", "spo_sample_prompts", "spo_advantages",
     "spo_advantages_static", "spo_advantages_apply",
-    "spo_tracker_update", "spo_tracker_update_repeats", "spo_loss_fwd", "spo_loss_bwd", "spo_loss_fwd_bwd", "spo_loss_mask_rows", "spo_loss_fwd_bwd_rows", "spo_loss_active_rows", "spo_loss_bwd_rows", "spo_workspace_bytes",
+    "spo_tracker_update", "spo_tracker_update_repeats", "spo_loss_fwd", "spo_loss_bwd", "spo_loss_fwd_bwd", "spo_loss_stats", "spo_loss_mask_rows", "spo_loss_fwd_bwd_rows", "spo_loss_active_rows", "spo_loss_bwd_rows", "spo_workspace_bytes",
     "spo_status_string", "spo_last_cuda_error", "spo_version", "spo_selftest_bounded_wait",
 ]
 
@@ -89,6 +89,8 @@ def lib():
                                        c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                                        c_void_p, c_int32, c_void_p, c_int32,
                                        c_void_p, c_size_t, P, c_void_p, c_void_p]
+        L.spo_loss_stats.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_int32, c_void_p, P,
+                                     c_void_p]
         L.spo_loss_mask_rows.argtypes = [c_void_p, c_int64, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
         L.spo_loss_fwd_bwd_rows.argtypes = [c_void_p, c_void_p, c_int32, c_void_p, c_void_p, c_void_p, c_void_p,
                                             c_int64, c_int32, c_int32, c_int32, c_void_p, c_int64, c_float,
@@ -225,6 +227,11 @@ def spo_loss_fwd_bwd(H, W, y, logp_old, mask, cu_seqlens, a_norm, grad_loss, los
                                   _ptr(logp), _ptr(lse), _ptr(coef), _ptr(seq_sums), _ptr(dH), _dtype_code(dH),
                                   _ptr(dW), int(dW_accumulate), _ptr(ws), ws.numel() * ws.element_size(),
                                   ctypes.byref(params), _ptr(d_status), _stream()), "spo_loss_fwd_bwd")
+
+
+def spo_loss_stats(logp, logp_old, mask, cu_seqlens, a_norm, out, params):
+    _check(lib().spo_loss_stats(_ptr(logp), _ptr(logp_old), _ptr(mask), _ptr(cu_seqlens), _ptr(a_norm), logp.numel(),
+                                cu_seqlens.numel() - 1, _ptr(out), ctypes.byref(params), _stream()), "spo_loss_stats")
 
 
 def spo_loss_mask_rows(mask, rows, d_count, ws):

@@ -484,6 +484,19 @@ int32_t spo_loss_fwd_bwd_rows(const void* H, const void* W, int32_t dtype, const
   return SPO_OK;
 }
 
+int32_t spo_loss_stats(const float* logp, const float* logp_old, const uint8_t* mask, const int32_t* cu_seqlens,
+                       const float* a_norm, int64_t T, int32_t S, float* out, const spo_params* params, void* stream) {
+  if (!params_ok(params) || !out || T < 0 || S < 0) return SPO_ERR_INVALID_ARG;
+  if (T > 0 && (!logp || !logp_old || !cu_seqlens || !a_norm || S < 1)) return SPO_ERR_INVALID_ARG;
+  if (T >= ((int64_t)1 << 31) - 256) return SPO_ERR_BAD_SHAPE;
+  if (!aligned16(logp) || !aligned16(logp_old) || !aligned16(cu_seqlens) || !aligned16(a_norm) || !aligned16(out))
+    return SPO_ERR_BAD_ALIGNMENT;
+  if (!device_is_sm100()) return SPO_ERR_UNSUPPORTED_ARCH;
+  cudaError_t e = launch_loss_stats(logp, logp_old, mask, cu_seqlens, a_norm, T, S, params->clip_lo, params->clip_hi, out,
+                                    (cudaStream_t)stream);
+  return e == cudaSuccess ? SPO_OK : cuda_fail(e);
+}
+
 size_t spo_workspace_bytes(int32_t which, int64_t T, int32_t d, int32_t V, int64_t N, int32_t B, int32_t M) {
   switch (which) {
     case SPO_WS_SAMPLE:

@@ -168,6 +168,9 @@ cudaError_t launch_bwd_bf16(const void* H, const void* W, const int32_t* y, cons
 // rows listed: coef[t] != 0 (coef given) or mask[t] != 0 (mask given, coef NULL)
 cudaError_t launch_active_rows(const float* coef, const uint8_t* mask, int64_t T, int32_t* rows, int32_t* d_count,
                                int32_t* block_cnt, cudaStream_t st);
+cudaError_t launch_loss_stats(const float* logp, const float* logp_old, const uint8_t* mask, const int32_t* cu_seqlens,
+                              const float* a_norm, int64_t T, int32_t S, float clip_lo, float clip_hi, float* out,
+                              cudaStream_t st);
 cudaError_t launch_compact_cu_seqlens(const int32_t* rows, int64_t n_act, const int32_t* cu_seqlens, int32_t S,
                                       int32_t* cu_act, cudaStream_t st);
 cudaError_t launch_scatter_scalars(const float* logp_act, const float* lse_act, const float* coef_act,

@@ -487,6 +487,76 @@ seq_level_apply_kernel(const uint8_t* __restrict__ mask, const int32_t* __restri
   }
 }
 
+// Diagnostics of the policy update over the unmasked tokens, one block (fixed reduction order):
+// count, mean ratio, share of tokens whose gradient the clip stops, two sampled KL estimates,
+// largest / smallest ratio, share of ratios outside the clip bounds.
+__global__ void __launch_bounds__(1024)
+loss_stats_kernel(const float* __restrict__ logp, const float* __restrict__ logp_old, const uint8_t* __restrict__ mask,
+                  const int32_t* __restrict__ cu_seqlens, const float* __restrict__ a_norm, int64_t T, int32_t S,
+                  float clip_lo, float clip_hi, float* __restrict__ out) {
+  const float hi_b = 1.0f + clip_hi, lo_b = 1.0f - clip_lo;
+  double acc[6] = {0.0, 0.0, 0.0, 0.0, 0.0, 0.0};     // count, ratio, stopped, -d, k3, outside
+  float rmax = -CUDART_INF_F, rmin = CUDART_INF_F;
+  for (int64_t t = threadIdx.x; t < T; t += 1024) {
+    if (mask && mask[t] == 0) continue;
+    int lo = 0, hi = S;
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if ((int64_t)cu_seqlens[mid] <= t) lo = mid; else hi = mid;
+    }
+    const float a = a_norm[lo];
+    const float d = logp[t] - logp_old[t];
+    const float r = expf(d);
+    const bool stopped = a > 0.0f ? r > hi_b : (a < 0.0f ? r < lo_b : false);
+    acc[0] += 1.0;
+    acc[1] += (double)r;
+    acc[2] += stopped ? 1.0 : 0.0;
+    acc[3] -= (double)d;
+    acc[4] += (double)r - 1.0 - (double)d;
+    acc[5] += (r > hi_b || r < lo_b) ? 1.0 : 0.0;
+    rmax = fmaxf(rmax, r);
+    rmin = fminf(rmin, r);
+  }
+  __shared__ double s_acc[32][6];
+  __shared__ float s_max[32], s_min[32];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+  for (int k = 0; k < 6; ++k) acc[k] = warp_sum_f64(acc[k]);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    rmax = fmaxf(rmax, __shfl_xor_sync(0xffffffffu, rmax, o));
+    rmin = fminf(rmin, __shfl_xor_sync(0xffffffffu, rmin, o));
+  }
+  if (lane == 0) {
+#pragma unroll
+    for (int k = 0; k < 6; ++k) s_acc[warp][k] = acc[k];
+    s_max[warp] = rmax; s_min[warp] = rmin;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double tot[6] = {0.0, 0.0, 0.0, 0.0, 0.0, 0.0};
+    float mx = -CUDART_INF_F, mn = CUDART_INF_F;
+    for (int w = 0; w < 32; ++w) {
+#pragma unroll
+      for (int k = 0; k < 6; ++k) tot[k] += s_acc[w][k];
+      mx = fmaxf(mx, s_max[w]); mn = fminf(mn, s_min[w]);
+    }
+    if (tot[0] > 0.0) {
+      out[0] = (float)tot[0];
+      out[1] = (float)(tot[1] / tot[0]);
+      out[2] = (float)(tot[2] / tot[0]);
+      out[3] = (float)(tot[3] / tot[0]);
+      out[4] = (float)(tot[4] / tot[0]);
+      out[5] = mx;
+      out[6] = mn;
+      out[7] = (float)(tot[5] / tot[0]);
+    } else {
+#pragma unroll
+      for (int k = 0; k < 8; ++k) out[k] = 0.0f;
+    }
+  }
+}
+
 // Sequence boundaries of the compacted batch: cu_act[s] = number of listed rows below cu_seqlens[s]
 // (rows is ascending, so a lower bound).
 __global__ void __launch_bounds__(256)
@@ -636,6 +706,13 @@ cudaError_t launch_gather_rows(const void* H, const int32_t* y, const float* lse
   gather_rows_kernel<<<(unsigned)blocks, 256, 0, st>>>(reinterpret_cast<const uint4*>(H), y, lse, coef, rows, n_act,
                                                        row_bytes / 16, reinterpret_cast<uint4*>(H_act), y_act, lse_act,
                                                        coef_act);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_loss_stats(const float* logp, const float* logp_old, const uint8_t* mask, const int32_t* cu_seqlens,
+                              const float* a_norm, int64_t T, int32_t S, float clip_lo, float clip_hi, float* out,
+                              cudaStream_t st) {
+  loss_stats_kernel<<<1, 1024, 0, st>>>(logp, logp_old, mask, cu_seqlens, a_norm, T, S, clip_lo, clip_hi, out);
   return cudaGetLastError();
 }
 

@@ -288,3 +288,29 @@ def test_backward_over_active_rows_with_nothing_active():
                         ws_bytes(B.WS_LOSS_BWD_ROWS, T=0, d=d, V=V), B.default_params(), status_word())
     torch.cuda.synchronize()
     assert float(dH.float().abs().max().item()) == 0.0 and float(dW.abs().max().item()) == 0.0
+
+
+def test_loss_stats_against_the_oracle():
+    """Diagnostics of the update (mean ratio, clipped share, KL estimates, extreme ratios) from the forward's logp."""
+    import torch
+    from paper_2509_13232_b200 import binding as B
+    from tests.helpers import dev
+    lb = _clip_batch(170, [900, 1300, 0, 700, 2500, 61], 128, 1500, True)
+    got = run_loss(lb)
+    p = B.default_params()
+    out = torch.full((8,), float("nan"), dtype=torch.float32, device="cuda")
+    B.spo_loss_stats(dev(got["logp"]), dev(lb.logp_old), dev(lb.mask), dev(lb.cu_seqlens), dev(lb.a_norm), out, p)
+    torch.cuda.synchronize()
+    want = O.loss_stats(got["logp"], lb.logp_old, lb.mask, lb.cu_seqlens, lb.a_norm, float(np.float32(p.clip_lo)),
+                        float(np.float32(p.clip_hi)))
+    assert 0.02 < want[2] < 0.9 and want[7] >= want[2]
+    np.testing.assert_allclose(out.cpu().numpy(), want, rtol=1e-5, atol=1e-6)
+    # the share it reports as stopped is the share of unmasked tokens the forward gave a zero coef
+    zero_adv = np.repeat(lb.a_norm, np.diff(lb.cu_seqlens)) == 0
+    stopped = ((got["coef"] == 0) & (lb.mask != 0) & ~zero_adv).sum() / want[0]
+    assert abs(stopped - want[2]) <= 2e-3              # tokens within rounding of a bound may fall on either side
+    # nothing unmasked: zeros
+    B.spo_loss_stats(dev(got["logp"]), dev(lb.logp_old), dev(np.zeros_like(lb.mask)), dev(lb.cu_seqlens), dev(lb.a_norm),
+                     out, p)
+    torch.cuda.synchronize()
+    assert float(out.abs().max().item()) == 0.0

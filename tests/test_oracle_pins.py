@@ -713,3 +713,32 @@ def test_gspo_gradients_against_central_finite_differences():
             arr[idx] = keep
             num[idx] = (up - dn) / (2 * step)
         assert np.linalg.norm(num - grad) <= 1e-6 * np.linalg.norm(grad)
+
+
+def test_loss_stats_hand_values_and_consistency_with_the_objective():
+    logp_old = np.log(np.array([0.5, 0.5, 0.5, 0.5, 0.5, 0.5]))
+    ratios = np.array([1.0, 1.5, 0.5, 1.1, 7.0, 0.6])
+    logp = logp_old + np.log(ratios)
+    mask = np.array([1, 1, 1, 1, 0, 1], dtype=np.uint8)
+    cu, a = [0, 3, 6], np.array([2.0, -1.0])
+    st = O.loss_stats(logp, logp_old, mask, cu, a)
+    live = ratios[[0, 1, 2, 3, 5]]
+    assert st[0] == 5
+    assert abs(st[1] - live.mean()) < 1e-14
+    # a > 0: 1.5 is above 1.28 (stopped), 0.5 is below 0.8 but on the side that still carries gradient;
+    # a < 0: 1.1 inside, 0.6 below 0.8 (stopped)
+    assert abs(st[2] - 2 / 5) < 1e-15
+    assert abs(st[3] + np.log(live).mean()) < 1e-14
+    assert abs(st[4] - (live - 1 - np.log(live)).mean()) < 1e-14 and st[4] >= 0
+    assert st[5] == 1.5 and st[6] == 0.5
+    assert abs(st[7] - 3 / 5) < 1e-15
+    # the tokens it counts as stopped are the unmasked ones whose coef the objective sets to zero
+    h, w, y = _tiny_loss_case(41, cu, 6)
+    base = O.loss_forward(h, w, y, np.zeros(6), mask, cu, a)["logp"]
+    fwd = O.loss_forward(h, w, y, base - np.log(ratios), mask, cu, a)
+    st2 = O.loss_stats(fwd["logp"], base - np.log(ratios), mask, cu, a)
+    assert abs(st2[2] - ((fwd["coef"] == 0) & (mask != 0)).sum() / 5) < 1e-15
+    # identical policies: ratio 1, both KL estimates 0, nothing clipped; nothing unmasked: zeros
+    same = O.loss_stats(logp_old, logp_old, None, cu, a)
+    np.testing.assert_allclose(same, [6, 1, 0, 0, 0, 1, 1, 0], atol=1e-15)
+    assert np.all(O.loss_stats(logp, logp_old, np.zeros(6, np.uint8), cu, a) == 0)
