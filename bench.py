@@ -412,6 +412,8 @@ SMALL_SHAPES = {
     "cfg2_tracker_scale": (1_000_000, 4096, 8192),
     "small_scaled": (1 << 28, 1 << 22, 8192),
     "small_scaled_26": (1 << 26, 1 << 22, 8192),      # a size that profiler captures with many passes can hold
+    "small_scaled_24": (1 << 24, 1 << 20, 8192),
+    "small_scaled_b24": (1 << 28, 1 << 24, 8192),     # the largest batch of the gather kernels
 }
 
 

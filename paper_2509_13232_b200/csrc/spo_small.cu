@@ -323,13 +323,21 @@ sample_accept_kernel(const int32_t* __restrict__ cand, int32_t M, int32_t B, con
   }
 }
 
+// One table entry fetched by id.  Gathers by random id use 8 of the bytes that come back; the
+// 64-byte prefetch-size hint keeps L2 from fetching a wider span from HBM for each of them.
+__device__ __forceinline__ float2 load_entry(const float2* p) {
+  float2 v;
+  asm volatile("ld.global.L2::64B.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "l"(p));
+  return v;
+}
+
 // ---------------------------------------------------------------------------
 // Advantages: A = r - alpha/(alpha+beta) gathered by id; batch mean / std; normalise.
 // ---------------------------------------------------------------------------
 __device__ __forceinline__ float gather_advantage(const float2* __restrict__ ab, int64_t N, int32_t id, float r,
                                                   bool& bad_id) {
   if (id < 0 || (int64_t)id >= N) { bad_id = true; return 0.0f; }
-  float2 e = __ldg(ab + id);
+  float2 e = load_entry(ab + id);
   float n = e.x + e.y;
   float v = n > 0.0f ? e.x / n : 0.5f;
   return r - v;
@@ -473,7 +481,7 @@ tracker_update_kernel(float2* __restrict__ ab, int64_t N, const int32_t* __restr
     for (int q = 0; q < U; ++q) {
       if (live[q] && (id[q] < 0 || (int64_t)id[q] >= N)) { flag(d_status, SPO_DEV_ID_OUT_OF_RANGE); live[q] = false; }
       if (live[q]) {
-        e[q] = ab[id[q]];
+        e[q] = load_entry(ab + id[q]);
         if (kl_is_table) div[q] = __ldg(kl + id[q]);
       }
     }
