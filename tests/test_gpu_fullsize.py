@@ -104,3 +104,21 @@ def test_full_size_sampled_rows_and_identities(workload, path):
     for t0 in range(0, T, 32768):
         rhs += float((step.dH[t0:t0 + 32768].double() * D["h"][t0:t0 + 32768].double()).sum().item())
     assert abs(lhs - rhs) <= 1e-3 * mag
+
+
+@pytest.mark.parametrize("path", ["onepass", "split"])
+def test_full_size_step_is_bitwise_reproducible(path):
+    """Two runs of the whole step at the cfg3 workload (eight chunks, lock-stepped CTA pairs, side warps,
+    chunk-by-chunk dW accumulation): every output identical bit for bit."""
+    import torch
+    import bench
+    step = bench.Step("cfg3_small_bf16", torch.device("cuda", 0), 0, path=path)
+    outs = []
+    for _ in range(2):
+        step.ab.copy_(step.ab0)
+        step.run()
+        torch.cuda.synchronize()
+        outs.append([t.clone() for t in (step.loss, step.logp, step.lse, step.coef, step.dH, step.dW, step.ids, step.ab)])
+    assert int(step.status[0].item()) == 0
+    for a, b in zip(*outs):
+        assert torch.equal(a, b)
