@@ -300,8 +300,9 @@ def loss_forward(h, w, y, logp_old, mask, cu_seqlens, a_norm,
     Returns a dict: loss, logp[T], lse[T], ratio[T], surrogate[T], unclipped[T]
     (bool: the gradient passes through the ratio), coef[T] = d loss / d logp_t
     = -u_t*a*ratio*unclipped with u_t the aggregation weight (mask/n_tok by
-    default, see aggregation_weights), n_tok, and seq_sums[S,3] = per sequence
-    (sum mask*logp, sum mask*(logp_old - logp), sum mask).
+    default, see aggregation_weights), n_tok, seq_sums[S,3] = per sequence
+    (sum mask*logp, sum mask*(logp_old - logp), sum mask), and entropy[T] =
+    -sum_v p log p of each row's softmax (a diagnostic).
     """
     z = logits(h, w)
     n_tok_rows = z.shape[0]
@@ -314,6 +315,10 @@ def loss_forward(h, w, y, logp_old, mask, cu_seqlens, a_norm,
     zmax = z.max(axis=1) if z.shape[1] else np.zeros(n_tok_rows)
     lse = zmax + np.log(np.exp(z - zmax[:, None]).sum(axis=1))
     logp = z[np.arange(n_tok_rows), y] - lse
+    # entropy of the policy's next-token distribution, -sum_v p log p = lse - sum_v p z (a diagnostic;
+    # Sec. 3.2 speaks of retaining policy entropy; it does not enter the objective)
+    p_full = np.exp(z - lse[:, None])
+    entropy = lse - (p_full * z).sum(axis=1)
     ratio = np.exp(logp - logp_old)
     seq = token_sequence_ids(cu_seqlens, n_tok_rows)
     a = np.asarray(a_norm, dtype=np.float64)[seq]
@@ -360,7 +365,7 @@ def loss_forward(h, w, y, logp_old, mask, cu_seqlens, a_norm,
     return {
         "loss": float(loss), "logp": logp, "lse": lse, "ratio": ratio,
         "surrogate": surrogate_t, "unclipped": unclipped, "coef": coef,
-        "n_tok": float(n_tok), "seq_sums": seq_sums,
+        "n_tok": float(n_tok), "seq_sums": seq_sums, "entropy": entropy,
     }
 
 

@@ -742,3 +742,24 @@ def test_loss_stats_hand_values_and_consistency_with_the_objective():
     same = O.loss_stats(logp_old, logp_old, None, cu, a)
     np.testing.assert_allclose(same, [6, 1, 0, 0, 0, 1, 1, 0], atol=1e-15)
     assert np.all(O.loss_stats(logp, logp_old, np.zeros(6, np.uint8), cu, a) == 0)
+
+
+def test_policy_entropy_against_library_and_closed_forms():
+    rng = np.random.default_rng(51)
+    t, d, v = 6, 5, 17
+    h, w = rng.standard_normal((t, d)), rng.standard_normal((v, d)) * 2.0
+    y = rng.integers(0, v, t)
+    cu, a = [0, 6], np.array([1.0])
+    fwd = O.loss_forward(h, w, y, np.zeros(t), None, cu, a)
+    p = scipy.special.softmax(h @ w.T, axis=1)
+    np.testing.assert_allclose(fwd["entropy"], scipy.stats.entropy(p, axis=1), rtol=1e-12)
+    # uniform logits: log V; one dominant logit: close to zero; two equal dominant logits: log 2
+    flat = O.loss_forward(h, np.zeros((v, d)), y, np.zeros(t), None, cu, a)
+    np.testing.assert_allclose(flat["entropy"], math.log(v), rtol=1e-13)
+    hh = np.zeros((1, 2)); hh[0, 0] = 1.0
+    ww = np.zeros((4, 2)); ww[0, 0] = 60.0; ww[1, 0] = 60.0
+    two = O.loss_forward(hh, ww, [0], np.zeros(1), None, [0, 1], a)
+    assert abs(two["entropy"][0] - math.log(2.0)) < 1e-12
+    ww[1, 0] = 0.0
+    one = O.loss_forward(hh, ww, [0], np.zeros(1), None, [0, 1], a)
+    assert 0.0 <= one["entropy"][0] < 1e-20
