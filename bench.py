@@ -105,7 +105,8 @@ class ClockSampler:
 class Step:
     """Device buffers of one workload and the call sequence of one step."""
 
-    def __init__(self, workload, device, rank, responses=None, custom=None, mask_frac=0.0, path="onepass"):
+    def __init__(self, workload, device, rank, responses=None, custom=None, mask_frac=0.0, path="onepass",
+                 entropy=False):
         import torch
         from paper_2509_13232_b200 import binding as B
         from paper_2509_13232_b200 import inputs
@@ -151,6 +152,7 @@ class Step:
         self.stats = torch.empty(4, **f32)
         self.loss = torch.zeros(4, **f32)
         self.logp, self.lse, self.coef = (torch.empty(self.T, **f32) for _ in range(3))
+        self.entropy = torch.empty(self.T, **f32) if entropy else None      # optional per-token policy entropy
         self.dH = torch.empty((self.T, d), dtype=torch.bfloat16, device=device)
         self.dW = torch.empty((V, d), **f32)
         self.status = torch.zeros(4, dtype=torch.int32, device=device)
@@ -209,7 +211,7 @@ class Step:
         self.B.spo_loss_fwd(D["h"] if h is None else h, D["w"], D["y"] if y is None else y,
                             D["logp_old"] if logp_old is None else logp_old, D["mask"] if mask is None else mask,
                             D["cu_seqlens"] if cu is None else cu, self.a_norm, self.loss, self.logp, self.lse,
-                            self.coef, None, self.ws_fwd, self.params, self.status)
+                            self.coef, None, self.ws_fwd, self.params, self.status, entropy=self.entropy)
 
     def bwd(self, h=None, y=None):
         D = self.data
@@ -238,7 +240,8 @@ class Step:
         self.B.spo_loss_fwd_bwd(D["h"] if h is None else h, D["w"], D["y"] if y is None else y,
                                 D["logp_old"] if logp_old is None else logp_old, D["mask"] if mask is None else mask,
                                 D["cu_seqlens"] if cu is None else cu, self.a_norm, 1.0, self.loss, self.logp,
-                                self.lse, self.coef, None, self.dH, self.dW, 0, self.ws_loss, self.params, self.status)
+                                self.lse, self.coef, None, self.dH, self.dW, 0, self.ws_loss, self.params, self.status,
+                                entropy=self.entropy)
 
     def loss_calls(self, h=None, y=None, logp_old=None, mask=None, cu=None):
         """The loss calls of one step on the chosen path."""
@@ -276,7 +279,7 @@ def run_ours(args, rank, world, local_rank):
         spo_build.build()
     if world > 1:
         dist.barrier()
-    step = Step(args.workload, device, rank, args.responses, args.custom, args.mask_frac, args.path)
+    step = Step(args.workload, device, rank, args.responses, args.custom, args.mask_frac, args.path, args.entropy)
     peaks = read_peaks()
 
     def barrier():
@@ -372,7 +375,7 @@ def run_ours(args, rank, world, local_rank):
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": "custom" if args.custom else args.workload, "responses": step.S, "tokens": step.T, "d": step.d, "V": step.V,
-                   "tracker_prompts": step.table_n, "l2": "inputs_exceed_l2", "loss_path": "onepass" if step.onepass else "split",
+                   "tracker_prompts": step.table_n, "l2": "inputs_exceed_l2", "loss_path": "onepass" if step.onepass else "split", "entropy_output": bool(args.entropy),
                    "bwd_chunks": step.bwd_chunks, "mask_frac": step.mask_frac,
                    "parallelism": "replicas" if world > 1 else "single"},
         "gpu_launches": step.launches * args.steps,
@@ -567,6 +570,7 @@ def main():
                          "spo_loss_bwd_rows)")
     ap.add_argument("--path", default="onepass", choices=["onepass", "split"],
                     help="loss as one spo_loss_fwd_bwd call (default) or as spo_loss_fwd + spo_loss_bwd")
+    ap.add_argument("--entropy", action="store_true", help="also ask the loss call for the per-token policy entropy")
     ap.add_argument("--responses", type=int, default=None,
                     help="use only the first S responses of the workload (small cases for profiling)")
     args = ap.parse_args()

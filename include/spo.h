@@ -259,6 +259,10 @@ int32_t spo_tracker_update_repeats(float* ab, int64_t N, const int32_t* ids, con
  *   logp, lse, coef   device out [T] fp32 each
  *   seq_sums    device out [S][3] fp32 = per response (sum mask*logp,
  *               sum mask*(logp_old-logp), sum mask), optional
+ *   entropy     device out [T] fp32, optional: entropy of each row's next-token distribution,
+ *               -sum_v p log p = lse - sum_v p z, in nats (a diagnostic: Sec. 3.2 speaks of retaining
+ *               policy entropy; it does not enter the objective).  Asking for it adds one multiply-add
+ *               per logit to the contraction's epilogue; NULL costs nothing.
  *   ws          device scratch, spo_workspace_bytes(SPO_WS_LOSS_FWD, T, d, V, 0, S, 0) bytes
  *               (the B argument of that query carries the number of responses S)
  * A target outside [0,V) sets SPO_DEV_ID_OUT_OF_RANGE (the row gets logp = -inf, coef = 0).
@@ -267,7 +271,7 @@ int32_t spo_loss_fwd(const void* H, const void* W, int32_t dtype,
                      const int32_t* y, const float* logp_old, const uint8_t* mask,
                      const int32_t* cu_seqlens, const float* a_norm,
                      int64_t T, int32_t d, int32_t V, int32_t S,
-                     float* loss, float* logp, float* lse, float* coef, float* seq_sums,
+                     float* loss, float* logp, float* lse, float* coef, float* seq_sums, float* entropy,
                      void* ws, size_t ws_bytes,
                      const spo_params* params, int32_t* d_status, void* stream);
 
@@ -319,7 +323,7 @@ int32_t spo_loss_fwd_bwd(const void* H, const void* W, int32_t dtype,
                          const int32_t* y, const float* logp_old, const uint8_t* mask,
                          const int32_t* cu_seqlens, const float* a_norm,
                          int64_t T, int32_t d, int32_t V, int32_t S, float grad_loss,
-                         float* loss, float* logp, float* lse, float* coef, float* seq_sums,
+                         float* loss, float* logp, float* lse, float* coef, float* seq_sums, float* entropy,
                          void* dH, int32_t dH_dtype, float* dW, int32_t dW_accumulate,
                          void* ws, size_t ws_bytes,
                          const spo_params* params, int32_t* d_status, void* stream);

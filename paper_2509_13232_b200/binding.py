@@ -79,14 +79,14 @@ def lib():
                                                  c_void_p, c_size_t, P, c_void_p, c_void_p]
         L.spo_loss_fwd.argtypes = [c_void_p, c_void_p, c_int32, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                                    c_int64, c_int32, c_int32, c_int32,
-                                   c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
+                                   c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                                    c_void_p, c_size_t, P, c_void_p, c_void_p]
         L.spo_loss_bwd.argtypes = [c_void_p, c_void_p, c_int32, c_void_p, c_void_p, c_void_p, c_float,
                                    c_int64, c_int32, c_int32, c_void_p, c_int32, c_void_p, c_int32,
                                    c_void_p, c_size_t, P, c_void_p, c_void_p]
         L.spo_loss_fwd_bwd.argtypes = [c_void_p, c_void_p, c_int32, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                                        c_int64, c_int32, c_int32, c_int32, c_float,
-                                       c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
+                                       c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                                        c_void_p, c_int32, c_void_p, c_int32,
                                        c_void_p, c_size_t, P, c_void_p, c_void_p]
         L.spo_loss_stats.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_int32, c_void_p, P,
@@ -198,13 +198,13 @@ def spo_tracker_update_repeats(ab, ids, r, kl, kl_is_table, ws, params, d_status
 
 
 def spo_loss_fwd(H, W, y, logp_old, mask, cu_seqlens, a_norm, loss, logp, lse, coef, seq_sums, ws, params,
-                 d_status):
+                 d_status, entropy=None):
     T, d = H.shape
     V = W.shape[0]
     S = cu_seqlens.numel() - 1
     _check(lib().spo_loss_fwd(_ptr(H), _ptr(W), _dtype_code(W), _ptr(y), _ptr(logp_old), _ptr(mask),
                               _ptr(cu_seqlens), _ptr(a_norm), T, d, V, S, _ptr(loss), _ptr(logp), _ptr(lse),
-                              _ptr(coef), _ptr(seq_sums), _ptr(ws), ws.numel() * ws.element_size(),
+                              _ptr(coef), _ptr(seq_sums), _ptr(entropy), _ptr(ws), ws.numel() * ws.element_size(),
                               ctypes.byref(params), _ptr(d_status), _stream()), "spo_loss_fwd")
 
 
@@ -218,15 +218,16 @@ def spo_loss_bwd(H, W, y, lse, coef, grad_loss, dH, dW, dW_accumulate, ws, param
 
 
 def spo_loss_fwd_bwd(H, W, y, logp_old, mask, cu_seqlens, a_norm, grad_loss, loss, logp, lse, coef, seq_sums, dH, dW,
-                     dW_accumulate, ws, params, d_status):
+                     dW_accumulate, ws, params, d_status, entropy=None):
     T, d = H.shape
     V = W.shape[0]
     S = cu_seqlens.numel() - 1
     _check(lib().spo_loss_fwd_bwd(_ptr(H), _ptr(W), _dtype_code(W), _ptr(y), _ptr(logp_old), _ptr(mask),
                                   _ptr(cu_seqlens), _ptr(a_norm), T, d, V, S, c_float(grad_loss), _ptr(loss),
-                                  _ptr(logp), _ptr(lse), _ptr(coef), _ptr(seq_sums), _ptr(dH), _dtype_code(dH),
-                                  _ptr(dW), int(dW_accumulate), _ptr(ws), ws.numel() * ws.element_size(),
-                                  ctypes.byref(params), _ptr(d_status), _stream()), "spo_loss_fwd_bwd")
+                                  _ptr(logp), _ptr(lse), _ptr(coef), _ptr(seq_sums), _ptr(entropy), _ptr(dH),
+                                  _dtype_code(dH), _ptr(dW), int(dW_accumulate), _ptr(ws),
+                                  ws.numel() * ws.element_size(), ctypes.byref(params), _ptr(d_status), _stream()),
+           "spo_loss_fwd_bwd")
 
 
 def spo_loss_stats(logp, logp_old, mask, cu_seqlens, a_norm, out, params):

@@ -84,7 +84,8 @@ namespace spo {
 static cudaError_t forward_launches(const void* H, const void* W, int32_t dtype, const int32_t* y,
                                     const float* logp_old, const uint8_t* mask, const int32_t* cu_seqlens,
                                     const float* a_norm, int64_t T, int32_t d, int32_t V, int32_t S, float* loss,
-                                    float* logp, float* lse, float* coef, float* seq_sums, char* w8, const FwdWs& L,
+                                    float* logp, float* lse, float* coef, float* seq_sums, float* entropy, char* w8,
+                                    const FwdWs& L,
                                     const spo_params* params, int32_t* d_status, cudaStream_t st) {
   FwdPartial* partials = reinterpret_cast<FwdPartial*>(w8 + L.partials);
   double* block_sums = reinterpret_cast<double*>(w8 + L.block_sums);
@@ -94,13 +95,14 @@ static cudaError_t forward_launches(const void* H, const void* W, int32_t dtype,
   cudaError_t e = launch_fwd_prepare(mask, T, cu_seqlens, S, params->agg_mode != 0 || seq_level, seq_cnt, counters, st);
   if (e != cudaSuccess) return e;
   if (dtype == SPO_DTYPE_BF16)
-    e = launch_fwd_bf16(H, W, y, T, d, V, partials, L.nsplit, reinterpret_cast<uint32_t*>(w8 + L.progress), d_status, st);
+    e = launch_fwd_bf16(H, W, y, T, d, V, partials, L.nsplit, entropy != nullptr,
+                        reinterpret_cast<uint32_t*>(w8 + L.progress), d_status, st);
   else
     e = launch_fwd_f32((const float*)H, (const float*)W, y, T, d, V, partials, st);
   if (e != cudaSuccess) return e;
   e = launch_fwd_finalize(partials, L.nsplit, y, logp_old, mask, cu_seqlens, a_norm, T, V, S, params->clip_lo,
-                          params->clip_hi, loss, logp, lse, coef, seq_sums, block_sums, counters, seq_cnt, params->agg_mode,
-                          params->surrogate, params->global_tokens, params->global_responses, L.fin_blocks, d_status, st);
+                          params->clip_hi, loss, logp, lse, coef, seq_sums, entropy, block_sums, counters, seq_cnt,
+                          params->agg_mode, params->surrogate, params->global_tokens, params->global_responses, L.fin_blocks, d_status, st);
   if (e != cudaSuccess || !seq_level) return e;
   return launch_seq_level_objective(logp, logp_old, mask, cu_seqlens, a_norm, T, S, params->clip_lo, params->clip_hi,
                                     counters, params->global_responses, reinterpret_cast<float*>(w8 + L.seq_coef),
@@ -225,19 +227,21 @@ static int32_t check_loss_shape(int32_t dtype, int64_t T, int32_t d, int32_t V) 
 int32_t spo_loss_fwd(const void* H, const void* W, int32_t dtype, const int32_t* y, const float* logp_old,
                      const uint8_t* mask, const int32_t* cu_seqlens, const float* a_norm, int64_t T, int32_t d,
                      int32_t V, int32_t S, float* loss, float* logp, float* lse, float* coef, float* seq_sums,
-                     void* ws, size_t ws_bytes, const spo_params* params, int32_t* d_status, void* stream) {
+                     float* entropy, void* ws, size_t ws_bytes, const spo_params* params, int32_t* d_status,
+                     void* stream) {
   int32_t rc = check_loss_shape(dtype, T, d, V);
   if (rc != SPO_OK) return rc;
   if (!params_ok(params) || !W || !loss || !ws || !cu_seqlens || S < 0) return SPO_ERR_INVALID_ARG;
   if (T > 0 && (!H || !y || !logp_old || !a_norm || !logp || !lse || !coef || S < 1)) return SPO_ERR_INVALID_ARG;
   if (!aligned16(H) || !aligned16(W) || !aligned16(y) || !aligned16(logp_old) || !aligned16(cu_seqlens) ||
-      !aligned16(a_norm) || !aligned16(logp) || !aligned16(lse) || !aligned16(coef) || !aligned16(ws))
+      !aligned16(a_norm) || !aligned16(logp) || !aligned16(lse) || !aligned16(coef) || !aligned16(entropy) ||
+      !aligned16(ws))
     return SPO_ERR_BAD_ALIGNMENT;
   if (!device_is_sm100()) return SPO_ERR_UNSUPPORTED_ARCH;
   const FwdWs L = fwd_ws_layout(T, d, V, dtype, S);
   if (ws_bytes < L.total) return SPO_ERR_WORKSPACE_TOO_SMALL;
   cudaError_t e = forward_launches(H, W, dtype, y, logp_old, mask, cu_seqlens, a_norm, T, d, V, S, loss, logp, lse, coef,
-                                   seq_sums, (char*)ws, L, params, d_status, (cudaStream_t)stream);
+                                   seq_sums, entropy, (char*)ws, L, params, d_status, (cudaStream_t)stream);
   return e == cudaSuccess ? SPO_OK : cuda_fail(e);
 }
 
@@ -272,8 +276,8 @@ int32_t spo_loss_bwd(const void* H, const void* W, int32_t dtype, const int32_t*
 int32_t spo_loss_fwd_bwd(const void* H, const void* W, int32_t dtype, const int32_t* y, const float* logp_old,
                          const uint8_t* mask, const int32_t* cu_seqlens, const float* a_norm, int64_t T, int32_t d,
                          int32_t V, int32_t S, float grad_loss, float* loss, float* logp, float* lse, float* coef,
-                         float* seq_sums, void* dH, int32_t dH_dtype, float* dW, int32_t dW_accumulate, void* ws,
-                         size_t ws_bytes, const spo_params* params, int32_t* d_status, void* stream) {
+                         float* seq_sums, float* entropy, void* dH, int32_t dH_dtype, float* dW, int32_t dW_accumulate,
+                         void* ws, size_t ws_bytes, const spo_params* params, int32_t* d_status, void* stream) {
   int32_t rc = check_loss_shape(dtype, T, d, V);
   if (rc != SPO_OK) return rc;
   if (dH_dtype != SPO_DTYPE_F32 && dH_dtype != SPO_DTYPE_BF16) return SPO_ERR_UNSUPPORTED_DTYPE;
@@ -281,7 +285,7 @@ int32_t spo_loss_fwd_bwd(const void* H, const void* W, int32_t dtype, const int3
   if (T > 0 && (!H || !y || !logp_old || !a_norm || !logp || !lse || !coef || !dH || S < 1)) return SPO_ERR_INVALID_ARG;
   if (!aligned16(H) || !aligned16(W) || !aligned16(y) || !aligned16(logp_old) || !aligned16(cu_seqlens) ||
       !aligned16(a_norm) || !aligned16(logp) || !aligned16(lse) || !aligned16(coef) || !aligned16(dH) ||
-      !aligned16(dW) || !aligned16(ws))
+      !aligned16(dW) || !aligned16(ws) || !aligned16(entropy))
     return SPO_ERR_BAD_ALIGNMENT;
   if (!device_is_sm100()) return SPO_ERR_UNSUPPORTED_ARCH;
   cudaStream_t st = (cudaStream_t)stream;
@@ -294,7 +298,7 @@ int32_t spo_loss_fwd_bwd(const void* H, const void* W, int32_t dtype, const int3
     FusedArgs a{};
     a.H = H; a.W = W; a.y = y; a.logp_old = logp_old; a.mask = mask; a.cu_seqlens = cu_seqlens; a.a_norm = a_norm;
     a.T = T; a.d = d; a.V = V; a.S = S; a.grad_loss = grad_loss;
-    a.loss = loss; a.logp = logp; a.lse = lse; a.coef = coef; a.seq_sums = seq_sums;
+    a.loss = loss; a.logp = logp; a.lse = lse; a.coef = coef; a.seq_sums = seq_sums; a.entropy = entropy;
     a.dH = dH; a.dH_dtype = dH_dtype; a.dW = dW; a.accumulate = dW_accumulate;
     a.params = params; a.d_status = d_status;
     e = launch_fused_bf16(a, w8, L, st);
@@ -304,7 +308,7 @@ int32_t spo_loss_fwd_bwd(const void* H, const void* W, int32_t dtype, const int3
   const FwdWs L = fwd_ws_layout(T, d, V, dtype, S);
   if (ws_bytes < L.total) return SPO_ERR_WORKSPACE_TOO_SMALL;
   if ((e = forward_launches(H, W, dtype, y, logp_old, mask, cu_seqlens, a_norm, T, d, V, S, loss, logp, lse, coef,
-                            seq_sums, w8, L, params, d_status, st)) != cudaSuccess)
+                            seq_sums, entropy, w8, L, params, d_status, st)) != cudaSuccess)
     return cuda_fail(e);
   e = launch_bwd_f32((const float*)H, (const float*)W, y, lse, coef, grad_loss, T, d, V, dH, dH_dtype, dW,
                      dW_accumulate, st);
@@ -474,7 +478,7 @@ int32_t spo_loss_fwd_bwd_rows(const void* H, const void* W, int32_t dtype, const
   FusedArgs a{};
   a.H = h_act; a.W = W; a.y = y_act; a.logp_old = lo_act; a.mask = nullptr; a.cu_seqlens = cu_act; a.a_norm = a_norm;
   a.T = T_act; a.d = d; a.V = V; a.S = S; a.grad_loss = grad_loss;
-  a.loss = loss; a.logp = logp_act; a.lse = lse_act; a.coef = coef_act; a.seq_sums = seq_sums;
+  a.loss = loss; a.logp = logp_act; a.lse = lse_act; a.coef = coef_act; a.seq_sums = seq_sums; a.entropy = nullptr;
   a.dH = dh_act; a.dH_dtype = dH_dtype; a.dW = dW; a.accumulate = dW_accumulate;
   a.params = params; a.d_status = d_status;
   if ((e = launch_fused_bf16(a, w8 + L.fused, L.inner, st)) != cudaSuccess) return cuda_fail(e);

@@ -59,7 +59,8 @@ cudaError_t launch_tracker_update_repeats(float* ab, int64_t N, const int32_t* i
 
 // ---- loss: pieces shared by the fp32 and bf16 paths ------------------------
 // Forward partial statistics of one vocabulary split, per token row:
-// (running max of z*log2(e), sum of 2^(z*log2(e) - max), target logit or -inf).
+// (running max of z*log2(e), sum e of 2^(z*log2(e) - max), target logit or -inf, and in `pad`
+// the sum of e*z when the entropy was asked for).
 struct FwdPartial { float m2, l, zt; float pad; };
 
 constexpr int kFinalizeThreads = 256;
@@ -101,7 +102,7 @@ cudaError_t launch_fwd_finalize(const FwdPartial* partials, int nsplit, const in
                                 const float* logp_old, const uint8_t* mask, const int32_t* cu_seqlens,
                                 const float* a_norm, int64_t T, int32_t V, int32_t S,
                                 float clip_lo, float clip_hi,
-                                float* loss, float* logp, float* lse, float* coef, float* seq_sums,
+                                float* loss, float* logp, float* lse, float* coef, float* seq_sums, float* entropy,
                                 double* block_sums, int32_t* counters, const int32_t* seq_cnt, int agg_mode,
                                 int surrogate, int32_t global_tokens, int32_t global_responses,
                                 int64_t fin_blocks, int32_t* d_status, cudaStream_t st,
@@ -147,7 +148,7 @@ struct FusedArgs {
   int64_t T;
   int32_t d, V, S;
   float grad_loss;
-  float *loss, *logp, *lse, *coef, *seq_sums;
+  float *loss, *logp, *lse, *coef, *seq_sums, *entropy;
   void* dH;
   int32_t dH_dtype;
   float* dW;
@@ -158,7 +159,8 @@ struct FusedArgs {
 cudaError_t launch_fused_bf16(const FusedArgs& a, char* ws, const FusedWs& L, cudaStream_t st);
 
 cudaError_t launch_fwd_bf16(const void* H, const void* W, const int32_t* y, int64_t T, int32_t d, int32_t V,
-                            FwdPartial* partials, int nsplit, uint32_t* progress, int32_t* d_status, cudaStream_t st);
+                            FwdPartial* partials, int nsplit, int want_entropy, uint32_t* progress, int32_t* d_status,
+                            cudaStream_t st);
 cudaError_t launch_bwd_bf16(const void* H, const void* W, const int32_t* y, const float* lse,
                             const float* coef, float grad_loss, int64_t T, int32_t d, int32_t V,
                             void* dH, int32_t dH_dtype, float* dW, int accumulate,

@@ -79,7 +79,7 @@ fwd_finalize_kernel(const FwdPartial* __restrict__ partials, int nsplit, const i
                     const int32_t* __restrict__ cu_seqlens, const float* __restrict__ a_norm,
                     int64_t T, int32_t V, int32_t S, float clip_lo, float clip_hi,
                     float* __restrict__ loss, float* __restrict__ logp_out, float* __restrict__ lse_out,
-                    float* __restrict__ coef_out, double* block_sums, int32_t* counters,
+                    float* __restrict__ coef_out, float* __restrict__ entropy_out, double* block_sums, int32_t* counters,
                     const int32_t* __restrict__ seq_cnt, int agg_mode, int surrogate, int32_t global_tokens,
                     int32_t global_responses, int32_t* d_status, FinalizeRange rg) {
   // This launch covers token rows [rg.t_begin, T_end); its blocks are blocks rg.block0.. of the
@@ -97,12 +97,15 @@ fwd_finalize_kernel(const FwdPartial* __restrict__ partials, int nsplit, const i
       m2 = fmaxf(m2, p.m2);
       zt = fmaxf(zt, p.zt);
     }
-    float l = 0.0f;
+    float l = 0.0f, ez = 0.0f;
     for (int s = 0; s < nsplit; ++s) {
       FwdPartial p = partials[(int64_t)s * rg.part_ld + tp];
-      l += p.l * exp2f(p.m2 - m2);
+      const float w = exp2f(p.m2 - m2);
+      l += p.l * w;
+      ez += p.pad * w;                       // sum_v e z of the split (filled when the entropy is asked for)
     }
     const float lse = (m2 + log2f(l)) * kLn2;
+    if (entropy_out) entropy_out[t] = lse - ez / l;      // -sum_v p log p = lse - sum_v p z
     const int32_t yt = y[t];
     float lp, coef = 0.0f;
     if (yt < 0 || yt >= V) {
@@ -221,7 +224,7 @@ fwd_f32_kernel(const float* __restrict__ H, const float* __restrict__ W, const i
   for (int k = threadIdx.x; k < d; k += 128) s_h[k] = H[t * d + k];
   __syncthreads();
   const int32_t yt = y[t];
-  float m2 = -CUDART_INF_F, l = 0.0f, zt = -CUDART_INF_F;
+  float m2 = -CUDART_INF_F, l = 0.0f, zt = -CUDART_INF_F, ez = 0.0f;
   for (int v = warp; v < V; v += 4) {
     const float* wr = W + (int64_t)v * d;
     float acc = 0.0f;
@@ -229,23 +232,25 @@ fwd_f32_kernel(const float* __restrict__ H, const float* __restrict__ W, const i
     const float z = warp_sum_f32(acc);
     const float z2 = z * kLog2e;
     const float mn = fmaxf(m2, z2);
-    l = l * exp2f(m2 - mn) + exp2f(z2 - mn);
+    const float down = exp2f(m2 - mn), e = exp2f(z2 - mn);
+    l = l * down + e;
+    ez = ez * down + e * z;
     m2 = mn;
     if (v == yt) zt = z;
   }
-  __shared__ float s_m[4], s_l[4], s_z[4];
-  if (lane == 0) { s_m[warp] = m2; s_l[warp] = l; s_z[warp] = zt; }
+  __shared__ float s_m[4], s_l[4], s_z[4], s_e[4];
+  if (lane == 0) { s_m[warp] = m2; s_l[warp] = l; s_z[warp] = zt; s_e[warp] = ez; }
   __syncthreads();
   if (threadIdx.x == 0) {
     float mm = fmaxf(fmaxf(s_m[0], s_m[1]), fmaxf(s_m[2], s_m[3]));
-    float ll = 0.0f, zz = -CUDART_INF_F;
+    float ll = 0.0f, zz = -CUDART_INF_F, ee = 0.0f;
 #pragma unroll
     for (int w = 0; w < 4; ++w) {
-      if (s_l[w] > 0.0f) ll += s_l[w] * exp2f(s_m[w] - mm);
+      if (s_l[w] > 0.0f) { ll += s_l[w] * exp2f(s_m[w] - mm); ee += s_e[w] * exp2f(s_m[w] - mm); }
       zz = fmaxf(zz, s_z[w]);
     }
     FwdPartial p;
-    p.m2 = mm; p.l = ll; p.zt = zz; p.pad = 0.0f;
+    p.m2 = mm; p.l = ll; p.zt = zz; p.pad = ee;
     partials[t] = p;
   }
 }
@@ -615,7 +620,7 @@ cudaError_t launch_fwd_finalize(const FwdPartial* partials, int nsplit, const in
                                 const float* logp_old, const uint8_t* mask, const int32_t* cu_seqlens,
                                 const float* a_norm, int64_t T, int32_t V, int32_t S,
                                 float clip_lo, float clip_hi,
-                                float* loss, float* logp, float* lse, float* coef, float* seq_sums,
+                                float* loss, float* logp, float* lse, float* coef, float* seq_sums, float* entropy,
                                 double* block_sums, int32_t* counters, const int32_t* seq_cnt, int agg_mode,
                                 int surrogate, int32_t global_tokens, int32_t global_responses,
                                 int64_t fin_blocks, int32_t* d_status, cudaStream_t st,
@@ -633,8 +638,8 @@ cudaError_t launch_fwd_finalize(const FwdPartial* partials, int nsplit, const in
   if (blocks == 0) return cudaSuccess;
   fwd_finalize_kernel<<<blocks, kFinalizeThreads, 0, st>>>(
       partials, nsplit, y, logp_old, mask, cu_seqlens, a_norm, T, V, S, clip_lo, clip_hi,
-      loss, logp, lse, coef, block_sums, counters, seq_cnt, agg_mode, surrogate, global_tokens, global_responses,
-      d_status, rg);
+      loss, logp, lse, coef, entropy, block_sums, counters, seq_cnt, agg_mode, surrogate, global_tokens,
+      global_responses, d_status, rg);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   if (seq_sums && S > 0 && rg.last) {

@@ -419,7 +419,10 @@ __device__ __forceinline__ Unit unit_of(int u, const GemmParams& p) {
 constexpr int SIDE_WARPS = 2;
 constexpr int kSideUnroll = 16;
 
-template <int MODE, bool SIDE = false>
+// ENT (FWD / E): also accumulate sum_v e z per row, from which the finalisation forms the entropy of
+// the row's softmax, lse - sum_v p z (one more multiply-add per logit; a separate instantiation so that
+// the kernels without it stay as they are).
+template <int MODE, bool SIDE = false, bool ENT = false>
 __global__ void __launch_bounds__(NUM_THREADS + (SIDE ? 32 * SIDE_WARPS : 0), 1)
 spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmParams p) {
   constexpr bool A_MN = (MODE == MODE_DW);
@@ -574,6 +577,7 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       const bool row_ok = grow < p.rows_valid;
       // per-row state
       float m2 = -CUDART_INF_F, l = 0.0f, zt = -CUDART_INF_F;             // FWD
+      float ez = 0.0f;                                                     // ENT: sum e z relative to m2
       int32_t yt = -1;
       float c = 0.0f, lse2 = 0.0f;                                         // G
       if (MODE == MODE_FWD || MODE == MODE_G || MODE == MODE_E) {
@@ -597,9 +601,11 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             uint32_t v[32];
             tmem_ld32(taddr + ch * 32, v);
             if (col0 + 32 > p.cols_valid) {                            // ragged last chunk of the vocabulary
+              // (with ENT a large finite value instead of -inf: its e is 0 either way and 0 * z stays 0)
+              const float fill = ENT ? -1.0e30f : -CUDART_INF_F;
 #pragma unroll
               for (int j = 0; j < 32; ++j)
-                if (col0 + j >= p.cols_valid) v[j] = __float_as_uint(-CUDART_INF_F);
+                if (col0 + j >= p.cols_valid) v[j] = __float_as_uint(fill);
             }
             float mx0 = __uint_as_float(v[0]), mx1 = __uint_as_float(v[1]);
 #pragma unroll
@@ -609,13 +615,21 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             }
             const float mn = fmaxf(m2, fmaxf(mx0, mx1) * kLog2e);
             const float neg = -mn;
-            float s0 = 0.0f, s1 = 0.0f;
+            float s0 = 0.0f, s1 = 0.0f, t0 = 0.0f, t1 = 0.0f;
 #pragma unroll
             for (int j = 0; j < 32; j += 2) {
-              s0 += fast_exp2(fmaf(__uint_as_float(v[j]), kLog2e, neg));
-              s1 += fast_exp2(fmaf(__uint_as_float(v[j + 1]), kLog2e, neg));
+              const float e0 = fast_exp2(fmaf(__uint_as_float(v[j]), kLog2e, neg));
+              const float e1 = fast_exp2(fmaf(__uint_as_float(v[j + 1]), kLog2e, neg));
+              s0 += e0;
+              s1 += e1;
+              if (ENT) {
+                t0 = fmaf(e0, __uint_as_float(v[j]), t0);
+                t1 = fmaf(e1, __uint_as_float(v[j + 1]), t1);
+              }
             }
-            l = fmaf(l, fast_exp2(m2 - mn), s0 + s1);
+            const float down = fast_exp2(m2 - mn);
+            l = fmaf(l, down, s0 + s1);
+            if (ENT) ez = fmaf(ez, down, t0 + t1);
             m2 = mn;
             if (yt >= col0 && yt < col0 + 32) {
               const int jj = yt - col0;
@@ -644,8 +658,9 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
               if (col0 + 64 > p.cols_valid) {                          // ragged end of the vocabulary
 #pragma unroll
                 for (int j = 0; j < 32; ++j) {
-                  if (col0 + j >= p.cols_valid) v0[j] = __float_as_uint(-CUDART_INF_F);
-                  if (col0 + 32 + j >= p.cols_valid) v1[j] = __float_as_uint(-CUDART_INF_F);
+                  const float fill = ENT ? -1.0e30f : -CUDART_INF_F;
+                  if (col0 + j >= p.cols_valid) v0[j] = __float_as_uint(fill);
+                  if (col0 + 32 + j >= p.cols_valid) v1[j] = __float_as_uint(fill);
                 }
               }
               float mx0 = __uint_as_float(v0[0]), mx1 = __uint_as_float(v0[1]);
@@ -667,7 +682,7 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 }
               }
               const float neg = -ref2;
-              float s0 = 0.0f, s1 = 0.0f, s2 = 0.0f, s3 = 0.0f;
+              float s0 = 0.0f, s1 = 0.0f, s2 = 0.0f, s3 = 0.0f, t0 = 0.0f, t1 = 0.0f;
 #pragma unroll
               for (int j = 0; j < 32; j += 2) {
                 const float e0 = fast_exp2(fmaf(__uint_as_float(v0[j]), kLog2e, neg));
@@ -675,11 +690,17 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 const float e2 = fast_exp2(fmaf(__uint_as_float(v1[j]), kLog2e, neg));
                 const float e3 = fast_exp2(fmaf(__uint_as_float(v1[j + 1]), kLog2e, neg));
                 s0 += e0; s1 += e1; s2 += e2; s3 += e3;
+                if (ENT) {
+                  t0 = fmaf(e0, __uint_as_float(v0[j]), fmaf(e1, __uint_as_float(v0[j + 1]), t0));
+                  t1 = fmaf(e2, __uint_as_float(v1[j]), fmaf(e3, __uint_as_float(v1[j + 1]), t1));
+                }
                 v0[j] = __float_as_uint(e0); v0[j + 1] = __float_as_uint(e1);
                 v1[j] = __float_as_uint(e2); v1[j + 1] = __float_as_uint(e3);
               }
               const float mn = fmaxf(m2, ref2);
-              l = fmaf(l, fast_exp2(m2 - mn), ((s0 + s1) + (s2 + s3)) * fast_exp2(ref2 - mn));
+              const float down = fast_exp2(m2 - mn), up = fast_exp2(ref2 - mn);
+              l = fmaf(l, down, ((s0 + s1) + (s2 + s3)) * up);
+              if (ENT) ez = fmaf(ez, down, (t0 + t1) * up);
               m2 = mn;
               bf16_values(v0, piece);
               bf16_values(v1, piece + 4);
@@ -769,7 +790,7 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       }
       if ((MODE == MODE_FWD || MODE == MODE_E) && ok && row_ok) {
         FwdPartial part;
-        part.m2 = m2; part.l = l; part.zt = zt; part.pad = 0.0f;
+        part.m2 = m2; part.l = l; part.zt = zt; part.pad = ez;
         p.partials[(int64_t)((u % p.nsplit) * 2 + half) * p.T + (grow - p.part_row0)] = part;
       }
     }
@@ -849,7 +870,7 @@ constexpr int kLockStepWindow = 1;
 // CTA pairs that can be resident at once (one CTA per SM).
 int group_count() { return sm_count() / CG; }
 
-template <int MODE, bool SIDE = false>
+template <int MODE, bool SIDE = false, bool ENT = false>
 cudaError_t launch_gemm(const CUtensorMap& a, const CUtensorMap& b, const GemmParams& p_in, uint32_t* progress,
                         cudaStream_t st) {
   constexpr int kThreads = NUM_THREADS + (SIDE ? 32 * SIDE_WARPS : 0);
@@ -858,7 +879,7 @@ cudaError_t launch_gemm(const CUtensorMap& a, const CUtensorMap& b, const GemmPa
   cudaGetDevice(&dev);
   if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
   if (max_groups[dev] == 0) {
-    cudaError_t e = cudaFuncSetAttribute(spo_gemm_kernel<MODE, SIDE>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    cudaError_t e = cudaFuncSetAttribute(spo_gemm_kernel<MODE, SIDE, ENT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (e != cudaSuccess) return e;
     // The kernel is persistent and its pairs pace one another, so the grid must not exceed what the
     // device can hold at one time.
@@ -874,7 +895,7 @@ cudaError_t launch_gemm(const CUtensorMap& a, const CUtensorMap& b, const GemmPa
     q.attrs = qa;
     q.numAttrs = 1;
     int n = 0;
-    e = cudaOccupancyMaxActiveClusters(&n, spo_gemm_kernel<MODE, SIDE>, &q);
+    e = cudaOccupancyMaxActiveClusters(&n, spo_gemm_kernel<MODE, SIDE, ENT>, &q);
     if (e != cudaSuccess) return e;
     if (n < 1) return cudaErrorLaunchOutOfResources;
     max_groups[dev] = n < group_count() ? n : group_count();
@@ -903,7 +924,7 @@ cudaError_t launch_gemm(const CUtensorMap& a, const CUtensorMap& b, const GemmPa
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, spo_gemm_kernel<MODE, SIDE>, a, b, p);
+  return cudaLaunchKernelEx(&cfg, spo_gemm_kernel<MODE, SIDE, ENT>, a, b, p);
 }
 
 // Operand box heights (rows per TMA box) for K-major operands.
@@ -951,7 +972,8 @@ int fwd_unit_splits(int64_t T, int32_t d, int32_t V) {
 int fwd_bf16_nsplit(int64_t T, int32_t d, int32_t V) { return 2 * fwd_unit_splits(T, d, V); }
 
 cudaError_t launch_fwd_bf16(const void* H, const void* W, const int32_t* y, int64_t T, int32_t d, int32_t V,
-                            FwdPartial* partials, int nsplit, uint32_t* progress, int32_t* d_status, cudaStream_t st) {
+                            FwdPartial* partials, int nsplit, int want_entropy, uint32_t* progress, int32_t* d_status,
+                            cudaStream_t st) {
   if (T == 0) return cudaSuccess;
   CUtensorMap ma, mb;
   if (!make_map(&ma, H, d, T, d, kBoxA) || !make_map(&mb, W, d, V, d, kBoxB)) return cudaErrorInvalidValue;
@@ -968,6 +990,7 @@ cudaError_t launch_fwd_bf16(const void* H, const void* W, const int32_t* y, int6
   p.partials = partials;
   p.T = T;
   p.d_status = d_status;
+  if (want_entropy) return launch_gemm<MODE_FWD, false, true>(ma, mb, p, progress, st);
   return launch_gemm<MODE_FWD>(ma, mb, p, progress, st);
 }
 
@@ -1138,7 +1161,7 @@ cudaError_t launch_fused_bf16(const FusedArgs& a, char* ws, const FusedWs& L, cu
   if (e != cudaSuccess) return e;
   if (T == 0) {
     e = launch_fwd_finalize(partials, 0, a.y, a.logp_old, a.mask, a.cu_seqlens, a.a_norm, 0, V, a.S, pr.clip_lo,
-                            pr.clip_hi, a.loss, a.logp, a.lse, a.coef, a.seq_sums, block_sums, counters, seq_cnt,
+                            pr.clip_hi, a.loss, a.logp, a.lse, a.coef, a.seq_sums, a.entropy, block_sums, counters, seq_cnt,
                             pr.agg_mode, pr.surrogate, pr.global_tokens, pr.global_responses, L.fin_blocks, a.d_status,
                             st);
     if (e != cudaSuccess) return e;
@@ -1200,11 +1223,14 @@ cudaError_t launch_fused_bf16(const FusedArgs& a, char* ws, const FusedWs& L, cu
       p.G = g_of(c); p.ldg = L.ldg;
       p.ref = ref_of(c); p.ref_ld = L.chunk_rows;
       p.d_status = a.d_status;
+      const bool ent = a.entropy != nullptr;
       if (c > 0) {
         p.side = e2g_job(c - 1);
-        e = launch_gemm<MODE_E, true>(mH_k, mW_k, p, progress, st);
+        e = ent ? launch_gemm<MODE_E, true, true>(mH_k, mW_k, p, progress, st)
+                : launch_gemm<MODE_E, true, false>(mH_k, mW_k, p, progress, st);
       } else {
-        e = launch_gemm<MODE_E, false>(mH_k, mW_k, p, progress, st);
+        e = ent ? launch_gemm<MODE_E, false, true>(mH_k, mW_k, p, progress, st)
+                : launch_gemm<MODE_E, false, false>(mH_k, mW_k, p, progress, st);
       }
       if (e != cudaSuccess) return e;
     }
@@ -1217,7 +1243,7 @@ cudaError_t launch_fused_bf16(const FusedArgs& a, char* ws, const FusedWs& L, cu
       rg.total_blocks = (int)L.fin_blocks;
       rg.last = (c == n_chunks - 1) ? 1 : 0;
       e = launch_fwd_finalize(partials, 2 * nsplit, a.y, a.logp_old, a.mask, a.cu_seqlens, a.a_norm, t0 + rows, V,
-                              a.S, pr.clip_lo, pr.clip_hi, a.loss, a.logp, a.lse, a.coef, a.seq_sums, block_sums,
+                              a.S, pr.clip_lo, pr.clip_hi, a.loss, a.logp, a.lse, a.coef, a.seq_sums, a.entropy, block_sums,
                               counters, seq_cnt, pr.agg_mode, pr.surrogate, pr.global_tokens, pr.global_responses,
                               L.fin_blocks, a.d_status, st, &rg);
       if (e != cudaSuccess) return e;

@@ -29,7 +29,7 @@ def ws_bytes(which, **kw):
 
 
 def run_loss(lb, params=None, grad_loss=1.0, dh_bf16=None, want_seq_sums=True, dw_init=None, mask_none=False,
-             one_pass=False):
+             one_pass=False, want_entropy=False):
     """Forward + backward through the binding for a LossBatch; returns numpy outputs.
     one_pass: a single spo_loss_fwd_bwd call instead of spo_loss_fwd followed by spo_loss_bwd."""
     import torch
@@ -48,6 +48,7 @@ def run_loss(lb, params=None, grad_loss=1.0, dh_bf16=None, want_seq_sums=True, d
     logp, lse, coef = (torch.full((max(T, 1),), float("nan"), **f32) for _ in range(3))
     seq = torch.zeros((max(S, 1), 3), **f32) if want_seq_sums else None
     st = status_word()
+    ent = torch.full((max(T, 1),), float("nan"), **f32) if want_entropy else None
     if dh_bf16 is None:
         dh_bf16 = lb.bf16
     dH = torch.full((max(T, 1), d), float("nan"), dtype=torch.bfloat16 if dh_bf16 else torch.float32, device="cuda")
@@ -60,10 +61,10 @@ def run_loss(lb, params=None, grad_loss=1.0, dh_bf16=None, want_seq_sums=True, d
     if one_pass:
         ws = ws_bytes(B.WS_LOSS_FWD_BWD, T=T, d=d, V=V, B=S)
         B.spo_loss_fwd_bwd(H, W, y, lo, mask, cu, an, grad_loss, loss, logp, lse, coef, seq, dH[:T], dW, acc, ws,
-                           params, st)
+                           params, st, entropy=ent)
     else:
         wsf = ws_bytes(B.WS_LOSS_FWD, T=T, d=d, V=V, B=S)
-        B.spo_loss_fwd(H, W, y, lo, mask, cu, an, loss, logp, lse, coef, seq, wsf, params, st)
+        B.spo_loss_fwd(H, W, y, lo, mask, cu, an, loss, logp, lse, coef, seq, wsf, params, st, entropy=ent)
         wsb = ws_bytes(B.WS_LOSS_BWD, T=T, d=d, V=V)
         B.spo_loss_bwd(H, W, y, lse, coef, grad_loss, dH, dW, acc, wsb, params, st)
     torch.cuda.synchronize()
@@ -71,6 +72,7 @@ def run_loss(lb, params=None, grad_loss=1.0, dh_bf16=None, want_seq_sums=True, d
         "loss": float(loss[0].item()), "logp": logp[:T].cpu().numpy(), "lse": lse[:T].cpu().numpy(),
         "coef": coef[:T].cpu().numpy(), "seq_sums": None if seq is None else seq[:S].cpu().numpy(),
         "dH": dH[:T].float().cpu().numpy(), "dW": dW.cpu().numpy(), "status": int(st[0].item()),
+        "entropy": None if ent is None else ent[:T].cpu().numpy(),
     }
 
 

@@ -80,7 +80,7 @@ def test_null_and_bad_arguments_are_rejected_on_the_host(lib):
     bad = B.default_params(rho_min=0.99, rho_max=0.9)
     assert lib.spo_tracker_update(fake, 10, fake, fake, fake, 0, 4, ctypes.byref(bad), None, None) == B.ERR_INVALID_ARG
     # loss: dtype, shape and alignment checks come before any device work
-    args_tail = (fake, fake, fake, fake, fake, fake, 1 << 30, ref, None, None)
+    args_tail = (fake, fake, fake, fake, fake, None, fake, 1 << 30, ref, None, None)
     assert lib.spo_loss_fwd(fake, fake, 7, fake, fake, None, fake, fake, 8, 64, 100, 1, *args_tail) == B.ERR_UNSUPPORTED_DTYPE
     assert lib.spo_loss_fwd(fake, fake, B.DTYPE_BF16, fake, fake, None, fake, fake, 8, 72, 100, 1, *args_tail) == B.ERR_BAD_SHAPE
     assert lib.spo_loss_fwd(odd, fake, B.DTYPE_BF16, fake, fake, None, fake, fake, 8, 64, 100, 1, *args_tail) == B.ERR_BAD_ALIGNMENT

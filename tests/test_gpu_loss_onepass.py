@@ -267,3 +267,31 @@ def test_unmasked_rows_only_with_everything_masked():
     assert len(got["rows"]) == 0 and got["loss"] == 0.0 and got["status"] == 0
     for k in ("logp", "lse", "coef", "dH", "dW", "seq_sums"):
         assert np.all(got[k] == 0.0), k
+
+
+@pytest.mark.parametrize("bf16,one_pass", [(True, True), (True, False), (False, False), (False, True)])
+def test_policy_entropy_output(bf16, one_pass):
+    """The optional per-token entropy of the softmax, accumulated in the contraction's epilogue:
+    equal to the oracle's -sum p log p, on both loss paths and element types, over several chunks
+    and a ragged vocabulary; asking for it changes no other output."""
+    lengths = [5000, 4100, 897] if bf16 else [40, 25, 1]
+    d, v = (128, 1211) if bf16 else (32, 257)
+    lb = inputs.loss_batch(180, lengths, d, v, 0.3, bf16, 0.1, target="softmax", mask_p=0.1)
+    want = oracle_loss(lb)
+    assert want["entropy"].min() < 0.5 * np.log(v) and want["entropy"].max() > 0.5      # a spread of peaked and flat rows
+    got = run_loss(lb, one_pass=one_pass, want_entropy=True)
+    tol = 2e-3 if bf16 else 1e-4
+    np.testing.assert_allclose(got["entropy"], want["entropy"], rtol=0, atol=tol)
+    plain = run_loss(lb, one_pass=one_pass)
+    assert plain["entropy"] is None and plain["loss"] == got["loss"]
+    for k in ("logp", "lse", "coef"):
+        np.testing.assert_array_equal(plain[k], got[k])
+    assert rel_fro(got["dH"], plain["dH"]) <= 1e-6 and rel_fro(got["dW"], plain["dW"]) <= 1e-6
+
+
+def test_policy_entropy_of_uniform_logits_is_log_v():
+    lb = inputs.loss_batch(181, [50, 78], 64, 300, 0.05, True, 0.05, target="uniform")
+    lb.w[:] = 0.0
+    for one_pass in (False, True):
+        got = run_loss(lb, one_pass=one_pass, want_entropy=True)
+        np.testing.assert_allclose(got["entropy"], np.log(300.0), atol=1e-5)

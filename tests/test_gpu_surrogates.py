@@ -69,6 +69,6 @@ def test_gspo_is_refused_by_the_one_pass_call_for_bf16():
     p = _params(surrogate=B.SUR_GSPO)
     fake = ctypes.c_void_p(0x1000)
     rc = B.lib().spo_loss_fwd_bwd(fake, fake, B.DTYPE_BF16, fake, fake, None, fake, fake, 8, 64, 100, 1, 1.0, fake, fake,
-                                  fake, fake, None, fake, B.DTYPE_BF16, fake, 0, fake, 1 << 40, ctypes.byref(p), None, None)
+                                  fake, fake, None, None, fake, B.DTYPE_BF16, fake, 0, fake, 1 << 40, ctypes.byref(p), None, None)
     assert rc == B.ERR_INVALID_ARG
     assert torch.cuda.is_available()
