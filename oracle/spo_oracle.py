@@ -6,10 +6,12 @@ with the CUDA path, imports nothing from it, and must never be called from the
 product path (only from tests, the smoke check and the CPU-baseline leg of the
 benchmark).
 
-Everything is numpy float64 unless a function name ends in ``_f32``: those
-restate, in IEEE fp32 as a fixed sequence of individually rounded operations, the few
-places where floating point decides an integer (the quantised sampling
-weights), so that both sides take that decision in the same precision.
+Everything is numpy float64.  Where floating point decides an integer (the
+sampled prompt ids) the decision itself is taken on integers: the selector
+(``sample_prompts``) receives the fp32 sampling weights as an input and
+quantises them exactly, so "bit-exact ids given the same uniforms and weights"
+needs no floating-point agreement beyond the weights themselves, which are
+checked against ``sampling_weights`` (the float64 definition) separately.
 
 Pinned by tests/test_oracle_pins.py against closed forms, brute force, finite
 differences and the constants the paper prints.  Pieces whose parameters the
@@ -128,6 +130,14 @@ def normalise_advantages(a, ddof=0, eps=1e-8):
     return (a - mu) / (sigma + eps), float(mu), sigma
 
 
+def near_zero_counts(a_raw, taus=(1e-4, 0.02)):
+    """How many raw advantages satisfy |A| <= tau, for each tolerance (Sec. 4, "Signal Efficiency
+    and Information Loss": the share of near-zero advantages is tracked on the unnormalised
+    advantages at tau = 1e-4 and tau = 0.02)."""
+    a = np.abs(np.asarray(a_raw, dtype=np.float64))
+    return [int((a <= float(t)).sum()) for t in taus]
+
+
 # --------------------------------------------------------------------------
 # Sec. 3.3 -- prioritised sampling
 # --------------------------------------------------------------------------
@@ -136,47 +146,6 @@ def sampling_weights(alpha, beta, eps_explore=EPS_EXPLORE):
     """w = sqrt(v(1-v)) + eps (Eq. "sampling_coef"), unnormalised."""
     v = value_estimate(alpha, beta)
     return np.sqrt(v * (1.0 - v)) + float(eps_explore)
-
-
-def sampling_weights_f32(alpha32, beta32, eps_explore=EPS_EXPLORE):
-    """The same weights in IEEE fp32 as a fixed sequence of individually rounded operations.
-
-    v(1-v) is formed as alpha*beta/(alpha+beta)^2, the same quantity without the
-    cancellation of 1-v near v = 1, and its square root as t/sqrt(t n^2):
-        n = alpha+beta; t = alpha*beta; den = n*n; x = t*den
-        2^-100 <= x <= 2^100 and alpha > 0 (every entry with both parameters positive that a tracker produces):
-            y0 = float32 with the bits 0x5f3759df - (bits(x) >> 1)      (reciprocal-square-root seed)
-            three Newton steps  y <- y * (1.5 - (0.5*x) * (y*y))
-            s = t * y
-        n == 0: s = 0.5;   alpha or beta zero with n > 0: s = 0
-        any other magnitude: s = sqrt((alpha/n) * (beta/n))
-        w = s + eps
-    numpy's float32 add, subtract, multiply, divide and sqrt are each correctly rounded and
-    nothing here is fused, so any IEEE implementation that performs these steps in this order
-    gives the same bits.  (This order of operations is this implementation's own choice for
-    Eq. "sampling_coef"; the pins hold it to the float64 definition.)
-    """
-    f = np.float32
-    a = np.asarray(alpha32, dtype=np.float32)
-    b = np.asarray(beta32, dtype=np.float32)
-    with np.errstate(all="ignore"):
-        n = a + b
-        t = a * b
-        den = n * n
-        x = t * den
-        h = f(0.5) * x
-        y = (np.uint32(0x5F3759DF) - (x.view(np.uint32) >> np.uint32(1))).view(np.float32)
-        for _ in range(3):
-            y = y * (f(1.5) - h * (y * y))
-        s = t * y
-        common = (x >= f(2.0 ** -100)) & (x <= f(2.0 ** 100)) & (a > f(0.0))
-        empty = n == f(0.0)
-        one_zero = (np.minimum(a, b) == f(0.0)) & (n > f(0.0))
-        n_safe = np.where(n > f(0.0), n, f(1.0))
-        rare = np.sqrt((a / n_safe) * (b / n_safe))
-        s = np.where(common, s, np.where(empty, f(0.5), np.where(one_zero, f(0.0), rare))).astype(np.float32)
-        w = s + f(eps_explore)
-    return w.astype(np.float32)
 
 
 def quantise_weights(w32):
@@ -272,7 +241,8 @@ SUR_GSPO = 2            # PPO-Clip on one sequence-level ratio per response
 
 
 def loss_forward(h, w, y, logp_old, mask, cu_seqlens, a_norm,
-                 clip_lo=CLIP_LO, clip_hi=CLIP_HI, agg_mode=AGG_TOKEN_MEAN, surrogate=SUR_PPO_CLIP):
+                 clip_lo=CLIP_LO, clip_hi=CLIP_HI, agg_mode=AGG_TOKEN_MEAN, surrogate=SUR_PPO_CLIP,
+                 dual_clip=None):
     """Token-level PPO-Clip surrogate of Sec. 3.2 with Clip-Higher bounds.
 
     Per token t (row of ``h``): z = W h_t; lse = log sum_v exp(z_v);
@@ -296,6 +266,12 @@ def loss_forward(h, w, y, logp_old, mask, cu_seqlens, a_norm,
                  d loss / d logp_t = -(1/S_act) * a_i * r_i * [unclipped_i] / n_i.
                  ``ratio``, ``surrogate`` and ``unclipped`` then hold each
                  token's response-level value.
+
+    ``dual_clip`` = c > 1 adds the second clip of dual-clip PPO (not in the paper; a variant
+    of its objective in the published form): for a negative advantage the term becomes
+    max(min(ratio*a, clip(ratio)*a), c*a), which stops the gradient once ratio > c (the
+    term is then the constant c*a); non-negative advantages are untouched.  It applies to
+    SUR_PPO_CLIP (per token) and SUR_GSPO (per response); SUR_CISPO has its own truncation.
 
     Returns a dict: loss, logp[T], lse[T], ratio[T], surrogate[T], unclipped[T]
     (bool: the gradient passes through the ratio), coef[T] = d loss / d logp_t
@@ -337,6 +313,10 @@ def loss_forward(h, w, y, logp_old, mask, cu_seqlens, a_norm,
         a_i = np.asarray(a_norm, dtype=np.float64)[:n_seq]
         term_i = np.minimum(r_i * a_i, np.minimum(np.maximum(r_i, lo_b), hi_b) * a_i)
         pass_i = np.where(a_i >= 0.0, r_i <= hi_b, r_i >= lo_b)
+        if dual_clip is not None:
+            neg = a_i < 0.0
+            term_i = np.where(neg, np.maximum(term_i, float(dual_clip) * a_i), term_i)
+            pass_i = pass_i & ~(neg & (r_i > float(dual_clip)))
         loss = -(term_i[live].sum() / s_act) if s_act > 0 else 0.0
         ratio = r_i[seq]
         surrogate_t = term_i[seq]
@@ -358,6 +338,12 @@ def loss_forward(h, w, y, logp_old, mask, cu_seqlens, a_norm,
             # ratio is on the inside of the bound that matters for the sign of a;
             # the boundary itself counts as inside.
             unclipped = np.where(a >= 0.0, ratio <= hi_b, ratio >= lo_b)
+            if dual_clip is not None:
+                # second clip for negative advantages: the term may not fall below c*a, and once
+                # ratio > c it is that constant (ratio == c counts as inside, like the other bounds)
+                neg = a < 0.0
+                surrogate_t = np.where(neg, np.maximum(surrogate_t, float(dual_clip) * a), surrogate_t)
+                unclipped = unclipped & ~(neg & (ratio > float(dual_clip)))
             coef = -(u * a * ratio * unclipped)
         else:
             raise ValueError("surrogate")
@@ -369,12 +355,13 @@ def loss_forward(h, w, y, logp_old, mask, cu_seqlens, a_norm,
     }
 
 
-def loss_stats(logp, logp_old, mask, cu_seqlens, a_norm, clip_lo=CLIP_LO, clip_hi=CLIP_HI):
+def loss_stats(logp, logp_old, mask, cu_seqlens, a_norm, clip_lo=CLIP_LO, clip_hi=CLIP_HI, dual_clip=None):
     """Per-step diagnostics of the policy update over the unmasked tokens (the quantities the
     paper's training curves are read by; none enters the objective):
       [0] n_tok            [1] mean importance ratio
       [2] share of tokens whose gradient the clip stops (ratio beyond the bound that matters
-          for the sign of their advantage; a zero advantage counts as not clipped)
+          for the sign of their advantage, or beyond ``dual_clip`` for a negative one; a zero
+          advantage counts as not clipped)
       [3] mean of logp_old - logp            (the plain sampled estimate of KL(old || new))
       [4] mean of ratio - 1 - log(ratio)     (a non-negative estimate of the same KL)
       [5] largest ratio    [6] smallest ratio
@@ -395,6 +382,8 @@ def loss_stats(logp, logp_old, mask, cu_seqlens, a_norm, clip_lo=CLIP_LO, clip_h
     ratio = np.exp(d)
     lo_b, hi_b = 1.0 - clip_lo, 1.0 + clip_hi
     stopped = np.where(a > 0.0, ratio > hi_b, np.where(a < 0.0, ratio < lo_b, False))
+    if dual_clip is not None:
+        stopped = stopped | ((a < 0.0) & (ratio > float(dual_clip)))
     out[0] = n
     out[1] = ratio.mean()
     out[2] = stopped.mean()
@@ -424,7 +413,7 @@ def loss_backward(h, w, y, lse, coef, grad_loss=1.0):
 
 
 def loss_rows(h_rows, w, y_rows, logp_old_rows, mask_rows, a_rows, n_tok,
-              clip_lo=CLIP_LO, clip_hi=CLIP_HI, grad_loss=1.0, v_chunk=8192):
+              clip_lo=CLIP_LO, clip_hi=CLIP_HI, grad_loss=1.0, v_chunk=8192, want_dw=False):
     """Row-local outputs for a handful of token rows of a large problem.
 
     Every per-token output of loss_forward and the dH row of loss_backward
@@ -432,7 +421,9 @@ def loss_rows(h_rows, w, y_rows, logp_old_rows, mask_rows, a_rows, n_tok,
     (the advantage of its sequence, n_tok).  This evaluates exactly those
     formulas for the given rows, streaming W in chunks of ``v_chunk`` rows so
     that W never has to exist in float64 at once.  Returns dict(logp, lse,
-    ratio, coef, dH).
+    ratio, coef, dH); with ``want_dw`` also dW = g^T H of these rows alone: dW of
+    the whole batch is the sum of its tokens' terms, so the contributions of a
+    partition of the rows add up to loss_backward's dW.
     """
     h = np.asarray(h_rows, dtype=np.float64)
     n, d = h.shape
@@ -457,4 +448,7 @@ def loss_rows(h_rows, w, y_rows, logp_old_rows, mask_rows, a_rows, n_tok,
     for v0 in range(0, v_total, v_chunk):
         wc = np.asarray(w[v0:v0 + v_chunk], dtype=np.float64)
         dh += g[:, v0:v0 + wc.shape[0]] @ wc
-    return {"logp": logp, "lse": lse, "ratio": ratio, "coef": coef, "dH": dh}
+    out = {"logp": logp, "lse": lse, "ratio": ratio, "coef": coef, "dH": dh}
+    if want_dw:
+        out["dW"] = g.T @ h
+    return out

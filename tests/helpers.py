@@ -10,6 +10,27 @@ def rel_fro(got, want):
     return np.linalg.norm(got - want) / (den if den > 0 else 1.0)
 
 
+def worst_row_tile_error(got, want, tile=256, floor_share=0.05):
+    """Largest relative Frobenius error over consecutive row tiles of a matrix (a whole-matrix norm
+    hides one wrong tile among hundreds).  Tiles whose reference norm is below floor_share x the
+    median tile norm carry (almost) no signal and are left out.  Returns (worst, checked, n_tiles,
+    last_tile_checked)."""
+    got = np.asarray(got, dtype=np.float64)
+    want = np.asarray(want, dtype=np.float64)
+    rows = want.shape[0]
+    n_tiles = -(-rows // tile)
+    norms = np.array([np.linalg.norm(want[i * tile:(i + 1) * tile]) for i in range(n_tiles)])
+    floor = floor_share * np.median(norms)
+    worst, checked = 0.0, 0
+    for i in range(n_tiles):
+        if norms[i] < floor or norms[i] == 0.0:
+            continue
+        sl = slice(i * tile, min((i + 1) * tile, rows))
+        worst = max(worst, np.linalg.norm(got[sl] - want[sl]) / norms[i])
+        checked += 1
+    return worst, checked, n_tiles, bool(norms[-1] >= floor and norms[-1] > 0.0)
+
+
 def dev(x, dtype=None):
     import torch
     t = torch.from_numpy(np.ascontiguousarray(x)).cuda()

@@ -175,6 +175,17 @@ def test_normalisation_affine_invariance_and_degenerate_cases():
 
 # ----------------------------------------------------------------- sampling
 
+def test_near_zero_counts_hand_values_and_tolerances_of_the_paper():
+    """Sec. 4 tracks |A| <= tau on the raw advantages at tau = 1e-4 and 0.02; the bound is inclusive."""
+    a = np.array([0.0, 1e-4, -1e-4, 1.0001e-4, 0.02, -0.020001, 0.5, -0.7])
+    assert O.near_zero_counts(a) == [3, 5]
+    assert O.near_zero_counts(a, taus=(0.0, 1.0)) == [1, 8]
+    assert O.near_zero_counts([]) == [0, 0]
+    # a tracker that predicts perfectly leaves every advantage at zero
+    al, be = np.array([8.0, 0.0]), np.array([0.0, 8.0])
+    assert O.near_zero_counts(O.raw_advantage(al, be, [0, 1], [1.0, 0.0])) == [2, 2]
+
+
 def test_weight_range_endpoints():
     eps = paper_constants()["eps_explore"]
     a = np.array([0.0, 8.0, 4.0])
@@ -185,34 +196,6 @@ def test_weight_range_endpoints():
     aa, bb = rng.uniform(0, 10, 1000), rng.uniform(0, 10, 1000)
     ww = O.sampling_weights(aa, bb, eps)
     assert ww.min() >= eps and ww.max() <= 0.5 + eps + 1e-15
-
-
-def test_fp32_weights_track_the_fp64_definition():
-    rng = np.random.default_rng(6)
-    a = rng.uniform(0, 20, 5000).astype(np.float32)
-    b = rng.uniform(0, 20, 5000).astype(np.float32)
-    a[:3], b[:3] = [0, 0, 5], [0, 5, 0]
-    w32 = O.sampling_weights_f32(a, b)
-    assert w32.dtype == np.float32
-    np.testing.assert_allclose(w32, O.sampling_weights(a, b), rtol=2e-6, atol=1e-7)
-    assert w32[0] == np.float32(0.55)
-
-
-def test_fp32_weights_uncommon_magnitudes_track_the_fp64_definition():
-    """Entries outside the range the Newton sequence serves (empty, a zero parameter, tiny, huge)
-    take the division / square-root branch; every branch stays within 1e-6 of the definition."""
-    a = np.array([0, 0, 5, 1e-30, 1, 1e-20, 1e25, 3e5, 2.0 ** -21, 1e-39, 1e18, 1e-19], dtype=np.float32)
-    b = np.array([0, 5, 0, 1, 1e-38, 1e-20, 1e25, 7e5, 2.0 ** -21, 1, 3e18, 4e-19], dtype=np.float32)
-    w32 = O.sampling_weights_f32(a, b)
-    want = O.sampling_weights(a.astype(np.float64), b.astype(np.float64))
-    assert np.all(np.isfinite(w32))
-    np.testing.assert_allclose(w32, want, rtol=1e-6)
-    assert w32[0] == np.float32(0.55) and w32[1] == np.float32(0.05) and w32[2] == np.float32(0.05)
-    rng = np.random.default_rng(8)
-    aa = (10.0 ** rng.uniform(-15, 15, 20000)).astype(np.float32)
-    bb = (10.0 ** rng.uniform(-15, 15, 20000)).astype(np.float32)
-    np.testing.assert_allclose(O.sampling_weights_f32(aa, bb),
-                               O.sampling_weights(aa.astype(np.float64), bb.astype(np.float64)), rtol=1e-6)
 
 
 def test_quantised_weights_are_exact_scalings():
@@ -271,7 +254,7 @@ def test_first_draw_frequencies_chi_square():
     n, draws = 64, 100_000
     a = rng.uniform(0, 8, n).astype(np.float32)
     b = rng.uniform(0, 8, n).astype(np.float32)
-    w = O.sampling_weights_f32(a, b)
+    w = O.sampling_weights(a, b).astype(np.float32)         # the selector takes fp32 weights as an input
     u = rng.random(draws).astype(np.float32)
     u = u[u < 1.0]
     counts = np.zeros(n)
@@ -487,6 +470,30 @@ def test_row_local_helper_equals_full_definition():
     np.testing.assert_allclose(sub["lse"], fwd["lse"][rows], atol=1e-13)
     np.testing.assert_allclose(sub["coef"], fwd["coef"][rows], atol=1e-15)
     np.testing.assert_allclose(sub["dH"], dh[rows], atol=1e-14)
+    assert "dW" not in sub
+
+
+def test_row_local_dw_contributions_of_a_partition_add_up_to_the_full_dw():
+    """dW = g^T H is a sum over tokens: the row blocks' contributions must add up to
+    loss_backward's dW (what the multi-chunk parity test at the real vocabulary relies on)."""
+    rng = np.random.default_rng(18)
+    t, d, v = 23, 6, 40
+    h, w = rng.standard_normal((t, d)), rng.standard_normal((v, d))
+    y = rng.integers(0, v, t)
+    cu, a = [0, 9, 23], np.array([0.8, -1.3])
+    mask = (rng.random(t) > 0.2).astype(np.uint8)
+    logp_old = rng.normal(-3.5, 0.3, t)
+    fwd = O.loss_forward(h, w, y, logp_old, mask, cu, a)
+    _, dw = O.loss_backward(h, w, y, fwd["lse"], fwd["coef"], grad_loss=0.7)
+    a_tok = np.repeat(a, np.diff(cu))
+    acc = np.zeros_like(dw)
+    for lo, hi in ((0, 7), (7, 8), (8, 23)):
+        sub = O.loss_rows(h[lo:hi], w, y[lo:hi], logp_old[lo:hi], mask[lo:hi], a_tok[lo:hi], fwd["n_tok"],
+                          grad_loss=0.7, v_chunk=16, want_dw=True)
+        acc += sub["dW"]
+    np.testing.assert_allclose(acc, dw, atol=1e-13)
+    # a transposed operand or a dropped block would not survive this: dW is [V, d], not symmetric
+    assert acc.shape == (v, d)
 
 
 def test_token_to_sequence_map():
@@ -763,3 +770,80 @@ def test_policy_entropy_against_library_and_closed_forms():
     ww[1, 0] = 0.0
     one = O.loss_forward(hh, ww, [0], np.zeros(1), None, [0, 1], a)
     assert 0.0 <= one["entropy"][0] < 1e-20
+
+
+# ------------------------------------------------------ dual clip (second clip for negative advantages)
+
+def test_dual_clip_hand_worked_table():
+    """term = max(min(r a, clip(r) a), c a) for a < 0; untouched for a >= 0.  c = 3, bounds 0.8 / 1.28."""
+    v = 4
+    z = np.zeros((6, v))
+    y = np.zeros(6, dtype=int)
+    base = -math.log(v)                                   # logp of every token
+    ratios = np.array([1.0, 2.0, 2.5, 4.0, 4.0, 0.5])
+    a = np.array([-1.0, -1.0, -1.0, -1.0, 1.0, -1.0])
+    logp_old = base - np.log(ratios)
+    args = _identity_problem(z, y, logp_old, a)
+    plain = O.loss_forward(*args)
+    dual = O.loss_forward(*args, dual_clip=3.0)
+    np.testing.assert_allclose(dual["ratio"], ratios, rtol=1e-14)
+    # plain PPO-Clip terms: a<0: min(r a, clip(r) a) = -max(r, clip(r))
+    np.testing.assert_allclose(plain["surrogate"], [-1.0, -2.0, -2.5, -4.0, 1.28, -0.8], rtol=1e-14)
+    # with the second clip the term is bounded below by c a = -3
+    np.testing.assert_allclose(dual["surrogate"], [-1.0, -2.0, -2.5, -3.0, 1.28, -0.8], rtol=1e-14)
+    assert dual["unclipped"].tolist() == [True, True, True, False, False, False]
+    assert plain["unclipped"].tolist() == [True, True, True, True, False, False]
+    np.testing.assert_allclose(dual["coef"], [1 / 6, 2 / 6, 2.5 / 6, 0.0, 0.0, 0.0], rtol=1e-14)
+    assert abs(dual["loss"] - (-(-1 - 2 - 2.5 - 3 + 1.28 - 0.8) / 6)) < 1e-14
+    # a bound no ratio reaches changes nothing
+    far = O.loss_forward(*args, dual_clip=100.0)
+    assert far["loss"] == plain["loss"] and np.array_equal(far["coef"], plain["coef"])
+
+
+def test_dual_clip_gradients_against_central_finite_differences():
+    rng = np.random.default_rng(61)
+    t, d, v = 6, 5, 9
+    h, w = rng.standard_normal((t, d)), rng.standard_normal((v, d)) * 0.5
+    y = rng.integers(0, v, t)
+    cu, a = [0, 3, 6], np.array([-0.9, 1.1])
+    base = O.loss_forward(h, w, y, np.zeros(t), None, cu, a)
+    # response 0 (a<0): ratios 1.1 (inside), 2.6 (beyond c = 2: constant term), 0.6 (first clip);
+    # response 1 (a>0): 1.1, 2.6 (clipped above), 0.9
+    logp_old = base["logp"] - np.log([1.1, 2.6, 0.6, 1.1, 2.6, 0.9])
+    fwd = O.loss_forward(h, w, y, logp_old, None, cu, a, dual_clip=2.0)
+    assert fwd["unclipped"].tolist() == [True, False, False, True, False, True]
+    dh, dw = O.loss_backward(h, w, y, fwd["lse"], fwd["coef"])
+    step = 1e-6
+    for arr, grad in ((h, dh), (w, dw)):
+        num = np.zeros_like(arr)
+        for idx in np.ndindex(arr.shape):
+            keep = arr[idx]
+            arr[idx] = keep + step
+            up = O.loss_forward(h, w, y, logp_old, None, cu, a, dual_clip=2.0)["loss"]
+            arr[idx] = keep - step
+            dn = O.loss_forward(h, w, y, logp_old, None, cu, a, dual_clip=2.0)["loss"]
+            arr[idx] = keep
+            num[idx] = (up - dn) / (2 * step)
+        assert np.linalg.norm(num - grad) <= 1e-6 * np.linalg.norm(grad)
+    # without the second clip token 1 would carry gradient
+    assert O.loss_forward(h, w, y, logp_old, None, cu, a)["coef"][1] != 0.0 and fwd["coef"][1] == 0.0
+
+
+def test_dual_clip_on_the_sequence_level_objective_and_in_the_diagnostics():
+    rng = np.random.default_rng(62)
+    t, d, v = 8, 4, 7
+    h, w = rng.standard_normal((t, d)), rng.standard_normal((v, d)) * 0.5
+    y = rng.integers(0, v, t)
+    cu, a = [0, 4, 8], np.array([-1.0, -0.5])
+    base = O.loss_forward(h, w, y, np.zeros(t), None, cu, a)
+    shift = np.concatenate([np.full(4, math.log(3.0)), np.full(4, math.log(1.1))])
+    logp_old = base["logp"] - shift                       # response ratios 3.0 and 1.1
+    g = O.loss_forward(h, w, y, logp_old, None, cu, a, surrogate=O.SUR_GSPO, dual_clip=2.0)
+    np.testing.assert_allclose(g["ratio"], np.repeat([3.0, 1.1], 4), rtol=1e-12)
+    assert abs(g["loss"] - (-(2.0 * -1.0 + 1.1 * -0.5) / 2)) < 1e-12      # c a for the first, r a for the second
+    assert np.all(g["coef"][:4] == 0.0) and np.all(g["coef"][4:] != 0.0)
+    # diagnostics: the share of stopped tokens counts the second clip and equals the zero-coef share
+    tok = O.loss_forward(h, w, y, logp_old, None, cu, a, dual_clip=2.0)
+    st = O.loss_stats(tok["logp"], logp_old, None, cu, a, dual_clip=2.0)
+    assert abs(st[2] - (tok["coef"] == 0.0).mean()) < 1e-15 and st[2] == 0.5
+    assert O.loss_stats(tok["logp"], logp_old, None, cu, a)[2] == 0.0
