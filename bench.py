@@ -149,7 +149,7 @@ class Step:
         self.params = B.default_params()
         self.ids = torch.empty(self.S, dtype=torch.int32, device=device)
         self.a_norm = torch.empty(self.S, **f32)
-        self.stats = torch.empty(4, **f32)
+        self.stats = torch.empty(8, **f32)
         self.loss = torch.zeros(4, **f32)
         self.logp, self.lse, self.coef = (torch.empty(self.T, **f32) for _ in range(3))
         self.entropy = torch.empty(self.T, **f32) if entropy else None      # optional per-token policy entropy
@@ -177,34 +177,34 @@ class Step:
                 self.ws_bwd = torch.empty(self.ws_bwd_bytes, **u8)
         chunk_rows = self.ws_bwd_bytes // (((V + 255) // 256) * 256 * 2)
         self.bwd_chunks = -(-self.T // chunk_rows)
-        # kernels launched by one step: sampling 3 (tile sums, search, accept), advantages 1, update 1, then
+        # kernels launched by one step: sampling 3 (tile sums, search, accept), advantages + update 1, then
         # split path: forward 3 (count, contraction, finalise), backward 3 per chunk;
-        # one-pass path: count 1, per chunk 4 (logits contraction [+ e->g of the chunk before on side warps],
-        # finalise, dH, dW), and one e->g kernel for the last chunk.  Memsets are not counted.
+        # one-pass path: count 1, first-tile pass 1, per chunk 4 (logits contraction, finalise, row scaling
+        # of H, dH) and one dW contraction per pair of chunks.  Memsets are not counted.
         self.flops_fwd = 2.0 * self.T * d * V
         chunks_act = -(-self.n_tok // chunk_rows)          # chunks of the compacted batch (masked workloads)
         if self.onepass and self.mask_frac > 0.0:
             # row list 3, gather 1, boundaries 1, one-pass on the compacted batch, two scatters
-            self.launches = 3 + 1 + 1 + 3 + 1 + 1 + (1 + 4 * chunks_act + 1) + 2
+            self.launches = 3 + 1 + 3 + 1 + 1 + (2 + 4 * chunks_act + -(-chunks_act // 2)) + 2
             self.flops_fwd = 2.0 * self.n_tok * d * V
             self.flops_bwd = 4.0 * self.n_tok * d * V
         elif self.onepass:
-            self.launches = 3 + 1 + 1 + 1 + 4 * self.bwd_chunks + 1
+            self.launches = 3 + 1 + 2 + 4 * self.bwd_chunks + -(-self.bwd_chunks // 2)
             self.flops_bwd = 4.0 * self.T * d * V
         elif self.mask_frac > 0.0:
             # forward over all rows; row list 3, gather 1, backward on the rows with gradient, scatter 1
-            self.launches = 3 + 1 + 1 + 3 + 3 + 1 + 3 * chunks_act + 1
+            self.launches = 3 + 1 + 3 + 3 + 1 + 3 * chunks_act + 1
             self.flops_bwd = 6.0 * self.n_tok * d * V
         else:
-            self.launches = 3 + 1 + 1 + 3 + 3 * self.bwd_chunks
+            self.launches = 3 + 1 + 3 + 3 * self.bwd_chunks
             self.flops_bwd = 6.0 * self.T * d * V
 
     def small(self):
         B = self.B
         B.spo_sample_prompts(self.ab, self.uniforms, self.S, self.ids, None, self.ws_sample, self.params, self.status)
-        B.spo_advantages(self.ab, self.ids, self.rewards, None, self.a_norm, self.stats, self.ws_adv, self.params,
-                         self.status)
-        B.spo_tracker_update(self.ab, self.ids, self.rewards, self.kl_table, 1, self.params, self.status)
+        # raw advantage (pre-update baseline), tracker update and normalisation in one pass over the entries
+        B.spo_advantages_update(self.ab, self.ids, self.rewards, self.kl_table, 1, None, self.a_norm, self.stats,
+                                self.ws_adv, self.params, self.status)
 
     def fwd(self, h=None, y=None, logp_old=None, mask=None, cu=None):
         D = self.data
@@ -440,7 +440,7 @@ def run_small_kernels(args, local_rank):
     n_draw = min(4096, Bn)
     out_ids = torch.empty(n_draw, dtype=torch.int32, device=dev)
     a_norm = torch.empty(Bn, device=dev)
-    stats = torch.empty(4, device=dev)
+    stats = torch.empty(8, device=dev)
     st = torch.zeros(4, dtype=torch.int32, device=dev)
     ws = torch.empty(B.spo_workspace_bytes(B.WS_SAMPLE, N=N, M=M), dtype=torch.uint8, device=dev)
     wsa = torch.empty(B.spo_workspace_bytes(B.WS_ADVANTAGES, B=Bn), dtype=torch.uint8, device=dev)

@@ -63,8 +63,8 @@ extern "C" {
  *             (no gradient through the weight): coef_t = -u_t w_t a for every unmasked token
  *   GSPO      one ratio per response, r_i = exp(mean over its unmasked tokens of logp_t - logp_old_t);
  *             (1/S_act) sum_i min(r_i a_i, clip(r_i) a_i); coef_t = -a_i r_i [unclipped_i] / (S_act n_i);
- *             agg_mode does not apply.  Needs every token of a response before any coef exists, so it
- *             runs in the two-call path only (spo_loss_fwd, spo_loss_bwd) */
+ *             agg_mode does not apply.  Needs every token of a response before any coef exists, so
+ *             spo_loss_fwd_bwd runs it as forward-then-backward (see there) */
 #define SPO_SUR_PPO_CLIP  0
 #define SPO_SUR_CISPO     1
 #define SPO_SUR_GSPO      2
@@ -102,6 +102,15 @@ typedef struct spo_params {
   int32_t global_tokens;     /* unmasked tokens of the whole mini-batch (n_tok) */
   int32_t global_responses;  /* responses with an unmasked token in the whole mini-batch (S_act) */
   int32_t surrogate;         /* SPO_SUR_*: which objective the loss calls evaluate */
+  /* Second clip of dual-clip PPO (not in the paper; 0 = off, the default).  With c = dual_clip > 1 a
+   * negative advantage's term becomes max(min(ratio a, clip(ratio) a), c a): once ratio > c the term
+   * is the constant c a and carries no gradient.  Applies to SPO_SUR_PPO_CLIP (per token) and
+   * SPO_SUR_GSPO (per response); SPO_SUR_CISPO has its own truncation and ignores it. */
+  float   dual_clip;
+  /* Tolerances of the near-zero-advantage counts (Sec. 4, signal efficiency: the share of raw
+   * advantages with |A| <= tau, tracked at tau = 1e-4 and tau = 0.02). */
+  float   near_zero_tau_lo;  /* 1e-4 */
+  float   near_zero_tau_hi;  /* 0.02 */
 } spo_params;
 
 int32_t spo_default_params(spo_params* p /* host, out */);
@@ -155,10 +164,13 @@ int32_t spo_sample_prompts(const float* ab, int64_t N, const float* uniforms, in
  *   r       device in  [B] fp32 rewards
  *   a_raw   device out [B] fp32, optional
  *   a_norm  device out [B] fp32
- *   stats   device out [4] fp32 = (mu, sigma, B, M2 = sum (A-mu)^2), optional; (mu, M2, B) of
- *           several ranks merge exactly (pairwise: M2 = M2a + M2b + (mub-mua)^2 Ba Bb/(Ba+Bb))
+ *   stats   device out [8] fp32 = (mu, sigma, B, M2 = sum (A-mu)^2, n_lo, n_hi, 0, 0), optional;
+ *           n_lo / n_hi = how many raw advantages satisfy |A| <= near_zero_tau_lo / _hi (Sec. 4,
+ *           signal efficiency; counts are exact up to 2^24).  (mu, M2, B) of several ranks merge
+ *           exactly (pairwise: M2 = M2a + M2b + (mub-mua)^2 Ba Bb/(Ba+Bb)); the counts add.
  *   ws      device scratch, spo_workspace_bytes(SPO_WS_ADVANTAGES, ..., B, ...) bytes
- * An id outside [0,N) sets SPO_DEV_ID_OUT_OF_RANGE and contributes A = 0.
+ * An id outside [0,N) sets SPO_DEV_ID_OUT_OF_RANGE and contributes A = 0; a negative or non-finite
+ * table entry sets SPO_DEV_NONFINITE and contributes A = 0 as well.
  */
 int32_t spo_advantages(const float* ab, int64_t N, const int32_t* ids, const float* r, int32_t B,
                        float* a_raw, float* a_norm, float* stats, void* ws, size_t ws_bytes,
@@ -185,7 +197,7 @@ int32_t spo_advantages_apply(const float* a_raw, int32_t B, float mu, float sigm
  * synchronise the device or fail outright.  Such a caller cannot produce the `ws`
  * buffer that spo_advantages asks for large batches.
  *
- * Here the block partials of the two-pass path live in a fixed 16 KB array inside the
+ * Here the block partials of the two-pass path live in a fixed 32 KB array inside the
  * library's device image (each GPU that loads the library holds it until the process
  * exits).  Consequences the caller must know:
  *   - B may not exceed SPO_ADVANTAGES_STATIC_MAX_B; a larger B returns SPO_ERR_BAD_SHAPE
@@ -217,6 +229,21 @@ int32_t spo_advantages_static(const float* ab, int64_t N, const int32_t* ids, co
 int32_t spo_tracker_update(float* ab, int64_t N, const int32_t* ids, const float* r, const float* kl,
                            int32_t kl_is_table, int32_t B,
                            const spo_params* params, int32_t* d_status, void* stream);
+
+/*
+ * spo_advantages and spo_tracker_update for the same batch in one pass over the table (Algorithm 1:
+ * "Compute raw advantage", "Update tracker", "Normalize advantages"): every entry ids[j] is read
+ * once, A_j = r_j - v(ids_j) is formed from the value as read (the pre-update baseline of Sec. 3.2),
+ * the entry is updated in place from that same value (Sec. 3.1) and the batch statistics and
+ * normalised advantages follow as in spo_advantages.  Results equal the two calls made in the
+ * paper's order; the table entry crosses the memory system once per step instead of twice.
+ * ids must be distinct (as for spo_tracker_update).  Arguments, scratch size (SPO_WS_ADVANTAGES)
+ * and status bits as in the two calls; an element with a bad id, table entry or reward contributes
+ * A = 0 and leaves its entry untouched, a NaN divergence leaves the entry untouched.
+ */
+int32_t spo_advantages_update(float* ab, int64_t N, const int32_t* ids, const float* r, const float* kl,
+                              int32_t kl_is_table, int32_t B, float* a_raw, float* a_norm, float* stats,
+                              void* ws, size_t ws_bytes, const spo_params* params, int32_t* d_status, void* stream);
 
 /*
  * Tracker update for batch SPO (appendix "Batch Extensions": every prompt rolled out G times per
@@ -265,7 +292,8 @@ int32_t spo_tracker_update_repeats(float* ab, int64_t N, const int32_t* ids, con
  *               per logit to the contraction's epilogue; NULL costs nothing.
  *   ws          device scratch, spo_workspace_bytes(SPO_WS_LOSS_FWD, T, d, V, 0, S, 0) bytes
  *               (the B argument of that query carries the number of responses S)
- * A target outside [0,V) sets SPO_DEV_ID_OUT_OF_RANGE (the row gets logp = -inf, coef = 0).
+ * A target outside [0,V) gives the row logp = -inf and coef = 0; it sets SPO_DEV_ID_OUT_OF_RANGE unless
+ * the row is masked out (masked rows may carry an ignore-index target such as -100).
  */
 int32_t spo_loss_fwd(const void* H, const void* W, int32_t dtype,
                      const int32_t* y, const float* logp_old, const uint8_t* mask,
@@ -300,23 +328,30 @@ int32_t spo_loss_bwd(const void* H, const void* W, int32_t dtype, const int32_t*
  * node of the training graph, so its upstream gradient (`grad_loss`, e.g. 1 or a loss scale) is
  * known before the forward runs; that is what lets the two halves share their logits.
  *
- * bf16: token rows are processed in chunks (the chunk of spo_loss_bwd).  The logits of a chunk
- * are contracted once; the epilogue keeps the online (max, sum-exp, target logit) of every row and
- * also stores each logit as e = 2^(z log2(e) - ref), bf16, with one fp32 reference exponent `ref`
- * per row and 64 columns (that group's largest logit, so e <= 1 and its relative error is bf16's
- * whatever the range of the logits).  After the chunk's rows are finalised (lse, coef), a streaming
- * kernel rewrites the buffer in place as g = grad_loss coef_t (1[v = y_t] - e 2^(ref - lse_t log2(e)))
- * and dH, dW follow as in spo_loss_bwd.  loss, logp, lse and coef never see the bf16 rounding of e;
- * dH and dW carry it in place of spo_loss_bwd's own bf16 rounding of g (same size).
+ * bf16: token rows are processed in chunks (the chunk of spo_loss_bwd).  A short launch first
+ * contracts every row with the first 512 vocabulary rows; the largest of those logits plus 40 binary
+ * orders is the row's reference exponent ref_t.  The logits of a chunk are then contracted once; the
+ * epilogue sums e = 2^(z log2(e) - ref_t) over the row (no running maximum is needed: fp32 and bf16
+ * keep their relative precision at any magnitude) and stores every e as bf16.  With l_t = sum_v e the
+ * softmax is e / l_t, so lse_t = (ref_t + log2 l_t) ln 2 and the logit gradient factors as
+ *   g[t,v] = rowscale_t (e[t,v] - l_t 1[v = y_t]),   rowscale_t = -grad_loss coef_t / l_t:
+ * after the chunk's rows are finalised the one target entry per row is patched in the stored chunk,
+ * dH = rowscale (e W) takes the factor in its epilogue and dW = e^T (rowscale H) reads a scaled bf16
+ * copy of the chunk's rows of H; the stored chunk is never rewritten.  dW is contracted over two
+ * chunks at a time.  loss, logp, lse and coef never see the bf16 rounding of e; dH and dW carry it
+ * (and dW the rounding of rowscale H) in place of spo_loss_bwd's own bf16 rounding of g.
+ * Range: a row whose largest logit exceeds the largest of its first 512 by more than 100 nats
+ * overflows the stored exponentials; such a row sets SPO_DEV_NONFINITE, gets lse = Inf, logp = -Inf,
+ * coef = 0 and takes no part in the gradients (use the two calls for such inputs).
  * fp32: the two SIMT halves run back to back (nothing to share).
  *
  *   arguments   as in spo_loss_fwd and spo_loss_bwd; lse and coef are outputs here.
- *               SPO_SUR_GSPO with bf16 inputs returns SPO_ERR_INVALID_ARG (a response's ratio needs all
- *               its tokens, which may lie in later chunks): use the two calls.
+ *               SPO_SUR_GSPO with bf16 inputs: a response's ratio needs the log-probs of all its tokens,
+ *               which may lie in later chunks, so the call runs the forward to the end and then the
+ *               chunked backward (four contractions, the cost of the two calls).
  *   ws          device scratch, spo_workspace_bytes(SPO_WS_LOSS_FWD_BWD, T, d, V, 0, S, 0) bytes:
- *               two chunk buffers when T exceeds one chunk (the chunks are software-pipelined: the
- *               e -> g pass of one chunk runs on spare warps of the next chunk's logits contraction),
- *               their reference exponents (1/32 of them) and the forward's partials
+ *               two chunk buffers when T exceeds one chunk, scaled copies of their rows of H, 36 bytes
+ *               per token row and the forward's partials
  * Status bits as spo_loss_fwd.
  */
 int32_t spo_loss_fwd_bwd(const void* H, const void* W, int32_t dtype,
@@ -327,6 +362,35 @@ int32_t spo_loss_fwd_bwd(const void* H, const void* W, int32_t dtype,
                          void* dH, int32_t dH_dtype, float* dW, int32_t dW_accumulate,
                          void* ws, size_t ws_bytes,
                          const spo_params* params, int32_t* d_status, void* stream);
+
+/*
+ * spo_loss_fwd_bwd for data-parallel ranks (Algorithm 1's mini-batch update spread over several GPUs:
+ * every rank holds part of the responses, W is replicated, and the ranks' dW must be summed).  dW is
+ * only final once its last contraction has run; this variant cuts that last launch into slabs of
+ * vocabulary rows and records a CUDA event behind each, so that the caller can start reducing slab k
+ * over the ranks on another stream (wait for events[k], then all-reduce rows row_begin[k] ..
+ * row_begin[k+1]-1 of dW) while slab k+1 is still being contracted; only the last slab's reduction is
+ * left exposed.  Results are those of spo_loss_fwd_bwd, bit for bit.
+ *
+ *   spo_dw_slab_rows   host only: writes row_begin[0..n] (row_begin[0] = 0, row_begin[n] = V) for a
+ *                      request of n_wanted slabs (1 .. SPO_MAX_DW_SLABS) and returns n <= n_wanted
+ *                      (slabs hold whole rounds of row tiles), or a negative status.
+ *   events             host array of n_wanted cudaEvent_t (created by the caller, e.g. with timing
+ *                      disabled); events[0..n) are recorded on `stream`.  Inputs for which the last
+ *                      contraction is not cut (fp32, SPO_SUR_GSPO, T = 0) record them all at the end.
+ * All other arguments as in spo_loss_fwd_bwd.  The library creates, waits on and destroys nothing.
+ */
+#define SPO_MAX_DW_SLABS 64
+int32_t spo_dw_slab_rows(int32_t V, int32_t d, int32_t n_wanted, int64_t* row_begin /* host, [n_wanted+1] */);
+int32_t spo_loss_fwd_bwd_slabs(const void* H, const void* W, int32_t dtype,
+                               const int32_t* y, const float* logp_old, const uint8_t* mask,
+                               const int32_t* cu_seqlens, const float* a_norm,
+                               int64_t T, int32_t d, int32_t V, int32_t S, float grad_loss,
+                               float* loss, float* logp, float* lse, float* coef, float* seq_sums, float* entropy,
+                               void* dH, int32_t dH_dtype, float* dW, int32_t dW_accumulate,
+                               void* ws, size_t ws_bytes,
+                               const spo_params* params, int32_t* d_status, void* stream,
+                               int32_t n_wanted, void* const* events /* host, [n_wanted] */);
 
 /*
  * Diagnostic (no counterpart in the paper): runs the kernels' bounded mbarrier wait on a barrier

@@ -27,8 +27,8 @@ SUR_PPO_CLIP, SUR_CISPO, SUR_GSPO = 0, 1, 2
 
 EXPORTS = [
     "spo_default_params", "spo_tracker_init", "spo_sample_prompts", "spo_advantages",
-    "spo_advantages_static", "spo_advantages_apply",
-    "spo_tracker_update", "spo_tracker_update_repeats", "spo_loss_fwd", "spo_loss_bwd", "spo_loss_fwd_bwd", "spo_loss_stats", "spo_loss_mask_rows", "spo_loss_fwd_bwd_rows", "spo_loss_active_rows", "spo_loss_bwd_rows", "spo_workspace_bytes",
+    "spo_advantages_static", "spo_advantages_apply", "spo_advantages_update",
+    "spo_tracker_update", "spo_tracker_update_repeats", "spo_loss_fwd", "spo_loss_bwd", "spo_loss_fwd_bwd", "spo_loss_fwd_bwd_slabs", "spo_dw_slab_rows", "spo_loss_stats", "spo_loss_mask_rows", "spo_loss_fwd_bwd_rows", "spo_loss_active_rows", "spo_loss_bwd_rows", "spo_workspace_bytes",
     "spo_status_string", "spo_last_cuda_error", "spo_version", "spo_selftest_bounded_wait",
 ]
 
@@ -38,7 +38,8 @@ class SpoParams(Structure):
         ("rho_min", c_float), ("rho_max", c_float), ("d_half", c_float), ("eps_explore", c_float),
         ("clip_lo", c_float), ("clip_hi", c_float), ("norm_eps", c_float), ("norm_ddof", c_int32),
         ("agg_mode", c_int32), ("global_tokens", c_int32), ("global_responses", c_int32),
-        ("surrogate", c_int32),
+        ("surrogate", c_int32), ("dual_clip", c_float), ("near_zero_tau_lo", c_float),
+        ("near_zero_tau_hi", c_float),
     ]
 
 
@@ -72,6 +73,8 @@ def lib():
                                      c_void_p, c_void_p, c_size_t, P, c_void_p, c_void_p]
         L.spo_advantages_static.argtypes = [c_void_p, c_int64, c_void_p, c_void_p, c_int32, c_void_p, c_void_p,
                                             c_void_p, P, c_void_p, c_void_p]
+        L.spo_advantages_update.argtypes = [c_void_p, c_int64, c_void_p, c_void_p, c_void_p, c_int32, c_int32,
+                                            c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, P, c_void_p, c_void_p]
         L.spo_advantages_apply.argtypes = [c_void_p, c_int32, c_float, c_float, c_void_p, P, c_void_p]
         L.spo_tracker_update.argtypes = [c_void_p, c_int64, c_void_p, c_void_p, c_void_p, c_int32, c_int32,
                                          P, c_void_p, c_void_p]
@@ -89,6 +92,8 @@ def lib():
                                        c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                                        c_void_p, c_int32, c_void_p, c_int32,
                                        c_void_p, c_size_t, P, c_void_p, c_void_p]
+        L.spo_loss_fwd_bwd_slabs.argtypes = list(L.spo_loss_fwd_bwd.argtypes) + [c_int32, POINTER(c_void_p)]
+        L.spo_dw_slab_rows.argtypes = [c_int32, c_int32, c_int32, POINTER(c_int64)]
         L.spo_loss_stats.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_int32, c_void_p, P,
                                      c_void_p]
         L.spo_loss_mask_rows.argtypes = [c_void_p, c_int64, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
@@ -167,6 +172,13 @@ def spo_advantages(ab, ids, r, a_raw, a_norm, stats, ws, params, d_status):
                                 ctypes.byref(params), _ptr(d_status), _stream()), "spo_advantages")
 
 
+def spo_advantages_update(ab, ids, r, kl, kl_is_table, a_raw, a_norm, stats, ws, params, d_status):
+    _check(lib().spo_advantages_update(_ptr(ab), ab.shape[0], _ptr(ids), _ptr(r), _ptr(kl), int(kl_is_table),
+                                       ids.numel(), _ptr(a_raw), _ptr(a_norm), _ptr(stats), _ptr(ws),
+                                       0 if ws is None else ws.numel() * ws.element_size(), ctypes.byref(params),
+                                       _ptr(d_status), _stream()), "spo_advantages_update")
+
+
 def spo_advantages_apply(a_raw, mu, sigma, a_norm, params):
     _check(lib().spo_advantages_apply(_ptr(a_raw), a_raw.numel(), c_float(mu), c_float(sigma), _ptr(a_norm),
                                       ctypes.byref(params), _stream()), "spo_advantages_apply")
@@ -228,6 +240,34 @@ def spo_loss_fwd_bwd(H, W, y, logp_old, mask, cu_seqlens, a_norm, grad_loss, los
                                   _dtype_code(dH), _ptr(dW), int(dW_accumulate), _ptr(ws),
                                   ws.numel() * ws.element_size(), ctypes.byref(params), _ptr(d_status), _stream()),
            "spo_loss_fwd_bwd")
+
+
+MAX_DW_SLABS = 64
+
+
+def spo_dw_slab_rows(V, d, n_wanted):
+    """Vocabulary-row bounds [0, ..., V] of the slabs a request for n_wanted slabs comes to (host only)."""
+    buf = (c_int64 * (n_wanted + 1))()
+    n = lib().spo_dw_slab_rows(V, d, n_wanted, buf)
+    if n < 0:
+        raise SpoError(n, "spo_dw_slab_rows")
+    return [int(buf[k]) for k in range(n + 1)]
+
+
+def spo_loss_fwd_bwd_slabs(H, W, y, logp_old, mask, cu_seqlens, a_norm, grad_loss, loss, logp, lse, coef, seq_sums, dH,
+                           dW, dW_accumulate, ws, params, d_status, events, entropy=None):
+    """spo_loss_fwd_bwd with the last dW contraction cut into len(events) slabs; `events` are
+    torch.cuda.Event objects that already own a CUDA event (recorded once), one is recorded behind each slab."""
+    T, d = H.shape
+    V = W.shape[0]
+    S = cu_seqlens.numel() - 1
+    handles = (c_void_p * len(events))(*[c_void_p(ev.cuda_event) for ev in events])
+    _check(lib().spo_loss_fwd_bwd_slabs(_ptr(H), _ptr(W), _dtype_code(W), _ptr(y), _ptr(logp_old), _ptr(mask),
+                                        _ptr(cu_seqlens), _ptr(a_norm), T, d, V, S, c_float(grad_loss), _ptr(loss),
+                                        _ptr(logp), _ptr(lse), _ptr(coef), _ptr(seq_sums), _ptr(entropy), _ptr(dH),
+                                        _dtype_code(dH), _ptr(dW), int(dW_accumulate), _ptr(ws),
+                                        ws.numel() * ws.element_size(), ctypes.byref(params), _ptr(d_status), _stream(),
+                                        len(events), handles), "spo_loss_fwd_bwd_slabs")
 
 
 def spo_loss_stats(logp, logp_old, mask, cu_seqlens, a_norm, out, params):

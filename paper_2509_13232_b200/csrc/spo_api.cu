@@ -56,10 +56,11 @@ FwdWs fwd_ws_layout(int64_t T, int32_t d, int32_t V, int32_t dtype, int32_t S) {
 
 static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-static inline int32_t cuda_fail(cudaError_t e) {
+int32_t record_cuda_error(cudaError_t e) {
   g_last_cuda_error = (int32_t)e;
   return SPO_ERR_CUDA;
 }
+static inline int32_t cuda_fail(cudaError_t e) { return record_cuda_error(e); }
 
 static bool params_ok(const spo_params* p) {
   if (!p) return false;
@@ -72,6 +73,8 @@ static bool params_ok(const spo_params* p) {
   if (p->agg_mode != SPO_AGG_TOKEN_MEAN && p->agg_mode != SPO_AGG_SEQ_MEAN) return false;
   if (p->global_tokens < 0 || p->global_responses < 0) return false;
   if (p->surrogate != SPO_SUR_PPO_CLIP && p->surrogate != SPO_SUR_CISPO && p->surrogate != SPO_SUR_GSPO) return false;
+  if (!(p->dual_clip == 0.0f || (p->dual_clip > 1.0f && p->dual_clip < 3.0e38f))) return false;
+  if (!(p->near_zero_tau_lo >= 0.0f) || !(p->near_zero_tau_hi >= 0.0f)) return false;
   return true;
 }
 
@@ -100,12 +103,11 @@ static cudaError_t forward_launches(const void* H, const void* W, int32_t dtype,
   else
     e = launch_fwd_f32((const float*)H, (const float*)W, y, T, d, V, partials, st);
   if (e != cudaSuccess) return e;
-  e = launch_fwd_finalize(partials, L.nsplit, y, logp_old, mask, cu_seqlens, a_norm, T, V, S, params->clip_lo,
-                          params->clip_hi, loss, logp, lse, coef, seq_sums, entropy, block_sums, counters, seq_cnt,
-                          params->agg_mode, params->surrogate, params->global_tokens, params->global_responses, L.fin_blocks, d_status, st);
+  e = launch_fwd_finalize(partials, L.nsplit, y, logp_old, mask, cu_seqlens, a_norm, T, V, S, loss, logp, lse, coef,
+                          seq_sums, entropy, block_sums, counters, seq_cnt, *params, L.fin_blocks, d_status, st);
   if (e != cudaSuccess || !seq_level) return e;
-  return launch_seq_level_objective(logp, logp_old, mask, cu_seqlens, a_norm, T, S, params->clip_lo, params->clip_hi,
-                                    counters, params->global_responses, reinterpret_cast<float*>(w8 + L.seq_coef),
+  return launch_seq_level_objective(logp, logp_old, mask, cu_seqlens, a_norm, T, S, *params, counters,
+                                    reinterpret_cast<float*>(w8 + L.seq_coef),
                                     reinterpret_cast<double*>(w8 + L.seq_term), coef, loss, st);
 }
 
@@ -129,6 +131,9 @@ int32_t spo_default_params(spo_params* p) {
   p->global_tokens = 0;
   p->global_responses = 0;
   p->surrogate = SPO_SUR_PPO_CLIP;
+  p->dual_clip = 0.0f;
+  p->near_zero_tau_lo = 1e-4f;
+  p->near_zero_tau_hi = 0.02f;
   return SPO_OK;
 }
 
@@ -171,8 +176,28 @@ int32_t spo_advantages(const float* ab, int64_t N, const int32_t* ids, const flo
     if (!ws) return SPO_ERR_INVALID_ARG;
     if (ws_bytes < spo_workspace_bytes(SPO_WS_ADVANTAGES, 0, 0, 0, N, B, 0)) return SPO_ERR_WORKSPACE_TOO_SMALL;
   }
-  cudaError_t e = launch_advantages(ab, N, ids, r, B, a_raw, a_norm, stats, (char*)ws, params->norm_eps,
-                                    params->norm_ddof, d_status, (cudaStream_t)stream);
+  cudaError_t e = launch_advantages(const_cast<float*>(ab), N, ids, r, B, a_raw, a_norm, stats, ws, *params, nullptr,
+                                    false, d_status, (cudaStream_t)stream);
+  return e == cudaSuccess ? SPO_OK : cuda_fail(e);
+}
+
+int32_t spo_advantages_update(float* ab, int64_t N, const int32_t* ids, const float* r, const float* kl,
+                              int32_t kl_is_table, int32_t B, float* a_raw, float* a_norm, float* stats, void* ws,
+                              size_t ws_bytes, const spo_params* params, int32_t* d_status, void* stream) {
+  if (!params_ok(params) || !ab || !ids || !r || !kl || !a_norm) return SPO_ERR_INVALID_ARG;
+  if (kl_is_table != 0 && kl_is_table != 1) return SPO_ERR_INVALID_ARG;
+  if (N < 1 || N >= ((int64_t)1 << 31) || B < 1) return SPO_ERR_BAD_SHAPE;
+  if (!aligned16(ab) || !aligned16(ids) || !aligned16(r) || !aligned16(kl) || !aligned16(a_raw) ||
+      !aligned16(a_norm) || !aligned16(stats) || !aligned16(ws))
+    return SPO_ERR_BAD_ALIGNMENT;
+  if (!device_is_sm100()) return SPO_ERR_UNSUPPORTED_ARCH;
+  if (B > kAdvSingleBlockMax) {
+    if (!ws) return SPO_ERR_INVALID_ARG;
+    if (ws_bytes < spo_workspace_bytes(SPO_WS_ADVANTAGES, 0, 0, 0, N, B, 0)) return SPO_ERR_WORKSPACE_TOO_SMALL;
+  }
+  const AdvUpdate upd = {kl, kl_is_table};
+  cudaError_t e = launch_advantages(ab, N, ids, r, B, a_raw, a_norm, stats, ws, *params, &upd, false, d_status,
+                                    (cudaStream_t)stream);
   return e == cudaSuccess ? SPO_OK : cuda_fail(e);
 }
 
@@ -273,11 +298,24 @@ int32_t spo_loss_bwd(const void* H, const void* W, int32_t dtype, const int32_t*
   return e == cudaSuccess ? SPO_OK : cuda_fail(e);
 }
 
-int32_t spo_loss_fwd_bwd(const void* H, const void* W, int32_t dtype, const int32_t* y, const float* logp_old,
-                         const uint8_t* mask, const int32_t* cu_seqlens, const float* a_norm, int64_t T, int32_t d,
-                         int32_t V, int32_t S, float grad_loss, float* loss, float* logp, float* lse, float* coef,
-                         float* seq_sums, float* entropy, void* dH, int32_t dH_dtype, float* dW, int32_t dW_accumulate,
-                         void* ws, size_t ws_bytes, const spo_params* params, int32_t* d_status, void* stream) {
+}  // extern "C"
+
+// Behind every slab of dW rows an event, when the caller asked for them (see spo_loss_fwd_bwd_slabs).
+// Paths that do not cut the last contraction record all of them at the end.
+static cudaError_t record_all(void* const* events, int n, cudaStream_t st) {
+  for (int k = 0; k < n; ++k) {
+    cudaError_t e = cudaEventRecord((cudaEvent_t)events[k], st);
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
+}
+
+static int32_t loss_fwd_bwd_impl(const void* H, const void* W, int32_t dtype, const int32_t* y, const float* logp_old,
+                                 const uint8_t* mask, const int32_t* cu_seqlens, const float* a_norm, int64_t T, int32_t d,
+                                 int32_t V, int32_t S, float grad_loss, float* loss, float* logp, float* lse, float* coef,
+                                 float* seq_sums, float* entropy, void* dH, int32_t dH_dtype, float* dW,
+                                 int32_t dW_accumulate, void* ws, size_t ws_bytes, const spo_params* params,
+                                 int32_t* d_status, void* stream, int32_t n_slabs, void* const* events) {
   int32_t rc = check_loss_shape(dtype, T, d, V);
   if (rc != SPO_OK) return rc;
   if (dH_dtype != SPO_DTYPE_F32 && dH_dtype != SPO_DTYPE_BF16) return SPO_ERR_UNSUPPORTED_DTYPE;
@@ -291,8 +329,28 @@ int32_t spo_loss_fwd_bwd(const void* H, const void* W, int32_t dtype, const int3
   cudaStream_t st = (cudaStream_t)stream;
   char* w8 = (char*)ws;
   cudaError_t e;
+  int slabs_used = 0;                      // slabs the caller's n_slabs comes to (its events 0 .. slabs_used-1 exist)
+  if (n_slabs > 0) {
+    int64_t bounds[SPO_MAX_DW_SLABS + 1];
+    slabs_used = dw_slab_rows(V, d, n_slabs, bounds);
+  }
+  if (dtype == SPO_DTYPE_BF16 && params->surrogate == SPO_SUR_GSPO) {
+    // A response's ratio needs the log-probs of all its tokens, and those may lie in later chunks than
+    // the rows whose gradient is being formed: the forward runs to the end first, then the chunked
+    // backward (four contractions per token, as spo_loss_fwd followed by spo_loss_bwd).
+    const FwdWs Lf = fwd_ws_layout(T, d, V, dtype, S);
+    const BwdWs Lb = bwd_ws_layout(T, d, V);
+    const size_t off_b = align_up(Lf.total, 256);
+    if (ws_bytes < off_b + Lb.total) return SPO_ERR_WORKSPACE_TOO_SMALL;
+    if ((e = forward_launches(H, W, dtype, y, logp_old, mask, cu_seqlens, a_norm, T, d, V, S, loss, logp, lse, coef,
+                              seq_sums, entropy, w8, Lf, params, d_status, st)) != cudaSuccess)
+      return cuda_fail(e);
+    e = launch_bwd_bf16(H, W, y, lse, coef, grad_loss, T, d, V, dH, dH_dtype, dW, dW_accumulate, w8 + off_b, Lb,
+                        d_status, st);
+    if (e == cudaSuccess && n_slabs > 0) e = record_all(events, slabs_used, st);
+    return e == cudaSuccess ? SPO_OK : cuda_fail(e);
+  }
   if (dtype == SPO_DTYPE_BF16) {
-    if (params->surrogate == SPO_SUR_GSPO) return SPO_ERR_INVALID_ARG;     // needs whole responses: two-call path
     const FusedWs L = fused_ws_layout(T, d, V, S);
     if (ws_bytes < L.total) return SPO_ERR_WORKSPACE_TOO_SMALL;
     FusedArgs a{};
@@ -301,6 +359,7 @@ int32_t spo_loss_fwd_bwd(const void* H, const void* W, int32_t dtype, const int3
     a.loss = loss; a.logp = logp; a.lse = lse; a.coef = coef; a.seq_sums = seq_sums; a.entropy = entropy;
     a.dH = dH; a.dH_dtype = dH_dtype; a.dW = dW; a.accumulate = dW_accumulate;
     a.params = params; a.d_status = d_status;
+    a.n_slabs = n_slabs; a.events = reinterpret_cast<cudaEvent_t*>(const_cast<void**>(events));
     e = launch_fused_bf16(a, w8, L, st);
     return e == cudaSuccess ? SPO_OK : cuda_fail(e);
   }
@@ -312,7 +371,42 @@ int32_t spo_loss_fwd_bwd(const void* H, const void* W, int32_t dtype, const int3
     return cuda_fail(e);
   e = launch_bwd_f32((const float*)H, (const float*)W, y, lse, coef, grad_loss, T, d, V, dH, dH_dtype, dW,
                      dW_accumulate, st);
+  if (e == cudaSuccess && n_slabs > 0) e = record_all(events, slabs_used, st);
   return e == cudaSuccess ? SPO_OK : cuda_fail(e);
+}
+
+extern "C" {
+
+int32_t spo_loss_fwd_bwd(const void* H, const void* W, int32_t dtype, const int32_t* y, const float* logp_old,
+                         const uint8_t* mask, const int32_t* cu_seqlens, const float* a_norm, int64_t T, int32_t d,
+                         int32_t V, int32_t S, float grad_loss, float* loss, float* logp, float* lse, float* coef,
+                         float* seq_sums, float* entropy, void* dH, int32_t dH_dtype, float* dW, int32_t dW_accumulate,
+                         void* ws, size_t ws_bytes, const spo_params* params, int32_t* d_status, void* stream) {
+  return loss_fwd_bwd_impl(H, W, dtype, y, logp_old, mask, cu_seqlens, a_norm, T, d, V, S, grad_loss, loss, logp, lse,
+                           coef, seq_sums, entropy, dH, dH_dtype, dW, dW_accumulate, ws, ws_bytes, params, d_status,
+                           stream, 0, nullptr);
+}
+
+int32_t spo_dw_slab_rows(int32_t V, int32_t d, int32_t n_wanted, int64_t* row_begin) {
+  if (V < 1 || d < 1 || n_wanted < 1 || n_wanted > SPO_MAX_DW_SLABS || !row_begin) return SPO_ERR_INVALID_ARG;
+  return dw_slab_rows(V, d, n_wanted, row_begin);
+}
+
+int32_t spo_loss_fwd_bwd_slabs(const void* H, const void* W, int32_t dtype, const int32_t* y, const float* logp_old,
+                               const uint8_t* mask, const int32_t* cu_seqlens, const float* a_norm, int64_t T,
+                               int32_t d, int32_t V, int32_t S, float grad_loss, float* loss, float* logp, float* lse,
+                               float* coef, float* seq_sums, float* entropy, void* dH, int32_t dH_dtype, float* dW,
+                               int32_t dW_accumulate, void* ws, size_t ws_bytes, const spo_params* params,
+                               int32_t* d_status, void* stream, int32_t n_wanted, void* const* events) {
+  if (n_wanted < 1 || n_wanted > SPO_MAX_DW_SLABS || !events || V < 1 || d < 1) return SPO_ERR_INVALID_ARG;
+  int64_t bounds[SPO_MAX_DW_SLABS + 1];
+  const int n = dw_slab_rows(V, d, n_wanted, bounds);
+  for (int k = 0; k < n; ++k)
+    if (!events[k]) return SPO_ERR_INVALID_ARG;
+  // dw_slab_rows(n) and the launch must agree on the cut: the launch is asked for the same n_wanted
+  return loss_fwd_bwd_impl(H, W, dtype, y, logp_old, mask, cu_seqlens, a_norm, T, d, V, S, grad_loss, loss, logp, lse,
+                           coef, seq_sums, entropy, dH, dH_dtype, dW, dW_accumulate, ws, ws_bytes, params, d_status,
+                           stream, n_wanted, events);
 }
 
 namespace {
@@ -380,12 +474,12 @@ int32_t spo_loss_bwd_rows(const void* H, const void* W, int32_t dtype, const int
   int32_t* y_act = reinterpret_cast<int32_t*>(w8 + L.y_act);
   float* lse_act = reinterpret_cast<float*>(w8 + L.lse_act);
   float* coef_act = reinterpret_cast<float*>(w8 + L.coef_act);
-  if ((e = launch_gather_rows(H, y, lse, coef, rows, T_act, d * 2, h_act, y_act, lse_act, coef_act, st)) != cudaSuccess)
+  if ((e = launch_gather_rows(H, y, lse, coef, rows, T_act, T, d * 2, h_act, y_act, lse_act, coef_act, d_status, st)) != cudaSuccess)
     return cuda_fail(e);
   if ((e = launch_bwd_bf16(h_act, W, y_act, lse_act, coef_act, grad_loss, T_act, d, V, dh_act, dH_dtype, dW,
                            dW_accumulate, w8 + L.bwd, L.inner, d_status, st)) != cudaSuccess)
     return cuda_fail(e);
-  if ((e = launch_scatter_rows(dh_act, rows, T_act, d * dh_elem, dH, st)) != cudaSuccess) return cuda_fail(e);
+  if ((e = launch_scatter_rows(dh_act, rows, T_act, T, d * dh_elem, dH, st)) != cudaSuccess) return cuda_fail(e);
   return SPO_OK;
 }
 
@@ -471,7 +565,7 @@ int32_t spo_loss_fwd_bwd_rows(const void* H, const void* W, int32_t dtype, const
   float* coef_act = reinterpret_cast<float*>(w8 + L.coef_act);
   int32_t* cu_act = reinterpret_cast<int32_t*>(w8 + L.cu_act);
   // the compacted batch: listed rows of H, y, logp_old, and the sequence boundaries among them
-  if ((e = launch_gather_rows(H, y, logp_old, logp_old, rows, T_act, d * 2, h_act, y_act, lo_act, logp_act, st)) !=
+  if ((e = launch_gather_rows(H, y, logp_old, logp_old, rows, T_act, T, d * 2, h_act, y_act, lo_act, logp_act, d_status, st)) !=
       cudaSuccess)
     return cuda_fail(e);
   if ((e = launch_compact_cu_seqlens(rows, T_act, cu_seqlens, S, cu_act, st)) != cudaSuccess) return cuda_fail(e);
@@ -482,9 +576,9 @@ int32_t spo_loss_fwd_bwd_rows(const void* H, const void* W, int32_t dtype, const
   a.dH = dh_act; a.dH_dtype = dH_dtype; a.dW = dW; a.accumulate = dW_accumulate;
   a.params = params; a.d_status = d_status;
   if ((e = launch_fused_bf16(a, w8 + L.fused, L.inner, st)) != cudaSuccess) return cuda_fail(e);
-  if ((e = launch_scatter_scalars(logp_act, lse_act, coef_act, rows, T_act, logp, lse, coef, st)) != cudaSuccess)
+  if ((e = launch_scatter_scalars(logp_act, lse_act, coef_act, rows, T_act, T, logp, lse, coef, st)) != cudaSuccess)
     return cuda_fail(e);
-  if ((e = launch_scatter_rows(dh_act, rows, T_act, d * dh_elem, dH, st)) != cudaSuccess) return cuda_fail(e);
+  if ((e = launch_scatter_rows(dh_act, rows, T_act, T, d * dh_elem, dH, st)) != cudaSuccess) return cuda_fail(e);
   return SPO_OK;
 }
 
@@ -496,7 +590,7 @@ int32_t spo_loss_stats(const float* logp, const float* logp_old, const uint8_t* 
   if (!aligned16(logp) || !aligned16(logp_old) || !aligned16(cu_seqlens) || !aligned16(a_norm) || !aligned16(out))
     return SPO_ERR_BAD_ALIGNMENT;
   if (!device_is_sm100()) return SPO_ERR_UNSUPPORTED_ARCH;
-  cudaError_t e = launch_loss_stats(logp, logp_old, mask, cu_seqlens, a_norm, T, S, params->clip_lo, params->clip_hi, out,
+  cudaError_t e = launch_loss_stats(logp, logp_old, mask, cu_seqlens, a_norm, T, S, *params, out,
                                     (cudaStream_t)stream);
   return e == cudaSuccess ? SPO_OK : cuda_fail(e);
 }
@@ -508,7 +602,7 @@ size_t spo_workspace_bytes(int32_t which, int64_t T, int32_t d, int32_t V, int64
       return sample_ws_layout(N, M).total;
     case SPO_WS_ADVANTAGES:
       if (B <= kAdvSingleBlockMax) return 256;
-      return align_up(sizeof(double) * 2 * (size_t)adv_blocks(B), 256);
+      return adv_partial_bytes(B);
     case SPO_WS_UPDATE_REPEATS:
       if (B < 0 || B > kRepeatsMaxBatch) return 0;
       return repeats_ws_layout(B).total;
@@ -531,7 +625,9 @@ size_t spo_workspace_bytes(int32_t which, int64_t T, int32_t d, int32_t V, int64
       if (T < 0 || V < 1 || d < 1) return 0;
       const size_t f32 = fwd_ws_layout(T, d, V, SPO_DTYPE_F32, B).total;
       if ((d % 64) != 0) return f32;
-      const size_t bf16 = fused_ws_layout(T, d, V, B).total;
+      size_t bf16 = fused_ws_layout(T, d, V, B).total;
+      const size_t two_call = align_up(fwd_ws_layout(T, d, V, SPO_DTYPE_BF16, B).total, 256) + bwd_ws_layout(T, d, V).total;
+      if (two_call > bf16) bf16 = two_call;         // the sequence-level objective runs forward, then backward
       return bf16 > f32 ? bf16 : f32;
     }
     default:

@@ -15,6 +15,7 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 
 int sm_count();                       // SMs of the current device (cached per device)
+int32_t record_cuda_error(cudaError_t e);   // remembers e for spo_last_cuda_error(); returns SPO_ERR_CUDA
 int device_is_sm100();                // 1 when the current device is compute capability 10.x
 
 // ---- sampler ------------------------------------------------------------
@@ -39,9 +40,12 @@ constexpr int kAdvSingleBlockMax = 8192;
 int adv_blocks(int32_t B);
 cudaError_t launch_advantages_apply(const float* a_raw, int32_t B, float mu, float sigma, float norm_eps, float* a_norm,
                                     cudaStream_t st);
-cudaError_t launch_advantages(const float* ab, int64_t N, const int32_t* ids, const float* r, int32_t B,
-                              float* a_raw, float* a_norm, float* stats, char* ws,
-                              float norm_eps, int32_t ddof, int32_t* d_status, cudaStream_t st);
+// Divergences for the fused advantage + update pass: [B] per batch entry, or [N] per prompt.
+struct AdvUpdate { const float* kl; int kl_is_table; };
+size_t adv_partial_bytes(int32_t B);   // block records of the two-pass path
+cudaError_t launch_advantages(float* ab, int64_t N, const int32_t* ids, const float* r, int32_t B,
+                              float* a_raw, float* a_norm, float* stats, void* partials, const spo_params& pr,
+                              const AdvUpdate* upd, bool force_two_pass, int32_t* d_status, cudaStream_t st);
 cudaError_t launch_tracker_update(float* ab, int64_t N, const int32_t* ids, const float* r,
                                   const float* kl, int kl_is_table, int32_t B,
                                   float rho_min, float rho_max, float d_half,
@@ -90,23 +94,36 @@ struct FinalizeRange {
   int last;             // 1 when this launch covers the final rows (per-response sums are taken then)
 };
 
+// Extra work of the finalisation in the one-pass forward+backward (G == nullptr: none).  With the
+// chunk's exponentials e = 2^(z log2e - ref_t) in G and l_t = sum_v e, the logit gradient is
+// g[t,v] = rowscale_t (e[t,v] - l_t 1[v = y_t]), rowscale_t = -grad_loss coef_t / l_t: the kernel
+// writes rowscale_t and replaces the one entry G[t][y_t] by e - l_t.
+struct OnePassFix {
+  uint16_t* G;          // bf16 [chunk rows][ldg]
+  int64_t ldg;
+  int64_t g_row0;       // token row held by row 0 of G
+  float* rowscale;      // [T], indexed by token row
+  float grad_loss;
+};
+
 // need_seq_counts: per-response unmasked counts and the number of responses that have any
 cudaError_t launch_fwd_prepare(const uint8_t* mask, int64_t T, const int32_t* cu_seqlens, int32_t S,
                                int need_seq_counts, int32_t* seq_cnt, int32_t* counters, cudaStream_t st);
 // Sequence-level objective: coef and loss from the finished logp of all tokens.
 cudaError_t launch_seq_level_objective(const float* logp, const float* logp_old, const uint8_t* mask,
                                        const int32_t* cu_seqlens, const float* a_norm, int64_t T, int32_t S,
-                                       float clip_lo, float clip_hi, const int32_t* counters, int32_t global_responses,
+                                       const spo_params& pr, const int32_t* counters,
                                        float* seq_coef, double* seq_term, float* coef, float* loss, cudaStream_t st);
 cudaError_t launch_fwd_finalize(const FwdPartial* partials, int nsplit, const int32_t* y,
                                 const float* logp_old, const uint8_t* mask, const int32_t* cu_seqlens,
                                 const float* a_norm, int64_t T, int32_t V, int32_t S,
-                                float clip_lo, float clip_hi,
                                 float* loss, float* logp, float* lse, float* coef, float* seq_sums, float* entropy,
-                                double* block_sums, int32_t* counters, const int32_t* seq_cnt, int agg_mode,
-                                int surrogate, int32_t global_tokens, int32_t global_responses,
+                                double* block_sums, int32_t* counters, const int32_t* seq_cnt, const spo_params& pr,
                                 int64_t fin_blocks, int32_t* d_status, cudaStream_t st,
-                                const FinalizeRange* range = nullptr);
+                                const FinalizeRange* range = nullptr, const OnePassFix* fix = nullptr);
+// out[i][:] = rowscale[t0 + i] * H[t0 + i][:] for i < rows (bf16 rows of row_bytes bytes; a zero factor gives zeros)
+cudaError_t launch_scale_rows(const void* H, const float* rowscale, int64_t t0, int64_t rows, int32_t row_bytes,
+                              void* out, cudaStream_t st);
 
 // fp32 SIMT path
 cudaError_t launch_fwd_f32(const float* H, const float* W, const int32_t* y, int64_t T, int32_t d, int32_t V,
@@ -127,15 +144,16 @@ BwdWs bwd_ws_layout(int64_t T, int32_t d, int32_t V);
 
 // one-pass forward+backward (bf16)
 struct FusedWs {
-  size_t g;             // n_buf x bf16 [chunk_rows][ldg]: e, then g, of one chunk each
-  size_t ref;           // n_buf x float [ldg/64][chunk_rows]: reference exponents of e
-  size_t g_bytes, ref_bytes;   // size of one of them
+  size_t g;             // slots x bf16 [chunk_rows][ldg], contiguous: the stored exponentials of one chunk each
+  size_t hs;            // slots x bf16 [chunk_rows][d], contiguous: the chunks' rows of H times their row scale
+  size_t pre;           // FwdPartial [2][T]: statistics of every row's first vocabulary tile
+  size_t rowscale;      // float [T]
   size_t partials;      // FwdPartial [2*nsplit][rows of the chunk]
   size_t progress, block_sums, counters, seq_cnt;
   size_t total;
   int64_t chunk_rows, ldg;
   int64_t fin_blocks;
-  int n_buf;            // 2 when there is more than one chunk (chunks are software-pipelined), else 1
+  int slots;            // chunks whose dW contribution is contracted in one launch (K = their rows together)
 };
 FusedWs fused_ws_layout(int64_t T, int32_t d, int32_t V, int32_t S);
 struct FusedArgs {
@@ -155,7 +173,15 @@ struct FusedArgs {
   int accumulate;
   const spo_params* params;
   int32_t* d_status;
+  // Data-parallel ranks reduce dW while its last contraction still runs: that launch is cut into
+  // `n_slabs` slabs of vocabulary rows and events[k] is recorded on the stream behind slab k
+  // (0 / NULL: one launch, no events).
+  int n_slabs;
+  cudaEvent_t* events;
 };
+// Vocabulary-row bounds of the slabs the last dW contraction is cut into: row_begin[0..n] with
+// row_begin[0] = 0 and row_begin[n] = V; returns n <= n_wanted (slabs hold whole rounds of row tiles).
+int dw_slab_rows(int32_t V, int32_t d, int n_wanted, int64_t* row_begin);
 cudaError_t launch_fused_bf16(const FusedArgs& a, char* ws, const FusedWs& L, cudaStream_t st);
 
 cudaError_t launch_fwd_bf16(const void* H, const void* W, const int32_t* y, int64_t T, int32_t d, int32_t V,
@@ -171,19 +197,19 @@ cudaError_t launch_bwd_bf16(const void* H, const void* W, const int32_t* y, cons
 cudaError_t launch_active_rows(const float* coef, const uint8_t* mask, int64_t T, int32_t* rows, int32_t* d_count,
                                int32_t* block_cnt, cudaStream_t st);
 cudaError_t launch_loss_stats(const float* logp, const float* logp_old, const uint8_t* mask, const int32_t* cu_seqlens,
-                              const float* a_norm, int64_t T, int32_t S, float clip_lo, float clip_hi, float* out,
+                              const float* a_norm, int64_t T, int32_t S, const spo_params& pr, float* out,
                               cudaStream_t st);
 cudaError_t launch_compact_cu_seqlens(const int32_t* rows, int64_t n_act, const int32_t* cu_seqlens, int32_t S,
                                       int32_t* cu_act, cudaStream_t st);
 cudaError_t launch_scatter_scalars(const float* logp_act, const float* lse_act, const float* coef_act,
-                                   const int32_t* rows, int64_t n_act, float* logp, float* lse, float* coef,
+                                   const int32_t* rows, int64_t n_act, int64_t T, float* logp, float* lse, float* coef,
                                    cudaStream_t st);
 size_t active_rows_ws_bytes(int64_t T);
 cudaError_t launch_gather_rows(const void* H, const int32_t* y, const float* lse, const float* coef,
-                               const int32_t* rows, int64_t n_act, int32_t row_bytes, void* H_act, int32_t* y_act,
-                               float* lse_act, float* coef_act, cudaStream_t st);
-cudaError_t launch_scatter_rows(const void* dH_act, const int32_t* rows, int64_t n_act, int32_t row_bytes, void* dH,
-                                cudaStream_t st);
+                               const int32_t* rows, int64_t n_act, int64_t T, int32_t row_bytes, void* H_act,
+                               int32_t* y_act, float* lse_act, float* coef_act, int32_t* d_status, cudaStream_t st);
+cudaError_t launch_scatter_rows(const void* dH_act, const int32_t* rows, int64_t n_act, int64_t T, int32_t row_bytes,
+                                void* dH, cudaStream_t st);
 
 cudaError_t launch_bounded_wait_probe(int32_t* d_status, uint32_t limit_us, int32_t* reached_end, cudaStream_t st);
 

@@ -81,7 +81,7 @@ fwd_finalize_kernel(const FwdPartial* __restrict__ partials, int nsplit, const i
                     float* __restrict__ loss, float* __restrict__ logp_out, float* __restrict__ lse_out,
                     float* __restrict__ coef_out, float* __restrict__ entropy_out, double* block_sums, int32_t* counters,
                     const int32_t* __restrict__ seq_cnt, int agg_mode, int surrogate, int32_t global_tokens,
-                    int32_t global_responses, int32_t* d_status, FinalizeRange rg) {
+                    int32_t global_responses, float dual_clip, int32_t* d_status, FinalizeRange rg, OnePassFix fix) {
   // This launch covers token rows [rg.t_begin, T_end); its blocks are blocks rg.block0.. of the
   // rg.total_blocks that cover all rows (one launch, or one per chunk of the one-pass path).
   const int64_t t = rg.t_begin + (int64_t)blockIdx.x * kFinalizeThreads + threadIdx.x;
@@ -107,9 +107,11 @@ fwd_finalize_kernel(const FwdPartial* __restrict__ partials, int nsplit, const i
     const float lse = (m2 + log2f(l)) * kLn2;
     if (entropy_out) entropy_out[t] = lse - ez / l;      // -sum_v p log p = lse - sum_v p z
     const int32_t yt = y[t];
+    const bool on = mask ? mask[t] != 0 : true;
     float lp, coef = 0.0f;
     if (yt < 0 || yt >= V) {
-      flag(d_status, SPO_DEV_ID_OUT_OF_RANGE);
+      // a masked row may carry an ignore-index target (-100, -1): it takes no part in the loss
+      if (on) flag(d_status, SPO_DEV_ID_OUT_OF_RANGE);
       lp = -CUDART_INF_F;
     } else {
       lp = zt - lse;
@@ -120,7 +122,6 @@ fwd_finalize_kernel(const FwdPartial* __restrict__ partials, int nsplit, const i
         if ((int64_t)cu_seqlens[mid] <= t) lo = mid; else hi = mid;
       }
       const float a = a_norm[lo];
-      const bool on = mask ? mask[t] != 0 : true;
       const float hi_b = 1.0f + clip_hi, lo_b = 1.0f - clip_lo;
       const float cut = fminf(fmaxf(ratio, lo_b), hi_b);
       // per unit of token weight: the objective's term and d term / d logp
@@ -130,7 +131,11 @@ fwd_finalize_kernel(const FwdPartial* __restrict__ partials, int nsplit, const i
         dsur = cut * a;
       } else {                                 // PPO-Clip (a sequence-level objective fills coef later)
         sur = fminf(ratio * a, cut * a);
-        const bool passes = a >= 0.0f ? ratio <= hi_b : ratio >= lo_b;
+        bool passes = a >= 0.0f ? ratio <= hi_b : ratio >= lo_b;
+        if (dual_clip > 0.0f && a < 0.0f) {    // second clip: the term may not fall below c a
+          sur = fmaxf(sur, dual_clip * a);
+          passes = passes && !(ratio > dual_clip);
+        }
         dsur = passes ? a * ratio : 0.0f;
       }
       if (on && n_tok > 0 && surrogate != SPO_SUR_GSPO) {
@@ -148,6 +153,19 @@ fwd_finalize_kernel(const FwdPartial* __restrict__ partials, int nsplit, const i
     logp_out[t] = lp;
     lse_out[t] = lse;
     coef_out[t] = coef;
+    if (fix.G) {
+      // one-pass path: m2 is the row's reference exponent (common to all its partials), l the sum of
+      // its stored exponentials.  A row whose logits outran the reference has l = Inf: reported, and
+      // it takes no part in the gradient (its logp is -Inf, so its coef is already zero).
+      if (!(l < CUDART_INF_F)) flag(d_status, SPO_DEV_NONFINITE);
+      float rsc = 0.0f;
+      if (coef != 0.0f && l > 0.0f && l < CUDART_INF_F) {
+        rsc = -fix.grad_loss * coef / l;
+        const float ey = exp2f(fmaf(zt, kLog2e, -m2));
+        reinterpret_cast<__nv_bfloat16*>(fix.G)[(t - fix.g_row0) * fix.ldg + yt] = __float2bfloat16_rn(ey - l);
+      }
+      fix.rowscale[t] = rsc;
+    }
   }
   __shared__ double s_part[kFinalizeThreads / 32];
   __shared__ int s_last;
@@ -396,27 +414,61 @@ active_write_kernel(const float* __restrict__ coef, const uint8_t* __restrict__ 
 // One warp per active row: copy the row of H (16-byte pieces) and its per-token scalars.
 __global__ void __launch_bounds__(256)
 gather_rows_kernel(const uint4* __restrict__ H, const int32_t* __restrict__ y, const float* __restrict__ lse,
-                   const float* __restrict__ coef, const int32_t* __restrict__ rows, int64_t n_act, int row_vec,
-                   uint4* __restrict__ H_act, int32_t* __restrict__ y_act, float* __restrict__ lse_act,
-                   float* __restrict__ coef_act) {
+                   const float* __restrict__ coef, const int32_t* __restrict__ rows, int64_t n_act, int64_t T,
+                   int row_vec, uint4* __restrict__ H_act, int32_t* __restrict__ y_act, float* __restrict__ lse_act,
+                   float* __restrict__ coef_act, int32_t* d_status) {
   const int lane = threadIdx.x & 31;
   for (int64_t i = ((int64_t)blockIdx.x * 256 + threadIdx.x) >> 5; i < n_act; i += ((int64_t)gridDim.x * 256) >> 5) {
     const int64_t t = rows[i];
+    if (t < 0 || t >= T) {                  // a row index outside the batch: reported, never dereferenced
+      if (lane == 0) { flag(d_status, SPO_DEV_ID_OUT_OF_RANGE); y_act[i] = 0; lse_act[i] = 0.0f; coef_act[i] = 0.0f; }
+      for (int k = lane; k < row_vec; k += 32) H_act[i * row_vec + k] = make_uint4(0u, 0u, 0u, 0u);
+      continue;
+    }
     for (int k = lane; k < row_vec; k += 32) H_act[i * row_vec + k] = __ldg(H + t * row_vec + k);
     if (lane == 0) { y_act[i] = y[t]; lse_act[i] = lse[t]; coef_act[i] = coef[t]; }
   }
 }
 
 __global__ void __launch_bounds__(256)
-scatter_rows_kernel(const uint4* __restrict__ dH_act, const int32_t* __restrict__ rows, int64_t n_act, int row_vec,
-                    uint4* __restrict__ dH) {
+scatter_rows_kernel(const uint4* __restrict__ dH_act, const int32_t* __restrict__ rows, int64_t n_act, int64_t T,
+                    int row_vec, uint4* __restrict__ dH) {
   const int lane = threadIdx.x & 31;
   for (int64_t i = ((int64_t)blockIdx.x * 256 + threadIdx.x) >> 5; i < n_act; i += ((int64_t)gridDim.x * 256) >> 5) {
     const int64_t t = rows[i];
+    if (t < 0 || t >= T) continue;          // reported by the gather of the same list
     for (int k = lane; k < row_vec; k += 32) dH[t * row_vec + k] = dH_act[i * row_vec + k];
   }
 }
 
+
+// One warp per row: out[i] = rowscale[t0 + i] * H[t0 + i], bf16, 16-byte pieces.
+__global__ void __launch_bounds__(256)
+scale_rows_kernel(const uint4* __restrict__ H, const float* __restrict__ rowscale, int64_t t0, int64_t rows,
+                  int row_vec, uint4* __restrict__ out) {
+  const int lane = threadIdx.x & 31;
+  for (int64_t i = ((int64_t)blockIdx.x * 256 + threadIdx.x) >> 5; i < rows; i += ((int64_t)gridDim.x * 256) >> 5) {
+    const float rs = rowscale[t0 + i];
+    const uint4* src = H + (t0 + i) * row_vec;
+    uint4* dst = out + i * row_vec;
+    for (int k = lane; k < row_vec; k += 32) {
+      uint4 v = make_uint4(0u, 0u, 0u, 0u);
+      if (rs != 0.0f) {
+        const uint4 h = __ldg(src + k);
+        const uint32_t w[4] = {h.x, h.y, h.z, h.w};
+        uint32_t o[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const __nv_bfloat162 pr2 = __floats2bfloat162_rn(__uint_as_float(w[q] << 16) * rs,
+                                                           __uint_as_float(w[q] & 0xFFFF0000u) * rs);
+          o[q] = *reinterpret_cast<const uint32_t*>(&pr2);
+        }
+        v = make_uint4(o[0], o[1], o[2], o[3]);
+      }
+      dst[k] = v;
+    }
+  }
+}
 
 // Sequence-level objective, one block per response: r = exp(mean over its unmasked tokens of
 // logp - logp_old), term = min(r a, clip(r) a), and the coef all its unmasked tokens share.
@@ -424,7 +476,7 @@ __global__ void __launch_bounds__(256)
 seq_level_terms_kernel(const float* __restrict__ logp, const float* __restrict__ logp_old,
                        const uint8_t* __restrict__ mask, const int32_t* __restrict__ cu_seqlens,
                        const float* __restrict__ a_norm, float clip_lo, float clip_hi,
-                       const int32_t* __restrict__ counters, int32_t global_responses,
+                       const int32_t* __restrict__ counters, int32_t global_responses, float dual_clip,
                        float* __restrict__ seq_coef, double* __restrict__ seq_term) {
   const int s = blockIdx.x;
   const int64_t lo = cu_seqlens[s], hi = cu_seqlens[s + 1];
@@ -450,7 +502,11 @@ seq_level_terms_kernel(const float* __restrict__ logp, const float* __restrict__
       const double a = (double)a_norm[s];
       const double hi_b = 1.0 + (double)clip_hi, lo_b = 1.0 - (double)clip_lo;
       term = fmin(r * a, fmin(fmax(r, lo_b), hi_b) * a);
-      const bool passes = a >= 0.0 ? r <= hi_b : r >= lo_b;
+      bool passes = a >= 0.0 ? r <= hi_b : r >= lo_b;
+      if (dual_clip > 0.0f && a < 0.0) {
+        term = fmax(term, (double)dual_clip * a);
+        passes = passes && !(r > (double)dual_clip);
+      }
       if (passes) c = (float)(-a * r / ((double)s_act * tc));
     }
     seq_coef[s] = c;
@@ -498,7 +554,7 @@ seq_level_apply_kernel(const uint8_t* __restrict__ mask, const int32_t* __restri
 __global__ void __launch_bounds__(1024)
 loss_stats_kernel(const float* __restrict__ logp, const float* __restrict__ logp_old, const uint8_t* __restrict__ mask,
                   const int32_t* __restrict__ cu_seqlens, const float* __restrict__ a_norm, int64_t T, int32_t S,
-                  float clip_lo, float clip_hi, float* __restrict__ out) {
+                  float clip_lo, float clip_hi, float dual_clip, float* __restrict__ out) {
   const float hi_b = 1.0f + clip_hi, lo_b = 1.0f - clip_lo;
   double acc[6] = {0.0, 0.0, 0.0, 0.0, 0.0, 0.0};     // count, ratio, stopped, -d, k3, outside
   float rmax = -CUDART_INF_F, rmin = CUDART_INF_F;
@@ -512,7 +568,7 @@ loss_stats_kernel(const float* __restrict__ logp, const float* __restrict__ logp
     const float a = a_norm[lo];
     const float d = logp[t] - logp_old[t];
     const float r = expf(d);
-    const bool stopped = a > 0.0f ? r > hi_b : (a < 0.0f ? r < lo_b : false);
+    const bool stopped = a > 0.0f ? r > hi_b : (a < 0.0f ? (r < lo_b || (dual_clip > 0.0f && r > dual_clip)) : false);
     acc[0] += 1.0;
     acc[1] += (double)r;
     acc[2] += stopped ? 1.0 : 0.0;
@@ -581,11 +637,12 @@ compact_cu_seqlens_kernel(const int32_t* __restrict__ rows, int64_t n_act, const
 // logp / lse / coef of the compacted rows back to their places in the full arrays.
 __global__ void __launch_bounds__(256)
 scatter_scalars_kernel(const float* __restrict__ logp_act, const float* __restrict__ lse_act,
-                       const float* __restrict__ coef_act, const int32_t* __restrict__ rows, int64_t n_act,
+                       const float* __restrict__ coef_act, const int32_t* __restrict__ rows, int64_t n_act, int64_t T,
                        float* __restrict__ logp, float* __restrict__ lse, float* __restrict__ coef) {
   const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
   if (i >= n_act) return;
   const int64_t t = rows[i];
+  if (t < 0 || t >= T) return;              // reported by the gather of the same list
   logp[t] = logp_act[i];
   lse[t] = lse_act[i];
   coef[t] = coef_act[i];
@@ -619,12 +676,10 @@ cudaError_t launch_fwd_prepare(const uint8_t* mask, int64_t T, const int32_t* cu
 cudaError_t launch_fwd_finalize(const FwdPartial* partials, int nsplit, const int32_t* y,
                                 const float* logp_old, const uint8_t* mask, const int32_t* cu_seqlens,
                                 const float* a_norm, int64_t T, int32_t V, int32_t S,
-                                float clip_lo, float clip_hi,
                                 float* loss, float* logp, float* lse, float* coef, float* seq_sums, float* entropy,
-                                double* block_sums, int32_t* counters, const int32_t* seq_cnt, int agg_mode,
-                                int surrogate, int32_t global_tokens, int32_t global_responses,
+                                double* block_sums, int32_t* counters, const int32_t* seq_cnt, const spo_params& pr,
                                 int64_t fin_blocks, int32_t* d_status, cudaStream_t st,
-                                const FinalizeRange* range) {
+                                const FinalizeRange* range, const OnePassFix* fix) {
   // Default: one launch over all rows.  With a range: rows [t_begin, T) of a larger batch whose
   // blocks are numbered from block0; T is then the end of the range and the per-response sums
   // are left to the launch that covers the last rows.
@@ -637,9 +692,9 @@ cudaError_t launch_fwd_finalize(const FwdPartial* partials, int nsplit, const in
   }
   if (blocks == 0) return cudaSuccess;
   fwd_finalize_kernel<<<blocks, kFinalizeThreads, 0, st>>>(
-      partials, nsplit, y, logp_old, mask, cu_seqlens, a_norm, T, V, S, clip_lo, clip_hi,
-      loss, logp, lse, coef, entropy, block_sums, counters, seq_cnt, agg_mode, surrogate, global_tokens,
-      global_responses, d_status, rg);
+      partials, nsplit, y, logp_old, mask, cu_seqlens, a_norm, T, V, S, pr.clip_lo, pr.clip_hi,
+      loss, logp, lse, coef, entropy, block_sums, counters, seq_cnt, pr.agg_mode, pr.surrogate, pr.global_tokens,
+      pr.global_responses, pr.dual_clip, d_status, rg, fix ? *fix : OnePassFix{nullptr, 0, 0, nullptr, 0.0f});
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   if (seq_sums && S > 0 && rg.last) {
@@ -651,11 +706,12 @@ cudaError_t launch_fwd_finalize(const FwdPartial* partials, int nsplit, const in
 
 cudaError_t launch_seq_level_objective(const float* logp, const float* logp_old, const uint8_t* mask,
                                        const int32_t* cu_seqlens, const float* a_norm, int64_t T, int32_t S,
-                                       float clip_lo, float clip_hi, const int32_t* counters, int32_t global_responses,
+                                       const spo_params& pr, const int32_t* counters,
                                        float* seq_coef, double* seq_term, float* coef, float* loss, cudaStream_t st) {
+  const int32_t global_responses = pr.global_responses;
   if (S > 0) {
-    seq_level_terms_kernel<<<S, 256, 0, st>>>(logp, logp_old, mask, cu_seqlens, a_norm, clip_lo, clip_hi, counters,
-                                              global_responses, seq_coef, seq_term);
+    seq_level_terms_kernel<<<S, 256, 0, st>>>(logp, logp_old, mask, cu_seqlens, a_norm, pr.clip_lo, pr.clip_hi, counters,
+                                              global_responses, pr.dual_clip, seq_coef, seq_term);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
   }
@@ -702,22 +758,34 @@ size_t active_rows_ws_bytes(int64_t T) {
 }
 
 cudaError_t launch_gather_rows(const void* H, const int32_t* y, const float* lse, const float* coef,
-                               const int32_t* rows, int64_t n_act, int32_t row_bytes, void* H_act, int32_t* y_act,
-                               float* lse_act, float* coef_act, cudaStream_t st) {
+                               const int32_t* rows, int64_t n_act, int64_t T, int32_t row_bytes, void* H_act,
+                               int32_t* y_act, float* lse_act, float* coef_act, int32_t* d_status, cudaStream_t st) {
   if (n_act == 0) return cudaSuccess;
   int64_t blocks = ceil_div(n_act * 32, 256);
   const int64_t cap = (int64_t)sm_count() * 16;
   if (blocks > cap) blocks = cap;
-  gather_rows_kernel<<<(unsigned)blocks, 256, 0, st>>>(reinterpret_cast<const uint4*>(H), y, lse, coef, rows, n_act,
+  gather_rows_kernel<<<(unsigned)blocks, 256, 0, st>>>(reinterpret_cast<const uint4*>(H), y, lse, coef, rows, n_act, T,
                                                        row_bytes / 16, reinterpret_cast<uint4*>(H_act), y_act, lse_act,
-                                                       coef_act);
+                                                       coef_act, d_status);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_scale_rows(const void* H, const float* rowscale, int64_t t0, int64_t rows, int32_t row_bytes,
+                              void* out, cudaStream_t st) {
+  if (rows == 0) return cudaSuccess;
+  int64_t blocks = ceil_div(rows * 32, 256);
+  const int64_t cap = (int64_t)sm_count() * 16;
+  if (blocks > cap) blocks = cap;
+  scale_rows_kernel<<<(unsigned)blocks, 256, 0, st>>>(reinterpret_cast<const uint4*>(H), rowscale, t0, rows,
+                                                      row_bytes / 16, reinterpret_cast<uint4*>(out));
   return cudaGetLastError();
 }
 
 cudaError_t launch_loss_stats(const float* logp, const float* logp_old, const uint8_t* mask, const int32_t* cu_seqlens,
-                              const float* a_norm, int64_t T, int32_t S, float clip_lo, float clip_hi, float* out,
+                              const float* a_norm, int64_t T, int32_t S, const spo_params& pr, float* out,
                               cudaStream_t st) {
-  loss_stats_kernel<<<1, 1024, 0, st>>>(logp, logp_old, mask, cu_seqlens, a_norm, T, S, clip_lo, clip_hi, out);
+  loss_stats_kernel<<<1, 1024, 0, st>>>(logp, logp_old, mask, cu_seqlens, a_norm, T, S, pr.clip_lo, pr.clip_hi,
+                                        pr.dual_clip, out);
   return cudaGetLastError();
 }
 
@@ -728,21 +796,21 @@ cudaError_t launch_compact_cu_seqlens(const int32_t* rows, int64_t n_act, const 
 }
 
 cudaError_t launch_scatter_scalars(const float* logp_act, const float* lse_act, const float* coef_act,
-                                   const int32_t* rows, int64_t n_act, float* logp, float* lse, float* coef,
+                                   const int32_t* rows, int64_t n_act, int64_t T, float* logp, float* lse, float* coef,
                                    cudaStream_t st) {
   if (n_act == 0) return cudaSuccess;
-  scatter_scalars_kernel<<<(unsigned)ceil_div(n_act, 256), 256, 0, st>>>(logp_act, lse_act, coef_act, rows, n_act, logp,
-                                                                        lse, coef);
+  scatter_scalars_kernel<<<(unsigned)ceil_div(n_act, 256), 256, 0, st>>>(logp_act, lse_act, coef_act, rows, n_act, T,
+                                                                        logp, lse, coef);
   return cudaGetLastError();
 }
 
-cudaError_t launch_scatter_rows(const void* dH_act, const int32_t* rows, int64_t n_act, int32_t row_bytes, void* dH,
-                                cudaStream_t st) {
+cudaError_t launch_scatter_rows(const void* dH_act, const int32_t* rows, int64_t n_act, int64_t T, int32_t row_bytes,
+                                void* dH, cudaStream_t st) {
   if (n_act == 0) return cudaSuccess;
   int64_t blocks = ceil_div(n_act * 32, 256);
   const int64_t cap = (int64_t)sm_count() * 16;
   if (blocks > cap) blocks = cap;
-  scatter_rows_kernel<<<(unsigned)blocks, 256, 0, st>>>(reinterpret_cast<const uint4*>(dH_act), rows, n_act,
+  scatter_rows_kernel<<<(unsigned)blocks, 256, 0, st>>>(reinterpret_cast<const uint4*>(dH_act), rows, n_act, T,
                                                         row_bytes / 16, reinterpret_cast<uint4*>(dH));
   return cudaGetLastError();
 }

@@ -5,11 +5,14 @@
 //         per token row in registers across the vocabulary tiles of its split.
 //   G   : the same contraction for one chunk of token rows; epilogue turns each logit
 //         into g = c_t (1[v=y_t] - e^{z-lse_t}) and writes it as bf16 into the chunk buffer.
-//   E   : the same contraction again, for the one-pass forward+backward: epilogue keeps the
-//         forward's online statistics AND writes every logit of the chunk as
-//         e = 2^(z log2e - ref), bf16, with one reference exponent per row and 64 columns;
-//         a streaming kernel turns e into g once the row's lse is known, so the backward
-//         needs no second logits contraction.
+//   E   : the same contraction again, for the one-pass forward+backward: epilogue sums the
+//         row's exponentials AND writes every logit of the chunk as e = 2^(z log2e - ref_t),
+//         bf16, against one reference exponent per token row that is fixed before the sweep.
+//         With l_t = sum_v e the softmax is p = e / l_t, so the logit gradient factors as
+//         g[t,v] = rowscale_t * (e[t,v] - l_t 1[v = y_t]): the finalisation kernel patches the
+//         one target entry per row, and a per-row scale (in DH's epilogue, and applied to the
+//         rows of H that DW reads) does the rest -- the stored chunk is never rewritten and the
+//         backward needs no second logits contraction.
 //   DH  : dH_chunk = G W        (A = G, K-major;  B = W read as an N-major operand)
 //   DW  : dW (+)= G^T H_chunk   (A = G read as an M-major operand; B = H, N-major)
 //
@@ -39,6 +42,8 @@
 #include <math_constants.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "spo_internal.h"
 
 namespace spo {
@@ -66,23 +71,9 @@ constexpr int kEpilogueSleepNs = 64;
 constexpr int kProducerSleepNs = 32;
 
 constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kRefMargin = 40.0f;     // binary orders between a row's reference exponent and its first tile's maximum
 
 enum : int { MODE_FWD = 0, MODE_G = 1, MODE_DH = 2, MODE_DW = 3, MODE_E = 4 };
-
-// Work description of the e -> g pass of the one-pass path (see e_to_g_rows).
-struct E2gJob {
-  __nv_bfloat16* G;        // [rows][ldg]
-  int64_t ldg;
-  const float* ref;        // [n_groups][ref_ld]
-  int64_t ref_ld;
-  int64_t rows;            // rows of the chunk that exist
-  int n_groups;            // ldg / 64
-  const int32_t* y;        // per-token arrays, indexed by row0 + chunk row
-  const float* lse;
-  const float* coef;
-  float grad_loss;
-  int64_t row0;
-};
 
 struct GemmParams {
   int m_tiles, n_tiles, nsplit, per_split;   // work decomposition: unit = (row tile, split of the column tiles)
@@ -102,9 +93,10 @@ struct GemmParams {
   int64_t part_row0;                         // global row that partial 0 of a split belongs to
   __nv_bfloat16* G;
   int64_t ldg;
-  float* ref;                                // E: reference exponent of (64-column group, chunk row), [groups][ref_ld]
-  int64_t ref_ld;
-  E2gJob side;                               // E with side warps: the previous chunk's e -> g (rows = 0: nothing)
+  const FwdPartial* pre;                     // E: statistics of every row's first vocabulary tile, [2][pre_ld] (both halves)
+  int64_t pre_ld;
+  const float* rowscale;                     // DH (one-pass): factor of each output row, indexed like the output; NULL = none
+  int m_tile0;                               // added to every unit's row tile (a launch that covers a slab of row tiles)
   // DH / DW
   void* out;
   int out_bf16;
@@ -301,6 +293,23 @@ __device__ __forceinline__ void g_values(const uint32_t (&v)[32], int col0, floa
                          pack_bf16(g[8 * q + 4], g[8 * q + 5]), pack_bf16(g[8 * q + 6], g[8 * q + 7]));
 }
 
+// Two floats to a bf16 pair, infinities replaced by the largest finite value (stored exponentials
+// of a row whose logits outrun the reference must not become Inf: Inf times a zero row scale is NaN).
+__device__ __forceinline__ uint32_t pack_bf16_finite(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.satfinite.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+
+__device__ __forceinline__ void bf16_values_finite(const uint32_t (&v)[32], uint4* out4) {
+#pragma unroll
+  for (int q = 0; q < 4; ++q)
+    out4[q] = make_uint4(pack_bf16_finite(__uint_as_float(v[8 * q + 0]), __uint_as_float(v[8 * q + 1])),
+                         pack_bf16_finite(__uint_as_float(v[8 * q + 2]), __uint_as_float(v[8 * q + 3])),
+                         pack_bf16_finite(__uint_as_float(v[8 * q + 4]), __uint_as_float(v[8 * q + 5])),
+                         pack_bf16_finite(__uint_as_float(v[8 * q + 6]), __uint_as_float(v[8 * q + 7])));
+}
+
 __device__ __forceinline__ void bf16_values(const uint32_t (&v)[32], uint4* out4) {
 #pragma unroll
   for (int q = 0; q < 4; ++q)
@@ -330,82 +339,11 @@ __host__ __device__ constexpr uint32_t instr_desc(bool a_mn, bool b_mn) {
 }
 
 
-// ---------------------------------------------------------------------------
-// One-pass forward+backward, second half: once a row's lse and coef exist, the stored
-// e = 2^(z log2e - ref) of a chunk become g = c_t (1[v = y_t] - e 2^(ref - lse_t log2e)), in place.
-// Streaming: 4 bytes per logit.  The work runs either as a kernel of its own or on four extra
-// warps of the next chunk's logits contraction, whose tensor-bound CTAs leave HBM nearly idle.
-// ---------------------------------------------------------------------------
-
-// One warp, 4 rows x 64 columns per step (lane -> row r = first_row + lane/8, 16-byte piece lane%8):
-// every warp-wide access is four whole 128-byte row pieces and the four references the warp needs
-// share a sector.  Rows without gradient are zero-filled without being read.
-template <int UNROLL>
-__device__ __forceinline__ void e_to_g_rows(const E2gJob& j, int64_t first_row, int g_begin, int g_end, int lane) {
-  const int64_t r = first_row + (lane >> 3);
-  if (r >= j.rows) return;
-  const int piece = lane & 7;
-  const float c = j.grad_loss * j.coef[j.row0 + r];
-  const float lse2 = j.lse[j.row0 + r] * kLog2e;
-  const int32_t yt = j.y[j.row0 + r];
-  uint4* grow = reinterpret_cast<uint4*>(j.G + r * j.ldg) + piece;      // + 8 per 64-column group
-  const float* rrow = j.ref + r;
-  if (c == 0.0f) {
-    for (int g = g_begin; g < g_end; ++g) grow[(int64_t)g * 8] = make_uint4(0u, 0u, 0u, 0u);
-    return;
-  }
-  const float nc = -c;
-  for (int g0 = g_begin; g0 < g_end; g0 += UNROLL) {
-    uint4 v[UNROLL];
-    float sc[UNROLL];
-#pragma unroll
-    for (int i = 0; i < UNROLL; ++i) {
-      if (g0 + i < g_end) {
-        v[i] = grow[(int64_t)(g0 + i) * 8];
-        sc[i] = rrow[(int64_t)(g0 + i) * j.ref_ld];
-      }
-    }
-#pragma unroll
-    for (int i = 0; i < UNROLL; ++i) {
-      if (g0 + i < g_end) {
-        const float scale = nc * fast_exp2(sc[i] - lse2);
-        const int col0 = (g0 + i) * 64 + piece * 8;
-        uint32_t w[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
-        float f[8];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          f[2 * q] = __uint_as_float(w[q] << 16) * scale;
-          f[2 * q + 1] = __uint_as_float(w[q] & 0xFFFF0000u) * scale;
-        }
-        if (yt >= col0 && yt < col0 + 8) {
-          const int jj = yt - col0;
-#pragma unroll
-          for (int q = 0; q < 8; ++q) if (q == jj) f[q] += c;
-        }
-        grow[(int64_t)(g0 + i) * 8] = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]),
-                                                 pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
-      }
-    }
-  }
-}
-
-constexpr int kE2gThreads = 256;
-constexpr int kE2gRows = 32;            // rows per block: 8 warps x 4 rows
-constexpr int kE2gUnroll = 4;
-
-__global__ void __launch_bounds__(kE2gThreads)
-e_to_g_kernel(const E2gJob job, int groups_per_block) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int g_begin = blockIdx.y * groups_per_block;
-  e_to_g_rows<kE2gUnroll>(job, (int64_t)blockIdx.x * kE2gRows + warp * 4, g_begin,
-                          min(g_begin + groups_per_block, job.n_groups), lane);
-}
-
 struct Unit { int m_tile, n_begin, n_end; };
 __device__ __forceinline__ Unit unit_of(int u, const GemmParams& p) {
   Unit r;
   const int split = u % p.nsplit;
-  r.m_tile = u / p.nsplit;
+  r.m_tile = u / p.nsplit + p.m_tile0;
   r.n_begin = split * p.per_split;
   r.n_end = min(r.n_begin + p.per_split, p.n_tiles);
   return r;
@@ -414,16 +352,11 @@ __device__ __forceinline__ Unit unit_of(int u, const GemmParams& p) {
 // ---------------------------------------------------------------------------
 // the kernel
 // ---------------------------------------------------------------------------
-// SIDE (E only): two more warps per CTA stream the previous chunk's e -> g while this chunk's
-// logits are contracted.
-constexpr int SIDE_WARPS = 2;
-constexpr int kSideUnroll = 16;
-
 // ENT (FWD / E): also accumulate sum_v e z per row, from which the finalisation forms the entropy of
 // the row's softmax, lse - sum_v p z (one more multiply-add per logit; a separate instantiation so that
 // the kernels without it stay as they are).
-template <int MODE, bool SIDE = false, bool ENT = false>
-__global__ void __launch_bounds__(NUM_THREADS + (SIDE ? 32 * SIDE_WARPS : 0), 1)
+template <int MODE, bool ENT = false>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
 spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmParams p) {
   constexpr bool A_MN = (MODE == MODE_DW);
   constexpr bool B_MN = (MODE == MODE_DH || MODE == MODE_DW);
@@ -580,10 +513,22 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       float ez = 0.0f;                                                     // ENT: sum e z relative to m2
       int32_t yt = -1;
       float c = 0.0f, lse2 = 0.0f;                                         // G
+      float rs = 1.0f;                                                     // DH: factor of this lane's output row
       if (MODE == MODE_FWD || MODE == MODE_G || MODE == MODE_E) {
         if (row_ok) yt = p.y[grow];
         if (MODE == MODE_G && row_ok) { c = p.grad_loss * p.coef[grow]; lse2 = p.lse[grow] * kLog2e; }
+        if (MODE == MODE_E) {
+          // Reference exponent of the row: the largest logit of its first vocabulary tile (found by a
+          // short launch beforehand) plus a margin, the same for every pair and column half that works
+          // on the row.  Exponentials are taken against it without a running maximum: bf16 and fp32
+          // keep their relative precision at any magnitude, so all that matters is that nothing
+          // overflows (row maximum up to kRefMargin + 109 binary orders above the first tile's) and
+          // that entries worth keeping do not underflow (anything within 126 - kRefMargin orders
+          // below the first tile's maximum survives).
+          m2 = row_ok ? fmaxf(p.pre[grow].m2, p.pre[p.pre_ld + grow].m2) + kRefMargin : 0.0f;
+        }
       }
+      if (MODE == MODE_DH && p.rowscale && row_ok) rs = p.rowscale[grow];
       for (int n = un.n_begin; n < un.n_end && ok; ++n, ++tile) {
         {                                   // one lane polls (with backoff); the warp reconverges on its verdict
           int good = 1;
@@ -638,41 +583,29 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             }
           }
         } else if (MODE == MODE_E) {
-          // Forward statistics and the stored exponentials in one pass.  Per 64 columns the row's
-          // largest logit gives the reference: e = 2^(z log2e - ref) <= 1 keeps full bf16 precision
-          // for the entries that matter whatever the range of the logits, and ref is written once
-          // per (64-column group, row) -- lanes are consecutive rows, so the store is coalesced.
-          __nv_bfloat16* obase = p.G + ((int64_t)un.m_tile * GROUP_M + warp_row0) * p.ldg;
-          float* ref_row = p.ref + (int64_t)un.m_tile * GROUP_M + row;
+          // Sum of the row's exponentials (and sum e z with ENT) and the stored exponentials in one
+          // pass, all against the row's fixed reference m2: no running maximum, no rescaling.
+          __nv_bfloat16* obase = p.G + ((int64_t)(un.m_tile - p.m_tile0) * GROUP_M + warp_row0) * p.ldg;
+          const float neg = -m2;
 #pragma unroll 1
           for (int r2 = 0; r2 < HALF_N / 64; ++r2) {
             const int col0 = col_half + r2 * 64;
             uint4 piece[8];
-            float ref2 = 0.0f;
             if (col0 < p.cols_valid) {
               uint32_t v0[32], v1[32];
               tmem_ld32_nowait(taddr + r2 * 64, v0);
               tmem_ld32_nowait(taddr + r2 * 64 + 32, v1);
               tmem_wait_ld(v0);
               tmem_wait_ld(v1);
-              if (col0 + 64 > p.cols_valid) {                          // ragged end of the vocabulary
+              if (col0 + 64 > p.cols_valid) {                          // ragged end of the vocabulary: e = 0
 #pragma unroll
                 for (int j = 0; j < 32; ++j) {
+                  // (with ENT a large finite value instead of -inf: its e is 0 either way and 0 * z stays 0)
                   const float fill = ENT ? -1.0e30f : -CUDART_INF_F;
                   if (col0 + j >= p.cols_valid) v0[j] = __float_as_uint(fill);
                   if (col0 + 32 + j >= p.cols_valid) v1[j] = __float_as_uint(fill);
                 }
               }
-              float mx0 = __uint_as_float(v0[0]), mx1 = __uint_as_float(v0[1]);
-              float mx2 = __uint_as_float(v1[0]), mx3 = __uint_as_float(v1[1]);
-#pragma unroll
-              for (int j = 2; j < 32; j += 2) {
-                mx0 = fmaxf(mx0, __uint_as_float(v0[j]));
-                mx1 = fmaxf(mx1, __uint_as_float(v0[j + 1]));
-                mx2 = fmaxf(mx2, __uint_as_float(v1[j]));
-                mx3 = fmaxf(mx3, __uint_as_float(v1[j + 1]));
-              }
-              ref2 = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * kLog2e;
               if (yt >= col0 && yt < col0 + 64) {
                 const int jj = yt - col0;
 #pragma unroll
@@ -681,7 +614,6 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                   if (j + 32 == jj) zt = __uint_as_float(v1[j]);
                 }
               }
-              const float neg = -ref2;
               float s0 = 0.0f, s1 = 0.0f, s2 = 0.0f, s3 = 0.0f, t0 = 0.0f, t1 = 0.0f;
 #pragma unroll
               for (int j = 0; j < 32; j += 2) {
@@ -697,18 +629,14 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 v0[j] = __float_as_uint(e0); v0[j + 1] = __float_as_uint(e1);
                 v1[j] = __float_as_uint(e2); v1[j + 1] = __float_as_uint(e3);
               }
-              const float mn = fmaxf(m2, ref2);
-              const float down = fast_exp2(m2 - mn), up = fast_exp2(ref2 - mn);
-              l = fmaf(l, down, ((s0 + s1) + (s2 + s3)) * up);
-              if (ENT) ez = fmaf(ez, down, (t0 + t1) * up);
-              m2 = mn;
-              bf16_values(v0, piece);
-              bf16_values(v1, piece + 4);
+              l += (s0 + s1) + (s2 + s3);
+              if (ENT) ez += t0 + t1;
+              bf16_values_finite(v0, piece);
+              bf16_values_finite(v1, piece + 4);
             } else {                                                   // pad columns: e = 0
 #pragma unroll
               for (int q = 0; q < 8; ++q) piece[q] = make_uint4(0u, 0u, 0u, 0u);
             }
-            ref_row[(int64_t)(col0 >> 6) * p.ref_ld] = ref2;
             stage_put(stage, lane, piece);
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
@@ -738,6 +666,13 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
               g_values(v0, col0, c, lse2, yt, p.cols_valid, piece);
               g_values(v1, col0 + 32, c, lse2, yt, p.cols_valid, piece + 4);
             } else {
+              if (p.rowscale) {                    // one-pass path: the row's factor (a zero factor gives exact zeros)
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                  v0[j] = __float_as_uint(rs == 0.0f ? 0.0f : __uint_as_float(v0[j]) * rs);
+                  v1[j] = __float_as_uint(rs == 0.0f ? 0.0f : __uint_as_float(v1[j]) * rs);
+                }
+              }
               bf16_values(v0, piece);
               bf16_values(v1, piece + 4);
             }
@@ -759,6 +694,10 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             if (col0 >= p.cols_valid) break;
             uint32_t v[32];
             tmem_ld32(taddr + ch * 32, v);
+            if (MODE == MODE_DH && p.rowscale) {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(rs == 0.0f ? 0.0f : __uint_as_float(v[j]) * rs);
+            }
             uint4 piece[8];
 #pragma unroll
             for (int q = 0; q < 8; ++q) piece[q] = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
@@ -794,12 +733,6 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         p.partials[(int64_t)((u % p.nsplit) * 2 + half) * p.T + (grow - p.part_row0)] = part;
       }
     }
-  } else if (SIDE) {
-    // ------------------------------------------------------------------ side warps: e -> g of the previous chunk
-    // Plain loads and stores on memory no other role of this launch touches; no waits.
-    const int sw = warp - (2 + EPI_WARPS);
-    for (int64_t rb = (int64_t)blockIdx.x * SIDE_WARPS + sw; rb * 4 < p.side.rows; rb += (int64_t)gridDim.x * SIDE_WARPS)
-      e_to_g_rows<kSideUnroll>(p.side, rb * 4, 0, p.side.n_groups, lane);
   }
 
   // ------------------------------------------------------------------ teardown
@@ -870,22 +803,23 @@ constexpr int kLockStepWindow = 1;
 // CTA pairs that can be resident at once (one CTA per SM).
 int group_count() { return sm_count() / CG; }
 
-template <int MODE, bool SIDE = false, bool ENT = false>
-cudaError_t launch_gemm(const CUtensorMap& a, const CUtensorMap& b, const GemmParams& p_in, uint32_t* progress,
-                        cudaStream_t st) {
-  constexpr int kThreads = NUM_THREADS + (SIDE ? 32 * SIDE_WARPS : 0);
-  static int max_groups[64] = {};            // CTA pairs that can be resident together, per device (0 = not yet asked)
+// CTA pairs of this instantiation that can be resident together on a device (0 = not yet asked).
+// The kernel is persistent and its pairs pace one another, so a grid must not exceed it.  One slot
+// per device, filled once; concurrent first calls compute the same value (atomic stores).
+template <int MODE, bool ENT>
+cudaError_t resident_groups(int* out) {
+  static std::atomic<int> cached[64];
   int dev = 0;
-  cudaGetDevice(&dev);
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
   if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-  if (max_groups[dev] == 0) {
-    cudaError_t e = cudaFuncSetAttribute(spo_gemm_kernel<MODE, SIDE, ENT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+  int n = cached[dev].load(std::memory_order_acquire);
+  if (n == 0) {
+    e = cudaFuncSetAttribute(spo_gemm_kernel<MODE, ENT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (e != cudaSuccess) return e;
-    // The kernel is persistent and its pairs pace one another, so the grid must not exceed what the
-    // device can hold at one time.
     cudaLaunchConfig_t q = {};
     q.gridDim = dim3(group_count() * CG, 1, 1);
-    q.blockDim = dim3(kThreads, 1, 1);
+    q.blockDim = dim3(NUM_THREADS, 1, 1);
     q.dynamicSmemBytes = SMEM_BYTES;
     cudaLaunchAttribute qa[1];
     qa[0].id = cudaLaunchAttributeClusterDimension;
@@ -894,12 +828,22 @@ cudaError_t launch_gemm(const CUtensorMap& a, const CUtensorMap& b, const GemmPa
     qa[0].val.clusterDim.z = 1;
     q.attrs = qa;
     q.numAttrs = 1;
-    int n = 0;
-    e = cudaOccupancyMaxActiveClusters(&n, spo_gemm_kernel<MODE, SIDE, ENT>, &q);
+    e = cudaOccupancyMaxActiveClusters(&n, spo_gemm_kernel<MODE, ENT>, &q);
     if (e != cudaSuccess) return e;
     if (n < 1) return cudaErrorLaunchOutOfResources;
-    max_groups[dev] = n < group_count() ? n : group_count();
+    if (n > group_count()) n = group_count();
+    cached[dev].store(n, std::memory_order_release);
   }
+  *out = n;
+  return cudaSuccess;
+}
+
+template <int MODE, bool ENT = false>
+cudaError_t launch_gemm(const CUtensorMap& a, const CUtensorMap& b, const GemmParams& p_in, uint32_t* progress,
+                        cudaStream_t st) {
+  int max_groups = 0;
+  cudaError_t e0 = resident_groups<MODE, ENT>(&max_groups);
+  if (e0 != cudaSuccess) return e0;
   const int units = p_in.m_tiles * p_in.nsplit;
   if (units <= 0) return cudaSuccess;
   GemmParams p = p_in;
@@ -911,10 +855,10 @@ cudaError_t launch_gemm(const CUtensorMap& a, const CUtensorMap& b, const GemmPa
     if (e != cudaSuccess) return e;
     p.progress = progress;
   }
-  const int groups = units < max_groups[dev] ? units : max_groups[dev];
+  const int groups = units < max_groups ? units : max_groups;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(groups * CG, 1, 1);
-  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.blockDim = dim3(NUM_THREADS, 1, 1);
   cfg.dynamicSmemBytes = SMEM_BYTES;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
@@ -924,7 +868,7 @@ cudaError_t launch_gemm(const CUtensorMap& a, const CUtensorMap& b, const GemmPa
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, spo_gemm_kernel<MODE, SIDE, ENT>, a, b, p);
+  return cudaLaunchKernelEx(&cfg, spo_gemm_kernel<MODE, ENT>, a, b, p);
 }
 
 // Operand box heights (rows per TMA box) for K-major operands.
@@ -990,7 +934,7 @@ cudaError_t launch_fwd_bf16(const void* H, const void* W, const int32_t* y, int6
   p.partials = partials;
   p.T = T;
   p.d_status = d_status;
-  if (want_entropy) return launch_gemm<MODE_FWD, false, true>(ma, mb, p, progress, st);
+  if (want_entropy) return launch_gemm<MODE_FWD, true>(ma, mb, p, progress, st);
   return launch_gemm<MODE_FWD>(ma, mb, p, progress, st);
 }
 
@@ -1014,47 +958,48 @@ BwdWs bwd_ws_layout(int64_t T, int32_t d, int32_t V) {
 
 namespace {
 
-// The two output contractions of one chunk whose g sits in the chunk buffer:
-// dH rows of the chunk = G W, then dW (+)= G^T H_chunk.
-cudaError_t launch_chunk_dh_dw(const CUtensorMap& mG_k, const CUtensorMap& mG_mn, const CUtensorMap& mW_mn,
-                               const CUtensorMap& mH_mn, int64_t t0, int64_t rows, int64_t T, int32_t d, int32_t V,
-                               void* dH, int32_t dH_dtype, float* dW, int dw_accumulate, uint32_t* progress,
-                               int32_t* d_status, cudaStream_t st) {
+// dH rows [t0, t0 + rows) = G W, where G is the chunk buffer (one-pass path: times `rowscale`, indexed by
+// token row, in the epilogue).
+cudaError_t launch_dh(const CUtensorMap& mG_k, const CUtensorMap& mW_mn, int64_t t0, int64_t rows, int64_t T,
+                      int32_t d, int32_t V, void* dH, int32_t dH_dtype, const float* rowscale, uint32_t* progress,
+                      int32_t* d_status, cudaStream_t st) {
   const int n_tiles_d = (int)ceil_div(d, BN);
-  cudaError_t e;
-  {
-    GemmParams p{};
-    p.m_tiles = (int)ceil_div(rows, GROUP_M);
-    p.n_tiles = n_tiles_d;
-    p.nsplit = n_tiles_d;
-    p.per_split = 1;
-    p.k_blocks = (int)ceil_div(V, BK);
-    p.a_row0 = 0;
-    p.b_k0 = 0;
-    p.rows_valid = T;
-    p.cols_valid = d;
-    p.out_row0 = t0;
-    p.out = dH; p.out_bf16 = (dH_dtype == SPO_DTYPE_BF16); p.ldo = d; p.accumulate = 0;
-    p.d_status = d_status;
-    if ((e = launch_gemm<MODE_DH>(mG_k, mW_mn, p, progress, st)) != cudaSuccess) return e;
-  }
-  {
-    GemmParams p{};
-    p.m_tiles = (int)ceil_div(V, GROUP_M);
-    p.n_tiles = n_tiles_d;
-    p.nsplit = n_tiles_d;
-    p.per_split = 1;
-    p.k_blocks = (int)ceil_div(rows, BK);
-    p.a_row0 = 0;
-    p.b_k0 = (int)t0;
-    p.rows_valid = V;
-    p.cols_valid = d;
-    p.out_row0 = 0;
-    p.out = dW; p.out_bf16 = 0; p.ldo = d; p.accumulate = dw_accumulate;
-    p.d_status = d_status;
-    if ((e = launch_gemm<MODE_DW>(mG_mn, mH_mn, p, progress, st)) != cudaSuccess) return e;
-  }
-  return cudaSuccess;
+  GemmParams p{};
+  p.m_tiles = (int)ceil_div(rows, GROUP_M);
+  p.n_tiles = n_tiles_d;
+  p.nsplit = n_tiles_d;
+  p.per_split = 1;
+  p.k_blocks = (int)ceil_div(V, BK);
+  p.rows_valid = T;
+  p.cols_valid = d;
+  p.out_row0 = t0;
+  p.out = dH; p.out_bf16 = (dH_dtype == SPO_DTYPE_BF16); p.ldo = d; p.accumulate = 0;
+  p.rowscale = rowscale;
+  p.d_status = d_status;
+  return launch_gemm<MODE_DH>(mG_k, mW_mn, p, progress, st);
+}
+
+// dW (+)= G^T Hk over `rows` token rows: G is the chunk buffer read as an M-major operand, Hk the
+// matching rows of the hidden states (read from row `h_row0` of their tensor map).  `tile0`, `tiles`:
+// the slab of 256-row vocabulary tiles this launch covers (the whole vocabulary: 0, all of them).
+cudaError_t launch_dw(const CUtensorMap& mG_mn, const CUtensorMap& mH_mn, int64_t h_row0, int64_t rows, int32_t d,
+                      int32_t V, float* dW, int dw_accumulate, int tile0, int tiles, uint32_t* progress,
+                      int32_t* d_status, cudaStream_t st) {
+  const int n_tiles_d = (int)ceil_div(d, BN);
+  GemmParams p{};
+  p.m_tiles = tiles;
+  p.m_tile0 = tile0;
+  p.n_tiles = n_tiles_d;
+  p.nsplit = n_tiles_d;
+  p.per_split = 1;
+  p.k_blocks = (int)ceil_div(rows, BK);
+  p.b_k0 = (int)h_row0;
+  p.rows_valid = V;
+  p.cols_valid = d;
+  p.out_row0 = 0;
+  p.out = dW; p.out_bf16 = 0; p.ldo = d; p.accumulate = dw_accumulate;
+  p.d_status = d_status;
+  return launch_gemm<MODE_DW>(mG_mn, mH_mn, p, progress, st);
 }
 
 }  // namespace
@@ -1101,21 +1046,31 @@ cudaError_t launch_bwd_bf16(const void* H, const void* W, const int32_t* y, cons
       if ((e = launch_gemm<MODE_G>(mH_k, mW_k, p, progress, st)) != cudaSuccess) return e;
     }
     // 2) dH rows of the chunk = G W;  3) dW (+)= G^T H_chunk
-    if ((e = launch_chunk_dh_dw(mG_k, mG_mn, mW_mn, mH_mn, t0, rows, T, d, V, dH, dH_dtype, dW,
-                                (accumulate || chunk > 0) ? 1 : 0, progress, d_status, st)) != cudaSuccess)
+    if ((e = launch_dh(mG_k, mW_mn, t0, rows, T, d, V, dH, dH_dtype, nullptr, progress, d_status, st)) != cudaSuccess)
+      return e;
+    if ((e = launch_dw(mG_mn, mH_mn, t0, rows, d, V, dW, (accumulate || chunk > 0) ? 1 : 0, 0,
+                       (int)ceil_div(V, GROUP_M), progress, d_status, st)) != cudaSuccess)
       return e;
   }
   return cudaSuccess;
 }
 
 // ---------------------------------------------------------------------------
-// One-pass forward+backward.  Per chunk of token rows: E contraction (forward statistics + stored
-// exponentials) -> per-token finalisation (lse, logp, coef, loss terms) -> e -> g in place ->
-// dH, dW.  Three contractions per token instead of the four of forward-then-backward.
-// The chunks are software-pipelined over two chunk buffers: the e -> g pass of chunk c (HBM-bound)
-// rides on side warps of chunk c+1's E launch (tensor-bound), so only the last chunk pays for it:
-//   E(0) fin(0) | E(1)+e2g(0) fin(1) DH(0) DW(0) | E(2)+e2g(1) fin(2) DH(1) DW(1) | ... | e2g(n-1) DH(n-1) DW(n-1)
+// One-pass forward+backward: three contractions per token instead of the four of
+// forward-then-backward.
+//   PRE      the logits of the first vocabulary tile for all rows (0.3 % of one contraction): their
+//            row maxima fix every row's reference exponent
+//   per chunk c of token rows, into slot c % slots of the chunk buffers:
+//     E(c)     logits contraction; epilogue: sum of exponentials, target logit, e = 2^(z log2e - ref) as bf16
+//     fin(c)   lse, logp, ratio, surrogate, coef, loss terms; row scale; the target entry of e patched
+//     scale(c) the chunk's rows of H times their row scale (bf16), the operand of the dW contraction
+//     DH(c)    dH rows = rowscale * (e W)
+//   per group of `slots` chunks:  DW   dW (+)= e^T (rowscale H) over the rows of the whole group
+// Contracting dW over several chunks at once divides its read-modify-write passes over the
+// [V x d] fp32 matrix (and its accumulator drains) by that number.
 // ---------------------------------------------------------------------------
+constexpr int kDwChunkGroup = 2;
+
 FusedWs fused_ws_layout(int64_t T, int32_t d, int32_t V, int32_t S) {
   FusedWs L{};
   const BwdWs b = bwd_ws_layout(T, d, V);
@@ -1123,7 +1078,8 @@ FusedWs fused_ws_layout(int64_t T, int32_t d, int32_t V, int32_t S) {
   L.ldg = b.ldg;
   const int n_tiles_v = (int)ceil_div(V, BN);
   const int64_t t_eff = T > 0 ? T : 1;
-  L.n_buf = t_eff > L.chunk_rows ? 2 : 1;
+  const int64_t n_chunks = ceil_div(t_eff, L.chunk_rows);
+  L.slots = (int)(n_chunks < kDwChunkGroup ? n_chunks : kDwChunkGroup);
   // partials: the full chunk and the (shorter) last chunk may pick different split counts
   const int64_t full_rows = t_eff < L.chunk_rows ? ceil_div(t_eff, GROUP_M) * GROUP_M : L.chunk_rows;
   size_t part_elems = (size_t)2 * pick_fwd_split(full_rows / GROUP_M, n_tiles_v, d) * (size_t)full_rows;
@@ -1134,11 +1090,11 @@ FusedWs fused_ws_layout(int64_t T, int32_t d, int32_t V, int32_t S) {
     if (e2 > part_elems) part_elems = e2;
   }
   L.fin_blocks = ceil_div(t_eff, kFinalizeThreads);
-  L.g_bytes = align_up((size_t)L.chunk_rows * (size_t)L.ldg * 2, 256);
-  L.ref_bytes = align_up(sizeof(float) * (size_t)(L.ldg / 64) * (size_t)L.chunk_rows, 256);
   size_t off = 0;
-  L.g = off;          off += L.g_bytes * (size_t)L.n_buf;
-  L.ref = off;        off += L.ref_bytes * (size_t)L.n_buf;
+  L.g = off;          off = align_up(off + (size_t)L.slots * (size_t)L.chunk_rows * (size_t)L.ldg * 2, 256);
+  L.hs = off;         off = align_up(off + (size_t)L.slots * (size_t)L.chunk_rows * (size_t)d * 2, 256);
+  L.pre = off;        off = align_up(off + sizeof(FwdPartial) * 2 * (size_t)t_eff, 256);
+  L.rowscale = off;   off = align_up(off + sizeof(float) * (size_t)t_eff, 256);
   L.partials = off;   off = align_up(off + sizeof(FwdPartial) * part_elems, 256);
   L.progress = off;   off = align_up(off + kProgressBytes, 256);
   L.block_sums = off; off = align_up(off + sizeof(double) * (size_t)L.fin_blocks, 256);
@@ -1148,124 +1104,169 @@ FusedWs fused_ws_layout(int64_t T, int32_t d, int32_t V, int32_t S) {
   return L;
 }
 
+namespace {
+// Row tiles (of GROUP_M vocabulary rows) per slab: whole rounds of units, so that no slab ends on a
+// partly filled round of CTA pairs.
+int slab_tiles(int32_t V, int32_t d, int n_wanted, int* n_out) {
+  const int tiles = (int)ceil_div(V, GROUP_M), n_tiles_d = (int)ceil_div(d, BN), groups = group_count();
+  int g = groups, b = n_tiles_d;                       // gcd
+  while (b) { const int t = g % b; g = b; b = t; }
+  const int quantum = groups / g;                      // row tiles whose units fill the pairs a whole number of times
+  if (n_wanted < 1) n_wanted = 1;
+  int per = tiles / n_wanted / quantum * quantum;      // rounded down: the last slab takes what is left over
+  if (per < quantum) per = quantum;
+  const int n = (int)ceil_div(tiles, per);
+  *n_out = n < n_wanted ? n : n_wanted;
+  return per;
+}
+}  // namespace
+
+int dw_slab_rows(int32_t V, int32_t d, int n_wanted, int64_t* row_begin) {
+  int n = 1;
+  const int per = slab_tiles(V, d, n_wanted, &n);
+  for (int k = 0; k < n; ++k) row_begin[k] = (int64_t)k * per * GROUP_M;
+  row_begin[n] = V;                                    // slab n-1 runs to the end of the vocabulary
+  return n;
+}
+
 cudaError_t launch_fused_bf16(const FusedArgs& a, char* ws, const FusedWs& L, cudaStream_t st) {
   FwdPartial* partials = reinterpret_cast<FwdPartial*>(ws + L.partials);
+  FwdPartial* pre = reinterpret_cast<FwdPartial*>(ws + L.pre);
+  float* rowscale = reinterpret_cast<float*>(ws + L.rowscale);
   uint32_t* progress = reinterpret_cast<uint32_t*>(ws + L.progress);
   double* block_sums = reinterpret_cast<double*>(ws + L.block_sums);
   int32_t* counters = reinterpret_cast<int32_t*>(ws + L.counters);
   int32_t* seq_cnt = reinterpret_cast<int32_t*>(ws + L.seq_cnt);
+  __nv_bfloat16* gbuf = reinterpret_cast<__nv_bfloat16*>(ws + L.g);
+  __nv_bfloat16* hsbuf = reinterpret_cast<__nv_bfloat16*>(ws + L.hs);
   const spo_params& pr = *a.params;
   const int64_t T = a.T;
   const int32_t d = a.d, V = a.V;
   cudaError_t e = launch_fwd_prepare(a.mask, T, a.cu_seqlens, a.S, pr.agg_mode != 0, seq_cnt, counters, st);
   if (e != cudaSuccess) return e;
   if (T == 0) {
-    e = launch_fwd_finalize(partials, 0, a.y, a.logp_old, a.mask, a.cu_seqlens, a.a_norm, 0, V, a.S, pr.clip_lo,
-                            pr.clip_hi, a.loss, a.logp, a.lse, a.coef, a.seq_sums, a.entropy, block_sums, counters, seq_cnt,
-                            pr.agg_mode, pr.surrogate, pr.global_tokens, pr.global_responses, L.fin_blocks, a.d_status,
-                            st);
+    e = launch_fwd_finalize(partials, 0, a.y, a.logp_old, a.mask, a.cu_seqlens, a.a_norm, 0, V, a.S, a.loss, a.logp,
+                            a.lse, a.coef, a.seq_sums, a.entropy, block_sums, counters, seq_cnt, pr, L.fin_blocks,
+                            a.d_status, st);
     if (e != cudaSuccess) return e;
-    if (!a.accumulate) return cudaMemsetAsync(a.dW, 0, sizeof(float) * (size_t)V * d, st);
+    if (!a.accumulate && (e = cudaMemsetAsync(a.dW, 0, sizeof(float) * (size_t)V * d, st)) != cudaSuccess) return e;
+    if (a.n_slabs > 0 && a.events) {              // nothing to contract: every slab is final at once
+      int n = 1;
+      slab_tiles(V, d, a.n_slabs, &n);
+      for (int k = 0; k < n; ++k)
+        if ((e = cudaEventRecord(a.events[k], st)) != cudaSuccess) return e;
+    }
     return cudaSuccess;
   }
-  CUtensorMap mH_k, mW_k, mW_mn, mH_mn;
+  CUtensorMap mH_k, mW_k, mW_mn;
   if (!make_map(&mH_k, a.H, d, T, d, kBoxA) || !make_map(&mW_k, a.W, d, V, d, kBoxB) ||
-      !make_map(&mW_mn, a.W, d, V, d, 64) || !make_map(&mH_mn, a.H, d, T, d, 64))
+      !make_map(&mW_mn, a.W, d, V, d, 64))
     return cudaErrorInvalidValue;
   const int n_tiles_v = (int)ceil_div(V, BN);
   const int n_chunks = (int)ceil_div(T, L.chunk_rows);
+  const bool ent = a.entropy != nullptr;
 
-  auto chunk_rows_of = [&](int c) {
-    const int64_t t0 = (int64_t)c * L.chunk_rows;
-    return (T - t0) < L.chunk_rows ? (T - t0) : L.chunk_rows;
-  };
-  auto g_of = [&](int c) { return reinterpret_cast<__nv_bfloat16*>(ws + L.g + L.g_bytes * (size_t)(c % L.n_buf)); };
-  auto ref_of = [&](int c) { return reinterpret_cast<float*>(ws + L.ref + L.ref_bytes * (size_t)(c % L.n_buf)); };
-  auto e2g_job = [&](int c) {
-    E2gJob j{};
-    j.G = g_of(c); j.ldg = L.ldg; j.ref = ref_of(c); j.ref_ld = L.chunk_rows;
-    j.rows = chunk_rows_of(c); j.n_groups = (int)(L.ldg / 64);
-    j.y = a.y; j.lse = a.lse; j.coef = a.coef; j.grad_loss = a.grad_loss; j.row0 = (int64_t)c * L.chunk_rows;
-    return j;
-  };
-  // dH rows of chunk c = G W, then dW (+)= G^T H_chunk
-  auto dh_dw = [&](int c) -> cudaError_t {
-    const int64_t t0 = (int64_t)c * L.chunk_rows, rows = chunk_rows_of(c);
-    CUtensorMap mG_k, mG_mn;
-    if (!make_map(&mG_k, g_of(c), V, rows, L.ldg, kBoxA) || !make_map(&mG_mn, g_of(c), V, rows, L.ldg, 64))
-      return cudaErrorInvalidValue;
-    return launch_chunk_dh_dw(mG_k, mG_mn, mW_mn, mH_mn, t0, rows, T, d, V, a.dH, a.dH_dtype, a.dW,
-                              (a.accumulate || c > 0) ? 1 : 0, progress, a.d_status, st);
-  };
-
-  for (int c = 0; c < n_chunks; ++c) {
-    const int64_t t0 = (int64_t)c * L.chunk_rows, rows = chunk_rows_of(c);
-    const int m_tiles = (int)ceil_div(rows, GROUP_M);
-    const int64_t rows_pad = (int64_t)m_tiles * GROUP_M;
-    // 1) logits of chunk c: online (max, sum, target logit) per row and split, e into the chunk buffer;
-    //    its side warps turn chunk c-1's e into g
-    const int nsplit = pick_fwd_split(m_tiles, n_tiles_v, d);
-    {
-      GemmParams p{};
-      p.m_tiles = m_tiles;
-      p.n_tiles = n_tiles_v;
-      p.nsplit = nsplit;
-      p.per_split = (int)ceil_div(n_tiles_v, p.nsplit);
-      p.k_blocks = (int)ceil_div(d, BK);
-      p.a_row0 = (int)t0;
-      p.rows_valid = T;
-      p.cols_valid = V;
-      p.out_row0 = t0;
-      p.y = a.y;
-      p.partials = partials;
-      p.T = rows_pad;
-      p.part_row0 = t0;
-      p.G = g_of(c); p.ldg = L.ldg;
-      p.ref = ref_of(c); p.ref_ld = L.chunk_rows;
-      p.d_status = a.d_status;
-      const bool ent = a.entropy != nullptr;
-      if (c > 0) {
-        p.side = e2g_job(c - 1);
-        e = ent ? launch_gemm<MODE_E, true, true>(mH_k, mW_k, p, progress, st)
-                : launch_gemm<MODE_E, true, false>(mH_k, mW_k, p, progress, st);
-      } else {
-        e = ent ? launch_gemm<MODE_E, false, true>(mH_k, mW_k, p, progress, st)
-                : launch_gemm<MODE_E, false, false>(mH_k, mW_k, p, progress, st);
-      }
-      if (e != cudaSuccess) return e;
-    }
-    // 2) lse, logp, ratio, clipped surrogate and coef of chunk c's rows; loss terms per block
-    {
-      FinalizeRange rg;
-      rg.t_begin = t0;
-      rg.part_ld = rows_pad;
-      rg.block0 = (int)(t0 / kFinalizeThreads);
-      rg.total_blocks = (int)L.fin_blocks;
-      rg.last = (c == n_chunks - 1) ? 1 : 0;
-      e = launch_fwd_finalize(partials, 2 * nsplit, a.y, a.logp_old, a.mask, a.cu_seqlens, a.a_norm, t0 + rows, V,
-                              a.S, pr.clip_lo, pr.clip_hi, a.loss, a.logp, a.lse, a.coef, a.seq_sums, a.entropy, block_sums,
-                              counters, seq_cnt, pr.agg_mode, pr.surrogate, pr.global_tokens, pr.global_responses,
-                              L.fin_blocks, a.d_status, st, &rg);
-      if (e != cudaSuccess) return e;
-    }
-    // 3) the two output contractions of chunk c-1, whose g is complete now
-    if (c > 0 && (e = dh_dw(c - 1)) != cudaSuccess) return e;
-  }
-  // last chunk: e -> g as a kernel of its own, then its output contractions
+  // PRE: first vocabulary tile of every row (the forward's kernel on one column tile)
   {
-    const int c = n_chunks - 1;
-    const E2gJob job = e2g_job(c);
-    const int64_t row_blocks = ceil_div(job.rows, kE2gRows);
-    int col_blocks = (int)ceil_div((int64_t)sm_count() * 16, row_blocks);       // enough blocks to fill the device
-    if (col_blocks < 1) col_blocks = 1;
-    if (col_blocks > job.n_groups) col_blocks = job.n_groups;
-    int per = (int)ceil_div(job.n_groups, col_blocks);
-    per = (int)ceil_div(per, kE2gUnroll) * kE2gUnroll;
-    col_blocks = (int)ceil_div(job.n_groups, per);
-    dim3 grid((unsigned)row_blocks, (unsigned)col_blocks, 1);
-    e_to_g_kernel<<<grid, kE2gThreads, 0, st>>>(job, per);
-    if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    if ((e = dh_dw(c)) != cudaSuccess) return e;
+    GemmParams p{};
+    p.m_tiles = (int)ceil_div(T, GROUP_M);
+    p.n_tiles = 1;
+    p.nsplit = 1;
+    p.per_split = 1;
+    p.k_blocks = (int)ceil_div(d, BK);
+    p.rows_valid = T;
+    p.cols_valid = V;
+    p.y = a.y;
+    p.partials = pre;
+    p.T = T;
+    p.d_status = a.d_status;
+    if ((e = launch_gemm<MODE_FWD>(mH_k, mW_k, p, progress, st)) != cudaSuccess) return e;
+  }
+
+  for (int c0 = 0; c0 < n_chunks; c0 += L.slots) {
+    int64_t group_rows = 0;
+    for (int c = c0; c < n_chunks && c < c0 + L.slots; ++c) {
+      const int slot = c - c0;
+      const int64_t t0 = (int64_t)c * L.chunk_rows;
+      const int64_t rows = (T - t0) < L.chunk_rows ? (T - t0) : L.chunk_rows;
+      const int m_tiles = (int)ceil_div(rows, GROUP_M);
+      const int64_t rows_pad = (int64_t)m_tiles * GROUP_M;
+      __nv_bfloat16* G = gbuf + (size_t)slot * (size_t)L.chunk_rows * (size_t)L.ldg;
+      // E: logits of chunk c
+      const int nsplit = pick_fwd_split(m_tiles, n_tiles_v, d);
+      {
+        GemmParams p{};
+        p.m_tiles = m_tiles;
+        p.n_tiles = n_tiles_v;
+        p.nsplit = nsplit;
+        p.per_split = (int)ceil_div(n_tiles_v, p.nsplit);
+        p.k_blocks = (int)ceil_div(d, BK);
+        p.a_row0 = (int)t0;
+        p.rows_valid = T;
+        p.cols_valid = V;
+        p.out_row0 = t0;
+        p.y = a.y;
+        p.partials = partials;
+        p.T = rows_pad;
+        p.part_row0 = t0;
+        p.G = G; p.ldg = L.ldg;
+        p.pre = pre; p.pre_ld = T;
+        p.d_status = a.d_status;
+        e = ent ? launch_gemm<MODE_E, true>(mH_k, mW_k, p, progress, st)
+                : launch_gemm<MODE_E, false>(mH_k, mW_k, p, progress, st);
+        if (e != cudaSuccess) return e;
+      }
+      // fin: per-token outputs of chunk c's rows, loss terms per block, row scale, patched target entries
+      {
+        FinalizeRange rg;
+        rg.t_begin = t0;
+        rg.part_ld = rows_pad;
+        rg.block0 = (int)(t0 / kFinalizeThreads);
+        rg.total_blocks = (int)L.fin_blocks;
+        rg.last = (c == n_chunks - 1) ? 1 : 0;
+        OnePassFix fix;
+        fix.G = reinterpret_cast<uint16_t*>(G);
+        fix.ldg = L.ldg;
+        fix.g_row0 = t0;
+        fix.rowscale = rowscale;
+        fix.grad_loss = a.grad_loss;
+        e = launch_fwd_finalize(partials, 2 * nsplit, a.y, a.logp_old, a.mask, a.cu_seqlens, a.a_norm, t0 + rows, V,
+                                a.S, a.loss, a.logp, a.lse, a.coef, a.seq_sums, a.entropy, block_sums, counters, seq_cnt,
+                                pr, L.fin_blocks, a.d_status, st, &rg, &fix);
+        if (e != cudaSuccess) return e;
+      }
+      // the chunk's rows of H times their row scale, behind the rows of the group's earlier chunks
+      e = launch_scale_rows(a.H, rowscale, t0, rows, d * 2, hsbuf + (size_t)slot * (size_t)L.chunk_rows * (size_t)d, st);
+      if (e != cudaSuccess) return e;
+      // DH: rows of chunk c
+      {
+        CUtensorMap mG_k;
+        if (!make_map(&mG_k, G, V, rows, L.ldg, kBoxA)) return cudaErrorInvalidValue;
+        e = launch_dh(mG_k, mW_mn, t0, rows, T, d, V, a.dH, a.dH_dtype, rowscale, progress, a.d_status, st);
+        if (e != cudaSuccess) return e;
+      }
+      group_rows += rows;        // only the group's last chunk can be short, so the rows stay contiguous
+    }
+    // DW over the group's rows
+    CUtensorMap mG_mn, mHs_mn;
+    if (!make_map(&mG_mn, gbuf, V, group_rows, L.ldg, 64) || !make_map(&mHs_mn, hsbuf, d, group_rows, d, 64))
+      return cudaErrorInvalidValue;
+    const int tiles = (int)ceil_div(V, GROUP_M);
+    const int dw_acc = (a.accumulate || c0 > 0) ? 1 : 0;
+    if (a.n_slabs > 0 && a.events && c0 + L.slots >= n_chunks) {
+      // the last contraction of dW, slab by slab: behind each slab its rows are final
+      int n = 1;
+      const int per = slab_tiles(V, d, a.n_slabs, &n);
+      for (int k = 0; k < n; ++k) {
+        const int t_begin = k * per, t_count = k == n - 1 ? tiles - t_begin : per;
+        e = launch_dw(mG_mn, mHs_mn, 0, group_rows, d, V, a.dW, dw_acc, t_begin, t_count, progress, a.d_status, st);
+        if (e != cudaSuccess) return e;
+        if ((e = cudaEventRecord(a.events[k], st)) != cudaSuccess) return e;
+      }
+    } else {
+      e = launch_dw(mG_mn, mHs_mn, 0, group_rows, d, V, a.dW, dw_acc, 0, tiles, progress, a.d_status, st);
+      if (e != cudaSuccess) return e;
+    }
   }
   return cudaSuccess;
 }

@@ -334,13 +334,24 @@ __device__ __forceinline__ float2 load_entry(const float2* p) {
 // ---------------------------------------------------------------------------
 // Advantages: A = r - alpha/(alpha+beta) gathered by id; batch mean / std; normalise.
 // ---------------------------------------------------------------------------
-__device__ __forceinline__ float gather_advantage(const float2* __restrict__ ab, int64_t N, int32_t id, float r,
-                                                  bool& bad_id) {
-  if (id < 0 || (int64_t)id >= N) { bad_id = true; return 0.0f; }
-  float2 e = load_entry(ab + id);
-  float n = e.x + e.y;
-  float v = n > 0.0f ? e.x / n : 0.5f;
-  return r - v;
+// Estimate of one entry, alpha/(alpha+beta); 0.5 for an empty entry.  A negative or non-finite
+// entry is reported through `bad_entry` (the caller skips the element).
+__device__ __forceinline__ float entry_estimate(float2 e, bool& bad_entry) {
+  const float n = e.x + e.y;
+  if ((fminf(e.x, e.y) < 0.0f) | !(n < CUDART_INF_F)) { bad_entry = true; return 0.5f; }
+  return n > 0.0f ? e.x / n : 0.5f;
+}
+
+// Batch statistics carried through the reductions: sum, sum of squares, and the two near-zero
+// counts (as doubles: exact, and they ride the same shuffles).
+struct AdvSums { double sum, sumsq, n_lo, n_hi; };
+
+__device__ __forceinline__ void adv_accumulate(AdvSums& s, float a, float tau_lo, float tau_hi) {
+  s.sum += a;
+  s.sumsq += (double)a * a;
+  const float m = fabsf(a);
+  s.n_lo += m <= tau_lo ? 1.0 : 0.0;
+  s.n_hi += m <= tau_hi ? 1.0 : 0.0;
 }
 
 __device__ __forceinline__ double warp_sum_f64(double v) {
@@ -349,25 +360,78 @@ __device__ __forceinline__ double warp_sum_f64(double v) {
   return v;
 }
 
-// Block-wide sum of two doubles; result valid in every thread.
+// Block-wide sum of the batch statistics (fixed order); result valid in every thread.
+// s_buf: THREADS / 32 entries of shared memory.
 template <int THREADS>
-__device__ __forceinline__ void block_sum2(double& a, double& b, double* s_a, double* s_b) {
+__device__ __forceinline__ void block_sum_adv(AdvSums& v, AdvSums* s_buf) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  a = warp_sum_f64(a);
-  b = warp_sum_f64(b);
-  if (lane == 0) { s_a[warp] = a; s_b[warp] = b; }
+  v.sum = warp_sum_f64(v.sum);
+  v.sumsq = warp_sum_f64(v.sumsq);
+  v.n_lo = warp_sum_f64(v.n_lo);
+  v.n_hi = warp_sum_f64(v.n_hi);
+  if (lane == 0) s_buf[warp] = v;
   __syncthreads();
-  double ta = 0.0, tb = 0.0;
+  AdvSums t = {0.0, 0.0, 0.0, 0.0};
 #pragma unroll
-  for (int w = 0; w < THREADS / 32; ++w) { ta += s_a[w]; tb += s_b[w]; }
-  a = ta; b = tb;
+  for (int w = 0; w < THREADS / 32; ++w) {
+    t.sum += s_buf[w].sum; t.sumsq += s_buf[w].sumsq; t.n_lo += s_buf[w].n_lo; t.n_hi += s_buf[w].n_hi;
+  }
+  v = t;
   __syncthreads();
 }
 
-__device__ __forceinline__ void mean_sigma(double sum, double sumsq, int32_t B, int32_t ddof, float& mu, float& sigma,
+__device__ __forceinline__ void write_stats(float* stats, float mu, float sigma, int32_t B, float m2, const AdvSums& t) {
+  stats[0] = mu; stats[1] = sigma; stats[2] = (float)B; stats[3] = m2;
+  stats[4] = (float)t.n_lo; stats[5] = (float)t.n_hi; stats[6] = 0.0f; stats[7] = 0.0f;
+}
+
+
+// What the fused advantage + update kernels need besides the advantage inputs.
+struct UpdateArgs {
+  const float* kl;       // [B] per batch entry, or [N] per prompt (kl_is_table)
+  int kl_is_table;
+  float rho_min, rho_max, inv_d_half;
+};
+
+constexpr unsigned kBadId = 1u, kBadValue = 2u;
+
+// One batch element: A = r - v(id) from the table as it stands (Sec. 3.2: the baseline is the
+// estimate before this batch's update) and, with UPDATE, the tracker update of the same entry from
+// the value just read (Sec. 3.1), so the entry crosses the memory system once per step.
+// Out-of-range ids, negative / non-finite entries and non-finite rewards or divergences are
+// reported in `bad`; the element then contributes A = 0 and its entry stays untouched.
+template <bool UPDATE>
+__device__ __forceinline__ float advantage_element(float2* __restrict__ ab, int64_t N, int32_t id, float r, int64_t j,
+                                                   const UpdateArgs& u, unsigned& bad) {
+  if (id < 0 || (int64_t)id >= N) { bad |= kBadId; return 0.0f; }
+  float2 e = load_entry(ab + id);
+  bool bad_entry = false;
+  const float v = entry_estimate(e, bad_entry);
+  if (bad_entry | !(fabsf(r) < CUDART_INF_F)) { bad |= kBadValue; return 0.0f; }
+  if (UPDATE) {
+    const float div = u.kl_is_table ? __ldg(u.kl + id) : u.kl[j];
+    if (isnan(div)) {
+      bad |= kBadValue;                      // entry untouched; the advantage itself is well defined
+    } else {
+      float rho = exp2f(-div * u.inv_d_half);
+      rho = fminf(fmaxf(rho, u.rho_min), u.rho_max);
+      e.x = fmaf(rho, e.x, r);
+      e.y = fmaf(rho, e.y, 1.0f - r);
+      ab[id] = e;
+    }
+  }
+  return r - v;
+}
+
+__device__ __forceinline__ void flag_bad(int32_t* d_status, unsigned bad) {
+  if (bad & kBadId) flag(d_status, SPO_DEV_ID_OUT_OF_RANGE);
+  if (bad & kBadValue) flag(d_status, SPO_DEV_NONFINITE);
+}
+
+__device__ __forceinline__ void mean_sigma(const AdvSums& t, int32_t B, int32_t ddof, float& mu, float& sigma,
                                            float& m2) {
-  double m = B > 0 ? sum / B : 0.0;
-  double ss = sumsq - sum * m;                 // sum (A - mu)^2
+  double m = B > 0 ? t.sum / B : 0.0;
+  double ss = t.sumsq - t.sum * m;             // sum (A - mu)^2
   if (ss < 0.0) ss = 0.0;
   int32_t den = B - ddof;
   double var = den > 0 ? ss / den : 0.0;
@@ -376,81 +440,80 @@ __device__ __forceinline__ void mean_sigma(double sum, double sumsq, int32_t B, 
   m2 = (float)ss;
 }
 
-// Whole batch in one block: one launch for gather, statistics and normalisation.
+struct NormArgs { float norm_eps; int32_t ddof; float tau_lo, tau_hi; };
+
+// Whole batch in one block: one launch for gather, (update,) statistics and normalisation.
+template <bool UPDATE>
 __global__ void __launch_bounds__(1024)
-advantages_single_kernel(const float2* __restrict__ ab, int64_t N, const int32_t* __restrict__ ids,
+advantages_single_kernel(float2* __restrict__ ab, int64_t N, const int32_t* __restrict__ ids,
                          const float* __restrict__ r, int32_t B, float* __restrict__ a_raw,
-                         float* __restrict__ a_norm, float* __restrict__ stats, float norm_eps, int32_t ddof,
+                         float* __restrict__ a_norm, float* __restrict__ stats, NormArgs na, UpdateArgs u,
                          int32_t* d_status) {
   constexpr int PER = kAdvSingleBlockMax / 1024;
-  __shared__ double s_a[32], s_b[32];
+  __shared__ AdvSums s_buf[32];
   float a[PER];
-  double sum = 0.0, sumsq = 0.0;
-  bool bad = false;
+  AdvSums t = {0.0, 0.0, 0.0, 0.0};
+  unsigned bad = 0;
 #pragma unroll
   for (int j = 0; j < PER; ++j) {
     int i = j * 1024 + threadIdx.x;
     a[j] = 0.0f;
     if (i < B) {
-      a[j] = gather_advantage(ab, N, ids[i], r[i], bad);
-      sum += a[j];
-      sumsq += (double)a[j] * a[j];
+      a[j] = advantage_element<UPDATE>(ab, N, ids[i], r[i], i, u, bad);
+      adv_accumulate(t, a[j], na.tau_lo, na.tau_hi);
       if (a_raw) a_raw[i] = a[j];
     }
   }
-  if (bad) flag(d_status, SPO_DEV_ID_OUT_OF_RANGE);
-  block_sum2<1024>(sum, sumsq, s_a, s_b);
+  flag_bad(d_status, bad);
+  block_sum_adv<1024>(t, s_buf);
   float mu, sigma, m2;
-  mean_sigma(sum, sumsq, B, ddof, mu, sigma, m2);
-  const float inv = 1.0f / (sigma + norm_eps);
+  mean_sigma(t, B, na.ddof, mu, sigma, m2);
+  const float inv = 1.0f / (sigma + na.norm_eps);
 #pragma unroll
   for (int j = 0; j < PER; ++j) {
     int i = j * 1024 + threadIdx.x;
     if (i < B) a_norm[i] = (a[j] - mu) * inv;
   }
-  if (stats && threadIdx.x == 0) { stats[0] = mu; stats[1] = sigma; stats[2] = (float)B; stats[3] = m2; }
+  if (stats && threadIdx.x == 0) write_stats(stats, mu, sigma, B, m2, t);
 }
 
-// Large batches, pass 1: raw advantages (stored into `tmp`) and per-block (sum, sum of squares).
+// Large batches, pass 1: raw advantages (stored into `tmp`), the update of the entries when fused,
+// and per-block statistics.
+template <bool UPDATE>
 __global__ void __launch_bounds__(256)
-advantages_partial_kernel(const float2* __restrict__ ab, int64_t N, const int32_t* __restrict__ ids,
+advantages_partial_kernel(float2* __restrict__ ab, int64_t N, const int32_t* __restrict__ ids,
                           const float* __restrict__ r, int32_t B, float* __restrict__ tmp,
-                          double2* __restrict__ partials, int32_t* d_status) {
-  __shared__ double s_a[8], s_b[8];
-  double sum = 0.0, sumsq = 0.0;
-  bool bad = false;
+                          AdvSums* __restrict__ partials, NormArgs na, UpdateArgs u, int32_t* d_status) {
+  __shared__ AdvSums s_buf[8];
+  AdvSums t = {0.0, 0.0, 0.0, 0.0};
+  unsigned bad = 0;
   for (int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x; i < B; i += (int64_t)gridDim.x * 256) {
-    float a = gather_advantage(ab, N, ids[i], r[i], bad);
+    const float a = advantage_element<UPDATE>(ab, N, ids[i], r[i], i, u, bad);
     tmp[i] = a;
-    sum += a;
-    sumsq += (double)a * a;
+    adv_accumulate(t, a, na.tau_lo, na.tau_hi);
   }
-  if (bad) flag(d_status, SPO_DEV_ID_OUT_OF_RANGE);
-  block_sum2<256>(sum, sumsq, s_a, s_b);
-  if (threadIdx.x == 0) partials[blockIdx.x] = make_double2(sum, sumsq);
+  flag_bad(d_status, bad);
+  block_sum_adv<256>(t, s_buf);
+  if (threadIdx.x == 0) partials[blockIdx.x] = t;
 }
 
 // Pass 2: every block folds the partials in the same fixed order, then normalises its span.
 __global__ void __launch_bounds__(256)
-advantages_normalise_kernel(const double2* __restrict__ partials, int n_partials, const float* tmp,
-                            int32_t B, float* a_norm, float* __restrict__ stats, float norm_eps,
-                            int32_t ddof) {
-  __shared__ double s_a[8], s_b[8];
-  double sum = 0.0, sumsq = 0.0;
+advantages_normalise_kernel(const AdvSums* __restrict__ partials, int n_partials, const float* tmp,
+                            int32_t B, float* a_norm, float* __restrict__ stats, NormArgs na) {
+  __shared__ AdvSums s_buf[8];
+  AdvSums t = {0.0, 0.0, 0.0, 0.0};
   for (int i = threadIdx.x; i < n_partials; i += 256) {
-    double2 p = partials[i];
-    sum += p.x;
-    sumsq += p.y;
+    const AdvSums p = partials[i];
+    t.sum += p.sum; t.sumsq += p.sumsq; t.n_lo += p.n_lo; t.n_hi += p.n_hi;
   }
-  block_sum2<256>(sum, sumsq, s_a, s_b);
+  block_sum_adv<256>(t, s_buf);
   float mu, sigma, m2;
-  mean_sigma(sum, sumsq, B, ddof, mu, sigma, m2);
-  const float inv = 1.0f / (sigma + norm_eps);
+  mean_sigma(t, B, na.ddof, mu, sigma, m2);
+  const float inv = 1.0f / (sigma + na.norm_eps);
   for (int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x; i < B; i += (int64_t)gridDim.x * 256)
     a_norm[i] = (tmp[i] - mu) * inv;
-  if (stats && blockIdx.x == 0 && threadIdx.x == 0) {
-    stats[0] = mu; stats[1] = sigma; stats[2] = (float)B; stats[3] = m2;
-  }
+  if (stats && blockIdx.x == 0 && threadIdx.x == 0) write_stats(stats, mu, sigma, B, m2, t);
 }
 
 // ---------------------------------------------------------------------------
@@ -675,23 +738,32 @@ int adv_blocks(int32_t B) {
   return (int)want;
 }
 
-cudaError_t launch_advantages(const float* ab, int64_t N, const int32_t* ids, const float* r, int32_t B,
-                              float* a_raw, float* a_norm, float* stats, char* ws,
-                              float norm_eps, int32_t ddof, int32_t* d_status, cudaStream_t st) {
-  const float2* ab2 = reinterpret_cast<const float2*>(ab);
-  if (B <= kAdvSingleBlockMax) {
-    advantages_single_kernel<<<1, 1024, 0, st>>>(ab2, N, ids, r, B, a_raw, a_norm, stats, norm_eps, ddof, d_status);
+// Advantages of a batch (and, with `upd`, the tracker update of the same entries in the same pass).
+// partials: scratch for adv_blocks(B) block records when B exceeds one block's capacity.
+cudaError_t launch_advantages(float* ab, int64_t N, const int32_t* ids, const float* r, int32_t B,
+                              float* a_raw, float* a_norm, float* stats, void* partials, const spo_params& pr,
+                              const AdvUpdate* upd, bool force_two_pass, int32_t* d_status, cudaStream_t st) {
+  float2* ab2 = reinterpret_cast<float2*>(ab);
+  const NormArgs na = {pr.norm_eps, pr.norm_ddof, pr.near_zero_tau_lo, pr.near_zero_tau_hi};
+  UpdateArgs u = {nullptr, 0, pr.rho_min, pr.rho_max, 1.0f / pr.d_half};
+  if (upd) { u.kl = upd->kl; u.kl_is_table = upd->kl_is_table; }
+  if (B <= kAdvSingleBlockMax && !force_two_pass) {
+    if (upd) advantages_single_kernel<true><<<1, 1024, 0, st>>>(ab2, N, ids, r, B, a_raw, a_norm, stats, na, u, d_status);
+    else advantages_single_kernel<false><<<1, 1024, 0, st>>>(ab2, N, ids, r, B, a_raw, a_norm, stats, na, u, d_status);
     return cudaGetLastError();
   }
   const int blocks = adv_blocks(B);
-  double2* partials = reinterpret_cast<double2*>(ws);
+  AdvSums* part = reinterpret_cast<AdvSums*>(partials);
   float* tmp = a_raw ? a_raw : a_norm;
-  advantages_partial_kernel<<<blocks, 256, 0, st>>>(ab2, N, ids, r, B, tmp, partials, d_status);
+  if (upd) advantages_partial_kernel<true><<<blocks, 256, 0, st>>>(ab2, N, ids, r, B, tmp, part, na, u, d_status);
+  else advantages_partial_kernel<false><<<blocks, 256, 0, st>>>(ab2, N, ids, r, B, tmp, part, na, u, d_status);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  advantages_normalise_kernel<<<blocks, 256, 0, st>>>(partials, blocks, tmp, B, a_norm, stats, norm_eps, ddof);
+  advantages_normalise_kernel<<<blocks, 256, 0, st>>>(part, blocks, tmp, B, a_norm, stats, na);
   return cudaGetLastError();
 }
+
+size_t adv_partial_bytes(int32_t B) { return align_up(sizeof(AdvSums) * (size_t)adv_blocks(B), 256); }
 
 cudaError_t launch_tracker_update(float* ab, int64_t N, const int32_t* ids, const float* r,
                                   const float* kl, int kl_is_table, int32_t B,
@@ -717,16 +789,16 @@ namespace {
 
 constexpr int kStaticAdvMaxBlocks = 1024;
 
-// Per-block (sum, sum of squares) partials of pass 1.  Lives in every GPU context that
-// loads this library, 16 KB, until the process exits.  In host code this name is only a
-// handle for cudaGetSymbolAddress, never a device address.
-static __device__ __align__(256) double2 g_adv_static_scratch[kStaticAdvMaxBlocks];
+// Per-block statistics records of pass 1.  Lives in every GPU context that loads this
+// library, 32 KB, until the process exits.  In host code this name is only a handle for
+// cudaGetSymbolAddress, never a device address.
+static __device__ __align__(256) AdvSums g_adv_static_scratch[kStaticAdvMaxBlocks];
 
 std::mutex g_adv_static_mutex;
-double2* g_adv_static_ptr[64] = {};
+AdvSums* g_adv_static_ptr[64] = {};
 
 // Device address of the scratch array for the current device (looked up once per device).
-cudaError_t adv_static_scratch(double2** out) {
+cudaError_t adv_static_scratch(AdvSums** out) {
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
@@ -736,7 +808,7 @@ cudaError_t adv_static_scratch(double2** out) {
     void* ptr = nullptr;
     e = cudaGetSymbolAddress(&ptr, g_adv_static_scratch);
     if (e != cudaSuccess) return e;
-    g_adv_static_ptr[dev] = static_cast<double2*>(ptr);
+    g_adv_static_ptr[dev] = static_cast<AdvSums*>(ptr);
   }
   *out = g_adv_static_ptr[dev];
   return cudaSuccess;
@@ -758,20 +830,14 @@ extern "C" int32_t spo_advantages_static(const float* ab, int64_t N, const int32
                         reinterpret_cast<uintptr_t>(a_norm) | reinterpret_cast<uintptr_t>(stats);
   if (all & 15u) return SPO_ERR_BAD_ALIGNMENT;
   if (!device_is_sm100()) return SPO_ERR_UNSUPPORTED_ARCH;
-  double2* partials = nullptr;
+  AdvSums* partials = nullptr;
   cudaError_t e = adv_static_scratch(&partials);
-  if (e != cudaSuccess) return SPO_ERR_CUDA;
-  int blocks = adv_blocks(B);
-  if (blocks > kStaticAdvMaxBlocks) blocks = kStaticAdvMaxBlocks;
-  cudaStream_t st = (cudaStream_t)stream;
-  const float2* ab2 = reinterpret_cast<const float2*>(ab);
-  float* tmp = a_raw ? a_raw : a_norm;
+  if (e != cudaSuccess) return record_cuda_error(e);
+  if (adv_blocks(B) > kStaticAdvMaxBlocks) return SPO_ERR_BAD_SHAPE;
   // Pass 1 overwrites partials[0..blocks) and pass 2 reads exactly those, so nothing left
   // over from an earlier call is ever read and nothing needs clearing.
-  advantages_partial_kernel<<<blocks, 256, 0, st>>>(ab2, N, ids, r, B, tmp, partials, d_status);
-  if ((e = cudaGetLastError()) != cudaSuccess) return SPO_ERR_CUDA;
-  advantages_normalise_kernel<<<blocks, 256, 0, st>>>(partials, blocks, tmp, B, a_norm, stats, params->norm_eps,
-                                                      params->norm_ddof);
-  if ((e = cudaGetLastError()) != cudaSuccess) return SPO_ERR_CUDA;
+  e = launch_advantages(const_cast<float*>(ab), N, ids, r, B, a_raw, a_norm, stats, partials, *params, nullptr,
+                        /*force_two_pass=*/true, d_status, (cudaStream_t)stream);
+  if (e != cudaSuccess) return record_cuda_error(e);
   return SPO_OK;
 }

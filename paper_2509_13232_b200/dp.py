@@ -4,7 +4,7 @@ Each rank holds its share of the mini-batch's responses and the replicated W and
 Three small exchanges make the ranks' results those of the whole mini-batch:
 
   1. advantage statistics: every rank calls spo_advantages for its raw advantages and
-     (mu, sigma, B, M2); `global_advantage_stats` gathers the 16-byte records, merges them and
+     (mu, sigma, B, M2, near-zero counts); `global_advantage_stats` gathers the 32-byte records, merges them and
      returns the mini-batch mu and sigma for spo_advantages_apply;
   2. denominators of the objective: `global_counts` sums the ranks' unmasked-token and active-
      response counts; they go into spo_params.global_tokens / global_responses;
@@ -41,7 +41,7 @@ def sigma_from(m2, n, ddof=0):
 
 
 def global_advantage_stats(stats, ddof=0, group=None):
-    """`stats` is this rank's [4] tensor (mu, sigma, B, M2) from spo_advantages.  Returns the
+    """`stats` is this rank's [8] tensor (mu, sigma, B, M2, n_lo, n_hi, 0, 0) from spo_advantages.  Returns the
     mini-batch (mu, sigma) as Python floats, identical on every rank."""
     import torch
     import torch.distributed as dist
@@ -72,3 +72,64 @@ def allreduce_sum(tensor, group=None):
     if dist.is_initialized() and dist.get_world_size(group) > 1:
         dist.all_reduce(tensor, op=dist.ReduceOp.SUM, group=group)
     return tensor
+
+
+def partition_by_tokens(lengths, world):
+    """Responses of one mini-batch dealt to `world` ranks so that the ranks' token counts are as even
+    as a greedy pass makes them: longest response first, each to the rank that holds the fewest tokens
+    so far (ties: lowest rank).  Returns one ascending list of response indices per rank; every rank
+    computes the same partition from the same lengths."""
+    order = sorted(range(len(lengths)), key=lambda i: (-int(lengths[i]), i))
+    load = [0] * world
+    parts = [[] for _ in range(world)]
+    for i in order:
+        r = min(range(world), key=lambda k: (load[k], k))
+        parts[r].append(i)
+        load[r] += int(lengths[i])
+    return [sorted(p) for p in parts]
+
+
+def slab_schedule(row_begin):
+    """(slab index, first row, end row) in the order the slabs of dW become final."""
+    return [(k, int(row_begin[k]), int(row_begin[k + 1])) for k in range(len(row_begin) - 1)]
+
+
+class SlabAllReduce:
+    """Sums dW over the ranks slab by slab while its last contraction still runs.
+
+    spo_loss_fwd_bwd_slabs records events[k] on the compute stream once rows row_begin[k] ..
+    row_begin[k+1]-1 of dW are final.  `reduce` makes a second stream wait for each event in turn and
+    issues the all-reduce of that slab there, so the transfer of slab k overlaps the contraction of
+    slab k+1; `finish` makes the compute stream wait for the last reduction.  Only torch.distributed
+    collectives are used (NCCL on GPUs); no kernel of the library reads another rank's memory.
+    """
+
+    def __init__(self, row_begin, device, group=None):
+        import torch
+        self.row_begin = [int(x) for x in row_begin]
+        self.group = group
+        self.stream = torch.cuda.Stream(device=device)
+        self.events = []
+        for _ in range(len(self.row_begin) - 1):
+            ev = torch.cuda.Event(enable_timing=False)
+            ev.record()                    # a torch event owns its CUDA event only after its first record
+            self.events.append(ev)
+        self.done = torch.cuda.Event(enable_timing=False)
+        self.works = []
+
+    def reduce(self, dW):
+        import torch
+        import torch.distributed as dist
+        self.works = []
+        with torch.cuda.stream(self.stream):
+            for k, lo, hi in slab_schedule(self.row_begin):
+                self.stream.wait_event(self.events[k])
+                if dist.is_initialized() and dist.get_world_size(self.group) > 1:
+                    self.works.append(dist.all_reduce(dW[lo:hi], op=dist.ReduceOp.SUM, group=self.group, async_op=True))
+            for w in self.works:
+                w.wait()                   # stream-level wait: the side stream orders behind the collectives
+            self.done.record(self.stream)
+
+    def finish(self):
+        import torch
+        torch.cuda.current_stream().wait_event(self.done)

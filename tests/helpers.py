@@ -104,7 +104,9 @@ def oracle_loss(lb, params=None, grad_loss=1.0, mask_none=False):
     mask = None if mask_none else lb.mask
     agg = 0 if params is None else int(params.agg_mode)
     sur = 0 if params is None else int(params.surrogate)
-    fwd = O.loss_forward(lb.h, lb.w, lb.y, lb.logp_old, mask, lb.cu_seqlens, lb.a_norm, clip_lo, clip_hi, agg, sur)
+    dual = None if params is None or params.dual_clip == 0.0 else float(np.float32(params.dual_clip))
+    fwd = O.loss_forward(lb.h, lb.w, lb.y, lb.logp_old, mask, lb.cu_seqlens, lb.a_norm, clip_lo, clip_hi, agg, sur,
+                         dual)
     dh, dw = O.loss_backward(lb.h, lb.w, lb.y, fwd["lse"], fwd["coef"], grad_loss)
     fwd["dH"], fwd["dW"] = dh, dw
     return fwd

@@ -47,7 +47,7 @@ def test_two_emulated_ranks_equal_the_whole_mini_batch(agg, one_pass):
     for s0, s1 in splits:
         a_raw = torch.empty(s1 - s0, dtype=torch.float32, device="cuda")
         a_tmp = torch.empty_like(a_raw)
-        stats = torch.zeros(4, dtype=torch.float32, device="cuda")
+        stats = torch.zeros(8, dtype=torch.float32, device="cuda")
         B.spo_advantages(ab_t, dev(ids[s0:s1]), dev(rewards[s0:s1]), a_raw, a_tmp, stats, ws_bytes(B.WS_ADVANTAGES, B=s1 - s0),
                          p0, status_word())
         torch.cuda.synchronize()

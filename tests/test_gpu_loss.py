@@ -108,6 +108,14 @@ def test_bf16_uniform_logits_and_bad_target():
     got = run_loss(lb)
     assert got["status"] & 1
     assert np.isneginf(got["logp"][3]) and got["coef"][3] == 0.0
+    # a masked row may carry an ignore-index target: no gradient, no status bit
+    lb.y[3] = -100
+    lb.mask[3] = 0
+    for one_pass in (False, True):
+        got = run_loss(lb, one_pass=one_pass)
+        assert got["status"] == 0 and got["coef"][3] == 0.0 and np.all(got["dH"][3] == 0.0)
+        keep = np.arange(len(lb.y)) != 3
+        np.testing.assert_allclose(got["logp"][keep], -np.log(300.0), atol=1e-5)
 
 
 def test_empty_batch_is_a_no_op_with_zero_loss():
@@ -267,6 +275,42 @@ def test_backward_over_active_rows_only(dh_f32):
     assert np.all(got_dh[inactive] == 0.0)
     assert rel_fro(got_dh, want["dH"]) <= 1e-2
     assert rel_fro(dW.cpu().numpy(), want["dW"]) <= 1e-2
+
+
+def test_row_lists_with_an_index_outside_the_batch_are_reported_not_dereferenced():
+    """spo_loss_bwd_rows / spo_loss_fwd_bwd_rows take the row list from the caller: an entry outside
+    [0, T) (a stale list, a list of another batch) sets the status bit and is skipped."""
+    import torch
+    from paper_2509_13232_b200 import binding as B
+    from tests.helpers import dev, status_word, ws_bytes
+    lb = _clip_batch(42, [60, 68], 64, 300, True)
+    T, d, V, S = 128, 64, 300, 2
+    H, W = dev(lb.h, torch.bfloat16), dev(lb.w, torch.bfloat16)
+    y, lo, cu, an = dev(lb.y), dev(lb.logp_old), dev(lb.cu_seqlens), dev(lb.a_norm)
+    f32 = dict(dtype=torch.float32, device="cuda")
+    rows_host = np.arange(0, T, 2, dtype=np.int32)
+    p = B.default_params()
+    for bad in (-1, T, 2 ** 31 - 1):
+        rows_bad = rows_host.copy()
+        rows_bad[5] = bad
+        rows = dev(rows_bad)
+        n = len(rows_bad)
+        loss = torch.zeros(4, **f32)
+        logp, lse, coef = (torch.zeros(T, **f32) for _ in range(3))
+        dH = torch.zeros((T, d), dtype=torch.bfloat16, device="cuda")
+        dW = torch.zeros((V, d), **f32)
+        st = status_word()
+        B.spo_loss_fwd_bwd_rows(H, W, y, lo, cu, an, rows, n, 1.0, loss, logp, lse, coef, None, dH, dW, 0,
+                                ws_bytes(B.WS_LOSS_FWD_BWD_ROWS, T=n, d=d, V=V, B=S), p, st)
+        torch.cuda.synchronize()
+        assert int(st[0].item()) & B.DEV_ID_OUT_OF_RANGE
+        assert torch.isfinite(dW).all() and torch.isfinite(dH.float()).all()
+        st = status_word()
+        B.spo_loss_bwd_rows(H, W, y, lse, coef, 1.0, rows, n, dH, dW, 0,
+                            ws_bytes(B.WS_LOSS_BWD_ROWS, T=n, d=d, V=V), p, st)
+        torch.cuda.synchronize()
+        assert int(st[0].item()) & B.DEV_ID_OUT_OF_RANGE
+        assert torch.isfinite(dW).all() and torch.isfinite(dH.float()).all()
 
 
 def test_backward_over_active_rows_with_nothing_active():

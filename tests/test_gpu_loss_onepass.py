@@ -2,11 +2,11 @@
 
 Same oracle, same inputs and same tolerances as the two-call path (bf16: loss / logp / lse within
 2e-3 absolute, gradients within 1e-2 relative Frobenius error; fp32: 1e-4 / 1e-4).  The one-pass
-path stores the logits of a chunk as bf16 exponentials relative to a per-row, per-64-column
-reference, so two things are checked beyond plain parity: the gradients keep their accuracy when
-the logits span a wide range (a peaked, trained-model-like distribution), and everything the
+path stores the logits of a chunk as bf16 exponentials relative to one reference exponent per
+row, so three things are checked beyond plain parity: the gradients keep their accuracy when
+the logits span a wide range (a peaked, trained-model-like distribution), everything the
 forward reports is independent of that storage (it agrees with the two-call forward to fp32
-rounding).
+rounding), and a row whose logits outrun its reference is reported and skipped.
 """
 
 import numpy as np
@@ -73,8 +73,8 @@ def test_forward_outputs_agree_with_the_two_call_path():
 @pytest.mark.parametrize("w_std", [0.5, 2.0])
 def test_wide_logit_range_keeps_gradient_accuracy(w_std):
     """Logits spanning tens to hundreds of nats (peaked rows, as a trained model gives): the stored
-    exponentials are relative to each 64-column group's own maximum, so the probabilities that
-    carry the gradient keep bf16 relative accuracy."""
+    exponentials are taken against one reference per row and bf16 keeps its relative precision at
+    any magnitude, so the probabilities that carry the gradient keep bf16 relative accuracy."""
     lb = inputs.loss_batch(133, [260, 300], 64, 3000, w_std, True, 0.1, target="softmax")
     z = lb.h.astype(np.float64) @ lb.w.astype(np.float64).T
     assert np.ptp(z, axis=1).mean() > 20.0
@@ -86,6 +86,34 @@ def test_wide_logit_range_keeps_gradient_accuracy(w_std):
     np.testing.assert_allclose(got["logp"], want["logp"], rtol=0, atol=tol)
     assert rel_fro(got["dH"], want["dH"]) <= 1e-2
     assert rel_fro(got["dW"], want["dW"]) <= 1e-2
+
+
+def test_a_row_that_outruns_its_reference_exponent_is_reported_and_skipped():
+    """The reference exponent of a row comes from its first 512 logits; a logit more than ~100 nats
+    above them overflows the stored exponentials.  Such a row must set the status bit, get
+    lse = Inf / logp = -Inf / coef = 0 and leave every gradient finite and, for all other rows,
+    equal to the oracle's with that row's coefficient zeroed.  (The two-call path has no such limit.)"""
+    from paper_2509_13232_b200 import binding as B
+    lb = inputs.loss_batch(134, [150, 170], 64, 1500, 0.05, True, 0.1, target="softmax")
+    t0, v0 = 77, 1000                                   # token row and a vocabulary row beyond the first tile
+    u = np.zeros(64, dtype=np.float32)
+    u[3] = 12.0
+    lb.h[t0], lb.w[v0] = u, u                           # logit 144 there; the other rows see at most |12 h_3| < 60
+    got = run_loss(lb, one_pass=True)
+    assert got["status"] == B.DEV_NONFINITE
+    assert np.isposinf(got["lse"][t0]) and np.isneginf(got["logp"][t0]) and got["coef"][t0] == 0.0
+    assert np.all(got["dH"][t0] == 0.0) and np.all(np.isfinite(got["dH"])) and np.all(np.isfinite(got["dW"]))
+    fwd = O.loss_forward(lb.h, lb.w, lb.y, lb.logp_old, lb.mask, lb.cu_seqlens, lb.a_norm)
+    keep = np.arange(lb.h.shape[0]) != t0
+    np.testing.assert_allclose(got["logp"][keep], fwd["logp"][keep], rtol=0, atol=4e-3)
+    coef = fwd["coef"].copy()
+    coef[t0] = 0.0
+    dh, dw = O.loss_backward(lb.h, lb.w, lb.y, fwd["lse"], coef)
+    assert rel_fro(got["coef"], coef) <= 1e-2
+    assert rel_fro(got["dH"], dh) <= 1e-2 and rel_fro(got["dW"], dw) <= 1e-2
+    # the two calls handle the same batch without a flag
+    two = run_loss(lb, one_pass=False)
+    assert two["status"] == 0 and abs(two["logp"][t0] - fwd["logp"][t0]) <= 2e-2
 
 
 def test_bf16_uniform_logits_and_bad_target():

@@ -66,7 +66,7 @@ def gpu_advantages(ab_t, ids, r, params, want_raw=True):
     b = len(ids)
     a_raw = torch.empty(b, dtype=torch.float32, device="cuda") if want_raw else None
     a_norm = torch.empty(b, dtype=torch.float32, device="cuda")
-    stats = torch.zeros(4, dtype=torch.float32, device="cuda")
+    stats = torch.zeros(8, dtype=torch.float32, device="cuda")
     st = status_word()
     ws = ws_bytes(B().WS_ADVANTAGES, B=b)
     B().spo_advantages(ab_t, dev(ids), dev(r), a_raw, a_norm, stats, ws, params, st)
@@ -368,3 +368,136 @@ def test_sampling_weights_over_thirty_decades_of_table_magnitudes():
     assert st == 0
     eps = np.float32(p.eps_explore)
     assert w.min() >= eps and w.max() <= np.float32(0.5) + eps          # the range Eq. "sampling_coef" gives
+
+
+def gpu_advantages_update(ab_t, ids, r, kl, is_table, params, want_raw=True):
+    import torch
+    b = len(ids)
+    a_raw = torch.full((b,), float("nan"), dtype=torch.float32, device="cuda") if want_raw else None
+    a_norm = torch.full((b,), float("nan"), dtype=torch.float32, device="cuda")
+    stats = torch.zeros(8, dtype=torch.float32, device="cuda")
+    st = status_word()
+    ws = ws_bytes(B().WS_ADVANTAGES, B=b)
+    B().spo_advantages_update(ab_t, dev(ids), dev(r), dev(kl), is_table, a_raw, a_norm, stats, ws, params, st)
+    torch.cuda.synchronize()
+    return (None if a_raw is None else a_raw.cpu().numpy()), a_norm.cpu().numpy(), stats.cpu().numpy(), int(st[0].item())
+
+
+@pytest.mark.parametrize("n,b,is_table", [(1_000_000, 4096, 1), (300_000, 200_000, 0), (50, 7, 0), (40_000, 8193, 1)])
+def test_fused_advantage_and_update_equals_the_two_steps_in_the_papers_order(n, b, is_table):
+    """One pass over the batch's entries: the advantage is formed from the estimate as read
+    (before this batch's update), then the entry is updated -- Algorithm 1's order.  Single-block
+    and two-pass sizes, divergences per entry and per prompt."""
+    rng = np.random.default_rng(900 + b)
+    ab = rng.uniform(0.1, 12.0, (n, 2)).astype(np.float32)
+    ab[rng.integers(0, n, max(1, n // 50))] = 0.0                  # some empty entries (v = 0.5, then v = r)
+    ids = rng.permutation(n)[:b].astype(np.int32)
+    a64, b64 = ab[:, 0].astype(np.float64), ab[:, 1].astype(np.float64)
+    v = O.value_estimate(a64, b64)
+    r = (rng.random(b) < v[ids]).astype(np.float32)
+    kl_table = rng.lognormal(-4, 1, n).astype(np.float32)
+    kl = kl_table[ids]
+    p = B().default_params(norm_ddof=1 if b == 8193 else 0)
+    ab_t = dev(ab)
+    a_raw, a_norm, stats, st = gpu_advantages_update(ab_t, ids, r, kl_table if is_table else kl, is_table, p,
+                                                     want_raw=(b != 8193))
+    assert st == 0
+    want_raw = O.raw_advantage(a64, b64, ids, r)
+    want_norm, mu, sigma = O.normalise_advantages(want_raw, p.norm_ddof, float(np.float32(p.norm_eps)))
+    if a_raw is not None:
+        np.testing.assert_allclose(a_raw, want_raw, rtol=RTOL, atol=ATOL)
+    np.testing.assert_allclose(a_norm, want_norm, rtol=RTOL, atol=2e-6)
+    np.testing.assert_allclose(stats[:3], [mu, sigma, b], rtol=RTOL, atol=ATOL)
+    a1, b1 = O.tracker_update(a64, b64, ids, r, kl.astype(np.float64), float(np.float32(p.d_half)))
+    out = ab_t.cpu().numpy()
+    np.testing.assert_allclose(out[:, 0], a1, rtol=RTOL, atol=ATOL)
+    np.testing.assert_allclose(out[:, 1], b1, rtol=RTOL, atol=ATOL)
+    # and it is the same as the two separate calls
+    ab_t2 = dev(ab)
+    a_raw2, a_norm2, stats2, _ = gpu_advantages(ab_t2, ids, r, p)
+    gpu_update(ab_t2, ids, r, kl_table if is_table else kl, is_table, p)
+    np.testing.assert_array_equal(a_norm2, a_norm)
+    np.testing.assert_array_equal(stats2, stats)
+    np.testing.assert_array_equal(ab_t2.cpu().numpy(), out)
+
+
+def test_fused_advantage_and_update_skips_bad_elements():
+    p = B().default_params()
+    ab = np.array([[2.0, 2.0], [1.0, 3.0], [3.0, 1.0], [-1.0, 2.0], [4.0, 4.0]], dtype=np.float32)
+    ab_t = dev(ab)
+    ids = np.array([0, 9, 2, 3, 4, 1], np.int32)
+    r = np.array([1.0, 1.0, np.nan, 1.0, 0.0, 1.0], np.float32)
+    kl = np.array([0.01, 0.01, 0.01, 0.01, np.nan, 0.02], np.float32)
+    a_raw, _, _, st = gpu_advantages_update(ab_t, ids, r, kl, 0, p)
+    assert st & B().DEV_ID_OUT_OF_RANGE and st & B().DEV_NONFINITE
+    # bad id, NaN reward, negative entry: A = 0, entry untouched; NaN divergence: A defined, entry untouched
+    np.testing.assert_allclose(a_raw, [0.5, 0.0, 0.0, 0.0, -0.5, 0.75], rtol=RTOL)
+    out = ab_t.cpu().numpy()
+    np.testing.assert_array_equal(out[2:5], ab[2:5])
+    a1, b1 = O.tracker_update(ab[:, 0].astype(np.float64), ab[:, 1].astype(np.float64), [0, 1], [1.0, 1.0],
+                              [np.float64(np.float32(0.01)), np.float64(np.float32(0.02))], float(np.float32(p.d_half)))
+    np.testing.assert_allclose(out[:2], np.stack([a1[:2], b1[:2]], 1), rtol=RTOL)
+
+
+def test_near_zero_advantage_counts():
+    """Sec. 4 tracks the share of raw advantages with |A| <= tau at tau = 1e-4 and 0.02."""
+    rng = np.random.default_rng(77)
+    p = B().default_params()
+    # hand case: estimates 1, 0.99, 0.5, 0 against rewards 1, 1, 1, 0 -> |A| = 0, 0.01, 0.5, 0
+    ab = np.array([[8.0, 0.0], [7.92, 0.08], [4.0, 4.0], [0.0, 8.0]], dtype=np.float32)
+    _, _, stats, st = gpu_advantages(dev(ab), np.arange(4, dtype=np.int32), np.array([1, 1, 1, 0], np.float32), p)
+    assert st == 0 and stats[4] == 2.0 and stats[5] == 3.0 and stats[6] == 0.0 and stats[7] == 0.0
+    # both code paths, against the oracle's counts, with tolerances set by the caller
+    n = 200_000
+    v = rng.beta(0.3, 0.3, n)                                      # many prompts nearly mastered or hopeless
+    ab = np.stack([v * 16.0, (1.0 - v) * 16.0], 1).astype(np.float32)
+    for b in (4096, 150_000):
+        ids = rng.permutation(n)[:b].astype(np.int32)
+        est = O.value_estimate(ab[ids, 0].astype(np.float64), ab[ids, 1].astype(np.float64))
+        r = (rng.random(b) < est).astype(np.float32)
+        for taus in ((1e-4, 0.02), (0.005, 0.1)):
+            pp = B().default_params(near_zero_tau_lo=taus[0], near_zero_tau_hi=taus[1])
+            a_raw, _, stats, st = gpu_advantages(dev(ab), ids, r, pp)
+            f32_taus = (float(np.float32(taus[0])), float(np.float32(taus[1])))
+            want = O.near_zero_counts(a_raw, f32_taus)             # the same fp32 advantages, so the counts are exact
+            assert st == 0 and [int(stats[4]), int(stats[5])] == want and want[1] > want[0] > 0
+            loose = O.near_zero_counts(O.raw_advantage(ab[:, 0].astype(np.float64), ab[:, 1].astype(np.float64), ids, r),
+                                       f32_taus)
+            assert abs(loose[1] - want[1]) <= 1 + b // 10_000        # float64 advantages: ties at tau may differ
+
+
+def test_update_from_an_empty_entry_gives_the_first_reward():
+    """The start without offline initialisation (appendix ablation): an entry (0, 0) estimates 0.5 and
+    after its first update the estimate is the reward itself, whatever the divergence."""
+    p = B().default_params()
+    n = 64
+    ab = np.zeros((n, 2), dtype=np.float32)
+    ab[1::2] = [2.0, 6.0]
+    ids = np.arange(0, n, 2, dtype=np.int32)                      # the empty entries
+    rng = np.random.default_rng(5)
+    r = rng.uniform(0, 1, len(ids)).astype(np.float32)
+    r[:4] = [0.0, 1.0, 1.0, 0.0]
+    kl = rng.lognormal(-4, 1, len(ids)).astype(np.float32)
+    for fused in (False, True):
+        ab_t = dev(ab)
+        if fused:
+            a_raw, _, _, st = gpu_advantages_update(ab_t, ids, r, kl, 0, p)
+        else:
+            a_raw, _, _, st = gpu_advantages(ab_t, ids, r, p)
+            st |= gpu_update(ab_t, ids, r, kl, 0, p)
+        assert st == 0
+        np.testing.assert_allclose(a_raw, r - 0.5, rtol=RTOL, atol=ATOL)
+        out = ab_t.cpu().numpy()
+        a1, b1 = O.tracker_update(np.zeros(n), np.zeros(n), ids, r, kl.astype(np.float64), float(np.float32(p.d_half)))
+        np.testing.assert_allclose(out[ids, 0], a1[ids], rtol=RTOL, atol=ATOL)
+        np.testing.assert_allclose(out[ids, 1], b1[ids], rtol=RTOL, atol=ATOL)
+        np.testing.assert_allclose(O.value_estimate(out[ids, 0], out[ids, 1]), r, rtol=RTOL, atol=ATOL)
+        np.testing.assert_array_equal(out[1::2], ab[1::2])
+
+
+def test_advantages_flag_bad_table_entries_and_rewards():
+    p = B().default_params()
+    ab = np.array([[2.0, 2.0], [np.inf, 1.0], [1.0, -3.0], [3.0, 1.0]], dtype=np.float32)
+    a_raw, _, _, st = gpu_advantages(dev(ab), np.array([0, 1, 2, 3], np.int32), np.array([1, 1, 1, np.inf], np.float32), p)
+    assert st & B().DEV_NONFINITE and not st & B().DEV_ID_OUT_OF_RANGE
+    np.testing.assert_array_equal(a_raw, [0.5, 0.0, 0.0, 0.0])

@@ -34,7 +34,7 @@ def _both(ab_t, ids, r, params, want_raw):
     for static in (False, True):
         a_raw = torch.full((b,), float("nan"), **f32) if want_raw else None
         a_norm = torch.full((b,), float("nan"), **f32)
-        stats = torch.zeros(4, **f32)
+        stats = torch.zeros(8, **f32)
         st = status_word()
         if static:
             B.spo_advantages_static(ab_t, ids_t, r_t, a_raw, a_norm, stats, params, st)
