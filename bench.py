@@ -35,9 +35,10 @@ if ROOT not in sys.path:
 METRIC = "response tokens/s, fused SPO loss fwd+bwd (d4096,V151936,bf16); % bf16 peak"
 UNIT = "tokens/s"
 TABLE_N = 1_000_000          # tracker table the step samples from and updates
-# DRAM read+write bytes of all launches of one cfg4 step, from ncu captures (profiles/); None = the
-# kernels of that path changed after the counters were taken
-CFG4_STEP_DRAM_BYTES = {"split": 1.23e12, "onepass": 1.03e12}
+# DRAM read+write bytes (dram__bytes_read.sum + dram__bytes_write.sum) of all launches of one cfg4 step:
+# one chunk's launches captured with ncu on a slice of the workload, times the chunks of a step.
+# None = the kernels of that path changed after the counters were taken.
+CFG4_STEP_DRAM_BYTES = {"split": 1.23e12, "onepass": None}
 
 LOSS_SHAPES = {
     # workload: (d, V, w_std, old-logprob noise, reward probability)
@@ -106,11 +107,14 @@ class Step:
     """Device buffers of one workload and the call sequence of one step."""
 
     def __init__(self, workload, device, rank, responses=None, custom=None, mask_frac=0.0, path="onepass",
-                 entropy=False):
+                 entropy=False, dp_world=None, dw_slabs=8):
+        """dp_world = N: this rank holds its share of ONE mini-batch split over N ranks by token count
+        (W and the tracker table replicated); None: the rank has a mini-batch of its own."""
         import torch
         from paper_2509_13232_b200 import binding as B
-        from paper_2509_13232_b200 import inputs
+        from paper_2509_13232_b200 import dp, inputs
         self.B, self.torch = B, torch
+        self.dp_world = dp_world
         if custom:                       # T,d,V: eight equal responses, weights scaled to unit-variance logits
             t_c, d, V = custom
             w_std, noise, rew_p = 1.3 / d ** 0.5, 0.02, 0.3
@@ -123,7 +127,15 @@ class Step:
             if responses:
                 lengths = lengths[:responses]
             cfg = int(workload[3])
-        data = inputs.loss_batch_device(cfg * 10 + rank, lengths, d, V, w_std, noise, device, adv_p=rew_p)
+        batch_cfg = cfg * 10 if dp_world else cfg * 10 + rank     # what the table, uniforms and W are seeded by
+        self.S_all = len(lengths)
+        self.n_tok_all = int(np.sum(lengths))
+        self.my_responses = None
+        if dp_world:
+            self.my_responses = np.asarray(dp.partition_by_tokens(lengths, dp_world)[rank], dtype=np.int64)
+            lengths = np.asarray(lengths)[self.my_responses]
+        data = inputs.loss_batch_device(cfg * 10 + rank, lengths, d, V, w_std, noise, device, adv_p=rew_p,
+                                        w_cfg=batch_cfg)
         self.data = data
         self.T, self.d, self.V, self.S = data["T"], d, V, data["S"]
         self.mask_frac = float(mask_frac)
@@ -139,7 +151,7 @@ class Step:
             data["mask"] = torch.from_numpy(m).to(device)
         self.n_tok = int(data["mask"].sum().item())
         self.table_n = TABLE_PROMPTS.get(workload, TABLE_N)
-        tb = inputs.tracker_batch(cfg * 10 + rank, self.table_n, self.S, 2 * self.S)
+        tb = inputs.tracker_batch(batch_cfg, self.table_n, self.S_all, 2 * self.S_all)
         f32 = dict(dtype=torch.float32, device=device)
         self.ab0 = torch.from_numpy(tb.ab).to(device)
         self.ab = self.ab0.clone()
@@ -147,8 +159,17 @@ class Step:
         self.uniforms = torch.from_numpy(tb.uniforms).to(device)
         self.rewards = data["rewards"]
         self.params = B.default_params()
-        self.ids = torch.empty(self.S, dtype=torch.int32, device=device)
-        self.a_norm = torch.empty(self.S, **f32)
+        self.ids = torch.empty(self.S_all, dtype=torch.int32, device=device)
+        self.a_norm_all = torch.empty(self.S_all, **f32)      # one value per response of the whole mini-batch
+        self.a_norm = self.a_norm_all                         # ... and of this rank's responses
+        if dp_world:
+            # every rank owns the rewards of its own responses; the full vector is put together each step
+            self.my_idx = torch.from_numpy(self.my_responses).to(device)
+            self.rewards_all = torch.zeros(self.S_all, **f32)
+            self.a_norm = torch.empty(self.S, **f32)
+            self.params.global_tokens = self.n_tok_all        # denominators of the whole mini-batch (mask is all ones)
+            self.params.global_responses = self.S_all
+            self.reducer = dp.SlabAllReduce(B.spo_dw_slab_rows(V, d, dw_slabs), device)
         self.stats = torch.empty(8, **f32)
         self.loss = torch.zeros(4, **f32)
         self.logp, self.lse, self.coef = (torch.empty(self.T, **f32) for _ in range(3))
@@ -157,8 +178,8 @@ class Step:
         self.dW = torch.empty((V, d), **f32)
         self.status = torch.zeros(4, dtype=torch.int32, device=device)
         u8 = dict(dtype=torch.uint8, device=device)
-        self.ws_sample = torch.empty(B.spo_workspace_bytes(B.WS_SAMPLE, N=self.table_n, M=2 * self.S), **u8)
-        self.ws_adv = torch.empty(B.spo_workspace_bytes(B.WS_ADVANTAGES, B=self.S), **u8)
+        self.ws_sample = torch.empty(B.spo_workspace_bytes(B.WS_SAMPLE, N=self.table_n, M=2 * self.S_all), **u8)
+        self.ws_adv = torch.empty(B.spo_workspace_bytes(B.WS_ADVANTAGES, B=self.S_all), **u8)
         self.ws_bwd_bytes = B.spo_workspace_bytes(B.WS_LOSS_BWD, T=self.T, d=d, V=V)
         if self.mask_frac > 0.0:        # row lists: unmasked rows (one-pass) or rows with gradient (split backward)
             self.rows = torch.empty(self.T, dtype=torch.int32, device=device)
@@ -201,10 +222,22 @@ class Step:
 
     def small(self):
         B = self.B
-        B.spo_sample_prompts(self.ab, self.uniforms, self.S, self.ids, None, self.ws_sample, self.params, self.status)
+        B.spo_sample_prompts(self.ab, self.uniforms, self.S_all, self.ids, None, self.ws_sample, self.params, self.status)
+        rewards = self.rewards
+        if self.dp_world:
+            # the table is replicated and every rank applies the whole batch's updates, so the rewards of
+            # all responses are needed everywhere: scatter this rank's into a zero vector and sum over ranks
+            # (S floats).  With them every rank also forms the batch-global normalisation by itself.
+            import torch.distributed as dist
+            self.rewards_all.zero_()
+            self.rewards_all.index_copy_(0, self.my_idx, self.rewards)
+            dist.all_reduce(self.rewards_all)
+            rewards = self.rewards_all
         # raw advantage (pre-update baseline), tracker update and normalisation in one pass over the entries
-        B.spo_advantages_update(self.ab, self.ids, self.rewards, self.kl_table, 1, None, self.a_norm, self.stats,
+        B.spo_advantages_update(self.ab, self.ids, rewards, self.kl_table, 1, None, self.a_norm_all, self.stats,
                                 self.ws_adv, self.params, self.status)
+        if self.dp_world:
+            self.torch.index_select(self.a_norm_all, 0, self.my_idx, out=self.a_norm)
 
     def fwd(self, h=None, y=None, logp_old=None, mask=None, cu=None):
         D = self.data
@@ -237,11 +270,20 @@ class Step:
                                     self.loss, self.logp, self.lse, self.coef, None, self.dH, self.dW, 0, self.ws_loss,
                                     self.params, self.status)
             return
-        self.B.spo_loss_fwd_bwd(D["h"] if h is None else h, D["w"], D["y"] if y is None else y,
-                                D["logp_old"] if logp_old is None else logp_old, D["mask"] if mask is None else mask,
-                                D["cu_seqlens"] if cu is None else cu, self.a_norm, 1.0, self.loss, self.logp,
-                                self.lse, self.coef, None, self.dH, self.dW, 0, self.ws_loss, self.params, self.status,
-                                entropy=self.entropy)
+        args = (D["h"] if h is None else h, D["w"], D["y"] if y is None else y,
+                D["logp_old"] if logp_old is None else logp_old, D["mask"] if mask is None else mask,
+                D["cu_seqlens"] if cu is None else cu, self.a_norm, 1.0, self.loss, self.logp,
+                self.lse, self.coef, None, self.dH, self.dW, 0, self.ws_loss, self.params, self.status)
+        if self.dp_world:
+            # the ranks' dW and loss add up to the mini-batch's; dW is summed slab by slab on a second
+            # stream while its last contraction still runs
+            import torch.distributed as dist
+            self.B.spo_loss_fwd_bwd_slabs(*args, self.reducer.events, entropy=self.entropy)
+            self.reducer.reduce(self.dW)
+            dist.all_reduce(self.loss)
+            self.reducer.finish()
+            return
+        self.B.spo_loss_fwd_bwd(*args, entropy=self.entropy)
 
     def loss_calls(self, h=None, y=None, logp_old=None, mask=None, cu=None):
         """The loss calls of one step on the chosen path."""
@@ -279,7 +321,11 @@ def run_ours(args, rank, world, local_rank):
         spo_build.build()
     if world > 1:
         dist.barrier()
-    step = Step(args.workload, device, rank, args.responses, args.custom, args.mask_frac, args.path, args.entropy)
+    dp_mode = args.parallelism == "dp" and world > 1
+    if dp_mode and (args.path != "onepass" or args.mask_frac > 0.0 or args.custom):
+        raise SystemExit("--parallelism dp runs the one-pass loss on the unmasked named workloads")
+    step = Step(args.workload, device, rank, args.responses, args.custom, args.mask_frac, args.path, args.entropy,
+                dp_world=world if dp_mode else None, dw_slabs=args.dw_slabs)
     peaks = read_peaks()
 
     def barrier():
@@ -369,15 +415,16 @@ def run_ours(args, rank, world, local_rank):
     ms_per_step = total_ms / args.steps
     value = tokens_all / (ms_per_step / 1e3)
     gemm_ms = (t_fwd + t_bwd) / args.steps
+    # tensor FLOPs of one rank's share over the slowest rank's time (per-GPU rate against a per-GPU peak)
     achieved = (step.flops_fwd + step.flops_bwd) / (gemm_ms / 1e3) / 1e12
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16", "data": "synthetic",
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "strong" if dp_mode else "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": "custom" if args.custom else args.workload, "responses": step.S, "tokens": step.T, "d": step.d, "V": step.V,
                    "tracker_prompts": step.table_n, "l2": "inputs_exceed_l2", "loss_path": "onepass" if step.onepass else "split", "entropy_output": bool(args.entropy),
                    "bwd_chunks": step.bwd_chunks, "mask_frac": step.mask_frac,
-                   "parallelism": "replicas" if world > 1 else "single"},
+                   "parallelism": ("dp%d" % world if dp_mode else "replicas%d" % world) if world > 1 else "single"},
         "gpu_launches": step.launches * args.steps,
         "device_status": status,
         "wall_s": wall,
@@ -395,9 +442,8 @@ def run_ours(args, rank, world, local_rank):
             "flops_per_token": (6 if step.onepass else 8) * step.d * step.V,
             "fwd_tflops": None if step.onepass else step.flops_fwd / (t_fwd / args.steps / 1e3) / 1e12,
             "bwd_tflops": None if step.onepass else step.flops_bwd / (t_bwd / args.steps / 1e3) / 1e12,
-            # DRAM read+write bytes of all launches of one step, from the ncu captures summarised in
-            # profiles/spo_loss_fwd_bwd_cfg4_16responses_full.md (one-pass) and
-            # profiles/spo_gemm_kernel_cfg4_16responses_full.md (split), scaled by token rows; null for other shapes.
+            # DRAM read+write bytes of all launches of one step (ncu counters of one chunk's launches, scaled by
+            # token rows); known for the full cfg4 workload only.
             "traffic": CFG4_STEP_DRAM_BYTES.get("onepass" if step.onepass else "split") if (
                 args.workload == "cfg4_8b_bf16" and not args.responses and not args.custom and not args.mask_frac) else None,
         },
@@ -406,7 +452,7 @@ def run_ours(args, rank, world, local_rank):
         "clocks": clocks.summary(),
     }
     if world == 1 and not args.no_cpu_baseline:
-        out["cpu_baseline"] = cpu_baseline_sample(step, args.cpu_tokens)
+        out["cpu_baseline"] = cpu_baseline_sample(args.workload, args.cpu_tokens)
     print(json.dumps(out), flush=True)
 
 
@@ -453,7 +499,16 @@ def run_small_kernels(args, local_rank):
         "spo_advantages": (lambda: B.spo_advantages(ab, ids, r, None, a_norm, stats, wsa, p, st), 28 * Bn,
                            1 if Bn <= 8192 else 2),
         "spo_tracker_update": (lambda: B.spo_tracker_update(ab, ids, r, kl, 0, p, st), 28 * Bn, 1),
+        # advantage + update in one pass over the entries: per element 4 B id, 4 B reward, 4 B divergence,
+        # 8 B entry read and written back, 4 B advantage written, read and written normalised = 36 B
+        "spo_advantages_update": (lambda: B.spo_advantages_update(ab, ids, r, kl, 0, None, a_norm, stats, wsa, p, st),
+                                  36 * Bn, 1 if Bn <= 8192 else 2),
     }
+    # What a random 8-byte read-modify-write costs the memory system: the entry comes in as a 64-byte
+    # DRAM burst (two 32-byte sectors) and its dirty 32-byte sector goes back later; the streamed arrays
+    # cost their own bytes.  Time of that traffic at the measured copy rate = the bound for the gathers.
+    gather_bound_bytes = {"spo_advantages": (64 + 20) * Bn, "spo_tracker_update": (64 + 32 + 12) * Bn,
+                          "spo_advantages_update": (64 + 32 + 28) * Bn}
     out_calls, total_ms, total_bytes, launches = {}, 0.0, 0, 0
     with ClockSampler(local_rank) as clocks:
         for name, (fn, nbytes, n_launch) in calls.items():
@@ -469,8 +524,12 @@ def run_small_kernels(args, local_rank):
             ms = ts[len(ts) // 2]
             out_calls[name] = {"ms": ms, "algorithmic_bytes": nbytes, "GB/s": nbytes / ms / 1e6,
                                "frac_of_hbm": nbytes / ms / 1e6 / peaks["hbm_gbs"]}
-            total_ms += ms
-            total_bytes += nbytes
+            if name in gather_bound_bytes:
+                bound_ms = gather_bound_bytes[name] / peaks["hbm_gbs"] / 1e6
+                out_calls[name].update({"random_access_bound_ms": bound_ms, "frac_of_random_access_bound": bound_ms / ms})
+            if name not in ("spo_advantages", "spo_tracker_update"):       # the fused call does their work in the step
+                total_ms += ms
+                total_bytes += nbytes
             launches += n_launch * args.steps
     dom = out_calls["spo_sample_prompts"]
     print(json.dumps({
@@ -496,9 +555,30 @@ def blas_threads():
         return os.cpu_count() or 1
 
 
-def oracle_slice_seconds(h, w, y, logp_old, a_tok, n_rows):
-    """Time the oracle, as it stands, on the first n_rows token rows (forward + backward)."""
+ORACLE_ROWS = 512      # token rows of the CPU-oracle sample (both the cpu_baseline leg and --impl reference)
+
+
+def oracle_sample(workload, n_rows):
+    """The bounded sample both CPU legs time: n_rows synthetic token rows of the workload's shape
+    (H ~ N(0,1), W ~ N(0, w_std), bf16-rounded, targets uniform), W widened to float64 once, here,
+    outside every timed region."""
+    from paper_2509_13232_b200 import inputs
+    d, V, w_std, _, _ = LOSS_SHAPES[workload]
+    rng = inputs.rng_for(int(workload[3]), 9)
+    h = inputs.round_to_bf16(rng.standard_normal((n_rows, d)).astype(np.float32)).astype(np.float64)
+    w = inputs.round_to_bf16((rng.standard_normal((V, d)) * w_std).astype(np.float32)).astype(np.float64)
+    y = rng.integers(0, V, n_rows).astype(np.int32)
+    lo = np.full(n_rows, -np.log(V), dtype=np.float32)
+    a_tok = np.full(n_rows, 0.5, dtype=np.float32)
+    text = ("oracle loss forward+backward on %d synthetic token rows at full d=%d, V=%d (numpy float64, W widened "
+            "once outside the timed region); the tracker/sampling steps are negligible beside it" % (n_rows, d, V))
+    return (h, w, y, lo, a_tok), text
+
+
+def oracle_slice_seconds(h, w, y, logp_old, a_tok):
+    """Time the oracle, as it stands, on the given token rows (forward + backward)."""
     from oracle import spo_oracle as O
+    n_rows = h.shape[0]
     cu = np.arange(n_rows + 1)
     t0 = time.perf_counter()
     fwd = O.loss_forward(h, w, y, logp_old, None, cu, a_tok)
@@ -506,51 +586,90 @@ def oracle_slice_seconds(h, w, y, logp_old, a_tok, n_rows):
     return time.perf_counter() - t0
 
 
-def cpu_baseline_sample(step, n_rows):
-    D = step.data
-    h = D["h"][:n_rows].float().cpu().numpy()
-    w = D["w"].float().cpu().numpy()
-    y = D["y"][:n_rows].cpu().numpy()
-    lo = D["logp_old"][:n_rows].cpu().numpy()
-    a_tok = np.full(n_rows, 0.5, dtype=np.float32)
-    sec = oracle_slice_seconds(h, w, y, lo, a_tok, n_rows)
-    return {"value": n_rows / sec, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
-            "sample": "loss forward+backward of the first %d token rows at full d=%d, V=%d (numpy float64); "
-                      "the tracker/sampling steps are negligible beside it" % (n_rows, step.d, step.V),
+def cpu_baseline_sample(workload, n_rows):
+    sample, text = oracle_sample(workload, n_rows)
+    sec = oracle_slice_seconds(*sample)
+    return {"value": n_rows / sec, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": text,
             "seconds": sec}
 
 
 def run_reference(args, rank, world):
-    """The reference arm: the float64 CPU oracle on a bounded sample per step (rank 0 only)."""
+    """The reference arm: the float64 CPU oracle on the same bounded sample per step (rank 0 only)."""
     if rank != 0:
         return
-    from paper_2509_13232_b200 import inputs
-    d, V, w_std, noise, _ = LOSS_SHAPES[args.workload]
+    d, V = LOSS_SHAPES[args.workload][:2]
     n_rows = args.cpu_tokens
-    rng = inputs.rng_for(int(args.workload[3]), 9)
-    h = inputs.round_to_bf16(rng.standard_normal((n_rows, d)).astype(np.float32))
-    w = inputs.round_to_bf16((rng.standard_normal((V, d)) * w_std).astype(np.float32))
-    y = rng.integers(0, V, n_rows).astype(np.int32)
-    lo = np.full(n_rows, -np.log(V), dtype=np.float32)
-    a_tok = np.full(n_rows, 0.5, dtype=np.float32)
+    sample, text = oracle_sample(args.workload, n_rows)
     for _ in range(args.warmup):
-        oracle_slice_seconds(h, w, y, lo, a_tok, n_rows)
+        oracle_slice_seconds(*sample)
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        oracle_slice_seconds(h, w, y, lo, a_tok, n_rows)
+        oracle_slice_seconds(*sample)
     sec = (time.perf_counter() - t0) / args.steps
     value = n_rows / sec
-    sample = ("each step = oracle loss forward+backward on %d synthetic token rows at full d=%d, V=%d "
-              "(numpy float64)" % (n_rows, d, V))
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": args.workload, "tokens": n_rows, "d": d, "V": V},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+                         "sample": "each step = " + text},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }), flush=True)
+
+
+def spawn_ranks(n):
+    """`python bench.py --gpus N` without a launcher: start N copies of this command, one per GPU, with
+    the rendezvous environment a launcher would give them (127.0.0.1, a free port).  Rank 0 prints the
+    JSON line.  Returns the worst exit code."""
+    import socket
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    procs = []
+    for r in range(n):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE=str(n), LOCAL_WORLD_SIZE=str(n),
+                   MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        env.setdefault("NCCL_DEBUG", "INFO")              # the communicator log (transport, NVLS) goes to stderr
+        env.setdefault("NCCL_DEBUG_SUBSYS", "INIT")
+        procs.append(subprocess.Popen([sys.executable, os.path.abspath(__file__)] + sys.argv[1:], env=env))
+    codes = [p.wait() for p in procs]
+    return max(abs(c) for c in codes)
+
+
+def rehearse_host(args, rank, world):
+    """The host side of a multi-rank run without any GPU: rendezvous over gloo, the token-balanced split
+    of the mini-batch, the dW slab plan, the reduction of timings and token counts, and the merge of
+    per-rank advantage statistics -- on dummy values.  Rank 0 prints the plan as one JSON line."""
+    import torch
+    import torch.distributed as dist
+    from paper_2509_13232_b200 import binding as B
+    from paper_2509_13232_b200 import dp, inputs
+    if world > 1:
+        dist.init_process_group("gloo")
+    try:
+        d, V = LOSS_SHAPES[args.workload][:2]
+        lengths = inputs.workload_lengths(args.workload)
+        if args.responses:
+            lengths = lengths[:args.responses]
+        parts = dp.partition_by_tokens(lengths, world)
+        mine = int(np.sum(np.asarray(lengths)[parts[rank]])) if parts[rank] else 0
+        times, tokens_all = reduce_over_ranks([100.0 + rank, 50.0 - rank], mine, world, torch.device("cpu"))
+        n_tok, n_resp = dp.global_counts(mine, len(parts[rank]))
+        rec = torch.tensor([float(rank), 1.0, float(len(parts[rank])), 2.0 * len(parts[rank]), 0, 0, 0, 0])
+        mu, sigma = dp.global_advantage_stats(rec)
+        slabs = B.spo_dw_slab_rows(V, d, args.dw_slabs)
+        if rank == 0:
+            print(json.dumps({"rehearsal": True, "n_ranks": world, "parallelism": args.parallelism,
+                              "tokens_per_rank": [int(np.sum(np.asarray(lengths)[p])) for p in parts],
+                              "responses_per_rank": [len(p) for p in parts], "tokens_all": tokens_all,
+                              "global_tokens": n_tok, "global_responses": n_resp, "max_times": times,
+                              "merged_mu_sigma": [mu, sigma], "dw_slab_rows": slabs,
+                              "dw_slab_order": dp.slab_schedule(slabs)}), flush=True)
+    finally:
+        if world > 1:
+            dist.destroy_process_group()
 
 
 def main():
@@ -571,23 +690,35 @@ def main():
     ap.add_argument("--path", default="onepass", choices=["onepass", "split"],
                     help="loss as one spo_loss_fwd_bwd call (default) or as spo_loss_fwd + spo_loss_bwd")
     ap.add_argument("--entropy", action="store_true", help="also ask the loss call for the per-token policy entropy")
+    ap.add_argument("--parallelism", default="replicas", choices=["replicas", "dp"],
+                    help="with more than one GPU: every rank its own mini-batch (weak scaling, no data-path "
+                         "collective), or ONE mini-batch split over the ranks by token count with dW summed over the "
+                         "ranks, overlapped slab by slab with its last contraction (strong scaling)")
+    ap.add_argument("--dw-slabs", type=int, default=8, help="slabs the last dW contraction is cut into (dp)")
+    ap.add_argument("--rehearse-host", action="store_true",
+                    help="no GPU work: start the ranks (gloo), plan the data-parallel split and the dW slabs, run the "
+                         "host-side exchanges on dummy values and print the plan (used by the CPU tests)")
     ap.add_argument("--responses", type=int, default=None,
                     help="use only the first S responses of the workload (small cases for profiling)")
     args = ap.parse_args()
+    if "WORLD_SIZE" not in os.environ and args.gpus > 1 and args.workload in LOSS_SHAPES and (
+            args.impl == "ours" or args.rehearse_host):
+        sys.exit(spawn_ranks(args.gpus))          # one process per GPU, as a launcher would start them
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.rehearse_host:
+        rehearse_host(args, rank, world)
+        return
     if args.workload in SMALL_SHAPES:
         if rank == 0:
             run_small_kernels(args, local_rank)
         return
+    if args.cpu_tokens is None:
+        args.cpu_tokens = ORACLE_ROWS
     if args.impl == "reference":
-        if args.cpu_tokens is None:
-            args.cpu_tokens = 16
         run_reference(args, rank, world)
         return
-    if args.cpu_tokens is None:
-        args.cpu_tokens = 512
     if world > 1:
         import torch
         import torch.distributed as dist

@@ -21,12 +21,19 @@ int device_is_sm100();                // 1 when the current device is compute ca
 // ---- sampler ------------------------------------------------------------
 constexpr int kSampleTile = 2048;     // table entries per partial-sum tile
 constexpr int kSuperTile = 1024;      // tiles per second-level sum
+// Tables of up to kSmallTableMax prompts take a second form of the same computation, made for latency
+// instead of bandwidth: tiles of kSmallTile entries, whose sums every block of the search scans into
+// shared memory (the draw needs two dependent global reads instead of some twenty).
+constexpr int kSmallTile = 256;
+constexpr int kSmallTilesMax = 4096;
+constexpr int64_t kSmallTableMax = (int64_t)kSmallTile * kSmallTilesMax;
 
 struct SampleWs {
   size_t super_sums, keys, vals, zeroed_bytes, tile_sums, cand, total;
   int64_t n_tiles;
   int n_super;
   int64_t hash_slots;
+  int small;            // 1: the small-table form (tiles of kSmallTile entries, no second-level sums)
 };
 SampleWs sample_ws_layout(int64_t N, int32_t M);
 

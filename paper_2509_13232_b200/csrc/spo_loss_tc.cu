@@ -798,7 +798,10 @@ bool make_map(CUtensorMap* m, const void* ptr, uint64_t inner, uint64_t outer, u
 }
 
 // How many tiles a CTA pair may run ahead of the slowest pair before it holds back.
-constexpr int kLockStepWindow = 1;
+#ifndef SPO_TUNE_WINDOW
+#define SPO_TUNE_WINDOW 1
+#endif
+constexpr int kLockStepWindow = SPO_TUNE_WINDOW;
 
 // CTA pairs that can be resident at once (one CTA per SM).
 int group_count() { return sm_count() / CG; }
@@ -849,6 +852,9 @@ cudaError_t launch_gemm(const CUtensorMap& a, const CUtensorMap& b, const GemmPa
   GemmParams p = p_in;
   p.window = kLockStepWindow;
   p.sync_kblocks = p.k_blocks;                 // compare progress once per tile
+#ifdef SPO_TUNE_SYNCKB
+  if (MODE == MODE_DH || MODE == MODE_DW) p.sync_kblocks = p.k_blocks < SPO_TUNE_SYNCKB ? p.k_blocks : SPO_TUNE_SYNCKB;
+#endif
   p.progress = nullptr;
   if (p.window > 0 && progress) {
     cudaError_t e = cudaMemsetAsync(progress, 0, kProgressBytes, st);
@@ -881,6 +887,9 @@ constexpr uint32_t kBoxB = BSUB_ROWS;
 // re-reads of W from HBM; the choice also avoids a short last split (pairs would fall out of step)
 // and a nearly empty last round of units.
 int pick_fwd_split(int64_t m_tiles, int n_tiles, int d) {
+#ifdef SPO_TUNE_NSPLIT
+  if (m_tiles > 8) return SPO_TUNE_NSPLIT < n_tiles ? SPO_TUNE_NSPLIT : n_tiles;
+#endif
   const int groups = group_count();
   const double a_tile = (double)GROUP_M * d * 2, b_tile = (double)BN * d * 2;
   const double l2_budget = 56e6;
@@ -1069,7 +1078,10 @@ cudaError_t launch_bwd_bf16(const void* H, const void* W, const int32_t* y, cons
 // Contracting dW over several chunks at once divides its read-modify-write passes over the
 // [V x d] fp32 matrix (and its accumulator drains) by that number.
 // ---------------------------------------------------------------------------
-constexpr int kDwChunkGroup = 2;
+#ifndef SPO_DW_CHUNK_GROUP
+#define SPO_DW_CHUNK_GROUP 1
+#endif
+constexpr int kDwChunkGroup = SPO_DW_CHUNK_GROUP;
 
 FusedWs fused_ws_layout(int64_t T, int32_t d, int32_t V, int32_t S) {
   FusedWs L{};

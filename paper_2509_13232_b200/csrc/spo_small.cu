@@ -257,6 +257,153 @@ sample_search_kernel(const float* __restrict__ ab, int64_t N, float eps, const f
   }
 }
 
+// ---------------------------------------------------------------------------
+// Small tables (N <= kSmallTableMax): the same draw, organised for latency.
+// ---------------------------------------------------------------------------
+// One block = one tile of kSmallTile entries: 128 threads, one float4 (two entries) each.
+template <bool EMIT>
+__global__ void __launch_bounds__(kSmallTile / 2)
+sample_small_sums_kernel(const float4* __restrict__ ab4, int64_t N, float eps, float2* __restrict__ out_w2,
+                         float* __restrict__ out_w, unsigned long long* __restrict__ tile_sums, int32_t* d_status) {
+  const int64_t p = (int64_t)blockIdx.x * (kSmallTile / 2) + threadIdx.x;
+  const int64_t n_pairs = N >> 1;
+  unsigned long long sum = 0;
+  if (p < n_pairs) {
+    const float4 e = __ldg(ab4 + p);
+    const float w0 = entry_weight(e.x, e.y, eps, d_status);
+    const float w1 = entry_weight(e.z, e.w, eps, d_status);
+    sum = quantise(w0) + quantise(w1);
+    if (EMIT) out_w2[p] = make_float2(w0, w1);
+  } else if (p == n_pairs && (N & 1)) {          // odd tail entry
+    const float* ab = reinterpret_cast<const float*>(ab4);
+    const float w0 = entry_weight(ab[2 * (N - 1)], ab[2 * (N - 1) + 1], eps, d_status);
+    sum = quantise(w0);
+    if (EMIT) out_w[N - 1] = w0;
+  }
+  sum = warp_sum_u64(sum);
+  __shared__ unsigned long long s_part[kSmallTile / 64];
+  if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = sum;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    unsigned long long t = 0;
+#pragma unroll
+    for (int w = 0; w < kSmallTile / 64; ++w) t += s_part[w];
+    tile_sums[blockIdx.x] = t;
+  }
+}
+
+constexpr int kSearchSmallThreads = 512;        // 16 warps, one draw each
+
+// Every block scans all tile sums into shared memory (inclusive prefix; at most 32 KB), then one warp
+// per uniform: 32-ary search of the prefix for the tile, one read of the tile's 256 entries (eight per
+// lane), warp scan, winner into the hash table as in sample_search_kernel.
+__global__ void __launch_bounds__(kSearchSmallThreads)
+sample_search_small_kernel(const float* __restrict__ ab, int64_t N, float eps, const float* __restrict__ uniforms,
+                           int32_t M, const unsigned long long* __restrict__ tile_sums, int n_tiles,
+                           int32_t* __restrict__ cand, int32_t* keys, int32_t* vals, uint32_t slot_mask,
+                           int32_t* d_status) {
+  __shared__ unsigned long long s_pre[kSmallTilesMax];
+  __shared__ unsigned long long s_warp[kSearchSmallThreads / 32];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  {
+    constexpr int PER = kSmallTilesMax / kSearchSmallThreads;          // consecutive tiles per thread (8)
+    unsigned long long v[PER], run = 0;
+#pragma unroll
+    for (int j = 0; j < PER; ++j) {
+      const int i = tid * PER + j;
+      v[j] = i < n_tiles ? tile_sums[i] : 0ull;
+      run += v[j];
+    }
+    const unsigned long long incl = warp_incl_scan_u64(run, lane);
+    if (lane == 31) s_warp[warp] = incl;
+    __syncthreads();
+    unsigned long long before = incl - run;
+    for (int w = 0; w < warp; ++w) before += s_warp[w];
+#pragma unroll
+    for (int j = 0; j < PER; ++j) {
+      before += v[j];
+      s_pre[tid * PER + j] = before;
+    }
+    __syncthreads();
+  }
+  const int k = blockIdx.x * (kSearchSmallThreads / 32) + warp;
+  if (k >= M) return;
+  const unsigned long long wtot = s_pre[n_tiles - 1];
+  const float u = uniforms[k];
+  if (wtot == 0 || !(u >= 0.0f) || !(u < 1.0f)) {
+    if (lane == 0) {
+      cand[k] = -1;
+      if (wtot != 0) flag(d_status, SPO_DEV_NONFINITE);
+      else if (k == 0) flag(d_status, SPO_DEV_ZERO_TOTAL_WEIGHT);
+    }
+    return;
+  }
+  const unsigned long long bigu = __float2ull_rz(u * 4294967296.0f);          // floor(u * 2^32), exact
+  const unsigned long long t = (__umul64hi(bigu, wtot) << 32) | ((bigu * wtot) >> 32);
+  // first tile whose inclusive prefix exceeds t (t < wtot, so there is one)
+  int lo = 0, n = n_tiles;
+  while (n > 32) {
+    const int chunk = (n + 31) >> 5;
+    int idx = lo + (lane + 1) * chunk - 1;
+    if (idx > lo + n - 1) idx = lo + n - 1;
+    const unsigned hit = __ballot_sync(0xffffffffu, s_pre[idx] > t);
+    const int f = __ffs(hit) - 1;                                      // hit != 0: the last probe is the range's end
+    lo += f * chunk;
+    n = min(chunk, n_tiles - lo);
+  }
+  const unsigned hit0 = __ballot_sync(0xffffffffu, lane < n && s_pre[lo + lane] > t);
+  const int tile = lo + __ffs(hit0) - 1;
+  const unsigned long long run = tile > 0 ? s_pre[tile - 1] : 0ull;
+  // the tile's entries: eight consecutive ones per lane
+  const int64_t base = (int64_t)tile * kSmallTile;
+  const int n_here = (int)(N - base < kSmallTile ? N - base : kSmallTile);
+  const int i0 = 8 * lane;
+  unsigned long long q[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) q[j] = 0ull;
+  if (i0 + 7 < n_here) {
+    const float4* ab4 = reinterpret_cast<const float4*>(ab) + (base + i0) / 2;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float4 e = __ldg(ab4 + j);
+      q[2 * j] = quantise(entry_weight(e.x, e.y, eps, d_status));
+      q[2 * j + 1] = quantise(entry_weight(e.z, e.w, eps, d_status));
+    }
+  } else {
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+      if (i0 + j < n_here) q[j] = quantise(entry_weight(ab[2 * (base + i0 + j)], ab[2 * (base + i0 + j) + 1], eps, d_status));
+  }
+  unsigned long long mine = 0;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) mine += q[j];
+  const unsigned long long incl = warp_incl_scan_u64(mine, lane);
+  const unsigned hit = __ballot_sync(0xffffffffu, run + incl > t);
+  int32_t found = -1;
+  if (hit) {
+    const int first = __ffs(hit) - 1;
+    unsigned long long r0 = run + __shfl_sync(0xffffffffu, incl - mine, first);
+    int j = 7;
+#pragma unroll
+    for (int jj = 0; jj < 7; ++jj) {
+      r0 += __shfl_sync(0xffffffffu, q[jj], first);
+      if (j == 7 && r0 > t) j = jj;
+    }
+    found = (int32_t)(base + 8 * first + j);
+  }
+  if (lane == 0) {
+    cand[k] = found;
+    if (found >= 0) {
+      uint32_t s = hash_id((uint32_t)found) & slot_mask;
+      for (uint32_t probe = 0; probe <= slot_mask; ++probe) {
+        const int32_t prev = atomicCAS(&keys[s], 0, found + 1);
+        if (prev == 0 || prev == found + 1) { atomicMax(&vals[s], M - k); break; }
+        s = (s + 1) & slot_mask;
+      }
+    }
+  }
+}
+
 // Keep the first occurrence of every candidate, in order, until B are accepted.  One block;
 // each pass covers 8192 draws, eight consecutive ones per thread.
 __global__ void __launch_bounds__(1024)
@@ -646,8 +793,9 @@ advantages_apply_kernel(const float* a_raw, int32_t B, float mu, float inv, floa
 
 SampleWs sample_ws_layout(int64_t N, int32_t M) {
   SampleWs L{};
-  L.n_tiles = ceil_div(N, kSampleTile);
-  L.n_super = (int)ceil_div(L.n_tiles, kSuperTile);
+  L.small = N <= kSmallTableMax ? 1 : 0;
+  L.n_tiles = ceil_div(N, L.small ? kSmallTile : kSampleTile);
+  L.n_super = L.small ? 1 : (int)ceil_div(L.n_tiles, kSuperTile);
   int64_t slots = 64;
   while (slots < 2 * (int64_t)M) slots <<= 1;
   L.hash_slots = slots;
@@ -680,6 +828,21 @@ cudaError_t launch_sample(const float* ab, int64_t N, const float* u, int32_t M,
   auto* vals = reinterpret_cast<int32_t*>(ws + L.vals);
   cudaError_t e;
   if ((e = cudaMemsetAsync(ws, 0, L.zeroed_bytes, st)) != cudaSuccess) return e;
+  if (L.small) {
+    const float4* ab4 = reinterpret_cast<const float4*>(ab);
+    if (out_w)
+      sample_small_sums_kernel<true><<<(unsigned)L.n_tiles, kSmallTile / 2, 0, st>>>(
+          ab4, N, eps, reinterpret_cast<float2*>(out_w), out_w, tile_sums, d_status);
+    else
+      sample_small_sums_kernel<false><<<(unsigned)L.n_tiles, kSmallTile / 2, 0, st>>>(ab4, N, eps, nullptr, nullptr,
+                                                                                     tile_sums, d_status);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    sample_search_small_kernel<<<(unsigned)ceil_div(M, kSearchSmallThreads / 32), kSearchSmallThreads, 0, st>>>(
+        ab, N, eps, u, M, tile_sums, (int)L.n_tiles, cand, keys, vals, (uint32_t)(L.hash_slots - 1), d_status);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    sample_accept_kernel<<<1, 1024, 0, st>>>(cand, M, B, keys, vals, (uint32_t)(L.hash_slots - 1), out_ids, d_status);
+    return cudaGetLastError();
+  }
   if (out_w)
     sample_tile_sums_kernel<true><<<(unsigned)L.n_tiles, 256, 0, st>>>(
         reinterpret_cast<const float4*>(ab), N, eps, reinterpret_cast<float2*>(out_w), out_w, tile_sums, super_sums,

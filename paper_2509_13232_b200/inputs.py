@@ -228,8 +228,11 @@ def cfg1_tiny():
 # device-side generation for sizes the host cannot hold comfortably
 # -------------------------------------------------------------------------
 
-def loss_batch_device(cfg, lengths, d, v, w_std, old_noise, device, adv_p=0.3, t_chunk=2048):
+def loss_batch_device(cfg, lengths, d, v, w_std, old_noise, device, adv_p=0.3, t_chunk=2048, w_cfg=None):
     """bf16 loss inputs generated on ``device`` with a seeded torch generator.
+
+    ``w_cfg`` seeds W by itself (default: ``cfg``): data-parallel ranks draw their own responses
+    (different ``cfg``) against the same replicated W (same ``w_cfg``).
 
     Returns a dict of torch tensors: h [T,d] bf16, w [V,d] bf16, y [T] int32,
     logp_old [T] fp32, mask [T] uint8, cu_seqlens [S+1] int32 and rewards [S]
@@ -243,7 +246,9 @@ def loss_batch_device(cfg, lengths, d, v, w_std, old_noise, device, adv_p=0.3, t
     g = torch.Generator(device=device)
     g.manual_seed(seed_for(cfg, 3))
     h = torch.randn((t, d), generator=g, device=device, dtype=torch.float32).to(torch.bfloat16)
-    w = (torch.randn((v, d), generator=g, device=device, dtype=torch.float32) * w_std).to(torch.bfloat16)
+    gw = torch.Generator(device=device)
+    gw.manual_seed(seed_for(cfg if w_cfg is None else w_cfg, 6))
+    w = (torch.randn((v, d), generator=gw, device=device, dtype=torch.float32) * w_std).to(torch.bfloat16)
     y = torch.empty(t, dtype=torch.int32, device=device)
     logp_old = torch.empty(t, dtype=torch.float32, device=device)
     for t0 in range(0, t, t_chunk):

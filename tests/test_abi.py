@@ -38,6 +38,8 @@ def test_default_params_are_the_papers(lib):
     assert abs(p.eps_explore - 0.05) < 1e-7
     assert abs(p.clip_lo - 0.2) < 1e-7 and abs(p.clip_hi - 0.28) < 1e-7
     assert p.norm_ddof == 0 and p.d_half > 0
+    assert abs(p.near_zero_tau_lo - 1e-4) < 1e-10 and abs(p.near_zero_tau_hi - 0.02) < 1e-8   # Sec. 4 tolerances
+    assert p.dual_clip == 0.0 and p.surrogate == B.SUR_PPO_CLIP and p.agg_mode == B.AGG_TOKEN_MEAN
 
 
 def test_status_strings_and_version(lib):
@@ -86,6 +88,31 @@ def test_null_and_bad_arguments_are_rejected_on_the_host(lib):
     assert lib.spo_loss_fwd(odd, fake, B.DTYPE_BF16, fake, fake, None, fake, fake, 8, 64, 100, 1, *args_tail) == B.ERR_BAD_ALIGNMENT
     assert lib.spo_loss_bwd(fake, fake, B.DTYPE_BF16, fake, fake, fake, 1.0, 8, 64, 100, fake, 5, fake, 0,
                             fake, 1 << 30, ref, None, None) == B.ERR_UNSUPPORTED_DTYPE
+
+
+def test_new_entry_points_reject_bad_arguments_on_the_host(lib):
+    p = B.default_params()
+    ref = ctypes.byref(p)
+    fake = ctypes.c_void_p(0x1000)
+    odd = ctypes.c_void_p(0x1004)
+    # fused advantage + update
+    assert lib.spo_advantages_update(None, 10, fake, fake, fake, 0, 4, None, fake, None, None, 0, ref, None, None) == B.ERR_INVALID_ARG
+    assert lib.spo_advantages_update(fake, 10, fake, fake, fake, 3, 4, None, fake, None, None, 0, ref, None, None) == B.ERR_INVALID_ARG
+    assert lib.spo_advantages_update(fake, 10, fake, fake, fake, 0, 0, None, fake, None, None, 0, ref, None, None) == B.ERR_BAD_SHAPE
+    assert lib.spo_advantages_update(fake, 10, fake, odd, fake, 0, 4, None, fake, None, None, 0, ref, None, None) == B.ERR_BAD_ALIGNMENT
+    # slab variant of the one-pass loss: the slab request is checked before anything else
+    loss_args = (fake, fake, B.DTYPE_BF16, fake, fake, None, fake, fake, 8, 64, 100, 1, 1.0, fake, fake, fake, fake, None,
+                 None, fake, B.DTYPE_BF16, fake, 0, fake, 1 << 40, ref, None, None)
+    evs = (ctypes.c_void_p * 4)(fake, fake, fake, fake)
+    assert lib.spo_loss_fwd_bwd_slabs(*loss_args, 0, evs) == B.ERR_INVALID_ARG
+    assert lib.spo_loss_fwd_bwd_slabs(*loss_args, 65, evs) == B.ERR_INVALID_ARG
+    assert lib.spo_loss_fwd_bwd_slabs(*loss_args, 4, None) == B.ERR_INVALID_ARG
+    none_first = (ctypes.c_void_p * 4)(None, fake, fake, fake)
+    assert lib.spo_loss_fwd_bwd_slabs(*loss_args, 4, none_first) == B.ERR_INVALID_ARG
+    # parameters outside their domain
+    for bad in (dict(dual_clip=1.0), dict(dual_clip=-2.0), dict(near_zero_tau_lo=-1.0), dict(surrogate=7)):
+        q = B.default_params(**bad)
+        assert lib.spo_advantages(fake, 10, fake, fake, 4, None, fake, None, None, 0, ctypes.byref(q), None, None) == B.ERR_INVALID_ARG
 
 
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):

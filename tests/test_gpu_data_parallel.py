@@ -76,3 +76,80 @@ def test_two_emulated_ranks_equal_the_whole_mini_batch(agg, one_pass):
     assert abs(loss_sum - want["loss"]) <= 2e-3
     assert rel_fro(np.concatenate(dhs, 0), want_dh) <= 1e-2
     assert rel_fro(dws[0] + dws[1], want_dw) <= 1e-2
+
+
+def _fwd_bwd(lb, params, events=None):
+    """One spo_loss_fwd_bwd (or, with events, spo_loss_fwd_bwd_slabs) call; returns (loss, dH, dW) tensors."""
+    import torch
+    from paper_2509_13232_b200 import binding as B
+    H, W = dev(lb.h, torch.bfloat16), dev(lb.w, torch.bfloat16)
+    T, d = H.shape
+    V, S = W.shape[0], len(lb.cu_seqlens) - 1
+    f32 = dict(dtype=torch.float32, device="cuda")
+    loss = torch.zeros(4, **f32)
+    logp, lse, coef = (torch.zeros(T, **f32) for _ in range(3))
+    dH = torch.zeros((T, d), dtype=torch.bfloat16, device="cuda")
+    dW = torch.full((V, d), float("nan"), **f32)
+    st = status_word()
+    args = (H, W, dev(lb.y), dev(lb.logp_old), dev(lb.mask), dev(lb.cu_seqlens), dev(lb.a_norm), 1.0, loss, logp, lse,
+            coef, None, dH, dW, 0, ws_bytes(B.WS_LOSS_FWD_BWD, T=T, d=d, V=V, B=S), params, st)
+    if events is None:
+        B.spo_loss_fwd_bwd(*args)
+    else:
+        B.spo_loss_fwd_bwd_slabs(*args, events)
+    return loss, dH, dW, st
+
+
+@pytest.mark.parametrize("lengths", [[700, 40, 520, 75], [5000, 4400, 9000, 1600]])
+def test_slab_cut_last_dw_contraction_is_bitwise_the_plain_call_and_reduces_in_slab_order(lengths):
+    """The data-parallel variant cuts the last dW launch into vocabulary slabs with an event behind
+    each.  One chunk and three chunks (the slabs belong to the last group of chunks only): results
+    equal spo_loss_fwd_bwd bit for bit, and two emulated ranks whose dW are added slab by slab, each
+    slab as soon as its event has passed on a second stream, give the whole mini-batch's dW."""
+    import torch
+    from paper_2509_13232_b200 import binding as B
+    v, d = 20000, 1024                      # 79 vocabulary row tiles, two hidden column tiles: slabs of 37 row tiles
+    small = sum(lengths) < 5000
+    if small:
+        lb = inputs.loss_batch(79, lengths, d, v, 0.02, True, 0.3, target="softmax", mask_p=0.1)
+    else:                                   # three chunks: too many logits for the host, generated on the device
+        data = inputs.loss_batch_device(79, np.asarray(lengths), d, v, 0.02, 0.3, torch.device("cuda", 0))
+        rng = inputs.rng_for(79, 5)
+        lb = inputs.LossBatch(h=data["h"].float().cpu().numpy(), w=data["w"].float().cpu().numpy(),
+                              y=data["y"].cpu().numpy(), logp_old=data["logp_old"].cpu().numpy(),
+                              mask=(rng.random(data["T"]) >= 0.1).astype(np.uint8),
+                              cu_seqlens=data["cu_seqlens"].cpu().numpy(),
+                              a_norm=rng.standard_normal(len(lengths)).astype(np.float32), bf16=True)
+    params = B.default_params()
+    plain = _fwd_bwd(lb, params)
+    rows = B.spo_dw_slab_rows(v, d, 6)
+    assert len(rows) - 1 == 3
+    red = dp.SlabAllReduce(rows, torch.device("cuda", 0))
+    cut = _fwd_bwd(lb, params, red.events)
+    red.reduce(cut[2])                       # one process: waits for every slab's event, no collective
+    red.finish()
+    torch.cuda.synchronize()
+    assert int(plain[3][0].item()) == 0 and int(cut[3][0].item()) == 0
+    for a, b in zip(plain[:3], cut[:3]):
+        assert torch.equal(a, b)
+    # two ranks, one after the other, each with the whole batch's denominators
+    n_tok, s_mid = int(lb.mask.sum()), 2
+    pg = B.default_params(global_tokens=n_tok, global_responses=len(lengths))
+    total = torch.zeros_like(plain[2])
+    side = torch.cuda.Stream()
+    for s0, s1 in ((0, s_mid), (s_mid, len(lengths))):
+        part = _slice_batch(lb, s0, s1)
+        evs = dp.SlabAllReduce(rows, torch.device("cuda", 0))
+        loss, dH, dW, st = _fwd_bwd(part, pg, evs.events)
+        with torch.cuda.stream(side):
+            for k, lo, hi in dp.slab_schedule(rows):
+                side.wait_event(evs.events[k])        # rows lo..hi of this rank's dW are final from here on
+                total[lo:hi] += dW[lo:hi]
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        assert int(st[0].item()) == 0
+    assert rel_fro(total.cpu().numpy(), plain[2].cpu().numpy()) <= 2e-3
+    if small:                               # ... and the oracle's, where the host can form the logits
+        want = O.loss_forward(lb.h, lb.w, lb.y, lb.logp_old, lb.mask, lb.cu_seqlens, lb.a_norm)
+        _, want_dw = O.loss_backward(lb.h, lb.w, lb.y, want["lse"], want["coef"])
+        assert rel_fro(total.cpu().numpy(), want_dw) <= 1e-2

@@ -34,6 +34,9 @@ def test_paper_constants_match_oracle_defaults():
     assert O.EPS_EXPLORE == c["eps_explore"]
     assert O.CLIP_LO == c["clip_low"] and O.CLIP_HI == c["clip_high"]
     assert O.N0_SAMPLES == c["n0"]
+    import inspect
+    taus = inspect.signature(O.near_zero_counts).parameters["taus"].default
+    assert tuple(taus) == (c["near_zero_tau_tight"], c["near_zero_tau_loose"])
 
 
 def test_init_effective_sample_size_is_window_min():
