@@ -198,26 +198,28 @@ class Step:
                 self.ws_bwd = torch.empty(self.ws_bwd_bytes, **u8)
         chunk_rows = self.ws_bwd_bytes // (((V + 255) // 256) * 256 * 2)
         self.bwd_chunks = -(-self.T // chunk_rows)
-        # kernels launched by one step: sampling 3 (tile sums, search, accept), advantages + update 1, then
+        # kernels launched by one step: sampling 4 (tile sums, their prefix, search, accept; 3 for tables above
+        # 2^20 prompts), advantages + update 1, then
         # split path: forward 3 (count, contraction, finalise), backward 3 per chunk;
-        # one-pass path: count 1, first-tile pass 1, per chunk 4 (logits contraction, finalise, row scaling
-        # of H, dH) and one dW contraction per pair of chunks.  Memsets are not counted.
+        # one-pass path: count 1, first-tile pass 1, per chunk 5 (logits contraction, finalise, row scaling
+        # of H, dH, dW).  Memsets are not counted.
         self.flops_fwd = 2.0 * self.T * d * V
+        n_samp = 4 if self.table_n <= (1 << 20) else 3
         chunks_act = -(-self.n_tok // chunk_rows)          # chunks of the compacted batch (masked workloads)
         if self.onepass and self.mask_frac > 0.0:
             # row list 3, gather 1, boundaries 1, one-pass on the compacted batch, two scatters
-            self.launches = 3 + 1 + 3 + 1 + 1 + (2 + 4 * chunks_act + -(-chunks_act // 2)) + 2
+            self.launches = n_samp + 1 + 3 + 1 + 1 + (2 + 5 * chunks_act) + 2
             self.flops_fwd = 2.0 * self.n_tok * d * V
             self.flops_bwd = 4.0 * self.n_tok * d * V
         elif self.onepass:
-            self.launches = 3 + 1 + 2 + 4 * self.bwd_chunks + -(-self.bwd_chunks // 2)
+            self.launches = n_samp + 1 + 2 + 5 * self.bwd_chunks
             self.flops_bwd = 4.0 * self.T * d * V
         elif self.mask_frac > 0.0:
             # forward over all rows; row list 3, gather 1, backward on the rows with gradient, scatter 1
-            self.launches = 3 + 1 + 3 + 3 + 1 + 3 * chunks_act + 1
+            self.launches = n_samp + 1 + 3 + 3 + 1 + 3 * chunks_act + 1
             self.flops_bwd = 6.0 * self.n_tok * d * V
         else:
-            self.launches = 3 + 1 + 3 + 3 * self.bwd_chunks
+            self.launches = n_samp + 1 + 3 + 3 * self.bwd_chunks
             self.flops_bwd = 6.0 * self.T * d * V
 
     def small(self):
@@ -495,7 +497,9 @@ def run_small_kernels(args, local_rank):
     flush = torch.empty(128 * 1024 * 1024, dtype=torch.float32, device=dev)
     calls = {
         "spo_tracker_init": (lambda: B.spo_tracker_init(ab2, v0, p), 12 * N, 1),
-        "spo_sample_prompts": (lambda: B.spo_sample_prompts(ab, u, n_draw, out_ids, None, ws, p, st), 8 * N, 3),
+        # launches: sums, prefix, search, accept for tables of up to 2^20 prompts; sums, search, accept above
+        "spo_sample_prompts": (lambda: B.spo_sample_prompts(ab, u, n_draw, out_ids, None, ws, p, st), 8 * N,
+                               4 if N <= (1 << 20) else 3),
         "spo_advantages": (lambda: B.spo_advantages(ab, ids, r, None, a_norm, stats, wsa, p, st), 28 * Bn,
                            1 if Bn <= 8192 else 2),
         "spo_tracker_update": (lambda: B.spo_tracker_update(ab, ids, r, kl, 0, p, st), 28 * Bn, 1),
@@ -522,8 +526,22 @@ def run_small_kernels(args, local_rank):
                     ts.append(e0.elapsed_time(e1))
             ts.sort()
             ms = ts[len(ts) // 2]
-            out_calls[name] = {"ms": ms, "algorithmic_bytes": nbytes, "GB/s": nbytes / ms / 1e6,
-                               "frac_of_hbm": nbytes / ms / 1e6 / peaks["hbm_gbs"]}
+            # the same call replayed from a CUDA graph: what the device needs for it once the host's launch
+            # calls (four per sampling call) are out of the way -- at the paper's sizes they are most of `ms`
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                fn()
+            tg = []
+            for i in range(args.warmup + args.steps):
+                flush.zero_()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(); graph.replay(); e1.record()
+                torch.cuda.synchronize()
+                if i >= args.warmup:
+                    tg.append(e0.elapsed_time(e1))
+            tg.sort()
+            out_calls[name] = {"ms": ms, "graph_ms": tg[len(tg) // 2], "algorithmic_bytes": nbytes,
+                               "GB/s": nbytes / ms / 1e6, "frac_of_hbm": nbytes / ms / 1e6 / peaks["hbm_gbs"]}
             if name in gather_bound_bytes:
                 bound_ms = gather_bound_bytes[name] / peaks["hbm_gbs"] / 1e6
                 out_calls[name].update({"random_access_bound_ms": bound_ms, "frac_of_random_access_bound": bound_ms / ms})

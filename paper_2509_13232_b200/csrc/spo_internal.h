@@ -29,7 +29,7 @@ constexpr int kSmallTilesMax = 4096;
 constexpr int64_t kSmallTableMax = (int64_t)kSmallTile * kSmallTilesMax;
 
 struct SampleWs {
-  size_t super_sums, keys, vals, zeroed_bytes, tile_sums, cand, total;
+  size_t super_sums, keys, vals, zeroed_bytes, tile_sums, cand, slot_of, first_draw, total;
   int64_t n_tiles;
   int n_super;
   int64_t hash_slots;

@@ -179,8 +179,8 @@ __global__ void __launch_bounds__(256)
 sample_search_kernel(const float* __restrict__ ab, int64_t N, float eps, const float* __restrict__ uniforms,
                      int32_t M, const unsigned long long* __restrict__ tile_sums,
                      const unsigned long long* __restrict__ super_sums, int64_t n_tiles, int n_super,
-                     int32_t* __restrict__ cand, int32_t* keys, int32_t* vals, uint32_t slot_mask,
-                     int32_t* d_status) {
+                     int32_t* __restrict__ cand, int32_t* __restrict__ slot_of, int32_t* keys, int32_t* vals,
+                     uint32_t slot_mask, int32_t* d_status) {
   const int lane = threadIdx.x & 31;
   const int k = (int)(((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5);
   if (k >= M) return;
@@ -250,7 +250,7 @@ sample_search_kernel(const float* __restrict__ ab, int64_t N, float eps, const f
       uint32_t s = hash_id((uint32_t)found) & slot_mask;
       for (uint32_t probe = 0; probe <= slot_mask; ++probe) {
         const int32_t prev = atomicCAS(&keys[s], 0, found + 1);
-        if (prev == 0 || prev == found + 1) { atomicMax(&vals[s], M - k); break; }
+        if (prev == 0 || prev == found + 1) { atomicMax(&vals[s], M - k); slot_of[k] = (int32_t)s; break; }
         s = (s + 1) & slot_mask;
       }
     }
@@ -264,10 +264,14 @@ sample_search_kernel(const float* __restrict__ ab, int64_t N, float eps, const f
 template <bool EMIT>
 __global__ void __launch_bounds__(kSmallTile / 2)
 sample_small_sums_kernel(const float4* __restrict__ ab4, int64_t N, float eps, float2* __restrict__ out_w2,
-                         float* __restrict__ out_w, unsigned long long* __restrict__ tile_sums, int32_t* d_status) {
+                         float* __restrict__ out_w, unsigned long long* __restrict__ tile_sums,
+                         int32_t* __restrict__ first_draw, int32_t* d_status) {
   const int64_t p = (int64_t)blockIdx.x * (kSmallTile / 2) + threadIdx.x;
   const int64_t n_pairs = N >> 1;
   unsigned long long sum = 0;
+  // first_draw[id] will hold the largest M - k over the draws k that pick prompt id: cleared here
+  if (p < n_pairs) reinterpret_cast<int2*>(first_draw)[p] = make_int2(0, 0);
+  else if (p == n_pairs && (N & 1)) first_draw[N - 1] = 0;
   if (p < n_pairs) {
     const float4 e = __ldg(ab4 + p);
     const float w0 = entry_weight(e.x, e.y, eps, d_status);
@@ -292,43 +296,53 @@ sample_small_sums_kernel(const float4* __restrict__ ab4, int64_t N, float eps, f
   }
 }
 
-constexpr int kSearchSmallThreads = 512;        // 16 warps, one draw each
-
-// Every block scans all tile sums into shared memory (inclusive prefix; at most 32 KB), then one warp
-// per uniform: 32-ary search of the prefix for the tile, one read of the tile's 256 entries (eight per
-// lane), warp scan, winner into the hash table as in sample_search_kernel.
-__global__ void __launch_bounds__(kSearchSmallThreads)
-sample_search_small_kernel(const float* __restrict__ ab, int64_t N, float eps, const float* __restrict__ uniforms,
-                           int32_t M, const unsigned long long* __restrict__ tile_sums, int n_tiles,
-                           int32_t* __restrict__ cand, int32_t* keys, int32_t* vals, uint32_t slot_mask,
-                           int32_t* d_status) {
-  __shared__ unsigned long long s_pre[kSmallTilesMax];
-  __shared__ unsigned long long s_warp[kSearchSmallThreads / 32];
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  {
-    constexpr int PER = kSmallTilesMax / kSearchSmallThreads;          // consecutive tiles per thread (8)
-    unsigned long long v[PER], run = 0;
+// Inclusive prefix of the (at most 4096) tile sums: one block, four consecutive values per thread.
+__global__ void __launch_bounds__(kSmallTilesMax / 4)
+sample_small_prefix_kernel(const unsigned long long* __restrict__ tile_sums, int n_tiles,
+                           unsigned long long* __restrict__ tile_prefix) {
+  constexpr int THREADS = kSmallTilesMax / 4, PER = 4;
+  unsigned long long v[PER], run = 0;
 #pragma unroll
-    for (int j = 0; j < PER; ++j) {
-      const int i = tid * PER + j;
-      v[j] = i < n_tiles ? tile_sums[i] : 0ull;
-      run += v[j];
-    }
-    const unsigned long long incl = warp_incl_scan_u64(run, lane);
-    if (lane == 31) s_warp[warp] = incl;
-    __syncthreads();
-    unsigned long long before = incl - run;
-    for (int w = 0; w < warp; ++w) before += s_warp[w];
-#pragma unroll
-    for (int j = 0; j < PER; ++j) {
-      before += v[j];
-      s_pre[tid * PER + j] = before;
-    }
-    __syncthreads();
+  for (int j = 0; j < PER; ++j) {
+    const int i = threadIdx.x * PER + j;
+    v[j] = i < n_tiles ? tile_sums[i] : 0ull;
+    run += v[j];
   }
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const unsigned long long incl = warp_incl_scan_u64(run, lane);
+  __shared__ unsigned long long s_warp[THREADS / 32];
+  if (lane == 31) s_warp[warp] = incl;
+  __syncthreads();
+  unsigned long long before = incl - run;
+  for (int w = 0; w < warp; ++w) before += s_warp[w];
+#pragma unroll
+  for (int j = 0; j < PER; ++j) {
+    const int i = threadIdx.x * PER + j;
+    before += v[j];
+    if (i < n_tiles) tile_prefix[i] = before;
+  }
+}
+
+constexpr int kSearchSmallThreads = 256;        // 8 warps, one draw each
+
+// One warp per uniform: a two-level 64-ary search of the inclusive prefix of the tile sums (at most
+// 4096 values, L2-resident: two dependent reads), one read of the tile's 256 entries (eight per lane),
+// warp scan.  The winner is entered as an integer maximum into first_draw[id] (the earliest draw of a
+// prompt has the largest M - k) and the draw remembers where to look (slot_of[k] = id).
+__global__ void __launch_bounds__(kSearchSmallThreads, 8)
+sample_search_small_kernel(const float* __restrict__ ab, int64_t N, float eps, const float* __restrict__ uniforms,
+                           int32_t M, const unsigned long long* __restrict__ pre, int n_tiles,
+                           int32_t* __restrict__ cand, int32_t* __restrict__ slot_of, int32_t* first_draw,
+                           int32_t* d_status) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int k = blockIdx.x * (kSearchSmallThreads / 32) + warp;
   if (k >= M) return;
-  const unsigned long long wtot = s_pre[n_tiles - 1];
+  // level 1: 64 probes at the ends of 64 equal spans of the prefix (two per lane); they do not depend
+  // on the uniform, so they are in flight together with it
+  const int span = (n_tiles + 63) >> 6;
+  const int i_a = min((2 * lane + 1) * span, n_tiles) - 1, i_b = min((2 * lane + 2) * span, n_tiles) - 1;
+  const unsigned long long p_a = pre[i_a], p_b = pre[i_b];
+  const unsigned long long wtot = __shfl_sync(0xffffffffu, p_b, 31);           // pre[n_tiles - 1]
   const float u = uniforms[k];
   if (wtot == 0 || !(u >= 0.0f) || !(u < 1.0f)) {
     if (lane == 0) {
@@ -340,20 +354,30 @@ sample_search_small_kernel(const float* __restrict__ ab, int64_t N, float eps, c
   }
   const unsigned long long bigu = __float2ull_rz(u * 4294967296.0f);          // floor(u * 2^32), exact
   const unsigned long long t = (__umul64hi(bigu, wtot) << 32) | ((bigu * wtot) >> 32);
-  // first tile whose inclusive prefix exceeds t (t < wtot, so there is one)
-  int lo = 0, n = n_tiles;
-  while (n > 32) {
-    const int chunk = (n + 31) >> 5;
-    int idx = lo + (lane + 1) * chunk - 1;
-    if (idx > lo + n - 1) idx = lo + n - 1;
-    const unsigned hit = __ballot_sync(0xffffffffu, s_pre[idx] > t);
-    const int f = __ffs(hit) - 1;                                      // hit != 0: the last probe is the range's end
-    lo += f * chunk;
-    n = min(chunk, n_tiles - lo);
+  // first span whose last prefix exceeds t (t < wtot, so there is one); the sum before it
+  const unsigned hit_a = __ballot_sync(0xffffffffu, p_a > t), hit_b = __ballot_sync(0xffffffffu, p_b > t);
+  const int fa = hit_a ? __ffs(hit_a) - 1 : 32, fb = __ffs(hit_b) - 1;        // spans 2 fa and 2 fb + 1
+  const int sp = (fa <= fb) ? 2 * fa : 2 * fb + 1;
+  // prefix at the end of span sp - 1: lane (sp-1)/2 holds it (p_a for an even span index, p_b for an odd one)
+  unsigned long long before_span = 0ull;
+  {
+    const unsigned long long from_a = __shfl_sync(0xffffffffu, p_a, sp > 0 ? (sp - 1) >> 1 : 0);
+    const unsigned long long from_b = __shfl_sync(0xffffffffu, p_b, sp > 0 ? (sp - 1) >> 1 : 0);
+    if (sp > 0) before_span = ((sp - 1) & 1) ? from_b : from_a;
   }
-  const unsigned hit0 = __ballot_sync(0xffffffffu, lane < n && s_pre[lo + lane] > t);
-  const int tile = lo + __ffs(hit0) - 1;
-  const unsigned long long run = tile > 0 ? s_pre[tile - 1] : 0ull;
+  // level 2: the span's own entries (at most 64: two per lane)
+  const int lo = sp * span, n = min(span, n_tiles - lo);
+  const unsigned long long q_a = lane < n ? pre[lo + lane] : ~0ull;
+  const unsigned long long q_b = lane + 32 < n ? pre[lo + 32 + lane] : ~0ull;
+  const unsigned h_a = __ballot_sync(0xffffffffu, q_a > t), h_b = __ballot_sync(0xffffffffu, q_b > t);
+  const int off_t = h_a ? __ffs(h_a) - 1 : 32 + __ffs(h_b) - 1;
+  const int tile = lo + off_t;
+  unsigned long long run = before_span;                                        // sum of all tiles before `tile`
+  if (off_t > 0) {
+    const unsigned long long r_a = __shfl_sync(0xffffffffu, q_a, (off_t - 1) & 31);
+    const unsigned long long r_b = __shfl_sync(0xffffffffu, q_b, (off_t - 1) & 31);
+    run = off_t - 1 < 32 ? r_a : r_b;
+  }
   // the tile's entries: eight consecutive ones per lane
   const int64_t base = (int64_t)tile * kSmallTile;
   const int n_here = (int)(N - base < kSmallTile ? N - base : kSmallTile);
@@ -363,11 +387,13 @@ sample_search_small_kernel(const float* __restrict__ ab, int64_t N, float eps, c
   for (int j = 0; j < 8; ++j) q[j] = 0ull;
   if (i0 + 7 < n_here) {
     const float4* ab4 = reinterpret_cast<const float4*>(ab) + (base + i0) / 2;
+    float4 e[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) e[j] = __ldg(ab4 + j);
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-      const float4 e = __ldg(ab4 + j);
-      q[2 * j] = quantise(entry_weight(e.x, e.y, eps, d_status));
-      q[2 * j + 1] = quantise(entry_weight(e.z, e.w, eps, d_status));
+      q[2 * j] = quantise(entry_weight(e[j].x, e[j].y, eps, d_status));
+      q[2 * j + 1] = quantise(entry_weight(e[j].z, e[j].w, eps, d_status));
     }
   } else {
 #pragma unroll
@@ -394,22 +420,18 @@ sample_search_small_kernel(const float* __restrict__ ab, int64_t N, float eps, c
   if (lane == 0) {
     cand[k] = found;
     if (found >= 0) {
-      uint32_t s = hash_id((uint32_t)found) & slot_mask;
-      for (uint32_t probe = 0; probe <= slot_mask; ++probe) {
-        const int32_t prev = atomicCAS(&keys[s], 0, found + 1);
-        if (prev == 0 || prev == found + 1) { atomicMax(&vals[s], M - k); break; }
-        s = (s + 1) & slot_mask;
-      }
+      atomicMax(&first_draw[found], M - k);
+      slot_of[k] = found;
     }
   }
 }
 
 // Keep the first occurrence of every candidate, in order, until B are accepted.  One block;
-// each pass covers 8192 draws, eight consecutive ones per thread.
+// each pass covers 8192 draws, eight consecutive ones per thread.  A draw is the first occurrence of
+// its prompt when the hash slot the search left it in still holds its own M - k (the largest wins).
 __global__ void __launch_bounds__(1024)
-sample_accept_kernel(const int32_t* __restrict__ cand, int32_t M, int32_t B, const int32_t* __restrict__ keys,
-                     const int32_t* __restrict__ vals, uint32_t slot_mask, int32_t* __restrict__ out_ids,
-                     int32_t* d_status) {
+sample_accept_kernel(const int32_t* __restrict__ cand, const int32_t* __restrict__ slot_of, int32_t M, int32_t B,
+                     const int32_t* __restrict__ vals, int32_t* __restrict__ out_ids, int32_t* d_status) {
   constexpr int PER = 8;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   __shared__ int s_warp[32];
@@ -419,26 +441,27 @@ sample_accept_kernel(const int32_t* __restrict__ cand, int32_t M, int32_t B, con
   for (int k0 = 0; k0 < M; k0 += 1024 * PER) {
     const int base_count = s_total;
     if (base_count >= B) break;
-    int32_t c[PER];
-    uint32_t slot[PER];
-    bool first[PER];
+    int32_t c[PER], sl[PER], best[PER];
+    const int kt = k0 + tid * PER;
+    if (kt + PER <= M) {                           // two 16-byte loads per array
+      const int4 c0 = *reinterpret_cast<const int4*>(cand + kt), c1 = *reinterpret_cast<const int4*>(cand + kt + 4);
+      const int4 s0 = *reinterpret_cast<const int4*>(slot_of + kt), s1 = *reinterpret_cast<const int4*>(slot_of + kt + 4);
+      c[0] = c0.x; c[1] = c0.y; c[2] = c0.z; c[3] = c0.w; c[4] = c1.x; c[5] = c1.y; c[6] = c1.z; c[7] = c1.w;
+      sl[0] = s0.x; sl[1] = s0.y; sl[2] = s0.z; sl[3] = s0.w; sl[4] = s1.x; sl[5] = s1.y; sl[6] = s1.z; sl[7] = s1.w;
+    } else {
 #pragma unroll
-    for (int j = 0; j < PER; ++j) {
-      const int k = k0 + tid * PER + j;
-      c[j] = k < M ? cand[k] : -1;
-      slot[j] = hash_id((uint32_t)c[j]) & slot_mask;
+      for (int j = 0; j < PER; ++j) {
+        c[j] = kt + j < M ? cand[kt + j] : -1;
+        sl[j] = kt + j < M ? slot_of[kt + j] : 0;
+      }
     }
+#pragma unroll
+    for (int j = 0; j < PER; ++j) best[j] = c[j] >= 0 ? __ldg(vals + sl[j]) : 0;     // eight independent reads
+    bool first[PER];
     int mine = 0;
 #pragma unroll
     for (int j = 0; j < PER; ++j) {
-      first[j] = false;
-      if (c[j] >= 0) {
-        uint32_t sl = slot[j];
-        for (uint32_t probe = 0; probe <= slot_mask; ++probe) {
-          if (keys[sl] == c[j] + 1) { first[j] = (vals[sl] == M - (k0 + tid * PER + j)); break; }
-          sl = (sl + 1) & slot_mask;
-        }
-      }
+      first[j] = c[j] >= 0 && best[j] == M - (kt + j);
       mine += first[j];
     }
     int incl = mine;
@@ -797,16 +820,18 @@ SampleWs sample_ws_layout(int64_t N, int32_t M) {
   L.n_tiles = ceil_div(N, L.small ? kSmallTile : kSampleTile);
   L.n_super = L.small ? 1 : (int)ceil_div(L.n_tiles, kSuperTile);
   int64_t slots = 64;
-  while (slots < 2 * (int64_t)M) slots <<= 1;
+  while (!L.small && slots < 2 * (int64_t)M) slots <<= 1;      // the small form keeps first draws per prompt, no hash table
   L.hash_slots = slots;
   size_t off = 0;
-  // one zero-filled region: super-tile sums, hash keys, hash values
+  // one zero-filled region: super-tile sums (small form: the ticket), hash keys, hash values
   L.super_sums = off;   off = align_up(off + sizeof(unsigned long long) * (size_t)L.n_super, 256);
   L.keys = off;         off = align_up(off + sizeof(int32_t) * (size_t)slots, 256);
   L.vals = off;         off = align_up(off + sizeof(int32_t) * (size_t)slots, 256);
   L.zeroed_bytes = off;
-  L.tile_sums = off;    off = align_up(off + sizeof(unsigned long long) * (size_t)L.n_tiles, 256);
+  L.tile_sums = off;    off = align_up(off + sizeof(unsigned long long) * (size_t)L.n_tiles * (L.small ? 2 : 1), 256);
   L.cand = off;         off = align_up(off + sizeof(int32_t) * (size_t)M, 256);
+  L.slot_of = off;      off = align_up(off + sizeof(int32_t) * (size_t)M, 256);
+  L.first_draw = off;   off = align_up(off + (L.small ? sizeof(int32_t) * (size_t)(N + 1) : 0), 256);
   L.total = off;
   return L;
 }
@@ -824,25 +849,32 @@ cudaError_t launch_sample(const float* ab, int64_t N, const float* u, int32_t M,
   auto* tile_sums = reinterpret_cast<unsigned long long*>(ws + L.tile_sums);
   auto* super_sums = reinterpret_cast<unsigned long long*>(ws + L.super_sums);
   auto* cand = reinterpret_cast<int32_t*>(ws + L.cand);
+  auto* slot_of = reinterpret_cast<int32_t*>(ws + L.slot_of);
   auto* keys = reinterpret_cast<int32_t*>(ws + L.keys);
   auto* vals = reinterpret_cast<int32_t*>(ws + L.vals);
   cudaError_t e;
-  if ((e = cudaMemsetAsync(ws, 0, L.zeroed_bytes, st)) != cudaSuccess) return e;
   if (L.small) {
+    // four launches, nothing to clear beforehand (the first kernel clears the first-draw array);
+    // the prefix of the tile sums sits behind the tile sums themselves
     const float4* ab4 = reinterpret_cast<const float4*>(ab);
+    unsigned long long* tile_prefix = tile_sums + L.n_tiles;
+    int32_t* first_draw = reinterpret_cast<int32_t*>(ws + L.first_draw);
     if (out_w)
       sample_small_sums_kernel<true><<<(unsigned)L.n_tiles, kSmallTile / 2, 0, st>>>(
-          ab4, N, eps, reinterpret_cast<float2*>(out_w), out_w, tile_sums, d_status);
+          ab4, N, eps, reinterpret_cast<float2*>(out_w), out_w, tile_sums, first_draw, d_status);
     else
-      sample_small_sums_kernel<false><<<(unsigned)L.n_tiles, kSmallTile / 2, 0, st>>>(ab4, N, eps, nullptr, nullptr,
-                                                                                     tile_sums, d_status);
+      sample_small_sums_kernel<false><<<(unsigned)L.n_tiles, kSmallTile / 2, 0, st>>>(
+          ab4, N, eps, nullptr, nullptr, tile_sums, first_draw, d_status);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    sample_small_prefix_kernel<<<1, kSmallTilesMax / 4, 0, st>>>(tile_sums, (int)L.n_tiles, tile_prefix);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     sample_search_small_kernel<<<(unsigned)ceil_div(M, kSearchSmallThreads / 32), kSearchSmallThreads, 0, st>>>(
-        ab, N, eps, u, M, tile_sums, (int)L.n_tiles, cand, keys, vals, (uint32_t)(L.hash_slots - 1), d_status);
+        ab, N, eps, u, M, tile_prefix, (int)L.n_tiles, cand, slot_of, first_draw, d_status);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    sample_accept_kernel<<<1, 1024, 0, st>>>(cand, M, B, keys, vals, (uint32_t)(L.hash_slots - 1), out_ids, d_status);
+    sample_accept_kernel<<<1, 1024, 0, st>>>(cand, slot_of, M, B, first_draw, out_ids, d_status);
     return cudaGetLastError();
   }
+  if ((e = cudaMemsetAsync(ws, 0, L.zeroed_bytes, st)) != cudaSuccess) return e;
   if (out_w)
     sample_tile_sums_kernel<true><<<(unsigned)L.n_tiles, 256, 0, st>>>(
         reinterpret_cast<const float4*>(ab), N, eps, reinterpret_cast<float2*>(out_w), out_w, tile_sums, super_sums,
@@ -852,10 +884,10 @@ cudaError_t launch_sample(const float* ab, int64_t N, const float* u, int32_t M,
         reinterpret_cast<const float4*>(ab), N, eps, nullptr, nullptr, tile_sums, super_sums, d_status);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   sample_search_kernel<<<(unsigned)ceil_div((int64_t)M * 32, 256), 256, 0, st>>>(
-      ab, N, eps, u, M, tile_sums, super_sums, L.n_tiles, L.n_super, cand, keys, vals, (uint32_t)(L.hash_slots - 1),
-      d_status);
+      ab, N, eps, u, M, tile_sums, super_sums, L.n_tiles, L.n_super, cand, slot_of, keys, vals,
+      (uint32_t)(L.hash_slots - 1), d_status);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
-  sample_accept_kernel<<<1, 1024, 0, st>>>(cand, M, B, keys, vals, (uint32_t)(L.hash_slots - 1), out_ids, d_status);
+  sample_accept_kernel<<<1, 1024, 0, st>>>(cand, slot_of, M, B, vals, out_ids, d_status);
   return cudaGetLastError();
 }
 
