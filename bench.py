@@ -107,7 +107,7 @@ class Step:
     """Device buffers of one workload and the call sequence of one step."""
 
     def __init__(self, workload, device, rank, responses=None, custom=None, mask_frac=0.0, path="onepass",
-                 entropy=False, dp_world=None, dw_slabs=8):
+                 entropy=False, dp_world=None, dw_slabs=8, surrogate="ppo_clip", dual_clip=0.0):
         """dp_world = N: this rank holds its share of ONE mini-batch split over N ranks by token count
         (W and the tracker table replicated); None: the rank has a mini-batch of its own."""
         import torch
@@ -158,7 +158,8 @@ class Step:
         self.kl_table = torch.from_numpy(tb.kl_table).to(device)
         self.uniforms = torch.from_numpy(tb.uniforms).to(device)
         self.rewards = data["rewards"]
-        self.params = B.default_params()
+        self.params = B.default_params(surrogate={"ppo_clip": B.SUR_PPO_CLIP, "cispo": B.SUR_CISPO,
+                                                  "gspo": B.SUR_GSPO}[surrogate], dual_clip=float(dual_clip))
         self.ids = torch.empty(self.S_all, dtype=torch.int32, device=device)
         self.a_norm_all = torch.empty(self.S_all, **f32)      # one value per response of the whole mini-batch
         self.a_norm = self.a_norm_all                         # ... and of this rank's responses
@@ -327,7 +328,11 @@ def run_ours(args, rank, world, local_rank):
     if dp_mode and (args.path != "onepass" or args.mask_frac > 0.0 or args.custom):
         raise SystemExit("--parallelism dp runs the one-pass loss on the unmasked named workloads")
     step = Step(args.workload, device, rank, args.responses, args.custom, args.mask_frac, args.path, args.entropy,
-                dp_world=world if dp_mode else None, dw_slabs=args.dw_slabs)
+                dp_world=world if dp_mode else None, dw_slabs=args.dw_slabs, surrogate=args.surrogate,
+                dual_clip=args.dual_clip)
+    if args.surrogate == "gspo" and step.onepass:
+        # a response's ratio needs all its tokens: spo_loss_fwd_bwd runs forward-then-backward for it
+        step.flops_bwd = 6.0 * step.T * step.d * step.V
     peaks = read_peaks()
 
     def barrier():
@@ -425,6 +430,7 @@ def run_ours(args, rank, world, local_rank):
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": "custom" if args.custom else args.workload, "responses": step.S, "tokens": step.T, "d": step.d, "V": step.V,
                    "tracker_prompts": step.table_n, "l2": "inputs_exceed_l2", "loss_path": "onepass" if step.onepass else "split", "entropy_output": bool(args.entropy),
+                   "surrogate": args.surrogate, "dual_clip": args.dual_clip,
                    "bwd_chunks": step.bwd_chunks, "mask_frac": step.mask_frac,
                    "parallelism": ("dp%d" % world if dp_mode else "replicas%d" % world) if world > 1 else "single"},
         "gpu_launches": step.launches * args.steps,
@@ -435,13 +441,13 @@ def run_ours(args, rank, world, local_rank):
         "roofline": {
             "bound": "tensor",
             "kernel": ("spo_gemm_kernel (E, DH, DW instantiations; all launches of a step; the duration is the whole "
-                       "spo_loss_fwd_bwd call, which also holds the streaming e->g and finalisation kernels)" if step.onepass
+                       "spo_loss_fwd_bwd call, which also holds the first-tile pass, the finalisation and the row-scaling kernels)" if step.onepass
                        else "spo_gemm_kernel (FWD, G, DH, DW instantiations; all launches of a step)"),
             "achieved": achieved, "peak": peaks["tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["tflops"],
             "peak_source": peaks["source"] + " sustained cuBLAS bf16",
             "frac_of_nominal_2250": achieved / 2250.0, "frac_of_burst": achieved / peaks["tflops_burst"],
             "flops_per_step": step.flops_fwd + step.flops_bwd,
-            "flops_per_token": (6 if step.onepass else 8) * step.d * step.V,
+            "flops_per_token": (step.flops_fwd + step.flops_bwd) / max(1, step.n_tok if step.mask_frac > 0.0 else step.T),
             "fwd_tflops": None if step.onepass else step.flops_fwd / (t_fwd / args.steps / 1e3) / 1e12,
             "bwd_tflops": None if step.onepass else step.flops_bwd / (t_bwd / args.steps / 1e3) / 1e12,
             # DRAM read+write bytes of all launches of one step (ncu counters of one chunk's launches, scaled by
@@ -707,6 +713,9 @@ def main():
                          "spo_loss_bwd_rows)")
     ap.add_argument("--path", default="onepass", choices=["onepass", "split"],
                     help="loss as one spo_loss_fwd_bwd call (default) or as spo_loss_fwd + spo_loss_bwd")
+    ap.add_argument("--surrogate", default="ppo_clip", choices=["ppo_clip", "cispo", "gspo"],
+                    help="objective of the loss calls: the paper's PPO-Clip, or one of the two it names as compatible")
+    ap.add_argument("--dual-clip", type=float, default=0.0, help="second clip for negative advantages (0 = off)")
     ap.add_argument("--entropy", action="store_true", help="also ask the loss call for the per-token policy entropy")
     ap.add_argument("--parallelism", default="replicas", choices=["replicas", "dp"],
                     help="with more than one GPU: every rank its own mini-batch (weak scaling, no data-path "

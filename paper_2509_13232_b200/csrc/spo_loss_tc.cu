@@ -191,6 +191,17 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       : "memory");
 }
 
+#ifdef SPO_TUNE_EHINT
+// Same load with an L2 eviction-priority policy (tuning builds only).
+__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar,
+                                                 uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar), "l"(policy)
+      : "memory");
+}
+#endif
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -435,6 +446,13 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
               if (rank == 0) mbar_expect_tx(full0 + 8 * s, CG * STAGE_BYTES);   // both CTAs' bytes land on the leader's barrier
               const uint32_t fb = map_to_cta(full0 + 8 * s, 0);
               if (!A_MN) {
+#ifdef SPO_TUNE_EHINT
+                if (MODE == MODE_E) {
+                  uint64_t pol;
+                  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+                  tma_load_2d_hint(sa, &tmA, kb * BK, p.a_row0 + row_base, fb, pol);
+                } else
+#endif
                 tma_load_2d(sa, &tmA, kb * BK, p.a_row0 + row_base, fb);
               } else {
 #pragma unroll
@@ -851,7 +869,10 @@ cudaError_t launch_gemm(const CUtensorMap& a, const CUtensorMap& b, const GemmPa
   if (units <= 0) return cudaSuccess;
   GemmParams p = p_in;
   p.window = kLockStepWindow;
-  p.sync_kblocks = p.k_blocks;                 // compare progress once per tile
+  // The pairs compare progress once per tile.  Comparing every 64 or 128 k-blocks inside the long
+  // tiles of DH / DW was measured too (SPO_TUNE_SYNCKB): same step time, and on one and the same GPU the
+  // same DRAM traffic (DH 14.2 against 14.7 GB per chunk, DW rather more than less).
+  p.sync_kblocks = p.k_blocks;
 #ifdef SPO_TUNE_SYNCKB
   if (MODE == MODE_DH || MODE == MODE_DW) p.sync_kblocks = p.k_blocks < SPO_TUNE_SYNCKB ? p.k_blocks : SPO_TUNE_SYNCKB;
 #endif
