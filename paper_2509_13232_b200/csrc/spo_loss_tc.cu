@@ -548,7 +548,7 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       }
       if (MODE == MODE_DH && p.rowscale && row_ok) rs = p.rowscale[grow];
       for (int n = un.n_begin; n < un.n_end && ok; ++n, ++tile) {
-        {                                   // one lane polls (with backoff); the warp reconverges on its verdict
+        {                                   // one lane polls (with backoff); the warp reconverges on the outcome
           int good = 1;
           if (lane == 0) good = mbar_wait<kEpilogueSleepNs>(tfull, tile & 1u, abort_flag, p.d_status) ? 1 : 0;
           good = __shfl_sync(0xffffffffu, good, 0);

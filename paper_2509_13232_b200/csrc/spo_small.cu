@@ -570,16 +570,14 @@ constexpr unsigned kBadId = 1u, kBadValue = 2u;
 // the value just read (Sec. 3.1), so the entry crosses the memory system once per step.
 // Out-of-range ids, negative / non-finite entries and non-finite rewards or divergences are
 // reported in `bad`; the element then contributes A = 0 and its entry stays untouched.
+// The arithmetic of one element once its entry (and divergence) are in registers.
 template <bool UPDATE>
-__device__ __forceinline__ float advantage_element(float2* __restrict__ ab, int64_t N, int32_t id, float r, int64_t j,
+__device__ __forceinline__ float advantage_compute(float2* __restrict__ ab, int32_t id, float2 e, float r, float div,
                                                    const UpdateArgs& u, unsigned& bad) {
-  if (id < 0 || (int64_t)id >= N) { bad |= kBadId; return 0.0f; }
-  float2 e = load_entry(ab + id);
   bool bad_entry = false;
   const float v = entry_estimate(e, bad_entry);
   if (bad_entry | !(fabsf(r) < CUDART_INF_F)) { bad |= kBadValue; return 0.0f; }
   if (UPDATE) {
-    const float div = u.kl_is_table ? __ldg(u.kl + id) : u.kl[j];
     if (isnan(div)) {
       bad |= kBadValue;                      // entry untouched; the advantage itself is well defined
     } else {
@@ -591,6 +589,16 @@ __device__ __forceinline__ float advantage_element(float2* __restrict__ ab, int6
     }
   }
   return r - v;
+}
+
+template <bool UPDATE>
+__device__ __forceinline__ float advantage_element(float2* __restrict__ ab, int64_t N, int32_t id, float r, int64_t j,
+                                                   const UpdateArgs& u, unsigned& bad) {
+  if (id < 0 || (int64_t)id >= N) { bad |= kBadId; return 0.0f; }
+  const float2 e = load_entry(ab + id);
+  float div = 0.0f;
+  if (UPDATE) div = u.kl_is_table ? __ldg(u.kl + id) : u.kl[j];
+  return advantage_compute<UPDATE>(ab, id, e, r, div, u, bad);
 }
 
 __device__ __forceinline__ void flag_bad(int32_t* d_status, unsigned bad) {
@@ -624,12 +632,35 @@ advantages_single_kernel(float2* __restrict__ ab, int64_t N, const int32_t* __re
   float a[PER];
   AdvSums t = {0.0, 0.0, 0.0, 0.0};
   unsigned bad = 0;
+  // The one block is bound by memory latency: first every id, reward and divergence of the thread's
+  // elements, then all their table entries, are requested together before any is used.
+  int32_t id[PER];
+  float rew[PER], div[PER];
+  float2 e[PER];
+  bool live[PER];
 #pragma unroll
   for (int j = 0; j < PER; ++j) {
-    int i = j * 1024 + threadIdx.x;
+    const int i = j * 1024 + threadIdx.x;
+    live[j] = i < B;
+    id[j] = live[j] ? ids[i] : 0;
+    rew[j] = live[j] ? r[i] : 0.0f;
+    div[j] = (UPDATE && live[j] && !u.kl_is_table) ? u.kl[i] : 0.0f;
+  }
+#pragma unroll
+  for (int j = 0; j < PER; ++j) {
+    e[j] = make_float2(0.0f, 0.0f);
+    if (live[j] && (id[j] < 0 || (int64_t)id[j] >= N)) { bad |= kBadId; live[j] = false; }
+    if (live[j]) {
+      e[j] = load_entry(ab + id[j]);
+      if (UPDATE && u.kl_is_table) div[j] = __ldg(u.kl + id[j]);
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < PER; ++j) {
+    const int i = j * 1024 + threadIdx.x;
     a[j] = 0.0f;
     if (i < B) {
-      a[j] = advantage_element<UPDATE>(ab, N, ids[i], r[i], i, u, bad);
+      if (live[j]) a[j] = advantage_compute<UPDATE>(ab, id[j], e[j], rew[j], div[j], u, bad);
       adv_accumulate(t, a[j], na.tau_lo, na.tau_hi);
       if (a_raw) a_raw[i] = a[j];
     }
