@@ -337,8 +337,8 @@ int32_t spo_loss_bwd(const void* H, const void* W, int32_t dtype, const int32_t*
  *   g[t,v] = rowscale_t (e[t,v] - l_t 1[v = y_t]),   rowscale_t = -grad_loss coef_t / l_t:
  * after the chunk's rows are finalised the one target entry per row is patched in the stored chunk,
  * dH = rowscale (e W) takes the factor in its epilogue and dW = e^T (rowscale H) reads a scaled bf16
- * copy of the chunk's rows of H; the stored chunk is never rewritten.  dW is contracted over two
- * chunks at a time.  loss, logp, lse and coef never see the bf16 rounding of e; dH and dW carry it
+ * copy of the chunk's rows of H; the stored chunk is never rewritten.
+ * loss, logp, lse and coef never see the bf16 rounding of e; dH and dW carry it
  * (and dW the rounding of rowscale H) in place of spo_loss_bwd's own bf16 rounding of g.
  * Range: a row whose largest logit exceeds the largest of its first 512 by more than 100 nats
  * overflows the stored exponentials; such a row sets SPO_DEV_NONFINITE, gets lse = Inf, logp = -Inf,
@@ -350,8 +350,8 @@ int32_t spo_loss_bwd(const void* H, const void* W, int32_t dtype, const int32_t*
  *               which may lie in later chunks, so the call runs the forward to the end and then the
  *               chunked backward (four contractions, the cost of the two calls).
  *   ws          device scratch, spo_workspace_bytes(SPO_WS_LOSS_FWD_BWD, T, d, V, 0, S, 0) bytes:
- *               two chunk buffers when T exceeds one chunk, scaled copies of their rows of H, 36 bytes
- *               per token row and the forward's partials
+ *               one chunk buffer (a few thousand token rows by V, bf16), a scaled bf16 copy of the chunk's
+ *               rows of H, 36 bytes per token row and the forward's partials
  * Status bits as spo_loss_fwd.
  */
 int32_t spo_loss_fwd_bwd(const void* H, const void* W, int32_t dtype,
