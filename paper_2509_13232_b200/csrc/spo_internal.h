@@ -70,8 +70,9 @@ cudaError_t launch_tracker_update_repeats(float* ab, int64_t N, const int32_t* i
 
 // ---- loss: pieces shared by the fp32 and bf16 paths ------------------------
 // Forward partial statistics of one vocabulary split, per token row:
-// (running max of z*log2(e), sum e of 2^(z*log2(e) - max), target logit or -inf, and in `pad`
-// the sum of e*z when the entropy was asked for).
+// (exponent m2 the sums are relative to, in log2 units: the running max of z*log2(e), or on the
+// one-pass path the row's fixed reference exponent; sum of 2^(z*log2(e) - m2); target logit or -inf;
+// and in `pad` the sum of e*z when the entropy was asked for).
 struct FwdPartial { float m2, l, zt; float pad; };
 
 constexpr int kFinalizeThreads = 256;
