@@ -142,8 +142,12 @@ int32_t spo_tracker_init(float* ab, const float* v0, int64_t N,
  *   ab        device in  [N][2]
  *   uniforms  device in  [M] fp32 in [0,1); M >= B (M = 2B is ample for N >> B)
  *   out_ids   device out [B] int32, in acceptance order
- *   out_w     device out [N] fp32 weights, optional
- *   ws        device scratch, spo_workspace_bytes(SPO_WS_SAMPLE, ..., N, B, M) bytes
+ *   out_w     device out [N] fp32 weights, optional (the ids do not depend on whether it is given;
+ *             given the same uniforms and these weights, the ids are fully determined by the
+ *             integer arithmetic above)
+ *   ws        device scratch, spo_workspace_bytes(SPO_WS_SAMPLE, ..., N, B, M) bytes (for tables of up
+ *             to 2^20 prompts it includes 4 bytes per prompt: the call is organised for latency there,
+ *             four short launches; larger tables are scanned at HBM speed)
  * Limits: 1 <= N < 2^31, 1 <= B <= M <= 2^20.
  * Device status: SPO_DEV_UNIFORMS_EXHAUSTED if fewer than B distinct candidates
  * (the tail of out_ids is then filled with -1), SPO_DEV_ZERO_TOTAL_WEIGHT,
