@@ -648,6 +648,12 @@ def spawn_ranks(n):
     the rendezvous environment a launcher would give them (127.0.0.1, a free port).  Rank 0 prints the
     JSON line.  Returns the worst exit code."""
     import socket
+    if "--rehearse-host" not in sys.argv:
+        import torch
+        have = torch.cuda.device_count()
+        if have < n:
+            sys.stderr.write("bench.py: --gpus %d asked for, %d CUDA device(s) visible\n" % (n, have))
+            return 2
     with socket.socket() as sock:
         sock.bind(("127.0.0.1", 0))
         port = sock.getsockname()[1]
@@ -658,7 +664,19 @@ def spawn_ranks(n):
         env.setdefault("NCCL_DEBUG", "INFO")              # the communicator log (transport, NVLS) goes to stderr
         env.setdefault("NCCL_DEBUG_SUBSYS", "INIT")
         procs.append(subprocess.Popen([sys.executable, os.path.abspath(__file__)] + sys.argv[1:], env=env))
-    codes = [p.wait() for p in procs]
+    # a rank that dies would leave the others waiting in a collective: stop them when one fails
+    codes = [None] * n
+    while any(c is None for c in codes):
+        for i, pr in enumerate(procs):
+            if codes[i] is None:
+                codes[i] = pr.poll()
+        if any(c not in (None, 0) for c in codes):
+            for i, pr in enumerate(procs):
+                if codes[i] is None:
+                    pr.terminate()
+                    codes[i] = pr.wait()
+            break
+        time.sleep(0.2)
     return max(abs(c) for c in codes)
 
 
