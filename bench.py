@@ -555,6 +555,19 @@ def run_small_kernels(args, local_rank):
                 total_ms += ms
                 total_bytes += nbytes
             launches += n_launch * args.steps
+    # reference for the gathers: the same random 8-byte rows fetched by a library primitive
+    idx64 = ids.to(torch.int64)
+    picked = torch.empty((Bn, 2), device=dev)
+    tr = []
+    for i in range(args.warmup + args.steps):
+        flush.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(); torch.index_select(ab, 0, idx64, out=picked); e1.record()
+        torch.cuda.synchronize()
+        if i >= args.warmup:
+            tr.append(e0.elapsed_time(e1))
+    tr.sort()
+    gather_ref_ms = tr[len(tr) // 2]
     dom = out_calls["spo_sample_prompts"]
     print(json.dumps({
         "metric": "tracker / advantage / sampling kernels, achieved HBM GB/s (algorithmic bytes)",
@@ -563,6 +576,8 @@ def run_small_kernels(args, local_rank):
         "data": "synthetic",
         "config": {"workload": args.workload, "N": N, "B": Bn, "M": M, "l2": "flushed_before_each_call"},
         "gpu_launches": launches, "device_status": int(st[0].item()), "calls": out_calls,
+        "random_gather_reference": {"what": "torch.index_select of the same B random 8-byte table rows", "ms": gather_ref_ms,
+                                    "accesses_per_s": Bn / gather_ref_ms * 1e3},
         "roofline": {"bound": "hbm", "kernel": "sample_tile_sums_kernel (within spo_sample_prompts)",
                      "achieved": dom["GB/s"], "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": dom["frac_of_hbm"],
                      "peak_source": peaks["source"] + " copy", "traffic": None},
