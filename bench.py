@@ -324,7 +324,7 @@ def run_ours(args, rank, world, local_rank):
         spo_build.build()
     if world > 1:
         dist.barrier()
-    dp_mode = args.parallelism == "dp" and world > 1
+    dp_mode = args.parallelism == "dp" and dist.is_available() and dist.is_initialized()
     if dp_mode and (args.path != "onepass" or args.mask_frac > 0.0 or args.custom):
         raise SystemExit("--parallelism dp runs the one-pass loss on the unmasked named workloads")
     step = Step(args.workload, device, rank, args.responses, args.custom, args.mask_frac, args.path, args.entropy,
@@ -432,7 +432,7 @@ def run_ours(args, rank, world, local_rank):
                    "tracker_prompts": step.table_n, "l2": "inputs_exceed_l2", "loss_path": "onepass" if step.onepass else "split", "entropy_output": bool(args.entropy),
                    "surrogate": args.surrogate, "dual_clip": args.dual_clip,
                    "bwd_chunks": step.bwd_chunks, "mask_frac": step.mask_frac,
-                   "parallelism": ("dp%d" % world if dp_mode else "replicas%d" % world) if world > 1 else "single"},
+                   "parallelism": "dp%d" % world if dp_mode else ("replicas%d" % world if world > 1 else "single")},
         "gpu_launches": step.launches * args.steps,
         "device_status": status,
         "wall_s": wall,
@@ -779,7 +779,10 @@ def main():
     if args.impl == "reference":
         run_reference(args, rank, world)
         return
-    if world > 1:
+    # a process group for N > 1 ranks, and for one rank under a launcher when the data-parallel step is asked
+    # for (its exchanges are then the identity: what that step costs by itself on one GPU)
+    grouped = world > 1 or (args.parallelism == "dp" and "WORLD_SIZE" in os.environ)
+    if grouped:
         import torch
         import torch.distributed as dist
         torch.cuda.set_device(local_rank)
@@ -787,7 +790,7 @@ def main():
     try:
         run_ours(args, rank, world, local_rank)
     finally:
-        if world > 1:
+        if grouped:
             import torch.distributed as dist
             dist.destroy_process_group()
 

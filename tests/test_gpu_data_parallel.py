@@ -153,3 +153,40 @@ def test_slab_cut_last_dw_contraction_is_bitwise_the_plain_call_and_reduces_in_s
         want = O.loss_forward(lb.h, lb.w, lb.y, lb.logp_old, lb.mask, lb.cu_seqlens, lb.a_norm)
         _, want_dw = O.loss_backward(lb.h, lb.w, lb.y, want["lse"], want["coef"])
         assert rel_fro(total.cpu().numpy(), want_dw) <= 1e-2
+
+
+def test_data_parallel_step_with_one_rank_equals_the_plain_step():
+    """The step bench.py runs under `--parallelism dp` (rewards put together over the ranks, whole-batch
+    advantages and tracker update on every rank, global denominators, slab-cut loss call with the
+    reductions behind the events) on a process group of ONE rank: every exchange is the identity, so
+    every output must equal the plain step's bit for bit.  (More ranks cannot run here; their host
+    logic is covered on gloo ranks.)"""
+    import os
+    import socket
+    import torch
+    import torch.distributed as dist
+    import bench
+    dev0 = torch.device("cuda", 0)
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    os.environ["MASTER_ADDR"], os.environ["MASTER_PORT"] = "127.0.0.1", str(port)
+    dist.init_process_group("nccl", rank=0, world_size=1, device_id=dev0)
+    try:
+        plain = bench.Step("cfg3_small_bf16", dev0, 0)
+        plain.run()
+        torch.cuda.synchronize()
+        keep = [t.clone() for t in (plain.loss, plain.logp, plain.coef, plain.dH, plain.dW, plain.ids, plain.ab,
+                                    plain.a_norm)]
+        assert int(plain.status[0].item()) == 0
+        del plain
+        torch.cuda.empty_cache()
+        part = bench.Step("cfg3_small_bf16", dev0, 0, dp_world=1, dw_slabs=8)
+        assert len(part.reducer.events) >= 2 and part.my_responses.tolist() == list(range(part.S_all))
+        part.run()
+        torch.cuda.synchronize()
+        assert int(part.status[0].item()) == 0
+        for a, b in zip(keep, (part.loss, part.logp, part.coef, part.dH, part.dW, part.ids, part.ab, part.a_norm)):
+            assert torch.equal(a, b)
+    finally:
+        dist.destroy_process_group()
