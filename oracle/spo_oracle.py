@@ -16,7 +16,8 @@ checked against ``sampling_weights`` (the float64 definition) separately.
 Pinned by tests/test_oracle_pins.py against closed forms, brute force, finite
 differences and the constants the paper prints.  Pieces whose parameters the
 paper never gives a value or a formula for (``d_half``; the two objectives
-Sec. 3.2 only names, ``SUR_CISPO`` and ``SUR_GSPO``; the whole-step
+Sec. 3.2 only names, ``SUR_CISPO`` and ``SUR_GSPO``; the optional second clip
+``dual_clip``, which is not in the paper at all; the whole-step
 composition, for which no worked example is printed) are "parity unpinned" by
 the paper itself and are pinned only through the identities listed in that
 test file.
