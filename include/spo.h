@@ -385,6 +385,7 @@ int32_t spo_loss_fwd_bwd(const void* H, const void* W, int32_t dtype,
  * All other arguments as in spo_loss_fwd_bwd.  The library creates, waits on and destroys nothing.
  */
 #define SPO_MAX_DW_SLABS 64
+#define SPO_MAX_DW_SHARDS 16
 int32_t spo_dw_slab_rows(int32_t V, int32_t d, int32_t n_wanted, int64_t* row_begin /* host, [n_wanted+1] */);
 int32_t spo_loss_fwd_bwd_slabs(const void* H, const void* W, int32_t dtype,
                                const int32_t* y, const float* logp_old, const uint8_t* mask,
@@ -395,6 +396,40 @@ int32_t spo_loss_fwd_bwd_slabs(const void* H, const void* W, int32_t dtype,
                                void* ws, size_t ws_bytes,
                                const spo_params* params, int32_t* d_status, void* stream,
                                int32_t n_wanted, void* const* events /* host, [n_wanted] */);
+
+/*
+ * spo_loss_fwd_bwd with the reduce-scatter of dW fused into its last contraction (data-parallel ranks whose
+ * optimizer is sharded over the vocabulary rows of W; Algorithm 1's mini-batch update spread over GPUs).
+ * The vocabulary rows are cut into n_shards equal shards of rows_per_shard rows (the last may be shorter);
+ * shard k lives in the memory of rank k (shard[k]: fp32 [rows_per_shard][d]; for k != own rank a pointer to
+ * PEER device memory mapped into this process).  The epilogue of the call's LAST dW contraction adds each
+ * finished tile of dW (the sum over all chunks of this rank's tokens) straight into the shard that owns its
+ * rows with vector store-reductions (`red.global.add` — over NVLink for a peer's shard; nothing is loaded
+ * from a peer and nothing waits on a peer), so the exchange overlaps the contraction tile by tile and no
+ * collective library call touches dW.  After every rank's call has completed (a barrier the caller
+ * provides: stream synchronise + process-group barrier), shard[own rank] holds the mini-batch's dW rows.
+ *   - Every shard must be zeroed by its owner, and that zeroing visible to all ranks, before any rank's call.
+ *   - dW is scratch here (it ends up holding the partial sums of the chunks before the last); dW_accumulate
+ *     still means "dW already holds a term to include".
+ *   - Summation order across ranks is not fixed: results are reproducible up to fp32 addition order.
+ *   - Inputs for which the last contraction is not this kernel (fp32, SPO_SUR_GSPO, T = 0) are followed by
+ *     a plain kernel that adds dW into the shards the same way.
+ * All other arguments and outputs as spo_loss_fwd_bwd.
+ */
+typedef struct spo_dw_shards {
+  int32_t n_shards;                       /* 1 .. SPO_MAX_DW_SHARDS */
+  int64_t rows_per_shard;                 /* n_shards * rows_per_shard >= V */
+  float*  shard[SPO_MAX_DW_SHARDS];       /* device pointers (own or peer memory), 16-byte aligned */
+} spo_dw_shards;
+int32_t spo_loss_fwd_bwd_scatter(const void* H, const void* W, int32_t dtype,
+                                 const int32_t* y, const float* logp_old, const uint8_t* mask,
+                                 const int32_t* cu_seqlens, const float* a_norm,
+                                 int64_t T, int32_t d, int32_t V, int32_t S, float grad_loss,
+                                 float* loss, float* logp, float* lse, float* coef, float* seq_sums, float* entropy,
+                                 void* dH, int32_t dH_dtype, float* dW, int32_t dW_accumulate,
+                                 void* ws, size_t ws_bytes,
+                                 const spo_params* params, int32_t* d_status, void* stream,
+                                 const spo_dw_shards* shards /* host */);
 
 /*
  * Diagnostic (no counterpart in the paper): runs the kernels' bounded mbarrier wait on a barrier

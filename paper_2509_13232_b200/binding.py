@@ -28,7 +28,7 @@ SUR_PPO_CLIP, SUR_CISPO, SUR_GSPO = 0, 1, 2
 EXPORTS = [
     "spo_default_params", "spo_tracker_init", "spo_sample_prompts", "spo_advantages",
     "spo_advantages_static", "spo_advantages_apply", "spo_advantages_update",
-    "spo_tracker_update", "spo_tracker_update_repeats", "spo_loss_fwd", "spo_loss_bwd", "spo_loss_fwd_bwd", "spo_loss_fwd_bwd_slabs", "spo_dw_slab_rows", "spo_loss_stats", "spo_loss_mask_rows", "spo_loss_fwd_bwd_rows", "spo_loss_active_rows", "spo_loss_bwd_rows", "spo_workspace_bytes",
+    "spo_tracker_update", "spo_tracker_update_repeats", "spo_loss_fwd", "spo_loss_bwd", "spo_loss_fwd_bwd", "spo_loss_fwd_bwd_slabs", "spo_dw_slab_rows", "spo_loss_fwd_bwd_scatter", "spo_loss_stats", "spo_loss_mask_rows", "spo_loss_fwd_bwd_rows", "spo_loss_active_rows", "spo_loss_bwd_rows", "spo_workspace_bytes",
     "spo_status_string", "spo_last_cuda_error", "spo_version", "spo_selftest_bounded_wait",
 ]
 
@@ -41,6 +41,13 @@ class SpoParams(Structure):
         ("surrogate", c_int32), ("dual_clip", c_float), ("near_zero_tau_lo", c_float),
         ("near_zero_tau_hi", c_float),
     ]
+
+
+MAX_DW_SHARDS = 16
+
+
+class SpoDwShards(Structure):
+    _fields_ = [("n_shards", c_int32), ("rows_per_shard", c_int64), ("shard", c_void_p * MAX_DW_SHARDS)]
 
 
 class SpoError(RuntimeError):
@@ -93,6 +100,7 @@ def lib():
                                        c_void_p, c_int32, c_void_p, c_int32,
                                        c_void_p, c_size_t, P, c_void_p, c_void_p]
         L.spo_loss_fwd_bwd_slabs.argtypes = list(L.spo_loss_fwd_bwd.argtypes) + [c_int32, POINTER(c_void_p)]
+        L.spo_loss_fwd_bwd_scatter.argtypes = list(L.spo_loss_fwd_bwd.argtypes) + [POINTER(SpoDwShards)]
         L.spo_dw_slab_rows.argtypes = [c_int32, c_int32, c_int32, POINTER(c_int64)]
         L.spo_loss_stats.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_int32, c_void_p, P,
                                      c_void_p]
@@ -268,6 +276,31 @@ def spo_loss_fwd_bwd_slabs(H, W, y, logp_old, mask, cu_seqlens, a_norm, grad_los
                                         _dtype_code(dH), _ptr(dW), int(dW_accumulate), _ptr(ws),
                                         ws.numel() * ws.element_size(), ctypes.byref(params), _ptr(d_status), _stream(),
                                         len(events), handles), "spo_loss_fwd_bwd_slabs")
+
+
+def dw_shards(shard_ptrs, rows_per_shard) -> SpoDwShards:
+    """Shard table for spo_loss_fwd_bwd_scatter: shard_ptrs[k] is the device address (an int, or a tensor) of the
+    fp32 [rows_per_shard][d] buffer that owns vocabulary rows k*rows_per_shard ..; it may be peer memory."""
+    sh = SpoDwShards()
+    sh.n_shards = len(shard_ptrs)
+    sh.rows_per_shard = int(rows_per_shard)
+    for k, ptr in enumerate(shard_ptrs):
+        sh.shard[k] = ptr if isinstance(ptr, int) else ptr.data_ptr()
+    return sh
+
+
+def spo_loss_fwd_bwd_scatter(H, W, y, logp_old, mask, cu_seqlens, a_norm, grad_loss, loss, logp, lse, coef, seq_sums,
+                             dH, dW, dW_accumulate, ws, params, d_status, shards, entropy=None):
+    """spo_loss_fwd_bwd whose last dW contraction adds the finished dW into the shards that own its rows."""
+    T, d = H.shape
+    V = W.shape[0]
+    S = cu_seqlens.numel() - 1
+    _check(lib().spo_loss_fwd_bwd_scatter(_ptr(H), _ptr(W), _dtype_code(W), _ptr(y), _ptr(logp_old), _ptr(mask),
+                                          _ptr(cu_seqlens), _ptr(a_norm), T, d, V, S, c_float(grad_loss), _ptr(loss),
+                                          _ptr(logp), _ptr(lse), _ptr(coef), _ptr(seq_sums), _ptr(entropy), _ptr(dH),
+                                          _dtype_code(dH), _ptr(dW), int(dW_accumulate), _ptr(ws),
+                                          ws.numel() * ws.element_size(), ctypes.byref(params), _ptr(d_status),
+                                          _stream(), ctypes.byref(shards)), "spo_loss_fwd_bwd_scatter")
 
 
 def spo_loss_stats(logp, logp_old, mask, cu_seqlens, a_norm, out, params):

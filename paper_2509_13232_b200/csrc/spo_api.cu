@@ -315,8 +315,18 @@ static int32_t loss_fwd_bwd_impl(const void* H, const void* W, int32_t dtype, co
                                  int32_t V, int32_t S, float grad_loss, float* loss, float* logp, float* lse, float* coef,
                                  float* seq_sums, float* entropy, void* dH, int32_t dH_dtype, float* dW,
                                  int32_t dW_accumulate, void* ws, size_t ws_bytes, const spo_params* params,
-                                 int32_t* d_status, void* stream, int32_t n_slabs, void* const* events) {
+                                 int32_t* d_status, void* stream, int32_t n_slabs, void* const* events,
+                                 const spo_dw_shards* shards = nullptr) {
   int32_t rc = check_loss_shape(dtype, T, d, V);
+  if (shards) {
+    if (shards->n_shards < 1 || shards->n_shards > SPO_MAX_DW_SHARDS || shards->rows_per_shard < 1 ||
+        (int64_t)shards->n_shards * shards->rows_per_shard < V)
+      return SPO_ERR_INVALID_ARG;
+    for (int k = 0; k < shards->n_shards; ++k) {
+      if (!shards->shard[k]) return SPO_ERR_INVALID_ARG;
+      if (!aligned16(shards->shard[k])) return SPO_ERR_BAD_ALIGNMENT;
+    }
+  }
   if (rc != SPO_OK) return rc;
   if (dH_dtype != SPO_DTYPE_F32 && dH_dtype != SPO_DTYPE_BF16) return SPO_ERR_UNSUPPORTED_DTYPE;
   if (!params_ok(params) || !W || !loss || !dW || !ws || !cu_seqlens || S < 0) return SPO_ERR_INVALID_ARG;
@@ -347,6 +357,7 @@ static int32_t loss_fwd_bwd_impl(const void* H, const void* W, int32_t dtype, co
       return cuda_fail(e);
     e = launch_bwd_bf16(H, W, y, lse, coef, grad_loss, T, d, V, dH, dH_dtype, dW, dW_accumulate, w8 + off_b, Lb,
                         d_status, st);
+    if (e == cudaSuccess && shards) e = launch_dw_scatter_add(dW, V, d, *shards, st);
     if (e == cudaSuccess && n_slabs > 0) e = record_all(events, slabs_used, st);
     return e == cudaSuccess ? SPO_OK : cuda_fail(e);
   }
@@ -360,6 +371,7 @@ static int32_t loss_fwd_bwd_impl(const void* H, const void* W, int32_t dtype, co
     a.dH = dH; a.dH_dtype = dH_dtype; a.dW = dW; a.accumulate = dW_accumulate;
     a.params = params; a.d_status = d_status;
     a.n_slabs = n_slabs; a.events = reinterpret_cast<cudaEvent_t*>(const_cast<void**>(events));
+    a.shards = shards;
     e = launch_fused_bf16(a, w8, L, st);
     return e == cudaSuccess ? SPO_OK : cuda_fail(e);
   }
@@ -371,6 +383,7 @@ static int32_t loss_fwd_bwd_impl(const void* H, const void* W, int32_t dtype, co
     return cuda_fail(e);
   e = launch_bwd_f32((const float*)H, (const float*)W, y, lse, coef, grad_loss, T, d, V, dH, dH_dtype, dW,
                      dW_accumulate, st);
+  if (e == cudaSuccess && shards) e = launch_dw_scatter_add(dW, V, d, *shards, st);
   if (e == cudaSuccess && n_slabs > 0) e = record_all(events, slabs_used, st);
   return e == cudaSuccess ? SPO_OK : cuda_fail(e);
 }
@@ -385,6 +398,18 @@ int32_t spo_loss_fwd_bwd(const void* H, const void* W, int32_t dtype, const int3
   return loss_fwd_bwd_impl(H, W, dtype, y, logp_old, mask, cu_seqlens, a_norm, T, d, V, S, grad_loss, loss, logp, lse,
                            coef, seq_sums, entropy, dH, dH_dtype, dW, dW_accumulate, ws, ws_bytes, params, d_status,
                            stream, 0, nullptr);
+}
+
+int32_t spo_loss_fwd_bwd_scatter(const void* H, const void* W, int32_t dtype, const int32_t* y, const float* logp_old,
+                                 const uint8_t* mask, const int32_t* cu_seqlens, const float* a_norm, int64_t T,
+                                 int32_t d, int32_t V, int32_t S, float grad_loss, float* loss, float* logp, float* lse,
+                                 float* coef, float* seq_sums, float* entropy, void* dH, int32_t dH_dtype, float* dW,
+                                 int32_t dW_accumulate, void* ws, size_t ws_bytes, const spo_params* params,
+                                 int32_t* d_status, void* stream, const spo_dw_shards* shards) {
+  if (!shards) return SPO_ERR_INVALID_ARG;
+  return loss_fwd_bwd_impl(H, W, dtype, y, logp_old, mask, cu_seqlens, a_norm, T, d, V, S, grad_loss, loss, logp, lse,
+                           coef, seq_sums, entropy, dH, dH_dtype, dW, dW_accumulate, ws, ws_bytes, params, d_status,
+                           stream, 0, nullptr, shards);
 }
 
 int32_t spo_dw_slab_rows(int32_t V, int32_t d, int32_t n_wanted, int64_t* row_begin) {

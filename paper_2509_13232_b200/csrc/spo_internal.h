@@ -186,7 +186,12 @@ struct FusedArgs {
   // (0 / NULL: one launch, no events).
   int n_slabs;
   cudaEvent_t* events;
+  // Reduce-scatter form (shards != NULL): the last dW contraction adds the finished dW, tile by tile, into
+  // the shards that own its vocabulary rows (spo_loss_fwd_bwd_scatter); dW itself is then scratch.
+  const spo_dw_shards* shards;
 };
+// dW[V][d] added into the shards that own its rows (the paths that do not fuse this into a contraction)
+cudaError_t launch_dw_scatter_add(const float* dW, int32_t V, int32_t d, const spo_dw_shards& sh, cudaStream_t st);
 // Vocabulary-row bounds of the slabs the last dW contraction is cut into: row_begin[0..n] with
 // row_begin[0] = 0 and row_begin[n] = V; returns n <= n_wanted (slabs hold whole rounds of row tiles).
 int dw_slab_rows(int32_t V, int32_t d, int n_wanted, int64_t* row_begin);

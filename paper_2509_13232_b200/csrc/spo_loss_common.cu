@@ -470,6 +470,22 @@ scale_rows_kernel(const uint4* __restrict__ H, const float* __restrict__ rowscal
   }
 }
 
+// dW added, row by row, into the shards that own its vocabulary rows (the reduce-scatter form of the
+// paths whose last contraction does not do it itself).  16-byte pieces, vector store-reductions.
+struct ShardTable { float* shard[SPO_MAX_DW_SHARDS]; int n; int64_t rows; };
+
+__global__ void __launch_bounds__(256)
+dw_scatter_add_kernel(const float4* __restrict__ dW, int64_t n_vec, int row_vec, ShardTable tb) {
+  for (int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x; i < n_vec; i += (int64_t)gridDim.x * 256) {
+    const int64_t v = i / row_vec;
+    const int owner = (int)(v / tb.rows);
+    const float4 x = dW[i];
+    float* dst = tb.shard[owner] + ((v - (int64_t)owner * tb.rows) * row_vec + (i - v * row_vec)) * 4;
+    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "f"(x.x), "f"(x.y), "f"(x.z), "f"(x.w)
+                 : "memory");
+  }
+}
+
 // Sequence-level objective, one block per response: r = exp(mean over its unmasked tokens of
 // logp - logp_old), term = min(r a, clip(r) a), and the coef all its unmasked tokens share.
 __global__ void __launch_bounds__(256)
@@ -778,6 +794,20 @@ cudaError_t launch_scale_rows(const void* H, const float* rowscale, int64_t t0, 
   if (blocks > cap) blocks = cap;
   scale_rows_kernel<<<(unsigned)blocks, 256, 0, st>>>(reinterpret_cast<const uint4*>(H), rowscale, t0, rows,
                                                       row_bytes / 16, reinterpret_cast<uint4*>(out));
+  return cudaGetLastError();
+}
+
+cudaError_t launch_dw_scatter_add(const float* dW, int32_t V, int32_t d, const spo_dw_shards& sh, cudaStream_t st) {
+  ShardTable tb{};
+  tb.n = sh.n_shards;
+  tb.rows = sh.rows_per_shard;
+  for (int k = 0; k < sh.n_shards; ++k) tb.shard[k] = sh.shard[k];
+  const int64_t n_vec = (int64_t)V * d / 4;
+  int64_t blocks = ceil_div(n_vec, 256 * 4);
+  const int64_t cap = (int64_t)sm_count() * 16;
+  if (blocks > cap) blocks = cap;
+  if (blocks < 1) blocks = 1;
+  dw_scatter_add_kernel<<<(unsigned)blocks, 256, 0, st>>>(reinterpret_cast<const float4*>(dW), n_vec, d / 4, tb);
   return cudaGetLastError();
 }
 

@@ -74,6 +74,7 @@ constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kRefMargin = 40.0f;     // binary orders between a row's reference exponent and its first tile's maximum
 
 enum : int { MODE_FWD = 0, MODE_G = 1, MODE_DH = 2, MODE_DW = 3, MODE_E = 4 };
+constexpr int kMaxDwShards = SPO_MAX_DW_SHARDS;
 
 struct GemmParams {
   int m_tiles, n_tiles, nsplit, per_split;   // work decomposition: unit = (row tile, split of the column tiles)
@@ -97,6 +98,11 @@ struct GemmParams {
   int64_t pre_ld;
   const float* rowscale;                     // DH (one-pass): factor of each output row, indexed like the output; NULL = none
   int m_tile0;                               // added to every unit's row tile (a launch that covers a slab of row tiles)
+  // DW, reduce-scatter form: instead of going to `out`, every tile (plus what `out` holds, when accumulating)
+  // is ADDED into the shard that owns its vocabulary rows; shard k = rows [k shard_rows, (k+1) shard_rows)
+  float* shard[kMaxDwShards];
+  int n_shards;                              // 0: plain output
+  int64_t shard_rows;
   // DH / DW
   void* out;
   int out_bf16;
@@ -726,7 +732,22 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
               const uint4 raw4 = stage_get(stage, lane, i, r, cc);
               if (grow_warp0 + r < p.rows_valid) {
                 float* dst = obase + (int64_t)r * p.ldo + col0 + cc * 4;
-                if (p.accumulate) {
+                if (MODE == MODE_DW && p.n_shards > 0) {
+                  // reduce-scatter form: this tile, plus the sum of the earlier chunks' tiles held in `out`,
+                  // goes to the owner of the vocabulary row (its memory may be another GPU's: a plain
+                  // peer store-reduction over NVLink, no load from there and nothing to wait for)
+                  float4 val = make_float4(__uint_as_float(raw4.x), __uint_as_float(raw4.y), __uint_as_float(raw4.z),
+                                           __uint_as_float(raw4.w));
+                  if (p.accumulate) {
+                    const float4 old = *reinterpret_cast<const float4*>(dst);
+                    val.x += old.x; val.y += old.y; val.z += old.z; val.w += old.w;
+                  }
+                  const int64_t vrow = grow_warp0 + r;
+                  const int owner = (int)(vrow / p.shard_rows);
+                  float* sdst = p.shard[owner] + (vrow - (int64_t)owner * p.shard_rows) * p.ldo + col0 + cc * 4;
+                  asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};"
+                               ::"l"(sdst), "f"(val.x), "f"(val.y), "f"(val.z), "f"(val.w) : "memory");
+                } else if (p.accumulate) {
                   // Added in L2, nothing comes back: no load latency in this (un-overlapped) epilogue.
                   // Each element receives exactly one addend per launch and launches are ordered on
                   // the stream, so the summation order is fixed.
@@ -1014,7 +1035,7 @@ cudaError_t launch_dh(const CUtensorMap& mG_k, const CUtensorMap& mW_mn, int64_t
 // the slab of 256-row vocabulary tiles this launch covers (the whole vocabulary: 0, all of them).
 cudaError_t launch_dw(const CUtensorMap& mG_mn, const CUtensorMap& mH_mn, int64_t h_row0, int64_t rows, int32_t d,
                       int32_t V, float* dW, int dw_accumulate, int tile0, int tiles, uint32_t* progress,
-                      int32_t* d_status, cudaStream_t st) {
+                      int32_t* d_status, cudaStream_t st, const spo_dw_shards* shards = nullptr) {
   const int n_tiles_d = (int)ceil_div(d, BN);
   GemmParams p{};
   p.m_tiles = tiles;
@@ -1028,6 +1049,11 @@ cudaError_t launch_dw(const CUtensorMap& mG_mn, const CUtensorMap& mH_mn, int64_
   p.cols_valid = d;
   p.out_row0 = 0;
   p.out = dW; p.out_bf16 = 0; p.ldo = d; p.accumulate = dw_accumulate;
+  if (shards) {
+    p.n_shards = shards->n_shards;
+    p.shard_rows = shards->rows_per_shard;
+    for (int k = 0; k < shards->n_shards; ++k) p.shard[k] = shards->shard[k];
+  }
   p.d_status = d_status;
   return launch_gemm<MODE_DW>(mG_mn, mH_mn, p, progress, st);
 }
@@ -1183,6 +1209,7 @@ cudaError_t launch_fused_bf16(const FusedArgs& a, char* ws, const FusedWs& L, cu
                             a.d_status, st);
     if (e != cudaSuccess) return e;
     if (!a.accumulate && (e = cudaMemsetAsync(a.dW, 0, sizeof(float) * (size_t)V * d, st)) != cudaSuccess) return e;
+    if (a.shards && a.accumulate && (e = launch_dw_scatter_add(a.dW, V, d, *a.shards, st)) != cudaSuccess) return e;
     if (a.n_slabs > 0 && a.events) {              // nothing to contract: every slab is final at once
       int n = 1;
       slab_tiles(V, d, a.n_slabs, &n);
@@ -1297,7 +1324,9 @@ cudaError_t launch_fused_bf16(const FusedArgs& a, char* ws, const FusedWs& L, cu
         if ((e = cudaEventRecord(a.events[k], st)) != cudaSuccess) return e;
       }
     } else {
-      e = launch_dw(mG_mn, mHs_mn, 0, group_rows, d, V, a.dW, dw_acc, 0, tiles, progress, a.d_status, st);
+      // reduce-scatter form: the call's last contraction sends the finished tiles to their owners
+      const spo_dw_shards* sh = (a.shards && c0 + L.slots >= n_chunks) ? a.shards : nullptr;
+      e = launch_dw(mG_mn, mHs_mn, 0, group_rows, d, V, a.dW, dw_acc, 0, tiles, progress, a.d_status, st, sh);
       if (e != cudaSuccess) return e;
     }
   }

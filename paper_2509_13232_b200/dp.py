@@ -133,3 +133,36 @@ class SlabAllReduce:
     def finish(self):
         import torch
         torch.cuda.current_stream().wait_event(self.done)
+
+
+class PeerShards:
+    """Vocabulary-row shards of dW, one per rank, that every rank can write: the target of
+    spo_loss_fwd_bwd_scatter.  Each rank owns an fp32 [rows_per_shard][d] buffer in memory that is mapped
+    into all ranks of the group (torch's symmetric memory); `table` is the shard table for the call.
+
+        shards.begin_step()      # zero this rank's shard; all ranks' zeroing is visible before anyone adds
+        binding.spo_loss_fwd_bwd_scatter(..., shards.table)
+        shards.end_step()        # every rank's additions have landed: shards.local holds this rank's rows of dW
+
+    The exchange itself is the library's: store-reductions into the owners' memory from the epilogue of the
+    last dW contraction (over NVLink for a peer's shard).  Not run on more than one GPU so far.
+    """
+
+    def __init__(self, V, d, device, group=None):
+        import torch
+        import torch.distributed as dist
+        import torch.distributed._symmetric_memory as symm_mem
+        from . import binding
+        group = group if group is not None else dist.group.WORLD
+        world = dist.get_world_size(group)
+        self.rows_per_shard = -(-int(V) // world)
+        self.local = symm_mem.empty((self.rows_per_shard, int(d)), dtype=torch.float32, device=device)
+        self.handle = symm_mem.rendezvous(self.local, group)
+        self.table = binding.dw_shards([int(p) for p in self.handle.buffer_ptrs], self.rows_per_shard)
+
+    def begin_step(self):
+        self.local.zero_()
+        self.handle.barrier()
+
+    def end_step(self):
+        self.handle.barrier()

@@ -109,6 +109,19 @@ def test_new_entry_points_reject_bad_arguments_on_the_host(lib):
     assert lib.spo_loss_fwd_bwd_slabs(*loss_args, 4, None) == B.ERR_INVALID_ARG
     none_first = (ctypes.c_void_p * 4)(None, fake, fake, fake)
     assert lib.spo_loss_fwd_bwd_slabs(*loss_args, 4, none_first) == B.ERR_INVALID_ARG
+    # reduce-scatter variant: the shard table is checked first
+    assert lib.spo_loss_fwd_bwd_scatter(*loss_args, None) == B.ERR_INVALID_ARG
+    sh = B.SpoDwShards()
+    sh.n_shards, sh.rows_per_shard = 2, 10                       # 20 rows < V = 100
+    sh.shard[0], sh.shard[1] = 0x1000, 0x2000
+    assert lib.spo_loss_fwd_bwd_scatter(*loss_args, ctypes.byref(sh)) == B.ERR_INVALID_ARG
+    sh.rows_per_shard = 50
+    sh.shard[1] = None
+    assert lib.spo_loss_fwd_bwd_scatter(*loss_args, ctypes.byref(sh)) == B.ERR_INVALID_ARG
+    sh.shard[1] = 0x2004
+    assert lib.spo_loss_fwd_bwd_scatter(*loss_args, ctypes.byref(sh)) == B.ERR_BAD_ALIGNMENT
+    sh.n_shards = 17
+    assert lib.spo_loss_fwd_bwd_scatter(*loss_args, ctypes.byref(sh)) == B.ERR_INVALID_ARG
     # parameters outside their domain
     for bad in (dict(dual_clip=1.0), dict(dual_clip=-2.0), dict(near_zero_tau_lo=-1.0), dict(surrogate=7)):
         q = B.default_params(**bad)

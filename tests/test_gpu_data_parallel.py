@@ -12,6 +12,12 @@ from tests.helpers import dev, rel_fro, run_loss, status_word, ws_bytes
 pytestmark = pytest.mark.gpu
 
 
+def _clip_batch_dp(cfg, lengths, d, v, bf16):
+    rng = np.random.default_rng(cfg)
+    a = rng.standard_normal(len(lengths)).astype(np.float32)
+    return inputs.loss_batch(cfg, lengths, d, v, 0.05, bf16, 0.3, target="softmax", mask_p=0.1, a_norm=a)
+
+
 def _slice_batch(lb, s0, s1):
     t0, t1 = int(lb.cu_seqlens[s0]), int(lb.cu_seqlens[s1])
     return inputs.LossBatch(h=lb.h[t0:t1], w=lb.w, y=lb.y[t0:t1], logp_old=lb.logp_old[t0:t1], mask=lb.mask[t0:t1],
@@ -190,3 +196,63 @@ def test_data_parallel_step_with_one_rank_equals_the_plain_step():
             assert torch.equal(a, b)
     finally:
         dist.destroy_process_group()
+
+
+def _scatter_call(lb, params, shards, dw_init=None):
+    """One spo_loss_fwd_bwd_scatter call; returns (loss, dH, dW scratch, status)."""
+    import torch
+    from paper_2509_13232_b200 import binding as B
+    tdt = torch.bfloat16 if lb.bf16 else torch.float32
+    H, W = dev(lb.h, tdt), dev(lb.w, tdt)
+    T, d = H.shape
+    V, S = W.shape[0], len(lb.cu_seqlens) - 1
+    f32 = dict(dtype=torch.float32, device="cuda")
+    loss = torch.zeros(4, **f32)
+    logp, lse, coef = (torch.zeros(max(T, 1), **f32) for _ in range(3))
+    dH = torch.zeros((max(T, 1), d), dtype=tdt, device="cuda")
+    dW = torch.full((V, d), float("nan"), **f32) if dw_init is None else dev(dw_init).clone()
+    st = status_word()
+    B.spo_loss_fwd_bwd_scatter(H, W, dev(lb.y), dev(lb.logp_old), dev(lb.mask), dev(lb.cu_seqlens), dev(lb.a_norm), 1.0,
+                               loss, logp, lse, coef, None, dH[:T], dW, 0 if dw_init is None else 1,
+                               ws_bytes(B.WS_LOSS_FWD_BWD, T=T, d=d, V=V, B=S), params, st, shards)
+    return loss, dH, dW, st
+
+
+@pytest.mark.parametrize("case", ["one_chunk", "three_chunks", "fp32", "gspo"])
+def test_reduce_scatter_form_two_emulated_ranks_fill_the_owners_shards(case):
+    """spo_loss_fwd_bwd_scatter: two ranks, one after the other on this GPU, each with its part of the
+    mini-batch and the whole batch's denominators, add their dW into three shards (local buffers standing
+    in for the owners' memory; the last shard is ragged).  Together the shards must hold the dW that one
+    plain call on the whole mini-batch gives; loss and dH are untouched by the variant."""
+    import torch
+    from paper_2509_13232_b200 import binding as B
+    bf16 = case != "fp32"
+    if case == "three_chunks":
+        lengths, d, v = [5000, 4400, 9000, 1600], 128, 3000
+    elif case == "fp32":
+        lengths, d, v = [30, 4, 51, 9], 32, 257
+    else:
+        lengths, d, v = [700, 40, 520, 75], 128, 3000
+    lb = _clip_batch_dp(160, lengths, d, v, bf16)
+    sur = B.SUR_GSPO if case == "gspo" else B.SUR_PPO_CLIP
+    n_tok = int(lb.mask.sum())
+    n_resp = sum(1 for a, b in zip(lb.cu_seqlens[:-1], lb.cu_seqlens[1:]) if lb.mask[int(a):int(b)].any())
+    whole = run_loss(lb, params=B.default_params(surrogate=sur), one_pass=True)
+    rows_per = -(-v // 3) + 5                                   # 3 shards, the last one shorter
+    bufs = [torch.zeros((rows_per, d), dtype=torch.float32, device="cuda") for _ in range(3)]
+    shards = B.dw_shards(bufs, rows_per)
+    pg = B.default_params(surrogate=sur, global_tokens=n_tok, global_responses=n_resp)
+    loss_sum, dhs = 0.0, []
+    for s0, s1 in ((0, 2), (2, len(lengths))):
+        part = _slice_batch(lb, s0, s1)
+        loss, dH, _, st = _scatter_call(part, pg, shards)
+        torch.cuda.synchronize()
+        assert int(st[0].item()) == 0
+        loss_sum += float(loss[0].item())
+        dhs.append(dH[:part.h.shape[0]].float().cpu().numpy())
+    got_dw = torch.cat(bufs, 0)[:v].cpu().numpy()
+    assert float(torch.cat(bufs, 0)[v:].abs().max().item()) == 0.0      # rows past the vocabulary stay untouched
+    tol = 2e-3 if bf16 else 1e-5
+    assert rel_fro(got_dw, whole["dW"]) <= tol
+    assert abs(loss_sum - whole["loss"]) <= (2e-3 if bf16 else 1e-5)
+    assert rel_fro(np.concatenate(dhs, 0), whole["dH"]) <= tol
