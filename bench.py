@@ -107,9 +107,12 @@ class Step:
     """Device buffers of one workload and the call sequence of one step."""
 
     def __init__(self, workload, device, rank, responses=None, custom=None, mask_frac=0.0, path="onepass",
-                 entropy=False, dp_world=None, dw_slabs=8, surrogate="ppo_clip", dual_clip=0.0):
+                 entropy=False, dp_world=None, dw_slabs=8, surrogate="ppo_clip", dual_clip=0.0, dw_reduce="allreduce"):
         """dp_world = N: this rank holds its share of ONE mini-batch split over N ranks by token count
-        (W and the tracker table replicated); None: the rank has a mini-batch of its own."""
+        (W and the tracker table replicated); None: the rank has a mini-batch of its own.
+        dw_reduce: "allreduce" sums dW over the ranks slab by slab behind the last contraction (every rank
+        ends with the whole dW); "scatter" has that contraction add its tiles into the vocabulary shard of
+        the owning rank's memory (every rank ends with its rows of dW in self.shards.local)."""
         import torch
         from paper_2509_13232_b200 import binding as B
         from paper_2509_13232_b200 import dp, inputs
@@ -170,7 +173,8 @@ class Step:
             self.a_norm = torch.empty(self.S, **f32)
             self.params.global_tokens = self.n_tok_all        # denominators of the whole mini-batch (mask is all ones)
             self.params.global_responses = self.S_all
-            self.reducer = dp.SlabAllReduce(B.spo_dw_slab_rows(V, d, dw_slabs), device)
+            self.shards = dp.PeerShards(V, d, device) if dw_reduce == "scatter" else None
+            self.reducer = None if self.shards else dp.SlabAllReduce(B.spo_dw_slab_rows(V, d, dw_slabs), device)
         self.stats = torch.empty(8, **f32)
         self.loss = torch.zeros(4, **f32)
         self.logp, self.lse, self.coef = (torch.empty(self.T, **f32) for _ in range(3))
@@ -281,6 +285,12 @@ class Step:
             # the ranks' dW and loss add up to the mini-batch's; dW is summed slab by slab on a second
             # stream while its last contraction still runs
             import torch.distributed as dist
+            if self.shards:
+                self.shards.begin_step()
+                self.B.spo_loss_fwd_bwd_scatter(*args, self.shards.table, entropy=self.entropy)
+                dist.all_reduce(self.loss)
+                self.shards.end_step()
+                return
             self.B.spo_loss_fwd_bwd_slabs(*args, self.reducer.events, entropy=self.entropy)
             self.reducer.reduce(self.dW)
             dist.all_reduce(self.loss)
@@ -329,7 +339,7 @@ def run_ours(args, rank, world, local_rank):
         raise SystemExit("--parallelism dp runs the one-pass loss on the unmasked named workloads")
     step = Step(args.workload, device, rank, args.responses, args.custom, args.mask_frac, args.path, args.entropy,
                 dp_world=world if dp_mode else None, dw_slabs=args.dw_slabs, surrogate=args.surrogate,
-                dual_clip=args.dual_clip)
+                dual_clip=args.dual_clip, dw_reduce=args.dw_reduce)
     if args.surrogate == "gspo" and step.onepass:
         # a response's ratio needs all its tokens: spo_loss_fwd_bwd runs forward-then-backward for it
         step.flops_bwd = 6.0 * step.T * step.d * step.V
@@ -432,7 +442,8 @@ def run_ours(args, rank, world, local_rank):
                    "tracker_prompts": step.table_n, "l2": "inputs_exceed_l2", "loss_path": "onepass" if step.onepass else "split", "entropy_output": bool(args.entropy),
                    "surrogate": args.surrogate, "dual_clip": args.dual_clip,
                    "bwd_chunks": step.bwd_chunks, "mask_frac": step.mask_frac,
-                   "parallelism": "dp%d" % world if dp_mode else ("replicas%d" % world if world > 1 else "single")},
+                   "parallelism": "dp%d" % world if dp_mode else ("replicas%d" % world if world > 1 else "single"),
+                   "dw_reduce": args.dw_reduce if dp_mode else None},
         "gpu_launches": step.launches * args.steps,
         "device_status": status,
         "wall_s": wall,
@@ -755,6 +766,10 @@ def main():
                          "collective), or ONE mini-batch split over the ranks by token count with dW summed over the "
                          "ranks, overlapped slab by slab with its last contraction (strong scaling)")
     ap.add_argument("--dw-slabs", type=int, default=8, help="slabs the last dW contraction is cut into (dp)")
+    ap.add_argument("--dw-reduce", choices=["allreduce", "scatter"], default="allreduce",
+                    help="dp: sum dW over the ranks with all-reduces per slab behind the last contraction (default), "
+                         "or have that contraction add its tiles into per-rank vocabulary shards in peer-mapped "
+                         "memory (spo_loss_fwd_bwd_scatter; every rank ends with its rows of dW)")
     ap.add_argument("--rehearse-host", action="store_true",
                     help="no GPU work: start the ranks (gloo), plan the data-parallel split and the dW slabs, run the "
                          "host-side exchanges on dummy values and print the plan (used by the CPU tests)")

@@ -7,7 +7,7 @@ import pytest
 
 from oracle import spo_oracle as O
 from paper_2509_13232_b200 import dp, inputs
-from tests.helpers import dev, rel_fro, run_loss, status_word, ws_bytes
+from tests.helpers import dev, oracle_loss, rel_fro, run_loss, status_word, worst_row_tile_error, ws_bytes
 
 pytestmark = pytest.mark.gpu
 
@@ -194,6 +194,18 @@ def test_data_parallel_step_with_one_rank_equals_the_plain_step():
         assert int(part.status[0].item()) == 0
         for a, b in zip(keep, (part.loss, part.logp, part.coef, part.dH, part.dW, part.ids, part.ab, part.a_norm)):
             assert torch.equal(a, b)
+        del part
+        torch.cuda.empty_cache()
+        # the same step with dW scattered into per-rank shards (one shard here): the sums are formed by
+        # store-reductions on top of a zeroed shard, so dW agrees to rounding instead of bit for bit
+        scat = bench.Step("cfg3_small_bf16", dev0, 0, dp_world=1, dw_reduce="scatter")
+        scat.run()
+        torch.cuda.synchronize()
+        assert int(scat.status[0].item()) == 0
+        for a, b in zip(keep[:4] + keep[5:], (scat.loss, scat.logp, scat.coef, scat.dH, scat.ids, scat.ab, scat.a_norm)):
+            assert torch.equal(a, b)
+        assert scat.shards.local.shape == keep[4].shape
+        assert rel_fro(scat.shards.local.cpu().numpy(), keep[4].cpu().numpy()) <= 1e-6
     finally:
         dist.destroy_process_group()
 
@@ -256,3 +268,39 @@ def test_reduce_scatter_form_two_emulated_ranks_fill_the_owners_shards(case):
     assert rel_fro(got_dw, whole["dW"]) <= tol
     assert abs(loss_sum - whole["loss"]) <= (2e-3 if bf16 else 1e-5)
     assert rel_fro(np.concatenate(dhs, 0), whole["dH"]) <= tol
+    want = oracle_loss(lb, params=B.default_params(surrogate=sur))     # and the float64 definition of the whole batch
+    assert rel_fro(got_dw, want["dW"]) <= (1e-2 if bf16 else 1e-4)
+    assert worst_row_tile_error(got_dw, want["dW"])[0] <= (2e-2 if bf16 else 1e-4)
+    assert abs(loss_sum - want["loss"]) <= (2e-3 if bf16 else 1e-5)
+
+
+def test_peer_shards_on_a_one_rank_group_hold_the_plain_dw():
+    """dp.PeerShards (shards in memory mapped into every rank of the group) with a group of one rank: the
+    table has one shard, this rank's, and after begin_step / the scatter call / end_step it holds the dW
+    of the plain call.  (Shards in a peer's memory need a second GPU.)"""
+    import os
+    import socket
+    import torch
+    import torch.distributed as dist
+    from paper_2509_13232_b200 import binding as B
+    dev0 = torch.device("cuda", 0)
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    os.environ["MASTER_ADDR"], os.environ["MASTER_PORT"] = "127.0.0.1", str(port)
+    dist.init_process_group("nccl", rank=0, world_size=1, device_id=dev0)
+    try:
+        d, v = 128, 3000
+        lb = _clip_batch_dp(161, [700, 40, 520, 75], d, v, True)
+        whole = run_loss(lb, params=B.default_params(), one_pass=True)
+        shards = dp.PeerShards(v, d, dev0)
+        assert shards.rows_per_shard == v and shards.table.n_shards == 1
+        for _ in range(2):                                     # a second step starts from a zeroed shard again
+            shards.begin_step()
+            _, _, _, st = _scatter_call(lb, B.default_params(), shards.table)
+            shards.end_step()
+            torch.cuda.synchronize()
+            assert int(st[0].item()) == 0
+            assert rel_fro(shards.local.cpu().numpy(), whole["dW"]) <= 2e-3
+    finally:
+        dist.destroy_process_group()
