@@ -38,7 +38,8 @@ TABLE_N = 1_000_000          # tracker table the step samples from and updates
 # DRAM read+write bytes (dram__bytes_read.sum + dram__bytes_write.sum) of all launches of one cfg4 step:
 # one chunk's launches captured with ncu on a slice of the workload, times the chunks of a step.
 # None = the kernels of that path changed after the counters were taken.
-CFG4_STEP_DRAM_BYTES = {"split": 1.23e12, "onepass": 1.02e12}
+CFG4_STEP_DRAM_BYTES = {"split": None, "onepass": None}
+DW_CHUNK_GROUP = 2           # chunks of token rows whose dW contraction shares one launch (the library's constant)
 
 LOSS_SHAPES = {
     # workload: (d, V, w_std, old-logprob noise, reward probability)
@@ -206,18 +207,18 @@ class Step:
         # kernels launched by one step: sampling 4 (tile sums, their prefix, search, accept; 3 for tables above
         # 2^20 prompts), advantages + update 1, then
         # split path: forward 3 (count, contraction, finalise), backward 3 per chunk;
-        # one-pass path: count 1, first-tile pass 1, per chunk 5 (logits contraction, finalise, row scaling
-        # of H, dH, dW).  Memsets are not counted.
+        # one-pass path: count 1, first-tile pass 1, per chunk 4 (logits contraction, finalise, row scaling
+        # of H, dH) and one dW contraction per DW_CHUNK_GROUP chunks.  Memsets are not counted.
         self.flops_fwd = 2.0 * self.T * d * V
         n_samp = 4 if self.table_n <= (1 << 20) else 3
         chunks_act = -(-self.n_tok // chunk_rows)          # chunks of the compacted batch (masked workloads)
         if self.onepass and self.mask_frac > 0.0:
             # row list 3, gather 1, boundaries 1, one-pass on the compacted batch, two scatters
-            self.launches = n_samp + 1 + 3 + 1 + 1 + (2 + 5 * chunks_act) + 2
+            self.launches = n_samp + 1 + 3 + 1 + 1 + (2 + 4 * chunks_act + -(-chunks_act // DW_CHUNK_GROUP)) + 2
             self.flops_fwd = 2.0 * self.n_tok * d * V
             self.flops_bwd = 4.0 * self.n_tok * d * V
         elif self.onepass:
-            self.launches = n_samp + 1 + 2 + 5 * self.bwd_chunks
+            self.launches = n_samp + 1 + 2 + 4 * self.bwd_chunks + -(-self.bwd_chunks // DW_CHUNK_GROUP)
             self.flops_bwd = 4.0 * self.T * d * V
         elif self.mask_frac > 0.0:
             # forward over all rows; row list 3, gather 1, backward on the rows with gradient, scatter 1

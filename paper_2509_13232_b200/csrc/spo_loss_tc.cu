@@ -62,13 +62,17 @@ constexpr int BSUB_ROWS = HALF_N / CG;               // B columns per CTA per ha
 constexpr int BSUB_BYTES = BSUB_ROWS * BK * 2;       // 16 KB
 constexpr int STAGE_BYTES = A_BYTES + 2 * BSUB_BYTES;  // 48 KB
 constexpr int EPI_WARPS = 8;
-constexpr int NUM_THREADS = 32 * (2 + EPI_WARPS);
+constexpr int PACER_WARP = 2 + EPI_WARPS;              // last warp: keeps the pairs' loads close together in time
+constexpr int NUM_THREADS = 32 * (3 + EPI_WARPS);
 constexpr int TMEM_COLS = 512;
 constexpr int STAGING_BYTES = 4096;                    // per epilogue warp: 32 rows x 128 bytes, for coalesced stores
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256 + EPI_WARPS * STAGING_BYTES;
 constexpr unsigned long long kWaitLimitNs = 4000000000ull;
 constexpr int kEpilogueSleepNs = 64;
 constexpr int kProducerSleepNs = 32;
+constexpr int kPacerSleepNs = 256;                     // between two looks at the other pairs' progress
+constexpr uint32_t kPacerMaxSpins = 1u << 24;          // the pacer gives up (and lets everyone run free) after this many looks
+constexpr int kHoldTries = 2048;                       // x 64 ns: longest time a producer holds back for the slowest pair
 
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kRefMargin = 40.0f;     // binary orders between a row's reference exponent and its first tile's maximum
@@ -109,10 +113,10 @@ struct GemmParams {
   int64_t ldo;
   int accumulate;
   int32_t* d_status;
-  // Soft lock-step between CTA pairs (FWD / G): progress[g] = tiles started by pair g (+1), ~0u when done.
+  // Soft lock-step between CTA pairs: progress[g] = k-blocks whose loads pair g has issued, ~0u when done;
+  // a pair holds its loads back while it is more than `window` k-blocks ahead of the slowest pair.
   uint32_t* progress;
   int window;
-  int sync_kblocks;                          // k-blocks between two progress comparisons
 };
 
 // ---------------------------------------------------------------------------
@@ -196,17 +200,6 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar)
       : "memory");
 }
-
-#ifdef SPO_TUNE_EHINT
-// Same load with an L2 eviction-priority policy (tuning builds only).
-__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar,
-                                                 uint64_t policy) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
-      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar), "l"(policy)
-      : "memory");
-}
-#endif
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -386,6 +379,8 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   const uint32_t full0 = bars, empty0 = bars + 8 * STAGES, tfull = bars + 16 * STAGES, tempty = tfull + 8;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen + STAGES * STAGE_BYTES + 16 * STAGES + 16);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + STAGES * STAGE_BYTES + 16 * STAGES + 24);
+  volatile uint32_t* pace_mine = reinterpret_cast<volatile uint32_t*>(gen + STAGES * STAGE_BYTES + 16 * STAGES + 32);
+  volatile uint32_t* pace_limit = pace_mine + 1;   // k-blocks this pair's producer may have issued (pacer -> producer)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();                    // 0 = leader of the pair
@@ -397,6 +392,8 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     mbar_init(tfull, 1);
     mbar_init(tempty, EPI_WARPS * CG);
     *abort_flag = 0;
+    *pace_mine = 0;
+    *pace_limit = p.progress ? (uint32_t)p.window : 0xFFFFFFFFu;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 0) {
@@ -411,37 +408,27 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
-    // Lane 0 issues the loads.  Every `sync_kblocks` k-blocks (once per tile) the whole warp compares
-    // this pair's step count with the other pairs' and holds back while it is more than `window`
-    // steps ahead of the slowest: pairs that sweep the same operand tiles then stay close enough in
-    // time for those tiles to be served from L2 instead of being streamed from HBM once per pair
-    // (without it the forward at 244k tokens read 0.8 TB from HBM per launch, with it 0.12 TB).
-    // The hold is bounded and advisory (after ~0.15 ms the pair goes on regardless), so it cannot
-    // dead-lock, and finished pairs publish ~0u so that they never hold anyone back.
-    uint32_t it = 0, tseq = 0;
+    // Lane 0 issues the loads.  Before each k-block it tells the pacer warp how far it is and holds
+    // back while it is ahead of what the pacer allows (the slowest pair's count plus `window`
+    // k-blocks): pairs that sweep the same operand tiles then stay close enough in time for those
+    // tiles to be served from L2 instead of being streamed from HBM once per pair (without any pacing
+    // the forward at 244k tokens read 0.8 TB from HBM per launch, with it 0.12 TB; dH at one look per
+    // tile read 17 GB per chunk, at a window of 32 k-blocks 8 GB).  Both words are in shared memory,
+    // so the loop pays two shared-memory accesses per k-block; the looks at the other pairs are the
+    // pacer's.  The hold is bounded and advisory (after ~0.13 ms the pair goes on regardless), so
+    // it cannot dead-lock, and finished pairs publish ~0u so that they never hold anyone back.
+    uint32_t it = 0;
     int ok = 1;
-    volatile uint32_t* progress = (rank == 0) ? p.progress : nullptr;
-    const uint32_t sync_kb = (uint32_t)p.sync_kblocks;
+    const bool paced = (rank == 0) && p.progress != nullptr;
     for (int u = group; u < total_units; u += n_groups) {
       const Unit un = unit_of(u, p);
       const int row_base = un.m_tile * GROUP_M + (int)rank * BM;       // this CTA's rows of the tile
       for (int n = un.n_begin; n < un.n_end; ++n) {
         const int col_base = n * BN + (int)rank * BSUB_ROWS;           // this CTA's columns of half 0
         for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
-          if (progress && (it % sync_kb) == 0) {                       // whole warp: publish and compare progress
-            ++tseq;
-            if (lane == 0) progress[group] = tseq;
-            if ((int)tseq > p.window) {
-              for (int tries = 0; tries < 128; ++tries) {
-                uint32_t mn = 0xFFFFFFFFu;
-                for (int g = lane; g < n_groups; g += 32) mn = min(mn, progress[g]);
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) mn = min(mn, __shfl_xor_sync(0xffffffffu, mn, o));
-                if (mn + (uint32_t)p.window >= tseq) break;
-                __nanosleep(128);
-              }
-            }
-            ok = __shfl_sync(0xffffffffu, ok, 0);
+          if (paced && lane == 0 && ok) {
+            *pace_mine = it;
+            for (int tries = 0; tries < kHoldTries && it > *pace_limit; ++tries) __nanosleep(64);
           }
           if (lane == 0 && ok) {
             const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
@@ -452,13 +439,6 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
               if (rank == 0) mbar_expect_tx(full0 + 8 * s, CG * STAGE_BYTES);   // both CTAs' bytes land on the leader's barrier
               const uint32_t fb = map_to_cta(full0 + 8 * s, 0);
               if (!A_MN) {
-#ifdef SPO_TUNE_EHINT
-                if (MODE == MODE_E) {
-                  uint64_t pol;
-                  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
-                  tma_load_2d_hint(sa, &tmA, kb * BK, p.a_row0 + row_base, fb, pol);
-                } else
-#endif
                 tma_load_2d(sa, &tmA, kb * BK, p.a_row0 + row_base, fb);
               } else {
 #pragma unroll
@@ -483,7 +463,7 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       }
     }
     __syncwarp();
-    if (progress && lane == 0) progress[group] = 0xFFFFFFFFu;          // done: never hold anyone back
+    if (paced && lane == 0) *pace_mine = 0xFFFFFFFFu;                  // done: the pacer publishes it and stops
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer (leader CTA)
     if (lane == 0 && rank == 0) {
@@ -666,8 +646,11 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             for (int i = 0; i < 8; ++i) {
               int r, cc;
               const uint4 val = stage_get(stage, lane, i, r, cc);
-              if (grow_warp0 + r < p.rows_valid)
-                *reinterpret_cast<uint4*>(obase + (int64_t)r * p.ldg + col0 + cc * 8) = val;
+              if (grow_warp0 + r < p.rows_valid) {
+                // streaming store: the chunk buffer is next read by another launch, and lines that stayed in
+                // L2 would push out the row strips of H that every tile of this sweep re-reads
+                __stcs(reinterpret_cast<uint4*>(obase + (int64_t)r * p.ldg + col0 + cc * 8), val);
+              }
             }
           }
         } else if (MODE == MODE_G || (MODE == MODE_DH && p.out_bf16)) {
@@ -774,6 +757,29 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     }
   }
 
+  else if (warp == PACER_WARP && rank == 0 && p.progress != nullptr) {
+    // ------------------------------------------------------------------ pacer (leader CTA)
+    // Publishes this pair's k-block count, reads every pair's, and hands the producer its limit.  A
+    // few loads and one sleep per turn; it ends when the producer has, or after kPacerMaxSpins turns
+    // (then with the limit lifted, so that nobody waits for a pacer that has gone).
+    volatile uint32_t* progress = p.progress;
+    for (uint32_t spins = 0;; ++spins) {
+      const uint32_t mine = *pace_mine;
+      if (lane == 0) progress[group] = mine;
+      if (mine == 0xFFFFFFFFu) break;
+      if (spins >= kPacerMaxSpins) {
+        if (lane == 0) { *pace_limit = 0xFFFFFFFFu; progress[group] = 0xFFFFFFFFu; }
+        break;
+      }
+      uint32_t mn = 0xFFFFFFFFu;
+      for (int g = lane; g < n_groups; g += 32) mn = min(mn, progress[g]);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) mn = min(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+      if (lane == 0) *pace_limit = (mn > 0xFFFFFFFFu - (uint32_t)p.window) ? 0xFFFFFFFFu : mn + (uint32_t)p.window;
+      __nanosleep(kPacerSleepNs);
+    }
+  }
+
   // ------------------------------------------------------------------ teardown
   __syncwarp();
   if (*abort_flag) {                       // let copies still in flight land before the CTA retires
@@ -836,11 +842,15 @@ bool make_map(CUtensorMap* m, const void* ptr, uint64_t inner, uint64_t outer, u
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// How many tiles a CTA pair may run ahead of the slowest pair before it holds back.
-#ifndef SPO_TUNE_WINDOW
-#define SPO_TUNE_WINDOW 1
+// How many k-blocks a CTA pair may run ahead of the slowest pair before it holds back.
+#ifndef SPO_TUNE_WINDOW_SWEEP
+#define SPO_TUNE_WINDOW_SWEEP 32
 #endif
-constexpr int kLockStepWindow = SPO_TUNE_WINDOW;
+#ifndef SPO_TUNE_WINDOW_STREAM
+#define SPO_TUNE_WINDOW_STREAM 16
+#endif
+constexpr int kWindowSweep = SPO_TUNE_WINDOW_SWEEP;
+constexpr int kWindowStream = SPO_TUNE_WINDOW_STREAM;
 
 // CTA pairs that can be resident at once (one CTA per SM).
 int group_count() { return sm_count() / CG; }
@@ -889,14 +899,9 @@ cudaError_t launch_gemm(const CUtensorMap& a, const CUtensorMap& b, const GemmPa
   const int units = p_in.m_tiles * p_in.nsplit;
   if (units <= 0) return cudaSuccess;
   GemmParams p = p_in;
-  p.window = kLockStepWindow;
-  // The pairs compare progress once per tile.  Comparing every 64 or 128 k-blocks inside the long
-  // tiles of DH / DW was measured too (SPO_TUNE_SYNCKB): same step time, and on one and the same GPU the
-  // same DRAM traffic (DH 14.2 against 14.7 GB per chunk, DW rather more than less).
-  p.sync_kblocks = p.k_blocks;
-#ifdef SPO_TUNE_SYNCKB
-  if (MODE == MODE_DH || MODE == MODE_DW) p.sync_kblocks = p.k_blocks < SPO_TUNE_SYNCKB ? p.k_blocks : SPO_TUNE_SYNCKB;
-#endif
+  // k-blocks a pair may run ahead of the slowest one.  E / FWD / G sweep short tiles (d / 64 k-blocks) and
+  // re-read their row strip per tile; dH / dW stream both operands through one long tile.
+  p.window = (MODE == MODE_DH || MODE == MODE_DW) ? kWindowStream : kWindowSweep;
   p.progress = nullptr;
   if (p.window > 0 && progress) {
     cudaError_t e = cudaMemsetAsync(progress, 0, kProgressBytes, st);
@@ -1126,7 +1131,7 @@ cudaError_t launch_bwd_bf16(const void* H, const void* W, const int32_t* y, cons
 // [V x d] fp32 matrix (and its accumulator drains) by that number.
 // ---------------------------------------------------------------------------
 #ifndef SPO_DW_CHUNK_GROUP
-#define SPO_DW_CHUNK_GROUP 1
+#define SPO_DW_CHUNK_GROUP 2
 #endif
 constexpr int kDwChunkGroup = SPO_DW_CHUNK_GROUP;
 
