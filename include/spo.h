@@ -354,8 +354,8 @@ int32_t spo_loss_bwd(const void* H, const void* W, int32_t dtype, const int32_t*
  *               which may lie in later chunks, so the call runs the forward to the end and then the
  *               chunked backward (four contractions, the cost of the two calls).
  *   ws          device scratch, spo_workspace_bytes(SPO_WS_LOSS_FWD_BWD, T, d, V, 0, S, 0) bytes:
- *               one chunk buffer (a few thousand token rows by V, bf16), a scaled bf16 copy of the chunk's
- *               rows of H, 36 bytes per token row and the forward's partials
+ *               two chunk buffers (a few thousand token rows by V each, bf16), scaled bf16 copies of those
+ *               chunks' rows of H, 36 bytes per token row and the forward's partials
  * Status bits as spo_loss_fwd.
  */
 int32_t spo_loss_fwd_bwd(const void* H, const void* W, int32_t dtype,

@@ -688,8 +688,11 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             for (int i = 0; i < 8; ++i) {
               int r, cc;
               const uint4 val = stage_get(stage, lane, i, r, cc);
-              if (grow_warp0 + r < p.rows_valid)
-                *reinterpret_cast<uint4*>(obase + (int64_t)r * ld + col0 + cc * 8) = val;
+              if (grow_warp0 + r < p.rows_valid) {
+                uint4* dst = reinterpret_cast<uint4*>(obase + (int64_t)r * ld + col0 + cc * 8);
+                if (MODE == MODE_G) __stcs(dst, val);        // chunk buffer: streaming, as in the E epilogue
+                else *dst = val;
+              }
             }
           }
         } else {
