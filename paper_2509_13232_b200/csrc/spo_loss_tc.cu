@@ -72,6 +72,7 @@ constexpr int kEpilogueSleepNs = 64;
 constexpr int kProducerSleepNs = 32;
 constexpr int kPacerSleepNs = 256;                     // between two looks at the other pairs' progress
 constexpr uint32_t kPacerMaxSpins = 1u << 24;          // the pacer gives up (and lets everyone run free) after this many looks
+constexpr int kLagCut = 8;                             // pairs more than this many windows behind are not waited for
 constexpr int kHoldTries = 2048;                       // x 64 ns: longest time a producer holds back for the slowest pair
 
 constexpr float kLog2e = 1.4426950408889634f;
@@ -774,8 +775,15 @@ spo_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         if (lane == 0) { *pace_limit = 0xFFFFFFFFu; progress[group] = 0xFFFFFFFFu; }
         break;
       }
+      // The slowest pair that is still within reach: one that is more than kLagCut windows behind this
+      // pair (its CTAs started late because another kernel held their SMs, say) cannot share L2
+      // lines with it any more, and waiting for it would only pass its delay on to everybody.
+      const uint32_t reach = (uint32_t)kLagCut * (uint32_t)p.window;
       uint32_t mn = 0xFFFFFFFFu;
-      for (int g = lane; g < n_groups; g += 32) mn = min(mn, progress[g]);
+      for (int g = lane; g < n_groups; g += 32) {
+        const uint32_t v = progress[g];
+        if (v >= mine || mine - v <= reach) mn = min(mn, v);
+      }
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) mn = min(mn, __shfl_xor_sync(0xffffffffu, mn, o));
       if (lane == 0) *pace_limit = (mn > 0xFFFFFFFFu - (uint32_t)p.window) ? 0xFFFFFFFFu : mn + (uint32_t)p.window;
