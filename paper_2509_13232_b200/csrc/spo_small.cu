@@ -260,12 +260,21 @@ sample_search_kernel(const float* __restrict__ ab, int64_t N, float eps, const f
 // ---------------------------------------------------------------------------
 // Small tables (N <= kSmallTableMax): the same draw, organised for latency.
 // ---------------------------------------------------------------------------
+// The four kernels of this path are a few microseconds each, so the gaps between them count.  Each one
+// lets the next be set up while it still runs (programmatic dependent launch): pdl_release() at the top
+// of a kernel allows its successor's blocks onto the SMs, pdl_wait() at the top of the successor holds them
+// until the predecessor has finished and its writes are visible.  Every kernel of the chain waits before
+// it touches anything a predecessor writes, so completion of one implies completion of all before it.
+__device__ __forceinline__ void pdl_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // One block = one tile of kSmallTile entries: 128 threads, one float4 (two entries) each.
 template <bool EMIT>
 __global__ void __launch_bounds__(kSmallTile / 2)
 sample_small_sums_kernel(const float4* __restrict__ ab4, int64_t N, float eps, float2* __restrict__ out_w2,
                          float* __restrict__ out_w, unsigned long long* __restrict__ tile_sums,
                          int32_t* __restrict__ first_draw, int32_t* d_status) {
+  pdl_release();
   const int64_t p = (int64_t)blockIdx.x * (kSmallTile / 2) + threadIdx.x;
   const int64_t n_pairs = N >> 1;
   unsigned long long sum = 0;
@@ -301,6 +310,8 @@ __global__ void __launch_bounds__(kSmallTilesMax / 4)
 sample_small_prefix_kernel(const unsigned long long* __restrict__ tile_sums, int n_tiles,
                            unsigned long long* __restrict__ tile_prefix) {
   constexpr int THREADS = kSmallTilesMax / 4, PER = 4;
+  pdl_release();
+  pdl_wait();
   unsigned long long v[PER], run = 0;
 #pragma unroll
   for (int j = 0; j < PER; ++j) {
@@ -336,14 +347,16 @@ sample_search_small_kernel(const float* __restrict__ ab, int64_t N, float eps, c
                            int32_t* d_status) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int k = blockIdx.x * (kSearchSmallThreads / 32) + warp;
+  pdl_release();
   if (k >= M) return;
+  const float u = uniforms[k];                   // an input: read before waiting for the prefix
+  pdl_wait();
   // level 1: 64 probes at the ends of 64 equal spans of the prefix (two per lane); they do not depend
   // on the uniform, so they are in flight together with it
   const int span = (n_tiles + 63) >> 6;
   const int i_a = min((2 * lane + 1) * span, n_tiles) - 1, i_b = min((2 * lane + 2) * span, n_tiles) - 1;
   const unsigned long long p_a = pre[i_a], p_b = pre[i_b];
   const unsigned long long wtot = __shfl_sync(0xffffffffu, p_b, 31);           // pre[n_tiles - 1]
-  const float u = uniforms[k];
   if (wtot == 0 || !(u >= 0.0f) || !(u < 1.0f)) {
     if (lane == 0) {
       cand[k] = -1;
@@ -437,6 +450,7 @@ sample_accept_kernel(const int32_t* __restrict__ cand, const int32_t* __restrict
   __shared__ int s_warp[32];
   __shared__ int s_total;
   if (tid == 0) s_total = 0;
+  pdl_wait();                                      // (returns at once when launched the ordinary way)
   __syncthreads();
   for (int k0 = 0; k0 < M; k0 += 1024 * PER) {
     const int base_count = s_total;
@@ -897,13 +911,28 @@ cudaError_t launch_sample(const float* ab, int64_t N, const float* u, int32_t M,
       sample_small_sums_kernel<false><<<(unsigned)L.n_tiles, kSmallTile / 2, 0, st>>>(
           ab4, N, eps, nullptr, nullptr, tile_sums, first_draw, d_status);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    sample_small_prefix_kernel<<<1, kSmallTilesMax / 4, 0, st>>>(tile_sums, (int)L.n_tiles, tile_prefix);
-    if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    sample_search_small_kernel<<<(unsigned)ceil_div(M, kSearchSmallThreads / 32), kSearchSmallThreads, 0, st>>>(
-        ab, N, eps, u, M, tile_prefix, (int)L.n_tiles, cand, slot_of, first_draw, d_status);
-    if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    sample_accept_kernel<<<1, 1024, 0, st>>>(cand, slot_of, M, B, first_draw, out_ids, d_status);
-    return cudaGetLastError();
+    // the other three may be set up while their predecessor runs (they wait for it on the device)
+    cudaLaunchAttribute early[1];
+    early[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    early[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.stream = st;
+    cfg.attrs = early;
+    cfg.numAttrs = 1;
+    cfg.gridDim = dim3(1);
+    cfg.blockDim = dim3(kSmallTilesMax / 4);
+    e = cudaLaunchKernelEx(&cfg, sample_small_prefix_kernel, (const unsigned long long*)tile_sums, (int)L.n_tiles,
+                           tile_prefix);
+    if (e != cudaSuccess) return e;
+    cfg.gridDim = dim3((unsigned)ceil_div(M, kSearchSmallThreads / 32));
+    cfg.blockDim = dim3(kSearchSmallThreads);
+    e = cudaLaunchKernelEx(&cfg, sample_search_small_kernel, ab, N, eps, u, M, (const unsigned long long*)tile_prefix,
+                           (int)L.n_tiles, cand, slot_of, first_draw, d_status);
+    if (e != cudaSuccess) return e;
+    cfg.gridDim = dim3(1);
+    cfg.blockDim = dim3(1024);
+    return cudaLaunchKernelEx(&cfg, sample_accept_kernel, (const int32_t*)cand, (const int32_t*)slot_of, M, B,
+                              (const int32_t*)first_draw, out_ids, d_status);
   }
   if ((e = cudaMemsetAsync(ws, 0, L.zeroed_bytes, st)) != cudaSuccess) return e;
   if (out_w)
