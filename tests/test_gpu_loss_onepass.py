@@ -14,7 +14,7 @@ import pytest
 
 from oracle import spo_oracle as O
 from paper_2509_13232_b200 import inputs
-from tests.helpers import oracle_loss, rel_fro, run_loss
+from tests.helpers import oracle_loss, rel_fro, run_loss, worst_row_tile_error
 from tests.test_gpu_loss import BF16_CASES, _clip_batch, check
 
 pytestmark = pytest.mark.gpu
@@ -55,6 +55,27 @@ def test_bf16_several_chunks_fp32_dh_and_dw_accumulate():
     assert rel_fro(got["dW"] - init, want["dW"]) <= 1e-2
     scale = np.maximum(1.0, want["seq_sums"][:, 2:3])
     np.testing.assert_allclose(got["seq_sums"] / scale, want["seq_sums"] / scale, rtol=0, atol=2e-3)
+
+
+def test_bf16_five_chunks_dw_contracted_two_chunks_at_a_time():
+    """dW is contracted over two chunks of token rows per launch: five chunks give a storing launch over
+    chunks 0 + 1, an adding one over 2 + 3 and an adding one over the short last chunk alone.  Checked
+    against the oracle per 256-row vocabulary tile (the ragged last tile included), both with a fresh dW
+    and on top of what the buffer held."""
+    lengths = [9000, 7000, 5200, 8100, 6400, 4300, 2500, 1100]
+    lb = inputs.loss_batch(137, lengths, 128, 1500, 0.05, True, 0.3, target="softmax", mask_p=0.1)
+    assert 4 * 9472 < lb.h.shape[0] < 5 * 9472
+    want = oracle_loss(lb)
+    for init in (None, np.full((1500, 128), -0.5, dtype=np.float32)):
+        got = run_loss(lb, dw_init=init, one_pass=True)
+        assert got["status"] == 0
+        assert abs(got["loss"] - want["loss"]) <= 2e-3
+        np.testing.assert_allclose(got["logp"], want["logp"], rtol=0, atol=2e-3)
+        assert rel_fro(got["dH"], want["dH"]) <= 1e-2
+        dw = got["dW"] if init is None else got["dW"] - init
+        assert rel_fro(dw, want["dW"]) <= 1e-2
+        worst, checked, n_tiles, last_checked = worst_row_tile_error(dw, want["dW"], 256)
+        assert n_tiles == 6 and checked == 6 and last_checked and worst <= 2e-2
 
 
 def test_forward_outputs_agree_with_the_two_call_path():
