@@ -38,7 +38,7 @@ TABLE_N = 1_000_000          # tracker table the step samples from and updates
 # DRAM read+write bytes (dram__bytes_read.sum + dram__bytes_write.sum) of all launches of one cfg4 step:
 # one chunk's launches captured with ncu on a slice of the workload, times the chunks of a step.
 # None = the kernels of that path changed after the counters were taken.
-CFG4_STEP_DRAM_BYTES = {"split": 9.19e11, "onepass": 6.74e11}
+CFG4_STEP_DRAM_BYTES = {"split": 9.19e11, "onepass": 6.9e11}
 DW_CHUNK_GROUP = 2           # chunks of token rows whose dW contraction shares one launch (the library's constant)
 
 LOSS_SHAPES = {
