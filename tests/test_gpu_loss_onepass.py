@@ -234,6 +234,28 @@ def test_results_are_bitwise_reproducible():
         np.testing.assert_array_equal(a[k], b[k])
 
 
+def test_results_do_not_depend_on_another_streams_kernels():
+    """The CTA pairs of a launch pace one another, and their holds are bounded and advisory: when another
+    stream's kernels take SMs away in the meantime (as a collective on a second stream would), the call
+    still ends, reports nothing, and gives bit for bit what it gives alone."""
+    import torch
+    lengths = [5000, 4100, 3000, 2900, 3100, 2907]
+    lb = inputs.loss_batch(96, lengths, 256, 4000, 0.05, True, 0.3, target="softmax", mask_p=0.1)
+    alone = run_loss(lb, one_pass=True)
+    assert alone["status"] == 0
+    side = torch.cuda.Stream()
+    x = torch.ones(32 << 20, dtype=torch.float32, device="cuda")
+    torch.cuda.synchronize()
+    with torch.cuda.stream(side):
+        for _ in range(400):
+            x.mul_(1.0001)
+    busy = run_loss(lb, one_pass=True)          # on the current stream, while the other one is busy
+    torch.cuda.synchronize()
+    assert busy["status"] == 0 and busy["loss"] == alone["loss"]
+    for k in ("logp", "lse", "coef", "dH", "dW"):
+        np.testing.assert_array_equal(busy[k], alone[k])
+
+
 def test_real_vocab_and_hidden_small_token_count_full_oracle():
     lb = inputs.loss_batch(41, [170, 1, 129], 4096, 151936, 0.02, True, 0.3, target="softmax", mask_p=0.1)
     got = run_loss(lb, one_pass=True)
