@@ -24,7 +24,7 @@
 // block of MACs) under the L2 bandwidth; the price is that the accumulator is not
 // double-buffered, so the epilogue is kept short: eight warps drain it in parallel.
 //
-// Pipeline per CTA (one CTA per SM, 320 threads):
+// Pipeline per CTA (one CTA per SM, 352 threads):
 //   warp 0 : allocates tensor memory; lane 0 issues the TMA loads (128-byte swizzle)
 //            of this CTA's operand parts into its 4-stage shared-memory ring; completion
 //            is signalled on the "full" mbarrier of the pair's leader CTA.
@@ -34,6 +34,9 @@
 //   warps 2-9 : epilogue; each owns the 32 accumulator lanes its warp id selects and one
 //            256-column half, reads them with tcgen05.ld and applies the mode's fused
 //            epilogue, then releases the accumulator ("tempty", on the leader).
+//   warp 10 : (leader CTA only) pacer: publishes how many k-blocks the pair has loaded, reads the
+//            other pairs' counts and tells warp 0 how far it may run ahead of the slowest, so
+//            that pairs sweeping the same operand tiles find them in L2.
 // Every mbarrier wait is bounded: when it runs out the CTA raises SPO_DEV_TIMEOUT,
 // all roles leave their loops, tensor memory is released and the kernel returns.
 #include <cuda.h>
