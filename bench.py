@@ -227,6 +227,8 @@ class Step:
         else:
             self.launches = n_samp + 1 + 3 + 3 * self.bwd_chunks
             self.flops_bwd = 6.0 * self.T * d * V
+        if dp_world and self.reducer is not None:
+            self.launches += len(self.reducer.events) - 1      # the last dW contraction runs as one launch per slab
 
     def small(self):
         B = self.B
